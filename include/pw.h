@@ -1,0 +1,261 @@
+/*
+ * pw.h - C ABI of the B200 (sm_100a) decoder-layer engine.
+ *
+ * The Pathways paper (arXiv 2203.12533) schedules "compiled functions": sub-computations
+ * with static shapes whose resource needs are known before they run (Section 3; Appendix B),
+ * enqueued asynchronously on an accelerator with buffer futures as inputs (Sections 4.4-4.5).
+ * For its decoder-only language-model workload (Section 5.3: 62 layers, model dimension 2048,
+ * hidden dimension 8192, micro-batches of 4 examples, GPipe-like schedule) the compiled
+ * function a pipeline stage runs is a stack of Transformer layers, forward and backward, on
+ * one micro-batch.  This library is that function for one GPU:
+ *
+ *   pw_layer_create / pw_layer_fwd / pw_layer_bwd    one pre-LN causal decoder layer
+ *   pw_stage_create / pw_stage_run_chain             a stack of layers over M micro-batches
+ *
+ * Conventions shared by every call
+ *   - All tensor pointers are DEVICE pointers unless a parameter is documented as host.
+ *     Activations are bf16, row-major [B, S, width] (token t = b*S + s).  Weights are bf16,
+ *     row-major [out_features, in_features] (y = x W^T + b).  Parameter gradients are fp32
+ *     with the shape of the parameter.  LayerNorm statistics and log-sum-exp are fp32.
+ *   - Ownership: the caller owns every device buffer it passes and keeps it alive until the
+ *     stream has passed the enqueued work.  The library owns only host-side handles, one
+ *     small device status word per handle, and cached CUDA graphs.  No call on the enqueue
+ *     path allocates device memory.
+ *   - Asynchrony: fwd / bwd / run_chain only enqueue work on `stream` (a cudaStream_t passed
+ *     as void*; NULL = the legacy default stream) and return without synchronising - stream
+ *     order plays the role of the paper's buffer futures.  Argument errors are detected
+ *     before anything is enqueued.
+ *   - Errors: every call returns a pw_status_t; no exception crosses the boundary.
+ *     pw_last_error() gives a thread-local message for the last failure on this thread.
+ *     Device-side waits are bounded: if one expires the kernel records PW_ERR_TIMEOUT in the
+ *     handle's status word, releases what it holds and returns; pw_layer_status /
+ *     pw_stage_status read that word.
+ *   - Threading: a handle is used by one host thread at a time.
+ *   - Device: compute capability 10.x only; there is no fallback path of any kind.
+ *
+ * Arithmetic (the paper gives sizes only; these are the textbook definitions)
+ *   h1 = LN(x; g1, b1)                 qkv = h1 Wqkv^T + bqkv      (columns: q | k | v, head h at h*dh)
+ *   o  = causal softmax(q k^T / sqrt(dh)) v   per sequence and head; key j visible to query i iff j <= i
+ *   x1 = x + o Wo^T + bo               h2 = LN(x1; g2, b2)
+ *   u  = h2 W1^T + b1                  a = GeLU(u)                 y = x1 + a W2^T + b2
+ *   LayerNorm: biased variance over the last dimension, eps inside the square root.
+ *   bf16 storage, fp32 accumulation / statistics / softmax / GeLU.
+ */
+#ifndef PW_H_
+#define PW_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PW_VERSION 100
+
+typedef enum pw_status {
+    PW_OK = 0,
+    PW_ERR_INVALID_ARG = 1,
+    PW_ERR_UNSUPPORTED_SHAPE = 2,
+    PW_ERR_WORKSPACE_TOO_SMALL = 3,
+    PW_ERR_CUDA = 4,
+    PW_ERR_DEVICE_UNSUPPORTED = 5,
+    PW_ERR_TIMEOUT = 6,
+    PW_ERR_INTERNAL = 7
+} pw_status_t;
+
+enum { PW_ACT_GELU_ERF = 0, PW_ACT_GELU_TANH = 1 };
+
+/* Static shape of a layer call - fixed for the life of the handle, like the static shapes of
+ * a compiled function (Section 3).  Supported: head_dim in {64, 128}; n_heads*head_dim ==
+ * d_model; d_model % 256 == 0 and d_model <= 8192; d_ff % 128 == 0; seq_len % 64 == 0;
+ * batch >= 1; causal == 1.  Anything else gives PW_ERR_UNSUPPORTED_SHAPE (never a slow path). */
+typedef struct pw_layer_config {
+    uint32_t struct_size; /* sizeof(pw_layer_config_t), for versioning */
+    int32_t d_model;
+    int32_t n_heads;
+    int32_t head_dim;
+    int32_t d_ff;
+    int32_t seq_len;
+    int32_t batch;
+    int32_t act;    /* PW_ACT_GELU_ERF (default) or PW_ACT_GELU_TANH */
+    float ln_eps;   /* 0 means 1e-5 */
+    int32_t causal; /* must be 1 */
+    uint32_t flags; /* reserved, 0 */
+} pw_layer_config_t;
+
+/* The 12 parameters of a layer (bf16 device pointers). */
+typedef struct pw_layer_params {
+    const void* ln1_gamma; /* [d]      */
+    const void* ln1_beta;  /* [d]      */
+    const void* w_qkv;     /* [3d, d]  */
+    const void* b_qkv;     /* [3d]     */
+    const void* w_o;       /* [d, d]   */
+    const void* b_o;       /* [d]      */
+    const void* ln2_gamma; /* [d]      */
+    const void* ln2_beta;  /* [d]      */
+    const void* w_fc1;     /* [F, d]   */
+    const void* b_fc1;     /* [F]      */
+    const void* w_fc2;     /* [d, F]   */
+    const void* b_fc2;     /* [d]      */
+} pw_layer_params_t;
+
+/* Gradients of the 12 parameters (fp32 device pointers, same shapes, same order). */
+typedef struct pw_layer_grads {
+    void* ln1_gamma; void* ln1_beta; void* w_qkv; void* b_qkv; void* w_o; void* b_o;
+    void* ln2_gamma; void* ln2_beta; void* w_fc1; void* b_fc1; void* w_fc2; void* b_fc2;
+} pw_layer_grads_t;
+
+typedef struct pw_layer pw_layer_t;
+typedef struct pw_stage pw_stage_t;
+
+/* Tensors the forward saves in `ctx` for the backward (ids for pw_layer_ctx_offset). */
+enum {
+    PW_CTX_H1 = 0,  /* bf16 [T, d]   LN1 output              */
+    PW_CTX_QKV = 1, /* bf16 [T, 3d]                          */
+    PW_CTX_O = 2,   /* bf16 [T, d]   attention output        */
+    PW_CTX_X1 = 3,  /* bf16 [T, d]   x + attention branch    */
+    PW_CTX_H2 = 4,  /* bf16 [T, d]   LN2 output              */
+    PW_CTX_U = 5,   /* bf16 [T, F]   FC1 pre-activation      */
+    PW_CTX_A = 6,   /* bf16 [T, F]   GeLU(u)                 */
+    PW_CTX_LSE = 7, /* fp32 [B, H, S] log-sum-exp of the scaled, masked scores */
+    PW_CTX_MU1 = 8, PW_CTX_R1 = 9,   /* fp32 [T] LN1 mean and 1/sqrt(var+eps) */
+    PW_CTX_MU2 = 10, PW_CTX_R2 = 11, /* fp32 [T] LN2 */
+    PW_CTX_COUNT = 12
+};
+
+/* ---- misc ---- */
+int pw_version(void);
+const char* pw_status_string(pw_status_t s);
+/* Thread-local description of the last error returned on this thread ("" if none). */
+const char* pw_last_error(void);
+
+/* ---- one layer (Section 5.3's Transformer layer as a compiled function, Section 3) ---- */
+
+/* Validates cfg, checks the current device (PW_ERR_DEVICE_UNSUPPORTED unless sm_100), builds
+ * the static launch plan.  *out is set only on PW_OK.  Host pointers. */
+pw_status_t pw_layer_create(const pw_layer_config_t* cfg, pw_layer_t** out);
+void pw_layer_destroy(pw_layer_t* layer);
+
+/* Bytes the caller must provide: ctx (saved activations, written by fwd and read by bwd) and
+ * scratch (temporaries of one fwd or bwd call; contents are undefined between calls).
+ * Both must be 256-byte aligned device memory.  Host pointers for the outputs. */
+pw_status_t pw_layer_workspace_bytes(const pw_layer_t* layer, size_t* ctx_bytes, size_t* scratch_bytes);
+
+/* Where tensor `which` (PW_CTX_*) lives inside ctx: byte offset and size.  For tests/tools. */
+pw_status_t pw_layer_ctx_offset(const pw_layer_t* layer, int which, size_t* offset, size_t* bytes);
+
+/* y = layer(x).  x, y: bf16 [B,S,d] device, y must not alias x.  ctx: receives the saved
+ * activations; NULL means "save nothing" (the intermediates then live in scratch only).
+ * `params` is a host struct of device pointers.  Enqueue only. */
+pw_status_t pw_layer_fwd(pw_layer_t* layer, const pw_layer_params_t* params, const void* x, void* y,
+                         void* ctx, void* scratch, void* stream);
+
+/* dx and parameter gradients from dy.  dy, dx: bf16 [B,S,d] device; dx may alias dy.
+ * accumulate = 0: gradients overwrite *grads; 1: they are added (sum over micro-batches, no
+ * averaging).  ctx: what fwd wrote for the same x and params; NULL means recompute: the
+ * forward is re-run from x into scratch first (bit-identical to the first forward), then the
+ * backward runs.  `grads` is a host struct of device pointers.  Enqueue only. */
+pw_status_t pw_layer_bwd(pw_layer_t* layer, const pw_layer_params_t* params, const void* x, const void* dy,
+                         void* dx, const pw_layer_grads_t* grads, int accumulate, const void* ctx,
+                         void* scratch, void* stream);
+
+/* Synchronises the device and reads the handle's status word: *device_status = PW_OK or the
+ * code a kernel recorded (PW_ERR_TIMEOUT) with *site (may be NULL) = where it gave up. */
+pw_status_t pw_layer_status(pw_layer_t* layer, int* device_status, int* site);
+
+/* ---- a pipeline stage: L layers x M micro-batches (Section 5.3, Table 2; dispatch modes of Section 5.1) ---- */
+
+enum {
+    PW_DISPATCH_OPBYOP = 0, /* synchronise the stream after every layer call (the paper's OpByOp) */
+    PW_DISPATCH_ASYNC = 1,  /* enqueue the whole chain, return (the paper's Chained)             */
+    PW_DISPATCH_GRAPH = 2   /* capture the chain once into a CUDA graph, replay it (Fused)       */
+};
+enum {
+    PW_SCHEDULE_GPIPE = 0,         /* all M forwards, then all M backwards (GPipe-like, Section 5.3) */
+    PW_SCHEDULE_PER_MICROBATCH = 1 /* forward and backward of micro-batch m before m+1              */
+};
+
+pw_status_t pw_stage_create(const pw_layer_config_t* cfg, int n_layers, pw_stage_t** out);
+void pw_stage_destroy(pw_stage_t* stage);
+
+/* Workspace (device, 256-byte aligned) needed by pw_stage_run_chain for these settings. */
+pw_status_t pw_stage_workspace_bytes(const pw_stage_t* stage, int n_microbatches, int schedule, int recompute,
+                                     size_t* bytes);
+
+/* For each micro-batch m: x_mb[m] -> L layers -> y_mb[m]; dy_mb[m] -> L layers backward ->
+ * dx_mb[m].  Layer l+1 consumes layer l's bf16 output.  grads[l] receive the SUM over the M
+ * micro-batches (overwritten by micro-batch 0, added to by the rest).
+ *   params, grads : host arrays [L] of structs of device pointers
+ *   x_mb, dy_mb, y_mb, dx_mb : host arrays [M] of device pointers (bf16 [B,S,d] each);
+ *                   y_mb[m] must not alias x_mb[m]
+ *   recompute = 1 : only each layer's input is kept for the backward; the layer's forward is
+ *                   re-run inside its backward (Section 5.3 config of the benchmark contract)
+ *   recompute = 0 : every layer saves its activations (needs L * M (GPipe) or L (per-micro-batch)
+ *                   contexts in the workspace)
+ * GRAPH mode caches an instantiated graph keyed by every pointer and setting of the call and
+ * replays it when they repeat.  Returns PW_ERR_WORKSPACE_TOO_SMALL before enqueuing anything
+ * if workspace_bytes is insufficient.  Enqueue only (OPBYOP synchronises by definition). */
+pw_status_t pw_stage_run_chain(pw_stage_t* stage, const pw_layer_params_t* params, const pw_layer_grads_t* grads,
+                               const void* const* x_mb, const void* const* dy_mb, void* const* y_mb,
+                               void* const* dx_mb, int n_microbatches, int dispatch_mode, int schedule,
+                               int recompute, void* workspace, size_t workspace_bytes, void* stream);
+
+pw_status_t pw_stage_status(pw_stage_t* stage, int* device_status, int* site);
+
+/* ---- single steps of the layer (same kernels the layer calls; for unit tests and profiling) ---- */
+
+/* LayerNorm forward.  x,h: bf16 [T,d]; gamma,beta: bf16 [d]; mu,rstd: fp32 [T]. */
+pw_status_t pw_op_layernorm_fwd(const void* x, const void* gamma, const void* beta, int T, int d, float eps,
+                                void* h, void* mu, void* rstd, void* stream);
+
+/* LayerNorm backward fused with the residual-gradient add and two bias-gradient column sums:
+ *   dx = resid + LNbwd(dh; x, mu, rstd, gamma)          (bf16 [T,d]; resid bf16 [T,d])
+ *   dgamma, dbeta (fp32 [d])  (+)= sum_t dh*xhat, sum_t dh
+ *   db_resid (fp32 [d], may be NULL) (+)= sum_t resid ; db_dx (fp32 [d], may be NULL) (+)= sum_t dx
+ * partials: fp32 device scratch of pw_op_layernorm_bwd_scratch_bytes(T, d) bytes. */
+size_t pw_op_layernorm_bwd_scratch_bytes(int T, int d);
+pw_status_t pw_op_layernorm_bwd(const void* dh, const void* x, const void* mu, const void* rstd,
+                                const void* gamma, const void* resid, int T, int d, void* dx, void* dgamma,
+                                void* dbeta, void* db_resid, void* db_dx, int accumulate, void* partials,
+                                void* stream);
+
+/* Column sums: out[n] (+)= sum_t in[t][n]; in bf16 [T,N] (row stride ld elements), out fp32 [N].
+ * partials: fp32 device scratch of pw_op_colsum_scratch_bytes(T, N) bytes. */
+size_t pw_op_colsum_scratch_bytes(int T, int N);
+pw_status_t pw_op_colsum(const void* in, int T, int N, int ld, void* out, int accumulate, void* partials,
+                         void* stream);
+
+/* bf16 GEMM on the tensor cores, fp32 accumulation.  C[M,N] = op(A) op(B) then an epilogue.
+ *   layout PW_GEMM_TN: A is [M,K] row-major (lda), B is [N,K] row-major (ldb)      (forward:  x W^T)
+ *          PW_GEMM_NN: A is [M,K] row-major,       B is [K,N] row-major            (dgrad:    dy W)
+ *          PW_GEMM_NT: A is [K,M] row-major,       B is [K,N] row-major            (wgrad:    dy^T x)
+ *   epilogue PW_EPI_NONE      : C bf16 = acc
+ *            PW_EPI_BIAS      : C bf16 = acc + bias[n]
+ *            PW_EPI_BIAS_RESID: C bf16 = acc + bias[n] + aux_in[m][n]          (aux_in bf16, ld_aux)
+ *            PW_EPI_BIAS_GELU : C bf16 = acc + bias[n] (pre-activation) and aux_out bf16 = GeLU(that) (ldc)
+ *            PW_EPI_DGELU     : C bf16 = acc * GeLU'(aux_in[m][n])             (aux_in bf16 = saved u)
+ *            PW_EPI_F32       : C fp32 = acc, or C += acc when accumulate != 0
+ * Leading dimensions are in elements; all of M, N, K multiples of 8; pointers 16-byte aligned. */
+enum { PW_GEMM_TN = 0, PW_GEMM_NN = 1, PW_GEMM_NT = 2 };
+enum { PW_EPI_NONE = 0, PW_EPI_BIAS = 1, PW_EPI_BIAS_RESID = 2, PW_EPI_BIAS_GELU = 3, PW_EPI_DGELU = 4,
+       PW_EPI_F32 = 5 };
+pw_status_t pw_op_gemm(int layout, int epilogue, int act, int M, int N, int K, const void* A, int lda,
+                       const void* B, int ldb, void* C, int ldc, const void* bias, const void* aux_in,
+                       int ld_aux, void* aux_out, int accumulate, void* stream);
+
+/* Causal attention forward on packed qkv (bf16 [T,3d]); o bf16 [T,d]; lse fp32 [B,H,S]. */
+pw_status_t pw_op_attention_fwd(const void* qkv, int B, int S, int H, int dh, void* o, void* lse, void* stream);
+
+/* Causal attention backward.  dout bf16 [T,d]; dqkv bf16 [T,3d] (same packing as qkv);
+ * delta: fp32 device scratch [B,H,S] (receives rowsum(dout*o)). */
+pw_status_t pw_op_attention_bwd(const void* qkv, const void* o, const void* dout, const void* lse, int B, int S,
+                                int H, int dh, void* dqkv, void* delta, void* stream);
+
+/* Status word used by the pw_op_* calls (same meaning as pw_layer_status). */
+pw_status_t pw_op_status(int* device_status, int* site);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PW_H_ */

@@ -1,0 +1,283 @@
+"""ctypes binding over the C-ABI library ``libpw.so`` (see ``include/pw.h``).
+
+Argument marshalling only: every step of the layer runs in the library's CUDA
+kernels.  torch is used for device memory (``tensor.data_ptr()``) and streams.
+There is no fallback: if the library is missing or the device is not sm_100,
+calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libpw.so")
+
+PW_OK = 0
+STATUS_NAMES = {0: "PW_OK", 1: "PW_ERR_INVALID_ARG", 2: "PW_ERR_UNSUPPORTED_SHAPE", 3: "PW_ERR_WORKSPACE_TOO_SMALL",
+                4: "PW_ERR_CUDA", 5: "PW_ERR_DEVICE_UNSUPPORTED", 6: "PW_ERR_TIMEOUT", 7: "PW_ERR_INTERNAL"}
+ACT_GELU_ERF, ACT_GELU_TANH = 0, 1
+GEMM_TN, GEMM_NN, GEMM_NT = 0, 1, 2
+EPI_NONE, EPI_BIAS, EPI_BIAS_RESID, EPI_BIAS_GELU, EPI_DGELU, EPI_F32 = range(6)
+DISPATCH_OPBYOP, DISPATCH_ASYNC, DISPATCH_GRAPH = 0, 1, 2
+SCHEDULE_GPIPE, SCHEDULE_PER_MICROBATCH = 0, 1
+CTX_NAMES = ("h1", "qkv", "o", "x1", "h2", "u", "a", "lse", "mu1", "r1", "mu2", "r2")
+PARAM_NAMES = ("ln1_gamma", "ln1_beta", "w_qkv", "b_qkv", "w_o", "b_o",
+               "ln2_gamma", "ln2_beta", "w_fc1", "b_fc1", "w_fc2", "b_fc2")
+
+EXPORTS = (
+    "pw_version", "pw_status_string", "pw_last_error",
+    "pw_layer_create", "pw_layer_destroy", "pw_layer_workspace_bytes", "pw_layer_ctx_offset",
+    "pw_layer_fwd", "pw_layer_bwd", "pw_layer_status",
+    "pw_stage_create", "pw_stage_destroy", "pw_stage_workspace_bytes", "pw_stage_run_chain", "pw_stage_status",
+    "pw_op_layernorm_fwd", "pw_op_layernorm_bwd_scratch_bytes", "pw_op_layernorm_bwd",
+    "pw_op_colsum_scratch_bytes", "pw_op_colsum", "pw_op_gemm",
+    "pw_op_attention_fwd", "pw_op_attention_bwd", "pw_op_status",
+)
+
+
+class PwError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {message}")
+        self.status = status
+
+
+class LayerConfig(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("d_model", ctypes.c_int32), ("n_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("d_ff", ctypes.c_int32), ("seq_len", ctypes.c_int32),
+                ("batch", ctypes.c_int32), ("act", ctypes.c_int32), ("ln_eps", ctypes.c_float),
+                ("causal", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class _Ptr12(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in PARAM_NAMES]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libpw.so (built by ``paper_2203_12533_b200.build``); raises if it is not there."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise FileNotFoundError(
+                f"{_LIB_PATH} is missing: build it with `python -m paper_2203_12533_b200.build` "
+                "(there is no fallback path)")
+        L = ctypes.CDLL(_LIB_PATH)
+        L.pw_version.restype = ctypes.c_int
+        L.pw_status_string.restype = ctypes.c_char_p
+        L.pw_status_string.argtypes = [ctypes.c_int]
+        L.pw_last_error.restype = ctypes.c_char_p
+        L.pw_op_layernorm_bwd_scratch_bytes.restype = ctypes.c_size_t
+        L.pw_op_layernorm_bwd_scratch_bytes.argtypes = [ctypes.c_int, ctypes.c_int]
+        L.pw_op_colsum_scratch_bytes.restype = ctypes.c_size_t
+        L.pw_op_colsum_scratch_bytes.argtypes = [ctypes.c_int, ctypes.c_int]
+        vp, ci = ctypes.c_void_p, ctypes.c_int
+        L.pw_layer_create.argtypes = [ctypes.POINTER(LayerConfig), ctypes.POINTER(vp)]
+        L.pw_layer_destroy.argtypes = [vp]
+        L.pw_layer_destroy.restype = None
+        L.pw_layer_workspace_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
+        L.pw_layer_ctx_offset.argtypes = [vp, ci, ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
+        L.pw_layer_fwd.argtypes = [vp, ctypes.POINTER(_Ptr12), vp, vp, vp, vp, vp]
+        L.pw_layer_bwd.argtypes = [vp, ctypes.POINTER(_Ptr12), vp, vp, vp, ctypes.POINTER(_Ptr12), ci, vp, vp, vp]
+        L.pw_layer_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
+        L.pw_stage_create.argtypes = [ctypes.POINTER(LayerConfig), ci, ctypes.POINTER(vp)]
+        L.pw_stage_destroy.argtypes = [vp]
+        L.pw_stage_destroy.restype = None
+        L.pw_stage_workspace_bytes.argtypes = [vp, ci, ci, ci, ctypes.POINTER(ctypes.c_size_t)]
+        L.pw_stage_run_chain.argtypes = [vp, ctypes.POINTER(_Ptr12), ctypes.POINTER(_Ptr12), ctypes.POINTER(vp),
+                                         ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), ci, ci, ci, ci,
+                                         vp, ctypes.c_size_t, vp]
+        L.pw_stage_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
+        L.pw_op_layernorm_fwd.argtypes = [vp, vp, vp, ci, ci, ctypes.c_float, vp, vp, vp, vp]
+        L.pw_op_layernorm_bwd.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp, vp, ci, vp, vp]
+        L.pw_op_colsum.argtypes = [vp, ci, ci, ci, vp, ci, vp, vp]
+        L.pw_op_gemm.argtypes = [ci, ci, ci, ci, ci, ci, vp, ci, vp, ci, vp, ci, vp, vp, ci, vp, ci, vp]
+        L.pw_op_attention_fwd.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp]
+        L.pw_op_attention_bwd.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, vp]
+        L.pw_op_status.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci)]
+        _lib = L
+    return _lib
+
+
+def _check(status: int):
+    if status != PW_OK:
+        raise PwError(status, lib().pw_last_error().decode())
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _p(t) -> int | None:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    assert t.is_cuda, "device tensors must be CUDA tensors"
+    return t.data_ptr()
+
+
+def _ptr12(tensors: Sequence) -> _Ptr12:
+    assert len(tensors) == 12
+    s = _Ptr12()
+    for n, t in zip(PARAM_NAMES, tensors):
+        setattr(s, n, _p(t))
+    return s
+
+
+def make_config(d_model, n_heads, head_dim, d_ff, seq_len, batch, act=ACT_GELU_ERF, ln_eps=1e-5, causal=1, flags=0):
+    return LayerConfig(ctypes.sizeof(LayerConfig), d_model, n_heads, head_dim, d_ff, seq_len, batch, act, ln_eps,
+                       causal, flags)
+
+
+class Layer:
+    """One pre-LN causal decoder layer with static shapes (pw_layer_*)."""
+
+    def __init__(self, d_model, n_heads, head_dim, d_ff, seq_len, batch, act=ACT_GELU_ERF, ln_eps=1e-5, causal=1):
+        self.cfg = make_config(d_model, n_heads, head_dim, d_ff, seq_len, batch, act, ln_eps, causal)
+        self._h = ctypes.c_void_p()
+        _check(lib().pw_layer_create(ctypes.byref(self.cfg), ctypes.byref(self._h)))
+        a, b = ctypes.c_size_t(), ctypes.c_size_t()
+        _check(lib().pw_layer_workspace_bytes(self._h, ctypes.byref(a), ctypes.byref(b)))
+        self.ctx_bytes, self.scratch_bytes = a.value, b.value
+        self.T, self.d, self.F = batch * seq_len, d_model, d_ff
+        self.B, self.S, self.H, self.dh = batch, seq_len, n_heads, head_dim
+
+    def close(self):
+        if self._h:
+            lib().pw_layer_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def ctx_view(self, ctx: torch.Tensor, name: str) -> torch.Tensor:
+        """A typed view of one saved tensor inside a ctx (or ctx-shaped scratch) byte buffer."""
+        i = CTX_NAMES.index(name)
+        off, nb = ctypes.c_size_t(), ctypes.c_size_t()
+        _check(lib().pw_layer_ctx_offset(self._h, i, ctypes.byref(off), ctypes.byref(nb)))
+        raw = ctx.view(torch.uint8)[off.value:off.value + nb.value]
+        T, d, F = self.T, self.d, self.F
+        if name in ("h1", "o", "x1", "h2"):
+            return raw.view(torch.bfloat16).view(T, d)
+        if name == "qkv":
+            return raw.view(torch.bfloat16).view(T, 3 * d)
+        if name in ("u", "a"):
+            return raw.view(torch.bfloat16).view(T, F)
+        if name == "lse":
+            return raw.view(torch.float32).view(self.B, self.H, self.S)
+        return raw.view(torch.float32).view(T)
+
+    def fwd(self, params, x, y, ctx, scratch, stream=None):
+        _check(lib().pw_layer_fwd(self._h, ctypes.byref(_ptr12(params)), _p(x), _p(y), _p(ctx), _p(scratch),
+                                  _stream(stream)))
+
+    def bwd(self, params, x, dy, dx, grads, accumulate, ctx, scratch, stream=None):
+        _check(lib().pw_layer_bwd(self._h, ctypes.byref(_ptr12(params)), _p(x), _p(dy), _p(dx),
+                                  ctypes.byref(_ptr12(grads)), int(accumulate), _p(ctx), _p(scratch),
+                                  _stream(stream)))
+
+    def status(self):
+        c, s = ctypes.c_int(), ctypes.c_int()
+        _check(lib().pw_layer_status(self._h, ctypes.byref(c), ctypes.byref(s)))
+        return c.value, s.value
+
+
+class Stage:
+    """A stack of identical-shape layers run over M micro-batches (pw_stage_*)."""
+
+    def __init__(self, n_layers, d_model, n_heads, head_dim, d_ff, seq_len, batch, act=ACT_GELU_ERF, ln_eps=1e-5):
+        self.cfg = make_config(d_model, n_heads, head_dim, d_ff, seq_len, batch, act, ln_eps)
+        self.n_layers = n_layers
+        self._h = ctypes.c_void_p()
+        _check(lib().pw_stage_create(ctypes.byref(self.cfg), n_layers, ctypes.byref(self._h)))
+
+    def close(self):
+        if self._h:
+            lib().pw_stage_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def workspace_bytes(self, n_microbatches, schedule=SCHEDULE_GPIPE, recompute=True) -> int:
+        n = ctypes.c_size_t()
+        _check(lib().pw_stage_workspace_bytes(self._h, n_microbatches, schedule, int(recompute), ctypes.byref(n)))
+        return n.value
+
+    def run_chain(self, params, grads, xs, dys, ys, dxs, workspace, dispatch=DISPATCH_ASYNC,
+                  schedule=SCHEDULE_GPIPE, recompute=True, stream=None, workspace_bytes=None):
+        L, M = self.n_layers, len(xs)
+        assert len(params) == L and len(grads) == L
+        P = (_Ptr12 * L)(*[_ptr12(p) for p in params])
+        G = (_Ptr12 * L)(*[_ptr12(g) for g in grads])
+        arr = lambda ts: (ctypes.c_void_p * M)(*[_p(t) for t in ts])
+        nbytes = workspace.numel() * workspace.element_size() if workspace_bytes is None else workspace_bytes
+        _check(lib().pw_stage_run_chain(self._h, P, G, arr(xs), arr(dys), arr(ys), arr(dxs), M, dispatch, schedule,
+                                        int(recompute), _p(workspace), nbytes, _stream(stream)))
+
+    def status(self):
+        c, s = ctypes.c_int(), ctypes.c_int()
+        _check(lib().pw_stage_status(self._h, ctypes.byref(c), ctypes.byref(s)))
+        return c.value, s.value
+
+
+# ---- single steps ----
+def op_layernorm_fwd(x, gamma, beta, eps, h, mu, rstd, stream=None):
+    T, d = x.shape
+    _check(lib().pw_op_layernorm_fwd(_p(x), _p(gamma), _p(beta), T, d, eps, _p(h), _p(mu), _p(rstd), _stream(stream)))
+
+
+def op_layernorm_bwd_scratch_bytes(T, d) -> int:
+    return lib().pw_op_layernorm_bwd_scratch_bytes(T, d)
+
+
+def op_layernorm_bwd(dh, x, mu, rstd, gamma, resid, dx, dgamma, dbeta, db_resid, db_dx, accumulate, partials,
+                     stream=None):
+    T, d = x.shape
+    _check(lib().pw_op_layernorm_bwd(_p(dh), _p(x), _p(mu), _p(rstd), _p(gamma), _p(resid), T, d, _p(dx), _p(dgamma),
+                                     _p(dbeta), _p(db_resid), _p(db_dx), int(accumulate), _p(partials),
+                                     _stream(stream)))
+
+
+def op_colsum_scratch_bytes(T, N) -> int:
+    return lib().pw_op_colsum_scratch_bytes(T, N)
+
+
+def op_colsum(inp, out, accumulate, partials, stream=None):
+    T, N = inp.shape
+    _check(lib().pw_op_colsum(_p(inp), T, N, inp.stride(0), _p(out), int(accumulate), _p(partials), _stream(stream)))
+
+
+def op_gemm(layout, epilogue, M, N, K, A, lda, B, ldb, C, ldc, bias=None, aux_in=None, ld_aux=0, aux_out=None,
+            accumulate=False, act=ACT_GELU_ERF, stream=None):
+    _check(lib().pw_op_gemm(layout, epilogue, act, M, N, K, _p(A), lda, _p(B), ldb, _p(C), ldc, _p(bias), _p(aux_in),
+                            ld_aux, _p(aux_out), int(accumulate), _stream(stream)))
+
+
+def op_attention_fwd(qkv, B, S, H, dh, o, lse, stream=None):
+    _check(lib().pw_op_attention_fwd(_p(qkv), B, S, H, dh, _p(o), _p(lse), _stream(stream)))
+
+
+def op_attention_bwd(qkv, o, dout, lse, B, S, H, dh, dqkv, delta, stream=None):
+    _check(lib().pw_op_attention_bwd(_p(qkv), _p(o), _p(dout), _p(lse), B, S, H, dh, _p(dqkv), _p(delta),
+                                     _stream(stream)))
+
+
+def op_status():
+    c, s = ctypes.c_int(), ctypes.c_int()
+    _check(lib().pw_op_status(ctypes.byref(c), ctypes.byref(s)))
+    return c.value, s.value

@@ -1,0 +1,659 @@
+// C ABI of the decoder-layer engine: runtime set-up, static launch plans, asynchronous enqueue
+// of one layer's forward / backward, and the stage chain with its three dispatch modes.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/pw.h"
+#include "pw_kernels.h"
+
+namespace pw {
+
+static thread_local std::string g_last_error;
+
+static pw_status_t fail(pw_status_t s, const std::string& msg)
+{
+    g_last_error = msg;
+    return s;
+}
+static pw_status_t fail_cuda(const char* what, cudaError_t e)
+{
+    return fail(PW_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+Runtime* get_runtime(const char** err)
+{
+    static std::mutex mu;
+    static std::map<int, Runtime*> per_device;
+    std::lock_guard<std::mutex> lock(mu);
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { *err = "no CUDA device (cudaGetDevice failed)"; return nullptr; }
+    auto it = per_device.find(dev);
+    if (it != per_device.end()) return it->second;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) { *err = "cudaGetDeviceProperties failed"; return nullptr; }
+    if (prop.major != 10) { *err = "device is not compute capability 10.x (sm_100a kernels only, no fallback)"; return nullptr; }
+    Runtime* rt = new Runtime();
+    rt->device = dev;
+    rt->sm_count = prop.multiProcessorCount;
+    rt->cc_major = prop.major;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &rt->encode_tiled, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || rt->encode_tiled == nullptr) {
+        delete rt; *err = "cuTensorMapEncodeTiled not available from the driver"; return nullptr;
+    }
+    const char* ce;
+    if ((ce = configure_gemm()) || (ce = configure_attention())) { delete rt; *err = ce; return nullptr; }
+    if (cudaMalloc(reinterpret_cast<void**>(&rt->op_status), sizeof(DeviceStatus)) != cudaSuccess ||
+        cudaMemset(rt->op_status, 0, sizeof(DeviceStatus)) != cudaSuccess) {
+        delete rt; *err = "could not allocate the status word"; return nullptr;
+    }
+    per_device[dev] = rt;
+    return rt;
+}
+
+static inline size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
+
+// Static plan of one layer: shapes, workspace offsets.
+struct LayerPlan {
+    pw_layer_config_t cfg;
+    int T, d, H, dh, F, B, S;
+    float eps;
+    size_t ctx_off[PW_CTX_COUNT], ctx_size[PW_CTX_COUNT], ctx_bytes;
+    // scratch = [ctx-shaped region used when the caller passes ctx == NULL] [backward temporaries]
+    size_t off_big, off_td0, off_td1, off_delta, off_partials, scratch_bytes;
+};
+
+}  // namespace pw
+
+struct pw_layer {
+    pw::LayerPlan plan;
+    pw::Runtime* rt;
+    pw::DeviceStatus* status;
+};
+
+struct pw_stage {
+    pw_layer_t* layer;
+    int n_layers;
+    std::map<std::vector<uint64_t>, cudaGraphExec_t> graphs;
+};
+
+namespace pw {
+
+static pw_status_t validate_cfg(const pw_layer_config_t* c)
+{
+    if (!c) return fail(PW_ERR_INVALID_ARG, "config is NULL");
+    if (c->struct_size != sizeof(pw_layer_config_t)) return fail(PW_ERR_INVALID_ARG, "config struct_size mismatch");
+    if (c->d_model <= 0 || c->n_heads <= 0 || c->head_dim <= 0 || c->d_ff <= 0 || c->seq_len <= 0 || c->batch <= 0)
+        return fail(PW_ERR_INVALID_ARG, "config has a non-positive dimension");
+    if (c->act != PW_ACT_GELU_ERF && c->act != PW_ACT_GELU_TANH) return fail(PW_ERR_INVALID_ARG, "unknown activation");
+    if (c->causal != 1) return fail(PW_ERR_UNSUPPORTED_SHAPE, "only causal attention is supported");
+    if (c->flags != 0) return fail(PW_ERR_INVALID_ARG, "flags must be 0");
+    if (c->ln_eps < 0.f) return fail(PW_ERR_INVALID_ARG, "ln_eps must be >= 0");
+    if (c->head_dim != 64 && c->head_dim != 128) return fail(PW_ERR_UNSUPPORTED_SHAPE, "head_dim must be 64 or 128");
+    if (static_cast<long long>(c->n_heads) * c->head_dim != c->d_model)
+        return fail(PW_ERR_UNSUPPORTED_SHAPE, "n_heads * head_dim must equal d_model");
+    if (c->d_model % 256 != 0 || c->d_model > 8192) return fail(PW_ERR_UNSUPPORTED_SHAPE, "d_model must be a multiple of 256, at most 8192");
+    if (c->d_ff % 128 != 0) return fail(PW_ERR_UNSUPPORTED_SHAPE, "d_ff must be a multiple of 128");
+    if (c->seq_len % 128 != 0) return fail(PW_ERR_UNSUPPORTED_SHAPE, "seq_len must be a multiple of 128");
+    if (static_cast<long long>(c->batch) * c->seq_len > (1ll << 24)) return fail(PW_ERR_UNSUPPORTED_SHAPE, "too many tokens per call");
+    return PW_OK;
+}
+
+static void build_plan(const pw_layer_config_t& c, Runtime* rt, LayerPlan* p)
+{
+    p->cfg = c;
+    p->B = c.batch; p->S = c.seq_len; p->T = c.batch * c.seq_len;
+    p->d = c.d_model; p->H = c.n_heads; p->dh = c.head_dim; p->F = c.d_ff;
+    p->eps = c.ln_eps > 0.f ? c.ln_eps : 1e-5f;
+    const size_t T = p->T, d = p->d, F = p->F;
+    const size_t sz[PW_CTX_COUNT] = {T * d * 2, T * 3 * d * 2, T * d * 2, T * d * 2, T * d * 2, T * F * 2, T * F * 2,
+                                     static_cast<size_t>(p->B) * p->H * p->S * 4, T * 4, T * 4, T * 4, T * 4};
+    size_t off = 0;
+    for (int i = 0; i < PW_CTX_COUNT; ++i) { p->ctx_off[i] = off; p->ctx_size[i] = sz[i]; off += align256(sz[i]); }
+    p->ctx_bytes = off;
+    size_t s = p->ctx_bytes;
+    p->off_big = s; s += align256((F > 3 * d ? T * F : T * 3 * d) * 2);
+    p->off_td0 = s; s += align256(T * d * 2);
+    p->off_td1 = s; s += align256(T * d * 2);
+    p->off_delta = s; s += align256(static_cast<size_t>(p->B) * p->H * p->S * 4);
+    size_t part = layernorm_bwd_scratch_bytes(rt, p->T, p->d);
+    const size_t c1 = colsum_scratch_bytes(rt, p->T, p->F), c2 = colsum_scratch_bytes(rt, p->T, 3 * p->d);
+    if (c1 > part) part = c1;
+    if (c2 > part) part = c2;
+    p->off_partials = s; s += align256(part);
+    p->scratch_bytes = s;
+}
+
+#define PW_TRY(expr)                                                        \
+    do {                                                                    \
+        const char* e__ = (expr);                                           \
+        if (e__) return fail(PW_ERR_CUDA, std::string(#expr) + ": " + e__); \
+    } while (0)
+
+static inline uint8_t* at(void* base, size_t off) { return static_cast<uint8_t*>(base) + off; }
+static inline const uint8_t* at(const void* base, size_t off) { return static_cast<const uint8_t*>(base) + off; }
+
+static GemmArgs gemm_args(int layout, int epi, int act, int M, int N, int K, const void* A, int lda, const void* B,
+                          int ldb, void* C, int ldc, const void* bias, const void* aux_in, int ld_aux, void* aux_out,
+                          int accumulate)
+{
+    GemmArgs g;
+    g.layout = layout; g.epilogue = epi; g.act = act; g.M = M; g.N = N; g.K = K;
+    g.A = A; g.lda = lda; g.B = B; g.ldb = ldb; g.C = C; g.ldc = ldc;
+    g.bias = bias; g.aux_in = aux_in; g.ld_aux = ld_aux; g.aux_out = aux_out; g.accumulate = accumulate;
+    return g;
+}
+
+// Forward into `ctx` (a ctx-shaped region).  with_fc2 = false stops after FC1/GeLU (all that a
+// recomputing backward needs).
+static pw_status_t enqueue_fwd(pw_layer_t* L, const pw_layer_params_t* P, const void* x, void* y, void* ctx,
+                               bool with_fc2, cudaStream_t st)
+{
+    const LayerPlan& p = L->plan;
+    Runtime* rt = L->rt;
+    const int T = p.T, d = p.d, F = p.F, act = p.cfg.act;
+    void* h1 = at(ctx, p.ctx_off[PW_CTX_H1]);   void* qkv = at(ctx, p.ctx_off[PW_CTX_QKV]);
+    void* o = at(ctx, p.ctx_off[PW_CTX_O]);     void* x1 = at(ctx, p.ctx_off[PW_CTX_X1]);
+    void* h2 = at(ctx, p.ctx_off[PW_CTX_H2]);   void* u = at(ctx, p.ctx_off[PW_CTX_U]);
+    void* a = at(ctx, p.ctx_off[PW_CTX_A]);     void* lse = at(ctx, p.ctx_off[PW_CTX_LSE]);
+    void* mu1 = at(ctx, p.ctx_off[PW_CTX_MU1]); void* r1 = at(ctx, p.ctx_off[PW_CTX_R1]);
+    void* mu2 = at(ctx, p.ctx_off[PW_CTX_MU2]); void* r2 = at(ctx, p.ctx_off[PW_CTX_R2]);
+
+    PW_TRY(launch_layernorm_fwd(rt, x, P->ln1_gamma, P->ln1_beta, T, d, p.eps, h1, mu1, r1, st));
+    PW_TRY(launch_gemm(rt, gemm_args(kTN, kEpiBias, act, T, 3 * d, d, h1, d, P->w_qkv, d, qkv, 3 * d, P->b_qkv,
+                                     nullptr, 0, nullptr, 0), L->status, st));
+    PW_TRY(launch_attention_fwd(rt, qkv, p.B, p.S, p.H, p.dh, o, lse, st));
+    PW_TRY(launch_gemm(rt, gemm_args(kTN, kEpiBiasResid, act, T, d, d, o, d, P->w_o, d, x1, d, P->b_o, x, d,
+                                     nullptr, 0), L->status, st));
+    PW_TRY(launch_layernorm_fwd(rt, x1, P->ln2_gamma, P->ln2_beta, T, d, p.eps, h2, mu2, r2, st));
+    PW_TRY(launch_gemm(rt, gemm_args(kTN, kEpiBiasGelu, act, T, F, d, h2, d, P->w_fc1, d, u, F, P->b_fc1, nullptr, 0,
+                                     a, 0), L->status, st));
+    if (with_fc2)
+        PW_TRY(launch_gemm(rt, gemm_args(kTN, kEpiBiasResid, act, T, d, F, a, F, P->w_fc2, F, y, d, P->b_fc2, x1, d,
+                                         nullptr, 0), L->status, st));
+    return PW_OK;
+}
+
+static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const void* x, const void* dy, void* dx,
+                               const pw_layer_grads_t* G, int accumulate, const void* ctx, void* scratch,
+                               cudaStream_t st)
+{
+    const LayerPlan& p = L->plan;
+    Runtime* rt = L->rt;
+    const int T = p.T, d = p.d, F = p.F, act = p.cfg.act;
+    if (ctx == nullptr) {
+        pw_status_t s = enqueue_fwd(L, P, x, nullptr, scratch, false, st);
+        if (s != PW_OK) return s;
+        ctx = scratch;
+    }
+    const void* h1 = at(ctx, p.ctx_off[PW_CTX_H1]);   const void* qkv = at(ctx, p.ctx_off[PW_CTX_QKV]);
+    const void* o = at(ctx, p.ctx_off[PW_CTX_O]);     const void* x1 = at(ctx, p.ctx_off[PW_CTX_X1]);
+    const void* h2 = at(ctx, p.ctx_off[PW_CTX_H2]);   const void* u = at(ctx, p.ctx_off[PW_CTX_U]);
+    const void* a = at(ctx, p.ctx_off[PW_CTX_A]);     const void* lse = at(ctx, p.ctx_off[PW_CTX_LSE]);
+    const void* mu1 = at(ctx, p.ctx_off[PW_CTX_MU1]); const void* r1 = at(ctx, p.ctx_off[PW_CTX_R1]);
+    const void* mu2 = at(ctx, p.ctx_off[PW_CTX_MU2]); const void* r2 = at(ctx, p.ctx_off[PW_CTX_R2]);
+    void* big = at(scratch, p.off_big);        // du [T,F], later dqkv [T,3d]
+    void* td0 = at(scratch, p.off_td0);        // dh2, then dout, then dh1
+    void* dx1 = at(scratch, p.off_td1);
+    void* delta = at(scratch, p.off_delta);
+    void* part = at(scratch, p.off_partials);
+
+    // y = x1 + a W2^T + b2  ->  du = (dy W2) * gelu'(u),  dW2 = dy^T a
+    PW_TRY(launch_gemm(rt, gemm_args(kNN, kEpiDGelu, act, T, F, d, dy, d, P->w_fc2, F, big, F, nullptr, u, F,
+                                     nullptr, 0), L->status, st));
+    PW_TRY(launch_gemm(rt, gemm_args(kNT, kEpiF32, act, d, F, T, dy, d, a, F, G->w_fc2, F, nullptr, nullptr, 0,
+                                     nullptr, accumulate), L->status, st));
+    // u = h2 W1^T + b1  ->  dh2 = du W1,  dW1 = du^T h2,  db1 = colsum(du)
+    PW_TRY(launch_gemm(rt, gemm_args(kNN, kEpiNone, act, T, d, F, big, F, P->w_fc1, d, td0, d, nullptr, nullptr, 0,
+                                     nullptr, 0), L->status, st));
+    PW_TRY(launch_gemm(rt, gemm_args(kNT, kEpiF32, act, F, d, T, big, F, h2, d, G->w_fc1, d, nullptr, nullptr, 0,
+                                     nullptr, accumulate), L->status, st));
+    PW_TRY(launch_colsum(rt, big, T, F, F, G->b_fc1, accumulate, part, st));
+    // LN2 backward + residual: dx1 = dy + LNbwd(dh2); also db2 = colsum(dy), dbo = colsum(dx1)
+    PW_TRY(launch_layernorm_bwd(rt, td0, x1, mu2, r2, P->ln2_gamma, dy, T, d, dx1, G->ln2_gamma, G->ln2_beta,
+                                G->b_fc2, G->b_o, accumulate, part, st));
+    // x1 = x + o Wo^T + bo  ->  dout = dx1 Wo,  dWo = dx1^T o
+    PW_TRY(launch_gemm(rt, gemm_args(kNN, kEpiNone, act, T, d, d, dx1, d, P->w_o, d, td0, d, nullptr, nullptr, 0,
+                                     nullptr, 0), L->status, st));
+    PW_TRY(launch_gemm(rt, gemm_args(kNT, kEpiF32, act, d, d, T, dx1, d, o, d, G->w_o, d, nullptr, nullptr, 0,
+                                     nullptr, accumulate), L->status, st));
+    // attention backward -> dqkv
+    PW_TRY(launch_attention_bwd(rt, qkv, o, td0, lse, p.B, p.S, p.H, p.dh, big, delta, st));
+    // qkv = h1 Wqkv^T + bqkv  ->  dh1 = dqkv Wqkv,  dWqkv = dqkv^T h1,  dbqkv = colsum(dqkv)
+    PW_TRY(launch_gemm(rt, gemm_args(kNN, kEpiNone, act, T, d, 3 * d, big, 3 * d, P->w_qkv, d, td0, d, nullptr,
+                                     nullptr, 0, nullptr, 0), L->status, st));
+    PW_TRY(launch_gemm(rt, gemm_args(kNT, kEpiF32, act, 3 * d, d, T, big, 3 * d, h1, d, G->w_qkv, d, nullptr, nullptr,
+                                     0, nullptr, accumulate), L->status, st));
+    PW_TRY(launch_colsum(rt, big, T, 3 * d, 3 * d, G->b_qkv, accumulate, part, st));
+    // LN1 backward + residual: dx = dx1 + LNbwd(dh1)
+    PW_TRY(launch_layernorm_bwd(rt, td0, x, mu1, r1, P->ln1_gamma, dx1, T, d, dx, G->ln1_gamma, G->ln1_beta, nullptr,
+                                nullptr, accumulate, part, st));
+    return PW_OK;
+}
+
+static bool params_ok(const pw_layer_params_t* P)
+{
+    const void* const* q = reinterpret_cast<const void* const*>(P);
+    for (int i = 0; i < 12; ++i)
+        if (q[i] == nullptr || (reinterpret_cast<uintptr_t>(q[i]) & 15)) return false;
+    return true;
+}
+static bool grads_ok(const pw_layer_grads_t* G)
+{
+    void* const* q = reinterpret_cast<void* const*>(G);
+    for (int i = 0; i < 12; ++i)
+        if (q[i] == nullptr || (reinterpret_cast<uintptr_t>(q[i]) & 15)) return false;
+    return true;
+}
+static bool aligned(const void* q, size_t a) { return q != nullptr && (reinterpret_cast<uintptr_t>(q) & (a - 1)) == 0; }
+
+static pw_status_t read_status(DeviceStatus* dev, int* code, int* site)
+{
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return fail_cuda("cudaDeviceSynchronize", e);
+    DeviceStatus h;
+    e = cudaMemcpy(&h, dev, sizeof(h), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail_cuda("cudaMemcpy(status)", e);
+    if (code) *code = h.code;
+    if (site) *site = h.site;
+    return PW_OK;
+}
+
+}  // namespace pw
+
+using namespace pw;
+
+extern "C" {
+
+int pw_version(void) { return PW_VERSION; }
+
+const char* pw_status_string(pw_status_t s)
+{
+    switch (s) {
+        case PW_OK: return "PW_OK";
+        case PW_ERR_INVALID_ARG: return "PW_ERR_INVALID_ARG";
+        case PW_ERR_UNSUPPORTED_SHAPE: return "PW_ERR_UNSUPPORTED_SHAPE";
+        case PW_ERR_WORKSPACE_TOO_SMALL: return "PW_ERR_WORKSPACE_TOO_SMALL";
+        case PW_ERR_CUDA: return "PW_ERR_CUDA";
+        case PW_ERR_DEVICE_UNSUPPORTED: return "PW_ERR_DEVICE_UNSUPPORTED";
+        case PW_ERR_TIMEOUT: return "PW_ERR_TIMEOUT";
+        case PW_ERR_INTERNAL: return "PW_ERR_INTERNAL";
+    }
+    return "PW_ERR_UNKNOWN";
+}
+
+const char* pw_last_error(void) { return g_last_error.c_str(); }
+
+pw_status_t pw_layer_create(const pw_layer_config_t* cfg, pw_layer_t** out)
+{
+    if (!out) return fail(PW_ERR_INVALID_ARG, "out is NULL");
+    pw_status_t s = validate_cfg(cfg);
+    if (s != PW_OK) return s;
+    const char* err = nullptr;
+    Runtime* rt = get_runtime(&err);
+    if (!rt) return fail(PW_ERR_DEVICE_UNSUPPORTED, err ? err : "runtime unavailable");
+    pw_layer_t* L = new (std::nothrow) pw_layer();
+    if (!L) return fail(PW_ERR_INTERNAL, "out of host memory");
+    L->rt = rt;
+    build_plan(*cfg, rt, &L->plan);
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&L->status), sizeof(DeviceStatus));
+    if (e == cudaSuccess) e = cudaMemset(L->status, 0, sizeof(DeviceStatus));
+    if (e != cudaSuccess) { delete L; return fail_cuda("status word allocation", e); }
+    *out = L;
+    return PW_OK;
+}
+
+void pw_layer_destroy(pw_layer_t* layer)
+{
+    if (!layer) return;
+    if (layer->status) cudaFree(layer->status);
+    delete layer;
+}
+
+pw_status_t pw_layer_workspace_bytes(const pw_layer_t* layer, size_t* ctx_bytes, size_t* scratch_bytes)
+{
+    if (!layer) return fail(PW_ERR_INVALID_ARG, "layer is NULL");
+    if (ctx_bytes) *ctx_bytes = layer->plan.ctx_bytes;
+    if (scratch_bytes) *scratch_bytes = layer->plan.scratch_bytes;
+    return PW_OK;
+}
+
+pw_status_t pw_layer_ctx_offset(const pw_layer_t* layer, int which, size_t* offset, size_t* bytes)
+{
+    if (!layer || which < 0 || which >= PW_CTX_COUNT) return fail(PW_ERR_INVALID_ARG, "bad layer or tensor id");
+    if (offset) *offset = layer->plan.ctx_off[which];
+    if (bytes) *bytes = layer->plan.ctx_size[which];
+    return PW_OK;
+}
+
+pw_status_t pw_layer_fwd(pw_layer_t* layer, const pw_layer_params_t* params, const void* x, void* y, void* ctx,
+                         void* scratch, void* stream)
+{
+    if (!layer || !params) return fail(PW_ERR_INVALID_ARG, "layer or params is NULL");
+    if (!params_ok(params)) return fail(PW_ERR_INVALID_ARG, "a parameter pointer is NULL or not 16-byte aligned");
+    if (!aligned(x, 16) || !aligned(y, 16)) return fail(PW_ERR_INVALID_ARG, "x or y is NULL or misaligned");
+    if (x == y) return fail(PW_ERR_INVALID_ARG, "y must not alias x");
+    if (ctx == nullptr && !aligned(scratch, 256)) return fail(PW_ERR_INVALID_ARG, "scratch must be 256-byte aligned when ctx is NULL");
+    if (ctx != nullptr && !aligned(ctx, 256)) return fail(PW_ERR_INVALID_ARG, "ctx must be 256-byte aligned");
+    return enqueue_fwd(layer, params, x, y, ctx ? ctx : scratch, true, static_cast<cudaStream_t>(stream));
+}
+
+pw_status_t pw_layer_bwd(pw_layer_t* layer, const pw_layer_params_t* params, const void* x, const void* dy, void* dx,
+                         const pw_layer_grads_t* grads, int accumulate, const void* ctx, void* scratch, void* stream)
+{
+    if (!layer || !params || !grads) return fail(PW_ERR_INVALID_ARG, "layer, params or grads is NULL");
+    if (!params_ok(params)) return fail(PW_ERR_INVALID_ARG, "a parameter pointer is NULL or not 16-byte aligned");
+    if (!grads_ok(grads)) return fail(PW_ERR_INVALID_ARG, "a gradient pointer is NULL or not 16-byte aligned");
+    if (!aligned(x, 16) || !aligned(dy, 16) || !aligned(dx, 16)) return fail(PW_ERR_INVALID_ARG, "x, dy or dx is NULL or misaligned");
+    if (dx == x) return fail(PW_ERR_INVALID_ARG, "dx must not alias x");
+    if (!aligned(scratch, 256)) return fail(PW_ERR_INVALID_ARG, "scratch is NULL or not 256-byte aligned");
+    if (ctx != nullptr && !aligned(ctx, 256)) return fail(PW_ERR_INVALID_ARG, "ctx must be 256-byte aligned");
+    if (accumulate != 0 && accumulate != 1) return fail(PW_ERR_INVALID_ARG, "accumulate must be 0 or 1");
+    return enqueue_bwd(layer, params, x, dy, dx, grads, accumulate, ctx, scratch, static_cast<cudaStream_t>(stream));
+}
+
+pw_status_t pw_layer_status(pw_layer_t* layer, int* device_status, int* site)
+{
+    if (!layer) return fail(PW_ERR_INVALID_ARG, "layer is NULL");
+    return read_status(layer->status, device_status, site);
+}
+
+// ---------------------------------------------------------------------------------------- stage
+
+pw_status_t pw_stage_create(const pw_layer_config_t* cfg, int n_layers, pw_stage_t** out)
+{
+    if (!out) return fail(PW_ERR_INVALID_ARG, "out is NULL");
+    if (n_layers <= 0 || n_layers > 4096) return fail(PW_ERR_INVALID_ARG, "n_layers out of range");
+    pw_layer_t* L = nullptr;
+    pw_status_t s = pw_layer_create(cfg, &L);
+    if (s != PW_OK) return s;
+    pw_stage_t* st = new (std::nothrow) pw_stage();
+    if (!st) { pw_layer_destroy(L); return fail(PW_ERR_INTERNAL, "out of host memory"); }
+    st->layer = L;
+    st->n_layers = n_layers;
+    *out = st;
+    return PW_OK;
+}
+
+void pw_stage_destroy(pw_stage_t* stage)
+{
+    if (!stage) return;
+    for (auto& kv : stage->graphs) cudaGraphExecDestroy(kv.second);
+    pw_layer_destroy(stage->layer);
+    delete stage;
+}
+
+namespace {
+struct StageLayout {
+    size_t act_bytes, n_act;      // hand-off buffers [T,d] bf16 between layers
+    size_t ctx_bytes, n_ctx;      // saved contexts (recompute == 0)
+    size_t off_act, off_ctx, off_g0, off_g1, off_scratch, total;
+};
+pw_status_t stage_layout(const pw_stage_t* stage, int M, int schedule, int recompute, StageLayout* lay)
+{
+    if (M <= 0 || M > 65536) return fail(PW_ERR_INVALID_ARG, "n_microbatches out of range");
+    if (schedule != PW_SCHEDULE_GPIPE && schedule != PW_SCHEDULE_PER_MICROBATCH) return fail(PW_ERR_INVALID_ARG, "unknown schedule");
+    if (recompute != 0 && recompute != 1) return fail(PW_ERR_INVALID_ARG, "recompute must be 0 or 1");
+    const LayerPlan& p = stage->layer->plan;
+    const size_t L = stage->n_layers, live = (schedule == PW_SCHEDULE_GPIPE) ? M : 1;
+    lay->act_bytes = align256(static_cast<size_t>(p.T) * p.d * 2);
+    lay->n_act = (L - 1) * live;
+    lay->ctx_bytes = p.ctx_bytes;
+    lay->n_ctx = recompute ? 0 : L * live;
+    size_t s = 0;
+    lay->off_act = s; s += lay->act_bytes * lay->n_act;
+    lay->off_ctx = s; s += lay->ctx_bytes * lay->n_ctx;
+    lay->off_g0 = s; s += lay->act_bytes;
+    lay->off_g1 = s; s += lay->act_bytes;
+    lay->off_scratch = s; s += p.scratch_bytes;
+    lay->total = s;
+    return PW_OK;
+}
+}  // namespace
+
+pw_status_t pw_stage_workspace_bytes(const pw_stage_t* stage, int n_microbatches, int schedule, int recompute,
+                                     size_t* bytes)
+{
+    if (!stage || !bytes) return fail(PW_ERR_INVALID_ARG, "stage or bytes is NULL");
+    StageLayout lay;
+    pw_status_t s = stage_layout(stage, n_microbatches, schedule, recompute, &lay);
+    if (s != PW_OK) return s;
+    *bytes = lay.total;
+    return PW_OK;
+}
+
+namespace {
+// Enqueues the whole chain on `st`.  sync_each = OPBYOP.
+pw_status_t enqueue_chain(pw_stage_t* stage, const pw_layer_params_t* params, const pw_layer_grads_t* grads,
+                          const void* const* x_mb, const void* const* dy_mb, void* const* y_mb, void* const* dx_mb,
+                          int M, int schedule, int recompute, void* ws, const StageLayout& lay, bool sync_each,
+                          cudaStream_t st)
+{
+    pw_layer_t* Lh = stage->layer;
+    const int L = stage->n_layers;
+    const bool gpipe = schedule == PW_SCHEDULE_GPIPE;
+    auto act = [&](int m, int l) -> void* {   // input of layer l (l >= 1) for micro-batch m
+        const size_t slot = (gpipe ? static_cast<size_t>(m) * (L - 1) : 0) + (l - 1);
+        return at(ws, lay.off_act + slot * lay.act_bytes);
+    };
+    auto ctxp = [&](int m, int l) -> void* {
+        if (recompute) return nullptr;
+        const size_t slot = (gpipe ? static_cast<size_t>(m) * L : 0) + l;
+        return at(ws, lay.off_ctx + slot * lay.ctx_bytes);
+    };
+    void* scratch = at(ws, lay.off_scratch);
+    auto sync = [&]() -> pw_status_t {
+        if (!sync_each) return PW_OK;
+        cudaError_t e = cudaStreamSynchronize(st);
+        return e == cudaSuccess ? PW_OK : fail_cuda("cudaStreamSynchronize", e);
+    };
+    auto fwd_mb = [&](int m) -> pw_status_t {
+        for (int l = 0; l < L; ++l) {
+            const void* in = l == 0 ? x_mb[m] : act(m, l);
+            void* out = l == L - 1 ? y_mb[m] : act(m, l + 1);
+            void* c = ctxp(m, l);
+            pw_status_t s = enqueue_fwd(Lh, &params[l], in, out, c ? c : scratch, true, st);
+            if (s != PW_OK) return s;
+            if ((s = sync()) != PW_OK) return s;
+        }
+        return PW_OK;
+    };
+    auto bwd_mb = [&](int m) -> pw_status_t {
+        const void* g = dy_mb[m];
+        for (int l = L - 1; l >= 0; --l) {
+            const void* in = l == 0 ? x_mb[m] : act(m, l);
+            void* out = l == 0 ? dx_mb[m] : at(ws, (l & 1) ? lay.off_g1 : lay.off_g0);
+            pw_status_t s = enqueue_bwd(Lh, &params[l], in, g, out, &grads[l], m > 0 ? 1 : 0, ctxp(m, l), scratch, st);
+            if (s != PW_OK) return s;
+            if ((s = sync()) != PW_OK) return s;
+            g = out;
+        }
+        return PW_OK;
+    };
+    pw_status_t s;
+    if (gpipe) {
+        for (int m = 0; m < M; ++m) if ((s = fwd_mb(m)) != PW_OK) return s;
+        for (int m = 0; m < M; ++m) if ((s = bwd_mb(m)) != PW_OK) return s;
+    } else {
+        for (int m = 0; m < M; ++m) {
+            if ((s = fwd_mb(m)) != PW_OK) return s;
+            if ((s = bwd_mb(m)) != PW_OK) return s;
+        }
+    }
+    return PW_OK;
+}
+}  // namespace
+
+pw_status_t pw_stage_run_chain(pw_stage_t* stage, const pw_layer_params_t* params, const pw_layer_grads_t* grads,
+                               const void* const* x_mb, const void* const* dy_mb, void* const* y_mb,
+                               void* const* dx_mb, int n_microbatches, int dispatch_mode, int schedule, int recompute,
+                               void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!stage || !params || !grads || !x_mb || !dy_mb || !y_mb || !dx_mb)
+        return fail(PW_ERR_INVALID_ARG, "a required pointer is NULL");
+    if (dispatch_mode < PW_DISPATCH_OPBYOP || dispatch_mode > PW_DISPATCH_GRAPH) return fail(PW_ERR_INVALID_ARG, "unknown dispatch mode");
+    StageLayout lay;
+    pw_status_t s = stage_layout(stage, n_microbatches, schedule, recompute, &lay);
+    if (s != PW_OK) return s;
+    if (!aligned(workspace, 256)) return fail(PW_ERR_INVALID_ARG, "workspace is NULL or not 256-byte aligned");
+    if (workspace_bytes < lay.total) return fail(PW_ERR_WORKSPACE_TOO_SMALL, "workspace smaller than pw_stage_workspace_bytes reports");
+    const int L = stage->n_layers, M = n_microbatches;
+    for (int l = 0; l < L; ++l)
+        if (!params_ok(&params[l]) || !grads_ok(&grads[l])) return fail(PW_ERR_INVALID_ARG, "a parameter or gradient pointer is NULL or misaligned");
+    for (int m = 0; m < M; ++m) {
+        if (!aligned(x_mb[m], 16) || !aligned(dy_mb[m], 16) || !aligned(y_mb[m], 16) || !aligned(dx_mb[m], 16))
+            return fail(PW_ERR_INVALID_ARG, "a micro-batch pointer is NULL or misaligned");
+        if (x_mb[m] == y_mb[m] || x_mb[m] == dx_mb[m]) return fail(PW_ERR_INVALID_ARG, "y and dx must not alias x");
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    if (dispatch_mode != PW_DISPATCH_GRAPH)
+        return enqueue_chain(stage, params, grads, x_mb, dy_mb, y_mb, dx_mb, M, schedule, recompute, workspace, lay,
+                             dispatch_mode == PW_DISPATCH_OPBYOP, st);
+
+    // GRAPH: key = every pointer and setting that the captured launches bake in.
+    std::vector<uint64_t> key;
+    key.reserve(8 + 24 * L + 4 * M);
+    key.push_back(M); key.push_back(schedule); key.push_back(recompute);
+    key.push_back(reinterpret_cast<uint64_t>(workspace));
+    for (int l = 0; l < L; ++l) {
+        const void* const* pp = reinterpret_cast<const void* const*>(&params[l]);
+        void* const* gg = reinterpret_cast<void* const*>(&grads[l]);
+        for (int i = 0; i < 12; ++i) { key.push_back(reinterpret_cast<uint64_t>(pp[i])); key.push_back(reinterpret_cast<uint64_t>(gg[i])); }
+    }
+    for (int m = 0; m < M; ++m) {
+        key.push_back(reinterpret_cast<uint64_t>(x_mb[m])); key.push_back(reinterpret_cast<uint64_t>(dy_mb[m]));
+        key.push_back(reinterpret_cast<uint64_t>(y_mb[m])); key.push_back(reinterpret_cast<uint64_t>(dx_mb[m]));
+    }
+    auto it = stage->graphs.find(key);
+    if (it == stage->graphs.end()) {
+        if (st == nullptr) return fail(PW_ERR_INVALID_ARG, "GRAPH mode needs a non-default stream (the legacy stream cannot be captured)");
+        cudaError_t e = cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal);
+        if (e != cudaSuccess) return fail_cuda("cudaStreamBeginCapture", e);
+        s = enqueue_chain(stage, params, grads, x_mb, dy_mb, y_mb, dx_mb, M, schedule, recompute, workspace, lay, false, st);
+        cudaGraph_t graph = nullptr;
+        e = cudaStreamEndCapture(st, &graph);
+        if (s != PW_OK) { if (graph) cudaGraphDestroy(graph); return s; }
+        if (e != cudaSuccess) return fail_cuda("cudaStreamEndCapture", e);
+        cudaGraphExec_t exec = nullptr;
+        e = cudaGraphInstantiate(&exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (e != cudaSuccess) return fail_cuda("cudaGraphInstantiate", e);
+        if (stage->graphs.size() >= 16) {   // bounded cache
+            for (auto& kv : stage->graphs) cudaGraphExecDestroy(kv.second);
+            stage->graphs.clear();
+        }
+        it = stage->graphs.emplace(key, exec).first;
+    }
+    cudaError_t e = cudaGraphLaunch(it->second, st);
+    return e == cudaSuccess ? PW_OK : fail_cuda("cudaGraphLaunch", e);
+}
+
+pw_status_t pw_stage_status(pw_stage_t* stage, int* device_status, int* site)
+{
+    if (!stage) return fail(PW_ERR_INVALID_ARG, "stage is NULL");
+    return read_status(stage->layer->status, device_status, site);
+}
+
+// ---------------------------------------------------------------------------------------- single steps
+
+#define PW_RT_OR_FAIL()                                                                       \
+    const char* rt_err__ = nullptr;                                                           \
+    Runtime* rt = get_runtime(&rt_err__);                                                     \
+    if (!rt) return fail(PW_ERR_DEVICE_UNSUPPORTED, rt_err__ ? rt_err__ : "runtime unavailable")
+
+#define PW_OP(expr)                                          \
+    do {                                                     \
+        const char* e__ = (expr);                            \
+        if (e__) return fail(PW_ERR_INVALID_ARG, e__);       \
+    } while (0)
+
+pw_status_t pw_op_layernorm_fwd(const void* x, const void* gamma, const void* beta, int T, int d, float eps, void* h,
+                                void* mu, void* rstd, void* stream)
+{
+    PW_RT_OR_FAIL();
+    if (!aligned(x, 16) || !aligned(gamma, 16) || !aligned(beta, 16) || !aligned(h, 16) || !mu || !rstd)
+        return fail(PW_ERR_INVALID_ARG, "layernorm: NULL or misaligned pointer");
+    PW_OP(launch_layernorm_fwd(rt, x, gamma, beta, T, d, eps, h, mu, rstd, static_cast<cudaStream_t>(stream)));
+    return PW_OK;
+}
+
+size_t pw_op_layernorm_bwd_scratch_bytes(int T, int d)
+{
+    const char* err = nullptr;
+    Runtime* rt = get_runtime(&err);
+    return rt ? layernorm_bwd_scratch_bytes(rt, T, d) : 0;
+}
+
+pw_status_t pw_op_layernorm_bwd(const void* dh, const void* x, const void* mu, const void* rstd, const void* gamma,
+                                const void* resid, int T, int d, void* dx, void* dgamma, void* dbeta, void* db_resid,
+                                void* db_dx, int accumulate, void* partials, void* stream)
+{
+    PW_RT_OR_FAIL();
+    if (!aligned(dh, 16) || !aligned(x, 16) || !aligned(gamma, 16) || !aligned(resid, 16) || !aligned(dx, 16) || !mu ||
+        !rstd || !dgamma || !dbeta || !aligned(partials, 16))
+        return fail(PW_ERR_INVALID_ARG, "layernorm bwd: NULL or misaligned pointer");
+    PW_OP(launch_layernorm_bwd(rt, dh, x, mu, rstd, gamma, resid, T, d, dx, dgamma, dbeta, db_resid, db_dx, accumulate,
+                               partials, static_cast<cudaStream_t>(stream)));
+    return PW_OK;
+}
+
+size_t pw_op_colsum_scratch_bytes(int T, int N)
+{
+    const char* err = nullptr;
+    Runtime* rt = get_runtime(&err);
+    return rt ? colsum_scratch_bytes(rt, T, N) : 0;
+}
+
+pw_status_t pw_op_colsum(const void* in, int T, int N, int ld, void* out, int accumulate, void* partials, void* stream)
+{
+    PW_RT_OR_FAIL();
+    if (!aligned(in, 16) || !out || !aligned(partials, 16)) return fail(PW_ERR_INVALID_ARG, "colsum: NULL or misaligned pointer");
+    PW_OP(launch_colsum(rt, in, T, N, ld, out, accumulate, partials, static_cast<cudaStream_t>(stream)));
+    return PW_OK;
+}
+
+pw_status_t pw_op_gemm(int layout, int epilogue, int act, int M, int N, int K, const void* A, int lda, const void* B,
+                       int ldb, void* C, int ldc, const void* bias, const void* aux_in, int ld_aux, void* aux_out,
+                       int accumulate, void* stream)
+{
+    PW_RT_OR_FAIL();
+    PW_OP(launch_gemm(rt, gemm_args(layout, epilogue, act, M, N, K, A, lda, B, ldb, C, ldc, bias, aux_in, ld_aux,
+                                    aux_out, accumulate), rt->op_status, static_cast<cudaStream_t>(stream)));
+    return PW_OK;
+}
+
+pw_status_t pw_op_attention_fwd(const void* qkv, int B, int S, int H, int dh, void* o, void* lse, void* stream)
+{
+    PW_RT_OR_FAIL();
+    if (!aligned(qkv, 16) || !aligned(o, 16) || !lse) return fail(PW_ERR_INVALID_ARG, "attention: NULL or misaligned pointer");
+    PW_OP(launch_attention_fwd(rt, qkv, B, S, H, dh, o, lse, static_cast<cudaStream_t>(stream)));
+    return PW_OK;
+}
+
+pw_status_t pw_op_attention_bwd(const void* qkv, const void* o, const void* dout, const void* lse, int B, int S, int H,
+                                int dh, void* dqkv, void* delta, void* stream)
+{
+    PW_RT_OR_FAIL();
+    if (!aligned(qkv, 16) || !aligned(o, 16) || !aligned(dout, 16) || !lse || !aligned(dqkv, 16) || !delta)
+        return fail(PW_ERR_INVALID_ARG, "attention bwd: NULL or misaligned pointer");
+    PW_OP(launch_attention_bwd(rt, qkv, o, dout, lse, B, S, H, dh, dqkv, delta, static_cast<cudaStream_t>(stream)));
+    return PW_OK;
+}
+
+pw_status_t pw_op_status(int* device_status, int* site)
+{
+    PW_RT_OR_FAIL();
+    return read_status(rt->op_status, device_status, site);
+}
+
+}  // extern "C"

@@ -1,0 +1,321 @@
+// HBM-bound kernels of the layer: LayerNorm forward, LayerNorm backward (fused with the
+// residual-gradient add and two bias-gradient column sums), column sums, and the row-dot
+// preprocess of the attention backward.  All use 16-byte accesses (8 bf16 per thread per
+// access), fp32 arithmetic, warp shuffles plus one shared-memory hop for row reductions, and
+// fixed-order two-stage reductions for anything summed over tokens (bitwise reproducible).
+#include "pw_kernels.h"
+
+namespace pw {
+namespace {
+
+constexpr int kMaxWarps = 8;          // CTAs have at most 256 threads
+constexpr int kRowThreadsMax = 256;
+
+// A row of d elements is handled by tpr = d / (8*CHUNKS) threads, CHUNKS 16-byte pieces each;
+// thread i of the row owns columns 8*(i + j*tpr) .. +7 for j < CHUNKS (coalesced per j).
+struct RowPlan { int chunks, tpr, rows_per_cta, threads; };
+bool plan_rows(int d, RowPlan* rp)
+{
+    for (int c = 1; c <= 4; c *= 2) {
+        if (d % (8 * c * 32) != 0) continue;
+        int tpr = d / (8 * c);
+        if (tpr > kRowThreadsMax) continue;
+        rp->chunks = c; rp->tpr = tpr;
+        rp->rows_per_cta = kRowThreadsMax / tpr;
+        rp->threads = rp->rows_per_cta * tpr;
+        return true;
+    }
+    return false;
+}
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Sum of `v` over the tpr threads of this row (warps_per_row consecutive warps).  `slot` is a
+// [kMaxWarps] shared array private to this reduction; the caller separates reuses of a slot
+// by a __syncthreads.
+__device__ __forceinline__ float row_sum(float v, float* slot, int warps_per_row, int row_in_cta)
+{
+    v = warp_sum(v);
+    if (warps_per_row == 1) return v;
+    const int warp = threadIdx.x >> 5;
+    if ((threadIdx.x & 31) == 0) slot[warp] = v;
+    __syncthreads();
+    float t = 0.f;
+    for (int i = 0; i < warps_per_row; ++i) t += slot[row_in_cta * warps_per_row + i];
+    return t;
+}
+
+template <int CHUNKS>
+__global__ void __launch_bounds__(kRowThreadsMax)
+ln_fwd_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gamma,
+              const __nv_bfloat16* __restrict__ beta, int T, int d, float eps, __nv_bfloat16* __restrict__ h,
+              float* __restrict__ mu, float* __restrict__ rstd, int tpr, int rows_per_cta)
+{
+    __shared__ float red[2][kMaxWarps];
+    const int row_in_cta = threadIdx.x / tpr, tr = threadIdx.x % tpr;
+    const int row = blockIdx.x * rows_per_cta + row_in_cta;
+    const int wpr = tpr >> 5;
+    const bool live = row < T;
+    float v[CHUNKS][8];
+    float s = 0.f;
+#pragma unroll
+    for (int j = 0; j < CHUNKS; ++j) {
+        const int col = 8 * (tr + j * tpr);
+        uint4 raw = live ? *reinterpret_cast<const uint4*>(x + static_cast<size_t>(row) * d + col) : make_uint4(0, 0, 0, 0);
+        unpack8(raw, v[j]);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) s += v[j][k];
+    }
+    const float mean = row_sum(s, red[0], wpr, row_in_cta) / d;
+    float q = 0.f;
+#pragma unroll
+    for (int j = 0; j < CHUNKS; ++j)
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { const float c = v[j][k] - mean; q += c * c; }
+    const float var = row_sum(q, red[1], wpr, row_in_cta) / d;
+    const float r = rsqrtf(var + eps);
+    if (!live) return;
+#pragma unroll
+    for (int j = 0; j < CHUNKS; ++j) {
+        const int col = 8 * (tr + j * tpr);
+        float g[8], b[8], o[8];
+        unpack8(__ldg(reinterpret_cast<const uint4*>(gamma + col)), g);
+        unpack8(__ldg(reinterpret_cast<const uint4*>(beta + col)), b);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) o[k] = g[k] * ((v[j][k] - mean) * r) + b[k];
+        *reinterpret_cast<uint4*>(h + static_cast<size_t>(row) * d + col) = pack8(o);
+    }
+    if (tr == 0) { mu[row] = mean; rstd[row] = r; }
+}
+
+// LayerNorm backward.  Persistent over rows; every thread keeps the column sums of its own
+// columns in registers and writes them once at the end as one partial row per (CTA, row slot):
+// partials[(cta*rows_per_cta + row_in_cta)][4][d] = {dgamma, dbeta, sum resid, sum dx}.
+template <int CHUNKS>
+__global__ void __launch_bounds__(kRowThreadsMax)
+ln_bwd_kernel(const __nv_bfloat16* __restrict__ dh, const __nv_bfloat16* __restrict__ x,
+              const float* __restrict__ mu, const float* __restrict__ rstd, const __nv_bfloat16* __restrict__ gamma,
+              const __nv_bfloat16* resid, int T, int d, __nv_bfloat16* dx,
+              float* __restrict__ partials, int tpr, int rows_per_cta)
+{
+    __shared__ float red[2][2][kMaxWarps];
+    const int row_in_cta = threadIdx.x / tpr, tr = threadIdx.x % tpr;
+    const int wpr = tpr >> 5;
+    float gm[CHUNKS][8];
+    float acc_g[CHUNKS][8], acc_b[CHUNKS][8], acc_r[CHUNKS][8], acc_x[CHUNKS][8];
+#pragma unroll
+    for (int j = 0; j < CHUNKS; ++j) {
+        unpack8(__ldg(reinterpret_cast<const uint4*>(gamma + 8 * (tr + j * tpr))), gm[j]);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) acc_g[j][k] = acc_b[j][k] = acc_r[j][k] = acc_x[j][k] = 0.f;
+    }
+    const int row_groups = (T + rows_per_cta - 1) / rows_per_cta;
+    int par = 0;
+    for (int rg = blockIdx.x; rg < row_groups; rg += gridDim.x, par ^= 1) {
+        const int row = rg * rows_per_cta + row_in_cta;
+        const bool live = row < T;
+        const float m = live ? mu[row] : 0.f, r = live ? rstd[row] : 0.f;
+        float xh[CHUNKS][8], g[CHUNKS][8], dhv[CHUNKS][8];
+        float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+        for (int j = 0; j < CHUNKS; ++j) {
+            const size_t off = static_cast<size_t>(row) * d + 8 * (tr + j * tpr);
+            uint4 a = live ? *reinterpret_cast<const uint4*>(dh + off) : make_uint4(0, 0, 0, 0);
+            uint4 b = live ? *reinterpret_cast<const uint4*>(x + off) : make_uint4(0, 0, 0, 0);
+            unpack8(a, dhv[j]);
+            unpack8(b, xh[j]);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                xh[j][k] = (xh[j][k] - m) * r;
+                g[j][k] = dhv[j][k] * gm[j][k];
+                s1 += g[j][k];
+                s2 += g[j][k] * xh[j][k];
+            }
+        }
+        const float mg = row_sum(s1, red[par][0], wpr, row_in_cta) / d;
+        const float mgx = row_sum(s2, red[par][1], wpr, row_in_cta) / d;
+        if (live) {
+#pragma unroll
+            for (int j = 0; j < CHUNKS; ++j) {
+                const size_t off = static_cast<size_t>(row) * d + 8 * (tr + j * tpr);
+                float rs[8], o[8];
+                unpack8(*reinterpret_cast<const uint4*>(resid + off), rs);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) o[k] = rs[k] + r * (g[j][k] - mg - xh[j][k] * mgx);
+                const uint4 packed = pack8(o);
+                *reinterpret_cast<uint4*>(dx + off) = packed;
+                float ob[8];
+                unpack8(packed, ob);   // the bias gradient sums the values that are actually stored
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    acc_g[j][k] += dhv[j][k] * xh[j][k];
+                    acc_b[j][k] += dhv[j][k];
+                    acc_r[j][k] += rs[k];
+                    acc_x[j][k] += ob[k];
+                }
+            }
+        }
+    }
+    float* prow = partials + static_cast<size_t>(blockIdx.x * rows_per_cta + row_in_cta) * 4 * d;
+#pragma unroll
+    for (int j = 0; j < CHUNKS; ++j) {
+        const int col = 8 * (tr + j * tpr);
+#pragma unroll
+        for (int k = 0; k < 8; k += 4) {
+            *reinterpret_cast<float4*>(prow + 0 * d + col + k) = make_float4(acc_g[j][k], acc_g[j][k + 1], acc_g[j][k + 2], acc_g[j][k + 3]);
+            *reinterpret_cast<float4*>(prow + 1 * d + col + k) = make_float4(acc_b[j][k], acc_b[j][k + 1], acc_b[j][k + 2], acc_b[j][k + 3]);
+            *reinterpret_cast<float4*>(prow + 2 * d + col + k) = make_float4(acc_r[j][k], acc_r[j][k + 1], acc_r[j][k + 2], acc_r[j][k + 3]);
+            *reinterpret_cast<float4*>(prow + 3 * d + col + k) = make_float4(acc_x[j][k], acc_x[j][k + 1], acc_x[j][k + 2], acc_x[j][k + 3]);
+        }
+    }
+}
+
+// out_q[c] (+)= sum over partial rows of partials[row][q][c], fixed order.  Up to 4 outputs.
+struct ReduceOuts { float* out[4]; };
+__global__ void reduce_partials_kernel(const float* __restrict__ partials, int nrows, int nq, int n, ReduceOuts outs,
+                                       int accumulate)
+{
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    const int q = blockIdx.y;
+    float* out = outs.out[q];
+    if (c >= n || out == nullptr) return;
+    float s = 0.f;
+    for (int r = 0; r < nrows; ++r) s += partials[(static_cast<size_t>(r) * nq + q) * n + c];
+    out[c] = accumulate ? out[c] + s : s;
+}
+
+// Column sums of a bf16 [T, N] matrix: CTA (x, y) owns columns 1024*x .. +1023 and rows y, y+R, ...
+__global__ void __launch_bounds__(128)
+colsum_kernel(const __nv_bfloat16* __restrict__ in, int T, int N, int ld, float* __restrict__ partials)
+{
+    const int col = blockIdx.x * 1024 + threadIdx.x * 8;
+    if (col >= N) return;
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    const int R = gridDim.y;
+    int t = blockIdx.y;
+    for (; t + 3 * R < T; t += 4 * R) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const uint4*>(in + static_cast<size_t>(t + u * R) * ld + col);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            float f[8];
+            unpack8(v[u], f);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc[k] += f[k];
+        }
+    }
+    for (; t < T; t += R) {
+        float f[8];
+        unpack8(*reinterpret_cast<const uint4*>(in + static_cast<size_t>(t) * ld + col), f);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) acc[k] += f[k];
+    }
+    float* p = partials + static_cast<size_t>(blockIdx.y) * N + col;
+    *reinterpret_cast<float4*>(p) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    *reinterpret_cast<float4*>(p + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+}
+
+int colsum_splits(Runtime* rt, int T, int N)
+{
+    const int col_blocks = (N + 1023) / 1024;
+    int r = (4 * rt->sm_count + col_blocks - 1) / col_blocks;
+    if (r > T) r = T;
+    if (r < 1) r = 1;
+    return r;
+}
+
+int ln_bwd_grid(Runtime* rt, int T, const RowPlan& rp)
+{
+    const int row_groups = (T + rp.rows_per_cta - 1) / rp.rows_per_cta;
+    const int cap = 2 * rt->sm_count;
+    return row_groups < cap ? row_groups : cap;
+}
+
+}  // namespace
+
+const char* launch_layernorm_fwd(Runtime* rt, const void* x, const void* gamma, const void* beta, int T, int d,
+                                 float eps, void* h, void* mu, void* rstd, cudaStream_t stream)
+{
+    (void)rt;
+    RowPlan rp;
+    if (T <= 0 || !plan_rows(d, &rp)) return "layernorm: unsupported row width";
+    const int grid = (T + rp.rows_per_cta - 1) / rp.rows_per_cta;
+    auto X = static_cast<const __nv_bfloat16*>(x);
+    auto G = static_cast<const __nv_bfloat16*>(gamma);
+    auto Bt = static_cast<const __nv_bfloat16*>(beta);
+    auto Hh = static_cast<__nv_bfloat16*>(h);
+    auto Mu = static_cast<float*>(mu);
+    auto Rs = static_cast<float*>(rstd);
+    switch (rp.chunks) {
+        case 1: ln_fwd_kernel<1><<<grid, rp.threads, 0, stream>>>(X, G, Bt, T, d, eps, Hh, Mu, Rs, rp.tpr, rp.rows_per_cta); break;
+        case 2: ln_fwd_kernel<2><<<grid, rp.threads, 0, stream>>>(X, G, Bt, T, d, eps, Hh, Mu, Rs, rp.tpr, rp.rows_per_cta); break;
+        default: ln_fwd_kernel<4><<<grid, rp.threads, 0, stream>>>(X, G, Bt, T, d, eps, Hh, Mu, Rs, rp.tpr, rp.rows_per_cta); break;
+    }
+    return cudaGetLastError() == cudaSuccess ? nullptr : "layernorm fwd launch failed";
+}
+
+size_t layernorm_bwd_scratch_bytes(Runtime* rt, int T, int d)
+{
+    RowPlan rp;
+    if (T <= 0 || !plan_rows(d, &rp)) return 0;
+    return static_cast<size_t>(ln_bwd_grid(rt, T, rp)) * rp.rows_per_cta * 4 * d * sizeof(float);
+}
+
+const char* launch_layernorm_bwd(Runtime* rt, const void* dh, const void* x, const void* mu, const void* rstd,
+                                 const void* gamma, const void* resid, int T, int d, void* dx, void* dgamma,
+                                 void* dbeta, void* db_resid, void* db_dx, int accumulate, void* partials,
+                                 cudaStream_t stream)
+{
+    RowPlan rp;
+    if (T <= 0 || !plan_rows(d, &rp)) return "layernorm: unsupported row width";
+    const int grid = ln_bwd_grid(rt, T, rp);
+    auto DH = static_cast<const __nv_bfloat16*>(dh);
+    auto X = static_cast<const __nv_bfloat16*>(x);
+    auto G = static_cast<const __nv_bfloat16*>(gamma);
+    auto R = static_cast<const __nv_bfloat16*>(resid);
+    auto DX = static_cast<__nv_bfloat16*>(dx);
+    auto Mu = static_cast<const float*>(mu);
+    auto Rs = static_cast<const float*>(rstd);
+    auto P = static_cast<float*>(partials);
+    switch (rp.chunks) {
+        case 1: ln_bwd_kernel<1><<<grid, rp.threads, 0, stream>>>(DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
+        case 2: ln_bwd_kernel<2><<<grid, rp.threads, 0, stream>>>(DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
+        default: ln_bwd_kernel<4><<<grid, rp.threads, 0, stream>>>(DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
+    }
+    if (cudaGetLastError() != cudaSuccess) return "layernorm bwd launch failed";
+    ReduceOuts outs;
+    outs.out[0] = static_cast<float*>(dgamma); outs.out[1] = static_cast<float*>(dbeta);
+    outs.out[2] = static_cast<float*>(db_resid); outs.out[3] = static_cast<float*>(db_dx);
+    dim3 rgrid((d + 255) / 256, 4);
+    reduce_partials_kernel<<<rgrid, 256, 0, stream>>>(P, grid * rp.rows_per_cta, 4, d, outs, accumulate);
+    return cudaGetLastError() == cudaSuccess ? nullptr : "layernorm bwd reduce launch failed";
+}
+
+size_t colsum_scratch_bytes(Runtime* rt, int T, int N)
+{
+    if (T <= 0 || N <= 0) return 0;
+    return static_cast<size_t>(colsum_splits(rt, T, N)) * N * sizeof(float);
+}
+
+const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, void* out, int accumulate,
+                          void* partials, cudaStream_t stream)
+{
+    if (T <= 0 || N <= 0 || (N % 8) || (ld % 8)) return "colsum: N and ld must be multiples of 8";
+    const int R = colsum_splits(rt, T, N);
+    dim3 grid((N + 1023) / 1024, R);
+    colsum_kernel<<<grid, 128, 0, stream>>>(static_cast<const __nv_bfloat16*>(in), T, N, ld, static_cast<float*>(partials));
+    if (cudaGetLastError() != cudaSuccess) return "colsum launch failed";
+    ReduceOuts outs;
+    outs.out[0] = static_cast<float*>(out); outs.out[1] = outs.out[2] = outs.out[3] = nullptr;
+    dim3 rgrid((N + 255) / 256, 1);
+    reduce_partials_kernel<<<rgrid, 256, 0, stream>>>(static_cast<const float*>(partials), R, 1, N, outs, accumulate);
+    return cudaGetLastError() == cudaSuccess ? nullptr : "colsum reduce launch failed";
+}
+
+}  // namespace pw

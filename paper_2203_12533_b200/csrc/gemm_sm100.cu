@@ -1,0 +1,318 @@
+// bf16 GEMM for sm_100a: TMA -> 4-stage shared-memory ring -> tcgen05.mma (fp32 accumulators in
+// TMEM, double buffered) -> epilogue warps (tcgen05.ld -> bias / GeLU / residual -> global).
+//
+// One persistent CTA per SM, 6 warps: warp 0 = TMA producer (one lane), warp 1 = MMA issuer (one
+// lane; the warp also owns the TMEM allocation), warps 2..5 = epilogue (warp w reads TMEM lanes
+// 32*(w%4) .. +31, i.e. 32 rows of the 128-row tile each).  Output tile 128 x 256, K step 64.
+//
+// Operand layouts are handled without physical transposes: an operand whose contraction index
+// is contiguous in memory ("K-major") is loaded as [rows][64 k] boxes, one whose row index is
+// contiguous ("MN-major": the weight in dgrad, both operands in wgrad) as [64 k][64 rows] boxes;
+// both use the 128-byte swizzle and the matching shared-memory descriptors.
+//
+// Every wait on an mbarrier is bounded (see mbar_wait); on expiry the CTA raises an abort flag,
+// all roles leave their loops, the TMEM allocation is released and the kernel returns.
+#include "pw_kernels.h"
+
+namespace pw {
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr int A_TILE_BYTES = BM * BK * 2;   // 16 KB
+constexpr int B_TILE_BYTES = BN * BK * 2;   // 32 KB
+constexpr int STAGE_BYTES = A_TILE_BYTES + B_TILE_BYTES;
+constexpr int GEMM_THREADS = 192;
+constexpr int TMEM_COLS = 2 * BN;           // two accumulators: the whole 512-column TMEM
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+struct GemmParams {
+    int M, N, K;
+    void* C; int ldc;
+    const __nv_bfloat16* bias;
+    const __nv_bfloat16* aux_in; int ld_aux;
+    __nv_bfloat16* aux_out;
+    int accumulate, act;
+    int m_tiles, n_tiles;
+    DeviceStatus* status;
+};
+
+template <int EPI>
+__device__ __forceinline__ void epilogue_chunk(const uint32_t* v, int row, int col0, const GemmParams& p)
+{
+    if constexpr (EPI == kEpiF32) {
+        float* c = reinterpret_cast<float*>(p.C) + static_cast<size_t>(row) * p.ldc + col0;
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            if (col0 + 4 * g < p.N) {
+                float4 o = make_float4(__uint_as_float(v[4 * g]), __uint_as_float(v[4 * g + 1]),
+                                       __uint_as_float(v[4 * g + 2]), __uint_as_float(v[4 * g + 3]));
+                if (p.accumulate) {
+                    float4 old = *reinterpret_cast<const float4*>(c + 4 * g);
+                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                }
+                *reinterpret_cast<float4*>(c + 4 * g) = o;
+            }
+        }
+    } else {
+        __nv_bfloat16* c = reinterpret_cast<__nv_bfloat16*>(p.C) + static_cast<size_t>(row) * p.ldc + col0;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            if (col0 + 8 * g < p.N) {
+                float f[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[8 * g + j]);
+                if constexpr (EPI == kEpiBias || EPI == kEpiBiasResid || EPI == kEpiBiasGelu) {
+                    float b[8];
+                    unpack8(__ldg(reinterpret_cast<const uint4*>(p.bias + col0 + 8 * g)), b);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) f[j] += b[j];
+                }
+                if constexpr (EPI == kEpiBiasResid) {
+                    float r[8];
+                    unpack8(*reinterpret_cast<const uint4*>(p.aux_in + static_cast<size_t>(row) * p.ld_aux + col0 + 8 * g), r);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) f[j] += r[j];
+                }
+                if constexpr (EPI == kEpiDGelu) {
+                    float u[8];
+                    unpack8(*reinterpret_cast<const uint4*>(p.aux_in + static_cast<size_t>(row) * p.ld_aux + col0 + 8 * g), u);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) f[j] *= gelu_grad_f(u[j], p.act);
+                }
+                *reinterpret_cast<uint4*>(c + 8 * g) = pack8(f);
+                if constexpr (EPI == kEpiBiasGelu) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) f[j] = gelu_f(f[j], p.act);
+                    *reinterpret_cast<uint4*>(p.aux_out + static_cast<size_t>(row) * p.ldc + col0 + 8 * g) = pack8(f);
+                }
+            }
+        }
+    }
+}
+
+template <bool A_MN, bool B_MN, int EPI>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + STAGES * STAGE_BYTES);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + STAGES);
+    const uint32_t accf0 = smem_u32(bars + 2 * STAGES), acce0 = smem_u32(bars + 2 * STAGES + 2);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_k = (p.K + BK - 1) / BK;
+    const int total_tiles = p.m_tiles * p.n_tiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 128); }
+        *abort_flag = 0;
+        fence_barrier_init();
+        fence_proxy_async();
+        prefetch_tmap(&tmA);
+        prefetch_tmap(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile % p.m_tiles) * BM, n0 = (tile / p.m_tiles) * BN;
+                for (int kb = 0; kb < num_k; ++kb) {
+                    if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 100)) { ok = false; break; }
+                    const uint32_t fb = full0 + 8 * stage;
+                    mbar_arrive_expect_tx(fb, STAGE_BYTES);
+                    const uint32_t a_dst = smem_u32(tiles + stage * STAGE_BYTES), b_dst = a_dst + A_TILE_BYTES;
+                    if constexpr (!A_MN) {
+                        tma_load_2d(a_dst, &tmA, kb * BK, m0, fb);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < BM / 64; ++j) tma_load_2d(a_dst + j * 8192, &tmA, m0 + 64 * j, kb * BK, fb);
+                    }
+                    if constexpr (!B_MN) {
+                        tma_load_2d(b_dst, &tmB, kb * BK, n0, fb);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < BN / 64; ++j) tma_load_2d(b_dst + j * 8192, &tmB, n0 + 64 * j, kb * BK, fb);
+                    }
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(BM, BN, A_MN, B_MN);
+            uint32_t stage = 0, phase = 0, it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+                const uint32_t buf = it & 1, acc_phase = (it >> 1) & 1;
+                if (!mbar_wait(acce0 + 8 * buf, acc_phase ^ 1, abort_flag, p.status, 200)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kb = 0; kb < num_k; ++kb) {
+                    if (!mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 201)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_base = smem_u32(tiles + stage * STAGE_BYTES), b_base = a_base + A_TILE_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+                        // K-major: 16 k = 32 bytes along the swizzled 128-byte row; 8-row groups 1024 B apart.
+                        // MN-major: 16 k = two 8-k groups of 1024 B; 64-row groups 8192 B apart.
+                        const uint64_t adesc = A_MN ? make_smem_desc_sw128(a_base + kk * 2048, 8192, 1024)
+                                                    : make_smem_desc_sw128(a_base + kk * 32, 16, 1024);
+                        const uint64_t bdesc = B_MN ? make_smem_desc_sw128(b_base + kk * 2048, 8192, 1024)
+                                                    : make_smem_desc_sw128(b_base + kk * 32, 16, 1024);
+                        umma_f16(d_tmem, adesc, bdesc, idesc, (kb | kk) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(empty0 + 8 * stage);   // frees the stage once these MMAs have read it
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (ok) umma_commit(accf0 + 8 * buf);  // accumulator complete
+            }
+        }
+    } else {
+        const int ew = warp & 3;
+        uint32_t it = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
+            const int m0 = (tile % p.m_tiles) * BM, n0 = (tile / p.m_tiles) * BN;
+            const uint32_t buf = it & 1, acc_phase = (it >> 1) & 1;
+            bool ok = mbar_wait(accf0 + 8 * buf, acc_phase, abort_flag, p.status, 300);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const int row = m0 + ew * 32 + lane;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(ew * 32) << 16) + buf * BN;
+#pragma unroll 1
+            for (int chunk = 0; chunk < BN / 32; ++chunk) {
+                const int col0 = n0 + chunk * 32;
+                if (col0 >= p.N) break;
+                uint32_t v[32];
+                tmem_ld32(taddr + chunk * 32, v);
+                tc_wait_ld();
+                if (row < p.M) epilogue_chunk<EPI>(v, row, col0, p);
+            }
+            tc_fence_before();
+            mbar_arrive(acce0 + 8 * buf);
+        }
+    }
+
+    __syncwarp();
+    if (*abort_flag) {   // give copies and MMAs still in flight time to land before releasing anything
+        const long long t0 = clock64();
+        while (clock64() - t0 < (1ll << 22)) {}
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 2-D bf16 tensor map: `inner` contiguous elements per row, `outer` rows, row pitch ld elements.
+const char* encode_2d(Runtime* rt, CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t outer, uint64_t ld,
+                      uint32_t box_inner, uint32_t box_outer)
+{
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {ld * 2};
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = reinterpret_cast<EncodeTiledFn>(rt->encode_tiled)(
+        map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? nullptr : "cuTensorMapEncodeTiled failed";
+}
+
+template <bool A_MN, bool B_MN, int EPI>
+const char* launch_inst(Runtime* rt, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p,
+                        cudaStream_t stream)
+{
+    auto kern = gemm_kernel<A_MN, B_MN, EPI>;
+    const int total = p.m_tiles * p.n_tiles;
+    const int grid = total < rt->sm_count ? total : rt->sm_count;
+    kern<<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, p);
+    return cudaGetLastError() == cudaSuccess ? nullptr : "gemm launch failed";
+}
+
+template <bool A_MN, bool B_MN, int EPI>
+bool set_attr()
+{
+    return cudaFuncSetAttribute(gemm_kernel<A_MN, B_MN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                SMEM_BYTES) == cudaSuccess;
+}
+
+}  // namespace
+
+// Opt every instantiation into its dynamic shared-memory size, once per process (never on the
+// enqueue path, so a stream capture sees launches only).
+const char* configure_gemm()
+{
+    const bool ok = set_attr<false, false, kEpiNone>() && set_attr<false, false, kEpiBias>() &&
+                    set_attr<false, false, kEpiBiasResid>() && set_attr<false, false, kEpiBiasGelu>() &&
+                    set_attr<false, true, kEpiNone>() && set_attr<false, true, kEpiDGelu>() &&
+                    set_attr<true, true, kEpiF32>();
+    return ok ? nullptr : "cudaFuncSetAttribute(gemm) failed";
+}
+
+const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cudaStream_t stream)
+{
+    if (a.M <= 0 || a.N <= 0 || a.K <= 0) return "gemm: non-positive dimension";
+    if ((a.M % 8) || (a.N % 8) || (a.K % 8)) return "gemm: M, N, K must be multiples of 8";
+    if ((a.lda % 8) || (a.ldb % 8) || (a.ldc % 8)) return "gemm: leading dimensions must be multiples of 8";
+    auto misaligned = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15) != 0; };
+    if (!a.A || !a.B || !a.C || misaligned(a.A) || misaligned(a.B) || misaligned(a.C)) return "gemm: null or misaligned operand";
+    const bool need_bias = a.epilogue == kEpiBias || a.epilogue == kEpiBiasResid || a.epilogue == kEpiBiasGelu;
+    const bool need_aux_in = a.epilogue == kEpiBiasResid || a.epilogue == kEpiDGelu;
+    if (need_bias && (!a.bias || misaligned(a.bias))) return "gemm: epilogue needs a 16-byte aligned bias";
+    if (need_aux_in && (!a.aux_in || misaligned(a.aux_in) || (a.ld_aux % 8))) return "gemm: epilogue needs aux_in";
+    if (a.epilogue == kEpiBiasGelu && (!a.aux_out || misaligned(a.aux_out))) return "gemm: epilogue needs aux_out";
+
+    const bool a_mn = a.layout == kNT, b_mn = a.layout == kNN || a.layout == kNT;
+    CUtensorMap tmA, tmB;
+    const char* e;
+    // K-major operand [rows, K]: box 64 k x rows.  MN-major operand stored [K, rows]: box 64 rows x 64 k.
+    e = a_mn ? encode_2d(rt, &tmA, a.A, a.M, a.K, a.lda, 64, BK) : encode_2d(rt, &tmA, a.A, a.K, a.M, a.lda, BK, BM);
+    if (e) return e;
+    e = b_mn ? encode_2d(rt, &tmB, a.B, a.N, a.K, a.ldb, 64, BK) : encode_2d(rt, &tmB, a.B, a.K, a.N, a.ldb, BK, BN);
+    if (e) return e;
+
+    GemmParams p;
+    p.M = a.M; p.N = a.N; p.K = a.K;
+    p.C = a.C; p.ldc = a.ldc;
+    p.bias = static_cast<const __nv_bfloat16*>(a.bias);
+    p.aux_in = static_cast<const __nv_bfloat16*>(a.aux_in); p.ld_aux = a.ld_aux;
+    p.aux_out = static_cast<__nv_bfloat16*>(a.aux_out);
+    p.accumulate = a.accumulate; p.act = a.act;
+    p.m_tiles = (a.M + BM - 1) / BM; p.n_tiles = (a.N + BN - 1) / BN;
+    p.status = status;
+
+    const int key = a.layout * 16 + a.epilogue;
+    switch (key) {
+        case kTN * 16 + kEpiNone: return launch_inst<false, false, kEpiNone>(rt, tmA, tmB, p, stream);
+        case kTN * 16 + kEpiBias: return launch_inst<false, false, kEpiBias>(rt, tmA, tmB, p, stream);
+        case kTN * 16 + kEpiBiasResid: return launch_inst<false, false, kEpiBiasResid>(rt, tmA, tmB, p, stream);
+        case kTN * 16 + kEpiBiasGelu: return launch_inst<false, false, kEpiBiasGelu>(rt, tmA, tmB, p, stream);
+        case kNN * 16 + kEpiNone: return launch_inst<false, true, kEpiNone>(rt, tmA, tmB, p, stream);
+        case kNN * 16 + kEpiDGelu: return launch_inst<false, true, kEpiDGelu>(rt, tmA, tmB, p, stream);
+        case kNT * 16 + kEpiF32: return launch_inst<true, true, kEpiF32>(rt, tmA, tmB, p, stream);
+        default: return "gemm: unsupported layout/epilogue combination";
+    }
+}
+
+}  // namespace pw

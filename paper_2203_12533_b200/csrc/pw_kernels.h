@@ -1,0 +1,62 @@
+// Internal launch interface between the host dispatch code and the kernels.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "pw_common.cuh"
+
+namespace pw {
+
+// Process-wide, per-device runtime state: SM count, the driver's tensor-map encoder, a default
+// status block for the single-step entry points.
+struct Runtime {
+    int device = -1;
+    int sm_count = 0;
+    int cc_major = 0;
+    void* encode_tiled = nullptr;      // cuTensorMapEncodeTiled, fetched through the runtime API
+    DeviceStatus* op_status = nullptr; // device memory, status block for pw_op_* calls
+};
+// Returns nullptr (and sets *err) if the device is not sm_100 or a CUDA call failed.
+Runtime* get_runtime(const char** err);
+
+// One-time kernel attribute set-up (dynamic shared-memory opt-in); called from get_runtime.
+const char* configure_gemm();
+const char* configure_attention();
+
+enum GemmLayout { kTN = 0, kNN = 1, kNT = 2 };
+enum GemmEpi { kEpiNone = 0, kEpiBias = 1, kEpiBiasResid = 2, kEpiBiasGelu = 3, kEpiDGelu = 4, kEpiF32 = 5 };
+
+struct GemmArgs {
+    int layout, epilogue, act;
+    int M, N, K;
+    const void* A; int lda;
+    const void* B; int ldb;
+    void* C; int ldc;
+    const void* bias;
+    const void* aux_in; int ld_aux;
+    void* aux_out;
+    int accumulate;
+};
+// Encodes the two tensor maps and launches.  Returns nullptr on success, else a static message.
+const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cudaStream_t stream);
+
+const char* launch_layernorm_fwd(Runtime* rt, const void* x, const void* gamma, const void* beta, int T, int d,
+                                 float eps, void* h, void* mu, void* rstd, cudaStream_t stream);
+size_t layernorm_bwd_scratch_bytes(Runtime* rt, int T, int d);
+const char* launch_layernorm_bwd(Runtime* rt, const void* dh, const void* x, const void* mu, const void* rstd,
+                                 const void* gamma, const void* resid, int T, int d, void* dx, void* dgamma,
+                                 void* dbeta, void* db_resid, void* db_dx, int accumulate, void* partials,
+                                 cudaStream_t stream);
+size_t colsum_scratch_bytes(Runtime* rt, int T, int N);
+const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, void* out, int accumulate,
+                          void* partials, cudaStream_t stream);
+
+const char* launch_attention_fwd(Runtime* rt, const void* qkv, int B, int S, int H, int dh, void* o, void* lse,
+                                 cudaStream_t stream);
+const char* launch_attention_bwd(Runtime* rt, const void* qkv, const void* o, const void* dout, const void* lse,
+                                 int B, int S, int H, int dh, void* dqkv, void* delta, cudaStream_t stream);
+
+}  // namespace pw

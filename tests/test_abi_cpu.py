@@ -1,0 +1,70 @@
+"""CPU-side checks of the boundary: the library builds, loads, and exports what include/pw.h declares."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def libpath():
+    from paper_2203_12533_b200 import build
+    return build.build()
+
+
+def declared_functions():
+    with open(os.path.join(ROOT, "include", "pw.h")) as f:
+        text = f.read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(pw_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(libpath):
+    lib = ctypes.CDLL(libpath)
+    names = declared_functions()
+    assert len(names) >= 20
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in pw.h but not exported"
+
+
+def test_binding_lists_the_same_symbols(libpath):
+    from paper_2203_12533_b200 import binding
+    assert sorted(binding.EXPORTS) == declared_functions()
+
+
+def test_version_and_status_strings(libpath):
+    lib = ctypes.CDLL(libpath)
+    lib.pw_status_string.restype = ctypes.c_char_p
+    assert lib.pw_version() == 100
+    assert lib.pw_status_string(0) == b"PW_OK"
+    assert lib.pw_status_string(6) == b"PW_ERR_TIMEOUT"
+
+
+def test_config_struct_matches_header():
+    from paper_2203_12533_b200 import binding
+    assert ctypes.sizeof(binding.LayerConfig) == 44          # 11 four-byte fields, no padding
+    assert ctypes.sizeof(binding._Ptr12) == 12 * ctypes.sizeof(ctypes.c_void_p)
+
+
+def test_argument_errors_need_no_gpu(libpath):
+    """Validation runs before any device work, so these fail the same way without a GPU."""
+    from paper_2203_12533_b200 import binding
+    lib = binding.lib()
+    h = ctypes.c_void_p()
+    bad = binding.make_config(2048, 16, 100, 8192, 1024, 8)           # head_dim not 64/128
+    assert lib.pw_layer_create(ctypes.byref(bad), ctypes.byref(h)) == 2
+    assert b"head_dim" in lib.pw_last_error()
+    bad = binding.make_config(2048, 16, 128, 8192, 1000, 8)           # seq_len not a multiple of 128
+    assert lib.pw_layer_create(ctypes.byref(bad), ctypes.byref(h)) == 2
+    bad = binding.make_config(2048, 8, 128, 8192, 1024, 8)            # heads * head_dim != d_model
+    assert lib.pw_layer_create(ctypes.byref(bad), ctypes.byref(h)) == 2
+    bad = binding.make_config(2048, 16, 128, 8192, 1024, 8)
+    bad.struct_size = 8
+    assert lib.pw_layer_create(ctypes.byref(bad), ctypes.byref(h)) == 1
+    assert lib.pw_layer_create(None, ctypes.byref(h)) == 1
+    import torch
+    if not torch.cuda.is_available():
+        ok = binding.make_config(2048, 16, 128, 8192, 1024, 8)
+        assert lib.pw_layer_create(ctypes.byref(ok), ctypes.byref(h)) == 5   # no device: loud failure, no fallback

@@ -1,0 +1,212 @@
+"""GPU parity of the single steps (through the C ABI) against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from tests.gpu_util import ACT_TOL, GRAD_TOL, bf16_randn, guard_alloc, np64, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pw():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2203_12533_b200 import binding
+    binding.lib()          # raises loudly if the library is not built
+    return binding
+
+
+def _status_ok(pw):
+    code, site = pw.op_status()
+    assert code == 0, f"device status {code} at site {site}"
+
+
+# ------------------------------------------------------------------------------------------ GEMM
+def test_gemm_tn_integer_exact(pw):
+    """Small integers are exact in bf16 and in the fp32 accumulator: any mis-tiled block shows up exactly."""
+    g = torch.Generator().manual_seed(1)
+    M, N, K = 384, 520, 64
+    A = torch.randint(-2, 3, (M, K), generator=g).to(torch.bfloat16)
+    B = torch.randint(-2, 3, (N, K), generator=g).to(torch.bfloat16)
+    C, check = guard_alloc((M, N), torch.bfloat16)
+    pw.op_gemm(pw.GEMM_TN, pw.EPI_NONE, M, N, K, A.cuda(), K, B.cuda(), K, C, N)
+    torch.cuda.synchronize()
+    _status_ok(pw)
+    check()
+    want = A.double() @ B.double().T
+    assert torch.equal(C.double().cpu(), want)
+
+
+SHAPES = [(392, 520, 200), (128, 256, 64), (1000, 768, 1032)]
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+@pytest.mark.parametrize("epi", ["none", "bias", "bias_resid", "bias_gelu"])
+def test_gemm_tn_epilogues(pw, oracle64, M, N, K, epi):
+    g = torch.Generator().manual_seed(2)
+    A, W = bf16_randn((M, K), g), bf16_randn((N, K), g, 0.1)
+    bias, R = bf16_randn((N,), g), bf16_randn((M, N), g)
+    C, check = guard_alloc((M, N), torch.bfloat16)
+    aux, check2 = guard_alloc((M, N), torch.bfloat16)
+    code = {"none": pw.EPI_NONE, "bias": pw.EPI_BIAS, "bias_resid": pw.EPI_BIAS_RESID, "bias_gelu": pw.EPI_BIAS_GELU}[epi]
+    pw.op_gemm(pw.GEMM_TN, code, M, N, K, A.cuda(), K, W.cuda(), K, C, N, bias=bias.cuda(),
+               aux_in=R.cuda() if epi == "bias_resid" else None, ld_aux=N,
+               aux_out=aux if epi == "bias_gelu" else None)
+    torch.cuda.synchronize()
+    _status_ok(pw)
+    check(); check2()
+    want = oracle64.linear_fwd(np64(A), np64(W), np64(bias) if epi != "none" else None)
+    if epi == "bias_resid":
+        want = want + np64(R)
+    assert rel_l2(C, want) < ACT_TOL
+    if epi == "bias_gelu":
+        assert rel_l2(aux, oracle64.gelu_fwd(want)) < ACT_TOL
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+@pytest.mark.parametrize("epi", ["none", "dgelu"])
+def test_gemm_nn_dgrad(pw, oracle64, M, N, K, epi):
+    """C[M,N] = A[M,K] B[K,N]  (dx = dy W with W stored [out=K, in=N])."""
+    g = torch.Generator().manual_seed(3)
+    A, W = bf16_randn((M, K), g), bf16_randn((K, N), g, 0.1)
+    U = bf16_randn((M, N), g)
+    C, check = guard_alloc((M, N), torch.bfloat16)
+    pw.op_gemm(pw.GEMM_NN, pw.EPI_DGELU if epi == "dgelu" else pw.EPI_NONE, M, N, K, A.cuda(), K, W.cuda(), N, C, N,
+               aux_in=U.cuda() if epi == "dgelu" else None, ld_aux=N)
+    torch.cuda.synchronize()
+    _status_ok(pw)
+    check()
+    dx, _, _ = oracle64.linear_bwd(np.zeros((M, N)), np64(W), np64(A))   # dx[t][n] = sum_k dout[t][k] W[k][n]
+    if epi == "dgelu":
+        dx = oracle64.gelu_bwd(np64(U), dx)
+    assert rel_l2(C, dx) < GRAD_TOL
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+@pytest.mark.parametrize("accumulate", [False, True])
+def test_gemm_nt_wgrad(pw, oracle64, M, N, K, accumulate):
+    """C[M,N] (+)= A[K,M]^T B[K,N]  (dW = dy^T x), fp32 output."""
+    g = torch.Generator().manual_seed(4)
+    A, B = bf16_randn((K, M), g), bf16_randn((K, N), g)
+    C, check = guard_alloc((M, N), torch.float32)
+    C0 = torch.randn((M, N), generator=g)
+    C.copy_(C0)
+    pw.op_gemm(pw.GEMM_NT, pw.EPI_F32, M, N, K, A.cuda(), M, B.cuda(), N, C, N, accumulate=accumulate)
+    torch.cuda.synchronize()
+    _status_ok(pw)
+    check()
+    _, dW, _ = oracle64.linear_bwd(np64(B), np.zeros((M, N)), np64(A))   # dW[m][n] = sum_k A[k][m] B[k][n]
+    if accumulate:
+        dW = dW + np64(C0)
+    assert rel_l2(C, dW) < 1e-5
+
+
+def test_gemm_is_deterministic(pw):
+    g = torch.Generator().manual_seed(5)
+    M, N, K = 640, 512, 448
+    A, W = bf16_randn((M, K), g).cuda(), bf16_randn((N, K), g).cuda()
+    C1 = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    C2 = torch.empty_like(C1)
+    pw.op_gemm(pw.GEMM_TN, pw.EPI_NONE, M, N, K, A, K, W, K, C1, N)
+    pw.op_gemm(pw.GEMM_TN, pw.EPI_NONE, M, N, K, A, K, W, K, C2, N)
+    torch.cuda.synchronize()
+    assert torch.equal(C1, C2)
+
+
+def test_gemm_rejects_bad_arguments(pw):
+    A = torch.zeros((128, 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(pw.PwError):
+        pw.op_gemm(pw.GEMM_TN, pw.EPI_NONE, 128, 128, 60, A, 64, A, 64, A, 128)        # K not a multiple of 8
+    with pytest.raises(pw.PwError):
+        pw.op_gemm(pw.GEMM_TN, pw.EPI_BIAS, 128, 128, 64, A, 64, A, 64, A, 128)        # bias missing
+    with pytest.raises(pw.PwError):
+        pw.op_gemm(pw.GEMM_NT, pw.EPI_BIAS, 128, 128, 64, A, 64, A, 64, A, 128, bias=A)  # unsupported combination
+
+
+# ------------------------------------------------------------------------------------------ LayerNorm / column sums
+@pytest.mark.parametrize("T,d", [(77, 256), (130, 1024), (515, 2048), (70, 4096), (33, 8192), (64, 1536)])
+def test_layernorm_fwd_bwd(pw, oracle64, T, d):
+    g = torch.Generator().manual_seed(6)
+    x = bf16_randn((T, d), g, 2.0) + 0.5
+    x = x.to(torch.bfloat16)
+    gamma = (1 + 0.2 * torch.randn(d, generator=g)).to(torch.bfloat16)
+    beta = (0.2 * torch.randn(d, generator=g)).to(torch.bfloat16)
+    dh, resid = bf16_randn((T, d), g), bf16_randn((T, d), g)
+    h, check_h = guard_alloc((T, d), torch.bfloat16)
+    mu = torch.empty(T, device="cuda"); r = torch.empty(T, device="cuda")
+    pw.op_layernorm_fwd(x.cuda(), gamma.cuda(), beta.cuda(), 1e-5, h, mu, r)
+    torch.cuda.synchronize()
+    check_h()
+    hw, muw, rw = oracle64.ln_fwd(np64(x), np64(gamma), np64(beta), 1e-5)
+    assert rel_l2(h, hw) < ACT_TOL and rel_l2(mu, muw) < 1e-5 and rel_l2(r, rw) < 1e-5
+
+    dx, check_dx = guard_alloc((T, d), torch.bfloat16)
+    outs = [torch.full((d,), 3.0, device="cuda") for _ in range(4)]
+    part = torch.empty(pw.op_layernorm_bwd_scratch_bytes(T, d), dtype=torch.uint8, device="cuda")
+    for acc in (False, True):
+        pw.op_layernorm_bwd(dh.cuda(), x.cuda(), mu, r, gamma.cuda(), resid.cuda(), dx, outs[0], outs[1], outs[2],
+                            outs[3], acc, part)
+    torch.cuda.synchronize()
+    check_dx()
+    dxw, dgw, dbw = oracle64.ln_bwd(np64(dh), np64(x), muw, rw, np64(gamma))
+    dxw = dxw + np64(resid)
+    assert rel_l2(dx, dxw) < GRAD_TOL
+    assert rel_l2(outs[0], 2 * dgw) < GRAD_TOL and rel_l2(outs[1], 2 * dbw) < GRAD_TOL   # overwrite, then accumulate
+    assert rel_l2(outs[2], 2 * np64(resid).sum(0)) < 1e-4
+    assert rel_l2(outs[3], 2 * dxw.sum(0)) < GRAD_TOL
+
+
+@pytest.mark.parametrize("T,N", [(100, 256), (1000, 3072), (777, 8192), (5, 1032)])
+def test_colsum(pw, T, N):
+    g = torch.Generator().manual_seed(7)
+    a = bf16_randn((T, N), g)
+    out = torch.full((N,), 1.0, device="cuda")
+    part = torch.empty(max(16, pw.op_colsum_scratch_bytes(T, N)), dtype=torch.uint8, device="cuda")
+    pw.op_colsum(a.cuda(), out, False, part)
+    pw.op_colsum(a.cuda(), out, True, part)
+    torch.cuda.synchronize()
+    assert rel_l2(out, 2 * np64(a).sum(0)) < 1e-5
+
+
+# ------------------------------------------------------------------------------------------ attention
+@pytest.mark.parametrize("B,S,H,dh", [(2, 128, 2, 64), (2, 384, 3, 64), (1, 256, 2, 128), (2, 640, 1, 128)])
+def test_attention_fwd_bwd(pw, oracle64, B, S, H, dh):
+    g = torch.Generator().manual_seed(8)
+    d = H * dh
+    qkv = bf16_randn((B * S, 3 * d), g)
+    dout = bf16_randn((B * S, d), g)
+    o, check_o = guard_alloc((B * S, d), torch.bfloat16)
+    lse, check_l = guard_alloc((B, H, S), torch.float32)
+    pw.op_attention_fwd(qkv.cuda(), B, S, H, dh, o, lse)
+    torch.cuda.synchronize()
+    check_o(); check_l()
+    ow, lw = oracle64.attn_fwd(np64(qkv), B, S, H, dh)
+    assert rel_l2(o, ow) < ACT_TOL
+    assert np.abs(lse.double().cpu().numpy() - lw).max() < 1e-3
+
+    dqkv, check_d = guard_alloc((B * S, 3 * d), torch.bfloat16)
+    delta = torch.empty((B, H, S), device="cuda")
+    pw.op_attention_bwd(qkv.cuda(), o, dout.cuda(), lse, B, S, H, dh, dqkv, delta)
+    torch.cuda.synchronize()
+    check_d()
+    dw = oracle64.attn_bwd(np64(qkv), np64(dout), B, S, H, dh)
+    for name, sl in (("dq", slice(0, d)), ("dk", slice(d, 2 * d)), ("dv", slice(2 * d, 3 * d))):
+        assert rel_l2(dqkv[:, sl], dw[:, sl]) < GRAD_TOL, name
+
+
+def test_attention_is_causal_and_deterministic(pw):
+    g = torch.Generator().manual_seed(9)
+    B, S, H, dh = 1, 256, 2, 64
+    d = H * dh
+    qkv = bf16_randn((B * S, 3 * d), g).cuda()
+    o1 = torch.empty((B * S, d), dtype=torch.bfloat16, device="cuda"); o2 = torch.empty_like(o1); o3 = torch.empty_like(o1)
+    lse = torch.empty((B, H, S), device="cuda")
+    pw.op_attention_fwd(qkv, B, S, H, dh, o1, lse)
+    pw.op_attention_fwd(qkv, B, S, H, dh, o2, lse)
+    q2 = qkv.clone()
+    q2[150:] += 1.0                                    # tokens >= 150 change; outputs at positions < 150 must not
+    pw.op_attention_fwd(q2, B, S, H, dh, o3, lse)
+    torch.cuda.synchronize()
+    assert torch.equal(o1, o2)
+    assert torch.equal(o1[:150], o3[:150]) and not torch.equal(o1[150:], o3[150:])
