@@ -33,3 +33,34 @@ def guard_alloc(shape, dtype, device="cuda", pad=256):
     def check():
         assert torch.isnan(buf[:pad]).all() and torch.isnan(buf[pad + n:]).all(), "write outside the output buffer"
     return view, check
+
+
+def dims_of(w):
+    """oracle.Dims for an inputs.Workload."""
+    from oracle import Dims
+    return Dims(w.batch, w.seq_len, w.d_model, w.n_heads, w.head_dim, w.d_ff)
+
+
+def make_layer(pw, w, act=0):
+    return pw.Layer(w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch, act=act)
+
+
+def zeros_like_params(w, device="cuda"):
+    return [torch.zeros(s, dtype=torch.float32, device=device) for s in w.param_shapes()]
+
+
+def run_layer_gpu(pw, layer, params_dev, x_dev, dy_dev, save_ctx=True, grads=None, accumulate=False):
+    """One forward + backward through the C ABI.  Returns dict(y, dx, grads, ctx, scratch)."""
+    T, d = layer.T, layer.d
+    y = torch.empty((T, d), dtype=torch.bfloat16, device="cuda")
+    dx = torch.empty_like(y)
+    ctx = torch.empty(layer.ctx_bytes, dtype=torch.uint8, device="cuda") if save_ctx else None
+    scratch = torch.empty(layer.scratch_bytes, dtype=torch.uint8, device="cuda")
+    if grads is None:
+        grads = [torch.full(p.shape, float("nan"), dtype=torch.float32, device="cuda") for p in params_dev]
+    layer.fwd(params_dev, x_dev, y, ctx, scratch)
+    layer.bwd(params_dev, x_dev, dy_dev, dx, grads, accumulate, ctx, scratch)
+    torch.cuda.synchronize()
+    code, site = layer.status()
+    assert code == 0, f"device status {code} at site {site}"
+    return dict(y=y, dx=dx, grads=grads, ctx=ctx, scratch=scratch)

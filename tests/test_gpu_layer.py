@@ -1,0 +1,201 @@
+"""GPU parity of the whole layer and of the stage chain (through the C ABI) against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2203_12533_b200 import inputs
+from tests.gpu_util import (ACT_TOL, GRAD_TOL, dims_of, make_layer, np64, rel_l2, run_layer_gpu)
+
+pytestmark = pytest.mark.gpu
+
+SAVED_BF16 = ("h1", "qkv", "o", "x1", "h2", "u", "a")
+
+
+@pytest.fixture(scope="module")
+def pw():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2203_12533_b200 import binding
+    binding.lib()
+    return binding
+
+
+def check_layer_against_oracle(pw, oracle, w, random_ln=False, act=0, save_ctx=True):
+    from oracle import Dims
+    D = dims_of(w)
+    D = Dims(D.B, D.S, D.d, D.H, D.dh, D.F, D.eps, act)
+    params = inputs.layer_params(w, seed=0, layer=0, random_ln=random_ln)
+    x, dy = inputs.microbatch(w, seed=0, m=0)
+    layer = make_layer(pw, w, act)
+    out = run_layer_gpu(pw, layer, [p.cuda() for p in params], x.cuda().view(-1, w.d_model),
+                        dy.cuda().view(-1, w.d_model), save_ctx=save_ctx)
+    cast = (lambda t: t.float().numpy()) if oracle.suf == "f32" else np64
+    ps = [cast(p) for p in params]
+    yw, sv = oracle.layer_fwd(D, ps, cast(x))
+    dxw, gw = oracle.layer_bwd(D, ps, cast(x), sv, cast(dy))
+    errs = {"y": rel_l2(out["y"], yw)}
+    store = out["ctx"] if save_ctx else out["scratch"]
+    for name in SAVED_BF16:
+        errs[name] = rel_l2(layer.ctx_view(store, name), sv[name])
+    for name in ("lse", "mu1", "r1", "mu2", "r2"):
+        errs[name] = rel_l2(layer.ctx_view(store, name), sv[name])
+    gerrs = {"dx": rel_l2(out["dx"], dxw)}
+    for name, g, want in zip(pw.PARAM_NAMES, out["grads"], gw):
+        gerrs["d" + name] = rel_l2(g, want)
+    assert max(errs.values()) < ACT_TOL, errs
+    assert max(gerrs.values()) < GRAD_TOL, gerrs
+    return errs, gerrs
+
+
+def test_cfg1_parity_all_tensors(pw, oracle64):
+    check_layer_against_oracle(pw, oracle64, inputs.WORKLOADS[1])
+
+
+def test_random_layernorm_params_and_tanh_gelu(pw, oracle64):
+    w = inputs.Workload("ragged", 512, 4, 128, 1152, 256, 3, sigma_w=0.05)    # T = 768, F not a multiple of 256
+    check_layer_against_oracle(pw, oracle64, w, random_ln=True)
+    check_layer_against_oracle(pw, oracle64, w, random_ln=True, act=1)
+
+
+def test_midsize_dh64(pw, oracle64):
+    w = inputs.Workload("mid", 768, 12, 64, 3072, 384, 2, sigma_w=0.03)
+    check_layer_against_oracle(pw, oracle64, w, random_ln=True)
+
+
+def test_recompute_matches_saved_bitwise_and_is_deterministic(pw):
+    w = inputs.WORKLOADS[1].with_(seq_len=256)
+    params = [p.cuda() for p in inputs.layer_params(w, random_ln=True)]
+    x, dy = inputs.microbatch(w)
+    x, dy = x.cuda().view(-1, w.d_model), dy.cuda().view(-1, w.d_model)
+    layer = make_layer(pw, w)
+    a = run_layer_gpu(pw, layer, params, x, dy, save_ctx=True)
+    b = run_layer_gpu(pw, layer, params, x, dy, save_ctx=False)     # backward re-runs the forward into scratch
+    c = run_layer_gpu(pw, layer, params, x, dy, save_ctx=True)
+    for other in (b, c):
+        assert torch.equal(a["y"], other["y"]) and torch.equal(a["dx"], other["dx"])
+        for g1, g2 in zip(a["grads"], other["grads"]):
+            assert torch.equal(g1, g2)
+
+
+def test_accumulate_adds(pw):
+    w = inputs.WORKLOADS[1]
+    params = [p.cuda() for p in inputs.layer_params(w)]
+    x, dy = inputs.microbatch(w)
+    x, dy = x.cuda().view(-1, w.d_model), dy.cuda().view(-1, w.d_model)
+    layer = make_layer(pw, w)
+    one = run_layer_gpu(pw, layer, params, x, dy)
+    acc = run_layer_gpu(pw, layer, params, x, dy, grads=[g.clone() for g in one["grads"]], accumulate=True)
+    for g1, g2 in zip(one["grads"], acc["grads"]):
+        assert rel_l2(g2, 2 * g1.double()) < 1e-6
+
+
+def test_dx_may_alias_dy(pw):
+    w = inputs.WORKLOADS[1]
+    params = [p.cuda() for p in inputs.layer_params(w)]
+    x, dy = inputs.microbatch(w)
+    x, dy = x.cuda().view(-1, w.d_model), dy.cuda().view(-1, w.d_model)
+    layer = make_layer(pw, w)
+    ref = run_layer_gpu(pw, layer, params, x, dy)
+    y = torch.empty_like(x)
+    ctx = torch.empty(layer.ctx_bytes, dtype=torch.uint8, device="cuda")
+    scratch = torch.empty(layer.scratch_bytes, dtype=torch.uint8, device="cuda")
+    g = dy.clone()
+    grads = [torch.empty_like(t) for t in ref["grads"]]
+    layer.fwd(params, x, y, ctx, scratch)
+    layer.bwd(params, x, g, g, grads, False, ctx, scratch)
+    torch.cuda.synchronize()
+    assert torch.equal(g, ref["dx"])
+
+
+def test_layer_argument_errors(pw):
+    w = inputs.WORKLOADS[1]
+    layer = make_layer(pw, w)
+    params = [p.cuda() for p in inputs.layer_params(w)]
+    x = torch.zeros((w.tokens, w.d_model), dtype=torch.bfloat16, device="cuda")
+    y = torch.empty_like(x)
+    ctx = torch.empty(layer.ctx_bytes, dtype=torch.uint8, device="cuda")
+    scratch = torch.empty(layer.scratch_bytes + 256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(pw.PwError) as e:
+        layer.fwd(params, x, x, ctx, scratch)                      # y aliases x
+    assert e.value.status == 1
+    with pytest.raises(pw.PwError):
+        layer.fwd(params, x, y, ctx[8:], scratch)                  # misaligned ctx
+    with pytest.raises(pw.PwError):
+        layer.fwd(params[:11] + [None], x, y, ctx, scratch)        # missing parameter
+    grads = [torch.zeros(p.shape, dtype=torch.float32, device="cuda") for p in params]
+    with pytest.raises(pw.PwError):
+        layer.bwd(params, x, y, y, grads, 2, ctx, scratch)         # accumulate must be 0/1
+    with pytest.raises(pw.PwError):
+        pw.Layer(2048, 16, 128, 8192, 1000, 8)                     # unsupported shape, no fallback
+    assert layer.status() == (0, 0)
+
+
+# ------------------------------------------------------------------------------------------ stage chain
+def run_chain_gpu(pw, w, L, M, dispatch, schedule, recompute, seed=0):
+    stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
+    params = [[p.cuda() for p in inputs.layer_params(w, seed, l, random_ln=True)] for l in range(L)]
+    grads = [[torch.full(p.shape, float("nan"), dtype=torch.float32, device="cuda") for p in ps] for ps in params]
+    mbs = [inputs.microbatch(w, seed, m) for m in range(M)]
+    xs = [x.cuda().view(-1, w.d_model) for x, _ in mbs]
+    dys = [dy.cuda().view(-1, w.d_model) for _, dy in mbs]
+    ys = [torch.empty_like(x) for x in xs]
+    dxs = [torch.empty_like(x) for x in xs]
+    ws = torch.empty(stage.workspace_bytes(M, schedule, recompute), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        reps = 2 if dispatch == pw.DISPATCH_GRAPH else 1           # second call replays the cached graph
+        for _ in range(reps):
+            stage.run_chain(params, grads, xs, dys, ys, dxs, ws, dispatch, schedule, recompute, stream=stream)
+    torch.cuda.synchronize()
+    assert stage.status() == (0, 0)
+    return ys, dxs, grads
+
+
+def test_chain_matches_oracle_and_modes_agree(pw, oracle64):
+    w = inputs.WORKLOADS[1].with_(seq_len=256, batch=1)
+    L, M = 3, 2
+    D = dims_of(w)
+    ref = run_chain_gpu(pw, w, L, M, pw.DISPATCH_ASYNC, pw.SCHEDULE_GPIPE, True)
+    pls = [[np64(p) for p in inputs.layer_params(w, 0, l, random_ln=True)] for l in range(L)]
+    mbs = [inputs.microbatch(w, 0, m) for m in range(M)]
+    bf16_roundtrip = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(torch.bfloat16).double().numpy()
+    ys, dxs, grads = oracle64.chain(D, pls, [np64(x) for x, _ in mbs], [np64(dy) for _, dy in mbs],
+                                    handoff=bf16_roundtrip)
+    for m in range(M):
+        assert rel_l2(ref[0][m], ys[m]) < ACT_TOL
+        assert rel_l2(ref[1][m], dxs[m]) < GRAD_TOL
+    for l in range(L):
+        for name, g, want in zip(pw.PARAM_NAMES, ref[2][l], grads[l]):
+            assert rel_l2(g, want) < GRAD_TOL, (l, name)
+    # every dispatch mode, schedule and save mode gives the same bits (same kernels, same order per tensor)
+    for dispatch, schedule, recompute in [(pw.DISPATCH_OPBYOP, pw.SCHEDULE_GPIPE, True),
+                                          (pw.DISPATCH_GRAPH, pw.SCHEDULE_GPIPE, True),
+                                          (pw.DISPATCH_ASYNC, pw.SCHEDULE_PER_MICROBATCH, True),
+                                          (pw.DISPATCH_ASYNC, pw.SCHEDULE_GPIPE, False),
+                                          (pw.DISPATCH_GRAPH, pw.SCHEDULE_PER_MICROBATCH, False)]:
+        other = run_chain_gpu(pw, w, L, M, dispatch, schedule, recompute)
+        for m in range(M):
+            assert torch.equal(ref[0][m], other[0][m]) and torch.equal(ref[1][m], other[1][m]), (dispatch, schedule, recompute)
+        for l in range(L):
+            for g1, g2 in zip(ref[2][l], other[2][l]):
+                assert torch.equal(g1, g2), (dispatch, schedule, recompute)
+
+
+def test_chain_workspace_too_small_is_reported_before_launch(pw):
+    w = inputs.WORKLOADS[1]
+    stage = pw.Stage(2, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
+    params = [[p.cuda() for p in inputs.layer_params(w, 0, l)] for l in range(2)]
+    grads = [[torch.zeros(p.shape, dtype=torch.float32, device="cuda") for p in ps] for ps in params]
+    x = torch.zeros((w.tokens, w.d_model), dtype=torch.bfloat16, device="cuda")
+    y, dy, dx = torch.empty_like(x), torch.zeros_like(x), torch.empty_like(x)
+    need = stage.workspace_bytes(1)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    with pytest.raises(pw.PwError) as e:
+        stage.run_chain(params, grads, [x], [dy], [y], [dx], ws, workspace_bytes=need - 1)
+    assert e.value.status == 3
+
+
+# ------------------------------------------------------------------------------------------ full benchmark size
+def test_cfg2_full_size_parity(pw, oracle32):
+    """The benchmark workload (d=2048, 16x128 heads, F=8192, S=1024, B=8) against the fp32 oracle."""
+    check_layer_against_oracle(pw, oracle32, inputs.WORKLOADS[2])
