@@ -1,0 +1,358 @@
+#!/usr/bin/env python
+"""Benchmark of the decoder-layer hot path on B200 (one process per GPU; N > 1 = independent replicas).
+
+    python bench.py --gpus 1 --steps 20 --warmup 3
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N --master-addr 127.0.0.1 --master-port P \
+        bench.py --gpus N --steps K --warmup W
+    python bench.py --impl reference ...        # the CPU oracle, timed on the host cores
+
+A "step" is one pass of the whole hot path over one batch of synthetic input: forward and
+backward of every layer of the workload on every micro-batch (workload 2, the default: one
+decoder layer d=2048, 16x128 heads, F=8192, S=1024, B=8).  Rank 0 prints ONE JSON line.
+
+Timing: CUDA events on the launching stream, after warm-up, barrier + synchronize on both
+sides, max over ranks.  Per-kernel-class times (for the roofline object) come from a second,
+instrumented pass of the same K steps in which the library brackets every launch with CUDA
+events; the headline number is from the un-instrumented pass.  The end-to-end number repeats
+the step with host buffers: pinned host -> device copies of x and dy and device -> host reads
+of y and dx inside the timed region.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram bytes read+written per GEMM launch (average over the 12 GEMM launches of a workload-2 step),
+# from the ncu capture summarised in profiles/; None until a capture exists for the workload.
+GEMM_DRAM_TRAFFIC_PER_LAUNCH = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    except Exception:
+        return dict(FALLBACK_PEAKS, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = index
+            if visible:
+                ids = [v for v in visible.split(",") if v.strip()]
+                if index < len(ids) and ids[index].strip().isdigit():
+                    phys = int(ids[index])
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4)}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for n, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def hw_flops_per_step(w) -> float:
+    """Executed FLOPs: model FLOPs plus, with recompute, one forward without the FC2 GEMM."""
+    per_call = w.model_flops_per_layer_call()
+    if w.recompute:
+        per_call += w.fwd_flops_per_layer_call() - 2.0 * w.tokens * w.d_model * w.d_ff
+    return per_call * w.n_layers * w.n_microbatches
+
+
+def oracle_step(oracle, D, params, x, dy):
+    y, sv = oracle.layer_fwd(D, params, x)
+    oracle.layer_bwd(D, params, x, sv, dy)
+
+
+def oracle_sample(w, batch):
+    """Inputs of a bounded sample of workload w (first `batch` sequences, one layer, one micro-batch)."""
+    from oracle import Dims
+    from paper_2203_12533_b200 import inputs
+    ws = w.with_(batch=batch)
+    D = Dims(ws.batch, ws.seq_len, ws.d_model, ws.n_heads, ws.head_dim, ws.d_ff)
+    params = [p.float().numpy() for p in inputs.layer_params(ws, 0, 0)]
+    x, dy = inputs.microbatch(ws, 0, 0)
+    return ws, D, params, x.float().numpy().reshape(ws.tokens, -1), dy.float().numpy().reshape(ws.tokens, -1)
+
+
+def run_reference(args, w):
+    """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle as oracle_mod
+    orc = oracle_mod.Oracle("f32")
+    batch = 1
+    ws, D, params, x, dy = oracle_sample(w, batch)
+    for _ in range(args.warmup):
+        oracle_step(orc, D, params, x, dy)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(orc, D, params, x, dy)
+    dt = time.perf_counter() - t0
+    value = ws.tokens * args.steps / dt
+    cores = oracle_mod.host_threads()
+    sample = (f"{batch} of {w.batch} sequences (S={w.seq_len}), one layer fwd+bwd per step, fp32 plain-loop C oracle")
+    line = {
+        "impl": "reference", "metric": "decoder-layer fwd+bwd tokens/s", "value": value, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "sample": sample},
+        "tflops_model": ws.model_flops_per_layer_call() * args.steps / dt / 1e12,
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2203_12533_b200 import binding as pw
+    from paper_2203_12533_b200 import inputs
+
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the product path)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    pw.lib()
+    peaks = load_peaks()
+    dev = torch.device("cuda", local)
+    L, M, T, d = w.n_layers, w.n_microbatches, w.tokens, w.d_model
+    dispatch = {"opbyop": pw.DISPATCH_OPBYOP, "async": pw.DISPATCH_ASYNC, "graph": pw.DISPATCH_GRAPH}[args.dispatch]
+    schedule = pw.SCHEDULE_GPIPE
+
+    stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
+    params = [[p.to(dev) for p in inputs.layer_params(w, args.seed, l)] for l in range(L)]
+    grads = [[torch.zeros(p.shape, dtype=torch.float32, device=dev) for p in ps] for ps in params]
+    host_x, host_dy = [], []
+    for m in range(M):
+        x, dy = inputs.microbatch(w, args.seed, m)
+        host_x.append(x.view(T, d).pin_memory())
+        host_dy.append(dy.view(T, d).pin_memory())
+    xs = [t.to(dev) for t in host_x]
+    dys = [t.to(dev) for t in host_dy]
+    ys = [torch.empty_like(t) for t in xs]
+    dxs = [torch.empty_like(t) for t in xs]
+    host_y = [torch.empty((T, d), dtype=torch.bfloat16).pin_memory() for _ in range(M)]
+    host_dx = [torch.empty((T, d), dtype=torch.bfloat16).pin_memory() for _ in range(M)]
+    ws_bytes = stage.workspace_bytes(M, schedule, w.recompute)
+    workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+
+    def step():
+        stage.run_chain(params, grads, xs, dys, ys, dxs, workspace, dispatch, schedule, w.recompute, stream=stream)
+
+    def step_e2e():
+        for m in range(M):
+            xs[m].copy_(host_x[m], non_blocking=True)
+            dys[m].copy_(host_dy[m], non_blocking=True)
+        step()
+        for m in range(M):
+            host_y[m].copy_(ys[m], non_blocking=True)
+            host_dx[m].copy_(dxs[m], non_blocking=True)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def timed(fn, steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for _ in range(steps):
+                fn()
+            e1.record(stream)
+        torch.cuda.synchronize(dev)
+        ms = e0.elapsed_time(e1)
+        barrier()
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            step()
+    torch.cuda.synchronize(dev)
+    code, site = stage.status()
+    if code != 0:
+        raise SystemExit(f"device status {code} at site {site} after warm-up")
+
+    n0 = stage.launch_count()
+    with ClockSampler(local) as clocks:
+        ms_total = timed(step, args.steps)
+    launches = stage.launch_count() - n0
+    ms_step = ms_total / args.steps
+    tokens_step = T * M
+    value = world * tokens_step / (ms_step * 1e-3)
+
+    # instrumented pass: per-kernel-class device time from CUDA events inside the library
+    prof = None
+    if dispatch != pw.DISPATCH_GRAPH:
+        stage.profile_begin()
+        with torch.cuda.stream(stream):
+            for _ in range(args.steps):
+                step()
+        prof = stage.profile_end()
+
+    # end to end through the public API with host buffers
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    with torch.cuda.stream(stream):
+        step_e2e()
+    ms_e2e = timed(step_e2e, e2e_steps) / e2e_steps
+    e2e_value = world * tokens_step / (ms_e2e * 1e-3)
+    code, site = stage.status()
+    if code != 0:
+        raise SystemExit(f"device status {code} at site {site}")
+
+    model_flops = w.model_flops_per_layer_call() * L * M
+    hw_flops = hw_flops_per_step(w)
+    line = {
+        "metric": "decoder-layer fwd+bwd tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "d_model": w.d_model, "heads": f"{w.n_heads}x{w.head_dim}", "d_ff": w.d_ff,
+                   "seq_len": w.seq_len, "microbatch": w.batch, "layers": L, "microbatches": M,
+                   "recompute": bool(w.recompute), "dispatch": args.dispatch, "parallelism": f"replicas x{world}",
+                   "l2": "working set per step (activations + weights + fp32 grads) is > 1 GB, far above the 126 MB L2"},
+        "tflops_model": world * model_flops / (ms_step * 1e-3) / 1e12,
+        "tflops_hw": world * hw_flops / (ms_step * 1e-3) / 1e12,
+        "frac_bf16_peak_burst": hw_flops / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
+        "frac_bf16_peak_sustained": hw_flops / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+        "peaks": peaks,
+        "clocks": clocks.summary(),
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "ms_per_step": ms_e2e, "steps": e2e_steps,
+                "h2d_bytes_per_step": 2 * M * T * d * 2, "d2h_bytes_per_step": 2 * M * T * d * 2},
+        "gpu_launches": int(launches),
+    }
+    if prof is not None:
+        kernels = {}
+        tot_ms = sum(v["ms"] for v in prof.values())
+        for name, v in prof.items():
+            if v["launches"] == 0:
+                continue
+            k = {"launches_per_step": v["launches"] / args.steps, "ms_per_step": v["ms"] / args.steps,
+                 "share": v["ms"] / tot_ms if tot_ms > 0 else None}
+            if v["flops"] > 0:
+                k["tflops"] = v["flops"] / (v["ms"] * 1e-3) / 1e12
+                k["frac_of_measured_bf16_burst"] = k["tflops"] / peaks["bf16_tflops"]
+            if v["bytes"] > 0:
+                k["gbs"] = v["bytes"] / (v["ms"] * 1e-3) / 1e9
+                k["frac_of_measured_hbm"] = k["gbs"] / peaks["hbm_gbs"]
+            kernels[name] = k
+        line["kernels"] = kernels
+        line["ms_per_step_instrumented"] = tot_ms / args.steps
+        g = [prof[n] for n in ("gemm_tn", "gemm_nn", "gemm_nt")]
+        g_flops, g_ms, g_n = sum(v["flops"] for v in g), sum(v["ms"] for v in g), sum(v["launches"] for v in g)
+        achieved = g_flops / (g_ms * 1e-3) / 1e12
+        line["roofline"] = {
+            "kernel": "gemm_kernel (tcgen05 bf16 GEMM: forward, dgrad and wgrad instantiations)",
+            "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+            "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst cuBLAS bf16)",
+            "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
+            "flops_per_launch": g_flops / g_n, "ms_per_launch": g_ms / g_n, "launches_per_step": g_n / args.steps,
+            "share_of_step": g_ms / tot_ms,
+            "traffic": GEMM_DRAM_TRAFFIC_PER_LAUNCH.get(w.name),
+        }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle as oracle_mod
+        orc = oracle_mod.Oracle("f32")
+        b = min(w.batch, args.cpu_sample_batch)
+        wsamp, D, ps, x, dy = oracle_sample(w, b)
+        t0 = time.perf_counter()
+        oracle_step(orc, D, ps, x, dy)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {
+            "value": wsamp.tokens / dt, "unit": "tokens/s", "cores": oracle_mod.host_threads(), "kind": "oracle",
+            "seconds": dt,
+            "sample": f"{b} of {w.batch} sequences (S={w.seq_len}) through one layer fwd+bwd, fp32 plain-loop C oracle, run once"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4])
+    ap.add_argument("--dispatch", default="async", choices=["opbyop", "async", "graph"])
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--cpu-sample-batch", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    from paper_2203_12533_b200 import inputs
+    w = inputs.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

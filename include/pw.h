@@ -164,6 +164,32 @@ pw_status_t pw_layer_bwd(pw_layer_t* layer, const pw_layer_params_t* params, con
  * code a kernel recorded (PW_ERR_TIMEOUT) with *site (may be NULL) = where it gave up. */
 pw_status_t pw_layer_status(pw_layer_t* layer, int* device_status, int* site);
 
+/* Per-kernel timing for benchmarks.  Between profile_begin and profile_end every kernel this
+ * handle launches is bracketed by CUDA events on the launching stream; profile_end synchronises
+ * that stream and sums the elapsed times by kernel class.  Not usable inside a captured graph
+ * (PW_DISPATCH_GRAPH returns PW_ERR_INVALID_ARG while profiling is on).  Host structs. */
+enum {
+    PW_K_GEMM_TN = 0,   /* forward GEMMs                      */
+    PW_K_GEMM_NN = 1,   /* data-gradient GEMMs                */
+    PW_K_GEMM_NT = 2,   /* weight-gradient GEMMs              */
+    PW_K_ATTN_FWD = 3,
+    PW_K_ATTN_BWD = 4,  /* delta + dq + dkdv kernels          */
+    PW_K_LN_FWD = 5,
+    PW_K_LN_BWD = 6,    /* main kernel + partial reduction    */
+    PW_K_COLSUM = 7,    /* main kernel + partial reduction    */
+    PW_K_COUNT = 8
+};
+typedef struct pw_profile {
+    uint64_t launches[PW_K_COUNT]; /* kernel launches per class since profile_begin      */
+    double ms[PW_K_COUNT];         /* summed device time per class, milliseconds         */
+    double flops[PW_K_COUNT];      /* executed tensor-core FLOPs (GEMM / attention classes; causal half only) */
+    double bytes[PW_K_COUNT];      /* algorithmic HBM bytes (LN / column-sum classes)    */
+} pw_profile_t;
+pw_status_t pw_layer_profile_begin(pw_layer_t* layer);
+pw_status_t pw_layer_profile_end(pw_layer_t* layer, pw_profile_t* out);
+/* Kernels launched through this handle since it was created (graph replays count their nodes). */
+pw_status_t pw_layer_launch_count(const pw_layer_t* layer, uint64_t* count);
+
 /* ---- a pipeline stage: L layers x M micro-batches (Section 5.3, Table 2; dispatch modes of Section 5.1) ---- */
 
 enum {
@@ -202,6 +228,9 @@ pw_status_t pw_stage_run_chain(pw_stage_t* stage, const pw_layer_params_t* param
                                int recompute, void* workspace, size_t workspace_bytes, void* stream);
 
 pw_status_t pw_stage_status(pw_stage_t* stage, int* device_status, int* site);
+pw_status_t pw_stage_profile_begin(pw_stage_t* stage);
+pw_status_t pw_stage_profile_end(pw_stage_t* stage, pw_profile_t* out);
+pw_status_t pw_stage_launch_count(const pw_stage_t* stage, uint64_t* count);
 
 /* ---- single steps of the layer (same kernels the layer calls; for unit tests and profiling) ---- */
 

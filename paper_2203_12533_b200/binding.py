@@ -32,7 +32,9 @@ EXPORTS = (
     "pw_version", "pw_status_string", "pw_last_error",
     "pw_layer_create", "pw_layer_destroy", "pw_layer_workspace_bytes", "pw_layer_ctx_offset",
     "pw_layer_fwd", "pw_layer_bwd", "pw_layer_status",
+    "pw_layer_profile_begin", "pw_layer_profile_end", "pw_layer_launch_count",
     "pw_stage_create", "pw_stage_destroy", "pw_stage_workspace_bytes", "pw_stage_run_chain", "pw_stage_status",
+    "pw_stage_profile_begin", "pw_stage_profile_end", "pw_stage_launch_count",
     "pw_op_layernorm_fwd", "pw_op_layernorm_bwd_scratch_bytes", "pw_op_layernorm_bwd",
     "pw_op_colsum_scratch_bytes", "pw_op_colsum", "pw_op_gemm",
     "pw_op_attention_fwd", "pw_op_attention_bwd", "pw_op_status",
@@ -50,6 +52,18 @@ class LayerConfig(ctypes.Structure):
                 ("head_dim", ctypes.c_int32), ("d_ff", ctypes.c_int32), ("seq_len", ctypes.c_int32),
                 ("batch", ctypes.c_int32), ("act", ctypes.c_int32), ("ln_eps", ctypes.c_float),
                 ("causal", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+KERNEL_CLASSES = ("gemm_tn", "gemm_nn", "gemm_nt", "attn_fwd", "attn_bwd", "ln_fwd", "ln_bwd", "colsum")
+
+
+class Profile(ctypes.Structure):
+    _fields_ = [("launches", ctypes.c_uint64 * 8), ("ms", ctypes.c_double * 8), ("flops", ctypes.c_double * 8),
+                ("bytes", ctypes.c_double * 8)]
+
+    def as_dict(self):
+        return {n: dict(launches=int(self.launches[i]), ms=float(self.ms[i]), flops=float(self.flops[i]),
+                        bytes=float(self.bytes[i])) for i, n in enumerate(KERNEL_CLASSES)}
 
 
 class _Ptr12(ctypes.Structure):
@@ -85,6 +99,12 @@ def lib() -> ctypes.CDLL:
         L.pw_layer_fwd.argtypes = [vp, ctypes.POINTER(_Ptr12), vp, vp, vp, vp, vp]
         L.pw_layer_bwd.argtypes = [vp, ctypes.POINTER(_Ptr12), vp, vp, vp, ctypes.POINTER(_Ptr12), ci, vp, vp, vp]
         L.pw_layer_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
+        L.pw_layer_profile_begin.argtypes = [vp]
+        L.pw_layer_profile_end.argtypes = [vp, ctypes.POINTER(Profile)]
+        L.pw_layer_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
+        L.pw_stage_profile_begin.argtypes = [vp]
+        L.pw_stage_profile_end.argtypes = [vp, ctypes.POINTER(Profile)]
+        L.pw_stage_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
         L.pw_stage_create.argtypes = [ctypes.POINTER(LayerConfig), ci, ctypes.POINTER(vp)]
         L.pw_stage_destroy.argtypes = [vp]
         L.pw_stage_destroy.restype = None
@@ -192,6 +212,19 @@ class Layer:
         _check(lib().pw_layer_status(self._h, ctypes.byref(c), ctypes.byref(s)))
         return c.value, s.value
 
+    def profile_begin(self):
+        _check(lib().pw_layer_profile_begin(self._h))
+
+    def profile_end(self) -> dict:
+        p = Profile()
+        _check(lib().pw_layer_profile_end(self._h, ctypes.byref(p)))
+        return p.as_dict()
+
+    def launch_count(self) -> int:
+        n = ctypes.c_uint64()
+        _check(lib().pw_layer_launch_count(self._h, ctypes.byref(n)))
+        return n.value
+
 
 class Stage:
     """A stack of identical-shape layers run over M micro-batches (pw_stage_*)."""
@@ -233,6 +266,19 @@ class Stage:
         c, s = ctypes.c_int(), ctypes.c_int()
         _check(lib().pw_stage_status(self._h, ctypes.byref(c), ctypes.byref(s)))
         return c.value, s.value
+
+    def profile_begin(self):
+        _check(lib().pw_stage_profile_begin(self._h))
+
+    def profile_end(self) -> dict:
+        p = Profile()
+        _check(lib().pw_stage_profile_end(self._h, ctypes.byref(p)))
+        return p.as_dict()
+
+    def launch_count(self) -> int:
+        n = ctypes.c_uint64()
+        _check(lib().pw_stage_launch_count(self._h, ctypes.byref(n)))
+        return n.value
 
 
 # ---- single steps ----

@@ -78,12 +78,23 @@ struct pw_layer {
     pw::LayerPlan plan;
     pw::Runtime* rt;
     pw::DeviceStatus* status;
+    uint64_t launches = 0;          // kernels launched (or replayed) through this handle
+    bool capturing = false;         // inside a stream capture: count launches into graph_nodes instead
+    uint64_t graph_nodes = 0;
+    // profiling: event pairs around every launch group
+    bool profiling = false;
+    struct Span { cudaEvent_t a, b; int cls; };
+    std::vector<Span> spans;
+    std::vector<cudaEvent_t> pool;
+    cudaStream_t prof_stream = nullptr;
+    pw_profile_t prof;
 };
 
 struct pw_stage {
     pw_layer_t* layer;
     int n_layers;
-    std::map<std::vector<uint64_t>, cudaGraphExec_t> graphs;
+    struct Cached { cudaGraphExec_t exec; uint64_t nodes; };
+    std::map<std::vector<uint64_t>, Cached> graphs;
 };
 
 namespace pw {
@@ -133,11 +144,32 @@ static void build_plan(const pw_layer_config_t& c, Runtime* rt, LayerPlan* p)
     p->scratch_bytes = s;
 }
 
-#define PW_TRY(expr)                                                        \
-    do {                                                                    \
-        const char* e__ = (expr);                                           \
-        if (e__) return fail(PW_ERR_CUDA, std::string(#expr) + ": " + e__); \
-    } while (0)
+// Runs one launch group, counting its kernels and (when profiling) bracketing it with events.
+struct LaunchScope {
+    pw_layer_t* L; int cls; cudaStream_t st; cudaEvent_t a = nullptr, b = nullptr;
+    static cudaEvent_t get_event(pw_layer_t* L)
+    {
+        if (!L->pool.empty()) { cudaEvent_t e = L->pool.back(); L->pool.pop_back(); return e; }
+        cudaEvent_t e = nullptr;
+        cudaEventCreate(&e);
+        return e;
+    }
+    LaunchScope(pw_layer_t* L_, int cls_, int nkernels, double flops, double bytes, cudaStream_t st_)
+        : L(L_), cls(cls_), st(st_)
+    {
+        if (L->capturing) L->graph_nodes += nkernels; else L->launches += nkernels;
+        if (L->profiling) {
+            L->prof.launches[cls] += nkernels; L->prof.flops[cls] += flops; L->prof.bytes[cls] += bytes;
+            L->prof_stream = st;
+            a = get_event(L); b = get_event(L);
+            if (a) cudaEventRecord(a, st);
+        }
+    }
+    ~LaunchScope()
+    {
+        if (L->profiling && a && b) { cudaEventRecord(b, st); L->spans.push_back({a, b, cls}); }
+    }
+};
 
 static inline uint8_t* at(void* base, size_t off) { return static_cast<uint8_t*>(base) + off; }
 static inline const uint8_t* at(const void* base, size_t off) { return static_cast<const uint8_t*>(base) + off; }
@@ -153,13 +185,68 @@ static GemmArgs gemm_args(int layout, int epi, int act, int M, int N, int K, con
     return g;
 }
 
+#define PW_DO(expr)                          \
+    do {                                     \
+        pw_status_t s__ = (expr);            \
+        if (s__ != PW_OK) return s__;        \
+    } while (0)
+
+static pw_status_t do_gemm(pw_layer_t* L, const GemmArgs& g, cudaStream_t st)
+{
+    const int cls = g.layout == kTN ? PW_K_GEMM_TN : g.layout == kNN ? PW_K_GEMM_NN : PW_K_GEMM_NT;
+    LaunchScope sc(L, cls, 1, 2.0 * g.M * g.N * g.K, 0.0, st);
+    const char* e = launch_gemm(L->rt, g, L->status, st);
+    return e ? fail(PW_ERR_CUDA, e) : PW_OK;
+}
+static pw_status_t do_ln_fwd(pw_layer_t* L, const void* x, const void* gamma, const void* beta, void* h, void* mu,
+                             void* rstd, cudaStream_t st)
+{
+    const LayerPlan& p = L->plan;
+    LaunchScope sc(L, PW_K_LN_FWD, 1, 0.0, 4.0 * p.T * p.d + 8.0 * p.T, st);
+    const char* e = launch_layernorm_fwd(L->rt, x, gamma, beta, p.T, p.d, p.eps, h, mu, rstd, st);
+    return e ? fail(PW_ERR_CUDA, e) : PW_OK;
+}
+static pw_status_t do_ln_bwd(pw_layer_t* L, const void* dh, const void* x, const void* mu, const void* rstd,
+                             const void* gamma, const void* resid, void* dx, void* dgamma, void* dbeta, void* db_resid,
+                             void* db_dx, int accumulate, void* partials, cudaStream_t st)
+{
+    const LayerPlan& p = L->plan;
+    LaunchScope sc(L, PW_K_LN_BWD, 2, 0.0, 8.0 * p.T * p.d + 8.0 * p.T, st);
+    const char* e = launch_layernorm_bwd(L->rt, dh, x, mu, rstd, gamma, resid, p.T, p.d, dx, dgamma, dbeta, db_resid,
+                                         db_dx, accumulate, partials, st);
+    return e ? fail(PW_ERR_CUDA, e) : PW_OK;
+}
+static pw_status_t do_colsum(pw_layer_t* L, const void* in, int N, void* out, int accumulate, void* partials,
+                             cudaStream_t st)
+{
+    const LayerPlan& p = L->plan;
+    LaunchScope sc(L, PW_K_COLSUM, 2, 0.0, 2.0 * p.T * N, st);
+    const char* e = launch_colsum(L->rt, in, p.T, N, N, out, accumulate, partials, st);
+    return e ? fail(PW_ERR_CUDA, e) : PW_OK;
+}
+// Attention FLOPs count the visible (causal) pairs only: 2 T (S+1) d forward, 2.5x that backward.
+static pw_status_t do_attn_fwd(pw_layer_t* L, const void* qkv, void* o, void* lse, cudaStream_t st)
+{
+    const LayerPlan& p = L->plan;
+    LaunchScope sc(L, PW_K_ATTN_FWD, 1, 2.0 * p.T * (p.S + 1.0) * p.d, 0.0, st);
+    const char* e = launch_attention_fwd(L->rt, qkv, p.B, p.S, p.H, p.dh, o, lse, st);
+    return e ? fail(PW_ERR_CUDA, e) : PW_OK;
+}
+static pw_status_t do_attn_bwd(pw_layer_t* L, const void* qkv, const void* o, const void* dout, const void* lse,
+                               void* dqkv, void* delta, cudaStream_t st)
+{
+    const LayerPlan& p = L->plan;
+    LaunchScope sc(L, PW_K_ATTN_BWD, 3, 5.0 * p.T * (p.S + 1.0) * p.d, 0.0, st);
+    const char* e = launch_attention_bwd(L->rt, qkv, o, dout, lse, p.B, p.S, p.H, p.dh, dqkv, delta, st);
+    return e ? fail(PW_ERR_CUDA, e) : PW_OK;
+}
+
 // Forward into `ctx` (a ctx-shaped region).  with_fc2 = false stops after FC1/GeLU (all that a
 // recomputing backward needs).
 static pw_status_t enqueue_fwd(pw_layer_t* L, const pw_layer_params_t* P, const void* x, void* y, void* ctx,
                                bool with_fc2, cudaStream_t st)
 {
     const LayerPlan& p = L->plan;
-    Runtime* rt = L->rt;
     const int T = p.T, d = p.d, F = p.F, act = p.cfg.act;
     void* h1 = at(ctx, p.ctx_off[PW_CTX_H1]);   void* qkv = at(ctx, p.ctx_off[PW_CTX_QKV]);
     void* o = at(ctx, p.ctx_off[PW_CTX_O]);     void* x1 = at(ctx, p.ctx_off[PW_CTX_X1]);
@@ -168,18 +255,18 @@ static pw_status_t enqueue_fwd(pw_layer_t* L, const pw_layer_params_t* P, const 
     void* mu1 = at(ctx, p.ctx_off[PW_CTX_MU1]); void* r1 = at(ctx, p.ctx_off[PW_CTX_R1]);
     void* mu2 = at(ctx, p.ctx_off[PW_CTX_MU2]); void* r2 = at(ctx, p.ctx_off[PW_CTX_R2]);
 
-    PW_TRY(launch_layernorm_fwd(rt, x, P->ln1_gamma, P->ln1_beta, T, d, p.eps, h1, mu1, r1, st));
-    PW_TRY(launch_gemm(rt, gemm_args(kTN, kEpiBias, act, T, 3 * d, d, h1, d, P->w_qkv, d, qkv, 3 * d, P->b_qkv,
-                                     nullptr, 0, nullptr, 0), L->status, st));
-    PW_TRY(launch_attention_fwd(rt, qkv, p.B, p.S, p.H, p.dh, o, lse, st));
-    PW_TRY(launch_gemm(rt, gemm_args(kTN, kEpiBiasResid, act, T, d, d, o, d, P->w_o, d, x1, d, P->b_o, x, d,
-                                     nullptr, 0), L->status, st));
-    PW_TRY(launch_layernorm_fwd(rt, x1, P->ln2_gamma, P->ln2_beta, T, d, p.eps, h2, mu2, r2, st));
-    PW_TRY(launch_gemm(rt, gemm_args(kTN, kEpiBiasGelu, act, T, F, d, h2, d, P->w_fc1, d, u, F, P->b_fc1, nullptr, 0,
-                                     a, 0), L->status, st));
+    PW_DO(do_ln_fwd(L, x, P->ln1_gamma, P->ln1_beta, h1, mu1, r1, st));
+    PW_DO(do_gemm(L, gemm_args(kTN, kEpiBias, act, T, 3 * d, d, h1, d, P->w_qkv, d, qkv, 3 * d, P->b_qkv,
+                                     nullptr, 0, nullptr, 0), st));
+    PW_DO(do_attn_fwd(L, qkv, o, lse, st));
+    PW_DO(do_gemm(L, gemm_args(kTN, kEpiBiasResid, act, T, d, d, o, d, P->w_o, d, x1, d, P->b_o, x, d,
+                                     nullptr, 0), st));
+    PW_DO(do_ln_fwd(L, x1, P->ln2_gamma, P->ln2_beta, h2, mu2, r2, st));
+    PW_DO(do_gemm(L, gemm_args(kTN, kEpiBiasGelu, act, T, F, d, h2, d, P->w_fc1, d, u, F, P->b_fc1, nullptr, 0,
+                                     a, 0), st));
     if (with_fc2)
-        PW_TRY(launch_gemm(rt, gemm_args(kTN, kEpiBiasResid, act, T, d, F, a, F, P->w_fc2, F, y, d, P->b_fc2, x1, d,
-                                         nullptr, 0), L->status, st));
+        PW_DO(do_gemm(L, gemm_args(kTN, kEpiBiasResid, act, T, d, F, a, F, P->w_fc2, F, y, d, P->b_fc2, x1, d,
+                                         nullptr, 0), st));
     return PW_OK;
 }
 
@@ -188,7 +275,6 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
                                cudaStream_t st)
 {
     const LayerPlan& p = L->plan;
-    Runtime* rt = L->rt;
     const int T = p.T, d = p.d, F = p.F, act = p.cfg.act;
     if (ctx == nullptr) {
         pw_status_t s = enqueue_fwd(L, P, x, nullptr, scratch, false, st);
@@ -208,34 +294,34 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
     void* part = at(scratch, p.off_partials);
 
     // y = x1 + a W2^T + b2  ->  du = (dy W2) * gelu'(u),  dW2 = dy^T a
-    PW_TRY(launch_gemm(rt, gemm_args(kNN, kEpiDGelu, act, T, F, d, dy, d, P->w_fc2, F, big, F, nullptr, u, F,
-                                     nullptr, 0), L->status, st));
-    PW_TRY(launch_gemm(rt, gemm_args(kNT, kEpiF32, act, d, F, T, dy, d, a, F, G->w_fc2, F, nullptr, nullptr, 0,
-                                     nullptr, accumulate), L->status, st));
+    PW_DO(do_gemm(L, gemm_args(kNN, kEpiDGelu, act, T, F, d, dy, d, P->w_fc2, F, big, F, nullptr, u, F,
+                                     nullptr, 0), st));
+    PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, d, F, T, dy, d, a, F, G->w_fc2, F, nullptr, nullptr, 0,
+                                     nullptr, accumulate), st));
     // u = h2 W1^T + b1  ->  dh2 = du W1,  dW1 = du^T h2,  db1 = colsum(du)
-    PW_TRY(launch_gemm(rt, gemm_args(kNN, kEpiNone, act, T, d, F, big, F, P->w_fc1, d, td0, d, nullptr, nullptr, 0,
-                                     nullptr, 0), L->status, st));
-    PW_TRY(launch_gemm(rt, gemm_args(kNT, kEpiF32, act, F, d, T, big, F, h2, d, G->w_fc1, d, nullptr, nullptr, 0,
-                                     nullptr, accumulate), L->status, st));
-    PW_TRY(launch_colsum(rt, big, T, F, F, G->b_fc1, accumulate, part, st));
+    PW_DO(do_gemm(L, gemm_args(kNN, kEpiNone, act, T, d, F, big, F, P->w_fc1, d, td0, d, nullptr, nullptr, 0,
+                                     nullptr, 0), st));
+    PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, F, d, T, big, F, h2, d, G->w_fc1, d, nullptr, nullptr, 0,
+                                     nullptr, accumulate), st));
+    PW_DO(do_colsum(L, big, F, G->b_fc1, accumulate, part, st));
     // LN2 backward + residual: dx1 = dy + LNbwd(dh2); also db2 = colsum(dy), dbo = colsum(dx1)
-    PW_TRY(launch_layernorm_bwd(rt, td0, x1, mu2, r2, P->ln2_gamma, dy, T, d, dx1, G->ln2_gamma, G->ln2_beta,
+    PW_DO(do_ln_bwd(L, td0, x1, mu2, r2, P->ln2_gamma, dy, dx1, G->ln2_gamma, G->ln2_beta,
                                 G->b_fc2, G->b_o, accumulate, part, st));
     // x1 = x + o Wo^T + bo  ->  dout = dx1 Wo,  dWo = dx1^T o
-    PW_TRY(launch_gemm(rt, gemm_args(kNN, kEpiNone, act, T, d, d, dx1, d, P->w_o, d, td0, d, nullptr, nullptr, 0,
-                                     nullptr, 0), L->status, st));
-    PW_TRY(launch_gemm(rt, gemm_args(kNT, kEpiF32, act, d, d, T, dx1, d, o, d, G->w_o, d, nullptr, nullptr, 0,
-                                     nullptr, accumulate), L->status, st));
+    PW_DO(do_gemm(L, gemm_args(kNN, kEpiNone, act, T, d, d, dx1, d, P->w_o, d, td0, d, nullptr, nullptr, 0,
+                                     nullptr, 0), st));
+    PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, d, d, T, dx1, d, o, d, G->w_o, d, nullptr, nullptr, 0,
+                                     nullptr, accumulate), st));
     // attention backward -> dqkv
-    PW_TRY(launch_attention_bwd(rt, qkv, o, td0, lse, p.B, p.S, p.H, p.dh, big, delta, st));
+    PW_DO(do_attn_bwd(L, qkv, o, td0, lse, big, delta, st));
     // qkv = h1 Wqkv^T + bqkv  ->  dh1 = dqkv Wqkv,  dWqkv = dqkv^T h1,  dbqkv = colsum(dqkv)
-    PW_TRY(launch_gemm(rt, gemm_args(kNN, kEpiNone, act, T, d, 3 * d, big, 3 * d, P->w_qkv, d, td0, d, nullptr,
-                                     nullptr, 0, nullptr, 0), L->status, st));
-    PW_TRY(launch_gemm(rt, gemm_args(kNT, kEpiF32, act, 3 * d, d, T, big, 3 * d, h1, d, G->w_qkv, d, nullptr, nullptr,
-                                     0, nullptr, accumulate), L->status, st));
-    PW_TRY(launch_colsum(rt, big, T, 3 * d, 3 * d, G->b_qkv, accumulate, part, st));
+    PW_DO(do_gemm(L, gemm_args(kNN, kEpiNone, act, T, d, 3 * d, big, 3 * d, P->w_qkv, d, td0, d, nullptr,
+                                     nullptr, 0, nullptr, 0), st));
+    PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, 3 * d, d, T, big, 3 * d, h1, d, G->w_qkv, d, nullptr, nullptr,
+                                     0, nullptr, accumulate), st));
+    PW_DO(do_colsum(L, big, 3 * d, G->b_qkv, accumulate, part, st));
     // LN1 backward + residual: dx = dx1 + LNbwd(dh1)
-    PW_TRY(launch_layernorm_bwd(rt, td0, x, mu1, r1, P->ln1_gamma, dx1, T, d, dx, G->ln1_gamma, G->ln1_beta, nullptr,
+    PW_DO(do_ln_bwd(L, td0, x, mu1, r1, P->ln1_gamma, dx1, dx, G->ln1_gamma, G->ln1_beta, nullptr,
                                 nullptr, accumulate, part, st));
     return PW_OK;
 }
@@ -315,6 +401,8 @@ pw_status_t pw_layer_create(const pw_layer_config_t* cfg, pw_layer_t** out)
 void pw_layer_destroy(pw_layer_t* layer)
 {
     if (!layer) return;
+    for (auto& sp : layer->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
+    for (auto e : layer->pool) cudaEventDestroy(e);
     if (layer->status) cudaFree(layer->status);
     delete layer;
 }
@@ -367,6 +455,40 @@ pw_status_t pw_layer_status(pw_layer_t* layer, int* device_status, int* site)
     return read_status(layer->status, device_status, site);
 }
 
+pw_status_t pw_layer_profile_begin(pw_layer_t* layer)
+{
+    if (!layer) return fail(PW_ERR_INVALID_ARG, "layer is NULL");
+    for (auto& sp : layer->spans) { layer->pool.push_back(sp.a); layer->pool.push_back(sp.b); }
+    layer->spans.clear();
+    std::memset(&layer->prof, 0, sizeof(layer->prof));
+    layer->profiling = true;
+    return PW_OK;
+}
+
+pw_status_t pw_layer_profile_end(pw_layer_t* layer, pw_profile_t* out)
+{
+    if (!layer || !out) return fail(PW_ERR_INVALID_ARG, "layer or out is NULL");
+    if (!layer->profiling) return fail(PW_ERR_INVALID_ARG, "profile_end without profile_begin");
+    layer->profiling = false;
+    cudaError_t e = cudaStreamSynchronize(layer->prof_stream);
+    if (e != cudaSuccess) return fail_cuda("cudaStreamSynchronize", e);
+    for (auto& sp : layer->spans) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, sp.a, sp.b) == cudaSuccess) layer->prof.ms[sp.cls] += ms;
+        layer->pool.push_back(sp.a); layer->pool.push_back(sp.b);
+    }
+    layer->spans.clear();
+    *out = layer->prof;
+    return PW_OK;
+}
+
+pw_status_t pw_layer_launch_count(const pw_layer_t* layer, uint64_t* count)
+{
+    if (!layer || !count) return fail(PW_ERR_INVALID_ARG, "layer or count is NULL");
+    *count = layer->launches;
+    return PW_OK;
+}
+
 // ---------------------------------------------------------------------------------------- stage
 
 pw_status_t pw_stage_create(const pw_layer_config_t* cfg, int n_layers, pw_stage_t** out)
@@ -387,7 +509,7 @@ pw_status_t pw_stage_create(const pw_layer_config_t* cfg, int n_layers, pw_stage
 void pw_stage_destroy(pw_stage_t* stage)
 {
     if (!stage) return;
-    for (auto& kv : stage->graphs) cudaGraphExecDestroy(kv.second);
+    for (auto& kv : stage->graphs) cudaGraphExecDestroy(kv.second.exec);
     pw_layer_destroy(stage->layer);
     delete stage;
 }
@@ -534,12 +656,16 @@ pw_status_t pw_stage_run_chain(pw_stage_t* stage, const pw_layer_params_t* param
         key.push_back(reinterpret_cast<uint64_t>(x_mb[m])); key.push_back(reinterpret_cast<uint64_t>(dy_mb[m]));
         key.push_back(reinterpret_cast<uint64_t>(y_mb[m])); key.push_back(reinterpret_cast<uint64_t>(dx_mb[m]));
     }
+    if (stage->layer->profiling) return fail(PW_ERR_INVALID_ARG, "per-kernel profiling is not available in GRAPH mode");
     auto it = stage->graphs.find(key);
     if (it == stage->graphs.end()) {
         if (st == nullptr) return fail(PW_ERR_INVALID_ARG, "GRAPH mode needs a non-default stream (the legacy stream cannot be captured)");
         cudaError_t e = cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal);
         if (e != cudaSuccess) return fail_cuda("cudaStreamBeginCapture", e);
+        stage->layer->capturing = true;
+        stage->layer->graph_nodes = 0;
         s = enqueue_chain(stage, params, grads, x_mb, dy_mb, y_mb, dx_mb, M, schedule, recompute, workspace, lay, false, st);
+        stage->layer->capturing = false;
         cudaGraph_t graph = nullptr;
         e = cudaStreamEndCapture(st, &graph);
         if (s != PW_OK) { if (graph) cudaGraphDestroy(graph); return s; }
@@ -549,19 +675,36 @@ pw_status_t pw_stage_run_chain(pw_stage_t* stage, const pw_layer_params_t* param
         cudaGraphDestroy(graph);
         if (e != cudaSuccess) return fail_cuda("cudaGraphInstantiate", e);
         if (stage->graphs.size() >= 16) {   // bounded cache
-            for (auto& kv : stage->graphs) cudaGraphExecDestroy(kv.second);
+            for (auto& kv : stage->graphs) cudaGraphExecDestroy(kv.second.exec);
             stage->graphs.clear();
         }
-        it = stage->graphs.emplace(key, exec).first;
+        it = stage->graphs.emplace(key, pw_stage::Cached{exec, stage->layer->graph_nodes}).first;
     }
-    cudaError_t e = cudaGraphLaunch(it->second, st);
-    return e == cudaSuccess ? PW_OK : fail_cuda("cudaGraphLaunch", e);
+    cudaError_t e = cudaGraphLaunch(it->second.exec, st);
+    if (e != cudaSuccess) return fail_cuda("cudaGraphLaunch", e);
+    stage->layer->launches += it->second.nodes;
+    return PW_OK;
 }
 
 pw_status_t pw_stage_status(pw_stage_t* stage, int* device_status, int* site)
 {
     if (!stage) return fail(PW_ERR_INVALID_ARG, "stage is NULL");
     return read_status(stage->layer->status, device_status, site);
+}
+pw_status_t pw_stage_profile_begin(pw_stage_t* stage)
+{
+    if (!stage) return fail(PW_ERR_INVALID_ARG, "stage is NULL");
+    return pw_layer_profile_begin(stage->layer);
+}
+pw_status_t pw_stage_profile_end(pw_stage_t* stage, pw_profile_t* out)
+{
+    if (!stage) return fail(PW_ERR_INVALID_ARG, "stage is NULL");
+    return pw_layer_profile_end(stage->layer, out);
+}
+pw_status_t pw_stage_launch_count(const pw_stage_t* stage, uint64_t* count)
+{
+    if (!stage) return fail(PW_ERR_INVALID_ARG, "stage is NULL");
+    return pw_layer_launch_count(stage->layer, count);
 }
 
 // ---------------------------------------------------------------------------------------- single steps
