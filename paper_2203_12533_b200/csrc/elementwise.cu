@@ -50,39 +50,57 @@ __device__ __forceinline__ float row_sum(float v, float* slot, int warps_per_row
     return t;
 }
 
-template <int CHUNKS>
+// LayerNorm forward.  A row is handled by W warps (W = 1 for d <= 2048), each lane holding CH
+// 16-byte pieces (lane i of warp w owns columns 8*(i + 32*(w + W*j)) .. +7, j < CH): all of a
+// lane's loads are issued at once, the statistics need only warp shuffles (plus one shared-memory
+// hop when W > 1).  256-thread CTAs hold 8/W rows.
+template <int CH>
 __global__ void __launch_bounds__(kRowThreadsMax)
 ln_fwd_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gamma,
               const __nv_bfloat16* __restrict__ beta, int T, int d, float eps, __nv_bfloat16* __restrict__ h,
-              float* __restrict__ mu, float* __restrict__ rstd, int tpr, int rows_per_cta)
+              float* __restrict__ mu, float* __restrict__ rstd, int W)
 {
     __shared__ float red[2][kMaxWarps];
-    const int row_in_cta = threadIdx.x / tpr, tr = threadIdx.x % tpr;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rows_per_cta = kMaxWarps / W;
+    const int row_in_cta = warp / W, wr = warp % W;
     const int row = blockIdx.x * rows_per_cta + row_in_cta;
-    const int wpr = tpr >> 5;
-    const bool live = row < T;
-    float v[CHUNKS][8];
+    const bool live = row < T && row_in_cta < rows_per_cta;
+    float v[CH][8];
     float s = 0.f;
 #pragma unroll
-    for (int j = 0; j < CHUNKS; ++j) {
-        const int col = 8 * (tr + j * tpr);
-        uint4 raw = live ? *reinterpret_cast<const uint4*>(x + static_cast<size_t>(row) * d + col) : make_uint4(0, 0, 0, 0);
+    for (int j = 0; j < CH; ++j) {
+        const int col = 8 * (lane + 32 * (wr + W * j));
+        const uint4 raw = live ? *reinterpret_cast<const uint4*>(x + static_cast<size_t>(row) * d + col) : make_uint4(0, 0, 0, 0);
         unpack8(raw, v[j]);
 #pragma unroll
         for (int k = 0; k < 8; ++k) s += v[j][k];
     }
-    const float mean = row_sum(s, red[0], wpr, row_in_cta) / d;
+    s = warp_sum(s);
+    if (W > 1) {
+        if (lane == 0) red[0][warp] = s;
+        __syncthreads();
+        s = 0.f;
+        for (int i = 0; i < W; ++i) s += red[0][row_in_cta * W + i];
+    }
+    const float mean = s / d;
     float q = 0.f;
 #pragma unroll
-    for (int j = 0; j < CHUNKS; ++j)
+    for (int j = 0; j < CH; ++j)
 #pragma unroll
         for (int k = 0; k < 8; ++k) { const float c = v[j][k] - mean; q += c * c; }
-    const float var = row_sum(q, red[1], wpr, row_in_cta) / d;
-    const float r = rsqrtf(var + eps);
+    q = warp_sum(q);
+    if (W > 1) {
+        if (lane == 0) red[1][warp] = q;
+        __syncthreads();
+        q = 0.f;
+        for (int i = 0; i < W; ++i) q += red[1][row_in_cta * W + i];
+    }
+    const float r = rsqrtf(q / d + eps);
     if (!live) return;
 #pragma unroll
-    for (int j = 0; j < CHUNKS; ++j) {
-        const int col = 8 * (tr + j * tpr);
+    for (int j = 0; j < CH; ++j) {
+        const int col = 8 * (lane + 32 * (wr + W * j));
         float g[8], b[8], o[8];
         unpack8(__ldg(reinterpret_cast<const uint4*>(gamma + col)), g);
         unpack8(__ldg(reinterpret_cast<const uint4*>(beta + col)), b);
@@ -90,12 +108,24 @@ ln_fwd_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restri
         for (int k = 0; k < 8; ++k) o[k] = g[k] * ((v[j][k] - mean) * r) + b[k];
         *reinterpret_cast<uint4*>(h + static_cast<size_t>(row) * d + col) = pack8(o);
     }
-    if (tr == 0) { mu[row] = mean; rstd[row] = r; }
+    if (wr == 0 && lane == 0) { mu[row] = mean; rstd[row] = r; }
+}
+
+// W warps per row and CH pieces per lane for a row of d elements (d a multiple of 256).
+bool plan_warp_rows(int d, int* W, int* CH)
+{
+    if (d % 256 != 0) return false;
+    const int total = d / 256;
+    for (int w = 1; w <= kMaxWarps; ++w)
+        if (total % w == 0 && total / w <= 8 && kMaxWarps % w == 0) { *W = w; *CH = total / w; return true; }
+    return false;
 }
 
 // LayerNorm backward.  Persistent over rows; every thread keeps the column sums of its own
 // columns in registers and writes them once at the end as one partial row per (CTA, row slot):
 // partials[(cta*rows_per_cta + row_in_cta)][4][d] = {dgamma, dbeta, sum resid, sum dx}.
+// The next row's three inputs are fetched before the current row's reduction, and the two row
+// sums share one barrier.
 template <int CHUNKS>
 __global__ void __launch_bounds__(kRowThreadsMax)
 ln_bwd_kernel(const __nv_bfloat16* __restrict__ dh, const __nv_bfloat16* __restrict__ x,
@@ -105,7 +135,7 @@ ln_bwd_kernel(const __nv_bfloat16* __restrict__ dh, const __nv_bfloat16* __restr
 {
     __shared__ float red[2][2][kMaxWarps];
     const int row_in_cta = threadIdx.x / tpr, tr = threadIdx.x % tpr;
-    const int wpr = tpr >> 5;
+    const int wpr = tpr >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     float gm[CHUNKS][8];
     float acc_g[CHUNKS][8], acc_b[CHUNKS][8], acc_r[CHUNKS][8], acc_x[CHUNKS][8];
 #pragma unroll
@@ -115,20 +145,34 @@ ln_bwd_kernel(const __nv_bfloat16* __restrict__ dh, const __nv_bfloat16* __restr
         for (int k = 0; k < 8; ++k) acc_g[j][k] = acc_b[j][k] = acc_r[j][k] = acc_x[j][k] = 0.f;
     }
     const int row_groups = (T + rows_per_cta - 1) / rows_per_cta;
+    uint4 n_dh[CHUNKS], n_x[CHUNKS], n_rs[CHUNKS];
+    float n_m = 0.f, n_r = 0.f;
+    auto fetch = [&](int rg) {
+        const int row = rg * rows_per_cta + row_in_cta;
+        const bool live = rg < row_groups && row < T;
+        n_m = live ? mu[row] : 0.f;
+        n_r = live ? rstd[row] : 0.f;
+#pragma unroll
+        for (int j = 0; j < CHUNKS; ++j) {
+            const size_t off = static_cast<size_t>(row) * d + 8 * (tr + j * tpr);
+            n_dh[j] = live ? *reinterpret_cast<const uint4*>(dh + off) : make_uint4(0, 0, 0, 0);
+            n_x[j] = live ? *reinterpret_cast<const uint4*>(x + off) : make_uint4(0, 0, 0, 0);
+            n_rs[j] = live ? *reinterpret_cast<const uint4*>(resid + off) : make_uint4(0, 0, 0, 0);
+        }
+    };
+    fetch(blockIdx.x);
     int par = 0;
     for (int rg = blockIdx.x; rg < row_groups; rg += gridDim.x, par ^= 1) {
         const int row = rg * rows_per_cta + row_in_cta;
         const bool live = row < T;
-        const float m = live ? mu[row] : 0.f, r = live ? rstd[row] : 0.f;
-        float xh[CHUNKS][8], g[CHUNKS][8], dhv[CHUNKS][8];
+        const float m = n_m, r = n_r;
+        float xh[CHUNKS][8], g[CHUNKS][8], dhv[CHUNKS][8], rs[CHUNKS][8];
         float s1 = 0.f, s2 = 0.f;
 #pragma unroll
         for (int j = 0; j < CHUNKS; ++j) {
-            const size_t off = static_cast<size_t>(row) * d + 8 * (tr + j * tpr);
-            uint4 a = live ? *reinterpret_cast<const uint4*>(dh + off) : make_uint4(0, 0, 0, 0);
-            uint4 b = live ? *reinterpret_cast<const uint4*>(x + off) : make_uint4(0, 0, 0, 0);
-            unpack8(a, dhv[j]);
-            unpack8(b, xh[j]);
+            unpack8(n_dh[j], dhv[j]);
+            unpack8(n_x[j], xh[j]);
+            unpack8(n_rs[j], rs[j]);
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 xh[j][k] = (xh[j][k] - m) * r;
@@ -137,16 +181,23 @@ ln_bwd_kernel(const __nv_bfloat16* __restrict__ dh, const __nv_bfloat16* __restr
                 s2 += g[j][k] * xh[j][k];
             }
         }
-        const float mg = row_sum(s1, red[par][0], wpr, row_in_cta) / d;
-        const float mgx = row_sum(s2, red[par][1], wpr, row_in_cta) / d;
+        fetch(rg + gridDim.x);            // next row's loads are in flight during the reduction
+        s1 = warp_sum(s1);
+        s2 = warp_sum(s2);
+        if (wpr > 1) {
+            if (lane == 0) { red[par][0][warp] = s1; red[par][1][warp] = s2; }
+            __syncthreads();
+            s1 = 0.f; s2 = 0.f;
+            for (int i = 0; i < wpr; ++i) { s1 += red[par][0][row_in_cta * wpr + i]; s2 += red[par][1][row_in_cta * wpr + i]; }
+        }
+        const float mg = s1 / d, mgx = s2 / d;
         if (live) {
 #pragma unroll
             for (int j = 0; j < CHUNKS; ++j) {
                 const size_t off = static_cast<size_t>(row) * d + 8 * (tr + j * tpr);
-                float rs[8], o[8];
-                unpack8(*reinterpret_cast<const uint4*>(resid + off), rs);
+                float o[8];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) o[k] = rs[k] + r * (g[j][k] - mg - xh[j][k] * mgx);
+                for (int k = 0; k < 8; ++k) o[k] = rs[j][k] + r * (g[j][k] - mg - xh[j][k] * mgx);
                 const uint4 packed = pack8(o);
                 *reinterpret_cast<uint4*>(dx + off) = packed;
                 float ob[8];
@@ -155,7 +206,7 @@ ln_bwd_kernel(const __nv_bfloat16* __restrict__ dh, const __nv_bfloat16* __restr
                 for (int k = 0; k < 8; ++k) {
                     acc_g[j][k] += dhv[j][k] * xh[j][k];
                     acc_b[j][k] += dhv[j][k];
-                    acc_r[j][k] += rs[k];
+                    acc_r[j][k] += rs[j][k];
                     acc_x[j][k] += ob[k];
                 }
             }
@@ -175,18 +226,30 @@ ln_bwd_kernel(const __nv_bfloat16* __restrict__ dh, const __nv_bfloat16* __restr
     }
 }
 
-// out_q[c] (+)= sum over partial rows of partials[row][q][c], fixed order.  Up to 4 outputs.
+// out_q[c] (+)= sum over partial rows of partials[row][q][c].  CTA = 32 columns x 8 row lanes:
+// row lane y adds rows y, y+8, ... in order, then the 8 lane sums are added in order, so the
+// result does not depend on scheduling.  Up to 4 outputs (grid.y = quantity).
 struct ReduceOuts { float* out[4]; };
-__global__ void reduce_partials_kernel(const float* __restrict__ partials, int nrows, int nq, int n, ReduceOuts outs,
-                                       int accumulate)
+__global__ void __launch_bounds__(256)
+reduce_partials_kernel(const float* __restrict__ partials, int nrows, int nq, int n, ReduceOuts outs, int accumulate)
 {
-    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    __shared__ float sm[8][33];
+    const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+    const int c = blockIdx.x * 32 + cx;
     const int q = blockIdx.y;
     float* out = outs.out[q];
-    if (c >= n || out == nullptr) return;
+    if (out == nullptr) return;
     float s = 0.f;
-    for (int r = 0; r < nrows; ++r) s += partials[(static_cast<size_t>(r) * nq + q) * n + c];
-    out[c] = accumulate ? out[c] + s : s;
+    if (c < n)
+        for (int r = ry; r < nrows; r += 8) s += partials[(static_cast<size_t>(r) * nq + q) * n + c];
+    sm[ry][cx] = s;
+    __syncthreads();
+    if (ry == 0 && c < n) {
+        float t = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) t += sm[i][cx];
+        out[c] = accumulate ? out[c] + t : t;
+    }
 }
 
 // Column sums of a bf16 [T, N] matrix: CTA (x, y) owns columns 1024*x .. +1023 and rows y, y+R, ...
@@ -233,7 +296,7 @@ int colsum_splits(Runtime* rt, int T, int N)
 int ln_bwd_grid(Runtime* rt, int T, const RowPlan& rp)
 {
     const int row_groups = (T + rp.rows_per_cta - 1) / rp.rows_per_cta;
-    const int cap = 2 * rt->sm_count;
+    const int cap = rt->sm_count;
     return row_groups < cap ? row_groups : cap;
 }
 
@@ -243,20 +306,22 @@ const char* launch_layernorm_fwd(Runtime* rt, const void* x, const void* gamma, 
                                  float eps, void* h, void* mu, void* rstd, cudaStream_t stream)
 {
     (void)rt;
-    RowPlan rp;
-    if (T <= 0 || !plan_rows(d, &rp)) return "layernorm: unsupported row width";
-    const int grid = (T + rp.rows_per_cta - 1) / rp.rows_per_cta;
+    int W = 0, CH = 0;
+    if (T <= 0 || !plan_warp_rows(d, &W, &CH)) return "layernorm: unsupported row width";
+    const int rows_per_cta = kMaxWarps / W;
+    const int grid = (T + rows_per_cta - 1) / rows_per_cta;
     auto X = static_cast<const __nv_bfloat16*>(x);
     auto G = static_cast<const __nv_bfloat16*>(gamma);
     auto Bt = static_cast<const __nv_bfloat16*>(beta);
     auto Hh = static_cast<__nv_bfloat16*>(h);
     auto Mu = static_cast<float*>(mu);
     auto Rs = static_cast<float*>(rstd);
-    switch (rp.chunks) {
-        case 1: ln_fwd_kernel<1><<<grid, rp.threads, 0, stream>>>(X, G, Bt, T, d, eps, Hh, Mu, Rs, rp.tpr, rp.rows_per_cta); break;
-        case 2: ln_fwd_kernel<2><<<grid, rp.threads, 0, stream>>>(X, G, Bt, T, d, eps, Hh, Mu, Rs, rp.tpr, rp.rows_per_cta); break;
-        default: ln_fwd_kernel<4><<<grid, rp.threads, 0, stream>>>(X, G, Bt, T, d, eps, Hh, Mu, Rs, rp.tpr, rp.rows_per_cta); break;
+#define PW_LN_FWD(N) case N: ln_fwd_kernel<N><<<grid, kRowThreadsMax, 0, stream>>>(X, G, Bt, T, d, eps, Hh, Mu, Rs, W); break
+    switch (CH) {
+        PW_LN_FWD(1); PW_LN_FWD(2); PW_LN_FWD(3); PW_LN_FWD(4); PW_LN_FWD(5); PW_LN_FWD(6); PW_LN_FWD(7); PW_LN_FWD(8);
+        default: return "layernorm: unsupported row width";
     }
+#undef PW_LN_FWD
     return cudaGetLastError() == cudaSuccess ? nullptr : "layernorm fwd launch failed";
 }
 
@@ -292,7 +357,7 @@ const char* launch_layernorm_bwd(Runtime* rt, const void* dh, const void* x, con
     ReduceOuts outs;
     outs.out[0] = static_cast<float*>(dgamma); outs.out[1] = static_cast<float*>(dbeta);
     outs.out[2] = static_cast<float*>(db_resid); outs.out[3] = static_cast<float*>(db_dx);
-    dim3 rgrid((d + 255) / 256, 4);
+    dim3 rgrid((d + 31) / 32, 4);
     reduce_partials_kernel<<<rgrid, 256, 0, stream>>>(P, grid * rp.rows_per_cta, 4, d, outs, accumulate);
     return cudaGetLastError() == cudaSuccess ? nullptr : "layernorm bwd reduce launch failed";
 }
@@ -313,7 +378,7 @@ const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, voi
     if (cudaGetLastError() != cudaSuccess) return "colsum launch failed";
     ReduceOuts outs;
     outs.out[0] = static_cast<float*>(out); outs.out[1] = outs.out[2] = outs.out[3] = nullptr;
-    dim3 rgrid((N + 255) / 256, 1);
+    dim3 rgrid((N + 31) / 32, 1);
     reduce_partials_kernel<<<rgrid, 256, 0, stream>>>(static_cast<const float*>(partials), R, 1, N, outs, accumulate);
     return cudaGetLastError() == cudaSuccess ? nullptr : "colsum reduce launch failed";
 }

@@ -12,79 +12,60 @@
 //
 // Every wait on an mbarrier is bounded (see mbar_wait); on expiry the CTA raises an abort flag,
 // all roles leave their loops, the TMEM allocation is released and the kernel returns.
+#include <cstdlib>
+
 #include "pw_kernels.h"
 
 namespace pw {
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
-constexpr int A_TILE_BYTES = BM * BK * 2;   // 16 KB
-constexpr int B_TILE_BYTES = BN * BK * 2;   // 32 KB
+constexpr int BM = 128, BN_MAX = 256, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr int A_TILE_BYTES = BM * BK * 2;       // 16 KB
+constexpr int B_TILE_BYTES = BN_MAX * BK * 2;   // 32 KB (a narrower tile uses the front of it)
 constexpr int STAGE_BYTES = A_TILE_BYTES + B_TILE_BYTES;
-constexpr int GEMM_THREADS = 192;
-constexpr int TMEM_COLS = 2 * BN;           // two accumulators: the whole 512-column TMEM
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int EPI_WARPS = 8;
+constexpr int GEMM_THREADS = 64 + 32 * EPI_WARPS;   // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
+constexpr int TMEM_COLS = 2 * BN_MAX;           // two accumulators: the whole 512-column TMEM
+constexpr int SLAB_BYTES = 4096;                // per epilogue warp: 32 rows x 128 bytes, swizzled
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * SLAB_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
 struct GemmParams {
     int M, N, K;
-    void* C; int ldc;
+    int bn;                      // tile width actually used: 128, 192 or 256
     const __nv_bfloat16* bias;
     const __nv_bfloat16* aux_in; int ld_aux;
-    __nv_bfloat16* aux_out;
     int accumulate, act;
     int m_tiles, n_tiles;
     DeviceStatus* status;
 };
 
+// One 8-column group of the bf16 epilogues: f = acc (+bias) (+residual | x GeLU'(u)).
 template <int EPI>
-__device__ __forceinline__ void epilogue_chunk(const uint32_t* v, int row, int col0, const GemmParams& p)
+__device__ __forceinline__ void epilogue_group(const uint32_t* v, int row, int c, const GemmParams& p, float* f)
 {
-    if constexpr (EPI == kEpiF32) {
-        float* c = reinterpret_cast<float*>(p.C) + static_cast<size_t>(row) * p.ldc + col0;
 #pragma unroll
-        for (int g = 0; g < 8; ++g) {
-            if (col0 + 4 * g < p.N) {
-                float4 o = make_float4(__uint_as_float(v[4 * g]), __uint_as_float(v[4 * g + 1]),
-                                       __uint_as_float(v[4 * g + 2]), __uint_as_float(v[4 * g + 3]));
-                if (p.accumulate) {
-                    float4 old = *reinterpret_cast<const float4*>(c + 4 * g);
-                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
-                }
-                *reinterpret_cast<float4*>(c + 4 * g) = o;
+    for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[j]);
+    if (c < p.N) {
+        if constexpr (EPI == kEpiBias || EPI == kEpiBiasResid || EPI == kEpiBiasGelu) {
+            float b[8];
+            unpack8(__ldg(reinterpret_cast<const uint4*>(p.bias + c)), b);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) f[j] += b[j];
+        }
+        if constexpr (EPI == kEpiBiasResid) {
+            if (row < p.M) {
+                float r[8];
+                unpack8(*reinterpret_cast<const uint4*>(p.aux_in + static_cast<size_t>(row) * p.ld_aux + c), r);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) f[j] += r[j];
             }
         }
-    } else {
-        __nv_bfloat16* c = reinterpret_cast<__nv_bfloat16*>(p.C) + static_cast<size_t>(row) * p.ldc + col0;
+        if constexpr (EPI == kEpiDGelu) {
+            if (row < p.M) {
+                float u[8];
+                unpack8(*reinterpret_cast<const uint4*>(p.aux_in + static_cast<size_t>(row) * p.ld_aux + c), u);
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            if (col0 + 8 * g < p.N) {
-                float f[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[8 * g + j]);
-                if constexpr (EPI == kEpiBias || EPI == kEpiBiasResid || EPI == kEpiBiasGelu) {
-                    float b[8];
-                    unpack8(__ldg(reinterpret_cast<const uint4*>(p.bias + col0 + 8 * g)), b);
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) f[j] += b[j];
-                }
-                if constexpr (EPI == kEpiBiasResid) {
-                    float r[8];
-                    unpack8(*reinterpret_cast<const uint4*>(p.aux_in + static_cast<size_t>(row) * p.ld_aux + col0 + 8 * g), r);
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) f[j] += r[j];
-                }
-                if constexpr (EPI == kEpiDGelu) {
-                    float u[8];
-                    unpack8(*reinterpret_cast<const uint4*>(p.aux_in + static_cast<size_t>(row) * p.ld_aux + col0 + 8 * g), u);
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) f[j] *= gelu_grad_f(u[j], p.act);
-                }
-                *reinterpret_cast<uint4*>(c + 8 * g) = pack8(f);
-                if constexpr (EPI == kEpiBiasGelu) {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) f[j] = gelu_f(f[j], p.act);
-                    *reinterpret_cast<uint4*>(p.aux_out + static_cast<size_t>(row) * p.ldc + col0 + 8 * g) = pack8(f);
-                }
+                for (int j = 0; j < 8; ++j) f[j] *= gelu_grad_f(u[j], p.act);
             }
         }
     }
@@ -92,11 +73,13 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t* v, int row, int c
 
 template <bool A_MN, bool B_MN, int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p)
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmAux, const GemmParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + STAGES * STAGE_BYTES);
+    uint8_t* slabs = tiles + STAGES * STAGE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(slabs + EPI_WARPS * SLAB_BYTES);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + STAGES);
     const uint32_t accf0 = smem_u32(bars + 2 * STAGES), acce0 = smem_u32(bars + 2 * STAGES + 2);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
@@ -105,15 +88,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_k = (p.K + BK - 1) / BK;
     const int total_tiles = p.m_tiles * p.n_tiles;
+    const int bn = p.bn;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 128); }
+        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 32 * EPI_WARPS); }
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async();
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
+        prefetch_tmap(&tmC);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
@@ -128,12 +113,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
+            const uint32_t stage_tx = A_TILE_BYTES + bn * BK * 2;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile % p.m_tiles) * BM, n0 = (tile / p.m_tiles) * BN;
+                const int m0 = (tile % p.m_tiles) * BM, n0 = (tile / p.m_tiles) * bn;
                 for (int kb = 0; kb < num_k; ++kb) {
                     if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 100)) { ok = false; break; }
                     const uint32_t fb = full0 + 8 * stage;
-                    mbar_arrive_expect_tx(fb, STAGE_BYTES);
+                    mbar_arrive_expect_tx(fb, stage_tx);
                     const uint32_t a_dst = smem_u32(tiles + stage * STAGE_BYTES), b_dst = a_dst + A_TILE_BYTES;
                     if constexpr (!A_MN) {
                         tma_load_2d(a_dst, &tmA, kb * BK, m0, fb);
@@ -144,8 +130,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     if constexpr (!B_MN) {
                         tma_load_2d(b_dst, &tmB, kb * BK, n0, fb);
                     } else {
-#pragma unroll
-                        for (int j = 0; j < BN / 64; ++j) tma_load_2d(b_dst + j * 8192, &tmB, n0 + 64 * j, kb * BK, fb);
+                        for (int j = 0; j < bn / 64; ++j) tma_load_2d(b_dst + j * 8192, &tmB, n0 + 64 * j, kb * BK, fb);
                     }
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
@@ -153,14 +138,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16(BM, BN, A_MN, B_MN);
+            const uint32_t idesc = make_idesc_bf16(BM, bn, A_MN, B_MN);
             uint32_t stage = 0, phase = 0, it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
                 const uint32_t buf = it & 1, acc_phase = (it >> 1) & 1;
                 if (!mbar_wait(acce0 + 8 * buf, acc_phase ^ 1, abort_flag, p.status, 200)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * BN;
+                const uint32_t d_tmem = tmem_base + buf * BN_MAX;
                 for (int kb = 0; kb < num_k; ++kb) {
                     if (!mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 201)) { ok = false; break; }
                     tc_fence_after();
@@ -182,29 +167,95 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
         }
     } else {
-        const int ew = warp & 3;
-        uint32_t it = 0;
+        // Epilogue: warp w may read TMEM lanes 32*(w%4)..+31; the two warps of a lane quarter take
+        // alternate column steps.  Each step goes TMEM -> registers -> swizzled shared slab -> one
+        // TMA store (rows >= M and columns >= N are clipped by the tensor map).
+        const int q = warp & 3, pi = (warp - 2) >> 2;
+        uint8_t* slab = slabs + (warp - 2) * SLAB_BYTES;
+        const uint32_t slab_u32 = smem_u32(slab);
+        uint8_t* my_row = slab + lane * 128;
+        uint32_t it = 0, nout = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
-            const int m0 = (tile % p.m_tiles) * BM, n0 = (tile / p.m_tiles) * BN;
+            const int m0 = (tile % p.m_tiles) * BM, n0 = (tile / p.m_tiles) * bn;
             const uint32_t buf = it & 1, acc_phase = (it >> 1) & 1;
             bool ok = mbar_wait(accf0 + 8 * buf, acc_phase, abort_flag, p.status, 300);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const int row = m0 + ew * 32 + lane;
-            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(ew * 32) << 16) + buf * BN;
+            const int row = m0 + q * 32 + lane;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * BN_MAX;
+            if constexpr (EPI == kEpiF32) {
+                const int nsteps = bn / 32;
 #pragma unroll 1
-            for (int chunk = 0; chunk < BN / 32; ++chunk) {
-                const int col0 = n0 + chunk * 32;
-                if (col0 >= p.N) break;
-                uint32_t v[32];
-                tmem_ld32(taddr + chunk * 32, v);
-                tc_wait_ld();
-                if (row < p.M) epilogue_chunk<EPI>(v, row, col0, p);
+                for (int s = pi; s < nsteps; s += 2) {
+                    const int col0 = n0 + s * 32;
+                    if (col0 >= p.N) break;
+                    uint32_t v[32];
+                    tmem_ld32(taddr + s * 32, v);
+                    tc_wait_ld();
+                    if (lane == 0) bulk_wait_read0();
+                    __syncwarp();
+#pragma unroll
+                    for (int g = 0; g < 8; ++g)
+                        *reinterpret_cast<uint4*>(my_row + ((g ^ (lane & 7)) << 4)) =
+                            make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (p.accumulate) tma_reduce_add_2d(&tmC, slab_u32, col0, m0 + q * 32);
+                        else tma_store_2d(&tmC, slab_u32, col0, m0 + q * 32);
+                        bulk_commit();
+                    }
+                }
+            } else {
+                // 32 columns per chunk; the slab is two 2 KB halves (32 rows x 64 bytes, 64-byte
+                // swizzle) used alternately, so one store is always in flight behind the math.
+                const int nchunks = bn / 32;
+                const uint32_t sw = (lane >> 1) & 3;
+#pragma unroll 1
+                for (int ch = pi; ch < nchunks; ch += 2) {
+                    const int col0 = n0 + ch * 32;
+                    if (col0 >= p.N) break;
+                    uint32_t v[32];
+                    tmem_ld32(taddr + ch * 32, v);
+                    tc_wait_ld();
+                    uint4 o[4], o2[4];
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        float f[8];
+                        epilogue_group<EPI>(v + 8 * g, row, col0 + g * 8, p, f);
+                        o[g] = pack8(f);
+                        if constexpr (EPI == kEpiBiasGelu) {
+                            // GeLU of the bf16 value stored as u: the backward reads u back and sees
+                            // exactly the argument the forward used
+                            unpack8(o[g], f);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) f[j] = gelu_f(f[j], p.act);
+                            o2[g] = pack8(f);
+                        }
+                    }
+                    constexpr int kOuts = (EPI == kEpiBiasGelu) ? 2 : 1;
+#pragma unroll
+                    for (int t = 0; t < kOuts; ++t) {
+                        const uint32_t half = (nout++ & 1u) * 2048u;
+                        if (lane == 0) bulk_wait_read1();
+                        __syncwarp();
+#pragma unroll
+                        for (int g = 0; g < 4; ++g)
+                            *reinterpret_cast<uint4*>(slab + half + lane * 64 + ((g ^ sw) << 4)) = (t == 0) ? o[g] : o2[g];
+                        fence_proxy_async();
+                        __syncwarp();
+                        if (lane == 0) {
+                            tma_store_2d(t == 0 ? &tmC : &tmAux, slab_u32 + half, col0, m0 + q * 32);
+                            bulk_commit();
+                        }
+                    }
+                }
             }
             tc_fence_before();
             mbar_arrive(acce0 + 8 * buf);
         }
+        if (lane == 0) bulk_wait0();
     }
 
     __syncwarp();
@@ -224,29 +275,30 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// 2-D bf16 tensor map: `inner` contiguous elements per row, `outer` rows, row pitch ld elements.
+// 2-D tensor map (bf16, or fp32 when f32 is set): `inner` contiguous elements per row, `outer`
+// rows, row pitch ld elements; 128-byte swizzle, so box_inner * element size must be 128 bytes.
 const char* encode_2d(Runtime* rt, CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t outer, uint64_t ld,
-                      uint32_t box_inner, uint32_t box_outer)
+                      uint32_t box_inner, uint32_t box_outer, bool f32 = false, bool swizzle64 = false)
 {
     cuuint64_t dims[2] = {inner, outer};
-    cuuint64_t strides[1] = {ld * 2};
+    cuuint64_t strides[1] = {ld * (f32 ? 4 : 2)};
     cuuint32_t box[2] = {box_inner, box_outer};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = reinterpret_cast<EncodeTiledFn>(rt->encode_tiled)(
-        map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? nullptr : "cuTensorMapEncodeTiled failed";
 }
 
 template <bool A_MN, bool B_MN, int EPI>
-const char* launch_inst(Runtime* rt, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p,
-                        cudaStream_t stream)
+const char* launch_inst(Runtime* rt, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
+                        const CUtensorMap& tmAux, const GemmParams& p, cudaStream_t stream)
 {
     auto kern = gemm_kernel<A_MN, B_MN, EPI>;
     const int total = p.m_tiles * p.n_tiles;
     const int grid = total < rt->sm_count ? total : rt->sm_count;
-    kern<<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, p);
+    kern<<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, tmC, tmAux, p);
     return cudaGetLastError() == cudaSuccess ? nullptr : "gemm launch failed";
 }
 
@@ -284,33 +336,52 @@ const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cu
     if (a.epilogue == kEpiBiasGelu && (!a.aux_out || misaligned(a.aux_out))) return "gemm: epilogue needs aux_out";
 
     const bool a_mn = a.layout == kNT, b_mn = a.layout == kNN || a.layout == kNT;
-    CUtensorMap tmA, tmB;
+    const bool f32_out = a.epilogue == kEpiF32;
+    if (f32_out && (a.ldc % 4)) return "gemm: fp32 ldc must be a multiple of 4";
+    // Tile width: the one that needs the least (rounds x width) on this many SMs; ties go to the
+    // wider tile (less operand traffic per FLOP).
+    const int m_tiles = (a.M + BM - 1) / BM;
+    // Tile width 256 unless that leaves most SMs without a tile (small problems are latency-bound;
+    // a narrower tile spreads them over more SMs).  Narrower tiles cost more operand traffic per
+    // FLOP and were measured slower whenever every SM already has work.
+    int bn = BN_MAX;
+    while (bn > 128 && static_cast<long long>(m_tiles) * ((a.N + bn - 1) / bn) * 2 <= rt->sm_count) bn -= 64;
+    {
+        static const int forced = [] { const char* v = getenv("PW_GEMM_BN"); return v ? atoi(v) : 0; }();
+        if (forced == 128 || forced == 192 || forced == 256) bn = forced;   // tuning aid
+    }
+    CUtensorMap tmA, tmB, tmC, tmAux;
     const char* e;
     // K-major operand [rows, K]: box 64 k x rows.  MN-major operand stored [K, rows]: box 64 rows x 64 k.
     e = a_mn ? encode_2d(rt, &tmA, a.A, a.M, a.K, a.lda, 64, BK) : encode_2d(rt, &tmA, a.A, a.K, a.M, a.lda, BK, BM);
     if (e) return e;
-    e = b_mn ? encode_2d(rt, &tmB, a.B, a.N, a.K, a.ldb, 64, BK) : encode_2d(rt, &tmB, a.B, a.K, a.N, a.ldb, BK, BN);
+    e = b_mn ? encode_2d(rt, &tmB, a.B, a.N, a.K, a.ldb, 64, BK) : encode_2d(rt, &tmB, a.B, a.K, a.N, a.ldb, BK, bn);
+    if (e) return e;
+
+    // Output maps: a store box is 32 rows x 32 columns (fp32: 128-byte rows, 128-byte swizzle;
+    // bf16: 64-byte rows, 64-byte swizzle).
+    e = encode_2d(rt, &tmC, a.C, a.N, a.M, a.ldc, 32, 32, f32_out, !f32_out);
+    if (e) return e;
+    e = encode_2d(rt, &tmAux, a.epilogue == kEpiBiasGelu ? a.aux_out : a.C, a.N, a.M, a.ldc, 32, 32, f32_out, !f32_out);
     if (e) return e;
 
     GemmParams p;
-    p.M = a.M; p.N = a.N; p.K = a.K;
-    p.C = a.C; p.ldc = a.ldc;
+    p.M = a.M; p.N = a.N; p.K = a.K; p.bn = bn;
     p.bias = static_cast<const __nv_bfloat16*>(a.bias);
     p.aux_in = static_cast<const __nv_bfloat16*>(a.aux_in); p.ld_aux = a.ld_aux;
-    p.aux_out = static_cast<__nv_bfloat16*>(a.aux_out);
     p.accumulate = a.accumulate; p.act = a.act;
-    p.m_tiles = (a.M + BM - 1) / BM; p.n_tiles = (a.N + BN - 1) / BN;
+    p.m_tiles = m_tiles; p.n_tiles = (a.N + bn - 1) / bn;
     p.status = status;
 
     const int key = a.layout * 16 + a.epilogue;
     switch (key) {
-        case kTN * 16 + kEpiNone: return launch_inst<false, false, kEpiNone>(rt, tmA, tmB, p, stream);
-        case kTN * 16 + kEpiBias: return launch_inst<false, false, kEpiBias>(rt, tmA, tmB, p, stream);
-        case kTN * 16 + kEpiBiasResid: return launch_inst<false, false, kEpiBiasResid>(rt, tmA, tmB, p, stream);
-        case kTN * 16 + kEpiBiasGelu: return launch_inst<false, false, kEpiBiasGelu>(rt, tmA, tmB, p, stream);
-        case kNN * 16 + kEpiNone: return launch_inst<false, true, kEpiNone>(rt, tmA, tmB, p, stream);
-        case kNN * 16 + kEpiDGelu: return launch_inst<false, true, kEpiDGelu>(rt, tmA, tmB, p, stream);
-        case kNT * 16 + kEpiF32: return launch_inst<true, true, kEpiF32>(rt, tmA, tmB, p, stream);
+        case kTN * 16 + kEpiNone: return launch_inst<false, false, kEpiNone>(rt, tmA, tmB, tmC, tmAux, p, stream);
+        case kTN * 16 + kEpiBias: return launch_inst<false, false, kEpiBias>(rt, tmA, tmB, tmC, tmAux, p, stream);
+        case kTN * 16 + kEpiBiasResid: return launch_inst<false, false, kEpiBiasResid>(rt, tmA, tmB, tmC, tmAux, p, stream);
+        case kTN * 16 + kEpiBiasGelu: return launch_inst<false, false, kEpiBiasGelu>(rt, tmA, tmB, tmC, tmAux, p, stream);
+        case kNN * 16 + kEpiNone: return launch_inst<false, true, kEpiNone>(rt, tmA, tmB, tmC, tmAux, p, stream);
+        case kNN * 16 + kEpiDGelu: return launch_inst<false, true, kEpiDGelu>(rt, tmA, tmB, tmC, tmAux, p, stream);
+        case kNT * 16 + kEpiF32: return launch_inst<true, true, kEpiF32>(rt, tmA, tmB, tmC, tmAux, p, stream);
         default: return "gemm: unsupported layout/epilogue combination";
     }
 }

@@ -39,24 +39,48 @@ __device__ __forceinline__ uint4 pack8(const float* f)
     return v;
 }
 
-// GeLU and its derivative in fp32 (erf form by default, tanh form selectable).
+// GeLU and its derivative in fp32.  The erf form uses the rational/exponential approximation
+// erfc(x) ~ (a1 t + ... + a5 t^5) exp(-x^2), t = 1/(1 + p x), x >= 0 (absolute error about 2e-7,
+// far below bf16 resolution); the exponential exp(-u^2/2) is shared with the density term of the
+// derivative.  act == 1 selects the tanh form.
+__device__ __forceinline__ void normal_cdf_pdf(float u, float& cdf, float& e /* exp(-u^2/2) */)
+{
+    const float ax = fabsf(u) * 0.7071067811865476f;
+    const float t = __frcp_rn(fmaf(0.3275911f, ax, 1.0f));
+    e = __expf(-ax * ax);
+    float poly = fmaf(t, 1.061405429f, -1.453152027f);
+    poly = fmaf(t, poly, 1.421413741f);
+    poly = fmaf(t, poly, -0.284496736f);
+    poly = fmaf(t, poly, 0.254829592f);
+    const float half_tail = 0.5f * poly * t * e;      // = erfc(|u|/sqrt2) / 2
+    cdf = u < 0.f ? half_tail : 1.0f - half_tail;
+}
+__device__ __forceinline__ float fast_tanh(float z)
+{
+    const float e2 = __expf(2.0f * z);
+    return 1.0f - __fdividef(2.0f, e2 + 1.0f);
+}
 __device__ __forceinline__ float gelu_f(float u, int act)
 {
     if (act == 1) {
-        float z = 0.7978845608028654f * (u + 0.044715f * u * u * u);
-        return 0.5f * u * (1.0f + tanhf(z));
+        const float z = 0.7978845608028654f * (u + 0.044715f * u * u * u);
+        return 0.5f * u * (1.0f + fast_tanh(z));
     }
-    return 0.5f * u * (1.0f + erff(u * 0.7071067811865476f));
+    float cdf, e;
+    normal_cdf_pdf(u, cdf, e);
+    return u * cdf;
 }
 __device__ __forceinline__ float gelu_grad_f(float u, int act)
 {
     if (act == 1) {
-        float z = 0.7978845608028654f * (u + 0.044715f * u * u * u);
-        float th = tanhf(z);
-        float dz = 0.7978845608028654f * (1.0f + 0.134145f * u * u);
+        const float z = 0.7978845608028654f * (u + 0.044715f * u * u * u);
+        const float th = fast_tanh(z);
+        const float dz = 0.7978845608028654f * (1.0f + 0.134145f * u * u);
         return 0.5f * (1.0f + th) + 0.5f * u * (1.0f - th * th) * dz;
     }
-    return 0.5f * (1.0f + erff(u * 0.7071067811865476f)) + u * __expf(-0.5f * u * u) * 0.3989422804014327f;
+    float cdf, e;
+    normal_cdf_pdf(u, cdf, e);
+    return fmaf(u * 0.3989422804014327f, e, cdf);
 }
 
 // ---------------------------------------------------------------- shared-memory addresses
@@ -132,6 +156,24 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
+// Shared -> global tiled store / fp32 reduce-add (out-of-range parts of the box are clipped).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(src) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, uint32_t src, int x, int y)
+{
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// All of this thread's bulk groups have finished READING shared memory (it may be rewritten).
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// At most the newest of this thread's bulk groups may still be reading shared memory.
+__device__ __forceinline__ void bulk_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+// All of this thread's bulk groups are complete.
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
