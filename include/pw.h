@@ -255,6 +255,26 @@ size_t pw_op_colsum_scratch_bytes(int T, int N);
 pw_status_t pw_op_colsum(const void* in, int T, int N, int ld, void* out, int accumulate, void* partials,
                          void* stream);
 
+/* Column sums for callers that cannot allocate device memory (the paper has no counterpart; this
+ * is a convenience of this library).  Same result as pw_op_colsum up to summation order, but the
+ * partial sums live in a 1 MiB array built into the library instead of a caller buffer, and the
+ * call itself allocates nothing on host-visible CUDA APIs: no cudaMalloc / cudaFree, no
+ * allocating library routine.  It is meant for code that runs when allocation is off the table:
+ * a serving loop whose memory pools already own all of HBM, a host callback, a plugin that is
+ * handed buffers but no allocator.
+ *   in  bf16 [T, N] device (row stride ld elements, ld >= N); out fp32 [N] device;
+ *   accumulate 0: out = sums, 1: out += sums.  N % 8 == 0, ld % 8 == 0.
+ * Limit: N <= 262144 columns (the array holds 262144 floats); beyond it the call returns
+ * PW_ERR_WORKSPACE_TOO_SMALL and launches nothing.  Fewer row groups are used than in
+ * pw_op_colsum when N is large, so the two may differ in the last fp32 bits.
+ * The first call on a device looks up the array's device address (once per device, with that
+ * device current); make that first call outside any stream capture.  Every call on a device
+ * shares the one array, which keeps the previous call's partial sums (each call overwrites the
+ * slots it later reads, so nothing needs clearing); calls whose kernels overlap on the GPU -
+ * different streams, or graphs replayed concurrently - race on it and must be serialised by the
+ * caller.  Each GPU that loads the library holds the 1 MiB until the process exits. */
+pw_status_t pw_op_colsum_noalloc(const void* in, int T, int N, int ld, void* out, int accumulate, void* stream);
+
 /* bf16 GEMM on the tensor cores, fp32 accumulation.  C[M,N] = op(A) op(B) then an epilogue.
  *   layout PW_GEMM_TN: A is [M,K] row-major (lda), B is [N,K] row-major (ldb)      (forward:  x W^T)
  *          PW_GEMM_NN: A is [M,K] row-major,       B is [K,N] row-major            (dgrad:    dy W)

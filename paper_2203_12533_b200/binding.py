@@ -36,7 +36,7 @@ EXPORTS = (
     "pw_stage_create", "pw_stage_destroy", "pw_stage_workspace_bytes", "pw_stage_run_chain", "pw_stage_status",
     "pw_stage_profile_begin", "pw_stage_profile_end", "pw_stage_launch_count",
     "pw_op_layernorm_fwd", "pw_op_layernorm_bwd_scratch_bytes", "pw_op_layernorm_bwd",
-    "pw_op_colsum_scratch_bytes", "pw_op_colsum", "pw_op_gemm",
+    "pw_op_colsum_scratch_bytes", "pw_op_colsum", "pw_op_colsum_noalloc", "pw_op_gemm",
     "pw_op_attention_fwd", "pw_op_attention_bwd", "pw_op_status",
 )
 
@@ -116,6 +116,7 @@ def lib() -> ctypes.CDLL:
         L.pw_op_layernorm_fwd.argtypes = [vp, vp, vp, ci, ci, ctypes.c_float, vp, vp, vp, vp]
         L.pw_op_layernorm_bwd.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp, vp, ci, vp, vp]
         L.pw_op_colsum.argtypes = [vp, ci, ci, ci, vp, ci, vp, vp]
+        L.pw_op_colsum_noalloc.argtypes = [vp, ci, ci, ci, vp, ci, vp]
         L.pw_op_gemm.argtypes = [ci, ci, ci, ci, ci, ci, vp, ci, vp, ci, vp, ci, vp, vp, ci, vp, ci, vp]
         L.pw_op_attention_fwd.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp]
         L.pw_op_attention_bwd.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, vp]
@@ -306,6 +307,17 @@ def op_colsum_scratch_bytes(T, N) -> int:
 def op_colsum(inp, out, accumulate, partials, stream=None):
     T, N = inp.shape
     _check(lib().pw_op_colsum(_p(inp), T, N, inp.stride(0), _p(out), int(accumulate), _p(partials), _stream(stream)))
+
+
+def op_colsum_noalloc(inp, out, accumulate, stream=None):
+    """Column sums of a bf16 [T, N] tensor into fp32 [N] without any device allocation.
+
+    For callers that may not allocate when they run (memory pools own all of HBM, host callbacks,
+    plugins without an allocator): the partial sums live in a 1 MiB array inside libpw.so, shared
+    by every call on the device, so overlapping calls must be serialised.  N <= 262144.
+    """
+    T, N = inp.shape
+    _check(lib().pw_op_colsum_noalloc(_p(inp), T, N, inp.stride(0), _p(out), int(accumulate), _stream(stream)))
 
 
 def op_gemm(layout, epilogue, M, N, K, A, lda, B, ldb, C, ldc, bias=None, aux_in=None, ld_aux=0, aux_out=None,

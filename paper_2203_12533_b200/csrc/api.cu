@@ -765,6 +765,17 @@ pw_status_t pw_op_colsum(const void* in, int T, int N, int ld, void* out, int ac
     return PW_OK;
 }
 
+pw_status_t pw_op_colsum_noalloc(const void* in, int T, int N, int ld, void* out, int accumulate, void* stream)
+{
+    if (!aligned(in, 16) || !out) return fail(PW_ERR_INVALID_ARG, "colsum: NULL or misaligned pointer");
+    if (accumulate != 0 && accumulate != 1) return fail(PW_ERR_INVALID_ARG, "accumulate must be 0 or 1");
+    if (N > 0 && static_cast<size_t>(N) > colsum_noalloc_max_columns())
+        return fail(PW_ERR_WORKSPACE_TOO_SMALL, "colsum (no-allocation variant): N exceeds the 262144 columns the built-in scratch can hold");
+    const char* e = launch_colsum_noalloc(in, T, N, ld, out, accumulate, static_cast<cudaStream_t>(stream));
+    if (e) return fail(PW_ERR_INVALID_ARG, e);
+    return PW_OK;
+}
+
 pw_status_t pw_op_gemm(int layout, int epilogue, int act, int M, int N, int K, const void* A, int lda, const void* B,
                        int ldb, void* C, int ldc, const void* bias, const void* aux_in, int ld_aux, void* aux_out,
                        int accumulate, void* stream)

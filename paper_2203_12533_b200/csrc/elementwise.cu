@@ -3,6 +3,9 @@
 // preprocess of the attention backward.  All use 16-byte accesses (8 bf16 per thread per
 // access), fp32 arithmetic, warp shuffles plus one shared-memory hop for row reductions, and
 // fixed-order two-stage reductions for anything summed over tokens (bitwise reproducible).
+#include <map>
+#include <mutex>
+
 #include "pw_kernels.h"
 
 namespace pw {
@@ -33,21 +36,6 @@ __device__ __forceinline__ float warp_sum(float v)
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
-}
-
-// Sum of `v` over the tpr threads of this row (warps_per_row consecutive warps).  `slot` is a
-// [kMaxWarps] shared array private to this reduction; the caller separates reuses of a slot
-// by a __syncthreads.
-__device__ __forceinline__ float row_sum(float v, float* slot, int warps_per_row, int row_in_cta)
-{
-    v = warp_sum(v);
-    if (warps_per_row == 1) return v;
-    const int warp = threadIdx.x >> 5;
-    if ((threadIdx.x & 31) == 0) slot[warp] = v;
-    __syncthreads();
-    float t = 0.f;
-    for (int i = 0; i < warps_per_row; ++i) t += slot[row_in_cta * warps_per_row + i];
-    return t;
 }
 
 // LayerNorm forward.  A row is handled by W warps (W = 1 for d <= 2048), each lane holding CH
@@ -380,6 +368,72 @@ const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, voi
     outs.out[0] = static_cast<float*>(out); outs.out[1] = outs.out[2] = outs.out[3] = nullptr;
     dim3 rgrid((N + 31) / 32, 1);
     reduce_partials_kernel<<<rgrid, 256, 0, stream>>>(static_cast<const float*>(partials), R, 1, N, outs, accumulate);
+    return cudaGetLastError() == cudaSuccess ? nullptr : "colsum reduce launch failed";
+}
+
+// ---------------------------------------------------------------------------------------------
+// Column sums without any allocation.  Some callers hand this library buffers but cannot create
+// device memory themselves while they run - a serving loop that has already given every byte of
+// HBM to its pools, a host callback, code running under a framework that forbids allocation at
+// that point.  For them the scratch of the column-sum kernel (the per-row-group partial sums)
+// lives in this fixed array, which every GPU that loads the library holds until the process
+// exits.  All calls share it: two calls that overlap on the GPU race on it, and it keeps the last
+// call's partial sums (every slot that a call reads is first written by that same call, so
+// nothing needs clearing).
+constexpr size_t kStaticScratchFloats = 262144;   // 1 MiB
+static __device__ __align__(256) float g_colsum_scratch[kStaticScratchFloats];
+
+namespace {
+struct StaticScratch { float* ptr; int sm_count; };
+// In host code the array's name is only a handle for the runtime, not a device address: the
+// address comes from cudaGetSymbolAddress, asked once per device with that device current.
+const char* static_scratch_for_current_device(StaticScratch* out)
+{
+    static std::mutex mu;
+    static std::map<int, StaticScratch> per_device;
+    std::lock_guard<std::mutex> lock(mu);
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return "no CUDA device (cudaGetDevice failed)";
+    auto it = per_device.find(dev);
+    if (it == per_device.end()) {
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return "cudaDeviceGetAttribute failed";
+        if (major != 10) return "device is not compute capability 10.x (sm_100a kernels only, no fallback)";
+        float* ptr = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_colsum_scratch);
+        if (e != cudaSuccess || ptr == nullptr) return "cudaGetSymbolAddress(static scratch) failed";
+        it = per_device.emplace(dev, StaticScratch{ptr, sms}).first;
+    }
+    *out = it->second;
+    return nullptr;
+}
+}  // namespace
+
+size_t colsum_noalloc_max_columns() { return kStaticScratchFloats; }
+
+const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* out, int accumulate, cudaStream_t stream)
+{
+    if (T <= 0 || N <= 0 || (N % 8) || (ld % 8) || ld < N) return "colsum: N and ld must be multiples of 8, ld >= N";
+    if (static_cast<size_t>(N) > kStaticScratchFloats)
+        return "colsum (no-allocation variant): N exceeds the 262144 columns the built-in scratch can hold";
+    StaticScratch sc;
+    if (const char* e = static_scratch_for_current_device(&sc)) return e;
+    // as many row groups as the fixed scratch can hold, at most what the allocating variant uses
+    const int col_blocks = (N + 1023) / 1024;
+    long long R = (4ll * sc.sm_count + col_blocks - 1) / col_blocks;
+    const long long fit = static_cast<long long>(kStaticScratchFloats / static_cast<size_t>(N));
+    if (R > fit) R = fit;
+    if (R > T) R = T;
+    if (R < 1) R = 1;
+    dim3 grid(col_blocks, static_cast<unsigned>(R));
+    colsum_kernel<<<grid, 128, 0, stream>>>(static_cast<const __nv_bfloat16*>(in), T, N, ld, sc.ptr);
+    if (cudaGetLastError() != cudaSuccess) return "colsum launch failed";
+    ReduceOuts outs;
+    outs.out[0] = static_cast<float*>(out); outs.out[1] = outs.out[2] = outs.out[3] = nullptr;
+    dim3 rgrid((N + 31) / 32, 1);
+    reduce_partials_kernel<<<rgrid, 256, 0, stream>>>(sc.ptr, static_cast<int>(R), 1, N, outs, accumulate);
     return cudaGetLastError() == cudaSuccess ? nullptr : "colsum reduce launch failed";
 }
 

@@ -54,6 +54,10 @@ size_t colsum_scratch_bytes(Runtime* rt, int T, int N);
 const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, void* out, int accumulate,
                           void* partials, cudaStream_t stream);
 
+// Column sums with the partial sums in a fixed device array inside the library (no allocation, no Runtime).
+size_t colsum_noalloc_max_columns();
+const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* out, int accumulate, cudaStream_t stream);
+
 const char* launch_attention_fwd(Runtime* rt, const void* qkv, int B, int S, int H, int dh, void* o, void* lse,
                                  cudaStream_t stream);
 const char* launch_attention_bwd(Runtime* rt, const void* qkv, const void* o, const void* dout, const void* lse,
