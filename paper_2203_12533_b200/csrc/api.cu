@@ -51,7 +51,7 @@ Runtime* get_runtime(const char** err)
         delete rt; *err = "cuTensorMapEncodeTiled not available from the driver"; return nullptr;
     }
     const char* ce;
-    if ((ce = configure_gemm()) || (ce = configure_attention())) { delete rt; *err = ce; return nullptr; }
+    if ((ce = configure_gemm()) || (ce = configure_attention()) || (ce = configure_attention_fwd())) { delete rt; *err = ce; return nullptr; }
     if (cudaMalloc(reinterpret_cast<void**>(&rt->op_status), sizeof(DeviceStatus)) != cudaSuccess ||
         cudaMemset(rt->op_status, 0, sizeof(DeviceStatus)) != cudaSuccess) {
         delete rt; *err = "could not allocate the status word"; return nullptr;
@@ -229,7 +229,7 @@ static pw_status_t do_attn_fwd(pw_layer_t* L, const void* qkv, void* o, void* ls
 {
     const LayerPlan& p = L->plan;
     LaunchScope sc(L, PW_K_ATTN_FWD, 1, 2.0 * p.T * (p.S + 1.0) * p.d, 0.0, st);
-    const char* e = launch_attention_fwd(L->rt, qkv, p.B, p.S, p.H, p.dh, o, lse, st);
+    const char* e = launch_attention_fwd(L->rt, qkv, p.B, p.S, p.H, p.dh, o, lse, L->status, st);
     return e ? fail(PW_ERR_CUDA, e) : PW_OK;
 }
 static pw_status_t do_attn_bwd(pw_layer_t* L, const void* qkv, const void* o, const void* dout, const void* lse,
@@ -790,7 +790,7 @@ pw_status_t pw_op_attention_fwd(const void* qkv, int B, int S, int H, int dh, vo
 {
     PW_RT_OR_FAIL();
     if (!aligned(qkv, 16) || !aligned(o, 16) || !lse) return fail(PW_ERR_INVALID_ARG, "attention: NULL or misaligned pointer");
-    PW_OP(launch_attention_fwd(rt, qkv, B, S, H, dh, o, lse, static_cast<cudaStream_t>(stream)));
+    PW_OP(launch_attention_fwd(rt, qkv, B, S, H, dh, o, lse, rt->op_status, static_cast<cudaStream_t>(stream)));
     return PW_OK;
 }
 

@@ -1,9 +1,7 @@
-// Fused causal attention, forward and backward, with online softmax (never materialises the
-// S x S score matrix).  Warp-level tensor-core path (mma.sync m16n8k16 bf16, fp32 accumulate),
-// cp.async double-buffered tiles in XOR-swizzled shared memory, ldmatrix operand fetch.
+// Causal attention backward (never materialises the S x S score matrix).  Warp-level
+// tensor-core path (mma.sync m16n8k16 bf16, fp32 accumulate), cp.async double-buffered tiles in
+// XOR-swizzled shared memory, ldmatrix operand fetch.  (The forward is in attention_fwd_sm100.cu.)
 //
-//   forward   : CTA = 128 queries of one (sequence, head), 8 warps x 16 query rows, key/value
-//               tiles of 64 up to the diagonal; writes o (bf16) and lse (fp32).
 //   backward  : delta = rowsum(dout * o); then two kernels so that every output is owned by one
 //               CTA (no atomics, bitwise reproducible):
 //                 dq   : CTA = 128 queries, loops over key/value tiles (S, dP, then dQ += dS K)
@@ -119,124 +117,6 @@ __device__ __forceinline__ void store_rows16(uint32_t tile_base, uint8_t* tile_p
         const int r = r0 + i / Tile<DH>::kChunks, ch = i % Tile<DH>::kChunks;
         const uint4 v = *reinterpret_cast<const uint4*>(tile_ptr + (Tile<DH>::addr(tile_base, r, ch * 8) - tile_base));
         *reinterpret_cast<uint4*>(g + static_cast<size_t>(r - r0) * ld + ch * 8) = v;
-    }
-}
-
-// ------------------------------------------------------------------------------------ forward
-template <int DH>
-__global__ void __launch_bounds__(kAttnThreads, 1)
-attn_fwd_kernel(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ o, float* __restrict__ lse,
-                int S, int H, float scale)
-{
-    extern __shared__ __align__(128) uint8_t smem[];
-    constexpr int QB = 128 * DH * 2, KB = 64 * DH * 2;
-    const uint32_t sQ = smem_u32(smem), sK = sQ + QB, sV = sK + 2 * KB;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int qblk = gridDim.x - 1 - blockIdx.x;            // longest rows first
-    const int b = blockIdx.y / H, h = blockIdx.y % H;
-    const int d = H * DH, ld = 3 * d;
-    const int q0 = qblk * 128;
-    const __nv_bfloat16* gq = qkv + static_cast<size_t>(b * S + q0) * ld + h * DH;
-    const __nv_bfloat16* gk = qkv + static_cast<size_t>(b * S) * ld + d + h * DH;
-    const __nv_bfloat16* gv = gk + d;
-    const int n_tiles = (q0 + 128) / 64;
-    const float sl2 = scale * kLog2e;
-
-    Tile<DH>::load(sQ, gq, ld, 128);
-    Tile<DH>::load(sK, gk, ld, 64);
-    Tile<DH>::load(sV, gv, ld, 64);
-    cp_async_commit();
-
-    uint32_t qf[DH / 16][4];
-    float oacc[DH / 8][4];
-#pragma unroll
-    for (int i = 0; i < DH / 8; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
-    float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
-    const int row_lo = q0 + warp * 16 + (lane >> 2), row_hi = row_lo + 8;
-
-    for (int t = 0; t < n_tiles; ++t) {
-        const int buf = t & 1;
-        if (t + 1 < n_tiles) {
-            Tile<DH>::load(sK + (buf ^ 1) * KB, gk + static_cast<size_t>(t + 1) * 64 * ld, ld, 64);
-            Tile<DH>::load(sV + (buf ^ 1) * KB, gv + static_cast<size_t>(t + 1) * 64 * ld, ld, 64);
-            cp_async_commit();
-            cp_async_wait<1>();
-        } else {
-            cp_async_wait<0>();
-        }
-        __syncthreads();
-        if (t == 0) {
-#pragma unroll
-            for (int ks = 0; ks < DH / 16; ++ks) load_a<DH>(sQ, warp * 16, ks * 16, qf[ks]);
-        }
-        const int kv0 = t * 64;
-        if (kv0 <= q0 + warp * 16 + 15) {                   // otherwise every key of the tile is masked for this warp
-            const uint32_t kb = sK + buf * KB, vb = sV + buf * KB;
-            float sacc[8][4];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f;
-#pragma unroll
-            for (int ks = 0; ks < DH / 16; ++ks) {
-#pragma unroll
-                for (int np = 0; np < 4; ++np) {
-                    uint32_t bb[4];
-                    load_b_nk<DH>(kb, np * 16, ks * 16, bb);
-                    mma16816(sacc[2 * np], qf[ks], bb[0], bb[1]);
-                    mma16816(sacc[2 * np + 1], qf[ks], bb[2], bb[3]);
-                }
-            }
-            if (kv0 + 63 > q0 + warp * 16) {                // tile crosses the diagonal for this warp
-#pragma unroll
-                for (int nb = 0; nb < 8; ++nb) {
-                    const int c = kv0 + nb * 8 + 2 * (lane & 3);
-                    if (c > row_lo) sacc[nb][0] = -INFINITY;
-                    if (c + 1 > row_lo) sacc[nb][1] = -INFINITY;
-                    if (c > row_hi) sacc[nb][2] = -INFINITY;
-                    if (c + 1 > row_hi) sacc[nb][3] = -INFINITY;
-                }
-            }
-            float mx_lo = -INFINITY, mx_hi = -INFINITY;
-#pragma unroll
-            for (int nb = 0; nb < 8; ++nb) {
-                mx_lo = fmaxf(mx_lo, fmaxf(sacc[nb][0], sacc[nb][1]));
-                mx_hi = fmaxf(mx_hi, fmaxf(sacc[nb][2], sacc[nb][3]));
-            }
-            const float mn_lo = fmaxf(m_lo, quad_max(mx_lo)), mn_hi = fmaxf(m_hi, quad_max(mx_hi));
-            const float a_lo = exp2f((m_lo - mn_lo) * sl2), a_hi = exp2f((m_hi - mn_hi) * sl2);
-            m_lo = mn_lo; m_hi = mn_hi;
-            float s_lo = 0.f, s_hi = 0.f;
-            uint32_t pf[4][4];
-#pragma unroll
-            for (int nb = 0; nb < 8; ++nb) {
-                const float p0 = exp2f((sacc[nb][0] - mn_lo) * sl2), p1 = exp2f((sacc[nb][1] - mn_lo) * sl2);
-                const float p2 = exp2f((sacc[nb][2] - mn_hi) * sl2), p3 = exp2f((sacc[nb][3] - mn_hi) * sl2);
-                s_lo += p0 + p1; s_hi += p2 + p3;
-                pf[nb >> 1][(nb & 1) * 2] = pack_bf16(p0, p1);
-                pf[nb >> 1][(nb & 1) * 2 + 1] = pack_bf16(p2, p3);
-            }
-            l_lo = l_lo * a_lo + quad_sum(s_lo);
-            l_hi = l_hi * a_hi + quad_sum(s_hi);
-#pragma unroll
-            for (int i = 0; i < DH / 8; ++i) { oacc[i][0] *= a_lo; oacc[i][1] *= a_lo; oacc[i][2] *= a_hi; oacc[i][3] *= a_hi; }
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-#pragma unroll
-                for (int np = 0; np < DH / 16; ++np) {
-                    uint32_t bb[4];
-                    load_b_kn<DH>(vb, ks * 16, np * 16, bb);
-                    mma16816(oacc[2 * np], pf[ks], bb[0], bb[1]);
-                    mma16816(oacc[2 * np + 1], pf[ks], bb[2], bb[3]);
-                }
-            }
-        }
-        __syncthreads();
-    }
-    store_rows16<DH>(sQ, smem, warp * 16, oacc, 1.f / l_lo, 1.f / l_hi,
-                     o + static_cast<size_t>(b * S + q0 + warp * 16) * d + h * DH, d);
-    if ((lane & 3) == 0) {
-        float* L = lse + (static_cast<size_t>(b) * H + h) * S;
-        L[row_lo] = m_lo * scale + logf(l_lo);
-        L[row_hi] = m_hi * scale + logf(l_hi);
     }
 }
 
@@ -506,7 +386,6 @@ const char* set_smem(K kern, int bytes)
                ? nullptr : "cudaFuncSetAttribute(attention) failed";
 }
 
-constexpr int fwd_smem(int dh) { return 128 * dh * 2 + 4 * 64 * dh * 2; }
 constexpr int dq_smem(int dh) { return 2 * 128 * dh * 2 + 4 * 64 * dh * 2; }
 constexpr int dkdv_smem(int dh) { return 2 * 128 * dh * 2 + 4 * 64 * dh * 2 + 4 * 64 * 4; }
 
@@ -515,32 +394,11 @@ constexpr int dkdv_smem(int dh) { return 2 * 128 * dh * 2 + 4 * 64 * dh * 2 + 4 
 const char* configure_attention()
 {
     const char* e;
-    if ((e = set_smem(attn_fwd_kernel<64>, fwd_smem(64)))) return e;
-    if ((e = set_smem(attn_fwd_kernel<128>, fwd_smem(128)))) return e;
     if ((e = set_smem(attn_bwd_dq_kernel<64>, dq_smem(64)))) return e;
     if ((e = set_smem(attn_bwd_dq_kernel<128>, dq_smem(128)))) return e;
     if ((e = set_smem(attn_bwd_dkdv_kernel<64>, dkdv_smem(64)))) return e;
     if ((e = set_smem(attn_bwd_dkdv_kernel<128>, dkdv_smem(128)))) return e;
     return nullptr;
-}
-
-const char* launch_attention_fwd(Runtime* rt, const void* qkv, int B, int S, int H, int dh, void* o, void* lse,
-                                 cudaStream_t stream)
-{
-    (void)rt;
-    if (B <= 0 || H <= 0 || S <= 0 || (S % 128) != 0 || (dh != 64 && dh != 128)) return "attention: unsupported shape";
-    const float scale = 1.0f / sqrtf(static_cast<float>(dh));
-    dim3 grid(S / 128, B * H);
-    const int smem = fwd_smem(dh);
-    auto Q = static_cast<const __nv_bfloat16*>(qkv);
-    auto O = static_cast<__nv_bfloat16*>(o);
-    auto L = static_cast<float*>(lse);
-    if (dh == 64) {
-        attn_fwd_kernel<64><<<grid, kAttnThreads, smem, stream>>>(Q, O, L, S, H, scale);
-    } else {
-        attn_fwd_kernel<128><<<grid, kAttnThreads, smem, stream>>>(Q, O, L, S, H, scale);
-    }
-    return cudaGetLastError() == cudaSuccess ? nullptr : "attention fwd launch failed";
 }
 
 const char* launch_attention_bwd(Runtime* rt, const void* qkv, const void* o, const void* dout, const void* lse,

@@ -25,6 +25,7 @@ Runtime* get_runtime(const char** err);
 // One-time kernel attribute set-up (dynamic shared-memory opt-in); called from get_runtime.
 const char* configure_gemm();
 const char* configure_attention();
+const char* configure_attention_fwd();
 
 enum GemmLayout { kTN = 0, kNN = 1, kNT = 2 };
 enum GemmEpi { kEpiNone = 0, kEpiBias = 1, kEpiBiasResid = 2, kEpiBiasGelu = 3, kEpiDGelu = 4, kEpiF32 = 5 };
@@ -59,7 +60,7 @@ size_t colsum_noalloc_max_columns();
 const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* out, int accumulate, cudaStream_t stream);
 
 const char* launch_attention_fwd(Runtime* rt, const void* qkv, int B, int S, int H, int dh, void* o, void* lse,
-                                 cudaStream_t stream);
+                                 DeviceStatus* status, cudaStream_t stream);
 const char* launch_attention_bwd(Runtime* rt, const void* qkv, const void* o, const void* dout, const void* lse,
                                  int B, int S, int H, int dh, void* dqkv, void* delta, cudaStream_t stream);
 
