@@ -237,7 +237,7 @@ static pw_status_t do_attn_bwd(pw_layer_t* L, const void* qkv, const void* o, co
 {
     const LayerPlan& p = L->plan;
     LaunchScope sc(L, PW_K_ATTN_BWD, 3, 5.0 * p.T * (p.S + 1.0) * p.d, 0.0, st);
-    const char* e = launch_attention_bwd(L->rt, qkv, o, dout, lse, p.B, p.S, p.H, p.dh, dqkv, delta, st);
+    const char* e = launch_attention_bwd(L->rt, qkv, o, dout, lse, p.B, p.S, p.H, p.dh, dqkv, delta, L->status, st);
     return e ? fail(PW_ERR_CUDA, e) : PW_OK;
 }
 
@@ -800,7 +800,7 @@ pw_status_t pw_op_attention_bwd(const void* qkv, const void* o, const void* dout
     PW_RT_OR_FAIL();
     if (!aligned(qkv, 16) || !aligned(o, 16) || !aligned(dout, 16) || !lse || !aligned(dqkv, 16) || !delta)
         return fail(PW_ERR_INVALID_ARG, "attention bwd: NULL or misaligned pointer");
-    PW_OP(launch_attention_bwd(rt, qkv, o, dout, lse, B, S, H, dh, dqkv, delta, static_cast<cudaStream_t>(stream)));
+    PW_OP(launch_attention_bwd(rt, qkv, o, dout, lse, B, S, H, dh, dqkv, delta, rt->op_status, static_cast<cudaStream_t>(stream)));
     return PW_OK;
 }
 

@@ -186,18 +186,19 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
             if (!ok) break;
             tc_fence_after();
             const bool diag = j == n_t - 1;
-            // pass 1: row maximum of the visible scores
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t v[32];
-                tmem_ld32(s_addr + c * 32, v);
-                tc_wait_ld();
+            // all 128 scores of the row in registers (four loads in flight, one wait)
+            uint32_t v[128];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float sv = __uint_as_float(v[i]);
-                    if (!diag || c * 32 + i <= r) mx = fmaxf(mx, sv);
-                }
+            for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, v + c * 32);
+            tc_wait_ld();
+            float mx = -INFINITY;
+            if (diag) {
+#pragma unroll
+                for (int i = 0; i < 128; ++i)
+                    if (i <= r) mx = fmaxf(mx, __uint_as_float(v[i]));
+            } else {
+#pragma unroll
+                for (int i = 0; i < 128; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
             }
             const float m_new = fmaxf(m_used, mx);
             const bool grow = (m_new - m_used) * sl2 > 8.0f;        // also true on the first tile (m_used = -inf)
@@ -209,34 +210,31 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                 l *= alpha;
 #pragma unroll 1
                 for (int c = 0; c < DH / 32; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(o_addr + c * 32, v);
+                    uint32_t w[32];
+                    tmem_ld32(o_addr + c * 32, w);
                     tc_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-                    tmem_st32(o_addr + c * 32, v);
+                    for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(__uint_as_float(w[i]) * alpha);
+                    tmem_st32(o_addr + c * 32, w);
                 }
             }
-            // pass 2: p = exp2((s - m) * scale * log2e), packed bf16 written over the S columns
+            // p = exp2((s - m) * scale * log2e), packed bf16 written over the S columns
             const float mb = m_used * sl2;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t v[32], pk[16];
-                tmem_ld32(s_addr + c * 32, v);
-                tc_wait_ld();
+            float ls = 0.f;
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    float p0 = ex2_approx(fmaf(__uint_as_float(v[i]), sl2, -mb));
-                    float p1 = ex2_approx(fmaf(__uint_as_float(v[i + 1]), sl2, -mb));
-                    if (diag) {
-                        if (c * 32 + i > r) p0 = 0.f;
-                        if (c * 32 + i + 1 > r) p1 = 0.f;
-                    }
-                    l += p0 + p1;
-                    pk[i >> 1] = pack_bf16(p0, p1);
+            for (int i = 0; i < 128; i += 2) {
+                float p0 = ex2_approx(fmaf(__uint_as_float(v[i]), sl2, -mb));
+                float p1 = ex2_approx(fmaf(__uint_as_float(v[i + 1]), sl2, -mb));
+                if (diag) {
+                    if (i > r) p0 = 0.f;
+                    if (i + 1 > r) p1 = 0.f;
                 }
-                tmem_st16(s_addr + c * 16, pk);
+                ls += p0 + p1;
+                v[i >> 1] = pack_bf16(p0, p1);
             }
+            l += ls;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_st16(s_addr + c * 16, v + c * 16);
             tc_wait_st();
             tc_fence_before();
             mbar_arrive(bar(11 + t));

@@ -62,6 +62,7 @@ const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* ou
 const char* launch_attention_fwd(Runtime* rt, const void* qkv, int B, int S, int H, int dh, void* o, void* lse,
                                  DeviceStatus* status, cudaStream_t stream);
 const char* launch_attention_bwd(Runtime* rt, const void* qkv, const void* o, const void* dout, const void* lse,
-                                 int B, int S, int H, int dh, void* dqkv, void* delta, cudaStream_t stream);
+                                 int B, int S, int H, int dh, void* dqkv, void* delta, DeviceStatus* status,
+                                 cudaStream_t stream);
 
 }  // namespace pw
