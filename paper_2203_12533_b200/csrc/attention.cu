@@ -13,26 +13,38 @@ const char* configure_attention_bwd_tc();
 namespace {
 
 // ------------------------------------------------------------------------------------ delta = rowsum(dout * o)
-__global__ void attn_delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ dout,
-                                  float* __restrict__ delta, int B, int S, int H, int dh)
+// Each thread handles four 16-byte pieces that are a whole block stride apart (all eight loads
+// are issued before any is used); the dh/8 threads of a (token, head) group reduce by shuffles.
+__global__ void __launch_bounds__(256)
+attn_delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ dout,
+                  float* __restrict__ delta, int B, int S, int H, int dh)
 {
     const int per_head = dh / 8;                             // threads per (token, head): 8 or 16
-    const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     const size_t total = static_cast<size_t>(B) * S * H * per_head;
-    float s = 0.f;
-    if (idx < total) {
-        float a[8], g[8];
-        unpack8(*reinterpret_cast<const uint4*>(o + idx * 8), a);
-        unpack8(*reinterpret_cast<const uint4*>(dout + idx * 8), g);
+    const size_t base = static_cast<size_t>(blockIdx.x) * 1024 + threadIdx.x;
+    uint4 a[4], g[4];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) s += a[k] * g[k];
+    for (int u = 0; u < 4; ++u) {
+        const size_t idx = base + u * 256;
+        a[u] = idx < total ? *reinterpret_cast<const uint4*>(o + idx * 8) : make_uint4(0, 0, 0, 0);
+        g[u] = idx < total ? *reinterpret_cast<const uint4*>(dout + idx * 8) : make_uint4(0, 0, 0, 0);
     }
-    for (int off = per_head >> 1; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-    if (idx < total && (idx % per_head) == 0) {
-        const size_t th = idx / per_head;                    // token * H + head
-        const size_t t = th / H, h = th % H;
-        const size_t b = t / S, sq = t % S;
-        delta[(b * H + h) * S + sq] = s;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const size_t idx = base + u * 256;
+        float fa[8], fg[8];
+        unpack8(a[u], fa);
+        unpack8(g[u], fg);
+        float s = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) s += fa[k] * fg[k];
+        for (int off = per_head >> 1; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+        if (idx < total && (idx % per_head) == 0) {
+            const size_t th = idx / per_head;                // token * H + head
+            const size_t t = th / H, h = th % H;
+            const size_t bb = t / S, sq = t % S;
+            delta[(bb * H + h) * S + sq] = s;
+        }
     }
 }
 
@@ -47,7 +59,7 @@ const char* launch_attention_bwd(Runtime* rt, const void* qkv, const void* o, co
     if (B <= 0 || H <= 0 || S <= 0 || (S % 128) != 0 || (dh != 64 && dh != 128)) return "attention: unsupported shape";
     {
         const size_t total = static_cast<size_t>(B) * S * H * (dh / 8);
-        attn_delta_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, stream>>>(
+        attn_delta_kernel<<<static_cast<unsigned>((total + 1023) / 1024), 256, 0, stream>>>(
             static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(dout), static_cast<float*>(delta), B, S, H, dh);
         if (cudaGetLastError() != cudaSuccess) return "attention delta launch failed";
     }

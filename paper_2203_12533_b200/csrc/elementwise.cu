@@ -115,7 +115,7 @@ bool plan_warp_rows(int d, int* W, int* CH)
 // The next row's three inputs are fetched before the current row's reduction, and the two row
 // sums share one barrier.
 template <int CHUNKS>
-__global__ void __launch_bounds__(kRowThreadsMax)
+__global__ void __launch_bounds__(kRowThreadsMax, CHUNKS == 1 ? 2 : 1)
 ln_bwd_kernel(const __nv_bfloat16* __restrict__ dh, const __nv_bfloat16* __restrict__ x,
               const float* __restrict__ mu, const float* __restrict__ rstd, const __nv_bfloat16* __restrict__ gamma,
               const __nv_bfloat16* resid, int T, int d, __nv_bfloat16* dx,
@@ -214,47 +214,51 @@ ln_bwd_kernel(const __nv_bfloat16* __restrict__ dh, const __nv_bfloat16* __restr
     }
 }
 
-// out_q[c] (+)= sum over partial rows of partials[row][q][c].  CTA = 32 columns x 8 row lanes:
-// row lane y adds rows y, y+8, ... in order, then the 8 lane sums are added in order, so the
+// out_q[c] (+)= sum over partial rows of partials[row][q][c].  CTA = 32 columns x 32 row lanes:
+// row lane y adds rows y, y+32, ... in order, then the 32 lane sums are added in order, so the
 // result does not depend on scheduling.  Up to 4 outputs (grid.y = quantity).
 struct ReduceOuts { float* out[4]; };
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 reduce_partials_kernel(const float* __restrict__ partials, int nrows, int nq, int n, ReduceOuts outs, int accumulate)
 {
-    __shared__ float sm[8][33];
+    __shared__ float sm[32][33];
     const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
     const int c = blockIdx.x * 32 + cx;
     const int q = blockIdx.y;
     float* out = outs.out[q];
     if (out == nullptr) return;
     float s = 0.f;
-    if (c < n)
-        for (int r = ry; r < nrows; r += 8) s += partials[(static_cast<size_t>(r) * nq + q) * n + c];
+    if (c < n) {
+#pragma unroll 4
+        for (int r = ry; r < nrows; r += 32) s += partials[(static_cast<size_t>(r) * nq + q) * n + c];
+    }
     sm[ry][cx] = s;
     __syncthreads();
     if (ry == 0 && c < n) {
         float t = 0.f;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) t += sm[i][cx];
+        for (int i = 0; i < 32; ++i) t += sm[i][cx];
         out[c] = accumulate ? out[c] + t : t;
     }
 }
 
-// Column sums of a bf16 [T, N] matrix: CTA (x, y) owns columns 1024*x .. +1023 and rows y, y+R, ...
-__global__ void __launch_bounds__(128)
+// Column sums of a bf16 [T, N] matrix: CTA (x, y) owns columns 2048*x .. +2047 and rows y, y+R, ...;
+// eight rows are in flight per thread.
+constexpr int kColsumCols = 2048;
+__global__ void __launch_bounds__(256)
 colsum_kernel(const __nv_bfloat16* __restrict__ in, int T, int N, int ld, float* __restrict__ partials)
 {
-    const int col = blockIdx.x * 1024 + threadIdx.x * 8;
+    const int col = blockIdx.x * kColsumCols + threadIdx.x * 8;
     if (col >= N) return;
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     const int R = gridDim.y;
     int t = blockIdx.y;
-    for (; t + 3 * R < T; t += 4 * R) {
-        uint4 v[4];
+    for (; t + 7 * R < T; t += 8 * R) {
+        uint4 v[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const uint4*>(in + static_cast<size_t>(t + u * R) * ld + col);
+        for (int u = 0; u < 8; ++u) v[u] = *reinterpret_cast<const uint4*>(in + static_cast<size_t>(t + u * R) * ld + col);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < 8; ++u) {
             float f[8];
             unpack8(v[u], f);
 #pragma unroll
@@ -274,7 +278,7 @@ colsum_kernel(const __nv_bfloat16* __restrict__ in, int T, int N, int ld, float*
 
 int colsum_splits(Runtime* rt, int T, int N)
 {
-    const int col_blocks = (N + 1023) / 1024;
+    const int col_blocks = (N + kColsumCols - 1) / kColsumCols;
     int r = (4 * rt->sm_count + col_blocks - 1) / col_blocks;
     if (r > T) r = T;
     if (r < 1) r = 1;
@@ -284,7 +288,7 @@ int colsum_splits(Runtime* rt, int T, int N)
 int ln_bwd_grid(Runtime* rt, int T, const RowPlan& rp)
 {
     const int row_groups = (T + rp.rows_per_cta - 1) / rp.rows_per_cta;
-    const int cap = rt->sm_count;
+    const int cap = (rp.chunks == 1 ? 2 : 1) * rt->sm_count;
     return row_groups < cap ? row_groups : cap;
 }
 
@@ -346,7 +350,7 @@ const char* launch_layernorm_bwd(Runtime* rt, const void* dh, const void* x, con
     outs.out[0] = static_cast<float*>(dgamma); outs.out[1] = static_cast<float*>(dbeta);
     outs.out[2] = static_cast<float*>(db_resid); outs.out[3] = static_cast<float*>(db_dx);
     dim3 rgrid((d + 31) / 32, 4);
-    reduce_partials_kernel<<<rgrid, 256, 0, stream>>>(P, grid * rp.rows_per_cta, 4, d, outs, accumulate);
+    reduce_partials_kernel<<<rgrid, 1024, 0, stream>>>(P, grid * rp.rows_per_cta, 4, d, outs, accumulate);
     return cudaGetLastError() == cudaSuccess ? nullptr : "layernorm bwd reduce launch failed";
 }
 
@@ -361,13 +365,13 @@ const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, voi
 {
     if (T <= 0 || N <= 0 || (N % 8) || (ld % 8)) return "colsum: N and ld must be multiples of 8";
     const int R = colsum_splits(rt, T, N);
-    dim3 grid((N + 1023) / 1024, R);
-    colsum_kernel<<<grid, 128, 0, stream>>>(static_cast<const __nv_bfloat16*>(in), T, N, ld, static_cast<float*>(partials));
+    dim3 grid((N + kColsumCols - 1) / kColsumCols, R);
+    colsum_kernel<<<grid, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(in), T, N, ld, static_cast<float*>(partials));
     if (cudaGetLastError() != cudaSuccess) return "colsum launch failed";
     ReduceOuts outs;
     outs.out[0] = static_cast<float*>(out); outs.out[1] = outs.out[2] = outs.out[3] = nullptr;
     dim3 rgrid((N + 31) / 32, 1);
-    reduce_partials_kernel<<<rgrid, 256, 0, stream>>>(static_cast<const float*>(partials), R, 1, N, outs, accumulate);
+    reduce_partials_kernel<<<rgrid, 1024, 0, stream>>>(static_cast<const float*>(partials), R, 1, N, outs, accumulate);
     return cudaGetLastError() == cudaSuccess ? nullptr : "colsum reduce launch failed";
 }
 
@@ -421,19 +425,19 @@ const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* ou
     StaticScratch sc;
     if (const char* e = static_scratch_for_current_device(&sc)) return e;
     // as many row groups as the fixed scratch can hold, at most what the allocating variant uses
-    const int col_blocks = (N + 1023) / 1024;
+    const int col_blocks = (N + kColsumCols - 1) / kColsumCols;
     long long R = (4ll * sc.sm_count + col_blocks - 1) / col_blocks;
     const long long fit = static_cast<long long>(kStaticScratchFloats / static_cast<size_t>(N));
     if (R > fit) R = fit;
     if (R > T) R = T;
     if (R < 1) R = 1;
     dim3 grid(col_blocks, static_cast<unsigned>(R));
-    colsum_kernel<<<grid, 128, 0, stream>>>(static_cast<const __nv_bfloat16*>(in), T, N, ld, sc.ptr);
+    colsum_kernel<<<grid, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(in), T, N, ld, sc.ptr);
     if (cudaGetLastError() != cudaSuccess) return "colsum launch failed";
     ReduceOuts outs;
     outs.out[0] = static_cast<float*>(out); outs.out[1] = outs.out[2] = outs.out[3] = nullptr;
     dim3 rgrid((N + 31) / 32, 1);
-    reduce_partials_kernel<<<rgrid, 256, 0, stream>>>(sc.ptr, static_cast<int>(R), 1, N, outs, accumulate);
+    reduce_partials_kernel<<<rgrid, 1024, 0, stream>>>(sc.ptr, static_cast<int>(R), 1, N, outs, accumulate);
     return cudaGetLastError() == cudaSuccess ? nullptr : "colsum reduce launch failed";
 }
 
