@@ -36,8 +36,26 @@ struct GemmParams {
     const __nv_bfloat16* aux_in; int ld_aux;
     int accumulate, act;
     int m_tiles, n_tiles;
+    int split_begin;             // tiles >= split_begin are issued as two half-width tiles (tail balancing)
+    int total_virtual;           // split_begin + 2 * (m_tiles*n_tiles - split_begin)
     DeviceStatus* status;
 };
+
+// Virtual tile v -> (m0, n0, width).  Full tiles are numbered m-fastest; the tiles of the last,
+// partly filled round are cut in two half-width tiles so that every SM gets one.
+__device__ __forceinline__ void tile_info(const GemmParams& p, int v, int& m0, int& n0, int& bn)
+{
+    int t = v, half = 0;
+    bn = p.bn;
+    if (v >= p.split_begin) {
+        const int hv = v - p.split_begin;
+        t = p.split_begin + (hv >> 1);
+        half = hv & 1;
+        bn = p.bn >> 1;
+    }
+    m0 = (t % p.m_tiles) * BM;
+    n0 = (t / p.m_tiles) * p.bn + half * (p.bn >> 1);
+}
 
 // One 8-column group of the bf16 epilogues: f = acc (+bias) (+residual | x GeLU'(u)).
 template <int EPI>
@@ -71,9 +89,91 @@ __device__ __forceinline__ void epilogue_group(const uint32_t* v, int row, int c
     }
 }
 
+// Epilogue of one accumulator tile for one warp: TMEM -> registers -> swizzled shared slab -> TMA
+// store (rows >= M and columns >= N are clipped by the tensor map).  `taddr` addresses this warp's
+// lane quarter of the accumulator, row0 is the first of its 32 rows, pi selects which of the two
+// warps of the quarter it is (they take alternate column chunks).
+template <int EPI>
+__device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, int bn, int pi, int lane, uint8_t* slab,
+                                              uint32_t slab_u32, uint32_t& nout, const CUtensorMap* tmC,
+                                              const CUtensorMap* tmAux, const GemmParams& p)
+{
+    const int row = row0 + lane;
+    uint8_t* my_row = slab + lane * 128;
+    if constexpr (EPI == kEpiF32) {
+        const int nsteps = bn / 32;
+#pragma unroll 1
+        for (int s = pi; s < nsteps; s += 2) {
+            const int col0 = n0 + s * 32;
+            if (col0 >= p.N) break;
+            uint32_t v[32];
+            tmem_ld32(taddr + s * 32, v);
+            tc_wait_ld();
+            if (lane == 0) bulk_wait_read0();
+            __syncwarp();
+#pragma unroll
+            for (int g = 0; g < 8; ++g)
+                *reinterpret_cast<uint4*>(my_row + ((g ^ (lane & 7)) << 4)) =
+                    make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+                if (p.accumulate) tma_reduce_add_2d(tmC, slab_u32, col0, row0);
+                else tma_store_2d(tmC, slab_u32, col0, row0);
+                bulk_commit();
+            }
+        }
+    } else {
+        // 32 columns per chunk; the slab is two 2 KB halves (32 rows x 64 bytes, 64-byte
+        // swizzle) used alternately, so one store is always in flight behind the math.
+        const int nchunks = bn / 32;
+        const uint32_t sw = (lane >> 1) & 3;
+#pragma unroll 1
+        for (int ch = pi; ch < nchunks; ch += 2) {
+            const int col0 = n0 + ch * 32;
+            if (col0 >= p.N) break;
+            uint32_t v[32];
+            tmem_ld32(taddr + ch * 32, v);
+            tc_wait_ld();
+            uint4 o[4], o2[4];
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                float f[8];
+                epilogue_group<EPI>(v + 8 * g, row, col0 + g * 8, p, f);
+                o[g] = pack8(f);
+                if constexpr (EPI == kEpiBiasGelu) {
+                    // GeLU of the bf16 value stored as u: the backward reads u back and sees
+                    // exactly the argument the forward used
+                    unpack8(o[g], f);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) f[j] = gelu_f(f[j], p.act);
+                    o2[g] = pack8(f);
+                }
+            }
+            constexpr int kOuts = (EPI == kEpiBiasGelu) ? 2 : 1;
+#pragma unroll
+            for (int t = 0; t < kOuts; ++t) {
+                const uint32_t half = (nout++ & 1u) * 2048u;
+                if (lane == 0) bulk_wait_read1();
+                __syncwarp();
+#pragma unroll
+                for (int g = 0; g < 4; ++g)
+                    *reinterpret_cast<uint4*>(slab + half + lane * 64 + ((g ^ sw) << 4)) = (t == 0) ? o[g] : o2[g];
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(t == 0 ? tmC : tmAux, slab_u32 + half, col0, row0);
+                    bulk_commit();
+                }
+            }
+        }
+    }
+}
+
 template <bool A_MN, bool B_MN, int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const __grid_constant__ CUtensorMap tmBh /* B with a half-width box */,
             const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmAux, const GemmParams p)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -87,8 +187,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_k = (p.K + BK - 1) / BK;
-    const int total_tiles = p.m_tiles * p.n_tiles;
-    const int bn = p.bn;
+    const int total_tiles = p.total_virtual;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
@@ -113,9 +212,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            const uint32_t stage_tx = A_TILE_BYTES + bn * BK * 2;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile % p.m_tiles) * BM, n0 = (tile / p.m_tiles) * bn;
+                int m0, n0, bn;
+                tile_info(p, tile, m0, n0, bn);
+                const uint32_t stage_tx = A_TILE_BYTES + bn * BK * 2;
+                const CUtensorMap* mapB = bn == p.bn ? &tmB : &tmBh;
                 for (int kb = 0; kb < num_k; ++kb) {
                     if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 100)) { ok = false; break; }
                     const uint32_t fb = full0 + 8 * stage;
@@ -128,7 +229,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         for (int j = 0; j < BM / 64; ++j) tma_load_2d(a_dst + j * 8192, &tmA, m0 + 64 * j, kb * BK, fb);
                     }
                     if constexpr (!B_MN) {
-                        tma_load_2d(b_dst, &tmB, kb * BK, n0, fb);
+                        tma_load_2d(b_dst, mapB, kb * BK, n0, fb);
                     } else {
                         for (int j = 0; j < bn / 64; ++j) tma_load_2d(b_dst + j * 8192, &tmB, n0 + 64 * j, kb * BK, fb);
                     }
@@ -138,10 +239,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = make_idesc_bf16(BM, bn, A_MN, B_MN);
+            const uint32_t idesc_full = make_idesc_bf16(BM, p.bn, A_MN, B_MN);
+            const uint32_t idesc_half = make_idesc_bf16(BM, p.bn >> 1, A_MN, B_MN);
             uint32_t stage = 0, phase = 0, it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+                const uint32_t idesc = tile >= p.split_begin ? idesc_half : idesc_full;
                 const uint32_t buf = it & 1, acc_phase = (it >> 1) & 1;
                 if (!mbar_wait(acce0 + 8 * buf, acc_phase ^ 1, abort_flag, p.status, 200)) break;
                 tc_fence_after();
@@ -173,85 +276,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int q = warp & 3, pi = (warp - 2) >> 2;
         uint8_t* slab = slabs + (warp - 2) * SLAB_BYTES;
         const uint32_t slab_u32 = smem_u32(slab);
-        uint8_t* my_row = slab + lane * 128;
         uint32_t it = 0, nout = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
-            const int m0 = (tile % p.m_tiles) * BM, n0 = (tile / p.m_tiles) * bn;
+            int m0, n0, bn;
+            tile_info(p, tile, m0, n0, bn);
             const uint32_t buf = it & 1, acc_phase = (it >> 1) & 1;
             bool ok = mbar_wait(accf0 + 8 * buf, acc_phase, abort_flag, p.status, 300);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const int row = m0 + q * 32 + lane;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * BN_MAX;
-            if constexpr (EPI == kEpiF32) {
-                const int nsteps = bn / 32;
-#pragma unroll 1
-                for (int s = pi; s < nsteps; s += 2) {
-                    const int col0 = n0 + s * 32;
-                    if (col0 >= p.N) break;
-                    uint32_t v[32];
-                    tmem_ld32(taddr + s * 32, v);
-                    tc_wait_ld();
-                    if (lane == 0) bulk_wait_read0();
-                    __syncwarp();
-#pragma unroll
-                    for (int g = 0; g < 8; ++g)
-                        *reinterpret_cast<uint4*>(my_row + ((g ^ (lane & 7)) << 4)) =
-                            make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-                    fence_proxy_async();
-                    __syncwarp();
-                    if (lane == 0) {
-                        if (p.accumulate) tma_reduce_add_2d(&tmC, slab_u32, col0, m0 + q * 32);
-                        else tma_store_2d(&tmC, slab_u32, col0, m0 + q * 32);
-                        bulk_commit();
-                    }
-                }
-            } else {
-                // 32 columns per chunk; the slab is two 2 KB halves (32 rows x 64 bytes, 64-byte
-                // swizzle) used alternately, so one store is always in flight behind the math.
-                const int nchunks = bn / 32;
-                const uint32_t sw = (lane >> 1) & 3;
-#pragma unroll 1
-                for (int ch = pi; ch < nchunks; ch += 2) {
-                    const int col0 = n0 + ch * 32;
-                    if (col0 >= p.N) break;
-                    uint32_t v[32];
-                    tmem_ld32(taddr + ch * 32, v);
-                    tc_wait_ld();
-                    uint4 o[4], o2[4];
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        float f[8];
-                        epilogue_group<EPI>(v + 8 * g, row, col0 + g * 8, p, f);
-                        o[g] = pack8(f);
-                        if constexpr (EPI == kEpiBiasGelu) {
-                            // GeLU of the bf16 value stored as u: the backward reads u back and sees
-                            // exactly the argument the forward used
-                            unpack8(o[g], f);
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) f[j] = gelu_f(f[j], p.act);
-                            o2[g] = pack8(f);
-                        }
-                    }
-                    constexpr int kOuts = (EPI == kEpiBiasGelu) ? 2 : 1;
-#pragma unroll
-                    for (int t = 0; t < kOuts; ++t) {
-                        const uint32_t half = (nout++ & 1u) * 2048u;
-                        if (lane == 0) bulk_wait_read1();
-                        __syncwarp();
-#pragma unroll
-                        for (int g = 0; g < 4; ++g)
-                            *reinterpret_cast<uint4*>(slab + half + lane * 64 + ((g ^ sw) << 4)) = (t == 0) ? o[g] : o2[g];
-                        fence_proxy_async();
-                        __syncwarp();
-                        if (lane == 0) {
-                            tma_store_2d(t == 0 ? &tmC : &tmAux, slab_u32 + half, col0, m0 + q * 32);
-                            bulk_commit();
-                        }
-                    }
-                }
-            }
+            epilogue_tile<EPI>(taddr, m0 + q * 32, n0, bn, pi, lane, slab, slab_u32, nout, &tmC, &tmAux, p);
             tc_fence_before();
             mbar_arrive(acce0 + 8 * buf);
         }
@@ -268,6 +303,152 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// CTA-pair variant (cta_group::2): a cluster of two CTAs computes one 256 x bn tile.  CTA r of the
+// pair loads its own 128 rows of A and its own half (bn/2 rows) of B - with plain per-CTA TMA loads
+// whose bytes are credited to the leader's "full" barrier - and the leader CTA issues one M = 256
+// MMA that reads both CTAs' shared memory and writes each CTA's 128 x bn accumulator into that
+// CTA's own TMEM.  Per FLOP this moves a third less data into shared memory than the one-CTA tile
+// and makes 128-wide tiles affordable, which removes most of the wave-quantisation loss on the
+// N = d_model GEMMs.  Barriers: full[s] (leader, 1 arrival + both CTAs' bytes), empty[s] and
+// acc_full[b] (one in each CTA, signalled by the leader's tcgen05.commit to both), acc_empty[b]
+// (leader, one arrival per epilogue warp of both CTAs).
+constexpr int P_STAGES = 6;
+constexpr int P_STAGE_BYTES = 32768;            // A: 128 x 64 (16 KB) + B half: up to 128 x 64 (16 KB)
+constexpr int P_SMEM_BYTES = P_STAGES * P_STAGE_BYTES + EPI_WARPS * SLAB_BYTES + 1024 + 256;
+
+template <bool A_MN, bool B_MN, int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmAux, const GemmParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* slabs = tiles + P_STAGES * P_STAGE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(slabs + EPI_WARPS * SLAB_BYTES);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + P_STAGES);
+    const uint32_t accf0 = smem_u32(bars + 2 * P_STAGES), acce0 = smem_u32(bars + 2 * P_STAGES + 2);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * P_STAGES + 4);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();            // 0 = leader
+    const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const int num_k = (p.K + BK - 1) / BK;
+    const int total_tiles = p.m_tiles * p.n_tiles;      // pair tiles: m_tiles counts 256-row blocks
+    const int bn = p.bn, half_n = bn >> 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < P_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 2 * EPI_WARPS); }
+        *abort_flag = 0;
+        fence_barrier_init();
+        fence_proxy_async();
+        prefetch_tmap(&tmA);
+        prefetch_tmap(&tmB);
+        prefetch_tmap(&tmC);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                 // both CTAs' barriers exist before anyone signals them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            const uint32_t pair_tx = 2u * (A_TILE_BYTES + half_n * BK * 2);
+            for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs) {
+                const int m0 = (tile % p.m_tiles) * 256 + rank * 128;
+                const int n0 = (tile / p.m_tiles) * bn + rank * half_n;
+                for (int kb = 0; kb < num_k; ++kb) {
+                    if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 700)) { ok = false; break; }
+                    const uint32_t fb = mapa_shared(full0 + 8 * stage, 0);     // the leader's barrier
+                    if (rank == 0) mbar_arrive_expect_tx(full0 + 8 * stage, pair_tx);
+                    const uint32_t a_dst = smem_u32(tiles + stage * P_STAGE_BYTES), b_dst = a_dst + A_TILE_BYTES;
+                    if constexpr (!A_MN) {
+                        tma_load_2d_pair(a_dst, &tmA, kb * BK, m0, fb);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) tma_load_2d_pair(a_dst + j * 8192, &tmA, m0 + 64 * j, kb * BK, fb);
+                    }
+                    if constexpr (!B_MN) {
+                        tma_load_2d_pair(b_dst, &tmB, kb * BK, n0, fb);
+                    } else {
+                        for (int j = 0; j < half_n / 64; ++j) tma_load_2d_pair(b_dst + j * 8192, &tmB, n0 + 64 * j, kb * BK, fb);
+                    }
+                    if (++stage == P_STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = make_idesc_bf16(256, bn, A_MN, B_MN);
+            uint32_t stage = 0, phase = 0, it = 0;
+            bool ok = true;
+            for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs, ++it) {
+                const uint32_t buf = it & 1, acc_phase = (it >> 1) & 1;
+                if (!mbar_wait(acce0 + 8 * buf, acc_phase ^ 1, abort_flag, p.status, 710)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BN_MAX;
+                for (int kb = 0; kb < num_k; ++kb) {
+                    if (!mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 711)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_base = smem_u32(tiles + stage * P_STAGE_BYTES), b_base = a_base + A_TILE_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+                        const uint64_t adesc = A_MN ? make_smem_desc_sw128(a_base + kk * 2048, 8192, 1024)
+                                                    : make_smem_desc_sw128(a_base + kk * 32, 16, 1024);
+                        const uint64_t bdesc = B_MN ? make_smem_desc_sw128(b_base + kk * 2048, 8192, 1024)
+                                                    : make_smem_desc_sw128(b_base + kk * 32, 16, 1024);
+                        umma_f16_pair(d_tmem, adesc, bdesc, idesc, (kb | kk) != 0 ? 1u : 0u);
+                    }
+                    umma_commit_pair(empty0 + 8 * stage, 3);     // frees the stage in both CTAs
+                    if (++stage == P_STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (ok) umma_commit_pair(accf0 + 8 * buf, 3);     // both CTAs' accumulators complete
+            }
+        }
+    } else {
+        const int q = warp & 3, pi = (warp - 2) >> 2;
+        uint8_t* slab = slabs + (warp - 2) * SLAB_BYTES;
+        const uint32_t slab_u32 = smem_u32(slab);
+        uint32_t it = 0, nout = 0;
+        for (int tile = pair_id; tile < total_tiles; tile += n_pairs, ++it) {
+            const int m0 = (tile % p.m_tiles) * 256 + rank * 128, n0 = (tile / p.m_tiles) * bn;
+            const uint32_t buf = it & 1, acc_phase = (it >> 1) & 1;
+            bool ok = mbar_wait(accf0 + 8 * buf, acc_phase, abort_flag, p.status, 720);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * BN_MAX;
+            epilogue_tile<EPI>(taddr, m0 + q * 32, n0, bn, pi, lane, slab, slab_u32, nout, &tmC, &tmAux, p);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_shared(acce0 + 8 * buf, 0));
+        }
+        if (lane == 0) bulk_wait0();
+    }
+
+    __syncwarp();
+    if (*abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < (1ll << 22)) {}
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                 // neither CTA releases TMEM or exits while its peer may still touch it
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
     }
 }
 
@@ -292,21 +473,35 @@ const char* encode_2d(Runtime* rt, CUtensorMap* map, const void* ptr, uint64_t i
 }
 
 template <bool A_MN, bool B_MN, int EPI>
-const char* launch_inst(Runtime* rt, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
-                        const CUtensorMap& tmAux, const GemmParams& p, cudaStream_t stream)
+const char* launch_inst(Runtime* rt, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmBh,
+                        const CUtensorMap& tmC, const CUtensorMap& tmAux, const GemmParams& p, cudaStream_t stream)
 {
     auto kern = gemm_kernel<A_MN, B_MN, EPI>;
     const int total = p.m_tiles * p.n_tiles;
     const int grid = total < rt->sm_count ? total : rt->sm_count;
-    kern<<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, tmC, tmAux, p);
+    kern<<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, tmBh, tmC, tmAux, p);
     return cudaGetLastError() == cudaSuccess ? nullptr : "gemm launch failed";
+}
+
+template <bool A_MN, bool B_MN, int EPI>
+const char* launch_pair(Runtime* rt, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC,
+                        const CUtensorMap& tmAux, const GemmParams& p, cudaStream_t stream)
+{
+    auto kern = gemm_pair_kernel<A_MN, B_MN, EPI>;
+    const int total = p.m_tiles * p.n_tiles;
+    const int max_pairs = rt->sm_count / 2;
+    const int pairs = total < max_pairs ? total : max_pairs;
+    kern<<<2 * pairs, GEMM_THREADS, P_SMEM_BYTES, stream>>>(tmA, tmB, tmC, tmAux, p);
+    return cudaGetLastError() == cudaSuccess ? nullptr : "gemm (CTA pair) launch failed";
 }
 
 template <bool A_MN, bool B_MN, int EPI>
 bool set_attr()
 {
     return cudaFuncSetAttribute(gemm_kernel<A_MN, B_MN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                SMEM_BYTES) == cudaSuccess;
+                                SMEM_BYTES) == cudaSuccess &&
+           cudaFuncSetAttribute(gemm_pair_kernel<A_MN, B_MN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                P_SMEM_BYTES) == cudaSuccess;
 }
 
 }  // namespace
@@ -320,6 +515,55 @@ const char* configure_gemm()
                     set_attr<false, true, kEpiNone>() && set_attr<false, true, kEpiDGelu>() &&
                     set_attr<true, true, kEpiF32>();
     return ok ? nullptr : "cudaFuncSetAttribute(gemm) failed";
+}
+
+static const char* launch_gemm_pair(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cudaStream_t stream)
+{
+    const bool a_mn = a.layout == kNT, b_mn = a.layout == kNN || a.layout == kNT;
+    const bool f32_out = a.epilogue == kEpiF32;
+    const int m_tiles = (a.M + 255) / 256, pairs = rt->sm_count / 2;
+    // Tile width: 256 unless the rounds it needs waste more than a 128-wide tiling does (a
+    // 128-wide pair tile moves as many operand bytes per FLOP as the one-CTA 256-wide tile).
+    int bn = 256;
+    {
+        static const int forced = [] { const char* v = getenv("PW_GEMM_BN"); return v ? atoi(v) : 0; }();
+        auto cost = [&](int w) {
+            const long long tiles = static_cast<long long>(m_tiles) * ((a.N + w - 1) / w);
+            const long long rounds = (tiles + pairs - 1) / pairs;
+            return static_cast<double>(rounds) * w * (w == 128 ? 1.6 : 1.0);   // 128-wide pair tiles measured ~1.6x slower per FLOP
+        };
+        if (cost(128) < cost(256)) bn = 128;
+        if (forced == 128 || forced == 256) bn = forced;
+    }
+    CUtensorMap tmA, tmB, tmC, tmAux;
+    const char* e;
+    e = a_mn ? encode_2d(rt, &tmA, a.A, a.M, a.K, a.lda, 64, BK) : encode_2d(rt, &tmA, a.A, a.K, a.M, a.lda, BK, BM);
+    if (e) return e;
+    e = b_mn ? encode_2d(rt, &tmB, a.B, a.N, a.K, a.ldb, 64, BK) : encode_2d(rt, &tmB, a.B, a.K, a.N, a.ldb, BK, bn / 2);
+    if (e) return e;
+    e = encode_2d(rt, &tmC, a.C, a.N, a.M, a.ldc, 32, 32, f32_out, !f32_out);
+    if (e) return e;
+    e = encode_2d(rt, &tmAux, a.epilogue == kEpiBiasGelu ? a.aux_out : a.C, a.N, a.M, a.ldc, 32, 32, f32_out, !f32_out);
+    if (e) return e;
+    GemmParams p;
+    p.M = a.M; p.N = a.N; p.K = a.K; p.bn = bn;
+    p.bias = static_cast<const __nv_bfloat16*>(a.bias);
+    p.aux_in = static_cast<const __nv_bfloat16*>(a.aux_in); p.ld_aux = a.ld_aux;
+    p.accumulate = a.accumulate; p.act = a.act;
+    p.m_tiles = m_tiles; p.n_tiles = (a.N + bn - 1) / bn;
+    p.split_begin = p.m_tiles * p.n_tiles; p.total_virtual = p.split_begin;
+    p.status = status;
+    const int key = a.layout * 16 + a.epilogue;
+    switch (key) {
+        case kTN * 16 + kEpiNone: return launch_pair<false, false, kEpiNone>(rt, tmA, tmB, tmC, tmAux, p, stream);
+        case kTN * 16 + kEpiBias: return launch_pair<false, false, kEpiBias>(rt, tmA, tmB, tmC, tmAux, p, stream);
+        case kTN * 16 + kEpiBiasResid: return launch_pair<false, false, kEpiBiasResid>(rt, tmA, tmB, tmC, tmAux, p, stream);
+        case kTN * 16 + kEpiBiasGelu: return launch_pair<false, false, kEpiBiasGelu>(rt, tmA, tmB, tmC, tmAux, p, stream);
+        case kNN * 16 + kEpiNone: return launch_pair<false, true, kEpiNone>(rt, tmA, tmB, tmC, tmAux, p, stream);
+        case kNN * 16 + kEpiDGelu: return launch_pair<false, true, kEpiDGelu>(rt, tmA, tmB, tmC, tmAux, p, stream);
+        case kNT * 16 + kEpiF32: return launch_pair<true, true, kEpiF32>(rt, tmA, tmB, tmC, tmAux, p, stream);
+        default: return "gemm: unsupported layout/epilogue combination";
+    }
 }
 
 const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cudaStream_t stream)
@@ -337,6 +581,8 @@ const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cu
 
     const bool a_mn = a.layout == kNT, b_mn = a.layout == kNN || a.layout == kNT;
     const bool f32_out = a.epilogue == kEpiF32;
+    static const int pair_mode = [] { const char* v = getenv("PW_GEMM_PAIR"); return v ? atoi(v) : 1; }();   // tuning aid
+    if (pair_mode && a.M >= 256) return launch_gemm_pair(rt, a, status, stream);
     if (f32_out && (a.ldc % 4)) return "gemm: fp32 ldc must be a multiple of 4";
     // Tile width: the one that needs the least (rounds x width) on this many SMs; ties go to the
     // wider tile (less operand traffic per FLOP).
@@ -350,12 +596,14 @@ const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cu
         static const int forced = [] { const char* v = getenv("PW_GEMM_BN"); return v ? atoi(v) : 0; }();
         if (forced == 128 || forced == 192 || forced == 256) bn = forced;   // tuning aid
     }
-    CUtensorMap tmA, tmB, tmC, tmAux;
+    CUtensorMap tmA, tmB, tmBh, tmC, tmAux;
     const char* e;
     // K-major operand [rows, K]: box 64 k x rows.  MN-major operand stored [K, rows]: box 64 rows x 64 k.
     e = a_mn ? encode_2d(rt, &tmA, a.A, a.M, a.K, a.lda, 64, BK) : encode_2d(rt, &tmA, a.A, a.K, a.M, a.lda, BK, BM);
     if (e) return e;
     e = b_mn ? encode_2d(rt, &tmB, a.B, a.N, a.K, a.ldb, 64, BK) : encode_2d(rt, &tmB, a.B, a.K, a.N, a.ldb, BK, bn);
+    if (e) return e;
+    e = b_mn ? encode_2d(rt, &tmBh, a.B, a.N, a.K, a.ldb, 64, BK) : encode_2d(rt, &tmBh, a.B, a.K, a.N, a.ldb, BK, bn / 2);
     if (e) return e;
 
     // Output maps: a store box is 32 rows x 32 columns (fp32: 128-byte rows, 128-byte swizzle;
@@ -372,16 +620,27 @@ const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cu
     p.accumulate = a.accumulate; p.act = a.act;
     p.m_tiles = m_tiles; p.n_tiles = (a.N + bn - 1) / bn;
     p.status = status;
+    {
+        // Tail balancing: when the last round would leave at least half of the SMs idle, its
+        // tiles are issued as two half-width tiles each.
+        const int total = p.m_tiles * p.n_tiles;
+        const int grid = total < rt->sm_count ? total : rt->sm_count;
+        const int rem = total % grid;
+        static const bool no_split = getenv("PW_GEMM_NO_SPLIT") != nullptr;   // tuning aid
+        p.split_begin = total;
+        if (bn == BN_MAX && rem > 0 && 2 * rem <= grid && !no_split) p.split_begin = total - rem;
+        p.total_virtual = p.split_begin + 2 * (total - p.split_begin);
+    }
 
     const int key = a.layout * 16 + a.epilogue;
     switch (key) {
-        case kTN * 16 + kEpiNone: return launch_inst<false, false, kEpiNone>(rt, tmA, tmB, tmC, tmAux, p, stream);
-        case kTN * 16 + kEpiBias: return launch_inst<false, false, kEpiBias>(rt, tmA, tmB, tmC, tmAux, p, stream);
-        case kTN * 16 + kEpiBiasResid: return launch_inst<false, false, kEpiBiasResid>(rt, tmA, tmB, tmC, tmAux, p, stream);
-        case kTN * 16 + kEpiBiasGelu: return launch_inst<false, false, kEpiBiasGelu>(rt, tmA, tmB, tmC, tmAux, p, stream);
-        case kNN * 16 + kEpiNone: return launch_inst<false, true, kEpiNone>(rt, tmA, tmB, tmC, tmAux, p, stream);
-        case kNN * 16 + kEpiDGelu: return launch_inst<false, true, kEpiDGelu>(rt, tmA, tmB, tmC, tmAux, p, stream);
-        case kNT * 16 + kEpiF32: return launch_inst<true, true, kEpiF32>(rt, tmA, tmB, tmC, tmAux, p, stream);
+        case kTN * 16 + kEpiNone: return launch_inst<false, false, kEpiNone>(rt, tmA, tmB, tmBh, tmC, tmAux, p, stream);
+        case kTN * 16 + kEpiBias: return launch_inst<false, false, kEpiBias>(rt, tmA, tmB, tmBh, tmC, tmAux, p, stream);
+        case kTN * 16 + kEpiBiasResid: return launch_inst<false, false, kEpiBiasResid>(rt, tmA, tmB, tmBh, tmC, tmAux, p, stream);
+        case kTN * 16 + kEpiBiasGelu: return launch_inst<false, false, kEpiBiasGelu>(rt, tmA, tmB, tmBh, tmC, tmAux, p, stream);
+        case kNN * 16 + kEpiNone: return launch_inst<false, true, kEpiNone>(rt, tmA, tmB, tmBh, tmC, tmAux, p, stream);
+        case kNN * 16 + kEpiDGelu: return launch_inst<false, true, kEpiDGelu>(rt, tmA, tmB, tmBh, tmC, tmAux, p, stream);
+        case kNT * 16 + kEpiF32: return launch_inst<true, true, kEpiF32>(rt, tmA, tmB, tmBh, tmC, tmAux, p, stream);
         default: return "gemm: unsupported layout/epilogue combination";
     }
 }
