@@ -94,8 +94,8 @@ __device__ __forceinline__ void epilogue_group(const uint32_t* v, int row, int c
 // lane quarter of the accumulator, row0 is the first of its 32 rows, pi selects which of the two
 // warps of the quarter it is (they take alternate column chunks).
 template <int EPI>
-__device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, int bn, int pi, int lane, uint8_t* slab,
-                                              uint32_t slab_u32, uint32_t& nout, const CUtensorMap* tmC,
+__device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, int bn, int pi, int pstride, int lane,
+                                              uint8_t* slab, uint32_t slab_u32, uint32_t& nout, const CUtensorMap* tmC,
                                               const CUtensorMap* tmAux, const GemmParams& p)
 {
     const int row = row0 + lane;
@@ -103,7 +103,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, 
     if constexpr (EPI == kEpiF32) {
         const int nsteps = bn / 32;
 #pragma unroll 1
-        for (int s = pi; s < nsteps; s += 2) {
+        for (int s = pi; s < nsteps; s += pstride) {
             const int col0 = n0 + s * 32;
             if (col0 >= p.N) break;
             uint32_t v[32];
@@ -129,7 +129,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, 
         const int nchunks = bn / 32;
         const uint32_t sw = (lane >> 1) & 3;
 #pragma unroll 1
-        for (int ch = pi; ch < nchunks; ch += 2) {
+        for (int ch = pi; ch < nchunks; ch += pstride) {
             const int col0 = n0 + ch * 32;
             if (col0 >= p.N) break;
             uint32_t v[32];
@@ -286,7 +286,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * BN_MAX;
-            epilogue_tile<EPI>(taddr, m0 + q * 32, n0, bn, pi, lane, slab, slab_u32, nout, &tmC, &tmAux, p);
+            epilogue_tile<EPI>(taddr, m0 + q * 32, n0, bn, pi, 2, lane, slab, slab_u32, nout, &tmC, &tmAux, p);
             tc_fence_before();
             mbar_arrive(acce0 + 8 * buf);
         }
@@ -316,19 +316,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 // N = d_model GEMMs.  Barriers: full[s] (leader, 1 arrival + both CTAs' bytes), empty[s] and
 // acc_full[b] (one in each CTA, signalled by the leader's tcgen05.commit to both), acc_empty[b]
 // (leader, one arrival per epilogue warp of both CTAs).
-constexpr int P_STAGES = 6;
+// The epilogues that evaluate GeLU / GeLU' are instruction-bound with 8 warps (two per scheduler),
+// so those instantiations run 16 epilogue warps and give up one pipeline stage for their slabs.
 constexpr int P_STAGE_BYTES = 32768;            // A: 128 x 64 (16 KB) + B half: up to 128 x 64 (16 KB)
-constexpr int P_SMEM_BYTES = P_STAGES * P_STAGE_BYTES + EPI_WARPS * SLAB_BYTES + 1024 + 256;
+template <int EPI> struct PairCfg {
+    static constexpr int kEpiWarps = (EPI == kEpiBiasGelu || EPI == kEpiDGelu) ? 16 : 8;
+    static constexpr int kStages = kEpiWarps == 16 ? 5 : 6;
+    static constexpr int kThreads = 64 + 32 * kEpiWarps;
+    static constexpr int kSmem = kStages * P_STAGE_BYTES + kEpiWarps * SLAB_BYTES + 1024 + 256;
+};
 
 template <bool A_MN, bool B_MN, int EPI>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairCfg<EPI>::kThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmAux, const GemmParams p)
 {
+    constexpr int P_STAGES = PairCfg<EPI>::kStages, NEPI = PairCfg<EPI>::kEpiWarps;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* slabs = tiles + P_STAGES * P_STAGE_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(slabs + EPI_WARPS * SLAB_BYTES);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(slabs + NEPI * SLAB_BYTES);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + P_STAGES);
     const uint32_t accf0 = smem_u32(bars + 2 * P_STAGES), acce0 = smem_u32(bars + 2 * P_STAGES + 2);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * P_STAGES + 4);
@@ -343,7 +350,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < P_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 2 * EPI_WARPS); }
+        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 2 * NEPI); }
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -430,7 +437,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * BN_MAX;
-            epilogue_tile<EPI>(taddr, m0 + q * 32, n0, bn, pi, lane, slab, slab_u32, nout, &tmC, &tmAux, p);
+            epilogue_tile<EPI>(taddr, m0 + q * 32, n0, bn, pi, NEPI / 4, lane, slab, slab_u32, nout, &tmC, &tmAux, p);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_shared(acce0 + 8 * buf, 0));
@@ -491,7 +498,7 @@ const char* launch_pair(Runtime* rt, const CUtensorMap& tmA, const CUtensorMap& 
     const int total = p.m_tiles * p.n_tiles;
     const int max_pairs = rt->sm_count / 2;
     const int pairs = total < max_pairs ? total : max_pairs;
-    kern<<<2 * pairs, GEMM_THREADS, P_SMEM_BYTES, stream>>>(tmA, tmB, tmC, tmAux, p);
+    kern<<<2 * pairs, PairCfg<EPI>::kThreads, PairCfg<EPI>::kSmem, stream>>>(tmA, tmB, tmC, tmAux, p);
     return cudaGetLastError() == cudaSuccess ? nullptr : "gemm (CTA pair) launch failed";
 }
 
@@ -501,7 +508,7 @@ bool set_attr()
     return cudaFuncSetAttribute(gemm_kernel<A_MN, B_MN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 SMEM_BYTES) == cudaSuccess &&
            cudaFuncSetAttribute(gemm_pair_kernel<A_MN, B_MN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                P_SMEM_BYTES) == cudaSuccess;
+                                PairCfg<EPI>::kSmem) == cudaSuccess;
 }
 
 }  // namespace
