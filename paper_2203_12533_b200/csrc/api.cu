@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -69,7 +70,7 @@ struct LayerPlan {
     float eps;
     size_t ctx_off[PW_CTX_COUNT], ctx_size[PW_CTX_COUNT], ctx_bytes;
     // scratch = [ctx-shaped region used when the caller passes ctx == NULL] [backward temporaries]
-    size_t off_big, off_td0, off_td1, off_delta, off_partials, scratch_bytes;
+    size_t off_big, off_td0, off_td1, off_delta, off_partials, off_partials2, scratch_bytes;
 };
 
 }  // namespace pw
@@ -78,6 +79,8 @@ struct pw_layer {
     pw::LayerPlan plan;
     pw::Runtime* rt;
     pw::DeviceStatus* status;
+    cudaStream_t aux = nullptr;     // side stream: weight gradients and bias column sums run beside the dgrad chain
+    cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     uint64_t launches = 0;          // kernels launched (or replayed) through this handle
     bool capturing = false;         // inside a stream capture: count launches into graph_nodes instead
     uint64_t graph_nodes = 0;
@@ -141,6 +144,7 @@ static void build_plan(const pw_layer_config_t& c, Runtime* rt, LayerPlan* p)
     if (c1 > part) part = c1;
     if (c2 > part) part = c2;
     p->off_partials = s; s += align256(part);
+    p->off_partials2 = s; s += align256(c1 > c2 ? c1 : c2);   // column sums on the side stream
     p->scratch_bytes = s;
 }
 
@@ -293,36 +297,64 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
     void* delta = at(scratch, p.off_delta);
     void* part = at(scratch, p.off_partials);
 
+    void* part2 = at(scratch, p.off_partials2);
+
+    // The weight gradients and the bias column sums hang off the dgrad chain, so they run on a
+    // side stream: their CTAs fill the SMs that the last, partly filled round of a dgrad GEMM
+    // leaves idle (and the HBM-bound kernels share SMs with GEMM CTAs).  Events order the two
+    // streams; the side stream always rejoins before this call returns, so a captured graph sees
+    // a plain fork/join.  While per-kernel profiling is on everything stays on one stream.
+    static const bool no_side = getenv("PW_NO_SIDE_STREAM") != nullptr;   // tuning aid
+    cudaStream_t ax = (L->profiling || no_side) ? st : L->aux;
+    auto order = [&](cudaEvent_t ev, cudaStream_t from, cudaStream_t to) -> pw_status_t {
+        if (from == to) return PW_OK;
+        cudaError_t e = cudaEventRecord(ev, from);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(to, ev, 0);
+        return e == cudaSuccess ? PW_OK : fail_cuda("stream ordering", e);
+    };
+    PW_DO(order(L->ev[0], st, ax));                      // side stream starts after everything already enqueued
     // y = x1 + a W2^T + b2  ->  du = (dy W2) * gelu'(u),  dW2 = dy^T a
+    PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, d, F, T, dy, d, a, F, G->w_fc2, F, nullptr, nullptr, 0,
+                                     nullptr, accumulate), ax));
     PW_DO(do_gemm(L, gemm_args(kNN, kEpiDGelu, act, T, F, d, dy, d, P->w_fc2, F, big, F, nullptr, u, F,
                                      nullptr, 0), st));
-    PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, d, F, T, dy, d, a, F, G->w_fc2, F, nullptr, nullptr, 0,
-                                     nullptr, accumulate), st));
+    PW_DO(order(L->ev[1], st, ax));                      // du ready
     // u = h2 W1^T + b1  ->  dh2 = du W1,  dW1 = du^T h2,  db1 = colsum(du)
+    PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, F, d, T, big, F, h2, d, G->w_fc1, d, nullptr, nullptr, 0,
+                                     nullptr, accumulate), ax));
+    PW_DO(do_colsum(L, big, F, G->b_fc1, accumulate, part2, ax));
+    if (ax != st) {                                      // remembered: du may be overwritten only after these two
+        cudaError_t e = cudaEventRecord(L->ev[2], ax);
+        if (e != cudaSuccess) return fail_cuda("stream ordering", e);
+    }
     PW_DO(do_gemm(L, gemm_args(kNN, kEpiNone, act, T, d, F, big, F, P->w_fc1, d, td0, d, nullptr, nullptr, 0,
                                      nullptr, 0), st));
-    PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, F, d, T, big, F, h2, d, G->w_fc1, d, nullptr, nullptr, 0,
-                                     nullptr, accumulate), st));
-    PW_DO(do_colsum(L, big, F, G->b_fc1, accumulate, part, st));
     // LN2 backward + residual: dx1 = dy + LNbwd(dh2); also db2 = colsum(dy), dbo = colsum(dx1)
     PW_DO(do_ln_bwd(L, td0, x1, mu2, r2, P->ln2_gamma, dy, dx1, G->ln2_gamma, G->ln2_beta,
                                 G->b_fc2, G->b_o, accumulate, part, st));
+    PW_DO(order(L->ev[3], st, ax));                      // dx1 ready
     // x1 = x + o Wo^T + bo  ->  dout = dx1 Wo,  dWo = dx1^T o
+    PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, d, d, T, dx1, d, o, d, G->w_o, d, nullptr, nullptr, 0,
+                                     nullptr, accumulate), ax));
     PW_DO(do_gemm(L, gemm_args(kNN, kEpiNone, act, T, d, d, dx1, d, P->w_o, d, td0, d, nullptr, nullptr, 0,
                                      nullptr, 0), st));
-    PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, d, d, T, dx1, d, o, d, G->w_o, d, nullptr, nullptr, 0,
-                                     nullptr, accumulate), st));
-    // attention backward -> dqkv
+    // attention backward -> dqkv (reuses the du buffer)
+    if (ax != st) {
+        cudaError_t e = cudaStreamWaitEvent(st, L->ev[2], 0);
+        if (e != cudaSuccess) return fail_cuda("stream ordering", e);
+    }
     PW_DO(do_attn_bwd(L, qkv, o, td0, lse, big, delta, st));
+    PW_DO(order(L->ev[4], st, ax));                      // dqkv ready
     // qkv = h1 Wqkv^T + bqkv  ->  dh1 = dqkv Wqkv,  dWqkv = dqkv^T h1,  dbqkv = colsum(dqkv)
+    PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, 3 * d, d, T, big, 3 * d, h1, d, G->w_qkv, d, nullptr, nullptr,
+                                     0, nullptr, accumulate), ax));
+    PW_DO(do_colsum(L, big, 3 * d, G->b_qkv, accumulate, part2, ax));
     PW_DO(do_gemm(L, gemm_args(kNN, kEpiNone, act, T, d, 3 * d, big, 3 * d, P->w_qkv, d, td0, d, nullptr,
                                      nullptr, 0, nullptr, 0), st));
-    PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, 3 * d, d, T, big, 3 * d, h1, d, G->w_qkv, d, nullptr, nullptr,
-                                     0, nullptr, accumulate), st));
-    PW_DO(do_colsum(L, big, 3 * d, G->b_qkv, accumulate, part, st));
     // LN1 backward + residual: dx = dx1 + LNbwd(dh1)
     PW_DO(do_ln_bwd(L, td0, x, mu1, r1, P->ln1_gamma, dx1, dx, G->ln1_gamma, G->ln1_beta, nullptr,
                                 nullptr, accumulate, part, st));
+    PW_DO(order(L->ev[5], ax, st));                      // join
     return PW_OK;
 }
 
@@ -393,7 +425,9 @@ pw_status_t pw_layer_create(const pw_layer_config_t* cfg, pw_layer_t** out)
     build_plan(*cfg, rt, &L->plan);
     cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&L->status), sizeof(DeviceStatus));
     if (e == cudaSuccess) e = cudaMemset(L->status, 0, sizeof(DeviceStatus));
-    if (e != cudaSuccess) { delete L; return fail_cuda("status word allocation", e); }
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&L->aux, cudaStreamNonBlocking);
+    for (int i = 0; i < 6 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&L->ev[i], cudaEventDisableTiming);
+    if (e != cudaSuccess) { pw_layer_destroy(L); return fail_cuda("handle resources (status word, side stream, events)", e); }
     *out = L;
     return PW_OK;
 }
@@ -403,6 +437,8 @@ void pw_layer_destroy(pw_layer_t* layer)
     if (!layer) return;
     for (auto& sp : layer->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     for (auto e : layer->pool) cudaEventDestroy(e);
+    for (auto e : layer->ev) if (e) cudaEventDestroy(e);
+    if (layer->aux) cudaStreamDestroy(layer->aux);
     if (layer->status) cudaFree(layer->status);
     delete layer;
 }

@@ -79,6 +79,20 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
         fence_barrier_init();
         fence_proxy_async();
         prefetch_tmap(&tmKV); prefetch_tmap(&tmQ); prefetch_tmap(&tmDO); prefetch_tmap(&tmOut);
+        // first loads go out before the TMEM allocation and the CTA-wide barrier
+        mbar_arrive_expect_tx(bar(0), 2 * L::kKV);
+        for (int kb = 0; kb < L::kBlocks; ++kb) {
+            tma_load_2d(sbase + L::kK + kb * 16384, &tmKV, d + h * DH + kb * 64, row_base + kv0, bar(0));
+            tma_load_2d(sbase + L::kV + kb * 16384, &tmKV, 2 * d + h * DH + kb * 64, row_base + kv0, bar(0));
+        }
+        for (int i = 0; i < n_u && i < L::kStages; ++i) {
+            mbar_arrive_expect_tx(bar(1 + i), 2 * L::kSub);
+            const uint32_t qs = sbase + L::kQ + i * 2 * L::kSub, gs = qs + L::kSub;
+            for (int kb = 0; kb < L::kBlocks; ++kb) {
+                tma_load_2d(qs + kb * 8192, &tmQ, h * DH + kb * 64, row_base + (u0 + i) * 64, bar(1 + i));
+                tma_load_2d(gs + kb * 8192, &tmDO, h * DH + kb * 64, row_base + (u0 + i) * 64, bar(1 + i));
+            }
+        }
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_slot), 512);
@@ -92,12 +106,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
 
     if (warp == 0) {
         if (lane == 0) {
-            mbar_arrive_expect_tx(bar(0), 2 * L::kKV);
-            for (int kb = 0; kb < L::kBlocks; ++kb) {
-                tma_load_2d(sbase + L::kK + kb * 16384, &tmKV, d + h * DH + kb * 64, row_base + kv0, bar(0));
-                tma_load_2d(sbase + L::kV + kb * 16384, &tmKV, 2 * d + h * DH + kb * 64, row_base + kv0, bar(0));
-            }
-            for (int i = 0; i < n_u; ++i) {
+            for (int i = L::kStages; i < n_u; ++i) {        // K_j, V_j and the first sub-tiles were requested in the prologue
                 const int s = i % L::kStages, ph = (i / L::kStages) & 1;
                 if (!mbar_wait(bar(5 + s), ph ^ 1, abort_flag, p.status, 500)) break;
                 mbar_arrive_expect_tx(bar(1 + s), 2 * L::kSub);
@@ -113,40 +122,41 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
         if (lane == 0) {
             constexpr uint32_t idesc_st = make_idesc_bf16(128, 64, false, false);
             constexpr uint32_t idesc_acc = make_idesc_bf16(128, DH, false, true);
+            const uint64_t desc_k = make_smem_desc_sw128(sbase + L::kK, 16, 1024);
+            const uint64_t desc_v = make_smem_desc_sw128(sbase + L::kV, 16, 1024);
             auto issue_scores = [&](int i) {                // S^T and dP^T of sub-tile i into buffer i & 1
                 const int s = i % L::kStages, hb = i & 1;
-                const uint32_t qs = sbase + L::kQ + s * 2 * L::kSub, gs = qs + L::kSub;
+                const uint32_t qs = sbase + L::kQ + s * 2 * L::kSub;
+                const uint64_t dq = make_smem_desc_sw128(qs, 16, 1024), dg = desc_advance(dq, L::kSub);
+                const uint32_t st = tmem_base + hb * 64;
 #pragma unroll
                 for (int kb = 0; kb < L::kBlocks; ++kb)
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        umma_f16(tmem_base + hb * 64, make_smem_desc_sw128(sbase + L::kK + kb * 16384 + kk * 32, 16, 1024),
-                                 make_smem_desc_sw128(qs + kb * 8192 + kk * 32, 16, 1024), idesc_st, (kb | kk) ? 1u : 0u);
-                    }
+                    for (int kk = 0; kk < 4; ++kk)
+                        umma_f16(st, desc_advance(desc_k, kb * 16384 + kk * 32), desc_advance(dq, kb * 8192 + kk * 32),
+                                 idesc_st, (kb | kk) ? 1u : 0u);
 #pragma unroll
                 for (int kb = 0; kb < L::kBlocks; ++kb)
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        umma_f16(tmem_base + 128 + hb * 64, make_smem_desc_sw128(sbase + L::kV + kb * 16384 + kk * 32, 16, 1024),
-                                 make_smem_desc_sw128(gs + kb * 8192 + kk * 32, 16, 1024), idesc_st, (kb | kk) ? 1u : 0u);
-                    }
+                    for (int kk = 0; kk < 4; ++kk)
+                        umma_f16(st + 128, desc_advance(desc_v, kb * 16384 + kk * 32), desc_advance(dg, kb * 8192 + kk * 32),
+                                 idesc_st, (kb | kk) ? 1u : 0u);
                 umma_commit(bar(9 + hb));
             };
             auto issue_acc = [&](int i) {                   // dV += P^T dO_u, dK += dS^T Q_u
                 const int s = i % L::kStages, hb = i & 1;
-                const uint32_t qs = sbase + L::kQ + s * 2 * L::kSub, gs = qs + L::kSub;
+                const uint32_t qs = sbase + L::kQ + s * 2 * L::kSub;
+                const uint64_t dq = make_smem_desc_sw128(qs, 8192, 1024), dg = desc_advance(dq, L::kSub);
+                const uint32_t pt = tmem_base + hb * 64;
+                const uint32_t first = i ? 1u : 0u;
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    const uint32_t acol = (ks >> 1) * 32 + (ks & 1) * 8;
-                    umma_f16_ta(tmem_base + 256, tmem_base + hb * 64 + acol,
-                                make_smem_desc_sw128(gs + ks * 2048, 8192, 1024), idesc_acc, (i | ks) ? 1u : 0u);
-                }
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_f16_ta(tmem_base + 256, pt + (ks >> 1) * 32 + (ks & 1) * 8, desc_advance(dg, ks * 2048), idesc_acc,
+                                ks ? 1u : first);
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    const uint32_t acol = (ks >> 1) * 32 + (ks & 1) * 8;
-                    umma_f16_ta(tmem_base + 384, tmem_base + 128 + hb * 64 + acol,
-                                make_smem_desc_sw128(qs + ks * 2048, 8192, 1024), idesc_acc, (i | ks) ? 1u : 0u);
-                }
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_f16_ta(tmem_base + 384, pt + 128 + (ks >> 1) * 32 + (ks & 1) * 8, desc_advance(dq, ks * 2048), idesc_acc,
+                                ks ? 1u : first);
                 umma_commit(bar(5 + s));                    // Q_u / dO_u stage free
             };
             bool ok = mbar_wait(bar(0), 0, abort_flag, p.status, 510) && mbar_wait(bar(1), 0, abort_flag, p.status, 511);
@@ -314,6 +324,22 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
         fence_barrier_init();
         fence_proxy_async();
         prefetch_tmap(&tmQ); prefetch_tmap(&tmDO); prefetch_tmap(&tmKV); prefetch_tmap(&tmOut);
+        // first loads go out before the TMEM allocation and the CTA-wide barrier
+        const int nq = hasB ? 2 : 1;
+        mbar_arrive_expect_tx(bar(0), nq * 2 * L::kTile);
+        for (int t = 0; t < nq; ++t)
+            for (int kb = 0; kb < L::kBlocks; ++kb) {
+                tma_load_2d(sbase + L::kQ + t * L::kTile + kb * 16384, &tmQ, h * DH + kb * 64, row_base + q0A + t * 128, bar(0));
+                tma_load_2d(sbase + L::kQ + (2 + t) * L::kTile + kb * 16384, &tmDO, h * DH + kb * 64, row_base + q0A + t * 128, bar(0));
+            }
+        for (int v = 0; v < 2 && v < n_kv; ++v) {
+            mbar_arrive_expect_tx(bar(1 + v), 2 * L::kSub);
+            const uint32_t ks = sbase + L::kKV + v * 2 * L::kSub, vs = ks + L::kSub;
+            for (int kb = 0; kb < L::kBlocks; ++kb) {
+                tma_load_2d(ks + kb * 8192, &tmKV, d + h * DH + kb * 64, row_base + v * 64, bar(1 + v));
+                tma_load_2d(vs + kb * 8192, &tmKV, 2 * d + h * DH + kb * 64, row_base + v * 64, bar(1 + v));
+            }
+        }
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_slot), 512);
@@ -327,16 +353,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
 
     if (warp == 0) {
         if (lane == 0) {
-            const int nq = hasB ? 2 : 1;
-            mbar_arrive_expect_tx(bar(0), nq * 2 * L::kTile);
-            for (int t = 0; t < nq; ++t)
-                for (int kb = 0; kb < L::kBlocks; ++kb) {
-                    tma_load_2d(sbase + L::kQ + t * L::kTile + kb * 16384, &tmQ, h * DH + kb * 64,
-                                row_base + q0A + t * 128, bar(0));
-                    tma_load_2d(sbase + L::kQ + (2 + t) * L::kTile + kb * 16384, &tmDO, h * DH + kb * 64,
-                                row_base + q0A + t * 128, bar(0));
-                }
-            for (int v = 0; v < n_kv; ++v) {
+            for (int v = 2; v < n_kv; ++v) {                // Q, dO and the first two sub-tiles were requested in the prologue
                 const int s = v & 1, ph = (v >> 1) & 1;
                 if (!mbar_wait(bar(3 + s), ph ^ 1, abort_flag, p.status, 600)) break;
                 mbar_arrive_expect_tx(bar(1 + s), 2 * L::kSub);
@@ -352,28 +369,31 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
             constexpr uint32_t idesc_sc = make_idesc_bf16(128, 64, false, false);
             constexpr uint32_t idesc_dq = make_idesc_bf16(128, DH, false, true);
             auto issue_scores = [&](int t, int s) {         // S_t = Q_t K_v^T, dP_t = dO_t V_v^T
-                const uint32_t qa = sbase + L::kQ + t * L::kTile, ga = sbase + L::kQ + (2 + t) * L::kTile;
-                const uint32_t ks = sbase + L::kKV + s * 2 * L::kSub, vs = ks + L::kSub;
+                const uint64_t dq = make_smem_desc_sw128(sbase + L::kQ + t * L::kTile, 16, 1024);
+                const uint64_t dg = desc_advance(dq, 2 * L::kTile);
+                const uint64_t dk = make_smem_desc_sw128(sbase + L::kKV + s * 2 * L::kSub, 16, 1024);
+                const uint64_t dv = desc_advance(dk, L::kSub);
+                const uint32_t dst = tmem_base + t * 256;
 #pragma unroll
                 for (int kb = 0; kb < L::kBlocks; ++kb)
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
-                        umma_f16(tmem_base + t * 256, make_smem_desc_sw128(qa + kb * 16384 + kk * 32, 16, 1024),
-                                 make_smem_desc_sw128(ks + kb * 8192 + kk * 32, 16, 1024), idesc_sc, (kb | kk) ? 1u : 0u);
+                        umma_f16(dst, desc_advance(dq, kb * 16384 + kk * 32), desc_advance(dk, kb * 8192 + kk * 32),
+                                 idesc_sc, (kb | kk) ? 1u : 0u);
 #pragma unroll
                 for (int kb = 0; kb < L::kBlocks; ++kb)
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
-                        umma_f16(tmem_base + t * 256 + 64, make_smem_desc_sw128(ga + kb * 16384 + kk * 32, 16, 1024),
-                                 make_smem_desc_sw128(vs + kb * 8192 + kk * 32, 16, 1024), idesc_sc, (kb | kk) ? 1u : 0u);
+                        umma_f16(dst + 64, desc_advance(dg, kb * 16384 + kk * 32), desc_advance(dv, kb * 8192 + kk * 32),
+                                 idesc_sc, (kb | kk) ? 1u : 0u);
                 umma_commit(bar(5 + t));
             };
             auto issue_dq = [&](int t, int s, bool acc) {   // dQ_t += dS_t K_v (dS packed in the S columns)
-                const uint32_t ks = sbase + L::kKV + s * 2 * L::kSub;
+                const uint64_t dk = make_smem_desc_sw128(sbase + L::kKV + s * 2 * L::kSub, 8192, 1024);
+                const uint32_t dst = tmem_base + t * 256 + 128, src = tmem_base + t * 256;
+                umma_f16_ta(dst, src, dk, idesc_dq, acc ? 1u : 0u);
 #pragma unroll
-                for (int kq = 0; kq < 4; ++kq)
-                    umma_f16_ta(tmem_base + t * 256 + 128, tmem_base + t * 256 + kq * 8,
-                                make_smem_desc_sw128(ks + kq * 2048, 8192, 1024), idesc_dq, (acc || kq) ? 1u : 0u);
+                for (int kq = 1; kq < 4; ++kq) umma_f16_ta(dst, src + kq * 8, desc_advance(dk, kq * 2048), idesc_dq, 1u);
             };
             bool ok = mbar_wait(bar(0), 0, abort_flag, p.status, 610) && mbar_wait(bar(1), 0, abort_flag, p.status, 611);
             if (ok) {

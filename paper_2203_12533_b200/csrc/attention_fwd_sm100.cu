@@ -76,6 +76,19 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
         fence_proxy_async();
         prefetch_tmap(&tmQKV);
         prefetch_tmap(&tmO);
+        // first loads go out before the TMEM allocation and the CTA-wide barrier
+        const int nq = hasB ? 2 : 1;
+        mbar_arrive_expect_tx(bar(0), nq * L::kTile);
+        for (int t = 0; t < nq; ++t)
+            for (int kb = 0; kb < L::kBlocks; ++kb)
+                tma_load_2d(sbase + L::kQ + t * L::kTile + kb * 16384, &tmQKV, h * DH + kb * 64,
+                            row_base + q0A + t * 128, bar(0));
+        mbar_arrive_expect_tx(bar(1), L::kTile);
+        mbar_arrive_expect_tx(bar(5), L::kTile);
+        for (int kb = 0; kb < L::kBlocks; ++kb) {
+            tma_load_2d(sbase + L::kK + kb * 16384, &tmQKV, d + h * DH + kb * 64, row_base, bar(1));
+            tma_load_2d(sbase + L::kV + kb * 16384, &tmQKV, 2 * d + h * DH + kb * 64, row_base, bar(5));
+        }
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_slot), 512);
@@ -88,13 +101,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
 
     if (warp == 0) {
         if (lane == 0) {
-            const int nq = hasB ? 2 : 1;
-            mbar_arrive_expect_tx(bar(0), nq * L::kTile);
-            for (int t = 0; t < nq; ++t)
-                for (int kb = 0; kb < L::kBlocks; ++kb)
-                    tma_load_2d(sbase + L::kQ + t * L::kTile + kb * 16384, &tmQKV, h * DH + kb * 64,
-                                row_base + q0A + t * 128, bar(0));
-            for (int j = 0; j < n_kv; ++j) {
+            for (int j = 1; j < n_kv; ++j) {                // Q and key tile 0 were requested in the prologue
                 const int s = j & 1, ph = (j >> 1) & 1;
                 if (!mbar_wait(bar(3 + s), ph ^ 1, abort_flag, p.status, 400)) break;
                 mbar_arrive_expect_tx(bar(1 + s), L::kTile);
@@ -114,22 +121,25 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
             constexpr uint32_t idesc_pv = make_idesc_bf16(128, DH, false, true);
             // S_t = Q_t K^T from K stage s
             auto issue_s = [&](int t, int s) {
-                const uint32_t qa = sbase + L::kQ + t * L::kTile, ka = sbase + L::kK + s * L::kTile;
+                const uint64_t dq = make_smem_desc_sw128(sbase + L::kQ + t * L::kTile, 16, 1024);
+                const uint64_t dk = make_smem_desc_sw128(sbase + L::kK + s * L::kTile, 16, 1024);
+                const uint32_t dst = tmem_base + t * 128;
 #pragma unroll
                 for (int kb = 0; kb < L::kBlocks; ++kb)
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
-                        umma_f16(tmem_base + t * 128, make_smem_desc_sw128(qa + kb * 16384 + kk * 32, 16, 1024),
-                                 make_smem_desc_sw128(ka + kb * 16384 + kk * 32, 16, 1024), idesc_s, (kb | kk) ? 1u : 0u);
+                        umma_f16(dst, desc_advance(dq, kb * 16384 + kk * 32), desc_advance(dk, kb * 16384 + kk * 32),
+                                 idesc_s, (kb | kk) ? 1u : 0u);
                 umma_commit(bar(9 + t));
             };
             // O_t (+)= P_t V from V stage s; P_t is bf16 packed in the first 64 columns of S_t
             auto issue_pv = [&](int t, int s, bool acc) {
-                const uint32_t va = sbase + L::kV + s * L::kTile;
+                const uint64_t dv = make_smem_desc_sw128(sbase + L::kV + s * L::kTile, 16384, 1024);
+                const uint32_t dst = tmem_base + 256 + t * 128, src = tmem_base + t * 128;
+                umma_f16_ta(dst, src, dv, idesc_pv, acc ? 1u : 0u);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    umma_f16_ta(tmem_base + 256 + t * 128, tmem_base + t * 128 + ks * 8,
-                                make_smem_desc_sw128(va + ks * 2048, 16384, 1024), idesc_pv, (acc || ks) ? 1u : 0u);
+                for (int ks = 1; ks < 8; ++ks)
+                    umma_f16_ta(dst, src + ks * 8, desc_advance(dv, ks * 2048), idesc_pv, 1u);
             };
             bool ok = mbar_wait(bar(0), 0, abort_flag, p.status, 410) && mbar_wait(bar(1), 0, abort_flag, p.status, 411);
             if (ok) {

@@ -350,6 +350,11 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t saddr, uint32_
     return d;
 }
 
+// Descriptor of the same operand starting `bytes` further on (bytes a multiple of 16, the new
+// start still inside the 256 KB shared-memory window, so the add never carries out of the
+// address field).  Lets the MMA-issuing thread build a descriptor once and step it with one add.
+__device__ __forceinline__ uint64_t desc_advance(uint64_t d, uint32_t bytes) { return d + (bytes >> 4); }
+
 // Instruction descriptor for kind::f16 with bf16 A/B and fp32 D.
 //   [4,6) D format (1 = f32)  [7,10) A format (1 = bf16)  [10,13) B format (1 = bf16)
 //   bit 15 A major (1 = MN-major)  bit 16 B major  [17,23) N >> 3  [24,29) M >> 4
