@@ -36,12 +36,15 @@ struct GemmParams {
     const __nv_bfloat16* aux_in; int ld_aux;
     int accumulate, act;
     int m_tiles, n_tiles;
+    int n_fastest;               // tile numbering: 1 = consecutive tiles share the A row panel, 0 = the B panel
     int split_begin;             // tiles >= split_begin are issued as two half-width tiles (tail balancing)
     int total_virtual;           // split_begin + 2 * (m_tiles*n_tiles - split_begin)
     DeviceStatus* status;
 };
 
-// Virtual tile v -> (m0, n0, width).  Full tiles are numbered m-fastest; the tiles of the last,
+// Virtual tile v -> (m0, n0, width).  Tiles that run at the same time should touch as few distinct
+// operand panels as possible (they have to sit in L2 together), so the numbering runs fastest along
+// the dimension with fewer tiles.  The tiles of the last,
 // partly filled round are cut in two half-width tiles so that every SM gets one.
 __device__ __forceinline__ void tile_info(const GemmParams& p, int v, int& m0, int& n0, int& bn)
 {
@@ -53,8 +56,10 @@ __device__ __forceinline__ void tile_info(const GemmParams& p, int v, int& m0, i
         half = hv & 1;
         bn = p.bn >> 1;
     }
-    m0 = (t % p.m_tiles) * BM;
-    n0 = (t / p.m_tiles) * p.bn + half * (p.bn >> 1);
+    const int mi = p.n_fastest ? t / p.n_tiles : t % p.m_tiles;
+    const int ni = p.n_fastest ? t % p.n_tiles : t / p.m_tiles;
+    m0 = mi * BM;
+    n0 = ni * p.bn + half * (p.bn >> 1);
 }
 
 // One 8-column group of the bf16 epilogues: f = acc (+bias) (+residual | x GeLU'(u)).
@@ -374,8 +379,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             bool ok = true;
             const uint32_t pair_tx = 2u * (A_TILE_BYTES + half_n * BK * 2);
             for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs) {
-                const int m0 = (tile % p.m_tiles) * 256 + rank * 128;
-                const int n0 = (tile / p.m_tiles) * bn + rank * half_n;
+                const int mi = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles;
+                const int ni = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
+                const int m0 = mi * 256 + rank * 128;
+                const int n0 = ni * bn + rank * half_n;
                 for (int kb = 0; kb < num_k; ++kb) {
                     if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 700)) { ok = false; break; }
                     const uint32_t fb = mapa_shared(full0 + 8 * stage, 0);     // the leader's barrier
@@ -430,7 +437,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const uint32_t slab_u32 = smem_u32(slab);
         uint32_t it = 0, nout = 0;
         for (int tile = pair_id; tile < total_tiles; tile += n_pairs, ++it) {
-            const int m0 = (tile % p.m_tiles) * 256 + rank * 128, n0 = (tile / p.m_tiles) * bn;
+            const int mi = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles;
+            const int ni = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
+            const int m0 = mi * 256 + rank * 128, n0 = ni * bn;
             const uint32_t buf = it & 1, acc_phase = (it >> 1) & 1;
             bool ok = mbar_wait(accf0 + 8 * buf, acc_phase, abort_flag, p.status, 720);
             ok = __all_sync(0xffffffffu, ok);
@@ -559,6 +568,7 @@ static const char* launch_gemm_pair(Runtime* rt, const GemmArgs& a, DeviceStatus
     p.accumulate = a.accumulate; p.act = a.act;
     p.m_tiles = m_tiles; p.n_tiles = (a.N + bn - 1) / bn;
     p.split_begin = p.m_tiles * p.n_tiles; p.total_virtual = p.split_begin;
+    p.n_fastest = p.n_tiles < p.m_tiles ? 1 : 0;
     p.status = status;
     const int key = a.layout * 16 + a.epilogue;
     switch (key) {
@@ -626,6 +636,7 @@ const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cu
     p.aux_in = static_cast<const __nv_bfloat16*>(a.aux_in); p.ld_aux = a.ld_aux;
     p.accumulate = a.accumulate; p.act = a.act;
     p.m_tiles = m_tiles; p.n_tiles = (a.N + bn - 1) / bn;
+    p.n_fastest = p.n_tiles < p.m_tiles ? 1 : 0;
     p.status = status;
     {
         // Tail balancing: when the last round would leave at least half of the SMs idle, its
