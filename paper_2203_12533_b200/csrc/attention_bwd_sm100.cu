@@ -184,13 +184,14 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
         bool ok = true;
         for (int i = 0; i < n_u; ++i) {
             const int hb = i & 1, qc0 = (u0 + i) * 64 + ch * 32;   // first query column of this thread's slice
-            float l2[32], dl[32];
+            // -lse*log2e and -delta of this slice's 32 queries, as two-wide operands
+            uint64_t nl2[16], ndl[16];
 #pragma unroll
             for (int g = 0; g < 8; ++g) {
                 const float4 a = __ldg(reinterpret_cast<const float4*>(lse_row + qc0) + g);
                 const float4 c = __ldg(reinterpret_cast<const float4*>(dl_row + qc0) + g);
-                l2[4 * g] = a.x * kLog2e; l2[4 * g + 1] = a.y * kLog2e; l2[4 * g + 2] = a.z * kLog2e; l2[4 * g + 3] = a.w * kLog2e;
-                dl[4 * g] = c.x; dl[4 * g + 1] = c.y; dl[4 * g + 2] = c.z; dl[4 * g + 3] = c.w;
+                nl2[2 * g] = pack_f32x2(-a.x * kLog2e, -a.y * kLog2e); nl2[2 * g + 1] = pack_f32x2(-a.z * kLog2e, -a.w * kLog2e);
+                ndl[2 * g] = pack_f32x2(-c.x, -c.y); ndl[2 * g + 1] = pack_f32x2(-c.z, -c.w);
             }
             ok = mbar_wait(bar(9 + hb), (i >> 1) & 1, abort_flag, p.status, 520);
             ok = __all_sync(0xffffffffu, ok);
@@ -202,16 +203,18 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
             tc_wait_ld();
             const bool diag = qc0 < kv0 + 128;               // some (key, query) pairs of this slice are masked
             uint32_t pp[16], dd[16];
+            const uint64_t sl2x2 = pack_f32x2(sl2, sl2);
 #pragma unroll
             for (int c = 0; c < 32; c += 2) {
-                float p0 = ex2_approx(fmaf(__uint_as_float(sv[c]), sl2, -l2[c]));
-                float p1 = ex2_approx(fmaf(__uint_as_float(sv[c + 1]), sl2, -l2[c + 1]));
+                float a0, a1, d0, d1;
+                unpack_f32x2(ffma2(pack_f32x2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), sl2x2, nl2[c >> 1]), a0, a1);
+                float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
                 if (diag) {
                     if (qc0 + c < kv0 + r) p0 = 0.f;
                     if (qc0 + c + 1 < kv0 + r) p1 = 0.f;
                 }
-                const float d0 = p0 * (__uint_as_float(dv[c]) - dl[c]);
-                const float d1 = p1 * (__uint_as_float(dv[c + 1]) - dl[c + 1]);
+                const uint64_t pv = pack_f32x2(p0, p1);
+                unpack_f32x2(fmul2(pv, fadd2(pack_f32x2(__uint_as_float(dv[c]), __uint_as_float(dv[c + 1])), ndl[c >> 1])), d0, d1);
                 pp[c >> 1] = pack_bf16(p0, p1);
                 dd[c >> 1] = pack_bf16(d0, d1);
             }
@@ -451,6 +454,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
             if (!ok) break;
             tc_fence_after();
             const bool diag = v * 64 + 63 > q0;              // some keys of this sub-tile are masked for some rows
+            const uint64_t sl2x2 = pack_f32x2(sl2, sl2), nlse2 = pack_f32x2(-lse2, -lse2), ndlt = pack_f32x2(-dlt, -dlt);
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 uint32_t sv[32], dv[32], ds[16];
@@ -459,14 +463,16 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
                 tc_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                    float p0 = ex2_approx(fmaf(__uint_as_float(sv[i]), sl2, -lse2));
-                    float p1 = ex2_approx(fmaf(__uint_as_float(sv[i + 1]), sl2, -lse2));
+                    float a0, a1, d0, d1;
+                    unpack_f32x2(ffma2(pack_f32x2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), sl2x2, nlse2), a0, a1);
+                    float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
                     if (diag) {
                         const int key = v * 64 + c * 32 + i;
                         if (key > q0 + r) p0 = 0.f;
                         if (key + 1 > q0 + r) p1 = 0.f;
                     }
-                    ds[i >> 1] = pack_bf16(p0 * (__uint_as_float(dv[i]) - dlt), p1 * (__uint_as_float(dv[i + 1]) - dlt));
+                    unpack_f32x2(fmul2(pack_f32x2(p0, p1), fadd2(pack_f32x2(__uint_as_float(dv[i]), __uint_as_float(dv[i + 1])), ndlt)), d0, d1);
+                    ds[i >> 1] = pack_bf16(d0, d1);
                 }
                 tmem_st16(s_addr + c * 16, ds);
             }

@@ -201,15 +201,20 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, v + c * 32);
             tc_wait_ld();
-            float mx = -INFINITY;
+            // row maximum: eight independent chains of three-input max (64 instructions for 128 scores)
+            float mxs[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) mxs[k] = -INFINITY;
             if (diag) {
 #pragma unroll
                 for (int i = 0; i < 128; ++i)
-                    if (i <= r) mx = fmaxf(mx, __uint_as_float(v[i]));
+                    if (i <= r) mxs[i & 7] = fmaxf(mxs[i & 7], __uint_as_float(v[i]));
             } else {
 #pragma unroll
-                for (int i = 0; i < 128; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+                for (int i = 0; i < 128; i += 2)
+                    mxs[(i >> 1) & 7] = fmax3(mxs[(i >> 1) & 7], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
             }
+            const float mx = fmaxf(fmax3(mxs[0], mxs[1], mxs[2]), fmax3(fmaxf(mxs[3], mxs[4]), fmaxf(mxs[5], mxs[6]), mxs[7]));
             const float m_new = fmaxf(m_used, mx);
             const bool grow = (m_new - m_used) * sl2 > 8.0f;        // also true on the first tile (m_used = -inf)
             if (j == 0) {
@@ -230,19 +235,32 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
             }
             // p = exp2((s - m) * scale * log2e), packed bf16 written over the S columns
             const float mb = m_used * sl2;
-            float ls = 0.f;
+            if (diag) {
+                float ls = 0.f;
 #pragma unroll
-            for (int i = 0; i < 128; i += 2) {
-                float p0 = ex2_approx(fmaf(__uint_as_float(v[i]), sl2, -mb));
-                float p1 = ex2_approx(fmaf(__uint_as_float(v[i + 1]), sl2, -mb));
-                if (diag) {
-                    if (i > r) p0 = 0.f;
-                    if (i + 1 > r) p1 = 0.f;
+                for (int i = 0; i < 128; i += 2) {
+                    float p0 = i > r ? 0.f : ex2_approx(fmaf(__uint_as_float(v[i]), sl2, -mb));
+                    float p1 = i + 1 > r ? 0.f : ex2_approx(fmaf(__uint_as_float(v[i + 1]), sl2, -mb));
+                    ls += p0 + p1;
+                    v[i >> 1] = pack_bf16(p0, p1);
                 }
-                ls += p0 + p1;
-                v[i >> 1] = pack_bf16(p0, p1);
+                l += ls;
+            } else {
+                // two scores per FMA / add instruction; the exponentials stay on the MUFU
+                const uint64_t sl2x2 = pack_f32x2(sl2, sl2), mbx2 = pack_f32x2(-mb, -mb);
+                uint64_t lsum[4] = {0ull, 0ull, 0ull, 0ull};
+#pragma unroll
+                for (int i = 0; i < 128; i += 2) {
+                    float a0, a1;
+                    unpack_f32x2(ffma2(pack_f32x2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), sl2x2, mbx2), a0, a1);
+                    const float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
+                    lsum[(i >> 1) & 3] = fadd2(lsum[(i >> 1) & 3], pack_f32x2(p0, p1));
+                    v[i >> 1] = pack_bf16(p0, p1);
+                }
+                float s0, s1;
+                unpack_f32x2(fadd2(fadd2(lsum[0], lsum[1]), fadd2(lsum[2], lsum[3])), s0, s1);
+                l += s0 + s1;
             }
-            l += ls;
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_st16(s_addr + c * 16, v + c * 16);
             tc_wait_st();
