@@ -88,7 +88,7 @@ __device__ __forceinline__ void epilogue_group(const uint32_t* v, int row, int c
                 float u[8];
                 unpack8(*reinterpret_cast<const uint4*>(p.aux_in + static_cast<size_t>(row) * p.ld_aux + c), u);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) f[j] *= gelu_grad_f(u[j], p.act);
+                for (int j = 0; j < 8; j += 2) gelu_grad_mul2(f[j], f[j + 1], u[j], u[j + 1], p.act);
             }
         }
     }
@@ -151,7 +151,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, 
                     // exactly the argument the forward used
                     unpack8(o[g], f);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) f[j] = gelu_f(f[j], p.act);
+                    for (int j = 0; j < 8; j += 2) gelu2(f[j], f[j + 1], p.act);
                     o2[g] = pack8(f);
                 }
             }

@@ -400,4 +400,42 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, bool a_mn_m
            (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
 }
 
+// GeLU / GeLU' of two values at once (erf form): the polynomial and scaling steps run as two-wide
+// fp32 instructions, the reciprocal and the exponential stay one MUFU op per value.
+//   half_tail = erfc(|u|/sqrt2)/2 = (b1 t + ... + b5 t^5) exp(-u^2/2),  t = 1/(1 + p|u|/sqrt2),  b = a/2
+__device__ __forceinline__ void normal_cdf_pdf2(float u0, float u1, uint64_t& cdf, uint64_t& e)
+{
+    const float au0 = fabsf(u0), au1 = fabsf(u1);
+    const uint64_t au = pack_f32x2(au0, au1);
+    float d0, d1, x0, x1;
+    unpack_f32x2(ffma2(au, pack_f32x2(0.23164189f, 0.23164189f), pack_f32x2(1.0f, 1.0f)), d0, d1);      // 1 + p |u| / sqrt2
+    unpack_f32x2(fmul2(fmul2(au, au), pack_f32x2(-0.72134752f, -0.72134752f)), x0, x1);                    // -u^2/2 * log2(e)
+    const uint64_t t = pack_f32x2(__frcp_rn(d0), __frcp_rn(d1));
+    e = pack_f32x2(ex2_approx(x0), ex2_approx(x1));
+    uint64_t poly = ffma2(t, pack_f32x2(0.5307027145f, 0.5307027145f), pack_f32x2(-0.7265760135f, -0.7265760135f));
+    poly = ffma2(t, poly, pack_f32x2(0.7107068705f, 0.7107068705f));
+    poly = ffma2(t, poly, pack_f32x2(-0.142248368f, -0.142248368f));
+    poly = ffma2(t, poly, pack_f32x2(0.127414796f, 0.127414796f));
+    const uint64_t ht = fmul2(fmul2(poly, t), e);
+    float h0, h1;
+    unpack_f32x2(ht, h0, h1);
+    cdf = pack_f32x2(u0 < 0.f ? h0 : 1.0f - h0, u1 < 0.f ? h1 : 1.0f - h1);
+}
+__device__ __forceinline__ void gelu2(float& u0, float& u1, int act)
+{
+    if (act == 1) { u0 = gelu_f(u0, 1); u1 = gelu_f(u1, 1); return; }
+    uint64_t cdf, e;
+    normal_cdf_pdf2(u0, u1, cdf, e);
+    unpack_f32x2(fmul2(pack_f32x2(u0, u1), cdf), u0, u1);
+}
+// g0, g1 *= GeLU'(u0), GeLU'(u1)
+__device__ __forceinline__ void gelu_grad_mul2(float& g0, float& g1, float u0, float u1, int act)
+{
+    if (act == 1) { g0 *= gelu_grad_f(u0, 1); g1 *= gelu_grad_f(u1, 1); return; }
+    uint64_t cdf, e;
+    normal_cdf_pdf2(u0, u1, cdf, e);
+    const uint64_t up = fmul2(pack_f32x2(u0, u1), pack_f32x2(0.3989422804f, 0.3989422804f));
+    unpack_f32x2(fmul2(pack_f32x2(g0, g1), ffma2(up, e, cdf)), g0, g1);
+}
+
 }  // namespace pw
