@@ -130,6 +130,14 @@ def test_layer_argument_errors(pw):
     assert layer.status() == (0, 0)
 
 
+@pytest.mark.parametrize("d,H,F,S", [(4096, 32, 16384, 256), (8192, 64, 32768, 128)], ids=["cfg3_width", "cfg4_width"])
+def test_wide_layers_at_reduced_token_count(pw, oracle32, d, H, F, S):
+    """The layer widths of workloads 3 and 4 (d = 4096 / 8192, 128-wide heads) on fewer tokens."""
+    sigma = 0.01 if d == 8192 else 0.02
+    w = inputs.Workload("wide", d, H, 128, F, S, 2 if d == 4096 else 1, sigma_w=sigma)
+    check_layer_against_oracle(pw, oracle32, w)
+
+
 # ------------------------------------------------------------------------------------------ stage chain
 def run_chain_gpu(pw, w, L, M, dispatch, schedule, recompute, seed=0):
     stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
