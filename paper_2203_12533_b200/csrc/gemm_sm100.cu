@@ -98,7 +98,7 @@ __device__ __forceinline__ void epilogue_group(const uint32_t* v, int row, int c
 // store (rows >= M and columns >= N are clipped by the tensor map).  `taddr` addresses this warp's
 // lane quarter of the accumulator, row0 is the first of its 32 rows, pi selects which of the two
 // warps of the quarter it is (they take alternate column chunks).
-template <int EPI>
+template <int EPI, bool SINGLE_SLAB = false>
 __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, int bn, int pi, int pstride, int lane,
                                               uint8_t* slab, uint32_t slab_u32, uint32_t& nout, const CUtensorMap* tmC,
                                               const CUtensorMap* tmAux, const GemmParams& p)
@@ -158,8 +158,8 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, 
             constexpr int kOuts = (EPI == kEpiBiasGelu) ? 2 : 1;
 #pragma unroll
             for (int t = 0; t < kOuts; ++t) {
-                const uint32_t half = (nout++ & 1u) * 2048u;
-                if (lane == 0) bulk_wait_read1();
+                const uint32_t half = SINGLE_SLAB ? 0u : (nout++ & 1u) * 2048u;
+                if (lane == 0) { if (SINGLE_SLAB) bulk_wait_read0(); else bulk_wait_read1(); }
                 __syncwarp();
 #pragma unroll
                 for (int g = 0; g < 4; ++g)
@@ -322,13 +322,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 // acc_full[b] (one in each CTA, signalled by the leader's tcgen05.commit to both), acc_empty[b]
 // (leader, one arrival per epilogue warp of both CTAs).
 // The epilogues that evaluate GeLU / GeLU' are instruction-bound with 8 warps (two per scheduler),
-// so those instantiations run 16 epilogue warps and give up one pipeline stage for their slabs.
+// so those instantiations run 16 epilogue warps and use one 2 KB output slab per warp instead of two.
 constexpr int P_STAGE_BYTES = 32768;            // A: 128 x 64 (16 KB) + B half: up to 128 x 64 (16 KB)
 template <int EPI> struct PairCfg {
     static constexpr int kEpiWarps = (EPI == kEpiBiasGelu || EPI == kEpiDGelu) ? 16 : 8;
-    static constexpr int kStages = kEpiWarps == 16 ? 5 : 6;
+    static constexpr int kStages = 6;
+    static constexpr int kSlab = kEpiWarps == 16 ? 2048 : SLAB_BYTES;   // 16 warps: one 2 KB slab each, no ping-pong
     static constexpr int kThreads = 64 + 32 * kEpiWarps;
-    static constexpr int kSmem = kStages * P_STAGE_BYTES + kEpiWarps * SLAB_BYTES + 1024 + 256;
+    static constexpr int kSmem = kStages * P_STAGE_BYTES + kEpiWarps * kSlab + 1024 + 256;
 };
 
 template <bool A_MN, bool B_MN, int EPI>
@@ -340,7 +341,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* slabs = tiles + P_STAGES * P_STAGE_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(slabs + NEPI * SLAB_BYTES);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(slabs + NEPI * PairCfg<EPI>::kSlab);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + P_STAGES);
     const uint32_t accf0 = smem_u32(bars + 2 * P_STAGES), acce0 = smem_u32(bars + 2 * P_STAGES + 2);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * P_STAGES + 4);
@@ -433,7 +434,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
     } else {
         const int q = warp & 3, pi = (warp - 2) >> 2;
-        uint8_t* slab = slabs + (warp - 2) * SLAB_BYTES;
+        uint8_t* slab = slabs + (warp - 2) * PairCfg<EPI>::kSlab;
         const uint32_t slab_u32 = smem_u32(slab);
         uint32_t it = 0, nout = 0;
         for (int tile = pair_id; tile < total_tiles; tile += n_pairs, ++it) {
@@ -446,7 +447,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * BN_MAX;
-            epilogue_tile<EPI>(taddr, m0 + q * 32, n0, bn, pi, NEPI / 4, lane, slab, slab_u32, nout, &tmC, &tmAux, p);
+            epilogue_tile<EPI, NEPI == 16>(taddr, m0 + q * 32, n0, bn, pi, NEPI / 4, lane, slab, slab_u32, nout, &tmC, &tmAux, p);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_shared(acce0 + 8 * buf, 0));
