@@ -16,12 +16,14 @@ namespace {
 // Each thread handles four 16-byte pieces that are a whole block stride apart (all eight loads
 // are issued before any is used); the dh/8 threads of a (token, head) group reduce by shuffles.
 __global__ void __launch_bounds__(256)
-attn_delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ dout,
-                  float* __restrict__ delta, int B, int S, int H, int dh)
+attn_delta_kernel(const __nv_bfloat16* o, const __nv_bfloat16* dout,
+                  float* delta, int B, int S, int H, int dh)
 {
     const int per_head = dh / 8;                             // threads per (token, head): 8 or 16
     const size_t total = static_cast<size_t>(B) * S * H * per_head;
     const size_t base = static_cast<size_t>(blockIdx.x) * 1024 + threadIdx.x;
+    grid_dep_launch();
+    grid_dep_wait();
     uint4 a[4], g[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
@@ -59,9 +61,9 @@ const char* launch_attention_bwd(Runtime* rt, const void* qkv, const void* o, co
     if (B <= 0 || H <= 0 || S <= 0 || (S % 128) != 0 || (dh != 64 && dh != 128)) return "attention: unsupported shape";
     {
         const size_t total = static_cast<size_t>(B) * S * H * (dh / 8);
-        attn_delta_kernel<<<static_cast<unsigned>((total + 1023) / 1024), 256, 0, stream>>>(
-            static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(dout), static_cast<float*>(delta), B, S, H, dh);
-        if (cudaGetLastError() != cudaSuccess) return "attention delta launch failed";
+        if (launch_k(attn_delta_kernel, dim3(static_cast<unsigned>((total + 1023) / 1024)), dim3(256), 0, stream,
+                     static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(dout), static_cast<float*>(delta), B, S, H, dh) != cudaSuccess)
+            return "attention delta launch failed";
     }
     if (const char* e = launch_attention_bwd_dq(rt, qkv, dout, lse, delta, B, S, H, dh, dqkv, status, stream)) return e;
     return launch_attention_bwd_dkdv(rt, qkv, dout, lse, delta, B, S, H, dh, dqkv, status, stream);

@@ -79,6 +79,10 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
         fence_barrier_init();
         fence_proxy_async();
         prefetch_tmap(&tmKV); prefetch_tmap(&tmQ); prefetch_tmap(&tmDO); prefetch_tmap(&tmOut);
+    }
+    grid_dep_launch();
+    grid_dep_wait();                                        // inputs come from the previous kernels
+    if (threadIdx.x == 0) {
         // first loads go out before the TMEM allocation and the CTA-wide barrier
         mbar_arrive_expect_tx(bar(0), 2 * L::kKV);
         for (int kb = 0; kb < L::kBlocks; ++kb) {
@@ -188,8 +192,8 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
             uint64_t nl2[16], ndl[16];
 #pragma unroll
             for (int g = 0; g < 8; ++g) {
-                const float4 a = __ldg(reinterpret_cast<const float4*>(lse_row + qc0) + g);
-                const float4 c = __ldg(reinterpret_cast<const float4*>(dl_row + qc0) + g);
+                const float4 a = *(reinterpret_cast<const float4*>(lse_row + qc0) + g);
+                const float4 c = *(reinterpret_cast<const float4*>(dl_row + qc0) + g);
                 nl2[2 * g] = pack_f32x2(-a.x * kLog2e, -a.y * kLog2e); nl2[2 * g + 1] = pack_f32x2(-a.z * kLog2e, -a.w * kLog2e);
                 ndl[2 * g] = pack_f32x2(-c.x, -c.y); ndl[2 * g + 1] = pack_f32x2(-c.z, -c.w);
             }
@@ -327,6 +331,10 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
         fence_barrier_init();
         fence_proxy_async();
         prefetch_tmap(&tmQ); prefetch_tmap(&tmDO); prefetch_tmap(&tmKV); prefetch_tmap(&tmOut);
+    }
+    grid_dep_launch();
+    grid_dep_wait();                                        // inputs come from the previous kernels
+    if (threadIdx.x == 0) {
         // first loads go out before the TMEM allocation and the CTA-wide barrier
         const int nq = hasB ? 2 : 1;
         mbar_arrive_expect_tx(bar(0), nq * 2 * L::kTile);
@@ -573,9 +581,10 @@ const char* launch_attention_bwd_dq(Runtime* rt, const void* qkv, const void* do
     p.lse = static_cast<const float*>(lse); p.delta = static_cast<const float*>(delta);
     p.status = status;
     dim3 grid((S + 255) / 256, B * H);
-    if (dh == 64) attn_bwd_dq_tc_kernel<64><<<grid, kThreads, DqSmem<64>::kBytes, stream>>>(tmQ, tmDO, tmKV, tmOut, p);
-    else attn_bwd_dq_tc_kernel<128><<<grid, kThreads, DqSmem<128>::kBytes, stream>>>(tmQ, tmDO, tmKV, tmOut, p);
-    return cudaGetLastError() == cudaSuccess ? nullptr : "attention bwd (dq) launch failed";
+    const cudaError_t e2 = dh == 64
+        ? launch_k(attn_bwd_dq_tc_kernel<64>, grid, dim3(kThreads), DqSmem<64>::kBytes, stream, tmQ, tmDO, tmKV, tmOut, p)
+        : launch_k(attn_bwd_dq_tc_kernel<128>, grid, dim3(kThreads), DqSmem<128>::kBytes, stream, tmQ, tmDO, tmKV, tmOut, p);
+    return e2 == cudaSuccess ? nullptr : "attention bwd (dq) launch failed";
 }
 
 // dK and dV parts of dqkv.  lse, delta: fp32 [B,H,S].
@@ -595,9 +604,10 @@ const char* launch_attention_bwd_dkdv(Runtime* rt, const void* qkv, const void* 
     p.lse = static_cast<const float*>(lse); p.delta = static_cast<const float*>(delta);
     p.status = status;
     dim3 grid(S / 128, B * H);
-    if (dh == 64) attn_bwd_dkdv_tc_kernel<64><<<grid, kThreads, KvSmem<64>::kBytes, stream>>>(tmKV, tmQ, tmDO, tmOut, p);
-    else attn_bwd_dkdv_tc_kernel<128><<<grid, kThreads, KvSmem<128>::kBytes, stream>>>(tmKV, tmQ, tmDO, tmOut, p);
-    return cudaGetLastError() == cudaSuccess ? nullptr : "attention bwd (dk, dv) launch failed";
+    const cudaError_t e2 = dh == 64
+        ? launch_k(attn_bwd_dkdv_tc_kernel<64>, grid, dim3(kThreads), KvSmem<64>::kBytes, stream, tmKV, tmQ, tmDO, tmOut, p)
+        : launch_k(attn_bwd_dkdv_tc_kernel<128>, grid, dim3(kThreads), KvSmem<128>::kBytes, stream, tmKV, tmQ, tmDO, tmOut, p);
+    return e2 == cudaSuccess ? nullptr : "attention bwd (dk, dv) launch failed";
 }
 
 }  // namespace pw

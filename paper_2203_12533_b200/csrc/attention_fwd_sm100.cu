@@ -76,6 +76,10 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
         fence_proxy_async();
         prefetch_tmap(&tmQKV);
         prefetch_tmap(&tmO);
+    }
+    grid_dep_launch();
+    grid_dep_wait();                                        // qkv comes from the previous kernel
+    if (threadIdx.x == 0) {
         // first loads go out before the TMEM allocation and the CTA-wide barrier
         const int nq = hasB ? 2 : 1;
         mbar_arrive_expect_tx(bar(0), nq * L::kTile);
@@ -357,9 +361,10 @@ const char* launch_attention_fwd(Runtime* rt, const void* qkv, int B, int S, int
     p.lse = static_cast<float*>(lse);
     p.status = status;
     dim3 grid((S + 255) / 256, B * H);
-    if (dh == 64) attn_fwd_tc_kernel<64><<<grid, kThreads, FwdSmem<64>::kBytes, stream>>>(tmQKV, tmO, p);
-    else attn_fwd_tc_kernel<128><<<grid, kThreads, FwdSmem<128>::kBytes, stream>>>(tmQKV, tmO, p);
-    return cudaGetLastError() == cudaSuccess ? nullptr : "attention fwd launch failed";
+    const cudaError_t e2 = dh == 64
+        ? launch_k(attn_fwd_tc_kernel<64>, grid, dim3(kThreads), FwdSmem<64>::kBytes, stream, tmQKV, tmO, p)
+        : launch_k(attn_fwd_tc_kernel<128>, grid, dim3(kThreads), FwdSmem<128>::kBytes, stream, tmQKV, tmO, p);
+    return e2 == cudaSuccess ? nullptr : "attention fwd launch failed";
 }
 
 }  // namespace pw

@@ -44,9 +44,9 @@ __device__ __forceinline__ float warp_sum(float v)
 // hop when W > 1).  256-thread CTAs hold 8/W rows.
 template <int CH>
 __global__ void __launch_bounds__(kRowThreadsMax)
-ln_fwd_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gamma,
-              const __nv_bfloat16* __restrict__ beta, int T, int d, float eps, __nv_bfloat16* __restrict__ h,
-              float* __restrict__ mu, float* __restrict__ rstd, int W)
+ln_fwd_kernel(const __nv_bfloat16* x, const __nv_bfloat16* gamma,
+              const __nv_bfloat16* beta, int T, int d, float eps, __nv_bfloat16* h,
+              float* mu, float* rstd, int W)
 {
     __shared__ float red[2][kMaxWarps];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -54,6 +54,8 @@ ln_fwd_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restri
     const int row_in_cta = warp / W, wr = warp % W;
     const int row = blockIdx.x * rows_per_cta + row_in_cta;
     const bool live = row < T && row_in_cta < rows_per_cta;
+    grid_dep_launch();
+    grid_dep_wait();
     float v[CH][8];
     float s = 0.f;
 #pragma unroll
@@ -90,8 +92,8 @@ ln_fwd_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restri
     for (int j = 0; j < CH; ++j) {
         const int col = 8 * (lane + 32 * (wr + W * j));
         float g[8], b[8], o[8];
-        unpack8(__ldg(reinterpret_cast<const uint4*>(gamma + col)), g);
-        unpack8(__ldg(reinterpret_cast<const uint4*>(beta + col)), b);
+        unpack8(*(reinterpret_cast<const uint4*>(gamma + col)), g);
+        unpack8(*(reinterpret_cast<const uint4*>(beta + col)), b);
 #pragma unroll
         for (int k = 0; k < 8; ++k) o[k] = g[k] * ((v[j][k] - mean) * r) + b[k];
         *reinterpret_cast<uint4*>(h + static_cast<size_t>(row) * d + col) = pack8(o);
@@ -116,19 +118,21 @@ bool plan_warp_rows(int d, int* W, int* CH)
 // sums share one barrier.
 template <int CHUNKS>
 __global__ void __launch_bounds__(kRowThreadsMax, CHUNKS == 1 ? 2 : 1)
-ln_bwd_kernel(const __nv_bfloat16* __restrict__ dh, const __nv_bfloat16* __restrict__ x,
-              const float* __restrict__ mu, const float* __restrict__ rstd, const __nv_bfloat16* __restrict__ gamma,
+ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
+              const float* mu, const float* rstd, const __nv_bfloat16* gamma,
               const __nv_bfloat16* resid, int T, int d, __nv_bfloat16* dx,
-              float* __restrict__ partials, int tpr, int rows_per_cta)
+              float* partials, int tpr, int rows_per_cta)
 {
     __shared__ float red[2][2][kMaxWarps];
     const int row_in_cta = threadIdx.x / tpr, tr = threadIdx.x % tpr;
     const int wpr = tpr >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    grid_dep_launch();
+    grid_dep_wait();
     float gm[CHUNKS][8];
     float acc_g[CHUNKS][8], acc_b[CHUNKS][8], acc_r[CHUNKS][8], acc_x[CHUNKS][8];
 #pragma unroll
     for (int j = 0; j < CHUNKS; ++j) {
-        unpack8(__ldg(reinterpret_cast<const uint4*>(gamma + 8 * (tr + j * tpr))), gm[j]);
+        unpack8(*(reinterpret_cast<const uint4*>(gamma + 8 * (tr + j * tpr))), gm[j]);
 #pragma unroll
         for (int k = 0; k < 8; ++k) acc_g[j][k] = acc_b[j][k] = acc_r[j][k] = acc_x[j][k] = 0.f;
     }
@@ -219,13 +223,15 @@ ln_bwd_kernel(const __nv_bfloat16* __restrict__ dh, const __nv_bfloat16* __restr
 // result does not depend on scheduling.  Up to 4 outputs (grid.y = quantity).
 struct ReduceOuts { float* out[4]; };
 __global__ void __launch_bounds__(1024)
-reduce_partials_kernel(const float* __restrict__ partials, int nrows, int nq, int n, ReduceOuts outs, int accumulate)
+reduce_partials_kernel(const float* partials, int nrows, int nq, int n, ReduceOuts outs, int accumulate)
 {
     __shared__ float sm[32][33];
     const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
     const int c = blockIdx.x * 32 + cx;
     const int q = blockIdx.y;
     float* out = outs.out[q];
+    grid_dep_launch();
+    grid_dep_wait();
     if (out == nullptr) return;
     float s = 0.f;
     if (c < n) {
@@ -246,9 +252,11 @@ reduce_partials_kernel(const float* __restrict__ partials, int nrows, int nq, in
 // eight rows are in flight per thread.
 constexpr int kColsumCols = 2048;
 __global__ void __launch_bounds__(256)
-colsum_kernel(const __nv_bfloat16* __restrict__ in, int T, int N, int ld, float* __restrict__ partials)
+colsum_kernel(const __nv_bfloat16* in, int T, int N, int ld, float* partials)
 {
     const int col = blockIdx.x * kColsumCols + threadIdx.x * 8;
+    grid_dep_launch();
+    grid_dep_wait();
     if (col >= N) return;
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     const int R = gridDim.y;
@@ -308,13 +316,14 @@ const char* launch_layernorm_fwd(Runtime* rt, const void* x, const void* gamma, 
     auto Hh = static_cast<__nv_bfloat16*>(h);
     auto Mu = static_cast<float*>(mu);
     auto Rs = static_cast<float*>(rstd);
-#define PW_LN_FWD(N) case N: ln_fwd_kernel<N><<<grid, kRowThreadsMax, 0, stream>>>(X, G, Bt, T, d, eps, Hh, Mu, Rs, W); break
+#define PW_LN_FWD(N) case N: le = launch_k(ln_fwd_kernel<N>, dim3(grid), dim3(kRowThreadsMax), 0, stream, X, G, Bt, T, d, eps, Hh, Mu, Rs, W); break
+    cudaError_t le = cudaSuccess;
     switch (CH) {
         PW_LN_FWD(1); PW_LN_FWD(2); PW_LN_FWD(3); PW_LN_FWD(4); PW_LN_FWD(5); PW_LN_FWD(6); PW_LN_FWD(7); PW_LN_FWD(8);
         default: return "layernorm: unsupported row width";
     }
 #undef PW_LN_FWD
-    return cudaGetLastError() == cudaSuccess ? nullptr : "layernorm fwd launch failed";
+    return le == cudaSuccess ? nullptr : "layernorm fwd launch failed";
 }
 
 size_t layernorm_bwd_scratch_bytes(Runtime* rt, int T, int d)
@@ -340,18 +349,19 @@ const char* launch_layernorm_bwd(Runtime* rt, const void* dh, const void* x, con
     auto Mu = static_cast<const float*>(mu);
     auto Rs = static_cast<const float*>(rstd);
     auto P = static_cast<float*>(partials);
+    cudaError_t le = cudaSuccess;
     switch (rp.chunks) {
-        case 1: ln_bwd_kernel<1><<<grid, rp.threads, 0, stream>>>(DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
-        case 2: ln_bwd_kernel<2><<<grid, rp.threads, 0, stream>>>(DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
-        default: ln_bwd_kernel<4><<<grid, rp.threads, 0, stream>>>(DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
+        case 1: le = launch_k(ln_bwd_kernel<1>, dim3(grid), dim3(rp.threads), 0, stream, DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
+        case 2: le = launch_k(ln_bwd_kernel<2>, dim3(grid), dim3(rp.threads), 0, stream, DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
+        default: le = launch_k(ln_bwd_kernel<4>, dim3(grid), dim3(rp.threads), 0, stream, DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
     }
-    if (cudaGetLastError() != cudaSuccess) return "layernorm bwd launch failed";
+    if (le != cudaSuccess) return "layernorm bwd launch failed";
     ReduceOuts outs;
     outs.out[0] = static_cast<float*>(dgamma); outs.out[1] = static_cast<float*>(dbeta);
     outs.out[2] = static_cast<float*>(db_resid); outs.out[3] = static_cast<float*>(db_dx);
     dim3 rgrid((d + 31) / 32, 4);
-    reduce_partials_kernel<<<rgrid, 1024, 0, stream>>>(P, grid * rp.rows_per_cta, 4, d, outs, accumulate);
-    return cudaGetLastError() == cudaSuccess ? nullptr : "layernorm bwd reduce launch failed";
+    return launch_k(reduce_partials_kernel, rgrid, dim3(1024), 0, stream, static_cast<const float*>(P), grid * rp.rows_per_cta, 4, d, outs, accumulate) == cudaSuccess
+               ? nullptr : "layernorm bwd reduce launch failed";
 }
 
 size_t colsum_scratch_bytes(Runtime* rt, int T, int N)
@@ -366,13 +376,13 @@ const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, voi
     if (T <= 0 || N <= 0 || (N % 8) || (ld % 8)) return "colsum: N and ld must be multiples of 8";
     const int R = colsum_splits(rt, T, N);
     dim3 grid((N + kColsumCols - 1) / kColsumCols, R);
-    colsum_kernel<<<grid, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(in), T, N, ld, static_cast<float*>(partials));
-    if (cudaGetLastError() != cudaSuccess) return "colsum launch failed";
+    if (launch_k(colsum_kernel, grid, dim3(256), 0, stream, static_cast<const __nv_bfloat16*>(in), T, N, ld, static_cast<float*>(partials)) != cudaSuccess)
+        return "colsum launch failed";
     ReduceOuts outs;
     outs.out[0] = static_cast<float*>(out); outs.out[1] = outs.out[2] = outs.out[3] = nullptr;
     dim3 rgrid((N + 31) / 32, 1);
-    reduce_partials_kernel<<<rgrid, 1024, 0, stream>>>(static_cast<const float*>(partials), R, 1, N, outs, accumulate);
-    return cudaGetLastError() == cudaSuccess ? nullptr : "colsum reduce launch failed";
+    return launch_k(reduce_partials_kernel, rgrid, dim3(1024), 0, stream, static_cast<const float*>(partials), R, 1, N, outs, accumulate) == cudaSuccess
+               ? nullptr : "colsum reduce launch failed";
 }
 
 // ---------------------------------------------------------------------------------------------

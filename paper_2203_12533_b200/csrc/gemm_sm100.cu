@@ -71,7 +71,7 @@ __device__ __forceinline__ void epilogue_group(const uint32_t* v, int row, int c
     if (c < p.N) {
         if constexpr (EPI == kEpiBias || EPI == kEpiBiasResid || EPI == kEpiBiasGelu) {
             float b[8];
-            unpack8(__ldg(reinterpret_cast<const uint4*>(p.bias + c)), b);
+            unpack8(*(reinterpret_cast<const uint4*>(p.bias + c)), b);
 #pragma unroll
             for (int j = 0; j < 8; ++j) f[j] += b[j];
         }
@@ -208,10 +208,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
         tmem_relinquish();
     }
+    grid_dep_launch();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    grid_dep_wait();                                    // inputs of this GEMM come from the previous kernel
 
     if (warp == 0) {
         if (lane == 0) {
@@ -370,9 +372,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
     tc_fence_before();
     __syncthreads();
+    grid_dep_launch();
     cluster_sync_all();                                 // both CTAs' barriers exist before anyone signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    grid_dep_wait();                                    // inputs of this GEMM come from the previous kernel
 
     if (warp == 0) {
         if (lane == 0) {
@@ -496,8 +500,8 @@ const char* launch_inst(Runtime* rt, const CUtensorMap& tmA, const CUtensorMap& 
     auto kern = gemm_kernel<A_MN, B_MN, EPI>;
     const int total = p.m_tiles * p.n_tiles;
     const int grid = total < rt->sm_count ? total : rt->sm_count;
-    kern<<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, tmBh, tmC, tmAux, p);
-    return cudaGetLastError() == cudaSuccess ? nullptr : "gemm launch failed";
+    return launch_k(kern, dim3(grid), dim3(GEMM_THREADS), SMEM_BYTES, stream, tmA, tmB, tmBh, tmC, tmAux, p) == cudaSuccess
+               ? nullptr : "gemm launch failed";
 }
 
 template <bool A_MN, bool B_MN, int EPI>
@@ -508,8 +512,8 @@ const char* launch_pair(Runtime* rt, const CUtensorMap& tmA, const CUtensorMap& 
     const int total = p.m_tiles * p.n_tiles;
     const int max_pairs = rt->sm_count / 2;
     const int pairs = total < max_pairs ? total : max_pairs;
-    kern<<<2 * pairs, PairCfg<EPI>::kThreads, PairCfg<EPI>::kSmem, stream>>>(tmA, tmB, tmC, tmAux, p);
-    return cudaGetLastError() == cudaSuccess ? nullptr : "gemm (CTA pair) launch failed";
+    return launch_k(kern, dim3(2 * pairs), dim3(PairCfg<EPI>::kThreads), PairCfg<EPI>::kSmem, stream, tmA, tmB, tmC, tmAux, p) == cudaSuccess
+               ? nullptr : "gemm (CTA pair) launch failed";
 }
 
 template <bool A_MN, bool B_MN, int EPI>

@@ -83,6 +83,18 @@ __device__ __forceinline__ float gelu_grad_f(float u, int act)
     return fmaf(u * 0.3989422804014327f, e, cdf);
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with the programmatic-serialization attribute may start while the previous
+// kernel of its stream is still running.  grid_dep_launch() lets the next kernel be scheduled as
+// early as possible; grid_dep_wait() blocks until the previous kernel has completed and its
+// memory is visible - every kernel calls it before its first global-memory access, so only the
+// launch latency and the on-chip set-up overlap.  Both are no-ops for a plain launch.
+// Consequence for every kernel here: no input pointer is `const __restrict__` and nothing is read
+// with __ldg - the compiler treats such loads as invariant over the kernel's lifetime and may hoist
+// them above the wait, where the producer has not written the data yet.
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------- shared-memory addresses
 __device__ __forceinline__ uint32_t smem_u32(const void* p)
 {

@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
+#include <stdlib.h>
 
 #include "pw_common.cuh"
 
@@ -26,6 +27,20 @@ Runtime* get_runtime(const char** err);
 const char* configure_gemm();
 const char* configure_attention();
 const char* configure_attention_fwd();
+
+// Launch with the programmatic-serialization attribute (see grid_dep_wait in pw_common.cuh).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args)
+{
+    static const bool pdl = getenv("PW_NO_PDL") == nullptr;   // tuning aid
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
 
 enum GemmLayout { kTN = 0, kNN = 1, kNT = 2 };
 enum GemmEpi { kEpiNone = 0, kEpiBias = 1, kEpiBiasResid = 2, kEpiBiasGelu = 3, kEpiDGelu = 4, kEpiF32 = 5 };
