@@ -52,7 +52,7 @@ Runtime* get_runtime(const char** err)
         delete rt; *err = "cuTensorMapEncodeTiled not available from the driver"; return nullptr;
     }
     const char* ce;
-    if ((ce = configure_gemm()) || (ce = configure_attention()) || (ce = configure_attention_fwd())) { delete rt; *err = ce; return nullptr; }
+    if ((ce = configure_gemm()) || (ce = configure_attention()) || (ce = configure_attention_fwd()) || (ce = configure_elementwise())) { delete rt; *err = ce; return nullptr; }
     if (cudaMalloc(reinterpret_cast<void**>(&rt->op_status), sizeof(DeviceStatus)) != cudaSuccess ||
         cudaMemset(rt->op_status, 0, sizeof(DeviceStatus)) != cudaSuccess) {
         delete rt; *err = "could not allocate the status word"; return nullptr;

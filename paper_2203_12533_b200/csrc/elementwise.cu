@@ -116,6 +116,31 @@ bool plan_warp_rows(int d, int* W, int* CH)
 // partials[(cta*rows_per_cta + row_in_cta)][4][d] = {dgamma, dbeta, sum resid, sum dx}.
 // The next row's three inputs are fetched before the current row's reduction, and the two row
 // sums share one barrier.
+constexpr int kLnBwdDepth = 4;
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, bool valid)
+{
+    const int n = valid ? 16 : 0;                       // 0: the 16 bytes are zero-filled, src is not read
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void unpack8_pairs(const uint4& v, uint64_t* p)
+{
+    p[0] = pack_f32x2(bf16_lo(v.x), bf16_hi(v.x)); p[1] = pack_f32x2(bf16_lo(v.y), bf16_hi(v.y));
+    p[2] = pack_f32x2(bf16_lo(v.z), bf16_hi(v.z)); p[3] = pack_f32x2(bf16_lo(v.w), bf16_hi(v.w));
+}
+__device__ __forceinline__ uint32_t pack_pair_bf16(uint64_t p)
+{
+    float lo, hi;
+    unpack_f32x2(p, lo, hi);
+    return pack_bf16(lo, hi);
+}
+__device__ __forceinline__ uint64_t splat2(float v) { return pack_f32x2(v, v); }
+
+// The kernel is bound by instruction issue as much as by memory, so all element-wise arithmetic
+// is two-wide fp32 (values of neighbouring columns packed in one 64-bit register).
 template <int CHUNKS>
 __global__ void __launch_bounds__(kRowThreadsMax, CHUNKS == 1 ? 2 : 1)
 ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
@@ -128,79 +153,101 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
     const int wpr = tpr >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     grid_dep_launch();
     grid_dep_wait();
-    float gm[CHUNKS][8];
-    float acc_g[CHUNKS][8], acc_b[CHUNKS][8], acc_r[CHUNKS][8], acc_x[CHUNKS][8];
+    uint64_t gm[CHUNKS][4];
+    uint64_t acc_g[CHUNKS][4], acc_b[CHUNKS][4], acc_r[CHUNKS][4], acc_x[CHUNKS][4];
 #pragma unroll
     for (int j = 0; j < CHUNKS; ++j) {
-        unpack8(*(reinterpret_cast<const uint4*>(gamma + 8 * (tr + j * tpr))), gm[j]);
+        unpack8_pairs(*(reinterpret_cast<const uint4*>(gamma + 8 * (tr + j * tpr))), gm[j]);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) acc_g[j][k] = acc_b[j][k] = acc_r[j][k] = acc_x[j][k] = 0.f;
+        for (int k = 0; k < 4; ++k) acc_g[j][k] = acc_b[j][k] = acc_r[j][k] = acc_x[j][k] = 0ull;
     }
     const int row_groups = (T + rows_per_cta - 1) / rows_per_cta;
-    uint4 n_dh[CHUNKS], n_x[CHUNKS], n_rs[CHUNKS];
+    // The three inputs of the rows this thread will handle travel through a private ring in
+    // shared memory, kLnBwdDepth - 1 rows ahead (16-byte asynchronous copies; a thread only ever
+    // reads what it fetched itself, so no barrier is involved).  Slot (stage, input, j) of thread
+    // t is ring[((stage * 3 + input) * CHUNKS + j) * blockDim.x + t].
+    extern __shared__ uint4 ln_bwd_ring[];
+    const uint32_t ring0 = smem_u32(ln_bwd_ring) + 16u * threadIdx.x;
+    const uint32_t slot_stride = 16u * blockDim.x;
+    auto issue = [&](int rg, int stage) {
+        const int row = rg * rows_per_cta + row_in_cta;
+        const bool live = rg < row_groups && row < T;
+#pragma unroll
+        for (int j = 0; j < CHUNKS; ++j) {
+            const size_t off = live ? static_cast<size_t>(row) * d + 8 * (tr + j * tpr) : 0;
+            const uint32_t dst = ring0 + (stage * 3 * CHUNKS + j) * slot_stride;
+            cp_async_16(dst, dh + off, live);
+            cp_async_16(dst + CHUNKS * slot_stride, x + off, live);
+            cp_async_16(dst + 2 * CHUNKS * slot_stride, resid + off, live);
+        }
+        cp_async_commit();
+    };
     float n_m = 0.f, n_r = 0.f;
-    auto fetch = [&](int rg) {
+    auto fetch_stats = [&](int rg) {
         const int row = rg * rows_per_cta + row_in_cta;
         const bool live = rg < row_groups && row < T;
         n_m = live ? mu[row] : 0.f;
         n_r = live ? rstd[row] : 0.f;
-#pragma unroll
-        for (int j = 0; j < CHUNKS; ++j) {
-            const size_t off = static_cast<size_t>(row) * d + 8 * (tr + j * tpr);
-            n_dh[j] = live ? *reinterpret_cast<const uint4*>(dh + off) : make_uint4(0, 0, 0, 0);
-            n_x[j] = live ? *reinterpret_cast<const uint4*>(x + off) : make_uint4(0, 0, 0, 0);
-            n_rs[j] = live ? *reinterpret_cast<const uint4*>(resid + off) : make_uint4(0, 0, 0, 0);
-        }
     };
-    fetch(blockIdx.x);
-    int par = 0;
+#pragma unroll
+    for (int s = 0; s < kLnBwdDepth - 1; ++s) issue(blockIdx.x + s * gridDim.x, s);
+    fetch_stats(blockIdx.x);
+    const float inv_d = 1.0f / d;
+    int par = 0, stage = 0;
     for (int rg = blockIdx.x; rg < row_groups; rg += gridDim.x, par ^= 1) {
         const int row = rg * rows_per_cta + row_in_cta;
         const bool live = row < T;
-        const float m = n_m, r = n_r;
-        float xh[CHUNKS][8], g[CHUNKS][8], dhv[CHUNKS][8], rs[CHUNKS][8];
-        float s1 = 0.f, s2 = 0.f;
+        const float r = n_r;
+        const uint64_t r2 = splat2(r), nmr2 = splat2(-n_m * r);
+        issue(rg + (kLnBwdDepth - 1) * gridDim.x, stage == 0 ? kLnBwdDepth - 1 : stage - 1);
+        cp_async_wait<kLnBwdDepth - 1>();                  // this row's copies have landed
+        uint64_t xh[CHUNKS][4], g[CHUNKS][4], dhv[CHUNKS][4], rs[CHUNKS][4];
+        uint64_t s1p = 0ull, s2p = 0ull;
 #pragma unroll
         for (int j = 0; j < CHUNKS; ++j) {
-            unpack8(n_dh[j], dhv[j]);
-            unpack8(n_x[j], xh[j]);
-            unpack8(n_rs[j], rs[j]);
+            const uint4* slot = ln_bwd_ring + (stage * 3 * CHUNKS + j) * blockDim.x + threadIdx.x;
+            unpack8_pairs(slot[0], dhv[j]);
+            unpack8_pairs(slot[CHUNKS * blockDim.x], xh[j]);
+            unpack8_pairs(slot[2 * CHUNKS * blockDim.x], rs[j]);
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                xh[j][k] = (xh[j][k] - m) * r;
-                g[j][k] = dhv[j][k] * gm[j][k];
-                s1 += g[j][k];
-                s2 += g[j][k] * xh[j][k];
+            for (int k = 0; k < 4; ++k) {
+                xh[j][k] = ffma2(xh[j][k], r2, nmr2);           // (x - mu) * rstd
+                g[j][k] = fmul2(dhv[j][k], gm[j][k]);
+                s1p = fadd2(s1p, g[j][k]);
+                s2p = ffma2(g[j][k], xh[j][k], s2p);
             }
         }
-        fetch(rg + gridDim.x);            // next row's loads are in flight during the reduction
-        s1 = warp_sum(s1);
-        s2 = warp_sum(s2);
+        stage = stage + 1 == kLnBwdDepth ? 0 : stage + 1;
+        fetch_stats(rg + gridDim.x);
+        float s1, s1b, s2, s2b;
+        unpack_f32x2(s1p, s1, s1b);
+        unpack_f32x2(s2p, s2, s2b);
+        s1 = warp_sum(s1 + s1b);
+        s2 = warp_sum(s2 + s2b);
         if (wpr > 1) {
             if (lane == 0) { red[par][0][warp] = s1; red[par][1][warp] = s2; }
             __syncthreads();
             s1 = 0.f; s2 = 0.f;
             for (int i = 0; i < wpr; ++i) { s1 += red[par][0][row_in_cta * wpr + i]; s2 += red[par][1][row_in_cta * wpr + i]; }
         }
-        const float mg = s1 / d, mgx = s2 / d;
+        const uint64_t nmg2 = splat2(-s1 * inv_d), nmgx2 = splat2(-s2 * inv_d);
         if (live) {
 #pragma unroll
             for (int j = 0; j < CHUNKS; ++j) {
                 const size_t off = static_cast<size_t>(row) * d + 8 * (tr + j * tpr);
-                float o[8];
+                uint32_t w[4];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) o[k] = rs[j][k] + r * (g[j][k] - mg - xh[j][k] * mgx);
-                const uint4 packed = pack8(o);
-                *reinterpret_cast<uint4*>(dx + off) = packed;
-                float ob[8];
-                unpack8(packed, ob);   // the bias gradient sums the values that are actually stored
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    acc_g[j][k] += dhv[j][k] * xh[j][k];
-                    acc_b[j][k] += dhv[j][k];
-                    acc_r[j][k] += rs[j][k];
-                    acc_x[j][k] += ob[k];
+                for (int k = 0; k < 4; ++k) {
+                    // dx = resid + rstd * (g - mean(g) - xh * mean(g * xh))
+                    const uint64_t t = ffma2(xh[j][k], nmgx2, fadd2(g[j][k], nmg2));
+                    w[k] = pack_pair_bf16(ffma2(r2, t, rs[j][k]));
+                    // the bias gradient sums the values that are actually stored
+                    acc_x[j][k] = fadd2(acc_x[j][k], pack_f32x2(bf16_lo(w[k]), bf16_hi(w[k])));
+                    acc_g[j][k] = ffma2(dhv[j][k], xh[j][k], acc_g[j][k]);
+                    acc_b[j][k] = fadd2(acc_b[j][k], dhv[j][k]);
+                    acc_r[j][k] = fadd2(acc_r[j][k], rs[j][k]);
                 }
+                *reinterpret_cast<uint4*>(dx + off) = make_uint4(w[0], w[1], w[2], w[3]);
             }
         }
     }
@@ -209,11 +256,12 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
     for (int j = 0; j < CHUNKS; ++j) {
         const int col = 8 * (tr + j * tpr);
 #pragma unroll
-        for (int k = 0; k < 8; k += 4) {
-            *reinterpret_cast<float4*>(prow + 0 * d + col + k) = make_float4(acc_g[j][k], acc_g[j][k + 1], acc_g[j][k + 2], acc_g[j][k + 3]);
-            *reinterpret_cast<float4*>(prow + 1 * d + col + k) = make_float4(acc_b[j][k], acc_b[j][k + 1], acc_b[j][k + 2], acc_b[j][k + 3]);
-            *reinterpret_cast<float4*>(prow + 2 * d + col + k) = make_float4(acc_r[j][k], acc_r[j][k + 1], acc_r[j][k + 2], acc_r[j][k + 3]);
-            *reinterpret_cast<float4*>(prow + 3 * d + col + k) = make_float4(acc_x[j][k], acc_x[j][k + 1], acc_x[j][k + 2], acc_x[j][k + 3]);
+        for (int k = 0; k < 4; k += 2) {
+            // two pairs = four consecutive columns
+            *reinterpret_cast<ulonglong2*>(prow + 0 * d + col + 2 * k) = make_ulonglong2(acc_g[j][k], acc_g[j][k + 1]);
+            *reinterpret_cast<ulonglong2*>(prow + 1 * d + col + 2 * k) = make_ulonglong2(acc_b[j][k], acc_b[j][k + 1]);
+            *reinterpret_cast<ulonglong2*>(prow + 2 * d + col + 2 * k) = make_ulonglong2(acc_r[j][k], acc_r[j][k + 1]);
+            *reinterpret_cast<ulonglong2*>(prow + 3 * d + col + 2 * k) = make_ulonglong2(acc_x[j][k], acc_x[j][k + 1]);
         }
     }
 }
@@ -326,6 +374,14 @@ const char* launch_layernorm_fwd(Runtime* rt, const void* x, const void* gamma, 
     return le == cudaSuccess ? nullptr : "layernorm fwd launch failed";
 }
 
+const char* configure_elementwise()
+{
+    cudaError_t e = cudaFuncSetAttribute(ln_bwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLnBwdDepth * 3 * 1 * kRowThreadsMax * 16);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ln_bwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLnBwdDepth * 3 * 2 * kRowThreadsMax * 16);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ln_bwd_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLnBwdDepth * 3 * 4 * kRowThreadsMax * 16);
+    return e == cudaSuccess ? nullptr : "could not raise the shared-memory limit of the layernorm kernels";
+}
+
 size_t layernorm_bwd_scratch_bytes(Runtime* rt, int T, int d)
 {
     RowPlan rp;
@@ -350,10 +406,11 @@ const char* launch_layernorm_bwd(Runtime* rt, const void* dh, const void* x, con
     auto Rs = static_cast<const float*>(rstd);
     auto P = static_cast<float*>(partials);
     cudaError_t le = cudaSuccess;
+    const size_t ring_bytes = static_cast<size_t>(kLnBwdDepth) * 3 * rp.chunks * rp.threads * 16;
     switch (rp.chunks) {
-        case 1: le = launch_k(ln_bwd_kernel<1>, dim3(grid), dim3(rp.threads), 0, stream, DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
-        case 2: le = launch_k(ln_bwd_kernel<2>, dim3(grid), dim3(rp.threads), 0, stream, DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
-        default: le = launch_k(ln_bwd_kernel<4>, dim3(grid), dim3(rp.threads), 0, stream, DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
+        case 1: le = launch_k(ln_bwd_kernel<1>, dim3(grid), dim3(rp.threads), ring_bytes, stream, DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
+        case 2: le = launch_k(ln_bwd_kernel<2>, dim3(grid), dim3(rp.threads), ring_bytes, stream, DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
+        default: le = launch_k(ln_bwd_kernel<4>, dim3(grid), dim3(rp.threads), ring_bytes, stream, DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
     }
     if (le != cudaSuccess) return "layernorm bwd launch failed";
     ReduceOuts outs;

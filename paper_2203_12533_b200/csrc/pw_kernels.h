@@ -27,6 +27,7 @@ Runtime* get_runtime(const char** err);
 const char* configure_gemm();
 const char* configure_attention();
 const char* configure_attention_fwd();
+const char* configure_elementwise();
 
 // Launch with the programmatic-serialization attribute (see grid_dep_wait in pw_common.cuh).
 template <typename... KArgs, typename... Args>
