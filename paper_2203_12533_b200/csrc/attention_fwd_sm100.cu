@@ -31,16 +31,55 @@ struct FwdSmem {
     static constexpr int kQ = 0;                            // two Q tiles
     static constexpr int kK = 2 * kTile;                    // two K stages
     static constexpr int kV = 4 * kTile;                    // two V stages
-    static constexpr int kBars = 6 * kTile;
+    static constexpr int kO = 6 * kTile;                    // output staging tile (shared by both query tiles)
+    static constexpr int kBars = 7 * kTile;
     static constexpr int kBytes = kBars + 256 + 1024;
 };
 
+// Timeline tracing of CTA 0 (one writer thread per role), compiled in only with -DPW_TRACE_ENABLE:
+// event = (tag << 48) | clock64.  Read back with pw_debug_trace_fwd (not part of the C ABI).
+#ifdef PW_TRACE_ENABLE
+__device__ long long g_trace[4][1024];
+__device__ int g_trace_n[4];
+// the event counter lives in a register of the writer thread (a global counter would stall it)
+__device__ __forceinline__ void trace(int role, int tag, int& n)
+{
+    if (blockIdx.x != 0 || (threadIdx.x & 31) != 0) return;
+    if (n < 1024) g_trace[role][n] = (static_cast<long long>(tag) << 48) | (clock64() & 0xffffffffffffll);
+    g_trace_n[role] = ++n;
+}
+#define PW_TRACE(role, tag) trace(role, tag, trace_n)
+#else
+#define PW_TRACE(role, tag) ((void)0)
+#endif
+
 struct FwdParams {
-    int S, H;
+    int S, H, B;
+    int pairs_per_seq;          // ceil(S / 256)
+    int n_items;                // B * H * pairs_per_seq
     float scale;
     float* lse;
     DeviceStatus* status;
+    int* sched;                 // {next ticket, CTAs done}
 };
+
+// Work items (one per sequence, head and pair of query tiles) are numbered heaviest first (latest
+// query tiles first) and handed out in that order: the producer thread draws the next number from
+// a global counter and passes it to the other roles through a two-slot ring in shared memory, so
+// the causal triangle balances itself over the CTAs.  Every CTA draws exactly one number past the
+// end; the last CTA to do so clears the counters for the next launch.
+struct FwdItem { int b, h, q0A, nA, nB; };
+__device__ __forceinline__ bool fwd_item(const FwdParams& p, int idx, FwdItem& it)
+{
+    if (idx >= p.n_items) return false;
+    const int BH = p.B * p.H;
+    const int pair = p.pairs_per_seq - 1 - idx / BH, bh = idx % BH;
+    it.b = bh / p.H; it.h = bh % p.H;
+    it.q0A = pair * 256;
+    it.nA = it.q0A / 128 + 1;                               // key tiles each query tile needs
+    it.nB = it.q0A + 128 < p.S ? it.nA + 1 : 0;
+    return true;
+}
 
 template <int DH>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -51,26 +90,57 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
     uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(sm);
     uint64_t* bars = reinterpret_cast<uint64_t*>(sm + L::kBars);
-    // barrier map: 0 q_full | 1,2 k_full | 3,4 k_empty | 5,6 v_full | 7,8 v_empty | 9,10 s_full | 11,12 p_full | 13,14 o_full
+    // barrier map (t = query tile, s = ring stage):
+    //   0+t q_full | 2+t q_empty | 4+s k_full | 6+s k_empty | 8+s v_full | 10+s v_empty
+    //   12+t s_full | 14+t p_full (128 arrivals) | 16+t o_full | 18+t o_empty (128 arrivals) | 20 staging free
+    //   21+i item_full | 23+i item_empty (9 arrivals: MMA warp + 8 softmax warps)
     const uint32_t bar0 = smem_u32(bars);
     auto bar = [&](int i) { return bar0 + 8u * i; };
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 26);
+    volatile int* item_slot = reinterpret_cast<volatile int*>(tmem_slot + 2);   // two entries
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    // draws the next item number; past the end, counts this CTA as done and lets the last one clear the counters
+    auto draw = [&]() {
+        const int idx = atomicAdd(p.sched, 1);
+        if (idx >= p.n_items && atomicAdd(p.sched + 1, 1) == static_cast<int>(gridDim.x) - 1) {
+            p.sched[0] = 0; p.sched[1] = 0;
+            __threadfence();
+        }
+        return idx;
+    };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int pair = gridDim.x - 1 - blockIdx.x;            // heaviest (latest) query tiles first
-    const int b = blockIdx.y / p.H, h = blockIdx.y % p.H;
     const int d = p.H * DH;
-    const int q0A = pair * 256, q0B = q0A + 128;
-    const bool hasB = q0B < p.S;
-    const int nA = q0A / 128 + 1, nB = hasB ? nA + 1 : 0;   // key tiles each query tile needs
-    const int n_kv = hasB ? nB : nA;
-    const int row_base = b * p.S;
+    int trace_n = 0;                                        // used by PW_TRACE only
+    (void)trace_n;
+
+    auto load_q = [&](const FwdItem& it, int t) {
+        mbar_arrive_expect_tx(bar(0 + t), L::kTile);
+        for (int kb = 0; kb < L::kBlocks; ++kb)
+            tma_load_2d(sbase + L::kQ + t * L::kTile + kb * 16384, &tmQKV, it.h * DH + kb * 64,
+                        it.b * p.S + it.q0A + t * 128, bar(0 + t));
+    };
+    auto load_k = [&](const FwdItem& it, int j, int s) {
+        mbar_arrive_expect_tx(bar(4 + s), L::kTile);
+        for (int kb = 0; kb < L::kBlocks; ++kb)
+            tma_load_2d(sbase + L::kK + s * L::kTile + kb * 16384, &tmQKV, d + it.h * DH + kb * 64,
+                        it.b * p.S + j * 128, bar(4 + s));
+    };
+    auto load_v = [&](const FwdItem& it, int j, int s) {
+        mbar_arrive_expect_tx(bar(8 + s), L::kTile);
+        for (int kb = 0; kb < L::kBlocks; ++kb)
+            tma_load_2d(sbase + L::kV + s * L::kTile + kb * 16384, &tmQKV, 2 * d + it.h * DH + kb * 64,
+                        it.b * p.S + j * 128, bar(8 + s));
+    };
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 11; ++i) mbar_init(bar(i), 1);
-        mbar_init(bar(11), 128); mbar_init(bar(12), 128);
-        mbar_init(bar(13), 1); mbar_init(bar(14), 1);
+        for (int i = 0; i < 14; ++i) mbar_init(bar(i), 1);
+        mbar_init(bar(14), 128); mbar_init(bar(15), 128);
+        mbar_init(bar(16), 1); mbar_init(bar(17), 1);
+        mbar_init(bar(18), 128); mbar_init(bar(19), 128);
+        mbar_init(bar(20), 1);
+        mbar_init(bar(21), 1); mbar_init(bar(22), 1);
+        mbar_init(bar(23), 9); mbar_init(bar(24), 9);
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -80,18 +150,16 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
     grid_dep_launch();
     grid_dep_wait();                                        // qkv comes from the previous kernel
     if (threadIdx.x == 0) {
-        // first loads go out before the TMEM allocation and the CTA-wide barrier
-        const int nq = hasB ? 2 : 1;
-        mbar_arrive_expect_tx(bar(0), nq * L::kTile);
-        for (int t = 0; t < nq; ++t)
-            for (int kb = 0; kb < L::kBlocks; ++kb)
-                tma_load_2d(sbase + L::kQ + t * L::kTile + kb * 16384, &tmQKV, h * DH + kb * 64,
-                            row_base + q0A + t * 128, bar(0));
-        mbar_arrive_expect_tx(bar(1), L::kTile);
-        mbar_arrive_expect_tx(bar(5), L::kTile);
-        for (int kb = 0; kb < L::kBlocks; ++kb) {
-            tma_load_2d(sbase + L::kK + kb * 16384, &tmQKV, d + h * DH + kb * 64, row_base, bar(1));
-            tma_load_2d(sbase + L::kV + kb * 16384, &tmQKV, 2 * d + h * DH + kb * 64, row_base, bar(5));
+        // the first item's first loads go out before the TMEM allocation and the CTA-wide barrier
+        FwdItem it;
+        const int idx0 = draw();
+        item_slot[0] = idx0;
+        mbar_arrive(bar(21));
+        if (fwd_item(p, idx0, it)) {
+            load_k(it, 0, 0);
+            load_q(it, 0);
+            if (it.nB) load_q(it, 1);
+            load_v(it, 0, 0);
         }
     }
     if (warp == 1) {
@@ -105,110 +173,214 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int j = 1; j < n_kv; ++j) {                // Q and key tile 0 were requested in the prologue
-                const int s = j & 1, ph = (j >> 1) & 1;
-                if (!mbar_wait(bar(3 + s), ph ^ 1, abort_flag, p.status, 400)) break;
-                mbar_arrive_expect_tx(bar(1 + s), L::kTile);
-                for (int kb = 0; kb < L::kBlocks; ++kb)
-                    tma_load_2d(sbase + L::kK + s * L::kTile + kb * 16384, &tmQKV, d + h * DH + kb * 64,
-                                row_base + j * 128, bar(1 + s));
-                if (!mbar_wait(bar(7 + s), ph ^ 1, abort_flag, p.status, 401)) break;
-                mbar_arrive_expect_tx(bar(5 + s), L::kTile);
-                for (int kb = 0; kb < L::kBlocks; ++kb)
-                    tma_load_2d(sbase + L::kV + s * L::kTile + kb * 16384, &tmQKV, 2 * d + h * DH + kb * 64,
-                                row_base + j * 128, bar(5 + s));
+            uint32_t n = 0;                                 // key/value tiles requested so far
+            uint32_t qn[2] = {0, 0};                        // items each query tile took part in
+            bool ok = true;
+            FwdItem it;
+            int idx = item_slot[0];
+            for (int k = 0; ok && fwd_item(p, idx, it); ++k) {
+                const int n_kv = it.nB ? it.nB : it.nA;
+                for (int j = 0; j < n_kv && ok; ++j, ++n) {
+                    const int s = n & 1;
+                    const uint32_t ph = (n >> 1) & 1;
+                    const bool early = k == 0 && j == 0;    // requested in the prologue
+                    if (!early) {
+                        if (!mbar_wait(bar(6 + s), ph ^ 1, abort_flag, p.status, 400)) { ok = false; break; }
+                        load_k(it, j, s);
+                        PW_TRACE(0, 1);
+                    }
+                    if (j == 0) {
+                        // Q follows the first key tile; its buffer is free once the previous item's
+                        // last S = Q K^T has been computed.
+                        for (int t = 0; t < (it.nB ? 2 : 1) && ok; ++t) {
+                            if (!early) {
+                                if (!mbar_wait(bar(2 + t), (qn[t] & 1) ^ 1, abort_flag, p.status, 402)) { ok = false; break; }
+                                load_q(it, t);
+                                PW_TRACE(0, 2);
+                            }
+                            ++qn[t];
+                        }
+                        if (!ok) break;
+                    }
+                    if (!early) {
+                        if (!mbar_wait(bar(10 + s), ph ^ 1, abort_flag, p.status, 401)) { ok = false; break; }
+                        load_v(it, j, s);
+                        PW_TRACE(0, 3);
+                    }
+                }
+                if (!ok) break;
+                // next item: its number goes into slot (k+1)&1 once every role has read what was there
+                const int kn = k + 1;
+                if (!mbar_wait(bar(23 + (kn & 1)), ((kn >> 1) & 1) ^ 1, abort_flag, p.status, 403)) break;
+                idx = draw();
+                item_slot[kn & 1] = idx;
+                mbar_arrive(bar(21 + (kn & 1)));
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
-            constexpr uint32_t idesc_pv = make_idesc_bf16(128, DH, false, true);
-            // S_t = Q_t K^T from K stage s
-            auto issue_s = [&](int t, int s) {
-                const uint64_t dq = make_smem_desc_sw128(sbase + L::kQ + t * L::kTile, 16, 1024);
-                const uint64_t dk = make_smem_desc_sw128(sbase + L::kK + s * L::kTile, 16, 1024);
-                const uint32_t dst = tmem_base + t * 128;
+        // The whole warp runs this role converged (waits and address arithmetic stay uniform);
+        // one elected lane issues the tcgen05 instructions.
+        constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
+        constexpr uint32_t idesc_pv = make_idesc_bf16(128, DH, false, true);
+        const uint32_t tb = __shfl_sync(0xffffffffu, tmem_base, 0);
+        const uint32_t sb = __shfl_sync(0xffffffffu, sbase, 0);
+        // S_t = Q_t K^T from K stage s
+        auto issue_s = [&](int t, int s) {
+            const uint64_t dq = make_smem_desc_sw128(sb + L::kQ + t * L::kTile, 16, 1024);
+            const uint64_t dk = make_smem_desc_sw128(sb + L::kK + s * L::kTile, 16, 1024);
+            const uint32_t dst = tb + t * 128;
+            if (elect_one()) {
 #pragma unroll
                 for (int kb = 0; kb < L::kBlocks; ++kb)
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
                         umma_f16(dst, desc_advance(dq, kb * 16384 + kk * 32), desc_advance(dk, kb * 16384 + kk * 32),
                                  idesc_s, (kb | kk) ? 1u : 0u);
-                umma_commit(bar(9 + t));
-            };
-            // O_t (+)= P_t V from V stage s; P_t is bf16 packed in the first 64 columns of S_t
-            auto issue_pv = [&](int t, int s, bool acc) {
-                const uint64_t dv = make_smem_desc_sw128(sbase + L::kV + s * L::kTile, 16384, 1024);
-                const uint32_t dst = tmem_base + 256 + t * 128, src = tmem_base + t * 128;
+                umma_commit(bar(12 + t));
+            }
+            __syncwarp();
+        };
+        // O_t (+)= P_t V from V stage s; P_t is bf16 packed in the first 64 columns of S_t
+        auto issue_pv = [&](int t, int s, bool acc) {
+            const uint64_t dv = make_smem_desc_sw128(sb + L::kV + s * L::kTile, 16384, 1024);
+            const uint32_t dst = tb + 256 + t * 128, src = tb + t * 128;
+            if (elect_one()) {
                 umma_f16_ta(dst, src, dv, idesc_pv, acc ? 1u : 0u);
 #pragma unroll
                 for (int ks = 1; ks < 8; ++ks)
                     umma_f16_ta(dst, src + ks * 8, desc_advance(dv, ks * 2048), idesc_pv, 1u);
-            };
-            bool ok = mbar_wait(bar(0), 0, abort_flag, p.status, 410) && mbar_wait(bar(1), 0, abort_flag, p.status, 411);
-            if (ok) {
+            }
+            __syncwarp();
+        };
+        auto commit = [&](int b) {
+            if (elect_one()) umma_commit(bar(b));
+            __syncwarp();
+        };
+        auto wait = [&](int b, uint32_t parity, int site) {
+            bool w = mbar_wait(bar(b), parity, abort_flag, p.status, site);
+            return __all_sync(0xffffffffu, w);
+        };
+        uint32_t n = 0;                                 // key/value tiles consumed before this item
+        uint32_t np[2] = {0, 0};                        // P tiles consumed per query tile
+        uint32_t qn[2] = {0, 0};                        // items each query tile took part in
+        bool ok = true;
+        FwdItem it;
+        for (int k = 0; ok; ++k) {
+            if (!wait(21 + (k & 1), (k >> 1) & 1, 423)) break;
+            const int idx = item_slot[k & 1];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(23 + (k & 1)));
+            if (!fwd_item(p, idx, it)) break;
+            const int nA = it.nA, nB = it.nB, n_kv = nB ? nB : nA;
+            {
+                const int s = n & 1;
+                const uint32_t ph = (n >> 1) & 1;
+                ok = wait(4 + s, ph, 411) && wait(0, qn[0] & 1, 410);
+                if (!ok) break;
                 tc_fence_after();
-                issue_s(0, 0);
-                if (hasB) issue_s(1, 0);
-                umma_commit(bar(3));
+                PW_TRACE(1, 9);
+                issue_s(0, s);
+                PW_TRACE(1, 1);
+                if (nA == 1) commit(2);                     // Q_A is not needed again
+                if (nB) {
+                    if (!wait(1, qn[1] & 1, 417)) { ok = false; break; }
+                    tc_fence_after();
+                    issue_s(1, s);
+                    PW_TRACE(1, 2);
+                    if (nB == 1) commit(3);
+                }
+                commit(6 + s);
             }
             for (int j = 0; j < n_kv && ok; ++j) {
-                const int s = j & 1, ph = (j >> 1) & 1, nxt = j + 1, sn = nxt & 1, phn = (nxt >> 1) & 1;
-                if (!mbar_wait(bar(5 + s), ph, abort_flag, p.status, 412)) { ok = false; break; }
+                const uint32_t nj = n + j, nn = nj + 1;
+                const int s = nj & 1, sn = nn & 1;
+                const uint32_t ph = (nj >> 1) & 1, phn = (nn >> 1) & 1;
+                if (!wait(8 + s, ph, 412)) { ok = false; break; }
                 bool k_waited = false;
                 if (j < nA) {
-                    if (!mbar_wait(bar(11), j & 1, abort_flag, p.status, 413)) { ok = false; break; }
+                    if (!wait(14, np[0] & 1, 413)) { ok = false; break; }
+                    ++np[0];
+                    // the previous item's O_A must have been read out before it is overwritten
+                    if (j == 0 && !wait(18, (qn[0] & 1) ^ 1, 418)) { ok = false; break; }
                     tc_fence_after();
                     issue_pv(0, s, j > 0);
-                    if (j == nA - 1) umma_commit(bar(13));
+                    PW_TRACE(1, 3);
+                    if (j == nA - 1) commit(16);
                 }
-                if (nxt < nA) {
-                    if (!mbar_wait(bar(1 + sn), phn, abort_flag, p.status, 414)) { ok = false; break; }
+                if (j + 1 < nA) {
+                    if (!wait(4 + sn, phn, 414)) { ok = false; break; }
                     k_waited = true;
                     tc_fence_after();
                     issue_s(0, sn);
+                    PW_TRACE(1, 1);
+                    if (j + 2 == nA) commit(2);
                 }
                 if (j < nB) {
-                    if (!mbar_wait(bar(12), j & 1, abort_flag, p.status, 415)) { ok = false; break; }
+                    if (!wait(15, np[1] & 1, 415)) { ok = false; break; }
+                    ++np[1];
+                    if (j == 0 && !wait(19, (qn[1] & 1) ^ 1, 419)) { ok = false; break; }
                     tc_fence_after();
                     issue_pv(1, s, j > 0);
-                    if (j == nB - 1) umma_commit(bar(14));
+                    PW_TRACE(1, 4);
+                    if (j == nB - 1) commit(17);
                 }
-                umma_commit(bar(7 + s));                    // V stage free once these MMAs are done
-                if (nxt < nB) {
-                    if (!k_waited && !mbar_wait(bar(1 + sn), phn, abort_flag, p.status, 416)) { ok = false; break; }
+                commit(10 + s);                             // V stage free once these MMAs are done
+                if (j + 1 < nB) {
+                    if (!k_waited && !wait(4 + sn, phn, 416)) { ok = false; break; }
                     tc_fence_after();
                     issue_s(1, sn);
+                    PW_TRACE(1, 2);
+                    if (j + 2 == nB) commit(3);
                 }
-                if (nxt < n_kv) umma_commit(bar(3 + sn));   // K stage free
+                if (j + 1 < n_kv) commit(6 + sn);           // K stage free
             }
+            n += n_kv;
+            ++qn[0];
+            if (nB) ++qn[1];
         }
     } else {
         const int t = (warp - 2) >> 2;                      // 0 = tile A, 1 = tile B
         const int q = warp & 3;                             // TMEM lane quarter this warp may touch
         const int r = q * 32 + lane;                        // query row inside the tile
-        const int n_t = t == 0 ? nA : nB;
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
         const uint32_t s_addr = tmem_base + lane_addr + t * 128;
         const uint32_t o_addr = tmem_base + lane_addr + 256 + t * 128;
         const float sl2 = p.scale * kLog2e;
-        float m_used = -INFINITY, l = 0.f;
+        uint32_t ns = 0, qn = 0;                            // S tiles and items this query tile has seen
+        uint32_t u_base = 0;                                // uses of the output staging tile before this item
         bool ok = true;
-        for (int j = 0; j < n_t; ++j) {
-            ok = mbar_wait(bar(9 + t), j & 1, abort_flag, p.status, 420);
+        FwdItem it;
+        for (int k = 0; ok; ++k) {
+        ok = mbar_wait(bar(21 + (k & 1)), (k >> 1) & 1, abort_flag, p.status, 424);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const int idx = item_slot[k & 1];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(23 + (k & 1)));
+        if (!fwd_item(p, idx, it)) break;
+        const int n_t = t == 0 ? it.nA : it.nB;
+        const uint32_t u = u_base + t;                      // staging order: A(k), B(k), A(k+1), ...
+        u_base += it.nB ? 2 : 1;
+        if (n_t == 0) continue;
+        const int q0 = it.q0A + t * 128;
+        float m_used = -INFINITY, l = 0.f;
+        for (int j = 0; j < n_t; ++j, ++ns) {
+            ok = mbar_wait(bar(12 + t), ns & 1, abort_flag, p.status, 420);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
+            if ((warp & 3) == 2 && lane == 0) PW_TRACE(2 + t, 1);
             const bool diag = j == n_t - 1;
             // all 128 scores of the row in registers (four loads in flight, one wait)
             uint32_t v[128];
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, v + c * 32);
             tc_wait_ld();
+            if ((warp & 3) == 2 && lane == 0) PW_TRACE(2 + t, 2);
             // row maximum: eight independent chains of three-input max (64 instructions for 128 scores)
             float mxs[8];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) mxs[k] = -INFINITY;
+            for (int i = 0; i < 8; ++i) mxs[i] = -INFINITY;
             if (diag) {
 #pragma unroll
                 for (int i = 0; i < 128; ++i)
@@ -238,6 +410,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                 }
             }
             // p = exp2((s - m) * scale * log2e), packed bf16 written over the S columns
+            if ((warp & 3) == 2 && lane == 0) PW_TRACE(2 + t, 3);
             const float mb = m_used * sl2;
             if (diag) {
                 float ls = 0.f;
@@ -265,25 +438,37 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                 unpack_f32x2(fadd2(fadd2(lsum[0], lsum[1]), fadd2(lsum[2], lsum[3])), s0, s1);
                 l += s0 + s1;
             }
+            if ((warp & 3) == 2 && lane == 0) PW_TRACE(2 + t, 4);
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_st16(s_addr + c * 16, v + c * 16);
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(bar(11 + t));
+            mbar_arrive(bar(14 + t));
+            if ((warp & 3) == 2 && lane == 0) PW_TRACE(2 + t, 5);
         }
-        if (ok && n_t > 0) {
-            ok = mbar_wait(bar(13 + t), 0, abort_flag, p.status, 421);
+        if (ok) {
+            ok = mbar_wait(bar(16 + t), qn & 1, abort_flag, p.status, 421);
             ok = __all_sync(0xffffffffu, ok);
         }
-        if (ok && n_t > 0) {
+        if (!ok) break;
+        {
             tc_fence_after();
+            if ((warp & 3) == 2 && lane == 0) PW_TRACE(2 + t, 6);
             const float inv_l = 1.0f / l;
-            uint8_t* stage = sm + L::kQ + t * L::kTile;     // the Q tile is idle now: reuse it for O
+            uint8_t* stage = sm + L::kO;
+            ok = mbar_wait(bar(20), (u & 1) ^ 1, abort_flag, p.status, 422);    // the previous user's store has read it
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if ((warp & 3) == 2 && lane == 0) PW_TRACE(2 + t, 7);
 #pragma unroll 1
             for (int c = 0; c < DH / 32; ++c) {
                 uint32_t v[32];
                 tmem_ld32(o_addr + c * 32, v);
                 tc_wait_ld();
+                if (c == DH / 32 - 1) {                     // O_t has left TMEM: the next item may overwrite it
+                    tc_fence_before();
+                    mbar_arrive(bar(18 + t));
+                }
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
                     float f[8];
@@ -293,17 +478,21 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                     *reinterpret_cast<uint4*>(stage + blk * 16384 + r * 128 + ((chunk ^ (r & 7)) << 4)) = pack8(f);
                 }
             }
-            p.lse[(static_cast<size_t>(b) * p.H + h) * p.S + (t == 0 ? q0A : q0B) + r] = m_used * p.scale + logf(l);
+            p.lse[(static_cast<size_t>(it.b) * p.H + it.h) * p.S + q0 + r] = m_used * p.scale + logf(l);
             fence_proxy_async();
             named_bar_sync(1 + t, 128);
             if ((warp & 3) == 2 && lane == 0) {
                 for (int kb = 0; kb < L::kBlocks; ++kb)
-                    tma_store_2d(&tmO, sbase + L::kQ + t * L::kTile + kb * 16384, h * DH + kb * 64,
-                                 row_base + (t == 0 ? q0A : q0B));
+                    tma_store_2d(&tmO, sbase + L::kO + kb * 16384, it.h * DH + kb * 64, it.b * p.S + q0);
                 bulk_commit();
-                bulk_wait0();
+                bulk_wait_read0();                          // the staging tile may be written again
+                mbar_arrive(bar(20));
+                PW_TRACE(2 + t, 8);
             }
+            ++qn;
         }
+        }
+        if ((warp & 3) == 2 && lane == 0) bulk_wait0();
     }
 
     __syncwarp();
@@ -339,6 +528,16 @@ const char* encode_rows(Runtime* rt, CUtensorMap* map, const void* ptr, uint64_t
 
 }  // namespace
 
+#ifdef PW_TRACE_ENABLE
+extern "C" int pw_debug_trace_fwd(long long* events, int* counts)
+{
+    if (cudaMemcpyFromSymbol(events, g_trace, sizeof(long long) * 4 * 1024) != cudaSuccess) return 1;
+    if (cudaMemcpyFromSymbol(counts, g_trace_n, sizeof(int) * 4) != cudaSuccess) return 1;
+    int zero[4] = {0, 0, 0, 0};
+    return cudaMemcpyToSymbol(g_trace_n, zero, sizeof(zero)) == cudaSuccess ? 0 : 1;
+}
+#endif
+
 const char* configure_attention_fwd()
 {
     if (cudaFuncSetAttribute(attn_fwd_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<64>::kBytes) != cudaSuccess ||
@@ -357,10 +556,13 @@ const char* launch_attention_fwd(Runtime* rt, const void* qkv, int B, int S, int
     if ((e = encode_rows(rt, &tmQKV, qkv, 3ull * d, static_cast<uint64_t>(B) * S))) return e;
     if ((e = encode_rows(rt, &tmO, o, d, static_cast<uint64_t>(B) * S))) return e;
     FwdParams p;
-    p.S = S; p.H = H; p.scale = 1.0f / sqrtf(static_cast<float>(dh));
+    p.S = S; p.H = H; p.B = B; p.scale = 1.0f / sqrtf(static_cast<float>(dh));
+    p.pairs_per_seq = (S + 255) / 256;
+    p.n_items = B * H * p.pairs_per_seq;
     p.lse = static_cast<float*>(lse);
     p.status = status;
-    dim3 grid((S + 255) / 256, B * H);
+    p.sched = status->sched + 0;
+    dim3 grid(p.n_items < rt->sm_count ? p.n_items : rt->sm_count);
     const cudaError_t e2 = dh == 64
         ? launch_k(attn_fwd_tc_kernel<64>, grid, dim3(kThreads), FwdSmem<64>::kBytes, stream, tmQKV, tmO, p)
         : launch_k(attn_fwd_tc_kernel<128>, grid, dim3(kThreads), FwdSmem<128>::kBytes, stream, tmQKV, tmO, p);

@@ -11,9 +11,12 @@ namespace pw {
 
 // Device status block owned by the runtime (one per handle): word 0 = status code
 // (0 = ok), word 1 = site id of the wait that gave up.
+// Words 2.. are the work counters of the persistent attention kernels: {next ticket, CTAs done}
+// per kernel.  They are zero between launches (the last CTA of a launch clears its pair).
 struct DeviceStatus {
     int code;
     int site;
+    int sched[6];               // [0,1] attention fwd, [2,3] dQ, [4,5] dK/dV
 };
 
 constexpr int kStatusTimeout = 6;  // == PW_ERR_TIMEOUT
@@ -158,6 +161,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         }
     }
     return true;
+}
+
+// One lane of the (converged) warp is picked; the rest of the warp's code stays uniform.
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "elect.sync _|P, 0xffffffff;\n\t"
+        "selp.b32 %0, 1, 0, P;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
 }
 
 // ---------------------------------------------------------------- TMA (tiled, no cluster qualifiers)
