@@ -26,11 +26,14 @@ constexpr int kThreads = 320;
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct BwdParams {
-    int S, H;
+    int S, H, B;
+    int tiles_per_seq;          // dQ: pairs of query tiles; dK/dV: key tiles
+    int n_items;                // B * H * tiles_per_seq
     float scale;
     const float* lse;
     const float* delta;
     DeviceStatus* status;
+    int* sched;                 // {next ticket, CTAs done} of this kernel
 };
 
 // ------------------------------------------------------------------------------------------- dK, dV
@@ -39,12 +42,30 @@ struct KvSmem {
     static constexpr int kBlocks = DH / 64;
     static constexpr int kKV = 128 * DH * 2;                 // K_j or V_j tile
     static constexpr int kSub = 64 * DH * 2;                 // one 64-row sub-tile of Q or dO
-    static constexpr int kStages = 4;
-    static constexpr int kK = 0, kV = kKV, kQ = 2 * kKV;     // ring: stage s holds Q_u at kQ + s*2*kSub, dO_u right after
+    static constexpr int kStages = 3;
+    static constexpr int kK = 0;                             // item buffer i: K_j at i*2*kKV, V_j right after (two buffers)
+    static constexpr int kQ = 4 * kKV;                       // ring: stage s holds Q_u at kQ + s*2*kSub, dO_u right after
     static constexpr int kBars = kQ + kStages * 2 * kSub;
     static constexpr int kBytes = kBars + 256 + 1024;
 };
 
+// Work items of the dK/dV kernel: one per (sequence, head, 128-key tile), heaviest first (key tile
+// 0 sees every query), drawn from a global counter by the producer thread.
+struct KvItem { int b, h, j, n_u; };
+__device__ __forceinline__ bool kv_item(const BwdParams& p, int idx, KvItem& it)
+{
+    if (idx >= p.n_items) return false;
+    const int BH = p.B * p.H;
+    const int bh = idx % BH;
+    it.j = idx / BH;
+    it.b = bh / p.H; it.h = bh % p.H;
+    it.n_u = p.S / 64 - 2 * it.j;                           // query sub-tiles 2j .. S/64 - 1
+    return true;
+}
+
+// Persistent: K_j / V_j are double-buffered across items (the finished item's buffer doubles as the
+// staging area of its dK / dV store while the next item's tiles are already in the other one); the
+// Q_u / dO_u ring, the S^T / dP^T buffers and every barrier phase run on across item boundaries.
 template <int DH>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 64 x 128 rows
@@ -58,23 +79,51 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
     uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(sm);
     uint64_t* bars = reinterpret_cast<uint64_t*>(sm + L::kBars);
-    // 0 kv_full | 1..4 q_full | 5..8 q_empty | 9,10 st_full | 11,12 p_full | 13 acc_full
+    // barrier map: 0,1 kv_full[buffer] | 2,3 kv_empty[buffer] | 4..6 q_full[stage] | 7..9 q_empty[stage]
+    //   10,11 st_full[hb] | 12,13 p_full[hb] (256 arrivals) | 14 acc_full | 15 acc_empty (256 arrivals)
+    //   16,17 item_full | 18,19 item_empty (9 arrivals)
     const uint32_t bar0 = smem_u32(bars);
     auto bar = [&](int i) { return bar0 + 8u * i; };
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* item_slot = reinterpret_cast<volatile int*>(tmem_slot + 2);   // two entries
+    auto draw = [&]() {
+        const int idx = atomicAdd(p.sched, 1);
+        if (idx >= p.n_items && atomicAdd(p.sched + 1, 1) == static_cast<int>(gridDim.x) - 1) {
+            p.sched[0] = 0; p.sched[1] = 0;
+            __threadfence();
+        }
+        return idx;
+    };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int j = blockIdx.x;                               // key tile; tile 0 has the most query sub-tiles
-    const int b = blockIdx.y / p.H, h = blockIdx.y % p.H;
     const int d = p.H * DH;
-    const int kv0 = j * 128, row_base = b * p.S;
-    const int u0 = 2 * j, n_u = p.S / 64 - u0;              // query sub-tiles u0 .. u0 + n_u - 1
+
+    auto load_kv = [&](const KvItem& it, int buf) {
+        mbar_arrive_expect_tx(bar(0 + buf), 2 * L::kKV);
+        const uint32_t ks = sbase + L::kK + buf * 2 * L::kKV, vs = ks + L::kKV;
+        for (int kb = 0; kb < L::kBlocks; ++kb) {
+            tma_load_2d(ks + kb * 16384, &tmKV, d + it.h * DH + kb * 64, it.b * p.S + it.j * 128, bar(0 + buf));
+            tma_load_2d(vs + kb * 16384, &tmKV, 2 * d + it.h * DH + kb * 64, it.b * p.S + it.j * 128, bar(0 + buf));
+        }
+    };
+    auto load_q = [&](const KvItem& it, int i, int s) {     // Q_u and dO_u, u = 2j + i
+        mbar_arrive_expect_tx(bar(4 + s), 2 * L::kSub);
+        const uint32_t qs = sbase + L::kQ + s * 2 * L::kSub, gs = qs + L::kSub;
+        const int qrow = it.b * p.S + (2 * it.j + i) * 64;
+        for (int kb = 0; kb < L::kBlocks; ++kb) {
+            tma_load_2d(qs + kb * 8192, &tmQ, it.h * DH + kb * 64, qrow, bar(4 + s));
+            tma_load_2d(gs + kb * 8192, &tmDO, it.h * DH + kb * 64, qrow, bar(4 + s));
+        }
+    };
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 11; ++i) mbar_init(bar(i), 1);
-        mbar_init(bar(11), 256); mbar_init(bar(12), 256);
-        mbar_init(bar(13), 1);
+        for (int i = 0; i < 12; ++i) mbar_init(bar(i), 1);
+        mbar_init(bar(12), 256); mbar_init(bar(13), 256);
+        mbar_init(bar(14), 1);
+        mbar_init(bar(15), 256);
+        mbar_init(bar(16), 1); mbar_init(bar(17), 1);
+        mbar_init(bar(18), 9); mbar_init(bar(19), 9);
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -82,20 +131,15 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
     }
     grid_dep_launch();
     grid_dep_wait();                                        // inputs come from the previous kernels
+    int early = 0;                                          // sub-tiles of the first item requested in the prologue
     if (threadIdx.x == 0) {
-        // first loads go out before the TMEM allocation and the CTA-wide barrier
-        mbar_arrive_expect_tx(bar(0), 2 * L::kKV);
-        for (int kb = 0; kb < L::kBlocks; ++kb) {
-            tma_load_2d(sbase + L::kK + kb * 16384, &tmKV, d + h * DH + kb * 64, row_base + kv0, bar(0));
-            tma_load_2d(sbase + L::kV + kb * 16384, &tmKV, 2 * d + h * DH + kb * 64, row_base + kv0, bar(0));
-        }
-        for (int i = 0; i < n_u && i < L::kStages; ++i) {
-            mbar_arrive_expect_tx(bar(1 + i), 2 * L::kSub);
-            const uint32_t qs = sbase + L::kQ + i * 2 * L::kSub, gs = qs + L::kSub;
-            for (int kb = 0; kb < L::kBlocks; ++kb) {
-                tma_load_2d(qs + kb * 8192, &tmQ, h * DH + kb * 64, row_base + (u0 + i) * 64, bar(1 + i));
-                tma_load_2d(gs + kb * 8192, &tmDO, h * DH + kb * 64, row_base + (u0 + i) * 64, bar(1 + i));
-            }
+        KvItem it;
+        const int idx0 = draw();
+        item_slot[0] = idx0;
+        mbar_arrive(bar(16));
+        if (kv_item(p, idx0, it)) {
+            load_kv(it, 0);
+            for (; early < it.n_u && early < L::kStages; ++early) load_q(it, early, early);
         }
     }
     if (warp == 1) {
@@ -110,29 +154,42 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int i = L::kStages; i < n_u; ++i) {        // K_j, V_j and the first sub-tiles were requested in the prologue
-                const int s = i % L::kStages, ph = (i / L::kStages) & 1;
-                if (!mbar_wait(bar(5 + s), ph ^ 1, abort_flag, p.status, 500)) break;
-                mbar_arrive_expect_tx(bar(1 + s), 2 * L::kSub);
-                const uint32_t qs = sbase + L::kQ + s * 2 * L::kSub, gs = qs + L::kSub;
-                const int qrow = row_base + (u0 + i) * 64;
-                for (int kb = 0; kb < L::kBlocks; ++kb) {
-                    tma_load_2d(qs + kb * 8192, &tmQ, h * DH + kb * 64, qrow, bar(1 + s));
-                    tma_load_2d(gs + kb * 8192, &tmDO, h * DH + kb * 64, qrow, bar(1 + s));
+            uint32_t m = 0;                                 // sub-tiles requested so far
+            bool ok = true;
+            KvItem it;
+            int idx = item_slot[0];
+            for (int k = 0; ok && kv_item(p, idx, it); ++k) {
+                if (k > 0) {
+                    if (!mbar_wait(bar(2 + (k & 1)), ((k >> 1) & 1) ^ 1, abort_flag, p.status, 501)) break;
+                    load_kv(it, k & 1);
                 }
+                for (int i = 0; i < it.n_u && ok; ++i, ++m) {
+                    if (k == 0 && i < early) continue;
+                    const int s = m % L::kStages;
+                    if (!mbar_wait(bar(7 + s), ((m / L::kStages) & 1) ^ 1, abort_flag, p.status, 500)) { ok = false; break; }
+                    load_q(it, i, s);
+                }
+                if (!ok) break;
+                const int kn = k + 1;
+                if (!mbar_wait(bar(18 + (kn & 1)), ((kn >> 1) & 1) ^ 1, abort_flag, p.status, 502)) break;
+                idx = draw();
+                item_slot[kn & 1] = idx;
+                mbar_arrive(bar(16 + (kn & 1)));
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc_st = make_idesc_bf16(128, 64, false, false);
-            constexpr uint32_t idesc_acc = make_idesc_bf16(128, DH, false, true);
-            const uint64_t desc_k = make_smem_desc_sw128(sbase + L::kK, 16, 1024);
-            const uint64_t desc_v = make_smem_desc_sw128(sbase + L::kV, 16, 1024);
-            auto issue_scores = [&](int i) {                // S^T and dP^T of sub-tile i into buffer i & 1
-                const int s = i % L::kStages, hb = i & 1;
-                const uint32_t qs = sbase + L::kQ + s * 2 * L::kSub;
-                const uint64_t dq = make_smem_desc_sw128(qs, 16, 1024), dg = desc_advance(dq, L::kSub);
-                const uint32_t st = tmem_base + hb * 64;
+        // converged warp, one elected lane issues (see the forward kernel)
+        constexpr uint32_t idesc_st = make_idesc_bf16(128, 64, false, false);
+        constexpr uint32_t idesc_acc = make_idesc_bf16(128, DH, false, true);
+        const uint32_t tb = __shfl_sync(0xffffffffu, tmem_base, 0);
+        const uint32_t sb = __shfl_sync(0xffffffffu, sbase, 0);
+        auto issue_scores = [&](uint32_t g, int buf) {      // S^T and dP^T of stream position g into buffer g & 1
+            const int s = g % L::kStages, hb = g & 1;
+            const uint64_t desc_k = make_smem_desc_sw128(sb + L::kK + buf * 2 * L::kKV, 16, 1024);
+            const uint64_t desc_v = desc_advance(desc_k, L::kKV);
+            const uint64_t dq = make_smem_desc_sw128(sb + L::kQ + s * 2 * L::kSub, 16, 1024), dg = desc_advance(dq, L::kSub);
+            const uint32_t st = tb + hb * 64;
+            if (elect_one()) {
 #pragma unroll
                 for (int kb = 0; kb < L::kBlocks; ++kb)
 #pragma unroll
@@ -145,100 +202,138 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
                     for (int kk = 0; kk < 4; ++kk)
                         umma_f16(st + 128, desc_advance(desc_v, kb * 16384 + kk * 32), desc_advance(dg, kb * 8192 + kk * 32),
                                  idesc_st, (kb | kk) ? 1u : 0u);
-                umma_commit(bar(9 + hb));
-            };
-            auto issue_acc = [&](int i) {                   // dV += P^T dO_u, dK += dS^T Q_u
-                const int s = i % L::kStages, hb = i & 1;
-                const uint32_t qs = sbase + L::kQ + s * 2 * L::kSub;
-                const uint64_t dq = make_smem_desc_sw128(qs, 8192, 1024), dg = desc_advance(dq, L::kSub);
-                const uint32_t pt = tmem_base + hb * 64;
-                const uint32_t first = i ? 1u : 0u;
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    umma_f16_ta(tmem_base + 256, pt + (ks >> 1) * 32 + (ks & 1) * 8, desc_advance(dg, ks * 2048), idesc_acc,
-                                ks ? 1u : first);
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    umma_f16_ta(tmem_base + 384, pt + 128 + (ks >> 1) * 32 + (ks & 1) * 8, desc_advance(dq, ks * 2048), idesc_acc,
-                                ks ? 1u : first);
-                umma_commit(bar(5 + s));                    // Q_u / dO_u stage free
-            };
-            bool ok = mbar_wait(bar(0), 0, abort_flag, p.status, 510) && mbar_wait(bar(1), 0, abort_flag, p.status, 511);
-            if (ok) { tc_fence_after(); issue_scores(0); }
-            for (int i = 0; i < n_u && ok; ++i) {
-                if (i + 1 < n_u) {
-                    const int sn = (i + 1) % L::kStages, phn = ((i + 1) / L::kStages) & 1;
-                    if (!mbar_wait(bar(1 + sn), phn, abort_flag, p.status, 512)) { ok = false; break; }
-                    tc_fence_after();
-                    issue_scores(i + 1);
-                }
-                if (!mbar_wait(bar(11 + (i & 1)), (i >> 1) & 1, abort_flag, p.status, 513)) { ok = false; break; }
-                tc_fence_after();
-                issue_acc(i);
+                umma_commit(bar(10 + hb));
             }
-            if (ok) umma_commit(bar(13));
+            __syncwarp();
+        };
+        auto issue_acc = [&](uint32_t g, bool first) {      // dV += P^T dO_u, dK += dS^T Q_u
+            const int s = g % L::kStages, hb = g & 1;
+            const uint64_t dq = make_smem_desc_sw128(sb + L::kQ + s * 2 * L::kSub, 8192, 1024), dg = desc_advance(dq, L::kSub);
+            const uint32_t pt = tb + hb * 64;
+            const uint32_t acc0 = first ? 0u : 1u;
+            if (elect_one()) {
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_f16_ta(tb + 256, pt + (ks >> 1) * 32 + (ks & 1) * 8, desc_advance(dg, ks * 2048), idesc_acc,
+                                ks ? 1u : acc0);
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_f16_ta(tb + 384, pt + 128 + (ks >> 1) * 32 + (ks & 1) * 8, desc_advance(dq, ks * 2048), idesc_acc,
+                                ks ? 1u : acc0);
+                umma_commit(bar(7 + s));                    // Q_u / dO_u stage free
+            }
+            __syncwarp();
+        };
+        auto wait = [&](int b, uint32_t parity, int site) {
+            const bool w = mbar_wait(bar(b), parity, abort_flag, p.status, site);
+            return __all_sync(0xffffffffu, w);
+        };
+        uint32_t g0 = 0;                                    // stream position of this item's first sub-tile
+        bool ok = true;
+        KvItem it;
+        for (int k = 0; ok; ++k) {
+            if (!wait(16 + (k & 1), (k >> 1) & 1, 514)) break;
+            const int idx = item_slot[k & 1];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(18 + (k & 1)));
+            if (!kv_item(p, idx, it)) break;
+            const int buf = k & 1, n_u = it.n_u;
+            ok = wait(0 + buf, (k >> 1) & 1, 510) && wait(4 + g0 % L::kStages, (g0 / L::kStages) & 1, 511);
+            if (!ok) break;
+            tc_fence_after();
+            issue_scores(g0, buf);
+            for (int i = 0; i < n_u && ok; ++i) {
+                const uint32_t g = g0 + i;
+                if (i + 1 < n_u) {
+                    const uint32_t gn = g + 1;
+                    if (!wait(4 + gn % L::kStages, (gn / L::kStages) & 1, 512)) { ok = false; break; }
+                    tc_fence_after();
+                    issue_scores(gn, buf);
+                }
+                if (!wait(12 + (g & 1), (g >> 1) & 1, 513)) { ok = false; break; }
+                // the previous item's dV / dK must have been read out before they are overwritten
+                if (i == 0 && !wait(15, (k & 1) ^ 1, 515)) { ok = false; break; }
+                tc_fence_after();
+                issue_acc(g, i == 0);
+            }
+            if (!ok) break;
+            if (elect_one()) umma_commit(bar(14));
+            __syncwarp();
+            g0 += n_u;
         }
     } else {
         const int q = warp & 3, ch = (warp - 2) >> 2;       // lane quarter, column half (32 of the 64 queries)
         const int r = q * 32 + lane;                        // key row inside the tile
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
         const float sl2 = p.scale * kLog2e;
-        const float* lse_row = p.lse + (static_cast<size_t>(b) * p.H + h) * p.S;
-        const float* dl_row = p.delta + (static_cast<size_t>(b) * p.H + h) * p.S;
+        uint32_t g = 0;                                     // stream position
         bool ok = true;
-        for (int i = 0; i < n_u; ++i) {
-            const int hb = i & 1, qc0 = (u0 + i) * 64 + ch * 32;   // first query column of this thread's slice
-            // -lse*log2e and -delta of this slice's 32 queries, as two-wide operands
-            uint64_t nl2[16], ndl[16];
-#pragma unroll
-            for (int g = 0; g < 8; ++g) {
-                const float4 a = *(reinterpret_cast<const float4*>(lse_row + qc0) + g);
-                const float4 c = *(reinterpret_cast<const float4*>(dl_row + qc0) + g);
-                nl2[2 * g] = pack_f32x2(-a.x * kLog2e, -a.y * kLog2e); nl2[2 * g + 1] = pack_f32x2(-a.z * kLog2e, -a.w * kLog2e);
-                ndl[2 * g] = pack_f32x2(-c.x, -c.y); ndl[2 * g + 1] = pack_f32x2(-c.z, -c.w);
-            }
-            ok = mbar_wait(bar(9 + hb), (i >> 1) & 1, abort_flag, p.status, 520);
+        KvItem it;
+        for (int k = 0; ok; ++k) {
+            ok = mbar_wait(bar(16 + (k & 1)), (k >> 1) & 1, abort_flag, p.status, 522);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            tc_fence_after();
-            uint32_t sv[32], dv[32];
-            tmem_ld32(tmem_base + lane_addr + hb * 64 + ch * 32, sv);
-            tmem_ld32(tmem_base + lane_addr + 128 + hb * 64 + ch * 32, dv);
-            tc_wait_ld();
-            const bool diag = qc0 < kv0 + 128;               // some (key, query) pairs of this slice are masked
-            uint32_t pp[16], dd[16];
-            const uint64_t sl2x2 = pack_f32x2(sl2, sl2);
+            const int idx = item_slot[k & 1];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(18 + (k & 1)));
+            if (!kv_item(p, idx, it)) break;
+            const int kv0 = it.j * 128, u0 = 2 * it.j;
+            const float* lse_row = p.lse + (static_cast<size_t>(it.b) * p.H + it.h) * p.S;
+            const float* dl_row = p.delta + (static_cast<size_t>(it.b) * p.H + it.h) * p.S;
+            for (int i = 0; i < it.n_u; ++i, ++g) {
+                const int hb = g & 1, qc0 = (u0 + i) * 64 + ch * 32;   // first query column of this thread's slice
+                // -lse*log2e and -delta of this slice's 32 queries, as two-wide operands
+                uint64_t nl2[16], ndl[16];
 #pragma unroll
-            for (int c = 0; c < 32; c += 2) {
-                float a0, a1, d0, d1;
-                unpack_f32x2(ffma2(pack_f32x2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), sl2x2, nl2[c >> 1]), a0, a1);
-                float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
-                if (diag) {
-                    if (qc0 + c < kv0 + r) p0 = 0.f;
-                    if (qc0 + c + 1 < kv0 + r) p1 = 0.f;
+                for (int gg = 0; gg < 8; ++gg) {
+                    const float4 a = *(reinterpret_cast<const float4*>(lse_row + qc0) + gg);
+                    const float4 c = *(reinterpret_cast<const float4*>(dl_row + qc0) + gg);
+                    nl2[2 * gg] = pack_f32x2(-a.x * kLog2e, -a.y * kLog2e); nl2[2 * gg + 1] = pack_f32x2(-a.z * kLog2e, -a.w * kLog2e);
+                    ndl[2 * gg] = pack_f32x2(-c.x, -c.y); ndl[2 * gg + 1] = pack_f32x2(-c.z, -c.w);
                 }
-                const uint64_t pv = pack_f32x2(p0, p1);
-                unpack_f32x2(fmul2(pv, fadd2(pack_f32x2(__uint_as_float(dv[c]), __uint_as_float(dv[c + 1])), ndl[c >> 1])), d0, d1);
-                pp[c >> 1] = pack_bf16(p0, p1);
-                dd[c >> 1] = pack_bf16(d0, d1);
+                ok = mbar_wait(bar(10 + hb), (g >> 1) & 1, abort_flag, p.status, 520);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t sv[32], dv[32];
+                tmem_ld32(tmem_base + lane_addr + hb * 64 + ch * 32, sv);
+                tmem_ld32(tmem_base + lane_addr + 128 + hb * 64 + ch * 32, dv);
+                tc_wait_ld();
+                const bool diag = qc0 < kv0 + 128;           // some (key, query) pairs of this slice are masked
+                uint32_t pp[16], dd[16];
+                const uint64_t sl2x2 = pack_f32x2(sl2, sl2);
+#pragma unroll
+                for (int c = 0; c < 32; c += 2) {
+                    float a0, a1, d0, d1;
+                    unpack_f32x2(ffma2(pack_f32x2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), sl2x2, nl2[c >> 1]), a0, a1);
+                    float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
+                    if (diag) {
+                        if (qc0 + c < kv0 + r) p0 = 0.f;
+                        if (qc0 + c + 1 < kv0 + r) p1 = 0.f;
+                    }
+                    const uint64_t pv = pack_f32x2(p0, p1);
+                    unpack_f32x2(fmul2(pv, fadd2(pack_f32x2(__uint_as_float(dv[c]), __uint_as_float(dv[c + 1])), ndl[c >> 1])), d0, d1);
+                    pp[c >> 1] = pack_bf16(p0, p1);
+                    dd[c >> 1] = pack_bf16(d0, d1);
+                }
+                // packed operands go back into this warp's own columns: P^T over S^T, dS^T over dP^T
+                tmem_st16(tmem_base + lane_addr + hb * 64 + ch * 32, pp);
+                tmem_st16(tmem_base + lane_addr + 128 + hb * 64 + ch * 32, dd);
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar(12 + hb));
             }
-            // packed operands go back into this warp's own columns: P^T over S^T, dS^T over dP^T
-            tmem_st16(tmem_base + lane_addr + hb * 64 + ch * 32, pp);
-            tmem_st16(tmem_base + lane_addr + 128 + hb * 64 + ch * 32, dd);
-            tc_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar(11 + hb));
-        }
-        if (ok) {
-            ok = mbar_wait(bar(13), 0, abort_flag, p.status, 521);
-            ok = __all_sync(0xffffffffu, ok);
-        }
-        if (ok) {
+            if (ok) {
+                ok = mbar_wait(bar(14), k & 1, abort_flag, p.status, 521);
+                ok = __all_sync(0xffffffffu, ok);
+            }
+            if (!ok) break;
             tc_fence_after();
             // this warp converts columns [ch*DH/2, +DH/2) of dV and dK and stages them over V_j / K_j
+            const int buf = k & 1;
 #pragma unroll 1
             for (int which = 0; which < 2; ++which) {
-                uint8_t* stage = sm + (which == 0 ? L::kV : L::kK);
+                uint8_t* stage = sm + L::kK + buf * 2 * L::kKV + (which == 0 ? L::kKV : 0);
                 const float mul = which == 0 ? 1.0f : p.scale;
 #pragma unroll 1
                 for (int c = 0; c < DH / 64; ++c) {
@@ -246,12 +341,16 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
                     uint32_t v[32];
                     tmem_ld32(tmem_base + lane_addr + 256 + which * 128 + col0, v);
                     tc_wait_ld();
+                    if (which == 1 && c == DH / 64 - 1) {    // dV and dK have left TMEM: the next item may overwrite them
+                        tc_fence_before();
+                        mbar_arrive(bar(15));
+                    }
 #pragma unroll
-                    for (int g = 0; g < 4; ++g) {
+                    for (int gq = 0; gq < 4; ++gq) {
                         float f[8];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[8 * g + i]) * mul;
-                        const int col = col0 + g * 8, blk = col >> 6, chunk = (col & 63) >> 3;
+                        for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[8 * gq + e]) * mul;
+                        const int col = col0 + gq * 8, blk = col >> 6, chunk = (col & 63) >> 3;
                         *reinterpret_cast<uint4*>(stage + blk * 16384 + r * 128 + ((chunk ^ (r & 7)) << 4)) = pack8(f);
                     }
                 }
@@ -259,14 +358,17 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
             fence_proxy_async();
             named_bar_sync(1, 256);
             if (warp == 2 && lane == 0) {
+                const uint32_t ks = sbase + L::kK + buf * 2 * L::kKV, vs = ks + L::kKV;
                 for (int kb = 0; kb < L::kBlocks; ++kb) {
-                    tma_store_2d(&tmOut, sbase + L::kK + kb * 16384, d + h * DH + kb * 64, row_base + kv0);
-                    tma_store_2d(&tmOut, sbase + L::kV + kb * 16384, 2 * d + h * DH + kb * 64, row_base + kv0);
+                    tma_store_2d(&tmOut, ks + kb * 16384, d + it.h * DH + kb * 64, it.b * p.S + kv0);
+                    tma_store_2d(&tmOut, vs + kb * 16384, 2 * d + it.h * DH + kb * 64, it.b * p.S + kv0);
                 }
                 bulk_commit();
-                bulk_wait0();
+                bulk_wait_read0();                          // the buffer may take another item's K / V
+                mbar_arrive(bar(2 + buf));
             }
         }
+        if (warp == 2 && lane == 0) bulk_wait0();
     }
 
     __syncwarp();
@@ -290,9 +392,25 @@ struct DqSmem {
     static constexpr int kSub = 64 * DH * 2;                 // 64-key sub-tile of K or V
     static constexpr int kQ = 0;                             // Q_A, Q_B, dO_A, dO_B
     static constexpr int kKV = 4 * kTile;                    // 2 stages x (K_v, V_v)
-    static constexpr int kBars = kKV + 4 * kSub;
+    static constexpr int kOut = kKV + 4 * kSub;              // dQ staging tile (shared by both query tiles)
+    static constexpr int kBars = kOut + kTile;
     static constexpr int kBytes = kBars + 256 + 1024;
 };
+
+// Work items of the dQ kernel: one per (sequence, head, pair of query tiles), heaviest first, drawn
+// from a global counter by the producer thread (same scheme as the forward kernel).
+struct DqItem { int b, h, q0A, nA, nB; };
+__device__ __forceinline__ bool dq_item(const BwdParams& p, int idx, DqItem& it)
+{
+    if (idx >= p.n_items) return false;
+    const int BH = p.B * p.H;
+    const int pair = p.tiles_per_seq - 1 - idx / BH, bh = idx % BH;
+    it.b = bh / p.H; it.h = bh % p.H;
+    it.q0A = pair * 256;
+    it.nA = it.q0A / 64 + 2;                                // 64-key sub-tiles each query tile needs
+    it.nB = it.q0A + 128 < p.S ? it.nA + 2 : 0;
+    return true;
+}
 
 template <int DH>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -307,26 +425,51 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
     uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(sm);
     uint64_t* bars = reinterpret_cast<uint64_t*>(sm + L::kBars);
-    // 0 q_full | 1,2 kv_full | 3,4 kv_empty | 5,6 s_full[t] | 7,8 ds_full[t] | 9,10 acc_full[t]
+    // barrier map (t = query tile, s = ring stage):
+    //   0+t q_full | 2+t q_empty | 4+s kv_full | 6+s kv_empty | 8+t s_full | 10+t ds_full (128 arrivals)
+    //   12+t acc_full | 14+t acc_empty (128 arrivals) | 16 staging free | 17+i item_full | 19+i item_empty (9 arrivals)
     const uint32_t bar0 = smem_u32(bars);
     auto bar = [&](int i) { return bar0 + 8u * i; };
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 22);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* item_slot = reinterpret_cast<volatile int*>(tmem_slot + 2);   // two entries
+    // draws the next item number; past the end, counts this CTA as done and lets the last one clear the counters
+    auto draw = [&]() {
+        const int idx = atomicAdd(p.sched, 1);
+        if (idx >= p.n_items && atomicAdd(p.sched + 1, 1) == static_cast<int>(gridDim.x) - 1) {
+            p.sched[0] = 0; p.sched[1] = 0;
+            __threadfence();
+        }
+        return idx;
+    };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int pair = gridDim.x - 1 - blockIdx.x;            // heaviest (latest) query tiles first
-    const int b = blockIdx.y / p.H, h = blockIdx.y % p.H;
     const int d = p.H * DH;
-    const int q0A = pair * 256, q0B = q0A + 128;
-    const bool hasB = q0B < p.S;
-    const int nA = q0A / 64 + 2, nB = hasB ? nA + 2 : 0;    // 64-key sub-tiles each query tile needs
-    const int n_kv = hasB ? nB : nA;
-    const int row_base = b * p.S;
+
+    auto load_q = [&](const DqItem& it, int t) {            // Q_t and dO_t
+        mbar_arrive_expect_tx(bar(0 + t), 2 * L::kTile);
+        for (int kb = 0; kb < L::kBlocks; ++kb) {
+            tma_load_2d(sbase + L::kQ + t * L::kTile + kb * 16384, &tmQ, it.h * DH + kb * 64, it.b * p.S + it.q0A + t * 128, bar(0 + t));
+            tma_load_2d(sbase + L::kQ + (2 + t) * L::kTile + kb * 16384, &tmDO, it.h * DH + kb * 64, it.b * p.S + it.q0A + t * 128, bar(0 + t));
+        }
+    };
+    auto load_kv = [&](const DqItem& it, int v, int s) {    // K_v and V_v (64 keys)
+        mbar_arrive_expect_tx(bar(4 + s), 2 * L::kSub);
+        const uint32_t ks = sbase + L::kKV + s * 2 * L::kSub, vs = ks + L::kSub;
+        for (int kb = 0; kb < L::kBlocks; ++kb) {
+            tma_load_2d(ks + kb * 8192, &tmKV, d + it.h * DH + kb * 64, it.b * p.S + v * 64, bar(4 + s));
+            tma_load_2d(vs + kb * 8192, &tmKV, 2 * d + it.h * DH + kb * 64, it.b * p.S + v * 64, bar(4 + s));
+        }
+    };
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 7; ++i) mbar_init(bar(i), 1);
-        mbar_init(bar(7), 128); mbar_init(bar(8), 128);
-        mbar_init(bar(9), 1); mbar_init(bar(10), 1);
+        for (int i = 0; i < 10; ++i) mbar_init(bar(i), 1);
+        mbar_init(bar(10), 128); mbar_init(bar(11), 128);
+        mbar_init(bar(12), 1); mbar_init(bar(13), 1);
+        mbar_init(bar(14), 128); mbar_init(bar(15), 128);
+        mbar_init(bar(16), 1);
+        mbar_init(bar(17), 1); mbar_init(bar(18), 1);
+        mbar_init(bar(19), 9); mbar_init(bar(20), 9);
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -335,21 +478,16 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
     grid_dep_launch();
     grid_dep_wait();                                        // inputs come from the previous kernels
     if (threadIdx.x == 0) {
-        // first loads go out before the TMEM allocation and the CTA-wide barrier
-        const int nq = hasB ? 2 : 1;
-        mbar_arrive_expect_tx(bar(0), nq * 2 * L::kTile);
-        for (int t = 0; t < nq; ++t)
-            for (int kb = 0; kb < L::kBlocks; ++kb) {
-                tma_load_2d(sbase + L::kQ + t * L::kTile + kb * 16384, &tmQ, h * DH + kb * 64, row_base + q0A + t * 128, bar(0));
-                tma_load_2d(sbase + L::kQ + (2 + t) * L::kTile + kb * 16384, &tmDO, h * DH + kb * 64, row_base + q0A + t * 128, bar(0));
-            }
-        for (int v = 0; v < 2 && v < n_kv; ++v) {
-            mbar_arrive_expect_tx(bar(1 + v), 2 * L::kSub);
-            const uint32_t ks = sbase + L::kKV + v * 2 * L::kSub, vs = ks + L::kSub;
-            for (int kb = 0; kb < L::kBlocks; ++kb) {
-                tma_load_2d(ks + kb * 8192, &tmKV, d + h * DH + kb * 64, row_base + v * 64, bar(1 + v));
-                tma_load_2d(vs + kb * 8192, &tmKV, 2 * d + h * DH + kb * 64, row_base + v * 64, bar(1 + v));
-            }
+        // the first item's first loads go out before the TMEM allocation and the CTA-wide barrier
+        DqItem it;
+        const int idx0 = draw();
+        item_slot[0] = idx0;
+        mbar_arrive(bar(17));
+        if (dq_item(p, idx0, it)) {
+            load_kv(it, 0, 0);
+            load_q(it, 0);
+            if (it.nB) load_q(it, 1);
+            load_kv(it, 1, 1);
         }
     }
     if (warp == 1) {
@@ -364,27 +502,54 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int v = 2; v < n_kv; ++v) {                // Q, dO and the first two sub-tiles were requested in the prologue
-                const int s = v & 1, ph = (v >> 1) & 1;
-                if (!mbar_wait(bar(3 + s), ph ^ 1, abort_flag, p.status, 600)) break;
-                mbar_arrive_expect_tx(bar(1 + s), 2 * L::kSub);
-                const uint32_t ks = sbase + L::kKV + s * 2 * L::kSub, vs = ks + L::kSub;
-                for (int kb = 0; kb < L::kBlocks; ++kb) {
-                    tma_load_2d(ks + kb * 8192, &tmKV, d + h * DH + kb * 64, row_base + v * 64, bar(1 + s));
-                    tma_load_2d(vs + kb * 8192, &tmKV, 2 * d + h * DH + kb * 64, row_base + v * 64, bar(1 + s));
+            uint32_t n = 0;                                 // key sub-tiles requested so far
+            uint32_t qn[2] = {0, 0};                        // items each query tile took part in
+            bool ok = true;
+            DqItem it;
+            int idx = item_slot[0];
+            for (int k = 0; ok && dq_item(p, idx, it); ++k) {
+                const int n_kv = it.nB ? it.nB : it.nA;
+                for (int v = 0; v < n_kv && ok; ++v, ++n) {
+                    const int s = n & 1;
+                    const uint32_t ph = (n >> 1) & 1;
+                    const bool early = k == 0 && v < 2;     // requested in the prologue
+                    if (!early) {
+                        if (!mbar_wait(bar(6 + s), ph ^ 1, abort_flag, p.status, 600)) { ok = false; break; }
+                        load_kv(it, v, s);
+                    }
+                    if (v == 0) {
+                        // Q_t / dO_t follow the first key sub-tile; their buffers are free once the
+                        // previous item's last scores of tile t have been computed
+                        for (int t = 0; t < (it.nB ? 2 : 1) && ok; ++t) {
+                            if (k > 0) {
+                                if (!mbar_wait(bar(2 + t), (qn[t] & 1) ^ 1, abort_flag, p.status, 601)) { ok = false; break; }
+                                load_q(it, t);
+                            }
+                            ++qn[t];
+                        }
+                    }
                 }
+                if (!ok) break;
+                const int kn = k + 1;
+                if (!mbar_wait(bar(19 + (kn & 1)), ((kn >> 1) & 1) ^ 1, abort_flag, p.status, 602)) break;
+                idx = draw();
+                item_slot[kn & 1] = idx;
+                mbar_arrive(bar(17 + (kn & 1)));
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc_sc = make_idesc_bf16(128, 64, false, false);
-            constexpr uint32_t idesc_dq = make_idesc_bf16(128, DH, false, true);
-            auto issue_scores = [&](int t, int s) {         // S_t = Q_t K_v^T, dP_t = dO_t V_v^T
-                const uint64_t dq = make_smem_desc_sw128(sbase + L::kQ + t * L::kTile, 16, 1024);
-                const uint64_t dg = desc_advance(dq, 2 * L::kTile);
-                const uint64_t dk = make_smem_desc_sw128(sbase + L::kKV + s * 2 * L::kSub, 16, 1024);
-                const uint64_t dv = desc_advance(dk, L::kSub);
-                const uint32_t dst = tmem_base + t * 256;
+        // converged warp, one elected lane issues (see the forward kernel)
+        constexpr uint32_t idesc_sc = make_idesc_bf16(128, 64, false, false);
+        constexpr uint32_t idesc_dq = make_idesc_bf16(128, DH, false, true);
+        const uint32_t tb = __shfl_sync(0xffffffffu, tmem_base, 0);
+        const uint32_t sb = __shfl_sync(0xffffffffu, sbase, 0);
+        auto issue_scores = [&](int t, int s) {             // S_t = Q_t K_v^T, dP_t = dO_t V_v^T
+            const uint64_t dq = make_smem_desc_sw128(sb + L::kQ + t * L::kTile, 16, 1024);
+            const uint64_t dg = desc_advance(dq, 2 * L::kTile);
+            const uint64_t dk = make_smem_desc_sw128(sb + L::kKV + s * 2 * L::kSub, 16, 1024);
+            const uint64_t dv = desc_advance(dk, L::kSub);
+            const uint32_t dst = tb + t * 256;
+            if (elect_one()) {
 #pragma unroll
                 for (int kb = 0; kb < L::kBlocks; ++kb)
 #pragma unroll
@@ -397,109 +562,171 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
                     for (int kk = 0; kk < 4; ++kk)
                         umma_f16(dst + 64, desc_advance(dg, kb * 16384 + kk * 32), desc_advance(dv, kb * 8192 + kk * 32),
                                  idesc_sc, (kb | kk) ? 1u : 0u);
-                umma_commit(bar(5 + t));
-            };
-            auto issue_dq = [&](int t, int s, bool acc) {   // dQ_t += dS_t K_v (dS packed in the S columns)
-                const uint64_t dk = make_smem_desc_sw128(sbase + L::kKV + s * 2 * L::kSub, 8192, 1024);
-                const uint32_t dst = tmem_base + t * 256 + 128, src = tmem_base + t * 256;
+                umma_commit(bar(8 + t));
+            }
+            __syncwarp();
+        };
+        auto issue_dq = [&](int t, int s, bool acc) {       // dQ_t += dS_t K_v (dS packed in the S columns)
+            const uint64_t dk = make_smem_desc_sw128(sb + L::kKV + s * 2 * L::kSub, 8192, 1024);
+            const uint32_t dst = tb + t * 256 + 128, src = tb + t * 256;
+            if (elect_one()) {
                 umma_f16_ta(dst, src, dk, idesc_dq, acc ? 1u : 0u);
 #pragma unroll
                 for (int kq = 1; kq < 4; ++kq) umma_f16_ta(dst, src + kq * 8, desc_advance(dk, kq * 2048), idesc_dq, 1u);
-            };
-            bool ok = mbar_wait(bar(0), 0, abort_flag, p.status, 610) && mbar_wait(bar(1), 0, abort_flag, p.status, 611);
-            if (ok) {
+            }
+            __syncwarp();
+        };
+        auto commit = [&](int b) {
+            if (elect_one()) umma_commit(bar(b));
+            __syncwarp();
+        };
+        auto wait = [&](int b, uint32_t parity, int site) {
+            const bool w = mbar_wait(bar(b), parity, abort_flag, p.status, site);
+            return __all_sync(0xffffffffu, w);
+        };
+        uint32_t n = 0;                                     // key sub-tiles consumed before this item
+        uint32_t nd[2] = {0, 0};                            // dS tiles consumed per query tile
+        uint32_t qn[2] = {0, 0};                            // items each query tile took part in
+        bool ok = true;
+        DqItem it;
+        for (int k = 0; ok; ++k) {
+            if (!wait(17 + (k & 1), (k >> 1) & 1, 616)) break;
+            const int idx = item_slot[k & 1];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(19 + (k & 1)));
+            if (!dq_item(p, idx, it)) break;
+            const int nA = it.nA, nB = it.nB, n_kv = nB ? nB : nA;
+            {
+                const int s = n & 1;
+                const uint32_t ph = (n >> 1) & 1;
+                ok = wait(4 + s, ph, 611) && wait(0, qn[0] & 1, 610);
+                if (!ok) break;
                 tc_fence_after();
-                issue_scores(0, 0);
-                if (hasB) issue_scores(1, 0);
+                issue_scores(0, s);
+                if (nB) {
+                    if (!wait(1, qn[1] & 1, 617)) { ok = false; break; }
+                    tc_fence_after();
+                    issue_scores(1, s);
+                }
             }
             for (int v = 0; v < n_kv && ok; ++v) {
-                const int s = v & 1, nxt = v + 1, sn = nxt & 1, phn = (nxt >> 1) & 1;
+                const uint32_t nv = n + v, nn = nv + 1;
+                const int s = nv & 1, sn = nn & 1;
+                const uint32_t phn = (nn >> 1) & 1;
                 bool k_waited = false;
                 if (v < nA) {
-                    if (!mbar_wait(bar(7), v & 1, abort_flag, p.status, 612)) { ok = false; break; }
+                    if (!wait(10, nd[0] & 1, 612)) { ok = false; break; }
+                    ++nd[0];
+                    // the previous item's dQ_A must have been read out before it is overwritten
+                    if (v == 0 && !wait(14, (qn[0] & 1) ^ 1, 618)) { ok = false; break; }
                     tc_fence_after();
                     issue_dq(0, s, v > 0);
-                    if (v == nA - 1) umma_commit(bar(9));
+                    if (v == nA - 1) commit(12);
                 }
-                if (nxt < nA) {
-                    if (!mbar_wait(bar(1 + sn), phn, abort_flag, p.status, 613)) { ok = false; break; }
+                if (v + 1 < nA) {
+                    if (!wait(4 + sn, phn, 613)) { ok = false; break; }
                     k_waited = true;
                     tc_fence_after();
                     issue_scores(0, sn);
+                    if (v + 2 == nA) commit(2);             // Q_A / dO_A are not needed again
                 }
                 if (v < nB) {
-                    if (!mbar_wait(bar(8), v & 1, abort_flag, p.status, 614)) { ok = false; break; }
+                    if (!wait(11, nd[1] & 1, 614)) { ok = false; break; }
+                    ++nd[1];
+                    if (v == 0 && !wait(15, (qn[1] & 1) ^ 1, 619)) { ok = false; break; }
                     tc_fence_after();
                     issue_dq(1, s, v > 0);
-                    if (v == nB - 1) umma_commit(bar(10));
+                    if (v == nB - 1) commit(13);
                 }
-                umma_commit(bar(3 + s));                    // K_v / V_v stage free
-                if (nxt < nB) {
-                    if (!k_waited && !mbar_wait(bar(1 + sn), phn, abort_flag, p.status, 615)) { ok = false; break; }
+                commit(6 + s);                              // K_v / V_v stage free
+                if (v + 1 < nB) {
+                    if (!k_waited && !wait(4 + sn, phn, 615)) { ok = false; break; }
                     tc_fence_after();
                     issue_scores(1, sn);
+                    if (v + 2 == nB) commit(3);
                 }
             }
+            n += n_kv;
+            ++qn[0];
+            if (nB) ++qn[1];
         }
     } else {
         const int t = (warp - 2) >> 2, q = warp & 3;
         const int r = q * 32 + lane;
-        const int q0 = t == 0 ? q0A : q0B;
-        const int n_t = t == 0 ? nA : nB;
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
         const uint32_t s_addr = tmem_base + lane_addr + t * 256;
         const float sl2 = p.scale * kLog2e;
-        float lse2 = 0.f, dlt = 0.f;
-        if (n_t > 0) {
-            const size_t idx = (static_cast<size_t>(b) * p.H + h) * p.S + q0 + r;
-            lse2 = p.lse[idx] * kLog2e;
-            dlt = p.delta[idx];
-        }
+        uint32_t ns = 0, qn = 0;                            // score tiles and items this query tile has seen
+        uint32_t u_base = 0;                                // uses of the staging tile before this item
         bool ok = true;
-        for (int v = 0; v < n_t; ++v) {
-            ok = mbar_wait(bar(5 + t), v & 1, abort_flag, p.status, 620);
+        DqItem it;
+        for (int k = 0; ok; ++k) {
+            ok = mbar_wait(bar(17 + (k & 1)), (k >> 1) & 1, abort_flag, p.status, 622);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            tc_fence_after();
-            const bool diag = v * 64 + 63 > q0;              // some keys of this sub-tile are masked for some rows
-            const uint64_t sl2x2 = pack_f32x2(sl2, sl2), nlse2 = pack_f32x2(-lse2, -lse2), ndlt = pack_f32x2(-dlt, -dlt);
+            const int idx = item_slot[k & 1];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(19 + (k & 1)));
+            if (!dq_item(p, idx, it)) break;
+            const int n_t = t == 0 ? it.nA : it.nB;
+            const uint32_t u = u_base + t;                  // staging order: A(k), B(k), A(k+1), ...
+            u_base += it.nB ? 2 : 1;
+            if (n_t == 0) continue;
+            const int q0 = it.q0A + t * 128;
+            const size_t row_idx = (static_cast<size_t>(it.b) * p.H + it.h) * p.S + q0 + r;
+            const float lse2 = p.lse[row_idx] * kLog2e, dlt = p.delta[row_idx];
+            for (int v = 0; v < n_t; ++v, ++ns) {
+                ok = mbar_wait(bar(8 + t), ns & 1, abort_flag, p.status, 620);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                const bool diag = v * 64 + 63 > q0;          // some keys of this sub-tile are masked for some rows
+                const uint64_t sl2x2 = pack_f32x2(sl2, sl2), nlse2 = pack_f32x2(-lse2, -lse2), ndlt = pack_f32x2(-dlt, -dlt);
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t sv[32], dv[32], ds[16];
-                tmem_ld32(s_addr + c * 32, sv);
-                tmem_ld32(s_addr + 64 + c * 32, dv);
-                tc_wait_ld();
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t sv[32], dv[32], ds[16];
+                    tmem_ld32(s_addr + c * 32, sv);
+                    tmem_ld32(s_addr + 64 + c * 32, dv);
+                    tc_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    float a0, a1, d0, d1;
-                    unpack_f32x2(ffma2(pack_f32x2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), sl2x2, nlse2), a0, a1);
-                    float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
-                    if (diag) {
-                        const int key = v * 64 + c * 32 + i;
-                        if (key > q0 + r) p0 = 0.f;
-                        if (key + 1 > q0 + r) p1 = 0.f;
+                    for (int i = 0; i < 32; i += 2) {
+                        float a0, a1, d0, d1;
+                        unpack_f32x2(ffma2(pack_f32x2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), sl2x2, nlse2), a0, a1);
+                        float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
+                        if (diag) {
+                            const int key = v * 64 + c * 32 + i;
+                            if (key > q0 + r) p0 = 0.f;
+                            if (key + 1 > q0 + r) p1 = 0.f;
+                        }
+                        unpack_f32x2(fmul2(pack_f32x2(p0, p1), fadd2(pack_f32x2(__uint_as_float(dv[i]), __uint_as_float(dv[i + 1])), ndlt)), d0, d1);
+                        ds[i >> 1] = pack_bf16(d0, d1);
                     }
-                    unpack_f32x2(fmul2(pack_f32x2(p0, p1), fadd2(pack_f32x2(__uint_as_float(dv[i]), __uint_as_float(dv[i + 1])), ndlt)), d0, d1);
-                    ds[i >> 1] = pack_bf16(d0, d1);
+                    tmem_st16(s_addr + c * 16, ds);
                 }
-                tmem_st16(s_addr + c * 16, ds);
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar(10 + t));
             }
-            tc_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar(7 + t));
-        }
-        if (ok && n_t > 0) {
-            ok = mbar_wait(bar(9 + t), 0, abort_flag, p.status, 621);
-            ok = __all_sync(0xffffffffu, ok);
-        }
-        if (ok && n_t > 0) {
+            if (ok) {
+                ok = mbar_wait(bar(12 + t), qn & 1, abort_flag, p.status, 621);
+                ok = __all_sync(0xffffffffu, ok);
+            }
+            if (ok) {
+                ok = mbar_wait(bar(16), (u & 1) ^ 1, abort_flag, p.status, 623);    // the previous user's store has read the staging tile
+                ok = __all_sync(0xffffffffu, ok);
+            }
+            if (!ok) break;
             tc_fence_after();
-            uint8_t* stage = sm + L::kQ + t * L::kTile;     // Q_t is idle now
+            uint8_t* stage = sm + L::kOut;
 #pragma unroll 1
             for (int c = 0; c < DH / 32; ++c) {
                 uint32_t v[32];
                 tmem_ld32(s_addr + 128 + c * 32, v);
                 tc_wait_ld();
+                if (c == DH / 32 - 1) {                     // dQ_t has left TMEM: the next item may overwrite it
+                    tc_fence_before();
+                    mbar_arrive(bar(14 + t));
+                }
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
                     float f[8];
@@ -513,11 +740,14 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
             named_bar_sync(1 + t, 128);
             if ((warp & 3) == 2 && lane == 0) {
                 for (int kb = 0; kb < L::kBlocks; ++kb)
-                    tma_store_2d(&tmOut, sbase + L::kQ + t * L::kTile + kb * 16384, h * DH + kb * 64, row_base + q0);
+                    tma_store_2d(&tmOut, sbase + L::kOut + kb * 16384, it.h * DH + kb * 64, it.b * p.S + q0);
                 bulk_commit();
-                bulk_wait0();
+                bulk_wait_read0();                          // the staging tile may be written again
+                mbar_arrive(bar(16));
             }
+            ++qn;
         }
+        if ((warp & 3) == 2 && lane == 0) bulk_wait0();
     }
 
     __syncwarp();
@@ -580,7 +810,9 @@ const char* launch_attention_bwd_dq(Runtime* rt, const void* qkv, const void* do
     p.S = S; p.H = H; p.scale = 1.0f / sqrtf(static_cast<float>(dh));
     p.lse = static_cast<const float*>(lse); p.delta = static_cast<const float*>(delta);
     p.status = status;
-    dim3 grid((S + 255) / 256, B * H);
+    p.B = B; p.tiles_per_seq = (S + 255) / 256; p.n_items = B * H * p.tiles_per_seq;
+    p.sched = status->sched + 2;
+    dim3 grid(p.n_items < rt->sm_count ? p.n_items : rt->sm_count);
     const cudaError_t e2 = dh == 64
         ? launch_k(attn_bwd_dq_tc_kernel<64>, grid, dim3(kThreads), DqSmem<64>::kBytes, stream, tmQ, tmDO, tmKV, tmOut, p)
         : launch_k(attn_bwd_dq_tc_kernel<128>, grid, dim3(kThreads), DqSmem<128>::kBytes, stream, tmQ, tmDO, tmKV, tmOut, p);
@@ -603,7 +835,9 @@ const char* launch_attention_bwd_dkdv(Runtime* rt, const void* qkv, const void* 
     p.S = S; p.H = H; p.scale = 1.0f / sqrtf(static_cast<float>(dh));
     p.lse = static_cast<const float*>(lse); p.delta = static_cast<const float*>(delta);
     p.status = status;
-    dim3 grid(S / 128, B * H);
+    p.B = B; p.tiles_per_seq = S / 128; p.n_items = B * H * p.tiles_per_seq;
+    p.sched = status->sched + 4;
+    dim3 grid(p.n_items < rt->sm_count ? p.n_items : rt->sm_count);
     const cudaError_t e2 = dh == 64
         ? launch_k(attn_bwd_dkdv_tc_kernel<64>, grid, dim3(kThreads), KvSmem<64>::kBytes, stream, tmKV, tmQ, tmDO, tmOut, p)
         : launch_k(attn_bwd_dkdv_tc_kernel<128>, grid, dim3(kThreads), KvSmem<128>::kBytes, stream, tmKV, tmQ, tmDO, tmOut, p);
