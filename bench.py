@@ -32,8 +32,9 @@ sys.path.insert(0, ROOT)
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram bytes read+written per GEMM launch (average over the 12 GEMM launches of a workload-2 step),
-# from the ncu capture summarised in profiles/; None until a capture exists for the workload.
-GEMM_DRAM_TRAFFIC_PER_LAUNCH = {}
+# from the ncu capture summarised in profiles/gemm_pair_kernel_cfg2_dram_traffic.md; None for
+# workloads without a capture.
+GEMM_DRAM_TRAFFIC_PER_LAUNCH = {"cfg2_d2048_s1024_b8": 223.0e6}
 
 
 def load_peaks():
@@ -382,7 +383,7 @@ def main():
     ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4])
     ap.add_argument("--dispatch", default="async", choices=["opbyop", "async", "graph"])
     ap.add_argument("--seed", type=int, default=0)
-    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--e2e-steps", type=int, default=30)
     ap.add_argument("--cpu-sample-batch", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -68,7 +68,7 @@ enum { PW_ACT_GELU_ERF = 0, PW_ACT_GELU_TANH = 1 };
 
 /* Static shape of a layer call - fixed for the life of the handle, like the static shapes of
  * a compiled function (Section 3).  Supported: head_dim in {64, 128}; n_heads*head_dim ==
- * d_model; d_model % 256 == 0 and d_model <= 8192; d_ff % 128 == 0; seq_len % 64 == 0;
+ * d_model; d_model % 256 == 0 and d_model <= 8192; d_ff % 128 == 0; seq_len % 128 == 0;
  * batch >= 1; causal == 1.  Anything else gives PW_ERR_UNSUPPORTED_SHAPE (never a slow path). */
 typedef struct pw_layer_config {
     uint32_t struct_size; /* sizeof(pw_layer_config_t), for versioning */

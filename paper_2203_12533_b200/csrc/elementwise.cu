@@ -38,6 +38,19 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
+__device__ __forceinline__ void unpack8_pairs(const uint4& v, uint64_t* p)
+{
+    p[0] = pack_f32x2(bf16_lo(v.x), bf16_hi(v.x)); p[1] = pack_f32x2(bf16_lo(v.y), bf16_hi(v.y));
+    p[2] = pack_f32x2(bf16_lo(v.z), bf16_hi(v.z)); p[3] = pack_f32x2(bf16_lo(v.w), bf16_hi(v.w));
+}
+__device__ __forceinline__ uint32_t pack_pair_bf16(uint64_t p)
+{
+    float lo, hi;
+    unpack_f32x2(p, lo, hi);
+    return pack_bf16(lo, hi);
+}
+__device__ __forceinline__ uint64_t splat2(float v) { return pack_f32x2(v, v); }
+
 // LayerNorm forward.  A row is handled by W warps (W = 1 for d <= 2048), each lane holding CH
 // 16-byte pieces (lane i of warp w owns columns 8*(i + 32*(w + W*j)) .. +7, j < CH): all of a
 // lane's loads are issued at once, the statistics need only warp shuffles (plus one shared-memory
@@ -56,17 +69,20 @@ ln_fwd_kernel(const __nv_bfloat16* x, const __nv_bfloat16* gamma,
     const bool live = row < T && row_in_cta < rows_per_cta;
     grid_dep_launch();
     grid_dep_wait();
-    float v[CH][8];
-    float s = 0.f;
+    // two-wide fp32 throughout: neighbouring columns share a 64-bit register
+    uint64_t v[CH][4];
+    uint64_t acc = 0ull;
 #pragma unroll
     for (int j = 0; j < CH; ++j) {
         const int col = 8 * (lane + 32 * (wr + W * j));
         const uint4 raw = live ? *reinterpret_cast<const uint4*>(x + static_cast<size_t>(row) * d + col) : make_uint4(0, 0, 0, 0);
-        unpack8(raw, v[j]);
+        unpack8_pairs(raw, v[j]);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) s += v[j][k];
+        for (int k = 0; k < 4; ++k) acc = fadd2(acc, v[j][k]);
     }
-    s = warp_sum(s);
+    float a0, a1;
+    unpack_f32x2(acc, a0, a1);
+    float s = warp_sum(a0 + a1);
     if (W > 1) {
         if (lane == 0) red[0][warp] = s;
         __syncthreads();
@@ -74,12 +90,14 @@ ln_fwd_kernel(const __nv_bfloat16* x, const __nv_bfloat16* gamma,
         for (int i = 0; i < W; ++i) s += red[0][row_in_cta * W + i];
     }
     const float mean = s / d;
-    float q = 0.f;
+    const uint64_t nmean = splat2(-mean);
+    acc = 0ull;
 #pragma unroll
     for (int j = 0; j < CH; ++j)
 #pragma unroll
-        for (int k = 0; k < 8; ++k) { const float c = v[j][k] - mean; q += c * c; }
-    q = warp_sum(q);
+        for (int k = 0; k < 4; ++k) { const uint64_t c = fadd2(v[j][k], nmean); acc = ffma2(c, c, acc); }
+    unpack_f32x2(acc, a0, a1);
+    float q = warp_sum(a0 + a1);
     if (W > 1) {
         if (lane == 0) red[1][warp] = q;
         __syncthreads();
@@ -88,15 +106,19 @@ ln_fwd_kernel(const __nv_bfloat16* x, const __nv_bfloat16* gamma,
     }
     const float r = rsqrtf(q / d + eps);
     if (!live) return;
+    const uint64_t r2 = splat2(r), nmr2 = splat2(-mean * r);
 #pragma unroll
     for (int j = 0; j < CH; ++j) {
         const int col = 8 * (lane + 32 * (wr + W * j));
-        float g[8], b[8], o[8];
-        unpack8(*(reinterpret_cast<const uint4*>(gamma + col)), g);
-        unpack8(*(reinterpret_cast<const uint4*>(beta + col)), b);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) o[k] = g[k] * ((v[j][k] - mean) * r) + b[k];
-        *reinterpret_cast<uint4*>(h + static_cast<size_t>(row) * d + col) = pack8(o);
+        uint64_t g[4], b[4];
+        unpack8_pairs(*(reinterpret_cast<const uint4*>(gamma + col)), g);
+        unpack8_pairs(*(reinterpret_cast<const uint4*>(beta + col)), b);
+        uint4 o;
+        o.x = pack_pair_bf16(ffma2(ffma2(v[j][0], r2, nmr2), g[0], b[0]));
+        o.y = pack_pair_bf16(ffma2(ffma2(v[j][1], r2, nmr2), g[1], b[1]));
+        o.z = pack_pair_bf16(ffma2(ffma2(v[j][2], r2, nmr2), g[2], b[2]));
+        o.w = pack_pair_bf16(ffma2(ffma2(v[j][3], r2, nmr2), g[3], b[3]));
+        *reinterpret_cast<uint4*>(h + static_cast<size_t>(row) * d + col) = o;
     }
     if (wr == 0 && lane == 0) { mu[row] = mean; rstd[row] = r; }
 }
@@ -125,19 +147,6 @@ __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, bool 
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-__device__ __forceinline__ void unpack8_pairs(const uint4& v, uint64_t* p)
-{
-    p[0] = pack_f32x2(bf16_lo(v.x), bf16_hi(v.x)); p[1] = pack_f32x2(bf16_lo(v.y), bf16_hi(v.y));
-    p[2] = pack_f32x2(bf16_lo(v.z), bf16_hi(v.z)); p[3] = pack_f32x2(bf16_lo(v.w), bf16_hi(v.w));
-}
-__device__ __forceinline__ uint32_t pack_pair_bf16(uint64_t p)
-{
-    float lo, hi;
-    unpack_f32x2(p, lo, hi);
-    return pack_bf16(lo, hi);
-}
-__device__ __forceinline__ uint64_t splat2(float v) { return pack_f32x2(v, v); }
 
 // The kernel is bound by instruction issue as much as by memory, so all element-wise arithmetic
 // is two-wide fp32 (values of neighbouring columns packed in one 64-bit register).
