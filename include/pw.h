@@ -293,7 +293,11 @@ pw_status_t pw_op_gemm(int layout, int epilogue, int act, int M, int N, int K, c
                        const void* B, int ldb, void* C, int ldc, const void* bias, const void* aux_in,
                        int ld_aux, void* aux_out, int accumulate, void* stream);
 
-/* Causal attention forward on packed qkv (bf16 [T,3d]); o bf16 [T,d]; lse fp32 [B,H,S]. */
+/* Causal attention forward on packed qkv (bf16 [T,3d]); o bf16 [T,d]; lse fp32 [B,H,S].
+ * The attention kernels are persistent and hand out their work through counters that live
+ * beside the status word: the pw_op_attention_* calls of one device share one set, so two of them
+ * must not run on the GPU at the same time (enqueue them on one stream, or order the streams). A
+ * layer handle owns its own counters; different handles may overlap freely. */
 pw_status_t pw_op_attention_fwd(const void* qkv, int B, int S, int H, int dh, void* o, void* lse, void* stream);
 
 /* Causal attention backward.  dout bf16 [T,d]; dqkv bf16 [T,3d] (same packing as qkv);
