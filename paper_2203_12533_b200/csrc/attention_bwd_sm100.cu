@@ -23,6 +23,7 @@ namespace pw {
 namespace {
 
 constexpr int kThreads = 320;
+constexpr int kDqThreads = 576;                            // producer warp, MMA warp, 2 x 8 element-wise warps
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct BwdParams {
@@ -413,7 +414,7 @@ __device__ __forceinline__ bool dq_item(const BwdParams& p, int idx, DqItem& it)
 }
 
 template <int DH>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kDqThreads, 1)
 attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64 x 128 rows
                       const __grid_constant__ CUtensorMap tmDO,   // dout, box 64 x 128 rows
                       const __grid_constant__ CUtensorMap tmKV,   // qkv, box 64 x 64 rows
@@ -426,8 +427,8 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
     const uint32_t sbase = smem_u32(sm);
     uint64_t* bars = reinterpret_cast<uint64_t*>(sm + L::kBars);
     // barrier map (t = query tile, s = ring stage):
-    //   0+t q_full | 2+t q_empty | 4+s kv_full | 6+s kv_empty | 8+t s_full | 10+t ds_full (128 arrivals)
-    //   12+t acc_full | 14+t acc_empty (128 arrivals) | 16 staging free | 17+i item_full | 19+i item_empty (9 arrivals)
+    //   0+t q_full | 2+t q_empty | 4+s kv_full | 6+s kv_empty | 8+t s_full | 10+t ds_full (256 arrivals)
+    //   12+t acc_full | 14+t acc_empty (256 arrivals) | 16 staging free | 17+i item_full | 19+i item_empty (17 arrivals)
     const uint32_t bar0 = smem_u32(bars);
     auto bar = [&](int i) { return bar0 + 8u * i; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 22);
@@ -464,12 +465,12 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < 10; ++i) mbar_init(bar(i), 1);
-        mbar_init(bar(10), 128); mbar_init(bar(11), 128);
+        mbar_init(bar(10), 256); mbar_init(bar(11), 256);
         mbar_init(bar(12), 1); mbar_init(bar(13), 1);
-        mbar_init(bar(14), 128); mbar_init(bar(15), 128);
+        mbar_init(bar(14), 256); mbar_init(bar(15), 256);
         mbar_init(bar(16), 1);
         mbar_init(bar(17), 1); mbar_init(bar(18), 1);
-        mbar_init(bar(19), 9); mbar_init(bar(20), 9);
+        mbar_init(bar(19), 17); mbar_init(bar(20), 17);
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -570,9 +571,11 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
             const uint64_t dk = make_smem_desc_sw128(sb + L::kKV + s * 2 * L::kSub, 8192, 1024);
             const uint32_t dst = tb + t * 256 + 128, src = tb + t * 256;
             if (elect_one()) {
+                // dS packed bf16: keys 0..31 in columns 0..15 of S_t, keys 32..63 in columns 32..47
                 umma_f16_ta(dst, src, dk, idesc_dq, acc ? 1u : 0u);
 #pragma unroll
-                for (int kq = 1; kq < 4; ++kq) umma_f16_ta(dst, src + kq * 8, desc_advance(dk, kq * 2048), idesc_dq, 1u);
+                for (int kq = 1; kq < 4; ++kq)
+                    umma_f16_ta(dst, src + (kq >> 1) * 32 + (kq & 1) * 8, desc_advance(dk, kq * 2048), idesc_dq, 1u);
             }
             __syncwarp();
         };
@@ -651,10 +654,15 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
             if (nB) ++qn[1];
         }
     } else {
-        const int t = (warp - 2) >> 2, q = warp & 3;
+        // Element-wise: two threads per query row.  Warps 2..9 serve tile A, 10..17 tile B; the lane
+        // quarter is warp % 4, the key half hf = (warp - 2) / 4 % 2: a thread owns 32 of the
+        // sub-tile's 64 keys and writes its packed dS over its own S columns.
+        const int t = (warp - 2) >> 3, hf = ((warp - 2) >> 2) & 1, q = warp & 3;
         const int r = q * 32 + lane;
+        const bool leader = hf == 0 && q == 2 && lane == 0;
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
-        const uint32_t s_addr = tmem_base + lane_addr + t * 256;
+        const uint32_t s_addr = tmem_base + lane_addr + t * 256 + hf * 32;       // my S columns; dP is 64 further
+        const uint32_t o_addr = tmem_base + lane_addr + t * 256 + 128 + hf * (DH / 2);
         const float sl2 = p.scale * kLog2e;
         uint32_t ns = 0, qn = 0;                            // score tiles and items this query tile has seen
         uint32_t u_base = 0;                                // uses of the staging tile before this item
@@ -675,33 +683,34 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
             const int q0 = it.q0A + t * 128;
             const size_t row_idx = (static_cast<size_t>(it.b) * p.H + it.h) * p.S + q0 + r;
             const float lse2 = p.lse[row_idx] * kLog2e, dlt = p.delta[row_idx];
+            const uint64_t sl2x2 = pack_f32x2(sl2, sl2), nlse2 = pack_f32x2(-lse2, -lse2), ndlt = pack_f32x2(-dlt, -dlt);
             for (int v = 0; v < n_t; ++v, ++ns) {
                 ok = mbar_wait(bar(8 + t), ns & 1, abort_flag, p.status, 620);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                const bool diag = v * 64 + 63 > q0;          // some keys of this sub-tile are masked for some rows
-                const uint64_t sl2x2 = pack_f32x2(sl2, sl2), nlse2 = pack_f32x2(-lse2, -lse2), ndlt = pack_f32x2(-dlt, -dlt);
+                const int key0 = v * 64 + hf * 32;            // first key of my slice
+                const bool diag = key0 + 31 > q0;            // some keys of this slice are masked for some rows
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
-                    uint32_t sv[32], dv[32], ds[16];
-                    tmem_ld32(s_addr + c * 32, sv);
-                    tmem_ld32(s_addr + 64 + c * 32, dv);
+                    uint32_t sv[16], dv[16], ds[8];
+                    tmem_ld16(s_addr + c * 16, sv);
+                    tmem_ld16(s_addr + 64 + c * 16, dv);
                     tc_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
+                    for (int i = 0; i < 16; i += 2) {
                         float a0, a1, d0, d1;
                         unpack_f32x2(ffma2(pack_f32x2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), sl2x2, nlse2), a0, a1);
                         float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
                         if (diag) {
-                            const int key = v * 64 + c * 32 + i;
+                            const int key = key0 + c * 16 + i;
                             if (key > q0 + r) p0 = 0.f;
                             if (key + 1 > q0 + r) p1 = 0.f;
                         }
                         unpack_f32x2(fmul2(pack_f32x2(p0, p1), fadd2(pack_f32x2(__uint_as_float(dv[i]), __uint_as_float(dv[i + 1])), ndlt)), d0, d1);
                         ds[i >> 1] = pack_bf16(d0, d1);
                     }
-                    tmem_st16(s_addr + c * 16, ds);
+                    tmem_st8(s_addr + c * 8, ds);            // over my own (already loaded) S columns
                 }
                 tc_wait_st();
                 tc_fence_before();
@@ -719,11 +728,11 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
             tc_fence_after();
             uint8_t* stage = sm + L::kOut;
 #pragma unroll 1
-            for (int c = 0; c < DH / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld32(s_addr + 128 + c * 32, v);
+            for (int c = 0; c < DH / 64; ++c) {
+                uint32_t w[32];
+                tmem_ld32(o_addr + c * 32, w);
                 tc_wait_ld();
-                if (c == DH / 32 - 1) {                     // dQ_t has left TMEM: the next item may overwrite it
+                if (c == DH / 64 - 1) {                     // this thread's part of dQ_t has left TMEM
                     tc_fence_before();
                     mbar_arrive(bar(14 + t));
                 }
@@ -731,14 +740,14 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
                 for (int g = 0; g < 4; ++g) {
                     float f[8];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[8 * g + i]) * p.scale;
-                    const int col = c * 32 + g * 8, blk = col >> 6, chunk = (col & 63) >> 3;
+                    for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(w[8 * g + i]) * p.scale;
+                    const int col = hf * (DH / 2) + c * 32 + g * 8, blk = col >> 6, chunk = (col & 63) >> 3;
                     *reinterpret_cast<uint4*>(stage + blk * 16384 + r * 128 + ((chunk ^ (r & 7)) << 4)) = pack8(f);
                 }
             }
             fence_proxy_async();
-            named_bar_sync(1 + t, 128);
-            if ((warp & 3) == 2 && lane == 0) {
+            named_bar_sync(1 + t, 256);
+            if (leader) {
                 for (int kb = 0; kb < L::kBlocks; ++kb)
                     tma_store_2d(&tmOut, sbase + L::kOut + kb * 16384, it.h * DH + kb * 64, it.b * p.S + q0);
                 bulk_commit();
@@ -747,7 +756,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmQ,    // qkv, box 64
             }
             ++qn;
         }
-        if ((warp & 3) == 2 && lane == 0) bulk_wait0();
+        if (leader) bulk_wait0();
     }
 
     __syncwarp();
@@ -814,8 +823,8 @@ const char* launch_attention_bwd_dq(Runtime* rt, const void* qkv, const void* do
     p.sched = status->sched + 2;
     dim3 grid(p.n_items < rt->sm_count ? p.n_items : rt->sm_count);
     const cudaError_t e2 = dh == 64
-        ? launch_k(attn_bwd_dq_tc_kernel<64>, grid, dim3(kThreads), DqSmem<64>::kBytes, stream, tmQ, tmDO, tmKV, tmOut, p)
-        : launch_k(attn_bwd_dq_tc_kernel<128>, grid, dim3(kThreads), DqSmem<128>::kBytes, stream, tmQ, tmDO, tmKV, tmOut, p);
+        ? launch_k(attn_bwd_dq_tc_kernel<64>, grid, dim3(kDqThreads), DqSmem<64>::kBytes, stream, tmQ, tmDO, tmKV, tmOut, p)
+        : launch_k(attn_bwd_dq_tc_kernel<128>, grid, dim3(kDqThreads), DqSmem<128>::kBytes, stream, tmQ, tmDO, tmKV, tmOut, p);
     return e2 == cudaSuccess ? nullptr : "attention bwd (dq) launch failed";
 }
 

@@ -21,7 +21,7 @@
 namespace pw {
 namespace {
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 576;                              // producer warp, MMA warp, 2 x 8 softmax warps
 constexpr float kLog2e = 1.4426950408889634f;
 
 template <int DH>
@@ -33,7 +33,9 @@ struct FwdSmem {
     static constexpr int kV = 4 * kTile;                    // two V stages
     static constexpr int kO = 6 * kTile;                    // output staging tile (shared by both query tiles)
     static constexpr int kBars = 7 * kTile;
-    static constexpr int kBytes = kBars + 256 + 1024;
+    static constexpr int kXch = kBars + 256;                // per-row exchange between the two threads of a row: [tile][half][128] fp32
+    static constexpr int kEnd = kXch + 2 * 2 * 128 * 4;
+    static constexpr int kBytes = kEnd + ((kEnd + 1024 <= 232448) ? 1024 : 232448 - kEnd);   // alignment slack (checked in the kernel)
 };
 
 // Timeline tracing of CTA 0 (one writer thread per role), compiled in only with -DPW_TRACE_ENABLE:
@@ -93,7 +95,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
     // barrier map (t = query tile, s = ring stage):
     //   0+t q_full | 2+t q_empty | 4+s k_full | 6+s k_empty | 8+s v_full | 10+s v_empty
     //   12+t s_full | 14+t p_full (128 arrivals) | 16+t o_full | 18+t o_empty (128 arrivals) | 20 staging free
-    //   21+i item_full | 23+i item_empty (9 arrivals: MMA warp + 8 softmax warps)
+    //   21+i item_full | 23+i item_empty (17 arrivals: MMA warp + 16 softmax warps)
     const uint32_t bar0 = smem_u32(bars);
     auto bar = [&](int i) { return bar0 + 8u * i; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 26);
@@ -111,6 +113,10 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int d = p.H * DH;
+    if (sm + L::kEnd > smem_raw + L::kBytes) {              // the alignment ate more than the slack (never seen; fail loudly)
+        if (threadIdx.x == 0 && atomicCAS(&p.status->code, 0, kStatusTimeout) == 0) p.status->site = 499;
+        return;
+    }
     int trace_n = 0;                                        // used by PW_TRACE only
     (void)trace_n;
 
@@ -135,12 +141,12 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < 14; ++i) mbar_init(bar(i), 1);
-        mbar_init(bar(14), 128); mbar_init(bar(15), 128);
+        mbar_init(bar(14), 256); mbar_init(bar(15), 256);
         mbar_init(bar(16), 1); mbar_init(bar(17), 1);
-        mbar_init(bar(18), 128); mbar_init(bar(19), 128);
+        mbar_init(bar(18), 256); mbar_init(bar(19), 256);
         mbar_init(bar(20), 1);
         mbar_init(bar(21), 1); mbar_init(bar(22), 1);
-        mbar_init(bar(23), 9); mbar_init(bar(24), 9);
+        mbar_init(bar(23), 17); mbar_init(bar(24), 17);
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -240,7 +246,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
             }
             __syncwarp();
         };
-        // O_t (+)= P_t V from V stage s; P_t is bf16 packed in the first 64 columns of S_t
+        // O_t (+)= P_t V from V stage s; P_t is bf16 packed over the S columns it came from: keys
+        // 0..63 in columns 0..31 of S_t, keys 64..127 in columns 64..95
         auto issue_pv = [&](int t, int s, bool acc) {
             const uint64_t dv = make_smem_desc_sw128(sb + L::kV + s * L::kTile, 16384, 1024);
             const uint32_t dst = tb + 256 + t * 128, src = tb + t * 128;
@@ -248,7 +255,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                 umma_f16_ta(dst, src, dv, idesc_pv, acc ? 1u : 0u);
 #pragma unroll
                 for (int ks = 1; ks < 8; ++ks)
-                    umma_f16_ta(dst, src + ks * 8, desc_advance(dv, ks * 2048), idesc_pv, 1u);
+                    umma_f16_ta(dst, src + (ks >> 2) * 64 + (ks & 3) * 8, desc_advance(dv, ks * 2048), idesc_pv, 1u);
             }
             __syncwarp();
         };
@@ -339,12 +346,21 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
             if (nB) ++qn[1];
         }
     } else {
-        const int t = (warp - 2) >> 2;                      // 0 = tile A, 1 = tile B
+        // Softmax: two threads per query row.  Warps 2..9 serve tile A, 10..17 tile B; inside a tile
+        // the warp's TMEM lane quarter is warp % 4 and its column half hf is (warp - 2) / 4 % 2: a
+        // thread owns 64 of the row's 128 scores (P goes back over the first 32 of their columns) and half of the
+        // O columns.  The two threads of a row swap their partial row maxima (and, at the end, row
+        // sums) through shared memory under a 256-thread named barrier - that barrier also orders
+        // every thread's S loads before any P store (P overwrites the S columns).
+        const int t = (warp - 2) >> 3;                      // 0 = tile A, 1 = tile B
+        const int hf = ((warp - 2) >> 2) & 1;               // column half
         const int q = warp & 3;                             // TMEM lane quarter this warp may touch
         const int r = q * 32 + lane;                        // query row inside the tile
+        const bool tracer = hf == 0 && q == 2 && lane == 0;
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
-        const uint32_t s_addr = tmem_base + lane_addr + t * 128;
-        const uint32_t o_addr = tmem_base + lane_addr + 256 + t * 128;
+        const uint32_t s_addr = tmem_base + lane_addr + t * 128 + hf * 64;       // my 64 scores
+        const uint32_t o_addr = tmem_base + lane_addr + 256 + t * 128 + hf * (DH / 2);
+        float* xch = reinterpret_cast<float*>(sm + L::kXch) + t * 256;           // [half][row]
         const float sl2 = p.scale * kLog2e;
         uint32_t ns = 0, qn = 0;                            // S tiles and items this query tile has seen
         uint32_t u_base = 0;                                // uses of the output staging tile before this item
@@ -369,38 +385,39 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            if ((warp & 3) == 2 && lane == 0) PW_TRACE(2 + t, 1);
+            if (tracer) PW_TRACE(2 + t, 1);
             const bool diag = j == n_t - 1;
-            // all 128 scores of the row in registers (four loads in flight, one wait)
-            uint32_t v[128];
+            const int lim = diag ? r - hf * 64 : 64;        // columns i > lim of my 64 are masked (diagonal tile)
+            // pass 1: row maximum, 32 scores at a time (keeps the register count under the 576-thread limit)
+            float mxs[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, v + c * 32);
-            tc_wait_ld();
-            if ((warp & 3) == 2 && lane == 0) PW_TRACE(2 + t, 2);
-            // row maximum: eight independent chains of three-input max (64 instructions for 128 scores)
-            float mxs[8];
+            for (int c = 0; c < 2; ++c) {
+                uint32_t v[32];
+                tmem_ld32(s_addr + c * 32, v);
+                tc_wait_ld();
+                if (diag) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) mxs[i] = -INFINITY;
-            if (diag) {
+                    for (int i = 0; i < 32; ++i) v[i] = c * 32 + i > lim ? 0xff800000u : v[i];
+                }
 #pragma unroll
-                for (int i = 0; i < 128; ++i)
-                    if (i <= r) mxs[i & 7] = fmaxf(mxs[i & 7], __uint_as_float(v[i]));
-            } else {
-#pragma unroll
-                for (int i = 0; i < 128; i += 2)
-                    mxs[(i >> 1) & 7] = fmax3(mxs[(i >> 1) & 7], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+                for (int i = 0; i < 32; i += 2)
+                    mxs[(i >> 1) & 3] = fmax3(mxs[(i >> 1) & 3], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
             }
-            const float mx = fmaxf(fmax3(mxs[0], mxs[1], mxs[2]), fmax3(fmaxf(mxs[3], mxs[4]), fmaxf(mxs[5], mxs[6]), mxs[7]));
+            if (tracer) PW_TRACE(2 + t, 2);
+            const float mine = fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3]));
+            xch[hf * 128 + r] = mine;
+            named_bar_sync(1 + t, 256);
+            const float mx = fmaxf(mine, xch[(hf ^ 1) * 128 + r]);
             const float m_new = fmaxf(m_used, mx);
             const bool grow = (m_new - m_used) * sl2 > 8.0f;        // also true on the first tile (m_used = -inf)
             if (j == 0) {
                 m_used = m_new;
-            } else if (__any_sync(0xffffffffu, grow)) {
+            } else if (__any_sync(0xffffffffu, grow)) {     // both threads of a row see the same values
                 const float alpha = grow ? ex2_approx((m_used - m_new) * sl2) : 1.0f;
                 if (grow) m_used = m_new;
                 l *= alpha;
 #pragma unroll 1
-                for (int c = 0; c < DH / 32; ++c) {
+                for (int c = 0; c < DH / 64; ++c) {
                     uint32_t w[32];
                     tmem_ld32(o_addr + c * 32, w);
                     tc_wait_ld();
@@ -409,42 +426,41 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                     tmem_st32(o_addr + c * 32, w);
                 }
             }
-            // p = exp2((s - m) * scale * log2e), packed bf16 written over the S columns
-            if ((warp & 3) == 2 && lane == 0) PW_TRACE(2 + t, 3);
+            if (tracer) PW_TRACE(2 + t, 3);
+            // pass 2: p = exp2((s - m) * scale * log2e), packed bf16 written over my own S columns
+            // (scores 0..31 -> columns 0..15, scores 32..63 -> columns 16..31: always behind the loads)
             const float mb = m_used * sl2;
-            if (diag) {
-                float ls = 0.f;
+            const uint64_t sl2x2 = pack_f32x2(sl2, sl2), mbx2 = pack_f32x2(-mb, -mb);
+            uint64_t lsum[2] = {0ull, 0ull};
 #pragma unroll
-                for (int i = 0; i < 128; i += 2) {
-                    float p0 = i > r ? 0.f : ex2_approx(fmaf(__uint_as_float(v[i]), sl2, -mb));
-                    float p1 = i + 1 > r ? 0.f : ex2_approx(fmaf(__uint_as_float(v[i + 1]), sl2, -mb));
-                    ls += p0 + p1;
-                    v[i >> 1] = pack_bf16(p0, p1);
+            for (int c = 0; c < 2; ++c) {
+                uint32_t v[32];
+                tmem_ld32(s_addr + c * 32, v);
+                tc_wait_ld();
+                if (diag) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = c * 32 + i > lim ? 0xff800000u : v[i];
                 }
-                l += ls;
-            } else {
-                // two scores per FMA / add instruction; the exponentials stay on the MUFU
-                const uint64_t sl2x2 = pack_f32x2(sl2, sl2), mbx2 = pack_f32x2(-mb, -mb);
-                uint64_t lsum[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
-                for (int i = 0; i < 128; i += 2) {
+                for (int i = 0; i < 32; i += 2) {
                     float a0, a1;
                     unpack_f32x2(ffma2(pack_f32x2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), sl2x2, mbx2), a0, a1);
                     const float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
-                    lsum[(i >> 1) & 3] = fadd2(lsum[(i >> 1) & 3], pack_f32x2(p0, p1));
+                    lsum[(i >> 1) & 1] = fadd2(lsum[(i >> 1) & 1], pack_f32x2(p0, p1));
                     v[i >> 1] = pack_bf16(p0, p1);
                 }
+                tmem_st16(s_addr + c * 16, v);
+            }
+            {
                 float s0, s1;
-                unpack_f32x2(fadd2(fadd2(lsum[0], lsum[1]), fadd2(lsum[2], lsum[3])), s0, s1);
+                unpack_f32x2(fadd2(lsum[0], lsum[1]), s0, s1);
                 l += s0 + s1;
             }
-            if ((warp & 3) == 2 && lane == 0) PW_TRACE(2 + t, 4);
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_st16(s_addr + c * 16, v + c * 16);
+            if (tracer) PW_TRACE(2 + t, 4);
             tc_wait_st();
             tc_fence_before();
             mbar_arrive(bar(14 + t));
-            if ((warp & 3) == 2 && lane == 0) PW_TRACE(2 + t, 5);
+            if (tracer) PW_TRACE(2 + t, 5);
         }
         if (ok) {
             ok = mbar_wait(bar(16 + t), qn & 1, abort_flag, p.status, 421);
@@ -453,19 +469,23 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
         if (!ok) break;
         {
             tc_fence_after();
-            if ((warp & 3) == 2 && lane == 0) PW_TRACE(2 + t, 6);
-            const float inv_l = 1.0f / l;
+            if (tracer) PW_TRACE(2 + t, 6);
+            // row sum = the two halves' sums (the partner's last read of this slot was before its last p_full arrival)
+            xch[hf * 128 + r] = l;
+            named_bar_sync(1 + t, 256);
+            const float l_row = l + xch[(hf ^ 1) * 128 + r];
+            const float inv_l = 1.0f / l_row;
             uint8_t* stage = sm + L::kO;
             ok = mbar_wait(bar(20), (u & 1) ^ 1, abort_flag, p.status, 422);    // the previous user's store has read it
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            if ((warp & 3) == 2 && lane == 0) PW_TRACE(2 + t, 7);
+            if (tracer) PW_TRACE(2 + t, 7);
 #pragma unroll 1
-            for (int c = 0; c < DH / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld32(o_addr + c * 32, v);
+            for (int c = 0; c < DH / 64; ++c) {
+                uint32_t w[32];
+                tmem_ld32(o_addr + c * 32, w);
                 tc_wait_ld();
-                if (c == DH / 32 - 1) {                     // O_t has left TMEM: the next item may overwrite it
+                if (c == DH / 64 - 1) {                     // this thread's part of O_t has left TMEM
                     tc_fence_before();
                     mbar_arrive(bar(18 + t));
                 }
@@ -473,15 +493,15 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                 for (int g = 0; g < 4; ++g) {
                     float f[8];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[8 * g + i]) * inv_l;
-                    const int col = c * 32 + g * 8, blk = col >> 6, chunk = (col & 63) >> 3;
+                    for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(w[8 * g + i]) * inv_l;
+                    const int col = hf * (DH / 2) + c * 32 + g * 8, blk = col >> 6, chunk = (col & 63) >> 3;
                     *reinterpret_cast<uint4*>(stage + blk * 16384 + r * 128 + ((chunk ^ (r & 7)) << 4)) = pack8(f);
                 }
             }
-            p.lse[(static_cast<size_t>(it.b) * p.H + it.h) * p.S + q0 + r] = m_used * p.scale + logf(l);
+            if (hf == 0) p.lse[(static_cast<size_t>(it.b) * p.H + it.h) * p.S + q0 + r] = m_used * p.scale + logf(l_row);
             fence_proxy_async();
-            named_bar_sync(1 + t, 128);
-            if ((warp & 3) == 2 && lane == 0) {
+            named_bar_sync(1 + t, 256);
+            if (tracer) {
                 for (int kb = 0; kb < L::kBlocks; ++kb)
                     tma_store_2d(&tmO, sbase + L::kO + kb * 16384, it.h * DH + kb * 64, it.b * p.S + q0);
                 bulk_commit();
@@ -492,7 +512,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
             ++qn;
         }
         }
-        if ((warp & 3) == 2 && lane == 0) bulk_wait0();
+        if (tracer) bulk_wait0();
     }
 
     __syncwarp();
