@@ -264,3 +264,88 @@ class Oracle:
             ys.append(acts[-1])
             dxs.append(g)
         return ys, dxs, grads
+
+    # -- first and last layer of the language model (embedding lookup, tied softmax head) --
+    def embed_fwd(self, ids, E):
+        ids = np.ascontiguousarray(ids, dtype=np.int32)
+        E = self._a(E)
+        T, d = ids.size, E.shape[1]
+        assert ids.min() >= 0 and ids.max() < E.shape[0]
+        x0 = np.empty((T, d), self.dtype)
+        self._fn("pwo_embed_fwd")(self._p(ids), self._p(E), ctypes.c_long(T), ctypes.c_long(d), self._p(x0))
+        return x0
+
+    def embed_bwd(self, ids, dx0, dE):
+        """dE[ids[t]] += dx0[t] (in place; dE is an array of the oracle's precision)."""
+        ids = np.ascontiguousarray(ids, dtype=np.int32)
+        dx0 = self._a(dx0)
+        assert dE.dtype == self.dtype and dE.flags.c_contiguous
+        T, d = dx0.shape
+        self._fn("pwo_embed_bwd")(self._p(ids), self._p(dx0), ctypes.c_long(T), ctypes.c_long(d), self._p(dE))
+        return dE
+
+    def head_fwd(self, hf, E, labels, want_logits=False):
+        """Returns (loss, lse[T]) or (loss, lse, logits[T,V])."""
+        hf, E = self._a(hf), self._a(E)
+        labels = np.ascontiguousarray(labels, dtype=np.int32)
+        T, d = hf.shape
+        V = E.shape[0]
+        assert E.shape == (V, d) and labels.size == T and labels.min() >= 0 and labels.max() < V
+        lse = np.empty(T, self.dtype)
+        loss = np.zeros(1, self.dtype)
+        logits = np.empty((T, V), self.dtype) if want_logits else None
+        self._fn("pwo_head_fwd")(self._p(hf), self._p(E), self._p(labels), ctypes.c_long(T), ctypes.c_long(d),
+                                 ctypes.c_long(V), self._p(logits) if want_logits else None, self._p(lse), self._p(loss))
+        return (float(loss[0]), lse, logits) if want_logits else (float(loss[0]), lse)
+
+    def head_bwd(self, hf, E, labels, lse, dE, want_dlogits=False):
+        """Returns dhf (and dlogits); adds the head's part of the tied gradient into dE."""
+        hf, E, lse = self._a(hf), self._a(E), self._a(lse)
+        labels = np.ascontiguousarray(labels, dtype=np.int32)
+        T, d = hf.shape
+        V = E.shape[0]
+        assert dE.shape == (V, d) and dE.dtype == self.dtype and dE.flags.c_contiguous
+        dhf = np.empty((T, d), self.dtype)
+        dz = np.empty((T, V), self.dtype) if want_dlogits else None
+        self._fn("pwo_head_bwd")(self._p(hf), self._p(E), self._p(labels), self._p(lse), ctypes.c_long(T),
+                                 ctypes.c_long(d), ctypes.c_long(V), self._p(dhf), self._p(dE),
+                                 self._p(dz) if want_dlogits else None)
+        return (dhf, dz) if want_dlogits else dhf
+
+    def lm_step(self, D: Dims, params_per_layer, E, lnf_gamma, lnf_beta, ids, labels, handoff=None):
+        """One training step of the small decoder LM: embedding -> L layers -> final LayerNorm ->
+        tied softmax head -> mean cross-entropy, and its backward.
+
+        Returns a dict: loss, grads (per layer, PARAM_NAMES order), dE (embedding + head parts),
+        dlnf_gamma, dlnf_beta, and the intermediates x0, hL (last layer output), hf, lse.
+        ``handoff`` as in chain().
+        """
+        L = len(params_per_layer)
+        E = self._a(E)
+        acts, saves = [self.embed_fwd(ids, E)], []
+        for l in range(L):
+            y, sv = self.layer_fwd(D, params_per_layer[l], acts[-1])
+            if handoff is not None:
+                y = self._a(handoff(y))
+            acts.append(y)
+            saves.append(sv)
+        hf, mu, r = self.ln_fwd(acts[-1], lnf_gamma, lnf_beta, D.eps)
+        if handoff is not None:
+            hf = self._a(handoff(hf))
+        loss, lse = self.head_fwd(hf, E, labels)
+        dE = np.zeros_like(E)
+        dhf = self.head_bwd(hf, E, labels, lse, dE)
+        if handoff is not None:
+            dhf = self._a(handoff(dhf))
+        g, dg, db = self.ln_bwd(dhf, acts[-1], mu, r, lnf_gamma)
+        if handoff is not None:
+            g = self._a(handoff(g))
+        grads = [None] * L
+        for l in reversed(range(L)):
+            g, grads[l] = self.layer_bwd(D, params_per_layer[l], acts[l], saves[l], g)
+            if handoff is not None:
+                g = self._a(handoff(g))
+        self.embed_bwd(ids, g, dE)
+        return {"loss": loss, "grads": grads, "dE": dE, "dlnf_gamma": dg, "dlnf_beta": db,
+                "x0": acts[0], "hL": acts[-1], "hf": hf, "lse": lse, "dx0": g}
+

@@ -392,3 +392,87 @@ void FN(pwo_layer_bwd)(long B, long S, long d, long H, long dh, long F, int act,
     free(da); free(du); free(dh2); free(dx1); free(dob); free(dqkv); free(dh1);
     free(gw); free(gb); free(gb2);
 }
+
+/* ---- First and last layer of the language model (Section 5.3: "an embedding layer first and a
+ * softmax layer last").  The paper gives no formula; these are the textbook ones, with the
+ * output projection tied to the embedding table (reading listed in the design notes). ---- */
+
+/* Embedding lookup: x0[t][:] = E[ids[t]][:]. */
+void FN(pwo_embed_fwd)(const int* ids, const REAL* E, long T, long d, REAL* x0)
+{
+    for (long t = 0; t < T; ++t)
+        for (long c = 0; c < d; ++c) x0[t * d + c] = E[(long)ids[t] * d + c];
+}
+
+/* Backward of the lookup: dE[ids[t]][:] += dx0[t][:], tokens visited in order. */
+void FN(pwo_embed_bwd)(const int* ids, const REAL* dx0, long T, long d, REAL* dE)
+{
+    for (long t = 0; t < T; ++t)
+        for (long c = 0; c < d; ++c) dE[(long)ids[t] * d + c] += dx0[t * d + c];
+}
+
+/* Tied softmax head with cross-entropy against integer labels:
+ *   z[t][v] = sum_c hf[t][c] E[v][c]
+ *   lse[t]  = log sum_v exp(z[t][v])          (computed as max + log sum exp(z - max))
+ *   loss    = (1/T) sum_t ( lse[t] - z[t][label[t]] )
+ * logits (may be NULL) receives z. */
+void FN(pwo_head_fwd)(const REAL* hf, const REAL* E, const int* labels, long T, long d, long V,
+                      REAL* logits, REAL* lse, REAL* loss)
+{
+    double total = 0.0;
+#pragma omp parallel for schedule(static) reduction(+ : total)
+    for (long t = 0; t < T; ++t) {
+        REAL* z = (REAL*)malloc(sizeof(REAL) * (size_t)V);
+        REAL mx = -INFINITY;
+        for (long v = 0; v < V; ++v) {
+            REAL acc = 0;
+            for (long c = 0; c < d; ++c) acc += hf[t * d + c] * E[v * d + c];
+            z[v] = acc;
+            if (acc > mx) mx = acc;
+        }
+        double sum = 0.0;
+        for (long v = 0; v < V; ++v) sum += exp((double)(z[v] - mx));
+        const double l = (double)mx + log(sum);
+        lse[t] = (REAL)l;
+        total += l - (double)z[labels[t]];
+        if (logits) for (long v = 0; v < V; ++v) logits[t * V + v] = z[v];
+        free(z);
+    }
+    *loss = (REAL)(total / (double)T);
+}
+
+/* Backward of the head for d loss = 1:
+ *   dz[t][v]  = ( exp(z[t][v] - lse[t]) - [v == label[t]] ) / T
+ *   dhf[t][c] = sum_v dz[t][v] E[v][c]
+ *   dE[v][c] += sum_t dz[t][v] hf[t][c]
+ * dlogits (may be NULL) receives dz.  z is recomputed from hf and E by the definition. */
+void FN(pwo_head_bwd)(const REAL* hf, const REAL* E, const int* labels, const REAL* lse, long T, long d, long V,
+                      REAL* dhf, REAL* dE, REAL* dlogits)
+{
+    REAL* dz = (REAL*)malloc(sizeof(REAL) * (size_t)T * (size_t)V);
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < T; ++t) {
+        for (long v = 0; v < V; ++v) {
+            REAL acc = 0;
+            for (long c = 0; c < d; ++c) acc += hf[t * d + c] * E[v * d + c];
+            REAL g = (REAL)exp((double)(acc - lse[t]));
+            if (v == (long)labels[t]) g -= (REAL)1;
+            dz[t * V + v] = g / (REAL)T;
+        }
+        for (long c = 0; c < d; ++c) {
+            REAL acc = 0;
+            for (long v = 0; v < V; ++v) acc += dz[t * V + v] * E[v * d + c];
+            dhf[t * d + c] = acc;
+        }
+    }
+#pragma omp parallel for schedule(static)
+    for (long v = 0; v < V; ++v)
+        for (long c = 0; c < d; ++c) {
+            REAL acc = 0;
+            for (long t = 0; t < T; ++t) acc += dz[t * V + v] * hf[t * d + c];
+            dE[v * d + c] += acc;
+        }
+    if (dlogits) memcpy(dlogits, dz, sizeof(REAL) * (size_t)T * (size_t)V);
+    free(dz);
+}
+

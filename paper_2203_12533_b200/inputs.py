@@ -22,6 +22,10 @@ draws, in this order: w_qkv, b_qkv, w_o, b_o, w_fc1, b_fc1, w_fc2, b_fc2
 ``random_ln=True`` (then gamma ~ 1 + N(0, 0.1), beta ~ N(0, 0.1), drawn after
 the weights).  Micro-batch m uses seed ``s*7919 + 100003 + m`` and draws
 x ~ N(0,1) [B,S,d] then dy ~ N(0,1) [B,S,d].
+The language-model workload (5) adds, from seed ``s*7919 + 200003``: the embedding table
+E ~ N(0, 0.02) [V,d] (also the output projection: tied), token ids and labels, both independent
+uniform integers in [0, V) (int32 [B,S]; the labels are not shifted ids), and the final
+LayerNorm's gamma = 1, beta = 0 (``random_ln`` as above).
 """
 from __future__ import annotations
 
@@ -114,3 +118,21 @@ def microbatch(w: Workload, seed: int = 0, m: int = 0):
     x = _bf16(torch.randn(shp, generator=g, dtype=torch.float32))
     dy = _bf16(torch.randn(shp, generator=g, dtype=torch.float32))
     return x, dy
+
+
+def lm_inputs(w: Workload, seed: int = 0, random_ln: bool = False):
+    """(E [V,d] bf16, lnf_gamma [d] bf16, lnf_beta [d] bf16, ids [B,S] int32, labels [B,S] int32), CPU tensors."""
+    assert w.vocab > 0
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed * 7919 + 200003)
+    E = _bf16(torch.randn((w.vocab, w.d_model), generator=g, dtype=torch.float32) * 0.02)
+    ids = torch.randint(0, w.vocab, (w.batch, w.seq_len), generator=g, dtype=torch.int32)
+    labels = torch.randint(0, w.vocab, (w.batch, w.seq_len), generator=g, dtype=torch.int32)
+    if random_ln:
+        gamma = _bf16(1.0 + 0.1 * torch.randn((w.d_model,), generator=g, dtype=torch.float32))
+        beta = _bf16(0.1 * torch.randn((w.d_model,), generator=g, dtype=torch.float32))
+    else:
+        gamma = torch.ones((w.d_model,), dtype=torch.bfloat16)
+        beta = torch.zeros((w.d_model,), dtype=torch.bfloat16)
+    return E, gamma, beta, ids, labels
+
