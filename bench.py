@@ -374,13 +374,199 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def lm_flops_per_step(w):
+    """(model, executed) FLOPs of one small-LM step: L layers + tied head (logits, dhf, dE: 6 T d V)."""
+    head = 6.0 * w.tokens * w.d_model * w.vocab
+    per_call = w.model_flops_per_layer_call()
+    extra = (w.fwd_flops_per_layer_call() - 2.0 * w.tokens * w.d_model * w.d_ff) if w.recompute else 0.0
+    return per_call * w.n_layers + head, (per_call + extra) * w.n_layers + head
+
+
+def oracle_lm_sample(w, layers):
+    """A bounded sample of the LM workload: its first sequence through `layers` layers and the full-vocabulary head."""
+    from oracle import Dims
+    from paper_2203_12533_b200 import inputs
+    ws = w.with_(batch=1, n_layers=layers)
+    D = Dims(ws.batch, ws.seq_len, ws.d_model, ws.n_heads, ws.head_dim, ws.d_ff)
+    pls = [[p.float().numpy() for p in inputs.layer_params(ws, 0, l)] for l in range(layers)]
+    E, g, b, ids, labels = inputs.lm_inputs(ws, 0)
+    return ws, D, pls, E.float().numpy(), g.float().numpy(), b.float().numpy(), ids.numpy().ravel(), labels.numpy().ravel()
+
+
+def run_ours_lm(args, w):
+    """Workload 5: the whole small language-model step (pw_lm_step) instead of a bare layer chain."""
+    import torch
+    import torch.distributed as dist
+    from paper_2203_12533_b200 import binding as pw
+    from paper_2203_12533_b200 import inputs
+
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the product path)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    pw.lib()
+    peaks = load_peaks()
+    dev = torch.device("cuda", local)
+    L, T, d, V = w.n_layers, w.tokens, w.d_model, w.vocab
+    stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
+    params = [[p.to(dev) for p in inputs.layer_params(w, args.seed, l)] for l in range(L)]
+    grads = [[torch.zeros(p.shape, dtype=torch.float32, device=dev) for p in ps] for ps in params]
+    E, g, b, ids, labels = inputs.lm_inputs(w, args.seed)
+    host_ids, host_labels = ids.pin_memory(), labels.pin_memory()
+    lm_params = (E.to(dev), g.to(dev), b.to(dev))
+    lm_grads = (torch.zeros(E.shape, dtype=torch.float32, device=dev), torch.zeros(d, device=dev), torch.zeros(d, device=dev))
+    dev_ids, dev_labels = [host_ids.to(dev), host_ids.to(dev)], [host_labels.to(dev), host_labels.to(dev)]
+    loss = torch.zeros(1, device=dev)
+    host_loss = torch.zeros(1).pin_memory()
+    workspace = torch.empty(stage.lm_workspace_bytes(V, w.recompute), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+    state = {"i": 0}
+
+    def step():
+        stage.lm_step(params, grads, lm_params, lm_grads, dev_ids[0], dev_labels[0], loss, V, workspace, w.recompute, stream=stream)
+
+    def step_e2e():
+        k = state["i"] & 1                                   # the copies are tiny: same stream, alternating buffers
+        dev_ids[k].copy_(host_ids, non_blocking=True)
+        dev_labels[k].copy_(host_labels, non_blocking=True)
+        stage.lm_step(params, grads, lm_params, lm_grads, dev_ids[k], dev_labels[k], loss, V, workspace, w.recompute, stream=stream)
+        host_loss.copy_(loss, non_blocking=True)
+        state["i"] += 1
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def timed(fn, steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for _ in range(steps):
+                fn()
+            e1.record(stream)
+        torch.cuda.synchronize(dev)
+        ms = e0.elapsed_time(e1)
+        barrier()
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            step()
+    torch.cuda.synchronize(dev)
+    if stage.status() != (0, 0):
+        raise SystemExit(f"device status {stage.status()} after warm-up")
+    n0 = stage.launch_count()
+    with ClockSampler(local) as clocks:
+        ms_step = timed(step, args.steps) / args.steps
+    launches = stage.launch_count() - n0
+    stage.profile_begin()
+    with torch.cuda.stream(stream):
+        for _ in range(args.steps):
+            step()
+    prof = stage.profile_end()
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    ms_e2e = timed(step_e2e, e2e_steps) / e2e_steps
+    if stage.status() != (0, 0):
+        raise SystemExit(f"device status {stage.status()}")
+    model_flops, hw_flops = lm_flops_per_step(w)
+    value = world * T / (ms_step * 1e-3)
+    line = {
+        "metric": "small-LM training step tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "d_model": d, "heads": f"{w.n_heads}x{w.head_dim}", "d_ff": w.d_ff,
+                   "seq_len": w.seq_len, "batch": w.batch, "layers": L, "vocab": V, "recompute": bool(w.recompute),
+                   "dispatch": "async", "parallelism": f"replicas x{world}",
+                   "l2": "working set per step (logits alone are 1 GB) is far above the 126 MB L2"},
+        "loss": float(loss.item()),
+        "tflops_model": world * model_flops / (ms_step * 1e-3) / 1e12,
+        "tflops_hw": world * hw_flops / (ms_step * 1e-3) / 1e12,
+        "frac_bf16_peak_burst": hw_flops / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
+        "frac_bf16_peak_sustained": hw_flops / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+        "peaks": peaks, "clocks": clocks.summary(),
+        "e2e": {"value": world * T / (ms_e2e * 1e-3), "unit": "tokens/s", "ms_per_step": ms_e2e, "steps": e2e_steps,
+                "how": "pinned host ids, labels -> device and the loss -> pinned host every step",
+                "h2d_bytes_per_step": 2 * T * 4, "d2h_bytes_per_step": 4},
+        "gpu_launches": int(launches),
+    }
+    kernels, tot_ms = {}, sum(v["ms"] for v in prof.values())
+    g_ms = g_flops = g_n = 0.0
+    for name, v in prof.items():
+        if v["launches"] == 0:
+            continue
+        k = {"launches_per_step": v["launches"] / args.steps, "ms_per_step": v["ms"] / args.steps, "share": v["ms"] / tot_ms}
+        if v["flops"] > 0:
+            k["tflops"] = v["flops"] / (v["ms"] * 1e-3) / 1e12
+            k["frac_of_measured_bf16_burst"] = k["tflops"] / peaks["bf16_tflops"]
+        if v["bytes"] > 0:
+            k["gbs"] = v["bytes"] / (v["ms"] * 1e-3) / 1e9
+            k["frac_of_measured_hbm"] = k["gbs"] / peaks["hbm_gbs"]
+        kernels[name] = k
+        if name.startswith("gemm"):
+            g_ms += v["ms"]; g_flops += v["flops"]; g_n += v["launches"]
+    line["kernels"] = kernels
+    achieved = g_flops / (g_ms * 1e-3) / 1e12
+    line["roofline"] = {"kernel": "gemm_pair_kernel (tcgen05 bf16 GEMM: layers and tied head)", "bound": "tensor",
+                        "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                        "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst cuBLAS bf16)",
+                        "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
+                        "flops_per_launch": g_flops / g_n, "ms_per_launch": g_ms / g_n,
+                        "launches_per_step": g_n / args.steps, "share_of_step": g_ms / tot_ms, "traffic": None}
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle as oracle_mod
+        orc = oracle_mod.Oracle("f32")
+        ws, D, pls, E_, g_, b_, ids_, labels_ = oracle_lm_sample(w, 1)
+        t0 = time.perf_counter()
+        orc.lm_step(D, pls, E_, g_, b_, ids_, labels_)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": ws.tokens / dt, "unit": "tokens/s", "cores": oracle_mod.host_threads(), "kind": "oracle",
+                                "seconds": dt, "sample": f"1 of {w.batch} sequences (S={w.seq_len}) through 1 of {L} layers and the full-vocabulary head, fwd+bwd, fp32 plain-loop C oracle, run once"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_reference_lm(args, w):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle as oracle_mod
+    orc = oracle_mod.Oracle("f32")
+    ws, D, pls, E, g, b, ids, labels = oracle_lm_sample(w, 1)
+    for _ in range(min(args.warmup, 1)):
+        orc.lm_step(D, pls, E, g, b, ids, labels)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        orc.lm_step(D, pls, E, g, b, ids, labels)
+    dt = time.perf_counter() - t0
+    value = ws.tokens * args.steps / dt
+    sample = f"1 of {w.batch} sequences (S={w.seq_len}) through 1 of {w.n_layers} layers and the full-vocabulary head per step, fp32 plain-loop C oracle"
+    print(json.dumps({
+        "impl": "reference", "metric": "small-LM training step tokens/s", "value": value, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": oracle_mod.host_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4])
+    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--dispatch", default="async", choices=["opbyop", "async", "graph"])
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=30)
@@ -390,9 +576,9 @@ def main():
     from paper_2203_12533_b200 import inputs
     w = inputs.WORKLOADS[args.workload]
     if args.impl == "reference":
-        run_reference(args, w)
+        (run_reference_lm if w.vocab else run_reference)(args, w)
     else:
-        run_ours(args, w)
+        (run_ours_lm if w.vocab else run_ours)(args, w)
 
 
 if __name__ == "__main__":

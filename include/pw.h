@@ -177,7 +177,9 @@ enum {
     PW_K_LN_FWD = 5,
     PW_K_LN_BWD = 6,    /* main kernel + partial reduction    */
     PW_K_COLSUM = 7,    /* main kernel + partial reduction    */
-    PW_K_COUNT = 8
+    PW_K_XENT = 8,      /* softmax / cross-entropy + loss mean (pw_lm_step)          */
+    PW_K_EMBED = 9,     /* embedding lookup and its scatter-add backward (pw_lm_step) */
+    PW_K_COUNT = 10
 };
 typedef struct pw_profile {
     uint64_t launches[PW_K_COUNT]; /* kernel launches per class since profile_begin      */
@@ -231,6 +233,34 @@ pw_status_t pw_stage_status(pw_stage_t* stage, int* device_status, int* site);
 pw_status_t pw_stage_profile_begin(pw_stage_t* stage);
 pw_status_t pw_stage_profile_end(pw_stage_t* stage, pw_profile_t* out);
 pw_status_t pw_stage_launch_count(const pw_stage_t* stage, uint64_t* count);
+
+/* ---- the whole small language model: embedding layer first, softmax layer last (Section 5.3) ----
+ * The paper names the two end layers but prints no formula; the reading built here: token
+ * embedding E [V,d] (no positional term), L decoder layers, a final LayerNorm, logits = hf E^T with
+ * the SAME table (tied), loss = mean over the T tokens of -log softmax(logits)[label].
+ *   ids, labels : int32 [B,S] device, values in [0, vocab) (anything else is reported through the
+ *                 status word as PW_ERR_INVALID_ARG and treated as 0)
+ *   loss        : one fp32 on the device
+ *   gradients   : overwritten (one batch per call): per-layer grads as in pw_layer_bwd,
+ *                 lm_grads->embedding fp32 [V,d] = head part + scatter-add of the input gradient
+ *                 (tokens added in increasing order: bitwise reproducible), lnf_gamma / lnf_beta fp32 [d]
+ * vocab % 8 == 0.  The logits (bf16 [T,V]) live in the workspace and are turned into their own
+ * gradient in place.  Enqueue only. */
+typedef struct pw_lm_params {
+    const void* embedding; /* bf16 [V, d]; also the output projection */
+    const void* lnf_gamma; /* bf16 [d] final LayerNorm */
+    const void* lnf_beta;  /* bf16 [d] */
+} pw_lm_params_t;
+typedef struct pw_lm_grads {
+    void* embedding; /* fp32 [V, d] */
+    void* lnf_gamma; /* fp32 [d] */
+    void* lnf_beta;  /* fp32 [d] */
+} pw_lm_grads_t;
+pw_status_t pw_lm_workspace_bytes(const pw_stage_t* stage, int vocab, int recompute, size_t* bytes);
+pw_status_t pw_lm_step(pw_stage_t* stage, const pw_layer_params_t* params, const pw_layer_grads_t* grads,
+                       const pw_lm_params_t* lm, const pw_lm_grads_t* lm_grads, const int32_t* ids,
+                       const int32_t* labels, float* loss, int vocab, int recompute, void* workspace,
+                       size_t workspace_bytes, void* stream);
 
 /* ---- single steps of the layer (same kernels the layer calls; for unit tests and profiling) ---- */
 
@@ -292,6 +322,19 @@ enum { PW_EPI_NONE = 0, PW_EPI_BIAS = 1, PW_EPI_BIAS_RESID = 2, PW_EPI_BIAS_GELU
 pw_status_t pw_op_gemm(int layout, int epilogue, int act, int M, int N, int K, const void* A, int lda,
                        const void* B, int ldb, void* C, int ldc, const void* bias, const void* aux_in,
                        int ld_aux, void* aux_out, int accumulate, void* stream);
+
+/* Embedding lookup x0[t] = E[ids[t]] (bf16 rows of d elements, d % 8 == 0) and its backward
+ * dE[ids[t]] += dx0[t] (fp32, tokens added in increasing t).  scratch: device,
+ * pw_op_embedding_bwd_scratch_bytes(T, V) bytes. */
+pw_status_t pw_op_embedding_fwd(const int32_t* ids, const void* E, int T, int d, int V, void* x0, void* stream);
+size_t pw_op_embedding_bwd_scratch_bytes(int T, int V);
+pw_status_t pw_op_embedding_bwd(const int32_t* ids, const void* dx0, int T, int d, int V, void* dE, void* scratch,
+                                void* stream);
+/* Softmax / cross-entropy over logits bf16 [T, ld] (V columns used, V % 8 == 0): lse fp32 [T],
+ * loss_rows fp32 [T] = lse - logit[label]; the logits are replaced by
+ * grad_scale * (softmax - onehot(label)). */
+pw_status_t pw_op_softmax_xent(void* logits, int ld, const int32_t* labels, int T, int V, float grad_scale,
+                               void* lse, void* loss_rows, void* stream);
 
 /* Causal attention forward on packed qkv (bf16 [T,3d]); o bf16 [T,d]; lse fp32 [B,H,S].
  * The attention kernels are persistent and hand out their work through counters that live

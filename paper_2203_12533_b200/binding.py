@@ -38,6 +38,8 @@ EXPORTS = (
     "pw_op_layernorm_fwd", "pw_op_layernorm_bwd_scratch_bytes", "pw_op_layernorm_bwd",
     "pw_op_colsum_scratch_bytes", "pw_op_colsum", "pw_op_colsum_noalloc", "pw_op_gemm",
     "pw_op_attention_fwd", "pw_op_attention_bwd", "pw_op_status",
+    "pw_lm_workspace_bytes", "pw_lm_step",
+    "pw_op_embedding_fwd", "pw_op_embedding_bwd_scratch_bytes", "pw_op_embedding_bwd", "pw_op_softmax_xent",
 )
 
 
@@ -54,16 +56,21 @@ class LayerConfig(ctypes.Structure):
                 ("causal", ctypes.c_int32), ("flags", ctypes.c_uint32)]
 
 
-KERNEL_CLASSES = ("gemm_tn", "gemm_nn", "gemm_nt", "attn_fwd", "attn_bwd", "ln_fwd", "ln_bwd", "colsum")
+KERNEL_CLASSES = ("gemm_tn", "gemm_nn", "gemm_nt", "attn_fwd", "attn_bwd", "ln_fwd", "ln_bwd", "colsum", "xent", "embed")
 
 
 class Profile(ctypes.Structure):
-    _fields_ = [("launches", ctypes.c_uint64 * 8), ("ms", ctypes.c_double * 8), ("flops", ctypes.c_double * 8),
-                ("bytes", ctypes.c_double * 8)]
+    _fields_ = [("launches", ctypes.c_uint64 * 10), ("ms", ctypes.c_double * 10), ("flops", ctypes.c_double * 10),
+                ("bytes", ctypes.c_double * 10)]
 
     def as_dict(self):
         return {n: dict(launches=int(self.launches[i]), ms=float(self.ms[i]), flops=float(self.flops[i]),
                         bytes=float(self.bytes[i])) for i, n in enumerate(KERNEL_CLASSES)}
+
+
+class _Ptr3(ctypes.Structure):
+    """pw_lm_params_t / pw_lm_grads_t: embedding table, final LayerNorm gamma, beta."""
+    _fields_ = [("embedding", ctypes.c_void_p), ("lnf_gamma", ctypes.c_void_p), ("lnf_beta", ctypes.c_void_p)]
 
 
 class _Ptr12(ctypes.Structure):
@@ -121,6 +128,14 @@ def lib() -> ctypes.CDLL:
         L.pw_op_attention_fwd.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp]
         L.pw_op_attention_bwd.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, vp]
         L.pw_op_status.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci)]
+        L.pw_lm_workspace_bytes.argtypes = [vp, ci, ci, ctypes.POINTER(ctypes.c_size_t)]
+        L.pw_lm_step.argtypes = [vp, ctypes.POINTER(_Ptr12), ctypes.POINTER(_Ptr12), ctypes.POINTER(_Ptr3),
+                                 ctypes.POINTER(_Ptr3), vp, vp, vp, ci, ci, vp, ctypes.c_size_t, vp]
+        L.pw_op_embedding_fwd.argtypes = [vp, vp, ci, ci, ci, vp, vp]
+        L.pw_op_embedding_bwd_scratch_bytes.restype = ctypes.c_size_t
+        L.pw_op_embedding_bwd_scratch_bytes.argtypes = [ci, ci]
+        L.pw_op_embedding_bwd.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp]
+        L.pw_op_softmax_xent.argtypes = [vp, ci, vp, ci, ci, ctypes.c_float, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -263,6 +278,25 @@ class Stage:
         _check(lib().pw_stage_run_chain(self._h, P, G, arr(xs), arr(dys), arr(ys), arr(dxs), M, dispatch, schedule,
                                         int(recompute), _p(workspace), nbytes, _stream(stream)))
 
+    def lm_workspace_bytes(self, vocab, recompute=False) -> int:
+        n = ctypes.c_size_t()
+        _check(lib().pw_lm_workspace_bytes(self._h, vocab, int(recompute), ctypes.byref(n)))
+        return n.value
+
+    def lm_step(self, params, grads, lm_params, lm_grads, ids, labels, loss, vocab, workspace, recompute=False,
+                stream=None, workspace_bytes=None):
+        """One training step of the small LM (pw_lm_step).  lm_params = (E, lnf_gamma, lnf_beta) bf16,
+        lm_grads = (dE, dlnf_gamma, dlnf_beta) fp32, ids / labels int32 [B,S], loss fp32 [1]."""
+        L = self.n_layers
+        assert len(params) == L and len(grads) == L
+        P = (_Ptr12 * L)(*[_ptr12(p) for p in params])
+        G = (_Ptr12 * L)(*[_ptr12(g) for g in grads])
+        lp = _Ptr3(*[_p(t) for t in lm_params])
+        lg = _Ptr3(*[_p(t) for t in lm_grads])
+        nbytes = workspace.numel() * workspace.element_size() if workspace_bytes is None else workspace_bytes
+        _check(lib().pw_lm_step(self._h, P, G, ctypes.byref(lp), ctypes.byref(lg), _p(ids), _p(labels), _p(loss), vocab,
+                                int(recompute), _p(workspace), nbytes, _stream(stream)))
+
     def status(self):
         c, s = ctypes.c_int(), ctypes.c_int()
         _check(lib().pw_stage_status(self._h, ctypes.byref(c), ctypes.byref(s)))
@@ -298,6 +332,26 @@ def op_layernorm_bwd(dh, x, mu, rstd, gamma, resid, dx, dgamma, dbeta, db_resid,
     _check(lib().pw_op_layernorm_bwd(_p(dh), _p(x), _p(mu), _p(rstd), _p(gamma), _p(resid), T, d, _p(dx), _p(dgamma),
                                      _p(dbeta), _p(db_resid), _p(db_dx), int(accumulate), _p(partials),
                                      _stream(stream)))
+
+
+def op_embedding_fwd(ids, E, x0, stream=None):
+    V, d = E.shape
+    _check(lib().pw_op_embedding_fwd(_p(ids), _p(E), ids.numel(), d, V, _p(x0), _stream(stream)))
+
+
+def op_embedding_bwd_scratch_bytes(T, V) -> int:
+    return lib().pw_op_embedding_bwd_scratch_bytes(T, V)
+
+
+def op_embedding_bwd(ids, dx0, dE, scratch, stream=None):
+    V, d = dE.shape
+    _check(lib().pw_op_embedding_bwd(_p(ids), _p(dx0), ids.numel(), d, V, _p(dE), _p(scratch), _stream(stream)))
+
+
+def op_softmax_xent(logits, labels, grad_scale, lse, loss_rows, stream=None):
+    T, V = logits.shape
+    _check(lib().pw_op_softmax_xent(_p(logits), logits.stride(0), _p(labels), T, V, grad_scale, _p(lse), _p(loss_rows),
+                                    _stream(stream)))
 
 
 def op_colsum_scratch_bytes(T, N) -> int:

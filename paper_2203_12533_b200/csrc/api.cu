@@ -743,6 +743,119 @@ pw_status_t pw_stage_launch_count(const pw_stage_t* stage, uint64_t* count)
     return pw_layer_launch_count(stage->layer, count);
 }
 
+// ---------------------------------------------------------------------------------------- language model step
+namespace {
+struct LmLayout {
+    size_t act_bytes, off_x0, off_acts, off_ctx, off_hf, off_mu, off_r, off_logits, off_lse, off_rows, off_g0, off_g1,
+        off_emb, off_scratch, total;
+};
+pw_status_t lm_layout(const pw_stage_t* stage, int vocab, int recompute, LmLayout* lay)
+{
+    if (vocab <= 0 || (vocab % 8)) return fail(PW_ERR_UNSUPPORTED_SHAPE, "vocab must be a positive multiple of 8");
+    if (recompute != 0 && recompute != 1) return fail(PW_ERR_INVALID_ARG, "recompute must be 0 or 1");
+    const LayerPlan& p = stage->layer->plan;
+    const size_t L = stage->n_layers, T = p.T;
+    lay->act_bytes = align256(T * p.d * 2);
+    size_t s = 0;
+    lay->off_x0 = s; s += lay->act_bytes;
+    lay->off_acts = s; s += lay->act_bytes * L;                 // output of every layer (the last one feeds the final LayerNorm)
+    lay->off_ctx = s; s += recompute ? 0 : p.ctx_bytes * L;
+    lay->off_hf = s; s += lay->act_bytes;
+    lay->off_mu = s; s += align256(T * 4);
+    lay->off_r = s; s += align256(T * 4);
+    lay->off_logits = s; s += align256(T * static_cast<size_t>(vocab) * 2);
+    lay->off_lse = s; s += align256(T * 4);
+    lay->off_rows = s; s += align256(T * 4);
+    lay->off_g0 = s; s += lay->act_bytes;
+    lay->off_g1 = s; s += lay->act_bytes;
+    lay->off_emb = s; s += align256(embedding_bwd_scratch_bytes(static_cast<int>(T), vocab));
+    lay->off_scratch = s; s += p.scratch_bytes;
+    lay->total = s;
+    return PW_OK;
+}
+}  // namespace
+
+pw_status_t pw_lm_workspace_bytes(const pw_stage_t* stage, int vocab, int recompute, size_t* bytes)
+{
+    if (!stage || !bytes) return fail(PW_ERR_INVALID_ARG, "stage or bytes is NULL");
+    LmLayout lay;
+    pw_status_t s = lm_layout(stage, vocab, recompute, &lay);
+    if (s != PW_OK) return s;
+    *bytes = lay.total;
+    return PW_OK;
+}
+
+pw_status_t pw_lm_step(pw_stage_t* stage, const pw_layer_params_t* params, const pw_layer_grads_t* grads,
+                       const pw_lm_params_t* lm, const pw_lm_grads_t* lm_grads, const int32_t* ids, const int32_t* labels,
+                       float* loss, int vocab, int recompute, void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!stage || !params || !grads || !lm || !lm_grads || !ids || !labels || !loss)
+        return fail(PW_ERR_INVALID_ARG, "a required pointer is NULL");
+    LmLayout lay;
+    pw_status_t s = lm_layout(stage, vocab, recompute, &lay);
+    if (s != PW_OK) return s;
+    if (!aligned(workspace, 256)) return fail(PW_ERR_INVALID_ARG, "workspace is NULL or not 256-byte aligned");
+    if (workspace_bytes < lay.total) return fail(PW_ERR_WORKSPACE_TOO_SMALL, "workspace smaller than pw_lm_workspace_bytes reports");
+    pw_layer_t* Lh = stage->layer;
+    const LayerPlan& p = Lh->plan;
+    const int L = stage->n_layers, T = p.T, d = p.d, V = vocab;
+    for (int l = 0; l < L; ++l)
+        if (!params_ok(&params[l]) || !grads_ok(&grads[l])) return fail(PW_ERR_INVALID_ARG, "a parameter or gradient pointer is NULL or misaligned");
+    if (!aligned(lm->embedding, 16) || !aligned(lm->lnf_gamma, 16) || !aligned(lm->lnf_beta, 16) ||
+        !aligned(lm_grads->embedding, 16) || !aligned(lm_grads->lnf_gamma, 16) || !aligned(lm_grads->lnf_beta, 16) ||
+        !aligned(ids, 4) || !aligned(labels, 4) || !aligned(loss, 4))
+        return fail(PW_ERR_INVALID_ARG, "a language-model pointer is NULL or misaligned");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    void* ws = workspace;
+    void* x0 = at(ws, lay.off_x0);
+    auto actp = [&](int l) -> void* { return at(ws, lay.off_acts + static_cast<size_t>(l) * lay.act_bytes); };   // output of layer l
+    auto ctxp = [&](int l) -> void* { return recompute ? nullptr : at(ws, lay.off_ctx + static_cast<size_t>(l) * p.ctx_bytes); };
+    void* scratch = at(ws, lay.off_scratch);
+    void* hf = at(ws, lay.off_hf); void* mu = at(ws, lay.off_mu); void* r = at(ws, lay.off_r);
+    void* logits = at(ws, lay.off_logits); void* lse = at(ws, lay.off_lse); void* rows = at(ws, lay.off_rows);
+    const char* e;
+
+    // forward: lookup, L layers, final LayerNorm, tied projection, softmax / cross-entropy
+    {
+        LaunchScope sc(Lh, PW_K_EMBED, 1, 0.0, 4.0 * T * d, st);
+        if ((e = launch_embedding_fwd(Lh->rt, ids, lm->embedding, T, d, V, x0, Lh->status, st))) return fail(PW_ERR_CUDA, e);
+    }
+    for (int l = 0; l < L; ++l) {
+        void* c = ctxp(l);
+        PW_DO(enqueue_fwd(Lh, &params[l], l == 0 ? x0 : actp(l - 1), actp(l), c ? c : scratch, true, st));
+    }
+    const void* hL = L > 0 ? actp(L - 1) : x0;
+    PW_DO(do_ln_fwd(Lh, hL, lm->lnf_gamma, lm->lnf_beta, hf, mu, r, st));
+    PW_DO(do_gemm(Lh, gemm_args(kTN, kEpiNone, 0, T, V, d, hf, d, lm->embedding, d, logits, V, nullptr, nullptr, 0,
+                                      nullptr, 0), st));
+    {
+        LaunchScope sc(Lh, PW_K_XENT, 2, 0.0, 4.0 * T * V + 12.0 * T, st);
+        if ((e = launch_softmax_xent(Lh->rt, logits, V, labels, T, V, 1.0f / static_cast<float>(T), lse, rows, Lh->status, st)))
+            return fail(PW_ERR_CUDA, e);
+        if ((e = launch_sum_scale(rows, T, 1.0f / static_cast<float>(T), loss, st))) return fail(PW_ERR_CUDA, e);
+    }
+    // backward: dhf = dz E, dE = dz^T hf, final LayerNorm, L layers, scatter-add of the input gradient
+    void* g0 = at(ws, lay.off_g0); void* g1 = at(ws, lay.off_g1);
+    PW_DO(do_gemm(Lh, gemm_args(kNN, kEpiNone, 0, T, d, V, logits, V, lm->embedding, d, g0, d, nullptr, nullptr, 0,
+                                      nullptr, 0), st));
+    PW_DO(do_gemm(Lh, gemm_args(kNT, kEpiF32, 0, V, d, T, logits, V, hf, d, lm_grads->embedding, d, nullptr, nullptr, 0,
+                                      nullptr, 0), st));
+    PW_DO(do_ln_bwd(Lh, g0, hL, mu, r, lm->lnf_gamma, nullptr, g1, lm_grads->lnf_gamma, lm_grads->lnf_beta, nullptr,
+                          nullptr, 0, at(scratch, p.off_partials), st));
+    const void* g = g1;
+    for (int l = L - 1; l >= 0; --l) {
+        void* out = (g == g1) ? g0 : g1;
+        PW_DO(enqueue_bwd(Lh, &params[l], l == 0 ? x0 : actp(l - 1), g, out, &grads[l], 0, ctxp(l), scratch, st));
+        g = out;
+    }
+    {
+        LaunchScope sc(Lh, PW_K_EMBED, 2, 0.0, 2.0 * T * d + 4.0 * (T + V), st);
+        if ((e = launch_embedding_bwd(Lh->rt, ids, g, T, d, V, lm_grads->embedding, at(ws, lay.off_emb), Lh->status, st)))
+            return fail(PW_ERR_CUDA, e);
+    }
+    return PW_OK;
+}
+
 // ---------------------------------------------------------------------------------------- single steps
 
 #define PW_RT_OR_FAIL()                                                                       \
@@ -837,6 +950,37 @@ pw_status_t pw_op_attention_bwd(const void* qkv, const void* o, const void* dout
     if (!aligned(qkv, 16) || !aligned(o, 16) || !aligned(dout, 16) || !lse || !aligned(dqkv, 16) || !delta)
         return fail(PW_ERR_INVALID_ARG, "attention bwd: NULL or misaligned pointer");
     PW_OP(launch_attention_bwd(rt, qkv, o, dout, lse, B, S, H, dh, dqkv, delta, rt->op_status, static_cast<cudaStream_t>(stream)));
+    return PW_OK;
+}
+
+pw_status_t pw_op_embedding_fwd(const int32_t* ids, const void* E, int T, int d, int V, void* x0, void* stream)
+{
+    PW_RT_OR_FAIL();
+    if (!aligned(ids, 4) || !aligned(E, 16) || !aligned(x0, 16)) return fail(PW_ERR_INVALID_ARG, "embedding: NULL or misaligned pointer");
+    PW_OP(launch_embedding_fwd(rt, ids, E, T, d, V, x0, rt->op_status, static_cast<cudaStream_t>(stream)));
+    return PW_OK;
+}
+
+size_t pw_op_embedding_bwd_scratch_bytes(int T, int V) { return embedding_bwd_scratch_bytes(T, V); }
+
+pw_status_t pw_op_embedding_bwd(const int32_t* ids, const void* dx0, int T, int d, int V, void* dE, void* scratch,
+                                void* stream)
+{
+    PW_RT_OR_FAIL();
+    if (!aligned(ids, 4) || !aligned(dx0, 16) || !aligned(dE, 16) || !aligned(scratch, 4))
+        return fail(PW_ERR_INVALID_ARG, "embedding bwd: NULL or misaligned pointer");
+    PW_OP(launch_embedding_bwd(rt, ids, dx0, T, d, V, dE, scratch, rt->op_status, static_cast<cudaStream_t>(stream)));
+    return PW_OK;
+}
+
+pw_status_t pw_op_softmax_xent(void* logits, int ld, const int32_t* labels, int T, int V, float grad_scale, void* lse,
+                               void* loss_rows, void* stream)
+{
+    PW_RT_OR_FAIL();
+    if (!aligned(logits, 16) || !aligned(labels, 4) || !aligned(lse, 4) || !aligned(loss_rows, 4))
+        return fail(PW_ERR_INVALID_ARG, "softmax-xent: NULL or misaligned pointer");
+    PW_OP(launch_softmax_xent(rt, logits, ld, labels, T, V, grad_scale, lse, loss_rows, rt->op_status,
+                              static_cast<cudaStream_t>(stream)));
     return PW_OK;
 }
 

@@ -187,7 +187,7 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
             const uint32_t dst = ring0 + (stage * 3 * CHUNKS + j) * slot_stride;
             cp_async_16(dst, dh + off, live);
             cp_async_16(dst + CHUNKS * slot_stride, x + off, live);
-            cp_async_16(dst + 2 * CHUNKS * slot_stride, resid + off, live);
+            cp_async_16(dst + 2 * CHUNKS * slot_stride, resid ? resid + off : dh + off, live && resid != nullptr);   // no residual: zeros
         }
         cp_async_commit();
     };

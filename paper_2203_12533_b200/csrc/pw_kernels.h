@@ -75,6 +75,16 @@ const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, voi
 size_t colsum_noalloc_max_columns();
 const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* out, int accumulate, cudaStream_t stream);
 
+// First / last layer of the language model (lm_head.cu).
+const char* launch_embedding_fwd(Runtime* rt, const void* ids, const void* E, int T, int d, int V, void* x0,
+                                 DeviceStatus* status, cudaStream_t stream);
+size_t embedding_bwd_scratch_bytes(int T, int V);
+const char* launch_embedding_bwd(Runtime* rt, const void* ids, const void* dx0, int T, int d, int V, void* dE,
+                                 void* scratch, DeviceStatus* status, cudaStream_t stream);
+const char* launch_softmax_xent(Runtime* rt, void* logits, int ld, const void* labels, int T, int V, float grad_scale,
+                                void* lse, void* loss_rows, DeviceStatus* status, cudaStream_t stream);
+const char* launch_sum_scale(const void* in, int n, float scale, void* out, cudaStream_t stream);
+
 const char* launch_attention_fwd(Runtime* rt, const void* qkv, int B, int S, int H, int dh, void* o, void* lse,
                                  DeviceStatus* status, cudaStream_t stream);
 const char* launch_attention_bwd(Runtime* rt, const void* qkv, const void* o, const void* dout, const void* lse,
