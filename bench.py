@@ -105,6 +105,22 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The slowest rank's time: what a multi-rank number is computed from (no-op for one rank)."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank: float, world: int, ms: float) -> float:
+    """Replicas: every rank processes the same number of units; the job's rate uses the slowest rank's time."""
+    return world * units_per_rank / (ms * 1e-3)
+
+
 def hw_flops_per_step(w) -> float:
     """Executed FLOPs: model FLOPs plus, with recompute, one forward without the FC2 GEMM."""
     per_call = w.model_flops_per_layer_call()
@@ -258,11 +274,7 @@ def run_ours(args, w):
         torch.cuda.synchronize(dev)
         ms = e0.elapsed_time(e1)
         barrier()
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(ms, world, dev)
 
     with torch.cuda.stream(stream):
         for _ in range(args.warmup):
@@ -278,7 +290,7 @@ def run_ours(args, w):
     launches = stage.launch_count() - n0
     ms_step = ms_total / args.steps
     tokens_step = T * M
-    value = world * tokens_step / (ms_step * 1e-3)
+    value = whole_job_value(tokens_step, world, ms_step)
 
     # instrumented pass: per-kernel-class device time from CUDA events inside the library
     prof = None
@@ -300,7 +312,7 @@ def run_ours(args, w):
     torch.cuda.synchronize(dev)
     e2e_state["i"] = 0
     ms_e2e = timed(step_e2e, e2e_steps) / e2e_steps
-    e2e_value = world * tokens_step / (ms_e2e * 1e-3)
+    e2e_value = whole_job_value(tokens_step, world, ms_e2e)
     code, site = stage.status()
     if code != 0:
         raise SystemExit(f"device status {code} at site {site}")
@@ -452,11 +464,7 @@ def run_ours_lm(args, w):
         torch.cuda.synchronize(dev)
         ms = e0.elapsed_time(e1)
         barrier()
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(ms, world, dev)
 
     with torch.cuda.stream(stream):
         for _ in range(args.warmup):
@@ -478,7 +486,7 @@ def run_ours_lm(args, w):
     if stage.status() != (0, 0):
         raise SystemExit(f"device status {stage.status()}")
     model_flops, hw_flops = lm_flops_per_step(w)
-    value = world * T / (ms_step * 1e-3)
+    value = whole_job_value(T, world, ms_step)
     line = {
         "metric": "small-LM training step tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,

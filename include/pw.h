@@ -350,6 +350,16 @@ pw_status_t pw_op_attention_bwd(const void* qkv, const void* o, const void* dout
 
 /* Status word used by the pw_op_* calls (same meaning as pw_layer_status). */
 pw_status_t pw_op_status(int* device_status, int* site);
+/* Clears the status word of the single-step calls (after a test has provoked an error). */
+pw_status_t pw_op_status_reset(void);
+/* Failure-path self-test.  Every device-side wait in this library is bounded; this call shows the
+ * mechanism working without hanging anything: it launches one warp that waits on a barrier
+ * nothing will ever signal, with a limit of limit_cycles SM cycles (clamped to [1e3, 2e9], i.e. at
+ * most about a second).  The wait gives up, the status word of the single-step calls records
+ * PW_ERR_TIMEOUT with site 990, and the kernel returns normally: *kernel_returned (host) = 1.
+ * Synchronises the stream.  pw_op_status then reports (PW_ERR_TIMEOUT, 990) until
+ * pw_op_status_reset. */
+pw_status_t pw_op_selftest_wait_timeout(uint64_t limit_cycles, int* kernel_returned, void* stream);
 
 #ifdef __cplusplus
 }

@@ -40,6 +40,7 @@ EXPORTS = (
     "pw_op_attention_fwd", "pw_op_attention_bwd", "pw_op_status",
     "pw_lm_workspace_bytes", "pw_lm_step",
     "pw_op_embedding_fwd", "pw_op_embedding_bwd_scratch_bytes", "pw_op_embedding_bwd", "pw_op_softmax_xent",
+    "pw_op_status_reset", "pw_op_selftest_wait_timeout",
 )
 
 
@@ -136,6 +137,7 @@ def lib() -> ctypes.CDLL:
         L.pw_op_embedding_bwd_scratch_bytes.argtypes = [ci, ci]
         L.pw_op_embedding_bwd.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp]
         L.pw_op_softmax_xent.argtypes = [vp, ci, vp, ci, ci, ctypes.c_float, vp, vp, vp]
+        L.pw_op_selftest_wait_timeout.argtypes = [ctypes.c_uint64, ctypes.POINTER(ci), vp]
         _lib = L
     return _lib
 
@@ -393,3 +395,15 @@ def op_status():
     c, s = ctypes.c_int(), ctypes.c_int()
     _check(lib().pw_op_status(ctypes.byref(c), ctypes.byref(s)))
     return c.value, s.value
+
+
+def op_status_reset():
+    _check(lib().pw_op_status_reset())
+
+
+def op_selftest_wait_timeout(limit_cycles=2_000_000, stream=None) -> int:
+    """Runs the bounded-wait self-test; returns 1 if the kernel's wait gave up and the kernel returned."""
+    r = ctypes.c_int(0)
+    _check(lib().pw_op_selftest_wait_timeout(limit_cycles, ctypes.byref(r), _stream(stream)))
+    return r.value
+

@@ -984,6 +984,36 @@ pw_status_t pw_op_softmax_xent(void* logits, int ld, const int32_t* labels, int 
     return PW_OK;
 }
 
+pw_status_t pw_op_selftest_wait_timeout(uint64_t limit_cycles, int* kernel_returned, void* stream)
+{
+    PW_RT_OR_FAIL();
+    if (!kernel_returned) return fail(PW_ERR_INVALID_ARG, "kernel_returned is NULL");
+    long long limit = static_cast<long long>(limit_cycles);
+    if (limit < 1000) limit = 1000;
+    if (limit > 2000000000ll) limit = 2000000000ll;            // about a second at most
+    int* flag = nullptr;
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&flag), sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(flag, 0, sizeof(int));
+    if (e != cudaSuccess) { if (flag) cudaFree(flag); return fail_cuda("self-test flag", e); }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const char* err = launch_wait_selftest(rt->op_status, limit, flag, st);
+    if (!err) {
+        e = cudaStreamSynchronize(st);
+        if (e == cudaSuccess) e = cudaMemcpy(kernel_returned, flag, sizeof(int), cudaMemcpyDeviceToHost);
+    }
+    cudaFree(flag);
+    if (err) return fail(PW_ERR_CUDA, err);
+    return e == cudaSuccess ? PW_OK : fail_cuda("self-test", e);
+}
+
+pw_status_t pw_op_status_reset(void)
+{
+    PW_RT_OR_FAIL();
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemset(rt->op_status, 0, 2 * sizeof(int));   // code and site; the work counters stay
+    return e == cudaSuccess ? PW_OK : fail_cuda("status reset", e);
+}
+
 pw_status_t pw_op_status(int* device_status, int* site)
 {
     PW_RT_OR_FAIL();

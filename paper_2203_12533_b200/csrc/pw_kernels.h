@@ -75,6 +75,9 @@ const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, voi
 size_t colsum_noalloc_max_columns();
 const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* out, int accumulate, cudaStream_t stream);
 
+// Bounded-wait self-test (selftest.cu): *returned (device int) becomes 1 when the wait gave up and the kernel went on.
+const char* launch_wait_selftest(DeviceStatus* status, long long limit, int* returned, cudaStream_t stream);
+
 // First / last layer of the language model (lm_head.cu).
 const char* launch_embedding_fwd(Runtime* rt, const void* ids, const void* E, int T, int d, int V, void* x0,
                                  DeviceStatus* status, cudaStream_t stream);

@@ -78,6 +78,8 @@ def test_softmax_xent_reports_a_label_outside_the_vocabulary(pw):
     torch.cuda.synchronize()
     assert pw.op_status()[0] == 1                                              # PW_ERR_INVALID_ARG recorded by the kernel
     assert torch.isfinite(lse).all()
+    pw.op_status_reset()
+    assert pw.op_status() == (0, 0)
 
 
 def run_lm_gpu(pw, w, seed=0, recompute=False, random_ln=True):
