@@ -1,0 +1,78 @@
+"""Single-GPU analogue of the paper's dispatch micro-benchmark (Section 5.1, Figures 5 and 6).
+
+The paper compares three ways of issuing a chain of small computations - one synchronous call
+per computation (OpByOp), one asynchronous call per computation (Chained) and the whole chain as
+one program (Fused) - and asks how long a computation must run before the host-side cost is
+hidden.  Here a computation is one decoder-layer call (forward + backward on one micro-batch) and
+the three modes are the dispatch modes of ``pw_stage_run_chain``: OPBYOP (synchronise after
+every layer call), ASYNC (enqueue everything) and GRAPH (one captured CUDA graph, replayed).
+
+    python -m paper_2203_12533_b200.dispatch_study [--layers 8] [--microbatches 8] [--reps 20]
+
+prints one JSON line per (sequence length, mode): layer calls per second and microseconds per
+call, for a chain of ``layers`` x ``microbatches`` x 2 calls at the width of workload 1.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import binding as pw
+from . import inputs
+
+
+def run(seq_len: int, layers: int, microbatches: int, reps: int, mode: int) -> float:
+    """Milliseconds per chain (L x M forward calls + L x M backward calls)."""
+    w = inputs.WORKLOADS[1].with_(seq_len=seq_len, n_layers=layers, n_microbatches=microbatches)
+    dev = torch.device("cuda")
+    stage = pw.Stage(layers, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
+    params = [[p.to(dev) for p in inputs.layer_params(w, 0, l)] for l in range(layers)]
+    grads = [[torch.zeros(p.shape, dtype=torch.float32, device=dev) for p in ps] for ps in params]
+    xs, dys = [], []
+    for m in range(microbatches):
+        x, dy = inputs.microbatch(w, 0, m)
+        xs.append(x.view(w.tokens, -1).to(dev))
+        dys.append(dy.view(w.tokens, -1).to(dev))
+    ys = [torch.empty_like(t) for t in xs]
+    dxs = [torch.empty_like(t) for t in xs]
+    ws = torch.empty(stage.workspace_bytes(microbatches, pw.SCHEDULE_GPIPE, True), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.Stream()
+
+    def chain():
+        stage.run_chain(params, grads, xs, dys, ys, dxs, ws, mode, pw.SCHEDULE_GPIPE, True, stream=stream)
+
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            chain()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            chain()
+        e1.record(stream)
+    torch.cuda.synchronize()
+    assert stage.status() == (0, 0)
+    return e0.elapsed_time(e1) / reps
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--layers", type=int, default=8)
+    ap.add_argument("--microbatches", type=int, default=8)
+    ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--seq-lens", type=int, nargs="+", default=[128, 256, 512, 1024, 2048])
+    args = ap.parse_args()
+    pw.lib()
+    modes = (("opbyop", pw.DISPATCH_OPBYOP), ("async", pw.DISPATCH_ASYNC), ("graph", pw.DISPATCH_GRAPH))
+    for S in args.seq_lens:
+        for name, mode in modes:
+            ms = run(S, args.layers, args.microbatches, args.reps, mode)
+            calls = 2 * args.layers * args.microbatches
+            print(json.dumps({"seq_len": S, "tokens_per_call": 2 * S, "mode": name, "ms_per_chain": ms,
+                              "us_per_layer_call": 1e3 * ms / calls, "layer_calls_per_s": calls / (ms * 1e-3)}), flush=True)
+
+
+if __name__ == "__main__":
+    main()
