@@ -87,8 +87,13 @@ __device__ __forceinline__ void epilogue_group(const uint32_t* v, int row, int c
             if (row < p.M) {
                 float u[8];
                 unpack8(*reinterpret_cast<const uint4*>(p.aux_in + static_cast<size_t>(row) * p.ld_aux + c), u);
+                if (p.act == 0) {                           // one uniform branch per group, not per pair
 #pragma unroll
-                for (int j = 0; j < 8; j += 2) gelu_grad_mul2(f[j], f[j + 1], u[j], u[j + 1], p.act);
+                    for (int j = 0; j < 8; j += 2) gelu_grad_mul2_erf(f[j], f[j + 1], u[j], u[j + 1]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; j += 2) gelu_grad_mul2(f[j], f[j + 1], u[j], u[j + 1], p.act);
+                }
             }
         }
     }
@@ -147,11 +152,14 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, 
                 epilogue_group<EPI>(v + 8 * g, row, col0 + g * 8, p, f);
                 o[g] = pack8(f);
                 if constexpr (EPI == kEpiBiasGelu) {
-                    // GeLU of the bf16 value stored as u: the backward reads u back and sees
-                    // exactly the argument the forward used
-                    unpack8(o[g], f);
+                    // GeLU of the pre-activation in fp32 (before its rounding to bf16 for storage)
+                    if (p.act == 0) {                       // one uniform branch per group, not per pair
 #pragma unroll
-                    for (int j = 0; j < 8; j += 2) gelu2(f[j], f[j + 1], p.act);
+                        for (int j = 0; j < 8; j += 2) gelu2_erf(f[j], f[j + 1]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 8; j += 2) gelu2(f[j], f[j + 1], p.act);
+                    }
                     o2[g] = pack8(f);
                 }
             }

@@ -461,18 +461,32 @@ __device__ __forceinline__ void normal_cdf_pdf2(float u0, float u1, uint64_t& cd
     poly = ffma2(t, poly, pack_f32x2(-0.142248368f, -0.142248368f));
     poly = ffma2(t, poly, pack_f32x2(0.127414796f, 0.127414796f));
     const uint64_t ht = fmul2(fmul2(poly, t), e);
-    float h0, h1;
-    unpack_f32x2(ht, h0, h1);
-    cdf = pack_f32x2(u0 < 0.f ? h0 : 1.0f - h0, u1 < 0.f ? h1 : 1.0f - h1);
+    // cdf = 1/2 + sign(u) (1/2 - half_tail): the sign of u is OR-ed into 1/2 - half_tail (>= 0), no compare / select
+    float g0, g1;
+    unpack_f32x2(ffma2(ht, pack_f32x2(-1.0f, -1.0f), pack_f32x2(0.5f, 0.5f)), g0, g1);
+    g0 = __uint_as_float(__float_as_uint(g0) | (__float_as_uint(u0) & 0x80000000u));
+    g1 = __uint_as_float(__float_as_uint(g1) | (__float_as_uint(u1) & 0x80000000u));
+    cdf = fadd2(pack_f32x2(g0, g1), pack_f32x2(0.5f, 0.5f));
 }
-__device__ __forceinline__ void gelu2(float& u0, float& u1, int act)
+__device__ __forceinline__ void gelu2_erf(float& u0, float& u1)
 {
-    if (act == 1) { u0 = gelu_f(u0, 1); u1 = gelu_f(u1, 1); return; }
     uint64_t cdf, e;
     normal_cdf_pdf2(u0, u1, cdf, e);
     unpack_f32x2(fmul2(pack_f32x2(u0, u1), cdf), u0, u1);
 }
+__device__ __forceinline__ void gelu2(float& u0, float& u1, int act)
+{
+    if (act == 1) { u0 = gelu_f(u0, 1); u1 = gelu_f(u1, 1); return; }
+    gelu2_erf(u0, u1);
+}
 // g0, g1 *= GeLU'(u0), GeLU'(u1)
+__device__ __forceinline__ void gelu_grad_mul2_erf(float& g0, float& g1, float u0, float u1)
+{
+    uint64_t cdf, e;
+    normal_cdf_pdf2(u0, u1, cdf, e);
+    const uint64_t up = fmul2(pack_f32x2(u0, u1), pack_f32x2(0.3989422804f, 0.3989422804f));
+    unpack_f32x2(fmul2(pack_f32x2(g0, g1), ffma2(up, e, cdf)), g0, g1);
+}
 __device__ __forceinline__ void gelu_grad_mul2(float& g0, float& g1, float u0, float u1, int act)
 {
     if (act == 1) { g0 *= gelu_grad_f(u0, 1); g1 *= gelu_grad_f(u1, 1); return; }
