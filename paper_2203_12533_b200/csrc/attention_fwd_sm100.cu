@@ -443,10 +443,19 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                 }
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                    float a0, a1;
-                    unpack_f32x2(ffma2(pack_f32x2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), sl2x2, mbx2), a0, a1);
-                    const float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
-                    lsum[(i >> 1) & 1] = fadd2(lsum[(i >> 1) & 1], pack_f32x2(p0, p1));
+                    // the MUFU bounds this loop: every fourth pair takes the FMA-pipe exponential
+                    const uint64_t a = ffma2(pack_f32x2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), sl2x2, mbx2);
+                    uint64_t pe;
+                    if (((i >> 1) & 3) == 3) {
+                        pe = exp2_poly2(a);
+                    } else {
+                        float a0, a1;
+                        unpack_f32x2(a, a0, a1);
+                        pe = pack_f32x2(ex2_approx(a0), ex2_approx(a1));
+                    }
+                    lsum[(i >> 1) & 1] = fadd2(lsum[(i >> 1) & 1], pe);
+                    float p0, p1;
+                    unpack_f32x2(pe, p0, p1);
                     v[i >> 1] = pack_bf16(p0, p1);
                 }
                 tmem_st16(s_addr + c * 16, v);

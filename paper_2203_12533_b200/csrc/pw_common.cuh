@@ -444,6 +444,28 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, bool a_mn_m
            (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
 }
 
+// 2^a for two values on the FMA / ALU pipes (no MUFU): a = n + f with n = round(a), f in [-0.5, 0.5];
+// 2^f by a cubic (relative error 1.1e-4, far below bf16 rounding), n added into the exponent field.
+// Inputs below -125 (masked scores are -inf) give about 2^-125.
+__device__ __forceinline__ uint64_t exp2_poly2(uint64_t a)
+{
+    float a0, a1;
+    unpack_f32x2(a, a0, a1);
+    const uint64_t ac = pack_f32x2(fmaxf(a0, -125.0f), fmaxf(a1, -125.0f));
+    const uint64_t t = fadd2(ac, pack_f32x2(12582912.0f, 12582912.0f));          // 1.5 * 2^23: integer part lands in the mantissa
+    const uint64_t fi = fadd2(t, pack_f32x2(-12582912.0f, -12582912.0f));
+    const uint64_t f = ffma2(fi, pack_f32x2(-1.0f, -1.0f), ac);
+    uint64_t q = ffma2(pack_f32x2(0.05459282f, 0.05459282f), f, pack_f32x2(0.24221784f, 0.24221784f));
+    q = ffma2(q, f, pack_f32x2(0.6933686f, 0.6933686f));
+    q = ffma2(q, f, pack_f32x2(1.0f, 1.0f));
+    float t0, t1, q0, q1;
+    unpack_f32x2(t, t0, t1);
+    unpack_f32x2(q, q0, q1);
+    const uint32_t r0 = __float_as_uint(q0) + (__float_as_uint(t0) << 23);
+    const uint32_t r1 = __float_as_uint(q1) + (__float_as_uint(t1) << 23);
+    return pack_f32x2(__uint_as_float(r0), __uint_as_float(r1));
+}
+
 // GeLU / GeLU' of two values at once (erf form): the polynomial and scaling steps run as two-wide
 // fp32 instructions, the reciprocal and the exponential stay one MUFU op per value.
 //   half_tail = erfc(|u|/sqrt2)/2 = (b1 t + ... + b5 t^5) exp(-u^2/2),  t = 1/(1 + p|u|/sqrt2),  b = a/2
