@@ -121,6 +121,53 @@ def whole_job_value(units_per_rank: float, world: int, ms: float) -> float:
     return world * units_per_rank / (ms * 1e-3)
 
 
+def isolated_elementwise(pw, w, peaks, dev, iters=30, nbuf=6):
+    """LayerNorm / column-sum kernels timed back to back through the single-step entry points on
+    HBM-resident inputs (a rotation of `nbuf` buffer sets, far larger than the 126 MB L2), so that
+    launch gaps and event brackets do not count: GB/s of algorithmic bytes vs the measured copy rate."""
+    import torch
+    T, d, F = w.tokens, w.d_model, w.d_ff
+    g = torch.Generator(device="cpu").manual_seed(1)
+    rnd = lambda *shape: torch.randn(shape, generator=g).to(torch.bfloat16).to(dev)
+    xs = [rnd(T, d) for _ in range(nbuf)]
+    hs = [torch.empty_like(x) for x in xs]
+    gamma, beta = torch.ones(d, dtype=torch.bfloat16, device=dev), torch.zeros(d, dtype=torch.bfloat16, device=dev)
+    mu, rs = torch.empty(T, device=dev), torch.empty(T, device=dev)
+    outs = [torch.zeros(d, device=dev) for _ in range(4)]
+    part = torch.empty(pw.op_layernorm_bwd_scratch_bytes(T, d), dtype=torch.uint8, device=dev)
+
+    def timeit(fn):
+        for i in range(3):
+            fn(i)
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        return e0.elapsed_time(e1) / iters
+
+    res = {}
+    ms = timeit(lambda i: pw.op_layernorm_fwd(xs[i % nbuf], gamma, beta, 1e-5, hs[i % nbuf], mu, rs))
+    res["ln_fwd"] = (ms, 4.0 * T * d + 8.0 * T)
+    dhs = [rnd(T, d) for _ in range(nbuf)]
+    ms = timeit(lambda i: pw.op_layernorm_bwd(dhs[i % nbuf], xs[i % nbuf], mu, rs, gamma, xs[(i + 1) % nbuf], hs[i % nbuf],
+                                               outs[0], outs[1], outs[2], outs[3], False, part))
+    res["ln_bwd"] = (ms, 8.0 * T * d + 8.0 * T)
+    del dhs
+    for name, N in (("colsum_ff", F), ("colsum_qkv", 3 * d)):
+        n = max(2, min(nbuf, int(1.5e9 // (2 * T * N))))
+        ins = [rnd(T, N) for _ in range(n)]
+        out = torch.zeros(N, device=dev)
+        sc = torch.empty(pw.op_colsum_scratch_bytes(T, N), dtype=torch.uint8, device=dev)
+        ms = timeit(lambda i: pw.op_colsum(ins[i % n], out, False, sc))
+        res[name] = (ms, 2.0 * T * N)
+        del ins
+    return {k: {"us": ms * 1e3, "gbs": b / (ms * 1e-3) / 1e9, "frac_of_measured_hbm": b / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+            for k, (ms, b) in res.items()}
+
+
 def hw_flops_per_step(w) -> float:
     """Executed FLOPs: model FLOPs plus, with recompute, one forward without the FC2 GEMM."""
     per_call = w.model_flops_per_layer_call()
@@ -368,6 +415,8 @@ def run_ours(args, w):
             "traffic": GEMM_DRAM_TRAFFIC_PER_LAUNCH.get(w.name),
         }
 
+    if rank == 0 and world == 1 and w.tokens * w.d_ff <= (1 << 27):
+        line["kernels_isolated"] = isolated_elementwise(pw, w, peaks, dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle as oracle_mod
         orc = oracle_mod.Oracle("f32")

@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <cstddef>
 #include <map>
 #include <mutex>
 #include <new>
@@ -383,6 +384,10 @@ static pw_status_t read_status(DeviceStatus* dev, int* code, int* site)
     if (e != cudaSuccess) return fail_cuda("cudaMemcpy(status)", e);
     if (code) *code = h.code;
     if (site) *site = h.site;
+    // A kernel that gave up may have left the work counters of the persistent attention kernels
+    // mid-count; the device is idle here, so they are put back to zero (the error stays recorded).
+    if (h.code != 0 && (h.sched[0] | h.sched[1] | h.sched[2] | h.sched[3] | h.sched[4] | h.sched[5]) != 0)
+        cudaMemset(reinterpret_cast<char*>(dev) + offsetof(DeviceStatus, sched), 0, sizeof(h.sched));
     return PW_OK;
 }
 
