@@ -274,7 +274,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
         FwdItem it;
         for (int k = 0; ok; ++k) {
             if (!wait(21 + (k & 1), (k >> 1) & 1, 423)) break;
-            const int idx = item_slot[k & 1];
+            const int idx = __shfl_sync(0xffffffffu, item_slot[k & 1], 0);   // broadcast: everything derived from it is warp-uniform
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(23 + (k & 1)));
             if (!fwd_item(p, idx, it)) break;
