@@ -350,6 +350,10 @@ pw_status_t pw_op_attention_bwd(const void* qkv, const void* o, const void* dout
 
 /* Status word used by the pw_op_* calls (same meaning as pw_layer_status). */
 pw_status_t pw_op_status(int* device_status, int* site);
+/* y[i] = x[i] * scale + shift on fp32 device vectors (y may alias x).  The node type of the
+ * paper's Figure 2 program (a(x) = x*2, b(x) = x+1, c(x) = x/2; f(v) = (b(a(v)), a(c(a(v))))): lets
+ * that worked example run through the same enqueue-only / captured-graph dispatch as the layers. */
+pw_status_t pw_op_affine_f32(const void* x, long long n, float scale, float shift, void* y, void* stream);
 /* Clears the status word of the single-step calls (after a test has provoked an error). */
 pw_status_t pw_op_status_reset(void);
 /* Failure-path self-test.  Every device-side wait in this library is bounded; this call shows the

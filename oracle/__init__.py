@@ -349,3 +349,17 @@ class Oracle:
         return {"loss": loss, "grads": grads, "dE": dE, "dlnf_gamma": dg, "dlnf_beta": db,
                 "x0": acts[0], "hL": acts[-1], "hf": hf, "lse": lse, "dx0": g}
 
+    # -- the element-wise computations of the Figure 2 program --
+    def affine(self, x, scale, shift):
+        x = self._a(x)
+        y = np.empty_like(x)
+        self._fn("pwo_affine")(self._p(x), ctypes.c_long(x.size), ctypes.c_double(scale), ctypes.c_double(shift), self._p(y))
+        return y
+
+    def figure2_program(self, v):
+        """f(v) = (b(a(v)), a(c(a(v)))) with a(x) = 2x, b(x) = x + 1, c(x) = x / 2 (Figure 2)."""
+        a = lambda t: self.affine(t, 2.0, 0.0)
+        b = lambda t: self.affine(t, 1.0, 1.0)
+        c = lambda t: self.affine(t, 0.5, 0.0)
+        return b(a(v)), a(c(a(v)))
+

@@ -476,3 +476,10 @@ void FN(pwo_head_bwd)(const REAL* hf, const REAL* E, const int* labels, const RE
     free(dz);
 }
 
+/* ---- The three one-line computations of the paper's Figure 2 program are all of the form
+ * y = x * scale + shift (a: x*2, b: x+1, c: x/2). ---- */
+void FN(pwo_affine)(const REAL* x, long n, double scale, double shift, REAL* y)
+{
+    for (long i = 0; i < n; ++i) y[i] = (REAL)((double)x[i] * scale + shift);
+}
+

@@ -40,7 +40,7 @@ EXPORTS = (
     "pw_op_attention_fwd", "pw_op_attention_bwd", "pw_op_status",
     "pw_lm_workspace_bytes", "pw_lm_step",
     "pw_op_embedding_fwd", "pw_op_embedding_bwd_scratch_bytes", "pw_op_embedding_bwd", "pw_op_softmax_xent",
-    "pw_op_status_reset", "pw_op_selftest_wait_timeout",
+    "pw_op_status_reset", "pw_op_selftest_wait_timeout", "pw_op_affine_f32",
 )
 
 
@@ -138,6 +138,7 @@ def lib() -> ctypes.CDLL:
         L.pw_op_embedding_bwd.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp]
         L.pw_op_softmax_xent.argtypes = [vp, ci, vp, ci, ci, ctypes.c_float, vp, vp, vp]
         L.pw_op_selftest_wait_timeout.argtypes = [ctypes.c_uint64, ctypes.POINTER(ci), vp]
+        L.pw_op_affine_f32.argtypes = [vp, ctypes.c_longlong, ctypes.c_float, ctypes.c_float, vp, vp]
         _lib = L
     return _lib
 
@@ -406,4 +407,8 @@ def op_selftest_wait_timeout(limit_cycles=2_000_000, stream=None) -> int:
     r = ctypes.c_int(0)
     _check(lib().pw_op_selftest_wait_timeout(limit_cycles, ctypes.byref(r), _stream(stream)))
     return r.value
+
+
+def op_affine_f32(x, scale, shift, y, stream=None):
+    _check(lib().pw_op_affine_f32(_p(x), x.numel(), scale, shift, _p(y), _stream(stream)))
 

@@ -989,6 +989,14 @@ pw_status_t pw_op_softmax_xent(void* logits, int ld, const int32_t* labels, int 
     return PW_OK;
 }
 
+pw_status_t pw_op_affine_f32(const void* x, long long n, float scale, float shift, void* y, void* stream)
+{
+    PW_RT_OR_FAIL();
+    if (!aligned(x, 4) || !aligned(y, 4)) return fail(PW_ERR_INVALID_ARG, "affine: NULL or misaligned pointer");
+    PW_OP(launch_affine_f32(x, n, scale, shift, y, static_cast<cudaStream_t>(stream)));
+    return PW_OK;
+}
+
 pw_status_t pw_op_selftest_wait_timeout(uint64_t limit_cycles, int* kernel_returned, void* stream)
 {
     PW_RT_OR_FAIL();

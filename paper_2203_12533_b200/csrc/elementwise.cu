@@ -123,6 +123,15 @@ ln_fwd_kernel(const __nv_bfloat16* x, const __nv_bfloat16* gamma,
     if (wr == 0 && lane == 0) { mu[row] = mean; rstd[row] = r; }
 }
 
+__global__ void __launch_bounds__(256)
+affine_f32_kernel(const float* x, long long n, float scale, float shift, float* y)
+{
+    grid_dep_launch();
+    grid_dep_wait();
+    const long long i = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
+    if (i < n) y[i] = fmaf(x[i], scale, shift);
+}
+
 // W warps per row and CH pieces per lane for a row of d elements (d a multiple of 256).
 bool plan_warp_rows(int d, int* W, int* CH)
 {
@@ -428,6 +437,18 @@ const char* launch_layernorm_bwd(Runtime* rt, const void* dh, const void* x, con
     dim3 rgrid((d + 31) / 32, 4);
     return launch_k(reduce_partials_kernel, rgrid, dim3(1024), 0, stream, static_cast<const float*>(P), grid * rp.rows_per_cta, 4, d, outs, accumulate) == cudaSuccess
                ? nullptr : "layernorm bwd reduce launch failed";
+}
+
+// y = x * scale + shift on fp32 vectors: the node type of the paper's Figure 2 program (a: x*2,
+// b: x+1, c: x/2), used to run that worked example through the dispatch paths.
+const char* launch_affine_f32(const void* x, long long n, float scale, float shift, void* y, cudaStream_t stream)
+{
+    if (n <= 0) return "affine: empty vector";
+    const long long blocks = (n + 255) / 256;
+    if (blocks > 0x7fffffffll) return "affine: vector too long";
+    return launch_k(affine_f32_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, stream, static_cast<const float*>(x), n,
+                    scale, shift, static_cast<float*>(y)) == cudaSuccess
+               ? nullptr : "affine launch failed";
 }
 
 size_t colsum_scratch_bytes(Runtime* rt, int T, int N)

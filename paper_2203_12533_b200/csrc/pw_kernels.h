@@ -75,6 +75,8 @@ const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, voi
 size_t colsum_noalloc_max_columns();
 const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* out, int accumulate, cudaStream_t stream);
 
+const char* launch_affine_f32(const void* x, long long n, float scale, float shift, void* y, cudaStream_t stream);
+
 // Bounded-wait self-test (selftest.cu): *returned (device int) becomes 1 when the wait gave up and the kernel went on.
 const char* launch_wait_selftest(DeviceStatus* status, long long limit, int* returned, cudaStream_t stream);
 

@@ -210,3 +210,38 @@ def test_attention_is_causal_and_deterministic(pw):
     torch.cuda.synchronize()
     assert torch.equal(o1, o2)
     assert torch.equal(o1[:150], o3[:150]) and not torch.equal(o1[150:], o3[150:])
+
+
+def test_figure2_program_on_a_stream_and_as_a_captured_graph(pw):
+    """The paper's Figure 2 worked example, f(v) = (b(a(v)), a(c(a(v)))), a = x*2, b = x+1, c = x/2,
+    run through the C ABI: enqueued on a stream and as a captured CUDA graph; both must give the
+    values the paper prints."""
+    import os
+    vals = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", "figure2_program.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                k, *nums = line.split()
+                vals[k] = torch.tensor([float(t) for t in nums], dtype=torch.float32)
+    v = vals["v"].cuda()
+    t1, t2, out0, out1 = (torch.empty_like(v) for _ in range(4))
+    stream = torch.cuda.Stream()
+
+    def program():
+        pw.op_affine_f32(v, 2.0, 0.0, t1, stream=stream)        # a(v)
+        pw.op_affine_f32(t1, 1.0, 1.0, out0, stream=stream)     # b(a(v))
+        pw.op_affine_f32(t1, 0.5, 0.0, t2, stream=stream)       # c(a(v))
+        pw.op_affine_f32(t2, 2.0, 0.0, out1, stream=stream)     # a(c(a(v)))
+
+    with torch.cuda.stream(stream):
+        program()
+    torch.cuda.synchronize()
+    assert torch.equal(out0.cpu(), vals["out0"]) and torch.equal(out1.cpu(), vals["out1"])
+    out0.zero_(); out1.zero_()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        program()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out0.cpu(), vals["out0"]) and torch.equal(out1.cpu(), vals["out1"])

@@ -363,3 +363,17 @@ def test_structure_matches_section_5_3_parameter_count():
     assert round(total / 1e9) == int(vals["params_billion"][0])
     assert abs(total - L * (4 * d * d + 2 * d * Fh)) / total < 1e-3     # biases and LN add < 0.1 %
     assert len(SAVED_NAMES) == 12 and len(PARAM_NAMES) == 12
+
+
+def test_figure2_program_reproduces_the_printed_values():
+    """The paper prints the input and both outputs of its Figure 2 example program."""
+    vals = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", "figure2_program.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                k, *nums = line.split()
+                vals[k] = np.array([float(t) for t in nums])
+    o = Oracle("f32")
+    out0, out1 = o.figure2_program(vals["v"])
+    assert np.array_equal(out0, vals["out0"].astype(np.float32))
+    assert np.array_equal(out1, vals["out1"].astype(np.float32))
