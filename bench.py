@@ -415,7 +415,7 @@ def run_ours(args, w):
             "traffic": GEMM_DRAM_TRAFFIC_PER_LAUNCH.get(w.name),
         }
 
-    if rank == 0 and world == 1 and w.tokens * w.d_ff <= (1 << 27):
+    if rank == 0 and world == 1 and not args.no_isolated and w.tokens * w.d_ff <= (1 << 27):
         line["kernels_isolated"] = isolated_elementwise(pw, w, peaks, dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle as oracle_mod
@@ -629,6 +629,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=30)
     ap.add_argument("--cpu-sample-batch", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-isolated", action="store_true", help="skip the back-to-back timing of the element-wise kernels")
     args = ap.parse_args()
     from paper_2203_12533_b200 import inputs
     w = inputs.WORKLOADS[args.workload]
