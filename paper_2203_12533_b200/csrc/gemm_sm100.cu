@@ -62,9 +62,10 @@ __device__ __forceinline__ void tile_info(const GemmParams& p, int v, int& m0, i
     n0 = ni * p.bn + half * (p.bn >> 1);
 }
 
-// One 8-column group of the bf16 epilogues: f = acc (+bias) (+residual | x GeLU'(u)).
+// One 8-column group of the bf16 epilogues: f = acc (+bias) (+residual | x GeLU'(u)).  `aux` holds the
+// group's 8 residual / pre-activation values, fetched by the caller ahead of the TMEM load.
 template <int EPI>
-__device__ __forceinline__ void epilogue_group(const uint32_t* v, int row, int c, const GemmParams& p, float* f)
+__device__ __forceinline__ void epilogue_group(const uint32_t* v, int row, int c, const GemmParams& p, const uint4& aux, float* f)
 {
 #pragma unroll
     for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[j]);
@@ -78,7 +79,7 @@ __device__ __forceinline__ void epilogue_group(const uint32_t* v, int row, int c
         if constexpr (EPI == kEpiBiasResid) {
             if (row < p.M) {
                 float r[8];
-                unpack8(*reinterpret_cast<const uint4*>(p.aux_in + static_cast<size_t>(row) * p.ld_aux + c), r);
+                unpack8(aux, r);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) f[j] += r[j];
             }
@@ -86,7 +87,7 @@ __device__ __forceinline__ void epilogue_group(const uint32_t* v, int row, int c
         if constexpr (EPI == kEpiDGelu) {
             if (row < p.M) {
                 float u[8];
-                unpack8(*reinterpret_cast<const uint4*>(p.aux_in + static_cast<size_t>(row) * p.ld_aux + c), u);
+                unpack8(aux, u);
                 if (p.act == 0) {                           // one uniform branch per group, not per pair
 #pragma unroll
                     for (int j = 0; j < 8; j += 2) gelu_grad_mul2_erf(f[j], f[j + 1], u[j], u[j + 1]);
@@ -142,17 +143,53 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, 
         for (int ch = pi; ch < nchunks; ch += pstride) {
             const int col0 = n0 + ch * 32;
             if (col0 >= p.N) break;
+            // residual / saved pre-activation of this chunk: requested before the TMEM load so that the
+            // (row-strided, L2-latency) reads overlap it
+            uint4 aux[4] = {};
+            if constexpr (EPI == kEpiBiasResid || EPI == kEpiDGelu) {
+                if (row < p.M) {
+#pragma unroll
+                    for (int g = 0; g < 4; ++g)
+                        if (col0 + g * 8 < p.N)
+                            aux[g] = *reinterpret_cast<const uint4*>(p.aux_in + static_cast<size_t>(row) * p.ld_aux + col0 + g * 8);
+                }
+            }
             uint32_t v[32];
             tmem_ld32(taddr + ch * 32, v);
             tc_wait_ld();
-            uint4 o[4], o2[4];
+            uint4 o[4];
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
                 float f[8];
-                epilogue_group<EPI>(v + 8 * g, row, col0 + g * 8, p, f);
+                epilogue_group<EPI>(v + 8 * g, row, col0 + g * 8, p, aux[g], f);
                 o[g] = pack8(f);
                 if constexpr (EPI == kEpiBiasGelu) {
-                    // GeLU of the pre-activation in fp32 (before its rounding to bf16 for storage)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) v[8 * g + j] = __float_as_uint(f[j]);   // fp32 pre-activation, kept for GeLU
+                }
+            }
+            auto store_chunk = [&](const uint4* src, const CUtensorMap* map) {
+                const uint32_t half = SINGLE_SLAB ? 0u : (nout++ & 1u) * 2048u;
+                if (lane == 0) { if (SINGLE_SLAB) bulk_wait_read0(); else bulk_wait_read1(); }
+                __syncwarp();
+#pragma unroll
+                for (int g = 0; g < 4; ++g)
+                    *reinterpret_cast<uint4*>(slab + half + lane * 64 + ((g ^ sw) << 4)) = src[g];
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(map, slab_u32 + half, col0, row0);
+                    bulk_commit();
+                }
+            };
+            store_chunk(o, tmC);
+            if constexpr (EPI == kEpiBiasGelu) {
+                // GeLU of the fp32 pre-activation, evaluated while the store above drains the slab
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    float f[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[8 * g + j]);
                     if (p.act == 0) {                       // one uniform branch per group, not per pair
 #pragma unroll
                         for (int j = 0; j < 8; j += 2) gelu2_erf(f[j], f[j + 1]);
@@ -160,24 +197,9 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, 
 #pragma unroll
                         for (int j = 0; j < 8; j += 2) gelu2(f[j], f[j + 1], p.act);
                     }
-                    o2[g] = pack8(f);
+                    o[g] = pack8(f);
                 }
-            }
-            constexpr int kOuts = (EPI == kEpiBiasGelu) ? 2 : 1;
-#pragma unroll
-            for (int t = 0; t < kOuts; ++t) {
-                const uint32_t half = SINGLE_SLAB ? 0u : (nout++ & 1u) * 2048u;
-                if (lane == 0) { if (SINGLE_SLAB) bulk_wait_read0(); else bulk_wait_read1(); }
-                __syncwarp();
-#pragma unroll
-                for (int g = 0; g < 4; ++g)
-                    *reinterpret_cast<uint4*>(slab + half + lane * 64 + ((g ^ sw) << 4)) = (t == 0) ? o[g] : o2[g];
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) {
-                    tma_store_2d(t == 0 ? tmC : tmAux, slab_u32 + half, col0, row0);
-                    bulk_commit();
-                }
+                store_chunk(o, tmAux);
             }
         }
     }
