@@ -207,3 +207,36 @@ def test_chain_workspace_too_small_is_reported_before_launch(pw):
 def test_cfg2_full_size_parity(pw, oracle32):
     """The benchmark workload (d=2048, 16x128 heads, F=8192, S=1024, B=8) against the fp32 oracle."""
     check_layer_against_oracle(pw, oracle32, inputs.WORKLOADS[2])
+
+
+# ------------------------------------------------------------------------------------------ full sizes of workloads 3 and 4
+@pytest.mark.parametrize("wid", [3, 4], ids=["cfg3_layer_full_size", "cfg4_full_size"])
+def test_full_size_wide_layer_by_the_causal_prefix_property(pw, oracle32, wid):
+    """One layer of workloads 3 / 4 at its full size (B x 2048 tokens, d = 4096 / 8192), checked through a
+    property that holds at any size: the model is causal and sequences are independent, so with an
+    upstream gradient that is zero outside the first P tokens of every sequence, the outputs on
+    those prefixes, their input gradients and ALL parameter gradients equal those of the problem
+    truncated to P tokens per sequence - which the oracle can compute - and dx is exactly zero
+    beyond the prefixes."""
+    w = inputs.WORKLOADS[wid].with_(n_layers=1, n_microbatches=1)
+    P = 64
+    params = inputs.layer_params(w, 0, 0, random_ln=True)
+    x, dy = inputs.microbatch(w, 0, 0)
+    dy = dy.clone()
+    dy[:, P:, :] = 0
+    layer = make_layer(pw, w)
+    out = run_layer_gpu(pw, layer, [p.cuda() for p in params], x.cuda().view(-1, w.d_model), dy.cuda().view(-1, w.d_model))
+    y = out["y"].view(w.batch, w.seq_len, w.d_model)
+    dx = out["dx"].view(w.batch, w.seq_len, w.d_model)
+    assert torch.count_nonzero(dx[:, P:, :]) == 0
+    wt = w.with_(seq_len=P)
+    D = dims_of(wt)
+    ps = [p.float().numpy() for p in params]
+    xt = x[:, :P, :].float().numpy().reshape(-1, w.d_model)
+    dyt = dy[:, :P, :].float().numpy().reshape(-1, w.d_model)
+    yw, sv = oracle32.layer_fwd(D, ps, xt)
+    dxw, gw = oracle32.layer_bwd(D, ps, xt, sv, dyt)
+    assert rel_l2(y[:, :P, :].reshape(-1, w.d_model), yw) < ACT_TOL
+    assert rel_l2(dx[:, :P, :].reshape(-1, w.d_model), dxw) < GRAD_TOL
+    errs = {name: rel_l2(g, want) for name, g, want in zip(pw.PARAM_NAMES, out["grads"], gw)}
+    assert max(errs.values()) < GRAD_TOL, errs
