@@ -240,3 +240,11 @@ def test_full_size_wide_layer_by_the_causal_prefix_property(pw, oracle32, wid):
     assert rel_l2(dx[:, :P, :].reshape(-1, w.d_model), dxw) < GRAD_TOL
     errs = {name: rel_l2(g, want) for name, g, want in zip(pw.PARAM_NAMES, out["grads"], gw)}
     assert max(errs.values()) < GRAD_TOL, errs
+
+
+def test_single_tile_layer(pw, oracle64):
+    """T = 128 tokens: one query tile per head (no second tile in the attention kernels), GEMMs on the one-CTA path."""
+    w = inputs.Workload("single_tile", 256, 2, 128, 640, 128, 1)
+    check_layer_against_oracle(pw, oracle64, w, random_ln=True)
+    w = inputs.Workload("odd_tiles", 768, 12, 64, 384, 384, 1, sigma_w=0.03)    # S = 3 x 128: the last pair has one tile
+    check_layer_against_oracle(pw, oracle64, w, random_ln=True, save_ctx=False)
