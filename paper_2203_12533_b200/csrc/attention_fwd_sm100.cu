@@ -246,8 +246,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
             }
             __syncwarp();
         };
-        // O_t (+)= P_t V from V stage s; P_t is bf16 packed over the S columns it came from: keys
-        // 0..63 in columns 0..31 of S_t, keys 64..127 in columns 64..95
+        // O_t (+)= P_t V from V stage s; P_t is bf16 packed over the S columns it came from: the 16
+        // keys of step ks sit in 8 columns at (ks/4)*64 + ((ks%4)/2)*32 + (ks%2)*8 of S_t
         auto issue_pv = [&](int t, int s, bool acc) {
             const uint64_t dv = make_smem_desc_sw128(sb + L::kV + s * L::kTile, 16384, 1024);
             const uint32_t dst = tb + 256 + t * 128, src = tb + t * 128;
@@ -255,7 +255,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                 umma_f16_ta(dst, src, dv, idesc_pv, acc ? 1u : 0u);
 #pragma unroll
                 for (int ks = 1; ks < 8; ++ks)
-                    umma_f16_ta(dst, src + (ks >> 2) * 64 + (ks & 3) * 8, desc_advance(dv, ks * 2048), idesc_pv, 1u);
+                    umma_f16_ta(dst, src + (ks >> 2) * 64 + ((ks & 3) >> 1) * 32 + (ks & 1) * 8, desc_advance(dv, ks * 2048), idesc_pv, 1u);
             }
             __syncwarp();
         };
@@ -388,20 +388,27 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
             if (tracer) PW_TRACE(2 + t, 1);
             const bool diag = j == n_t - 1;
             const int lim = diag ? r - hf * 64 : 64;        // columns i > lim of my 64 are masked (diagonal tile)
-            // pass 1: row maximum, 32 scores at a time (keeps the register count under the 576-thread limit)
+            // pass 1: row maximum.  Scores 0..31 are read, used and dropped; scores 32..63 stay in
+            // registers for the second pass (all 64 would not fit under the 576-thread register limit).
             float mxs[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
+            uint32_t vk[32];
+            {
                 uint32_t v[32];
-                tmem_ld32(s_addr + c * 32, v);
+                tmem_ld32(s_addr, v);
+                tmem_ld32(s_addr + 32, vk);
                 tc_wait_ld();
                 if (diag) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = c * 32 + i > lim ? 0xff800000u : v[i];
+                    for (int i = 0; i < 32; ++i) {
+                        v[i] = i > lim ? 0xff800000u : v[i];
+                        vk[i] = 32 + i > lim ? 0xff800000u : vk[i];
+                    }
                 }
 #pragma unroll
-                for (int i = 0; i < 32; i += 2)
-                    mxs[(i >> 1) & 3] = fmax3(mxs[(i >> 1) & 3], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+                for (int i = 0; i < 32; i += 2) {
+                    mxs[(i >> 1) & 1] = fmax3(mxs[(i >> 1) & 1], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+                    mxs[2 + ((i >> 1) & 1)] = fmax3(mxs[2 + ((i >> 1) & 1)], __uint_as_float(vk[i]), __uint_as_float(vk[i + 1]));
+                }
             }
             if (tracer) PW_TRACE(2 + t, 2);
             const float mine = fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3]));
@@ -427,20 +434,12 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                 }
             }
             if (tracer) PW_TRACE(2 + t, 3);
-            // pass 2: p = exp2((s - m) * scale * log2e), packed bf16 written over my own S columns
-            // (scores 0..31 -> columns 0..15, scores 32..63 -> columns 16..31: always behind the loads)
+            // pass 2: p = exp2((s - m) * scale * log2e), packed bf16 written over my own S columns: first the
+            // kept scores 32..63 (into columns 32..47, their own), then scores 0..31 re-read (into columns 0..15)
             const float mb = m_used * sl2;
             const uint64_t sl2x2 = pack_f32x2(sl2, sl2), mbx2 = pack_f32x2(-mb, -mb);
             uint64_t lsum[2] = {0ull, 0ull};
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t v[32];
-                tmem_ld32(s_addr + c * 32, v);
-                tc_wait_ld();
-                if (diag) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = c * 32 + i > lim ? 0xff800000u : v[i];
-                }
+            auto exps = [&](uint32_t* v) {
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
                     // the MUFU bounds this loop: every fourth pair takes the FMA-pipe exponential
@@ -458,7 +457,19 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                     unpack_f32x2(pe, p0, p1);
                     v[i >> 1] = pack_bf16(p0, p1);
                 }
-                tmem_st16(s_addr + c * 16, v);
+            };
+            {
+                uint32_t v[32];
+                tmem_ld32(s_addr, v);                        // in flight while the kept half is processed
+                exps(vk);
+                tmem_st16(s_addr + 32, vk);
+                tc_wait_ld();
+                if (diag) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = i > lim ? 0xff800000u : v[i];
+                }
+                exps(v);
+                tmem_st16(s_addr, v);
             }
             {
                 float s0, s1;
