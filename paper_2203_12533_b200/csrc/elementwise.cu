@@ -159,7 +159,10 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 
 // The kernel is bound by instruction issue as much as by memory, so all element-wise arithmetic
 // is two-wide fp32 (values of neighbouring columns packed in one 64-bit register).
-template <int CHUNKS>
+// BIAS_SUMS: also produce the column sums of the residual gradient and of dx (the two bias
+// gradients that the LN2 backward of a layer yields for free); without them the partial rows hold
+// two quantities instead of four.
+template <int CHUNKS, bool BIAS_SUMS>
 __global__ void __launch_bounds__(kRowThreadsMax, CHUNKS == 1 ? 2 : 1)
 ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
               const float* mu, const float* rstd, const __nv_bfloat16* gamma,
@@ -260,16 +263,17 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
                     const uint64_t t = ffma2(xh[j][k], nmgx2, fadd2(g[j][k], nmg2));
                     w[k] = pack_pair_bf16(ffma2(r2, t, rs[j][k]));
                     // the bias gradient sums the values that are actually stored
-                    acc_x[j][k] = fadd2(acc_x[j][k], pack_f32x2(bf16_lo(w[k]), bf16_hi(w[k])));
+                    if (BIAS_SUMS) acc_x[j][k] = fadd2(acc_x[j][k], pack_f32x2(bf16_lo(w[k]), bf16_hi(w[k])));
                     acc_g[j][k] = ffma2(dhv[j][k], xh[j][k], acc_g[j][k]);
                     acc_b[j][k] = fadd2(acc_b[j][k], dhv[j][k]);
-                    acc_r[j][k] = fadd2(acc_r[j][k], rs[j][k]);
+                    if (BIAS_SUMS) acc_r[j][k] = fadd2(acc_r[j][k], rs[j][k]);
                 }
                 *reinterpret_cast<uint4*>(dx + off) = make_uint4(w[0], w[1], w[2], w[3]);
             }
         }
     }
-    float* prow = partials + static_cast<size_t>(blockIdx.x * rows_per_cta + row_in_cta) * 4 * d;
+    constexpr int NQ = BIAS_SUMS ? 4 : 2;
+    float* prow = partials + static_cast<size_t>(blockIdx.x * rows_per_cta + row_in_cta) * NQ * d;
 #pragma unroll
     for (int j = 0; j < CHUNKS; ++j) {
         const int col = 8 * (tr + j * tpr);
@@ -278,8 +282,10 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
             // two pairs = four consecutive columns
             *reinterpret_cast<ulonglong2*>(prow + 0 * d + col + 2 * k) = make_ulonglong2(acc_g[j][k], acc_g[j][k + 1]);
             *reinterpret_cast<ulonglong2*>(prow + 1 * d + col + 2 * k) = make_ulonglong2(acc_b[j][k], acc_b[j][k + 1]);
-            *reinterpret_cast<ulonglong2*>(prow + 2 * d + col + 2 * k) = make_ulonglong2(acc_r[j][k], acc_r[j][k + 1]);
-            *reinterpret_cast<ulonglong2*>(prow + 3 * d + col + 2 * k) = make_ulonglong2(acc_x[j][k], acc_x[j][k + 1]);
+            if (BIAS_SUMS) {
+                *reinterpret_cast<ulonglong2*>(prow + 2 * d + col + 2 * k) = make_ulonglong2(acc_r[j][k], acc_r[j][k + 1]);
+                *reinterpret_cast<ulonglong2*>(prow + 3 * d + col + 2 * k) = make_ulonglong2(acc_x[j][k], acc_x[j][k + 1]);
+            }
         }
     }
 }
@@ -394,9 +400,10 @@ const char* launch_layernorm_fwd(Runtime* rt, const void* x, const void* gamma, 
 
 const char* configure_elementwise()
 {
-    cudaError_t e = cudaFuncSetAttribute(ln_bwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLnBwdDepth * 3 * 1 * kRowThreadsMax * 16);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(ln_bwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLnBwdDepth * 3 * 2 * kRowThreadsMax * 16);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(ln_bwd_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLnBwdDepth * 3 * 4 * kRowThreadsMax * 16);
+    cudaError_t e = cudaSuccess;
+#define PW_LN_ATTR(C, B) if (e == cudaSuccess) e = cudaFuncSetAttribute(ln_bwd_kernel<C, B>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLnBwdDepth * 3 * C * kRowThreadsMax * 16)
+    PW_LN_ATTR(1, true); PW_LN_ATTR(1, false); PW_LN_ATTR(2, true); PW_LN_ATTR(2, false); PW_LN_ATTR(4, true); PW_LN_ATTR(4, false);
+#undef PW_LN_ATTR
     return e == cudaSuccess ? nullptr : "could not raise the shared-memory limit of the layernorm kernels";
 }
 
@@ -425,17 +432,21 @@ const char* launch_layernorm_bwd(Runtime* rt, const void* dh, const void* x, con
     auto P = static_cast<float*>(partials);
     cudaError_t le = cudaSuccess;
     const size_t ring_bytes = static_cast<size_t>(kLnBwdDepth) * 3 * rp.chunks * rp.threads * 16;
+    const bool sums = db_resid != nullptr || db_dx != nullptr;
+#define PW_LN_BWD(C, B) le = launch_k(ln_bwd_kernel<C, B>, dim3(grid), dim3(rp.threads), ring_bytes, stream, DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta)
     switch (rp.chunks) {
-        case 1: le = launch_k(ln_bwd_kernel<1>, dim3(grid), dim3(rp.threads), ring_bytes, stream, DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
-        case 2: le = launch_k(ln_bwd_kernel<2>, dim3(grid), dim3(rp.threads), ring_bytes, stream, DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
-        default: le = launch_k(ln_bwd_kernel<4>, dim3(grid), dim3(rp.threads), ring_bytes, stream, DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta); break;
+        case 1: if (sums) PW_LN_BWD(1, true); else PW_LN_BWD(1, false); break;
+        case 2: if (sums) PW_LN_BWD(2, true); else PW_LN_BWD(2, false); break;
+        default: if (sums) PW_LN_BWD(4, true); else PW_LN_BWD(4, false); break;
     }
+#undef PW_LN_BWD
     if (le != cudaSuccess) return "layernorm bwd launch failed";
     ReduceOuts outs;
     outs.out[0] = static_cast<float*>(dgamma); outs.out[1] = static_cast<float*>(dbeta);
     outs.out[2] = static_cast<float*>(db_resid); outs.out[3] = static_cast<float*>(db_dx);
-    dim3 rgrid((d + 31) / 32, 4);
-    return launch_k(reduce_partials_kernel, rgrid, dim3(1024), 0, stream, static_cast<const float*>(P), grid * rp.rows_per_cta, 4, d, outs, accumulate) == cudaSuccess
+    const int nq = sums ? 4 : 2;
+    dim3 rgrid((d + 31) / 32, nq);
+    return launch_k(reduce_partials_kernel, rgrid, dim3(1024), 0, stream, static_cast<const float*>(P), grid * rp.rows_per_cta, nq, d, outs, accumulate) == cudaSuccess
                ? nullptr : "layernorm bwd reduce launch failed";
 }
 
