@@ -245,3 +245,52 @@ def test_figure2_program_on_a_stream_and_as_a_captured_graph(pw):
     graph.replay()
     torch.cuda.synchronize()
     assert torch.equal(out0.cpu(), vals["out0"]) and torch.equal(out1.cpu(), vals["out1"])
+
+
+def test_gemm_random_shapes_all_layouts(pw, oracle64):
+    """Twelve seeded random shapes (multiples of 8 between 8 and ~1600, so tile tails in every
+    dimension, one-CTA and CTA-pair kernels, partly filled rounds) through every layout."""
+    rng = np.random.default_rng(11)
+    g = torch.Generator().manual_seed(12)
+    for case in range(12):
+        M, N, K = (int(8 * rng.integers(1, 200)) for _ in range(3))
+        layout = (pw.GEMM_TN, pw.GEMM_NN, pw.GEMM_NT)[case % 3]
+        A, Bm = bf16_randn((M, K), g), bf16_randn((K, N), g, 0.1)          # mathematical operands: C = A @ Bm
+        want = np64(A) @ np64(Bm)
+        if layout == pw.GEMM_TN:
+            a_dev, lda, b_dev, ldb = A.cuda(), K, Bm.t().contiguous().cuda(), K      # B stored [N, K]
+        elif layout == pw.GEMM_NN:
+            a_dev, lda, b_dev, ldb = A.cuda(), K, Bm.cuda(), N                        # B stored [K, N]
+        else:
+            a_dev, lda, b_dev, ldb = A.t().contiguous().cuda(), M, Bm.cuda(), N      # A stored [K, M]
+        f32 = layout == pw.GEMM_NT
+        C, check = guard_alloc((M, N), torch.float32 if f32 else torch.bfloat16)
+        pw.op_gemm(layout, pw.EPI_F32 if f32 else pw.EPI_NONE, M, N, K, a_dev, lda, b_dev, ldb, C, N)
+        torch.cuda.synchronize()
+        _status_ok(pw)
+        check()
+        assert rel_l2(C, want) < (1e-5 if f32 else ACT_TOL), (case, layout, M, N, K)
+
+
+def test_attention_random_shapes(pw, oracle64):
+    """Seeded random (B, S, H, dh): odd and even tile counts, more and fewer work items than SMs."""
+    rng = np.random.default_rng(13)
+    g = torch.Generator().manual_seed(14)
+    for case in range(5):
+        B, S, H = int(rng.integers(1, 4)), 128 * int(rng.integers(1, 6)), int(rng.integers(1, 5))
+        dh = (64, 128)[case % 2]
+        d = H * dh
+        qkv = bf16_randn((B * S, 3 * d), g)
+        dout = bf16_randn((B * S, d), g)
+        o = torch.empty((B * S, d), dtype=torch.bfloat16, device="cuda")
+        lse = torch.empty((B, H, S), device="cuda")
+        dqkv = torch.empty((B * S, 3 * d), dtype=torch.bfloat16, device="cuda")
+        delta = torch.empty((B, H, S), device="cuda")
+        pw.op_attention_fwd(qkv.cuda(), B, S, H, dh, o, lse)
+        pw.op_attention_bwd(qkv.cuda(), o, dout.cuda(), lse, B, S, H, dh, dqkv, delta)
+        torch.cuda.synchronize()
+        _status_ok(pw)
+        ow, lsew = oracle64.attn_fwd(np64(qkv), B, S, H, dh)
+        assert rel_l2(o, ow) < ACT_TOL, (case, B, S, H, dh)
+        assert np.allclose(lse.cpu().numpy(), lsew, atol=2e-3), (case, B, S, H, dh)
+        assert rel_l2(dqkv, oracle64.attn_bwd(np64(qkv), np64(dout), B, S, H, dh)) < GRAD_TOL, (case, B, S, H, dh)
