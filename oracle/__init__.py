@@ -356,6 +356,26 @@ class Oracle:
         self._fn("pwo_affine")(self._p(x), ctypes.c_long(x.size), ctypes.c_double(scale), ctypes.c_double(shift), self._p(y))
         return y
 
+    # -- gradient apply (plain SGD on a master copy; bf16 working copy) --
+    def round_bf16(self, x):
+        """x rounded to bf16 (round to nearest, ties to even), kept in the working precision."""
+        x = self._a(x)
+        f = self._fn("pwo_round_bf16")
+        f.restype = ctypes.c_float if self.suf == "f32" else ctypes.c_double
+        ctype = ctypes.c_float if self.suf == "f32" else ctypes.c_double
+        f.argtypes = [ctype]
+        return np.array([f(ctype(float(v))) for v in x.ravel()], dtype=self.dtype).reshape(x.shape)
+
+    def sgd_apply(self, master, grad, lr, grad_scale=1.0):
+        """(master - lr * grad_scale * grad, that rounded to bf16); the inputs are not modified."""
+        m = self._a(master).copy()
+        g = self._a(grad)
+        assert m.shape == g.shape
+        p = np.empty_like(m)
+        self._fn("pwo_sgd_apply")(self._p(m), self._p(g), ctypes.c_long(m.size), ctypes.c_double(lr),
+                                  ctypes.c_double(grad_scale), self._p(p))
+        return m, p
+
     def figure2_program(self, v):
         """f(v) = (b(a(v)), a(c(a(v)))) with a(x) = 2x, b(x) = x + 1, c(x) = x / 2 (Figure 2)."""
         a = lambda t: self.affine(t, 2.0, 0.0)

@@ -28,7 +28,9 @@
  * cross-entropy) are pinned by closed forms (zero table -> ln V, gradient rows summing
  * to zero), scipy's logsumexp, torch's cross_entropy + autograd in double, central
  * differences through the whole small-LM step and the initial-loss window of the
- * workload recipe; the Figure 2 program by the values the paper prints.
+ * workload recipe; the Figure 2 program by the values the paper prints; the gradient
+ * apply by a library bf16 conversion, the closed form after k equal steps, the exact
+ * minimiser of a quadratic and the first-order loss decrease of the small-LM step.
  * Nothing is "parity unpinned".
  *
  * Layout conventions (all row-major, all REAL):
@@ -488,3 +490,29 @@ void FN(pwo_affine)(const REAL* x, long n, double scale, double shift, REAL* y)
     for (long i = 0; i < n; ++i) y[i] = (REAL)((double)x[i] * scale + shift);
 }
 
+
+/* ---- Gradient apply ----
+ * In the appendix's trace of data-parallel training over two islands, each island applies
+ * the gradients it received before it starts the next step.  The paper names no optimizer,
+ * so this is plain stochastic gradient descent on a full-precision master copy of a
+ * parameter tensor, with the bf16 working copy derived from the master afterwards:
+ *     master <- master - lr * grad_scale * grad          (grad_scale: e.g. 1 / micro-batches)
+ *     param  =  master rounded to bf16 (8 significant bits, round to nearest, ties to even)
+ * The rounding is the definition written out: split x = m * 2^e with 0.5 <= |m| < 1, round
+ * m * 2^8 to the nearest integer (ties to even: the default rounding mode of nearbyint) and
+ * scale back.  Values below the bf16 normal range do not occur in this workload. */
+REAL FN(pwo_round_bf16)(REAL x)
+{
+    if (x == 0 || !isfinite((double)x)) return x;
+    int e;
+    const double m = frexp((double)x, &e);
+    return (REAL)ldexp(nearbyint(ldexp(m, 8)), e - 8);
+}
+
+void FN(pwo_sgd_apply)(REAL* master, const REAL* grad, long n, double lr, double grad_scale, REAL* param)
+{
+    for (long i = 0; i < n; ++i) {
+        master[i] = (REAL)((double)master[i] - lr * grad_scale * (double)grad[i]);
+        param[i] = FN(pwo_round_bf16)(master[i]);
+    }
+}
