@@ -164,6 +164,18 @@ def isolated_elementwise(pw, w, peaks, dev, iters=30, nbuf=6):
         ms = timeit(lambda i: pw.op_colsum(ins[i % n], out, False, sc))
         res[name] = (ms, 2.0 * T * N)
         del ins
+    # gradient apply over one layer's parameter tensors (a rotation of two sets: 14 bytes per element)
+    shapes = [(d,), (d,), (3 * d, d), (3 * d,), (d, d), (d,), (d,), (d,), (F, d), (F,), (d, F), (d,)]
+    n_el = sum(int(torch.Size(sh).numel()) for sh in shapes)
+    sets = []
+    for _ in range(2 if n_el * 10 * 2 < 40e9 else 1):
+        ps = [torch.zeros(sh, dtype=torch.bfloat16, device=dev) for sh in shapes]
+        ms_ = [torch.zeros(sh, device=dev) for sh in shapes]
+        gs = [torch.full(sh, 1e-3, device=dev) for sh in shapes]
+        sets.append(list(zip(ps, ms_, gs)))
+    ms = timeit(lambda i: pw.sgd_apply(sets[i % len(sets)], 1e-3))
+    res["sgd_apply"] = (ms, 14.0 * n_el)
+    del sets
     return {k: {"us": ms * 1e3, "gbs": b / (ms * 1e-3) / 1e9, "frac_of_measured_hbm": b / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
             for k, (ms, b) in res.items()}
 

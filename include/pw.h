@@ -354,6 +354,28 @@ pw_status_t pw_op_status(int* device_status, int* site);
  * paper's Figure 2 program (a(x) = x*2, b(x) = x+1, c(x) = x/2; f(v) = (b(a(v)), a(c(a(v))))): lets
  * that worked example run through the same enqueue-only / captured-graph dispatch as the layers. */
 pw_status_t pw_op_affine_f32(const void* x, long long n, float scale, float shift, void* y, void* stream);
+/* Gradient apply.  In the appendix's trace of data-parallel training each island applies the
+ * gradients it received before the next step; the paper names no optimizer, so this is plain
+ * stochastic gradient descent on an fp32 master copy with the bf16 working copy re-derived from it:
+ *     master[i] <- master[i] - lr * grad_scale * grad[i]     (one fused multiply-add per element)
+ *     param[i]   = bf16(master[i])                           (round to nearest even)
+ * for every element of every item.  items is a HOST array of n_items entries; every pointer in it is
+ * a DEVICE pointer owned by the caller: param bf16 [n] (read only when init_master != 0, always
+ * written), master fp32 [n] (read unless init_master != 0, always written), grad fp32 [n] (read only;
+ * e.g. a member of pw_layer_grads_t).  Items must not overlap.  init_master != 0 takes the old master
+ * from param instead (first step, or lr = 0 to only create the master copy).  grad_scale is for
+ * sums over micro-batches (1 / count).  Any alignment of the element type works; 16-byte aligned
+ * tensors take the vector path.  Enqueue-only on `stream`; one launch per 24 items.
+ * Errors: PW_ERR_INVALID_ARG for NULL / misaligned pointers, n < 0, n_items <= 0, lr < 0 or not
+ * finite, grad_scale <= 0 or not finite; n == 0 items are skipped. */
+typedef struct {
+    void* param;       /* device, bf16 [n] */
+    void* master;      /* device, fp32 [n] */
+    const void* grad;  /* device, fp32 [n] */
+    int64_t n;
+} pw_apply_item_t;
+pw_status_t pw_sgd_apply(const pw_apply_item_t* items, int n_items, float lr, float grad_scale, int init_master,
+                         void* stream);
 /* Clears the status word of the single-step calls (after a test has provoked an error). */
 pw_status_t pw_op_status_reset(void);
 /* Failure-path self-test.  Every device-side wait in this library is bounded; this call shows the

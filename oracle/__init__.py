@@ -360,11 +360,7 @@ class Oracle:
     def round_bf16(self, x):
         """x rounded to bf16 (round to nearest, ties to even), kept in the working precision."""
         x = self._a(x)
-        f = self._fn("pwo_round_bf16")
-        f.restype = ctypes.c_float if self.suf == "f32" else ctypes.c_double
-        ctype = ctypes.c_float if self.suf == "f32" else ctypes.c_double
-        f.argtypes = [ctype]
-        return np.array([f(ctype(float(v))) for v in x.ravel()], dtype=self.dtype).reshape(x.shape)
+        return self.sgd_apply(x, np.zeros_like(x), 0.0)[1]            # a step of rate zero only rounds
 
     def sgd_apply(self, master, grad, lr, grad_scale=1.0):
         """(master - lr * grad_scale * grad, that rounded to bf16); the inputs are not modified."""

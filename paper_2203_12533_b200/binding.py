@@ -40,7 +40,7 @@ EXPORTS = (
     "pw_op_attention_fwd", "pw_op_attention_bwd", "pw_op_status",
     "pw_lm_workspace_bytes", "pw_lm_step",
     "pw_op_embedding_fwd", "pw_op_embedding_bwd_scratch_bytes", "pw_op_embedding_bwd", "pw_op_softmax_xent",
-    "pw_op_status_reset", "pw_op_selftest_wait_timeout", "pw_op_affine_f32",
+    "pw_op_status_reset", "pw_op_selftest_wait_timeout", "pw_op_affine_f32", "pw_sgd_apply",
 )
 
 
@@ -55,6 +55,11 @@ class LayerConfig(ctypes.Structure):
                 ("head_dim", ctypes.c_int32), ("d_ff", ctypes.c_int32), ("seq_len", ctypes.c_int32),
                 ("batch", ctypes.c_int32), ("act", ctypes.c_int32), ("ln_eps", ctypes.c_float),
                 ("causal", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class ApplyItem(ctypes.Structure):
+    _fields_ = [("param", ctypes.c_void_p), ("master", ctypes.c_void_p), ("grad", ctypes.c_void_p),
+                ("n", ctypes.c_int64)]
 
 
 KERNEL_CLASSES = ("gemm_tn", "gemm_nn", "gemm_nt", "attn_fwd", "attn_bwd", "ln_fwd", "ln_bwd", "colsum", "xent", "embed")
@@ -139,6 +144,8 @@ def lib() -> ctypes.CDLL:
         L.pw_op_softmax_xent.argtypes = [vp, ci, vp, ci, ci, ctypes.c_float, vp, vp, vp]
         L.pw_op_selftest_wait_timeout.argtypes = [ctypes.c_uint64, ctypes.POINTER(ci), vp]
         L.pw_op_affine_f32.argtypes = [vp, ctypes.c_longlong, ctypes.c_float, ctypes.c_float, vp, vp]
+        L.pw_sgd_apply.argtypes = [ctypes.POINTER(ApplyItem), ctypes.c_int, ctypes.c_float, ctypes.c_float,
+                                   ctypes.c_int, vp]
         _lib = L
     return _lib
 
@@ -412,3 +419,14 @@ def op_selftest_wait_timeout(limit_cycles=2_000_000, stream=None) -> int:
 def op_affine_f32(x, scale, shift, y, stream=None):
     _check(lib().pw_op_affine_f32(_p(x), x.numel(), scale, shift, _p(y), _stream(stream)))
 
+
+def sgd_apply(items, lr, grad_scale=1.0, init_master=False, stream=None):
+    """items: (param bf16, master fp32, grad fp32) device tensors of equal element counts.
+    master -= lr * grad_scale * grad and param = bf16(master), in place, for every item."""
+    arr = (ApplyItem * max(len(items), 1))()
+    for i, (p, m, g) in enumerate(items):
+        assert p.numel() == m.numel() == g.numel(), "param, master and grad must have the same number of elements"
+        assert p.is_contiguous() and m.is_contiguous() and g.is_contiguous()
+        assert p.element_size() == 2 and m.element_size() == 4 and g.element_size() == 4
+        arr[i] = ApplyItem(_p(p), _p(m), _p(g), p.numel())
+    _check(lib().pw_sgd_apply(arr, len(items), lr, grad_scale, int(bool(init_master)), _stream(stream)))

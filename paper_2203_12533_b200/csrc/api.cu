@@ -7,6 +7,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <cstddef>
+#include <cmath>
 #include <map>
 #include <mutex>
 #include <new>
@@ -994,6 +995,25 @@ pw_status_t pw_op_affine_f32(const void* x, long long n, float scale, float shif
     PW_RT_OR_FAIL();
     if (!aligned(x, 4) || !aligned(y, 4)) return fail(PW_ERR_INVALID_ARG, "affine: NULL or misaligned pointer");
     PW_OP(launch_affine_f32(x, n, scale, shift, y, static_cast<cudaStream_t>(stream)));
+    return PW_OK;
+}
+
+pw_status_t pw_sgd_apply(const pw_apply_item_t* items, int n_items, float lr, float grad_scale, int init_master,
+                         void* stream)
+{
+    PW_RT_OR_FAIL();
+    if (!items || n_items <= 0) return fail(PW_ERR_INVALID_ARG, "gradient apply: no items");
+    if (!(lr >= 0.0f) || !(grad_scale > 0.0f) || !std::isfinite(lr) || !std::isfinite(grad_scale))
+        return fail(PW_ERR_INVALID_ARG, "gradient apply: lr must be finite and >= 0, grad_scale finite and > 0");
+    std::vector<ApplyItem> v(static_cast<size_t>(n_items));
+    for (int i = 0; i < n_items; ++i) {
+        const pw_apply_item_t& a = items[i];
+        if (a.n < 0) return fail(PW_ERR_INVALID_ARG, "gradient apply: negative element count");
+        if (a.n > 0 && (!aligned(a.param, 2) || !aligned(a.master, 4) || !aligned(a.grad, 4)))
+            return fail(PW_ERR_INVALID_ARG, "gradient apply: NULL or misaligned pointer");
+        v[static_cast<size_t>(i)] = ApplyItem{a.param, a.master, a.grad, static_cast<long long>(a.n)};
+    }
+    PW_OP(launch_sgd_apply(v.data(), n_items, lr * grad_scale, init_master, static_cast<cudaStream_t>(stream)));
     return PW_OK;
 }
 

@@ -77,6 +77,12 @@ const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* ou
 
 const char* launch_affine_f32(const void* x, long long n, float scale, float shift, void* y, cudaStream_t stream);
 
+// Gradient apply (optimizer.cu): master -= step * grad, param = bf16(master), for every item; with
+// init_master the old master is taken from param instead of being read.
+constexpr int kApplyMaxItems = 24;                      // tensors served by one launch
+struct ApplyItem { void* param; void* master; const void* grad; long long n; };
+const char* launch_sgd_apply(const ApplyItem* items, int n_items, float step, int init_master, cudaStream_t stream);
+
 // Bounded-wait self-test (selftest.cu): *returned (device int) becomes 1 when the wait gave up and the kernel went on.
 const char* launch_wait_selftest(DeviceStatus* status, long long limit, int* returned, cudaStream_t stream);
 
