@@ -498,14 +498,28 @@ def run_ours_lm(args, w):
     stream = torch.cuda.Stream(device=dev)
     state = {"i": 0}
 
+    apply_items = None
+    if args.apply_lr is not None:
+        flat_p = [p for ps in params for p in ps] + list(lm_params)
+        flat_g = [x for gs in grads for x in gs] + list(lm_grads)
+        flat_m = [torch.empty(p.shape, dtype=torch.float32, device=dev) for p in flat_p]
+        apply_items = list(zip(flat_p, flat_m, flat_g))
+        with torch.cuda.stream(stream):
+            pw.sgd_apply(apply_items, 0.0, init_master=True, stream=stream)      # master copies from the bf16 parameters
+    apply_launches = 0 if apply_items is None else -(-len(apply_items) // pw.APPLY_ITEMS_PER_LAUNCH)
+
     def step():
         stage.lm_step(params, grads, lm_params, lm_grads, dev_ids[0], dev_labels[0], loss, V, workspace, w.recompute, stream=stream)
+        if apply_items is not None:
+            pw.sgd_apply(apply_items, args.apply_lr, stream=stream)
 
     def step_e2e():
         k = state["i"] & 1                                   # the copies are tiny: same stream, alternating buffers
         dev_ids[k].copy_(host_ids, non_blocking=True)
         dev_labels[k].copy_(host_labels, non_blocking=True)
         stage.lm_step(params, grads, lm_params, lm_grads, dev_ids[k], dev_labels[k], loss, V, workspace, w.recompute, stream=stream)
+        if apply_items is not None:
+            pw.sgd_apply(apply_items, args.apply_lr, stream=stream)
         host_loss.copy_(loss, non_blocking=True)
         state["i"] += 1
 
@@ -536,12 +550,21 @@ def run_ours_lm(args, w):
     n0 = stage.launch_count()
     with ClockSampler(local) as clocks:
         ms_step = timed(step, args.steps) / args.steps
-    launches = stage.launch_count() - n0
+    launches = stage.launch_count() - n0 + apply_launches * args.steps
+    loss_after_timed = float(loss.item())
     stage.profile_begin()
     with torch.cuda.stream(stream):
         for _ in range(args.steps):
             step()
     prof = stage.profile_end()
+    apply_info = None
+    if apply_items is not None:
+        n_el = sum(p.numel() for p, _, _ in apply_items)
+        ms_apply = timed(lambda: pw.sgd_apply(apply_items, 0.0, stream=stream), args.steps) / args.steps   # rate 0: same traffic
+        gbs = 14.0 * n_el / (ms_apply * 1e-3) / 1e9
+        apply_info = {"lr": args.apply_lr, "optimizer": "plain SGD, fp32 master copies, bf16 working copies",
+                      "tensors": len(apply_items), "elements": n_el, "launches_per_step": apply_launches,
+                      "ms_per_step_alone": ms_apply, "gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"]}
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     ms_e2e = timed(step_e2e, e2e_steps) / e2e_steps
     if stage.status() != (0, 0):
@@ -556,7 +579,7 @@ def run_ours_lm(args, w):
                    "seq_len": w.seq_len, "batch": w.batch, "layers": L, "vocab": V, "recompute": bool(w.recompute),
                    "dispatch": "async", "parallelism": f"replicas x{world}",
                    "l2": "working set per step (logits alone are 1 GB) is far above the 126 MB L2"},
-        "loss": float(loss.item()),
+        "loss": loss_after_timed,
         "tflops_model": world * model_flops / (ms_step * 1e-3) / 1e12,
         "tflops_hw": world * hw_flops / (ms_step * 1e-3) / 1e12,
         "frac_bf16_peak_burst": hw_flops / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
@@ -567,6 +590,9 @@ def run_ours_lm(args, w):
                 "h2d_bytes_per_step": 2 * T * 4, "d2h_bytes_per_step": 4},
         "gpu_launches": int(launches),
     }
+    if apply_info is not None:
+        line["metric"] = "small-LM training step with gradient apply tokens/s"
+        line["apply"] = apply_info
     kernels, tot_ms = {}, sum(v["ms"] for v in prof.values())
     g_ms = g_flops = g_n = 0.0
     for name, v in prof.items():
@@ -642,9 +668,13 @@ def main():
     ap.add_argument("--cpu-sample-batch", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-isolated", action="store_true", help="skip the back-to-back timing of the element-wise kernels")
+    ap.add_argument("--apply-lr", type=float, default=None,
+                    help="workload 5 only: every step also applies the gradients (plain SGD, this rate) to all parameters")
     args = ap.parse_args()
     from paper_2203_12533_b200 import inputs
     w = inputs.WORKLOADS[args.workload]
+    if args.apply_lr is not None and (not w.vocab or args.impl != "ours" or args.apply_lr < 0):
+        raise SystemExit("--apply-lr needs --workload 5, --impl ours and a rate >= 0")
     if args.impl == "reference":
         (run_reference_lm if w.vocab else run_reference)(args, w)
     else:

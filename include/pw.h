@@ -365,7 +365,8 @@ pw_status_t pw_op_affine_f32(const void* x, long long n, float scale, float shif
  * e.g. a member of pw_layer_grads_t).  Items must not overlap.  init_master != 0 takes the old master
  * from param instead (first step, or lr = 0 to only create the master copy).  grad_scale is for
  * sums over micro-batches (1 / count).  Any alignment of the element type works; 16-byte aligned
- * tensors take the vector path.  Enqueue-only on `stream`; one launch per 24 items.
+ * tensors take the vector path.  Enqueue-only on `stream`; one launch per 64 items
+ * (items with n == 0 do not count).
  * Errors: PW_ERR_INVALID_ARG for NULL / misaligned pointers, n < 0, n_items <= 0, lr < 0 or not
  * finite, grad_scale <= 0 or not finite; n == 0 items are skipped. */
 typedef struct {

@@ -57,6 +57,9 @@ class LayerConfig(ctypes.Structure):
                 ("causal", ctypes.c_int32), ("flags", ctypes.c_uint32)]
 
 
+APPLY_ITEMS_PER_LAUNCH = 64      # tensors one launch of the gradient apply serves
+
+
 class ApplyItem(ctypes.Structure):
     _fields_ = [("param", ctypes.c_void_p), ("master", ctypes.c_void_p), ("grad", ctypes.c_void_p),
                 ("n", ctypes.c_int64)]

@@ -79,7 +79,7 @@ const char* launch_affine_f32(const void* x, long long n, float scale, float shi
 
 // Gradient apply (optimizer.cu): master -= step * grad, param = bf16(master), for every item; with
 // init_master the old master is taken from param instead of being read.
-constexpr int kApplyMaxItems = 24;                      // tensors served by one launch
+constexpr int kApplyMaxItems = 64;                      // tensors served by one launch
 struct ApplyItem { void* param; void* master; const void* grad; long long n; };
 const char* launch_sgd_apply(const ApplyItem* items, int n_items, float step, int init_master, cudaStream_t stream);
 

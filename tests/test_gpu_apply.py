@@ -81,7 +81,7 @@ def test_sgd_apply_unaligned_views_and_neighbours_untouched(pw, oracle32, oracle
 
 def test_sgd_apply_many_items_span_several_launches(pw, oracle32, oracle64):
     gen = torch.Generator().manual_seed(23)
-    sizes = [int(s) for s in torch.randint(0, 3 * CHUNK, (61,), generator=gen)]
+    sizes = [int(s) for s in torch.randint(0, 2 * CHUNK, (150,), generator=gen)]
     sizes[5] = 0
     masters = [torch.randn(n, generator=gen) for n in sizes]
     grads = [torch.randn(n, generator=gen) for n in sizes]
