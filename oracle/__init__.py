@@ -372,6 +372,15 @@ class Oracle:
                                   ctypes.c_double(grad_scale), self._p(p))
         return m, p
 
+    def dp_sgd_apply(self, master, grads_per_rank, lr, grad_scale=1.0):
+        """Data-parallel form of the gradient apply: every replica's gradient of the same tensor is
+        added up (in rank order) and the sum is applied once; all replicas then hold the same
+        parameters.  Returns (new master, bf16 working copy)."""
+        total = self._a(grads_per_rank[0]).copy()
+        for g in grads_per_rank[1:]:
+            total = total + self._a(g)
+        return self.sgd_apply(master, total, lr, grad_scale)
+
     def figure2_program(self, v):
         """f(v) = (b(a(v)), a(c(a(v)))) with a(x) = 2x, b(x) = x + 1, c(x) = x / 2 (Figure 2)."""
         a = lambda t: self.affine(t, 2.0, 0.0)

@@ -91,3 +91,28 @@ def test_applying_the_lm_gradients_lowers_the_loss_by_rate_times_gradient_norm(o
         drops.append(out["loss"] - o64.lm_step(D, ps2, E2, g2, b2, ids, labels)["loss"])
         assert abs(drops[-1] - lr * gnorm2) < 0.02 * lr * gnorm2, (lr, drops[-1], lr * gnorm2)
     assert drops[0] > drops[1] > 0
+
+
+def test_data_parallel_apply_is_one_step_on_the_summed_gradient(o64):
+    """Two replicas with half the batch each and grad_scale 1/2 take the step of the mean gradient;
+    one replica is the plain apply; for a loss that is a sum over examples the replicas' summed
+    gradients equal the gradient of the whole batch (checked on a least-squares problem)."""
+    rng = np.random.default_rng(8)
+    m0 = rng.standard_normal(300)
+    gs = [rng.standard_normal(300) for _ in range(4)]
+    m1, p1 = o64.dp_sgd_apply(m0, gs, 0.1, 0.25)
+    assert np.allclose(m1, m0 - 0.1 * np.mean(gs, axis=0), rtol=0, atol=1e-15)
+    assert np.array_equal(p1, o64.round_bf16(m1))
+    ma, pa = o64.dp_sgd_apply(m0, gs[:1], 0.1)
+    mb, pb = o64.sgd_apply(m0, gs[0], 0.1)
+    assert np.array_equal(ma, mb) and np.array_equal(pa, pb)
+    mr, _ = o64.dp_sgd_apply(m0, gs[::-1], 0.1, 0.25)                  # order only changes the rounding
+    assert np.allclose(mr, m1, rtol=0, atol=1e-15)
+    # least squares: loss = sum_i (a_i . w - y_i)^2 / 2 over 8 examples, split 3 + 5 over two replicas
+    A, y, w = rng.standard_normal((8, 6)), rng.standard_normal(8), rng.standard_normal(6)
+    grad = lambda rows: A[rows].T @ (A[rows] @ w - y[rows])
+    whole, _ = o64.sgd_apply(w, grad(slice(0, 8)), 0.05)
+    split, _ = o64.dp_sgd_apply(w, [grad(slice(0, 3)), grad(slice(3, 8))], 0.05)
+    assert np.allclose(whole, split, rtol=0, atol=1e-14)
+    full_loss = lambda v: 0.5 * float(((A @ v - y) ** 2).sum())
+    assert full_loss(split) < full_loss(w)
