@@ -377,6 +377,39 @@ typedef struct {
 } pw_apply_item_t;
 pw_status_t pw_sgd_apply(const pw_apply_item_t* items, int n_items, float lr, float grad_scale, int init_master,
                          void* stream);
+/* Data-parallel gradient apply over peer memory: the two-island data-parallel training of Section
+ * 5.3 and the appendix trace (each island computes gradients, the islands exchange them, each
+ * applies them), for replicas that are GPUs of one NVLink domain, one process each.  Every replica
+ * keeps ALL its parameter gradients in one flat fp32 buffer and ALL its bf16 parameters in one flat
+ * bf16 buffer (n_total elements each, same layout on every replica), both mapped into every other
+ * replica (pw_shared_*).  Replica `rank` owns elements [lo, hi) (pw_dp_slice: equal slices, a
+ * multiple of 8 elements) and holds the fp32 master of that slice only.  The call, for i in [lo, hi):
+ *     g = grads[0][i] + grads[1][i] + ... + grads[world-1][i]      (fp32, this order)
+ *     master_slice[i - lo] <- master_slice[i - lo] - lr * grad_scale * g
+ *     params[k][i] = bf16(master_slice[i - lo])  for every replica k
+ * i.e. reduce-scatter, step and all-gather of the working copy in one kernel of plain peer loads and
+ * stores (no multicast, no waiting inside the kernel).  grads / params: HOST arrays of `world` DEVICE
+ * pointers in rank order (entry `rank` is this replica's own buffer, the others are mapped peers).
+ * init_master != 0 takes the old master from this replica's own params.
+ * ORDERING IS THE CALLER'S: every replica's gradients must be complete before any replica's call
+ * starts, and no replica may read params (next forward) or rewrite grads (next backward) before
+ * every replica's call has finished - e.g. a one-element NCCL all-reduce on the same stream before
+ * and after, or host barriers after a stream synchronize.  Enqueue-only on `stream`.
+ * Errors: PW_ERR_INVALID_ARG for world outside [1, 8], a bad rank, NULL / misaligned buffers, bad
+ * lr / grad_scale.  A replica whose slice is empty launches nothing. */
+pw_status_t pw_dp_slice(int64_t n_total, int world, int rank, int64_t* lo, int64_t* hi);   /* host only, needs no GPU */
+pw_status_t pw_dp_reduce_apply(int rank, int world, const void* const* grads, void* const* params, void* master_slice,
+                               int64_t n_total, float lr, float grad_scale, int init_master, void* stream);
+/* Device buffers that other processes can map (CUDA IPC).  pw_shared_alloc: cudaMalloc of `bytes` on
+ * the current device plus a 64-byte handle to send to the other replicas (any host channel);
+ * pw_shared_open: map another process's buffer (same GPU or a peer GPU of the node; peer access is
+ * enabled on demand) - the handle's maker cannot open it itself; pw_shared_close / pw_shared_free
+ * undo them.  Close every mapping before the owner frees the buffer. */
+typedef struct { unsigned char bytes[64]; } pw_ipc_handle_t;
+pw_status_t pw_shared_alloc(size_t bytes, void** dev_ptr, pw_ipc_handle_t* handle);
+pw_status_t pw_shared_free(void* dev_ptr);
+pw_status_t pw_shared_open(const pw_ipc_handle_t* handle, void** dev_ptr);
+pw_status_t pw_shared_close(void* dev_ptr);
 /* Clears the status word of the single-step calls (after a test has provoked an error). */
 pw_status_t pw_op_status_reset(void);
 /* Failure-path self-test.  Every device-side wait in this library is bounded; this call shows the

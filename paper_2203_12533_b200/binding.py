@@ -41,6 +41,7 @@ EXPORTS = (
     "pw_lm_workspace_bytes", "pw_lm_step",
     "pw_op_embedding_fwd", "pw_op_embedding_bwd_scratch_bytes", "pw_op_embedding_bwd", "pw_op_softmax_xent",
     "pw_op_status_reset", "pw_op_selftest_wait_timeout", "pw_op_affine_f32", "pw_sgd_apply",
+    "pw_dp_slice", "pw_dp_reduce_apply", "pw_shared_alloc", "pw_shared_free", "pw_shared_open", "pw_shared_close",
 )
 
 
@@ -57,6 +58,11 @@ class LayerConfig(ctypes.Structure):
                 ("causal", ctypes.c_int32), ("flags", ctypes.c_uint32)]
 
 
+class IpcHandle(ctypes.Structure):
+    _fields_ = [("bytes", ctypes.c_ubyte * 64)]
+
+
+DP_MAX_WORLD = 8
 APPLY_ITEMS_PER_LAUNCH = 64      # tensors one launch of the gradient apply serves
 
 
@@ -147,6 +153,14 @@ def lib() -> ctypes.CDLL:
         L.pw_op_softmax_xent.argtypes = [vp, ci, vp, ci, ci, ctypes.c_float, vp, vp, vp]
         L.pw_op_selftest_wait_timeout.argtypes = [ctypes.c_uint64, ctypes.POINTER(ci), vp]
         L.pw_op_affine_f32.argtypes = [vp, ctypes.c_longlong, ctypes.c_float, ctypes.c_float, vp, vp]
+        L.pw_dp_slice.argtypes = [ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int64),
+                                  ctypes.POINTER(ctypes.c_int64)]
+        L.pw_dp_reduce_apply.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(vp), ctypes.POINTER(vp), vp, ctypes.c_int64,
+                                         ctypes.c_float, ctypes.c_float, ctypes.c_int, vp]
+        L.pw_shared_alloc.argtypes = [ctypes.c_size_t, ctypes.POINTER(vp), ctypes.POINTER(IpcHandle)]
+        L.pw_shared_free.argtypes = [vp]
+        L.pw_shared_open.argtypes = [ctypes.POINTER(IpcHandle), ctypes.POINTER(vp)]
+        L.pw_shared_close.argtypes = [vp]
         L.pw_sgd_apply.argtypes = [ctypes.POINTER(ApplyItem), ctypes.c_int, ctypes.c_float, ctypes.c_float,
                                    ctypes.c_int, vp]
         _lib = L
@@ -433,3 +447,43 @@ def sgd_apply(items, lr, grad_scale=1.0, init_master=False, stream=None):
         assert p.element_size() == 2 and m.element_size() == 4 and g.element_size() == 4
         arr[i] = ApplyItem(_p(p), _p(m), _p(g), p.numel())
     _check(lib().pw_sgd_apply(arr, len(items), lr, grad_scale, int(bool(init_master)), _stream(stream)))
+
+
+def dp_slice(n_total, world, rank):
+    """Elements [lo, hi) of the flat index space that replica `rank` owns (host arithmetic only)."""
+    lo, hi = ctypes.c_int64(), ctypes.c_int64()
+    _check(lib().pw_dp_slice(n_total, world, rank, ctypes.byref(lo), ctypes.byref(hi)))
+    return lo.value, hi.value
+
+
+def dp_reduce_apply(rank, grad_ptrs, param_ptrs, master_slice, n_total, lr, grad_scale, init_master=False, stream=None):
+    """grad_ptrs / param_ptrs: device addresses (ints) of every replica's flat buffers, in rank order."""
+    world = len(grad_ptrs)
+    assert len(param_ptrs) == world
+    g = (ctypes.c_void_p * world)(*grad_ptrs)
+    p = (ctypes.c_void_p * world)(*param_ptrs)
+    _check(lib().pw_dp_reduce_apply(rank, world, g, p, _p(master_slice), n_total, lr, grad_scale, int(bool(init_master)),
+                                    _stream(stream)))
+
+
+def shared_alloc(nbytes):
+    """(device address, 64-byte handle) of a new device buffer that other processes can map."""
+    ptr, h = ctypes.c_void_p(), IpcHandle()
+    _check(lib().pw_shared_alloc(nbytes, ctypes.byref(ptr), ctypes.byref(h)))
+    return ptr.value, bytes(h.bytes)
+
+
+def shared_free(ptr):
+    _check(lib().pw_shared_free(ptr))
+
+
+def shared_open(handle: bytes):
+    h = IpcHandle()
+    ctypes.memmove(h.bytes, handle, 64)
+    ptr = ctypes.c_void_p()
+    _check(lib().pw_shared_open(ctypes.byref(h), ctypes.byref(ptr)))
+    return ptr.value
+
+
+def shared_close(ptr):
+    _check(lib().pw_shared_close(ptr))

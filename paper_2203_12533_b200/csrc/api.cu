@@ -1017,6 +1017,99 @@ pw_status_t pw_sgd_apply(const pw_apply_item_t* items, int n_items, float lr, fl
     return PW_OK;
 }
 
+pw_status_t pw_dp_slice(int64_t n_total, int world, int rank, int64_t* lo, int64_t* hi)
+{
+    if (n_total < 0 || world < 1 || world > kDpMaxWorld || rank < 0 || rank >= world || !lo || !hi)
+        return fail(PW_ERR_INVALID_ARG, "dp slice: need n_total >= 0, 1 <= world <= 8, 0 <= rank < world, non-NULL outputs");
+    long long a, b;
+    dp_slice(static_cast<long long>(n_total), world, rank, &a, &b);
+    *lo = a; *hi = b;
+    return PW_OK;
+}
+
+pw_status_t pw_dp_reduce_apply(int rank, int world, const void* const* grads, void* const* params, void* master_slice,
+                               int64_t n_total, float lr, float grad_scale, int init_master, void* stream)
+{
+    PW_RT_OR_FAIL();
+    if (world < 1 || world > kDpMaxWorld || rank < 0 || rank >= world)
+        return fail(PW_ERR_INVALID_ARG, "data-parallel apply: need 1 <= world <= 8 and 0 <= rank < world");
+    if (!grads || !params || n_total < 0) return fail(PW_ERR_INVALID_ARG, "data-parallel apply: NULL pointer table or negative size");
+    if (!(lr >= 0.0f) || !(grad_scale > 0.0f) || !std::isfinite(lr) || !std::isfinite(grad_scale))
+        return fail(PW_ERR_INVALID_ARG, "data-parallel apply: lr must be finite and >= 0, grad_scale finite and > 0");
+    for (int k = 0; k < world; ++k)
+        if (!aligned(grads[k], 4) || !aligned(params[k], 2))
+            return fail(PW_ERR_INVALID_ARG, "data-parallel apply: NULL or misaligned replica buffer");
+    long long lo, hi;
+    dp_slice(static_cast<long long>(n_total), world, rank, &lo, &hi);
+    if (hi > lo && !aligned(master_slice, 4)) return fail(PW_ERR_INVALID_ARG, "data-parallel apply: NULL or misaligned master slice");
+    PW_OP(launch_dp_reduce_apply(rank, world, grads, params, master_slice, static_cast<long long>(n_total), lr * grad_scale,
+                                 init_master, static_cast<cudaStream_t>(stream)));
+    return PW_OK;
+}
+
+// Device buffers that other processes can map.  Allocated here with cudaMalloc (a whole allocation
+// of its own: the handle then names exactly this buffer) and opened by the other replicas with
+// lazy peer access, which covers both another process on the same GPU and a process on a peer GPU.
+namespace {
+std::mutex g_shared_mu;
+std::map<void*, int> g_shared_owned;     // pointers from pw_shared_alloc
+std::map<void*, int> g_shared_opened;    // pointers from pw_shared_open
+}  // namespace
+
+pw_status_t pw_shared_alloc(size_t bytes, void** dev_ptr, pw_ipc_handle_t* handle)
+{
+    if (!dev_ptr || !handle || bytes == 0) return fail(PW_ERR_INVALID_ARG, "shared alloc: NULL output or zero size");
+    static_assert(sizeof(cudaIpcMemHandle_t) <= sizeof(handle->bytes), "handle too small");
+    void* p = nullptr;
+    cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) return fail_cuda("shared alloc", e);
+    cudaIpcMemHandle_t h;
+    e = cudaIpcGetMemHandle(&h, p);
+    if (e != cudaSuccess) { cudaFree(p); return fail_cuda("shared alloc: export handle", e); }
+    std::memset(handle->bytes, 0, sizeof(handle->bytes));
+    std::memcpy(handle->bytes, &h, sizeof(h));
+    { std::lock_guard<std::mutex> lock(g_shared_mu); g_shared_owned[p] = 1; }
+    *dev_ptr = p;
+    return PW_OK;
+}
+
+pw_status_t pw_shared_free(void* dev_ptr)
+{
+    {
+        std::lock_guard<std::mutex> lock(g_shared_mu);
+        auto it = g_shared_owned.find(dev_ptr);
+        if (it == g_shared_owned.end()) return fail(PW_ERR_INVALID_ARG, "shared free: not a pointer from pw_shared_alloc");
+        g_shared_owned.erase(it);
+    }
+    const cudaError_t e = cudaFree(dev_ptr);
+    return e == cudaSuccess ? PW_OK : fail_cuda("shared free", e);
+}
+
+pw_status_t pw_shared_open(const pw_ipc_handle_t* handle, void** dev_ptr)
+{
+    if (!handle || !dev_ptr) return fail(PW_ERR_INVALID_ARG, "shared open: NULL argument");
+    cudaIpcMemHandle_t h;
+    std::memcpy(&h, handle->bytes, sizeof(h));
+    void* p = nullptr;
+    const cudaError_t e = cudaIpcOpenMemHandle(&p, h, cudaIpcMemLazyEnablePeerAccess);
+    if (e != cudaSuccess) return fail_cuda("shared open (a handle cannot be opened by the process that made it)", e);
+    { std::lock_guard<std::mutex> lock(g_shared_mu); g_shared_opened[p] = 1; }
+    *dev_ptr = p;
+    return PW_OK;
+}
+
+pw_status_t pw_shared_close(void* dev_ptr)
+{
+    {
+        std::lock_guard<std::mutex> lock(g_shared_mu);
+        auto it = g_shared_opened.find(dev_ptr);
+        if (it == g_shared_opened.end()) return fail(PW_ERR_INVALID_ARG, "shared close: not a pointer from pw_shared_open");
+        g_shared_opened.erase(it);
+    }
+    const cudaError_t e = cudaIpcCloseMemHandle(dev_ptr);
+    return e == cudaSuccess ? PW_OK : fail_cuda("shared close", e);
+}
+
 pw_status_t pw_op_selftest_wait_timeout(uint64_t limit_cycles, int* kernel_returned, void* stream)
 {
     PW_RT_OR_FAIL();

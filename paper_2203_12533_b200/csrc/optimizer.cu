@@ -103,7 +103,126 @@ sgd_apply_kernel(const __grid_constant__ ApplyTable tab, float step)
     }
 }
 
+// Data-parallel form over peer memory.  Every replica (one process per GPU) has the gradients and
+// the bf16 parameters of all tensors in one flat buffer each, mapped into every other replica's
+// address space.  Replica `rank` owns the elements [lo, hi) of the flat index space and keeps the
+// fp32 master of that slice only.  For its slice this kernel
+//     reads the gradient of every replica (plain loads from peer memory, rank order 0..world-1:
+//     the sum has one fixed order), applies the step to its master slice, and
+//     stores the new bf16 values into every replica's parameter buffer (plain stores to peers),
+// i.e. reduce-scatter, optimizer step and all-gather of the working copy in one pass: 4 bytes per
+// element come in over the links and 2 go out, instead of the 8 + 8 of an fp32 all-reduce followed
+// by a local apply.  The kernel waits on nothing: the caller orders it after every replica's
+// backward pass and orders the next forward pass after every replica's kernel (stream-ordered or
+// host barriers), so a missing peer can delay the host but never spin a GPU.
+struct DpTable {
+    const float* grad[kDpMaxWorld];
+    __nv_bfloat16* param[kDpMaxWorld];
+};
+
+__device__ __forceinline__ void add8(float (&acc)[8], const float4& a, const float4& b)
+{
+    acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
+    acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
+}
+
+template <bool INIT>
+__global__ void __launch_bounds__(kApplyThreads)
+dp_reduce_apply_kernel(const __grid_constant__ DpTable tab, int world, int rank, float* master, long long lo,
+                       long long hi, float step, int vec)
+{
+    grid_dep_launch();
+    const long long i = lo + (static_cast<long long>(blockIdx.x) * kApplyThreads + threadIdx.x) * 8;
+    grid_dep_wait();
+    if (i >= hi) return;
+    if (vec && i + 8 <= hi) {
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int k0 = 0; k0 < world; k0 += 4) {                       // four replicas' loads in flight at a time
+            float4 g[4][2];
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (k0 + q < world) {
+                    const float4* src = reinterpret_cast<const float4*>(tab.grad[k0 + q] + i);
+                    g[q][0] = __ldcv(src);                             // peers rewrite these every step: never from L1
+                    g[q][1] = __ldcv(src + 1);
+                }
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (k0 + q < world) add8(acc, g[q][0], g[q][1]);
+        }
+        float m[8];
+        if (INIT) {
+            const uint4 w = *reinterpret_cast<const uint4*>(tab.param[rank] + i);
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                m[2 * q] = __uint_as_float(ww[q] << 16);
+                m[2 * q + 1] = __uint_as_float(ww[q] & 0xffff0000u);
+            }
+        } else {
+            const float4 a = __ldcs(reinterpret_cast<const float4*>(master + (i - lo)));
+            const float4 b = __ldcs(reinterpret_cast<const float4*>(master + (i - lo)) + 1);
+            m[0] = a.x; m[1] = a.y; m[2] = a.z; m[3] = a.w; m[4] = b.x; m[5] = b.y; m[6] = b.z; m[7] = b.w;
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) m[e] = fmaf(-step, acc[e], m[e]);
+        __stcs(reinterpret_cast<float4*>(master + (i - lo)), make_float4(m[0], m[1], m[2], m[3]));
+        __stcs(reinterpret_cast<float4*>(master + (i - lo)) + 1, make_float4(m[4], m[5], m[6], m[7]));
+        uint4 o;
+        o.x = pack_bf16x2(m[0], m[1]); o.y = pack_bf16x2(m[2], m[3]);
+        o.z = pack_bf16x2(m[4], m[5]); o.w = pack_bf16x2(m[6], m[7]);
+        for (int k = 0; k < world; ++k) *reinterpret_cast<uint4*>(tab.param[k] + i) = o;
+        return;
+    }
+    const long long end = (i + 8 < hi) ? i + 8 : hi;
+    for (long long j = i; j < end; ++j) {
+        float g = 0.f;
+        for (int k = 0; k < world; ++k) g += *reinterpret_cast<const volatile float*>(tab.grad[k] + j);
+        const float m0 = INIT ? __bfloat162float(tab.param[rank][j]) : master[j - lo];
+        const float m1 = fmaf(-step, g, m0);
+        master[j - lo] = m1;
+        const __nv_bfloat16 w = __float2bfloat16_rn(m1);
+        for (int k = 0; k < world; ++k) tab.param[k][j] = w;
+    }
+}
+
 }  // namespace
+
+void dp_slice(long long n_total, int world, int rank, long long* lo, long long* hi)
+{
+    long long per = (n_total + world - 1) / world;
+    per = (per + 7) / 8 * 8;                                          // slices start on 16-byte boundaries of the bf16 buffer
+    long long a = per * rank, b = a + per;
+    if (a > n_total) a = n_total;
+    if (b > n_total) b = n_total;
+    *lo = a; *hi = b;
+}
+
+const char* launch_dp_reduce_apply(int rank, int world, const void* const* grads, void* const* params, void* master,
+                                   long long n_total, float step, int init_master, cudaStream_t stream)
+{
+    if (world < 1 || world > kDpMaxWorld || rank < 0 || rank >= world) return "data-parallel apply: bad rank or world size";
+    DpTable tab;
+    uintptr_t bits = reinterpret_cast<uintptr_t>(master);
+    for (int k = 0; k < kDpMaxWorld; ++k) {
+        tab.grad[k] = k < world ? static_cast<const float*>(grads[k]) : nullptr;
+        tab.param[k] = k < world ? static_cast<__nv_bfloat16*>(params[k]) : nullptr;
+        if (k < world) bits |= reinterpret_cast<uintptr_t>(grads[k]) | reinterpret_cast<uintptr_t>(params[k]);
+    }
+    long long lo, hi;
+    dp_slice(n_total, world, rank, &lo, &hi);
+    if (hi <= lo) return nullptr;                                     // this replica owns nothing
+    const long long per_block = static_cast<long long>(kApplyThreads) * 8;
+    const long long blocks = (hi - lo + per_block - 1) / per_block;
+    if (blocks > 0x7fffffffll) return "data-parallel apply: too many elements for one call";
+    const int vec = (bits & 15) == 0;
+    const cudaError_t e = init_master
+        ? launch_k(dp_reduce_apply_kernel<true>, dim3(static_cast<unsigned>(blocks)), dim3(kApplyThreads), 0, stream, tab, world, rank,
+                   static_cast<float*>(master), lo, hi, step, vec)
+        : launch_k(dp_reduce_apply_kernel<false>, dim3(static_cast<unsigned>(blocks)), dim3(kApplyThreads), 0, stream, tab, world, rank,
+                   static_cast<float*>(master), lo, hi, step, vec);
+    return e == cudaSuccess ? nullptr : "data-parallel apply launch failed";
+}
 
 const char* launch_sgd_apply(const ApplyItem* items, int n_items, float step, int init_master, cudaStream_t stream)
 {

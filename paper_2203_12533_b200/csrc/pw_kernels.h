@@ -83,6 +83,14 @@ constexpr int kApplyMaxItems = 64;                      // tensors served by one
 struct ApplyItem { void* param; void* master; const void* grad; long long n; };
 const char* launch_sgd_apply(const ApplyItem* items, int n_items, float step, int init_master, cudaStream_t stream);
 
+// Data-parallel gradient apply over peer memory (optimizer.cu).  grads / params: host arrays of `world`
+// device pointers (flat fp32 gradient and bf16 parameter buffers of every replica, n_total elements
+// each); master: this replica's fp32 slice [lo, hi) as given by dp_slice.
+constexpr int kDpMaxWorld = 8;
+void dp_slice(long long n_total, int world, int rank, long long* lo, long long* hi);
+const char* launch_dp_reduce_apply(int rank, int world, const void* const* grads, void* const* params, void* master,
+                                   long long n_total, float step, int init_master, cudaStream_t stream);
+
 // Bounded-wait self-test (selftest.cu): *returned (device int) becomes 1 when the wait gave up and the kernel went on.
 const char* launch_wait_selftest(DeviceStatus* status, long long limit, int* returned, cudaStream_t stream);
 

@@ -61,3 +61,85 @@ def test_reference_arm_under_torchrun_prints_one_line_from_rank_0():
     d = json.loads(lines[0])
     assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["value"] > 0
     assert d["cpu_baseline"]["kind"] == "oracle" and d["e2e"]["h2d_bytes_per_step"] == 0
+
+
+class _FakeLibrary:
+    """Stands in for the CUDA library in the host-logic test of the data-parallel replica: buffers
+    are numbers, handles name their owner, and every call is recorded."""
+
+    def __init__(self, rank):
+        self.rank, self.calls, self.next = rank, [], 1000 * (rank + 1)
+
+    def shared_alloc(self, nbytes):
+        self.next += 1
+        self.calls.append(("alloc", nbytes))
+        return self.next, f"{self.rank}:{self.next}".encode().ljust(64, b"\0")
+
+    def shared_free(self, ptr): self.calls.append(("free", ptr))
+
+    def shared_open(self, handle):
+        owner, ptr = handle.rstrip(b"\0").decode().split(":")
+        assert int(owner) != self.rank, "a replica must not open its own handle"
+        self.calls.append(("open", int(owner), int(ptr)))
+        return 100000 * (int(owner) + 1) + int(ptr)
+
+    def shared_close(self, ptr): self.calls.append(("close", ptr))
+
+    def dp_slice(self, n, world, rank):
+        per = -(-(-(-n // world)) // 8) * 8
+        return min(per * rank, n), min(per * rank + per, n)
+
+    def dp_reduce_apply(self, rank, gp, pp, master, n, lr, scale, init_master=False, stream=None):
+        self.calls.append(("apply", rank, tuple(gp), tuple(pp), n, lr, scale, init_master))
+
+    def tensor_at(self, ptr, numel, dtype, device): return torch.zeros(numel, dtype=dtype)
+
+    def empty_master(self, numel, device): return torch.zeros(max(numel, 1))
+
+    def synchronize(self, device, stream=None): self.calls.append(("sync",))
+
+
+def _replica_main(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    from paper_2203_12533_b200 import data_parallel
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+    fake = _FakeLibrary(rank)
+    rep = data_parallel.Replica([(3, 5), (7,), (16,)], torch.device("cpu"), library=fake)
+    rep.reduce_apply(0.5, init_master=True)
+    rep.reduce_apply(0.25, grad_scale=1.0)
+    info = {"offsets": rep.offsets, "total": rep.total, "slice": (rep.lo, rep.hi), "grad_ptrs": rep.grad_ptrs,
+            "param_ptrs": rep.param_ptrs, "shapes": [tuple(t.shape) for t in rep.params]}
+    rep.close()
+    info["calls"] = fake.calls
+    out[rank] = info
+    dist.destroy_process_group()
+
+
+def test_replica_host_logic_with_two_gloo_ranks():
+    """Arena layout, slice ownership, handle exchange in rank order, default gradient scale, and the
+    close-before-free order, with the CUDA library replaced by a recorder."""
+    world, port = 2, _free_port()
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_replica_main, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    for r in range(world):
+        info = res[r]
+        assert info["offsets"] == [0, 16, 24] and info["total"] == 40          # 15 -> 16, 7 -> 8, 16
+        assert info["shapes"] == [(3, 5), (7,), (16,)]
+        own_g, own_p = 1000 * (r + 1) + 1, 1000 * (r + 1) + 2
+        other = 1 - r
+        peer_g, peer_p = 100000 * (other + 1) + 1000 * (other + 1) + 1, 100000 * (other + 1) + 1000 * (other + 1) + 2
+        want_g = [own_g, peer_g] if r == 0 else [peer_g, own_g]
+        want_p = [own_p, peer_p] if r == 0 else [peer_p, own_p]
+        assert info["grad_ptrs"] == want_g and info["param_ptrs"] == want_p      # rank order, own buffer at own rank
+        applies = [c for c in info["calls"] if c[0] == "apply"]
+        assert applies[0] == ("apply", r, tuple(want_g), tuple(want_p), 40, 0.5, 0.5, True)    # scale defaults to 1 / world
+        assert applies[1] == ("apply", r, tuple(want_g), tuple(want_p), 40, 0.25, 1.0, False)
+        names = [c[0] for c in info["calls"]]
+        assert names.count("open") == 2 and names.count("close") == 2 and names.count("free") == 2
+        assert max(i for i, n in enumerate(names) if n == "close") < min(i for i, n in enumerate(names) if n == "free")
+        # a host synchronise before each barrier around each apply (gloo backend: host ordering)
+        first_apply = names.index("apply")
+        assert "sync" in names[:first_apply] and "sync" in names[first_apply + 1:]
+    assert res[0]["slice"] == (0, 24) and res[1]["slice"] == (24, 40)
