@@ -485,12 +485,28 @@ def run_ours_lm(args, w):
     dev = torch.device("cuda", local)
     L, T, d, V = w.n_layers, w.tokens, w.d_model, w.vocab
     stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
-    params = [[p.to(dev) for p in inputs.layer_params(w, args.seed, l)] for l in range(L)]
-    grads = [[torch.zeros(p.shape, dtype=torch.float32, device=dev) for p in ps] for ps in params]
     E, g, b, ids, labels = inputs.lm_inputs(w, args.seed)
+    cpu_params = [inputs.layer_params(w, args.seed, l) for l in range(L)]
+    replica = None
+    if args.data_parallel:
+        # every parameter and every gradient lives in the replica's two flat, peer-mapped buffers
+        from paper_2203_12533_b200 import data_parallel
+        flat_cpu = [p for ps in cpu_params for p in ps] + [E, g, b]
+        replica = data_parallel.Replica([tuple(p.shape) for p in flat_cpu], dev)
+        for dst, src in zip(replica.params, flat_cpu):
+            dst.copy_(src)
+        per = len(cpu_params[0])
+        params = [replica.params[l * per:(l + 1) * per] for l in range(L)]
+        grads = [replica.grads[l * per:(l + 1) * per] for l in range(L)]
+        lm_params, lm_grads = tuple(replica.params[L * per:]), tuple(replica.grads[L * per:])
+        if world > 1:                                        # each replica trains on its own batch
+            _, _, _, ids, labels = inputs.lm_inputs(w, args.seed + 1000 * rank)
+    else:
+        params = [[p.to(dev) for p in ps] for ps in cpu_params]
+        grads = [[torch.zeros(p.shape, dtype=torch.float32, device=dev) for p in ps] for ps in params]
+        lm_params = (E.to(dev), g.to(dev), b.to(dev))
+        lm_grads = (torch.zeros(E.shape, dtype=torch.float32, device=dev), torch.zeros(d, device=dev), torch.zeros(d, device=dev))
     host_ids, host_labels = ids.pin_memory(), labels.pin_memory()
-    lm_params = (E.to(dev), g.to(dev), b.to(dev))
-    lm_grads = (torch.zeros(E.shape, dtype=torch.float32, device=dev), torch.zeros(d, device=dev), torch.zeros(d, device=dev))
     dev_ids, dev_labels = [host_ids.to(dev), host_ids.to(dev)], [host_labels.to(dev), host_labels.to(dev)]
     loss = torch.zeros(1, device=dev)
     host_loss = torch.zeros(1).pin_memory()
@@ -499,7 +515,10 @@ def run_ours_lm(args, w):
     state = {"i": 0}
 
     apply_items = None
-    if args.apply_lr is not None:
+    if replica is not None:
+        with torch.cuda.stream(stream):
+            replica.reduce_apply(0.0, init_master=True, stream=stream)           # master slices from the bf16 parameters
+    elif args.apply_lr is not None:
         flat_p = [p for ps in params for p in ps] + list(lm_params)
         flat_g = [x for gs in grads for x in gs] + list(lm_grads)
         flat_m = [torch.empty(p.shape, dtype=torch.float32, device=dev) for p in flat_p]
@@ -507,19 +526,25 @@ def run_ours_lm(args, w):
         with torch.cuda.stream(stream):
             pw.sgd_apply(apply_items, 0.0, init_master=True, stream=stream)      # master copies from the bf16 parameters
     apply_launches = 0 if apply_items is None else -(-len(apply_items) // pw.APPLY_ITEMS_PER_LAUNCH)
+    if replica is not None:
+        apply_launches = 1
+
+    def apply(lr):
+        if replica is not None:
+            replica.reduce_apply(lr, stream=stream)
+        elif apply_items is not None:
+            pw.sgd_apply(apply_items, lr, stream=stream)
 
     def step():
         stage.lm_step(params, grads, lm_params, lm_grads, dev_ids[0], dev_labels[0], loss, V, workspace, w.recompute, stream=stream)
-        if apply_items is not None:
-            pw.sgd_apply(apply_items, args.apply_lr, stream=stream)
+        apply(args.apply_lr)
 
     def step_e2e():
         k = state["i"] & 1                                   # the copies are tiny: same stream, alternating buffers
         dev_ids[k].copy_(host_ids, non_blocking=True)
         dev_labels[k].copy_(host_labels, non_blocking=True)
         stage.lm_step(params, grads, lm_params, lm_grads, dev_ids[k], dev_labels[k], loss, V, workspace, w.recompute, stream=stream)
-        if apply_items is not None:
-            pw.sgd_apply(apply_items, args.apply_lr, stream=stream)
+        apply(args.apply_lr)
         host_loss.copy_(loss, non_blocking=True)
         state["i"] += 1
 
@@ -558,13 +583,21 @@ def run_ours_lm(args, w):
             step()
     prof = stage.profile_end()
     apply_info = None
-    if apply_items is not None:
-        n_el = sum(p.numel() for p, _, _ in apply_items)
-        ms_apply = timed(lambda: pw.sgd_apply(apply_items, 0.0, stream=stream), args.steps) / args.steps   # rate 0: same traffic
-        gbs = 14.0 * n_el / (ms_apply * 1e-3) / 1e9
+    if apply_items is not None or replica is not None:
+        n_el = replica.total if replica is not None else sum(p.numel() for p, _, _ in apply_items)
+        ms_apply = timed(lambda: apply(0.0), args.steps) / args.steps            # rate 0: same traffic
         apply_info = {"lr": args.apply_lr, "optimizer": "plain SGD, fp32 master copies, bf16 working copies",
-                      "tensors": len(apply_items), "elements": n_el, "launches_per_step": apply_launches,
-                      "ms_per_step_alone": ms_apply, "gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"]}
+                      "tensors": len(replica.shapes) if replica is not None else len(apply_items), "elements": n_el,
+                      "launches_per_step": apply_launches, "ms_per_step_alone": ms_apply}
+        if replica is None or world == 1:
+            gbs = 14.0 * n_el / (ms_apply * 1e-3) / 1e9     # grad 4 + master 4 + 4 + bf16 copy 2 bytes per element, all local
+            apply_info.update({"gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"]})
+        else:
+            # per replica: 4 bytes per element of its slice from each peer come in, 2 bytes per element go out to each peer
+            link_in = 4.0 * (n_el / world) * (world - 1)
+            apply_info.update({"mode": "data parallel: fused reduce-scatter + step + all-gather over peer memory",
+                               "link_bytes_in_per_replica": link_in, "link_gbs_in": link_in / (ms_apply * 1e-3) / 1e9,
+                               "frac_of_measured_peer_copy_770": link_in / (ms_apply * 1e-3) / 1e9 / 770.0})
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     ms_e2e = timed(step_e2e, e2e_steps) / e2e_steps
     if stage.status() != (0, 0):
@@ -577,7 +610,9 @@ def run_ours_lm(args, w):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "d_model": d, "heads": f"{w.n_heads}x{w.head_dim}", "d_ff": w.d_ff,
                    "seq_len": w.seq_len, "batch": w.batch, "layers": L, "vocab": V, "recompute": bool(w.recompute),
-                   "dispatch": "async", "parallelism": f"replicas x{world}",
+                   "dispatch": "async",
+                   "parallelism": (f"data parallel x{world} (gradients summed and applied through peer memory)"
+                                   if args.data_parallel else f"replicas x{world}"),
                    "l2": "working set per step (logits alone are 1 GB) is far above the 126 MB L2"},
         "loss": loss_after_timed,
         "tflops_model": world * model_flops / (ms_step * 1e-3) / 1e12,
@@ -627,6 +662,8 @@ def run_ours_lm(args, w):
                                 "seconds": dt, "sample": f"1 of {w.batch} sequences (S={w.seq_len}) through 1 of {L} layers and the full-vocabulary head, fwd+bwd, fp32 plain-loop C oracle, run once"}
     if rank == 0:
         print(json.dumps(line), flush=True)
+    if replica is not None:
+        replica.close()
     if world > 1:
         dist.destroy_process_group()
 
@@ -668,6 +705,9 @@ def main():
     ap.add_argument("--cpu-sample-batch", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-isolated", action="store_true", help="skip the back-to-back timing of the element-wise kernels")
+    ap.add_argument("--data-parallel", action="store_true",
+                    help="with --apply-lr: the ranks are data-parallel replicas; gradients are summed and applied through peer "
+                         "memory by the fused kernel (each rank draws its own token batch)")
     ap.add_argument("--apply-lr", type=float, default=None,
                     help="workload 5 only: every step also applies the gradients (plain SGD, this rate) to all parameters")
     args = ap.parse_args()
@@ -675,6 +715,8 @@ def main():
     w = inputs.WORKLOADS[args.workload]
     if args.apply_lr is not None and (not w.vocab or args.impl != "ours" or args.apply_lr < 0):
         raise SystemExit("--apply-lr needs --workload 5, --impl ours and a rate >= 0")
+    if args.data_parallel and args.apply_lr is None:
+        raise SystemExit("--data-parallel needs --apply-lr")
     if args.impl == "reference":
         (run_reference_lm if w.vocab else run_reference)(args, w)
     else:

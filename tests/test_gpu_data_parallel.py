@@ -149,3 +149,56 @@ def test_two_processes_map_each_others_buffers(pw, oracle64, tmp_path):
         master = want_m
     got_m = np.concatenate([res[r]["master"][:res[r]["hi"] - res[r]["lo"]].numpy() for r in range(world)])
     assert np.all(np.abs(got_m - master) <= 1e-6 * (np.abs(master) + 1.0))
+
+
+def test_lm_training_through_a_replica_matches_separate_tensors(pw):
+    """The small language model trained for three steps with all parameters and gradients in a
+    replica's flat buffers (one replica: its own gradients only) gives the same losses and the same
+    parameters, bit for bit, as with separate tensors and the plain apply."""
+    from paper_2203_12533_b200 import data_parallel, inputs
+    w = inputs.Workload("lm_small", 256, 4, 64, 1024, 128, 2, n_layers=2, vocab=512)
+    L, lr, steps = w.n_layers, 0.1, 3
+    cpu_params = [inputs.layer_params(w, 0, l, random_ln=True) for l in range(L)]
+    E0, g0, b0, ids, labels = inputs.lm_inputs(w, 0, random_ln=True)
+    ids, labels = ids.cuda(), labels.cuda()
+    stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
+    ws = torch.empty(stage.lm_workspace_bytes(w.vocab, False), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+
+    def run(params, grads, ends, end_grads, apply):
+        loss, losses = torch.zeros(1, device="cuda"), []
+        with torch.cuda.stream(stream):
+            for s in range(steps):
+                stage.lm_step(params, grads, tuple(ends), end_grads, ids, labels, loss, w.vocab, ws, False, stream=stream)
+                losses.append(loss.clone())
+                apply(s)
+        torch.cuda.synchronize()
+        assert stage.status() == (0, 0)
+        return [x.item() for x in losses]
+
+    # separate tensors
+    params = [[p.cuda() for p in ps] for ps in cpu_params]
+    ends = [E0.cuda(), g0.cuda(), b0.cuda()]
+    grads = [[torch.zeros(p.shape, device="cuda") for p in ps] for ps in params]
+    end_grads = [torch.zeros(t.shape, device="cuda") for t in ends]
+    flat_p = [p for ps in params for p in ps] + ends
+    flat_g = [x for gs in grads for x in gs] + end_grads
+    flat_m = [torch.empty(p.shape, device="cuda") for p in flat_p]
+    a = run(params, grads, ends, end_grads,
+            lambda s: pw.sgd_apply(list(zip(flat_p, flat_m, flat_g)), lr, init_master=(s == 0), stream=stream))
+
+    # one replica's flat buffers
+    flat_cpu = [p for ps in cpu_params for p in ps] + [E0, g0, b0]
+    rep = data_parallel.Replica([tuple(p.shape) for p in flat_cpu], torch.device("cuda", 0))
+    try:
+        for dst, src in zip(rep.params, flat_cpu):
+            dst.copy_(src)
+        per = len(cpu_params[0])
+        b = run([rep.params[l * per:(l + 1) * per] for l in range(L)], [rep.grads[l * per:(l + 1) * per] for l in range(L)],
+                rep.params[L * per:], rep.grads[L * per:],
+                lambda s: rep.reduce_apply(lr, init_master=(s == 0), stream=stream))
+        assert a == b and a[-1] < a[0]
+        for x, y in zip(flat_p, rep.params):
+            assert torch.equal(x, y)
+    finally:
+        rep.close()
