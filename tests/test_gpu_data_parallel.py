@@ -202,3 +202,48 @@ def test_lm_training_through_a_replica_matches_separate_tensors(pw):
             assert torch.equal(x, y)
     finally:
         rep.close()
+
+
+def test_two_pipeline_stages_in_two_processes_match_one_chain(pw, tmp_path):
+    """Two stage processes (two layers each, three micro-batches, GPipe) whose last kernels store
+    straight into the neighbour's mapped buffers, against the same four layers run as one chain in
+    this process: outputs, input gradients and every parameter gradient agree bit for bit."""
+    from paper_2203_12533_b200 import inputs
+    from tests import pp_worker
+    world, port = 2, _free_port()
+    procs = [subprocess.Popen([sys.executable, os.path.join(ROOT, "tests", "pp_worker.py"), str(r), str(world), str(port), str(tmp_path)],
+                              cwd=ROOT, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True) for r in range(world)]
+    outs = []
+    for p in procs:
+        try:
+            outs.append(p.communicate(timeout=240)[0])
+        except subprocess.TimeoutExpired:
+            for q in procs:
+                q.kill()
+            raise
+    assert all(p.returncode == 0 for p in procs), "\n".join(o[-1500:] for o in outs)
+    res = [torch.load(os.path.join(tmp_path, f"stage{r}.pt")) for r in range(world)]
+    assert all(r["status"] == (0, 0) for r in res)
+    M = pp_worker.MICRO
+    assert res[0]["signals"] == [("send", 1)] * M + [("recv", 1)] * M
+    assert res[1]["signals"] == [("recv", 0)] * M + [("send", 0)] * M
+
+    w = pp_worker.workload()
+    L = w.n_layers
+    stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
+    params = [[p.cuda() for p in inputs.layer_params(w, 0, l, random_ln=True)] for l in range(L)]
+    grads = [[torch.zeros(p.shape, dtype=torch.float32, device="cuda") for p in ps] for ps in params]
+    mbs = [inputs.microbatch(w, 0, m) for m in range(M)]
+    xs, dys = [x.cuda() for x, _ in mbs], [dy.cuda() for _, dy in mbs]
+    ys, dxs = [torch.empty_like(x) for x in xs], [torch.empty_like(x) for x in xs]
+    ws = torch.empty(stage.workspace_bytes(M, pw.SCHEDULE_GPIPE, False), dtype=torch.uint8, device="cuda")
+    stage.run_chain(params, grads, xs, dys, ys, dxs, ws, schedule=pw.SCHEDULE_GPIPE, recompute=False)
+    torch.cuda.synchronize()
+    assert stage.status() == (0, 0)
+    for m in range(M):
+        assert torch.equal(res[1]["y"][m], ys[m].view(-1, w.d_model).cpu())
+        assert torch.equal(res[0]["dx"][m], dxs[m].view(-1, w.d_model).cpu())
+    per = pp_worker.LAYERS_PER_STAGE
+    for l in range(L):
+        for got, want in zip(res[l // per]["grads"][l % per], grads[l]):
+            assert torch.equal(got, want.cpu())

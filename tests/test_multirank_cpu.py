@@ -143,3 +143,66 @@ def test_replica_host_logic_with_two_gloo_ranks():
         first_apply = names.index("apply")
         assert "sync" in names[:first_apply] and "sync" in names[first_apply + 1:]
     assert res[0]["slice"] == (0, 24) and res[1]["slice"] == (24, 40)
+
+
+class _FakeLayer:
+    T, d, ctx_bytes, scratch_bytes = 4, 8, 16, 16
+
+    def __init__(self): self.calls = []
+
+    def fwd(self, params, x, y, ctx, scratch, stream=None):
+        self.calls.append(("fwd", params, y if isinstance(y, int) else "local"))
+
+    def bwd(self, params, x, dy, dx, grads, accumulate, ctx, scratch, stream=None):
+        self.calls.append(("bwd", params, dx if isinstance(dx, int) else "local", bool(accumulate)))
+
+
+def _stage_main(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    from paper_2203_12533_b200 import pipeline_parallel
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+    fake, layer = _FakeLibrary(rank), _FakeLayer()
+    st = pipeline_parallel.PipelineStage(layer, 2, 3, torch.device("cpu"), library=fake)
+    st.run(["p0", "p1"], ["g0", "g1"], stream="s")
+    out[rank] = {"signals": st.signals, "calls": layer.calls, "lib": fake.calls, "first": st.is_first, "last": st.is_last,
+                 "y_ptrs": st._y_ptrs, "dx_ptrs": st._dx_ptrs,
+                 "own_y": [t.data_ptr() for t in st.y_out] if st.is_last else None,
+                 "own_dx": [t.data_ptr() for t in st.dx_out] if st.is_first else None}
+    st.close()
+    dist.destroy_process_group()
+
+
+def test_pipeline_stage_host_logic_with_three_gloo_ranks():
+    """Three stages, two layers each, three micro-batches: GPipe order of the layer calls, the last
+    kernel of a stage writes into the neighbour's mapped buffer, gradients accumulate from the
+    second micro-batch on, and the send / receive pattern cannot deadlock (it completes)."""
+    world, port = 3, _free_port()
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_stage_main, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    M = 3
+    assert res[0]["signals"] == [("send", 1)] * M + [("recv", 1)] * M
+    assert res[1]["signals"] == [("recv", 0), ("send", 2)] * M + [("recv", 2), ("send", 0)] * M
+    assert res[2]["signals"] == [("recv", 1)] * M + [("send", 1)] * M
+    act_bytes = _FakeLayer.T * _FakeLayer.d * 2
+    for r in range(world):
+        calls = res[r]["calls"]
+        fw, bw = [c for c in calls if c[0] == "fwd"], [c for c in calls if c[0] == "bwd"]
+        assert calls == fw + bw and len(fw) == 2 * M and len(bw) == 2 * M          # all forwards first
+        assert [c[1] for c in fw] == ["p0", "p1"] * M and [c[1] for c in bw] == ["p1", "p0"] * M
+        assert [c[3] for c in bw] == [False, False] + [True] * 4                    # overwrite, then accumulate
+        opens = [c for c in res[r]["lib"] if c[0] == "open"]
+        if r < world - 1:                                                           # y of the last layer: next stage's x_in
+            base = 100000 * (r + 2) + 1000 * (r + 2) + 1
+            assert res[r]["y_ptrs"] == [base + m * act_bytes for m in range(M)]
+            assert [c[2] for c in fw[1::2]] == res[r]["y_ptrs"] and ("open", r + 1, 1000 * (r + 2) + 1) in opens
+        else:
+            assert [c[2] for c in fw[1::2]] == res[r]["own_y"] and all(c[2] == "local" for c in fw[0::2])
+        if r > 0:                                                                   # dx of the first layer: previous stage's dy_in
+            base = 100000 * r + 1000 * r + 2
+            assert res[r]["dx_ptrs"] == [base + m * act_bytes for m in range(M)]
+            assert [c[2] for c in bw[1::2]] == res[r]["dx_ptrs"] and ("open", r - 1, 1000 * r + 2) in opens
+        else:
+            assert [c[2] for c in bw[1::2]] == res[r]["own_dx"] and all(c[2] == "local" for c in bw[0::2])
+        assert len(opens) == (1 if r in (0, world - 1) else 2)
