@@ -254,7 +254,8 @@ def run_ours(args, w):
     dispatch = {"opbyop": pw.DISPATCH_OPBYOP, "async": pw.DISPATCH_ASYNC, "graph": pw.DISPATCH_GRAPH}[args.dispatch]
     schedule = pw.SCHEDULE_GPIPE
 
-    stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
+    stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch,
+                     flags=pw.FLAG_LEAN_CTX if args.lean else 0)
     params = [[p.to(dev) for p in inputs.layer_params(w, args.seed, l)] for l in range(L)]
     grads = [[torch.zeros(p.shape, dtype=torch.float32, device=dev) for p in ps] for ps in params]
     host_x, host_dy = [], []
@@ -384,7 +385,8 @@ def run_ours(args, w):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "d_model": w.d_model, "heads": f"{w.n_heads}x{w.head_dim}", "d_ff": w.d_ff,
                    "seq_len": w.seq_len, "microbatch": w.batch, "layers": L, "microbatches": M,
-                   "recompute": bool(w.recompute), "dispatch": args.dispatch, "parallelism": f"replicas x{world}",
+                   "recompute": bool(w.recompute), "lean_ctx": bool(args.lean), "workspace_bytes": int(ws_bytes),
+                   "dispatch": args.dispatch, "parallelism": f"replicas x{world}",
                    "l2": "working set per step (activations + weights + fp32 grads) is > 1 GB, far above the 126 MB L2"},
         "tflops_model": world * model_flops / (ms_step * 1e-3) / 1e12,
         "tflops_hw": world * hw_flops / (ms_step * 1e-3) / 1e12,
@@ -484,7 +486,8 @@ def run_ours_lm(args, w):
     peaks = load_peaks()
     dev = torch.device("cuda", local)
     L, T, d, V = w.n_layers, w.tokens, w.d_model, w.vocab
-    stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
+    stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch,
+                     flags=pw.FLAG_LEAN_CTX if args.lean else 0)
     E, g, b, ids, labels = inputs.lm_inputs(w, args.seed)
     cpu_params = [inputs.layer_params(w, args.seed, l) for l in range(L)]
     replica = None
@@ -610,6 +613,7 @@ def run_ours_lm(args, w):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "d_model": d, "heads": f"{w.n_heads}x{w.head_dim}", "d_ff": w.d_ff,
                    "seq_len": w.seq_len, "batch": w.batch, "layers": L, "vocab": V, "recompute": bool(w.recompute),
+                   "lean_ctx": bool(args.lean), "workspace_bytes": int(workspace.numel()),
                    "dispatch": "async",
                    "parallelism": (f"data parallel x{world} (gradients summed and applied through peer memory)"
                                    if args.data_parallel else f"replicas x{world}"),
@@ -705,6 +709,8 @@ def main():
     ap.add_argument("--cpu-sample-batch", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-isolated", action="store_true", help="skip the back-to-back timing of the element-wise kernels")
+    ap.add_argument("--lean", action="store_true",
+                    help="lean save set: the forward keeps neither LayerNorm output nor GeLU(u); the backward re-derives them")
     ap.add_argument("--data-parallel", action="store_true",
                     help="with --apply-lr: the ranks are data-parallel replicas; gradients are summed and applied through peer "
                          "memory by the fused kernel (each rank draws its own token batch)")

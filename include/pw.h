@@ -65,6 +65,13 @@ typedef enum pw_status {
 } pw_status_t;
 
 enum { PW_ACT_GELU_ERF = 0, PW_ACT_GELU_TANH = 1 };
+/* Layer flags.  PW_FLAG_LEAN_CTX: the forward does not keep the two LayerNorm outputs (h1, h2) nor
+ * GeLU(u) in ctx - 2 T d + T F of the 7 T d + 2 T F bf16 elements a full ctx holds (40 % at
+ * F = 4 d).  The backward re-derives them into scratch (two LayerNorm forwards from x and x1 with
+ * the same bits as the first time, and GeLU of the bf16 pre-activations u, which may differ from
+ * the forward's GeLU of the fp32 pre-activations in the last bf16 bit).  pw_layer_ctx_offset reports
+ * size 0 for the three tensors; pw_layer_fwd then needs `scratch` even when ctx is given. */
+enum { PW_FLAG_LEAN_CTX = 1u };
 
 /* Static shape of a layer call - fixed for the life of the handle, like the static shapes of
  * a compiled function (Section 3).  Supported: head_dim in {64, 128}; n_heads*head_dim ==
@@ -81,7 +88,7 @@ typedef struct pw_layer_config {
     int32_t act;    /* PW_ACT_GELU_ERF (default) or PW_ACT_GELU_TANH */
     float ln_eps;   /* 0 means 1e-5 */
     int32_t causal; /* must be 1 */
-    uint32_t flags; /* reserved, 0 */
+    uint32_t flags; /* 0, or PW_FLAG_LEAN_CTX */
 } pw_layer_config_t;
 
 /* The 12 parameters of a layer (bf16 device pointers). */
@@ -147,6 +154,7 @@ pw_status_t pw_layer_ctx_offset(const pw_layer_t* layer, int which, size_t* offs
 
 /* y = layer(x).  x, y: bf16 [B,S,d] device, y must not alias x.  ctx: receives the saved
  * activations; NULL means "save nothing" (the intermediates then live in scratch only).
+ * scratch may be NULL only if ctx is given and the layer is not PW_FLAG_LEAN_CTX.
  * `params` is a host struct of device pointers.  Enqueue only. */
 pw_status_t pw_layer_fwd(pw_layer_t* layer, const pw_layer_params_t* params, const void* x, void* y,
                          void* ctx, void* scratch, void* stream);
@@ -179,7 +187,8 @@ enum {
     PW_K_COLSUM = 7,    /* main kernel + partial reduction    */
     PW_K_XENT = 8,      /* softmax / cross-entropy + loss mean (pw_lm_step)          */
     PW_K_EMBED = 9,     /* embedding lookup and its scatter-add backward (pw_lm_step) */
-    PW_K_COUNT = 10
+    PW_K_GELU = 10,     /* GeLU(u) re-derived in the backward of a PW_FLAG_LEAN_CTX layer */
+    PW_K_COUNT = 11
 };
 typedef struct pw_profile {
     uint64_t launches[PW_K_COUNT]; /* kernel launches per class since profile_begin      */

@@ -20,6 +20,7 @@ PW_OK = 0
 STATUS_NAMES = {0: "PW_OK", 1: "PW_ERR_INVALID_ARG", 2: "PW_ERR_UNSUPPORTED_SHAPE", 3: "PW_ERR_WORKSPACE_TOO_SMALL",
                 4: "PW_ERR_CUDA", 5: "PW_ERR_DEVICE_UNSUPPORTED", 6: "PW_ERR_TIMEOUT", 7: "PW_ERR_INTERNAL"}
 ACT_GELU_ERF, ACT_GELU_TANH = 0, 1
+FLAG_LEAN_CTX = 1
 GEMM_TN, GEMM_NN, GEMM_NT = 0, 1, 2
 EPI_NONE, EPI_BIAS, EPI_BIAS_RESID, EPI_BIAS_GELU, EPI_DGELU, EPI_F32 = range(6)
 DISPATCH_OPBYOP, DISPATCH_ASYNC, DISPATCH_GRAPH = 0, 1, 2
@@ -71,12 +72,13 @@ class ApplyItem(ctypes.Structure):
                 ("n", ctypes.c_int64)]
 
 
-KERNEL_CLASSES = ("gemm_tn", "gemm_nn", "gemm_nt", "attn_fwd", "attn_bwd", "ln_fwd", "ln_bwd", "colsum", "xent", "embed")
+KERNEL_CLASSES = ("gemm_tn", "gemm_nn", "gemm_nt", "attn_fwd", "attn_bwd", "ln_fwd", "ln_bwd", "colsum", "xent", "embed",
+                  "gelu")
 
 
 class Profile(ctypes.Structure):
-    _fields_ = [("launches", ctypes.c_uint64 * 10), ("ms", ctypes.c_double * 10), ("flops", ctypes.c_double * 10),
-                ("bytes", ctypes.c_double * 10)]
+    _fields_ = [("launches", ctypes.c_uint64 * 11), ("ms", ctypes.c_double * 11), ("flops", ctypes.c_double * 11),
+                ("bytes", ctypes.c_double * 11)]
 
     def as_dict(self):
         return {n: dict(launches=int(self.launches[i]), ms=float(self.ms[i]), flops=float(self.flops[i]),
@@ -203,8 +205,8 @@ def make_config(d_model, n_heads, head_dim, d_ff, seq_len, batch, act=ACT_GELU_E
 class Layer:
     """One pre-LN causal decoder layer with static shapes (pw_layer_*)."""
 
-    def __init__(self, d_model, n_heads, head_dim, d_ff, seq_len, batch, act=ACT_GELU_ERF, ln_eps=1e-5, causal=1):
-        self.cfg = make_config(d_model, n_heads, head_dim, d_ff, seq_len, batch, act, ln_eps, causal)
+    def __init__(self, d_model, n_heads, head_dim, d_ff, seq_len, batch, act=ACT_GELU_ERF, ln_eps=1e-5, causal=1, flags=0):
+        self.cfg = make_config(d_model, n_heads, head_dim, d_ff, seq_len, batch, act, ln_eps, causal, flags)
         self._h = ctypes.c_void_p()
         _check(lib().pw_layer_create(ctypes.byref(self.cfg), ctypes.byref(self._h)))
         a, b = ctypes.c_size_t(), ctypes.c_size_t()
@@ -229,6 +231,8 @@ class Layer:
         i = CTX_NAMES.index(name)
         off, nb = ctypes.c_size_t(), ctypes.c_size_t()
         _check(lib().pw_layer_ctx_offset(self._h, i, ctypes.byref(off), ctypes.byref(nb)))
+        if nb.value == 0:
+            raise KeyError(f"{name} is not kept in this layer's ctx (lean save set)")
         raw = ctx.view(torch.uint8)[off.value:off.value + nb.value]
         T, d, F = self.T, self.d, self.F
         if name in ("h1", "o", "x1", "h2"):
@@ -272,8 +276,8 @@ class Layer:
 class Stage:
     """A stack of identical-shape layers run over M micro-batches (pw_stage_*)."""
 
-    def __init__(self, n_layers, d_model, n_heads, head_dim, d_ff, seq_len, batch, act=ACT_GELU_ERF, ln_eps=1e-5):
-        self.cfg = make_config(d_model, n_heads, head_dim, d_ff, seq_len, batch, act, ln_eps)
+    def __init__(self, n_layers, d_model, n_heads, head_dim, d_ff, seq_len, batch, act=ACT_GELU_ERF, ln_eps=1e-5, flags=0):
+        self.cfg = make_config(d_model, n_heads, head_dim, d_ff, seq_len, batch, act, ln_eps, 1, flags)
         self.n_layers = n_layers
         self._h = ctypes.c_void_p()
         _check(lib().pw_stage_create(ctypes.byref(self.cfg), n_layers, ctypes.byref(self._h)))

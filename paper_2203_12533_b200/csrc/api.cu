@@ -73,6 +73,9 @@ struct LayerPlan {
     size_t ctx_off[PW_CTX_COUNT], ctx_size[PW_CTX_COUNT], ctx_bytes;
     // scratch = [ctx-shaped region used when the caller passes ctx == NULL] [backward temporaries]
     size_t off_big, off_td0, off_td1, off_delta, off_partials, off_partials2, scratch_bytes;
+    // lean ctx: h1, h2, a (and the statistics the re-derivation writes again) live in scratch
+    bool lean;
+    size_t off_lean_h1, off_lean_h2, off_lean_a, off_lean_stats;
 };
 
 }  // namespace pw
@@ -112,7 +115,7 @@ static pw_status_t validate_cfg(const pw_layer_config_t* c)
         return fail(PW_ERR_INVALID_ARG, "config has a non-positive dimension");
     if (c->act != PW_ACT_GELU_ERF && c->act != PW_ACT_GELU_TANH) return fail(PW_ERR_INVALID_ARG, "unknown activation");
     if (c->causal != 1) return fail(PW_ERR_UNSUPPORTED_SHAPE, "only causal attention is supported");
-    if (c->flags != 0) return fail(PW_ERR_INVALID_ARG, "flags must be 0");
+    if ((c->flags & ~static_cast<uint32_t>(PW_FLAG_LEAN_CTX)) != 0) return fail(PW_ERR_INVALID_ARG, "unknown flag");
     if (c->ln_eps < 0.f) return fail(PW_ERR_INVALID_ARG, "ln_eps must be >= 0");
     if (c->head_dim != 64 && c->head_dim != 128) return fail(PW_ERR_UNSUPPORTED_SHAPE, "head_dim must be 64 or 128");
     if (static_cast<long long>(c->n_heads) * c->head_dim != c->d_model)
@@ -131,8 +134,10 @@ static void build_plan(const pw_layer_config_t& c, Runtime* rt, LayerPlan* p)
     p->d = c.d_model; p->H = c.n_heads; p->dh = c.head_dim; p->F = c.d_ff;
     p->eps = c.ln_eps > 0.f ? c.ln_eps : 1e-5f;
     const size_t T = p->T, d = p->d, F = p->F;
-    const size_t sz[PW_CTX_COUNT] = {T * d * 2, T * 3 * d * 2, T * d * 2, T * d * 2, T * d * 2, T * F * 2, T * F * 2,
-                                     static_cast<size_t>(p->B) * p->H * p->S * 4, T * 4, T * 4, T * 4, T * 4};
+    p->lean = (c.flags & PW_FLAG_LEAN_CTX) != 0;
+    size_t sz[PW_CTX_COUNT] = {T * d * 2, T * 3 * d * 2, T * d * 2, T * d * 2, T * d * 2, T * F * 2, T * F * 2,
+                               static_cast<size_t>(p->B) * p->H * p->S * 4, T * 4, T * 4, T * 4, T * 4};
+    if (p->lean) sz[PW_CTX_H1] = sz[PW_CTX_H2] = sz[PW_CTX_A] = 0;
     size_t off = 0;
     for (int i = 0; i < PW_CTX_COUNT; ++i) { p->ctx_off[i] = off; p->ctx_size[i] = sz[i]; off += align256(sz[i]); }
     p->ctx_bytes = off;
@@ -147,6 +152,13 @@ static void build_plan(const pw_layer_config_t& c, Runtime* rt, LayerPlan* p)
     if (c2 > part) part = c2;
     p->off_partials = s; s += align256(part);
     p->off_partials2 = s; s += align256(c1 > c2 ? c1 : c2);   // column sums on the side stream
+    p->off_lean_h1 = p->off_lean_h2 = p->off_lean_a = p->off_lean_stats = 0;
+    if (p->lean) {
+        p->off_lean_h1 = s; s += align256(T * d * 2);
+        p->off_lean_h2 = s; s += align256(T * d * 2);
+        p->off_lean_a = s; s += align256(T * F * 2);
+        p->off_lean_stats = s; s += 2 * align256(T * 4);
+    }
     p->scratch_bytes = s;
 }
 
@@ -250,14 +262,16 @@ static pw_status_t do_attn_bwd(pw_layer_t* L, const void* qkv, const void* o, co
 // Forward into `ctx` (a ctx-shaped region).  with_fc2 = false stops after FC1/GeLU (all that a
 // recomputing backward needs).
 static pw_status_t enqueue_fwd(pw_layer_t* L, const pw_layer_params_t* P, const void* x, void* y, void* ctx,
-                               bool with_fc2, cudaStream_t st)
+                               void* scratch, bool with_fc2, cudaStream_t st)
 {
     const LayerPlan& p = L->plan;
     const int T = p.T, d = p.d, F = p.F, act = p.cfg.act;
-    void* h1 = at(ctx, p.ctx_off[PW_CTX_H1]);   void* qkv = at(ctx, p.ctx_off[PW_CTX_QKV]);
+    void* h1 = p.lean ? at(scratch, p.off_lean_h1) : at(ctx, p.ctx_off[PW_CTX_H1]);
+    void* h2 = p.lean ? at(scratch, p.off_lean_h2) : at(ctx, p.ctx_off[PW_CTX_H2]);
+    void* a = p.lean ? at(scratch, p.off_lean_a) : at(ctx, p.ctx_off[PW_CTX_A]);
+    void* qkv = at(ctx, p.ctx_off[PW_CTX_QKV]);
     void* o = at(ctx, p.ctx_off[PW_CTX_O]);     void* x1 = at(ctx, p.ctx_off[PW_CTX_X1]);
-    void* h2 = at(ctx, p.ctx_off[PW_CTX_H2]);   void* u = at(ctx, p.ctx_off[PW_CTX_U]);
-    void* a = at(ctx, p.ctx_off[PW_CTX_A]);     void* lse = at(ctx, p.ctx_off[PW_CTX_LSE]);
+    void* u = at(ctx, p.ctx_off[PW_CTX_U]);     void* lse = at(ctx, p.ctx_off[PW_CTX_LSE]);
     void* mu1 = at(ctx, p.ctx_off[PW_CTX_MU1]); void* r1 = at(ctx, p.ctx_off[PW_CTX_R1]);
     void* mu2 = at(ctx, p.ctx_off[PW_CTX_MU2]); void* r2 = at(ctx, p.ctx_off[PW_CTX_R2]);
 
@@ -282,15 +296,19 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
 {
     const LayerPlan& p = L->plan;
     const int T = p.T, d = p.d, F = p.F, act = p.cfg.act;
+    bool rederive = p.lean;                              // h1, h2, a are not in a lean ctx
     if (ctx == nullptr) {
-        pw_status_t s = enqueue_fwd(L, P, x, nullptr, scratch, false, st);
+        pw_status_t s = enqueue_fwd(L, P, x, nullptr, scratch, scratch, false, st);
         if (s != PW_OK) return s;
         ctx = scratch;
+        rederive = false;                                // the forward that just ran left them in scratch
     }
-    const void* h1 = at(ctx, p.ctx_off[PW_CTX_H1]);   const void* qkv = at(ctx, p.ctx_off[PW_CTX_QKV]);
+    const void* h1 = p.lean ? at(scratch, p.off_lean_h1) : at(ctx, p.ctx_off[PW_CTX_H1]);
+    const void* h2 = p.lean ? at(scratch, p.off_lean_h2) : at(ctx, p.ctx_off[PW_CTX_H2]);
+    const void* a = p.lean ? at(scratch, p.off_lean_a) : at(ctx, p.ctx_off[PW_CTX_A]);
+    const void* qkv = at(ctx, p.ctx_off[PW_CTX_QKV]);
     const void* o = at(ctx, p.ctx_off[PW_CTX_O]);     const void* x1 = at(ctx, p.ctx_off[PW_CTX_X1]);
-    const void* h2 = at(ctx, p.ctx_off[PW_CTX_H2]);   const void* u = at(ctx, p.ctx_off[PW_CTX_U]);
-    const void* a = at(ctx, p.ctx_off[PW_CTX_A]);     const void* lse = at(ctx, p.ctx_off[PW_CTX_LSE]);
+    const void* u = at(ctx, p.ctx_off[PW_CTX_U]);     const void* lse = at(ctx, p.ctx_off[PW_CTX_LSE]);
     const void* mu1 = at(ctx, p.ctx_off[PW_CTX_MU1]); const void* r1 = at(ctx, p.ctx_off[PW_CTX_R1]);
     const void* mu2 = at(ctx, p.ctx_off[PW_CTX_MU2]); const void* r2 = at(ctx, p.ctx_off[PW_CTX_R2]);
     void* big = at(scratch, p.off_big);        // du [T,F], later dqkv [T,3d]
@@ -315,6 +333,16 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
         return e == cudaSuccess ? PW_OK : fail_cuda("stream ordering", e);
     };
     PW_DO(order(L->ev[0], st, ax));                      // side stream starts after everything already enqueued
+    // Lean ctx: the three operands of the weight-gradient GEMMs that were not kept are made again on
+    // the side stream, each just before the GEMM that reads it.  The statistics the LayerNorm kernel
+    // writes once more go to scratch (the ctx is read-only here).
+    void* lean_st1 = p.lean ? at(scratch, p.off_lean_stats) : nullptr;
+    void* lean_st2 = p.lean ? at(scratch, p.off_lean_stats + align256(static_cast<size_t>(T) * 4)) : nullptr;
+    if (rederive) {
+        LaunchScope sc(L, PW_K_GELU, 1, 0.0, 4.0 * T * F, ax);
+        const char* e = launch_gelu_fwd(L->rt, u, const_cast<void*>(a), static_cast<long long>(T) * F, act, ax);
+        if (e) return fail(PW_ERR_CUDA, e);
+    }
     // y = x1 + a W2^T + b2  ->  du = (dy W2) * gelu'(u),  dW2 = dy^T a
     PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, d, F, T, dy, d, a, F, G->w_fc2, F, nullptr, nullptr, 0,
                                      nullptr, accumulate), ax));
@@ -322,6 +350,7 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
                                      nullptr, 0), st));
     PW_DO(order(L->ev[1], st, ax));                      // du ready
     // u = h2 W1^T + b1  ->  dh2 = du W1,  dW1 = du^T h2,  db1 = colsum(du)
+    if (rederive) PW_DO(do_ln_fwd(L, x1, P->ln2_gamma, P->ln2_beta, const_cast<void*>(h2), lean_st1, lean_st2, ax));
     PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, F, d, T, big, F, h2, d, G->w_fc1, d, nullptr, nullptr, 0,
                                      nullptr, accumulate), ax));
     PW_DO(do_colsum(L, big, F, G->b_fc1, accumulate, part2, ax));
@@ -348,6 +377,7 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
     PW_DO(do_attn_bwd(L, qkv, o, td0, lse, big, delta, st));
     PW_DO(order(L->ev[4], st, ax));                      // dqkv ready
     // qkv = h1 Wqkv^T + bqkv  ->  dh1 = dqkv Wqkv,  dWqkv = dqkv^T h1,  dbqkv = colsum(dqkv)
+    if (rederive) PW_DO(do_ln_fwd(L, x, P->ln1_gamma, P->ln1_beta, const_cast<void*>(h1), lean_st1, lean_st2, ax));
     PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, 3 * d, d, T, big, 3 * d, h1, d, G->w_qkv, d, nullptr, nullptr,
                                      0, nullptr, accumulate), ax));
     PW_DO(do_colsum(L, big, 3 * d, G->b_qkv, accumulate, part2, ax));
@@ -474,7 +504,8 @@ pw_status_t pw_layer_fwd(pw_layer_t* layer, const pw_layer_params_t* params, con
     if (x == y) return fail(PW_ERR_INVALID_ARG, "y must not alias x");
     if (ctx == nullptr && !aligned(scratch, 256)) return fail(PW_ERR_INVALID_ARG, "scratch must be 256-byte aligned when ctx is NULL");
     if (ctx != nullptr && !aligned(ctx, 256)) return fail(PW_ERR_INVALID_ARG, "ctx must be 256-byte aligned");
-    return enqueue_fwd(layer, params, x, y, ctx ? ctx : scratch, true, static_cast<cudaStream_t>(stream));
+    if (layer->plan.lean && !aligned(scratch, 256)) return fail(PW_ERR_INVALID_ARG, "a lean-ctx layer needs a 256-byte aligned scratch in fwd");
+    return enqueue_fwd(layer, params, x, y, ctx ? ctx : scratch, scratch, true, static_cast<cudaStream_t>(stream));
 }
 
 pw_status_t pw_layer_bwd(pw_layer_t* layer, const pw_layer_params_t* params, const void* x, const void* dy, void* dx,
@@ -625,7 +656,7 @@ pw_status_t enqueue_chain(pw_stage_t* stage, const pw_layer_params_t* params, co
             const void* in = l == 0 ? x_mb[m] : act(m, l);
             void* out = l == L - 1 ? y_mb[m] : act(m, l + 1);
             void* c = ctxp(m, l);
-            pw_status_t s = enqueue_fwd(Lh, &params[l], in, out, c ? c : scratch, true, st);
+            pw_status_t s = enqueue_fwd(Lh, &params[l], in, out, c ? c : scratch, scratch, true, st);
             if (s != PW_OK) return s;
             if ((s = sync()) != PW_OK) return s;
         }
@@ -828,7 +859,7 @@ pw_status_t pw_lm_step(pw_stage_t* stage, const pw_layer_params_t* params, const
     }
     for (int l = 0; l < L; ++l) {
         void* c = ctxp(l);
-        PW_DO(enqueue_fwd(Lh, &params[l], l == 0 ? x0 : actp(l - 1), actp(l), c ? c : scratch, true, st));
+        PW_DO(enqueue_fwd(Lh, &params[l], l == 0 ? x0 : actp(l - 1), actp(l), c ? c : scratch, scratch, true, st));
     }
     const void* hL = L > 0 ? actp(L - 1) : x0;
     PW_DO(do_ln_fwd(Lh, hL, lm->lnf_gamma, lm->lnf_beta, hf, mu, r, st));

@@ -132,6 +132,39 @@ affine_f32_kernel(const float* x, long long n, float scale, float shift, float* 
     if (i < n) y[i] = fmaf(x[i], scale, shift);
 }
 
+// a = GeLU(u) on bf16 tensors: the backward pass of a layer that did not keep `a` re-derives it from
+// the pre-activations it did keep.  8 elements per thread and iteration; 4 bytes per element.
+__device__ __forceinline__ uint4 gelu8(const uint4& w, int act)
+{
+    const uint32_t in[4] = {w.x, w.y, w.z, w.w};
+    uint32_t out[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        float lo = __uint_as_float(in[q] << 16), hi = __uint_as_float(in[q] & 0xffff0000u);
+        gelu2(lo, hi, act);
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out[q]) : "f"(hi), "f"(lo));
+    }
+    return make_uint4(out[0], out[1], out[2], out[3]);
+}
+
+__global__ void __launch_bounds__(256)
+gelu_fwd_kernel(const __nv_bfloat16* u, __nv_bfloat16* a, long long n8, int act)
+{
+    grid_dep_launch();
+    grid_dep_wait();
+    const long long stride = static_cast<long long>(gridDim.x) * 256;
+    long long i = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
+    for (; i + 3 * stride < n8; i += 4 * stride) {                    // four loads in flight per thread
+        uint4 w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) w[j] = __ldcs(reinterpret_cast<const uint4*>(u + (i + j * stride) * 8));
+#pragma unroll
+        for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(a + (i + j * stride) * 8) = gelu8(w[j], act);
+    }
+    for (; i < n8; i += stride)
+        *reinterpret_cast<uint4*>(a + i * 8) = gelu8(*reinterpret_cast<const uint4*>(u + i * 8), act);
+}
+
 // W warps per row and CH pieces per lane for a row of d elements (d a multiple of 256).
 bool plan_warp_rows(int d, int* W, int* CH)
 {
@@ -460,6 +493,18 @@ const char* launch_affine_f32(const void* x, long long n, float scale, float shi
     return launch_k(affine_f32_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, stream, static_cast<const float*>(x), n,
                     scale, shift, static_cast<float*>(y)) == cudaSuccess
                ? nullptr : "affine launch failed";
+}
+
+const char* launch_gelu_fwd(Runtime* rt, const void* u, void* a, long long n, int act, cudaStream_t stream)
+{
+    if (n <= 0 || (n % 8) != 0) return "gelu: element count must be a positive multiple of 8";
+    const long long n8 = n / 8;
+    long long blocks = (n8 + 255) / 256;
+    const long long cap = static_cast<long long>(rt->sm_count) * 16;
+    if (blocks > cap) blocks = cap;
+    return launch_k(gelu_fwd_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, stream, static_cast<const __nv_bfloat16*>(u),
+                    static_cast<__nv_bfloat16*>(a), n8, act) == cudaSuccess
+               ? nullptr : "gelu launch failed";
 }
 
 size_t colsum_scratch_bytes(Runtime* rt, int T, int N)

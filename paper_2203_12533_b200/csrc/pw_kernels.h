@@ -75,6 +75,9 @@ const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, voi
 size_t colsum_noalloc_max_columns();
 const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* out, int accumulate, cudaStream_t stream);
 
+// a = GeLU(u), bf16 -> bf16, n a multiple of 8.
+const char* launch_gelu_fwd(Runtime* rt, const void* u, void* a, long long n, int act, cudaStream_t stream);
+
 const char* launch_affine_f32(const void* x, long long n, float scale, float shift, void* y, cudaStream_t stream);
 
 // Gradient apply (optimizer.cu): master -= step * grad, param = bf16(master), for every item; with
