@@ -706,7 +706,7 @@ def main():
     ap.add_argument("--dispatch", default="async", choices=["opbyop", "async", "graph"])
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=30)
-    ap.add_argument("--cpu-sample-batch", type=int, default=2)
+    ap.add_argument("--cpu-sample-batch", type=int, default=6, help="sequences of the workload the timed oracle run processes (about 13 s of host time on workload 2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-isolated", action="store_true", help="skip the back-to-back timing of the element-wise kernels")
     ap.add_argument("--lean", action="store_true",
