@@ -400,8 +400,8 @@ void FN(pwo_layer_bwd)(long B, long S, long d, long H, long dh, long F, int act,
     free(gw); free(gb); free(gb2);
 }
 
-/* ---- First and last layer of the language model (Section 5.3: "an embedding layer first and a
- * softmax layer last").  The paper gives no formula; these are the textbook ones, with the
+/* ---- First and last layer of the language model (Section 5.3 names an embedding layer first and a
+ * softmax layer last).  The paper gives no formula; these are the textbook ones, with the
  * output projection tied to the embedding table (reading listed in the design notes). ---- */
 
 /* Embedding lookup: x0[t][:] = E[ids[t]][:]. */
