@@ -11,7 +11,7 @@ import pytest
 import torch
 
 from tests import dp_worker
-from tests.gpu_util import np64
+from tests.gpu_util import np64, rel_l2
 
 pytestmark = pytest.mark.gpu
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -247,3 +247,56 @@ def test_two_pipeline_stages_in_two_processes_match_one_chain(pw, tmp_path):
     for l in range(L):
         for got, want in zip(res[l // per]["grads"][l % per], grads[l]):
             assert torch.equal(got, want.cpu())
+
+
+def test_two_replicas_train_like_one_process_on_the_whole_batch(pw, tmp_path):
+    """Two replicas (two sequences each, own tokens, gradients averaged through the mapped buffers)
+    against one process that runs all four sequences as one batch with the plain apply: the mean of
+    the replica losses follows the whole-batch loss step by step and the parameters end up together
+    (different batch shapes round differently, so this is a tolerance check, not a bitwise one)."""
+    from tests import dp_lm_worker as wk
+    world, port = 2, _free_port()
+    procs = [subprocess.Popen([sys.executable, os.path.join(ROOT, "tests", "dp_lm_worker.py"), str(r), str(world), str(port), str(tmp_path)],
+                              cwd=ROOT, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True) for r in range(world)]
+    outs = []
+    for p in procs:
+        try:
+            outs.append(p.communicate(timeout=240)[0])
+        except subprocess.TimeoutExpired:
+            for q in procs:
+                q.kill()
+            raise
+    assert all(p.returncode == 0 for p in procs), "\n".join(o[-1500:] for o in outs)
+    res = [torch.load(os.path.join(tmp_path, f"lm_rank{r}.pt")) for r in range(world)]
+    assert all(r["status"] == (0, 0) for r in res)
+    for a, b in zip(res[0]["params"], res[1]["params"]):
+        assert torch.equal(a, b)                                      # replicas stay identical
+
+    w = wk.workload(world * wk.SEQS_PER_REPLICA)
+    L = w.n_layers
+    layers, ends = wk.initial_parameters()
+    params = [[p.cuda() for p in ps] for ps in layers]
+    ends = [t.cuda() for t in ends]
+    toks = [wk.replica_tokens(r) for r in range(world)]
+    ids = torch.cat([t[0] for t in toks]).cuda()
+    labels = torch.cat([t[1] for t in toks]).cuda()
+    grads = [[torch.zeros(p.shape, device="cuda") for p in ps] for ps in params]
+    end_grads = [torch.zeros(t.shape, device="cuda") for t in ends]
+    flat_p = [p for ps in params for p in ps] + ends
+    flat_g = [x for gs in grads for x in gs] + end_grads
+    flat_m = [torch.empty(p.shape, device="cuda") for p in flat_p]
+    stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
+    ws = torch.empty(stage.lm_workspace_bytes(w.vocab, False), dtype=torch.uint8, device="cuda")
+    loss, whole = torch.zeros(1, device="cuda"), []
+    for s in range(wk.STEPS):
+        stage.lm_step(params, grads, tuple(ends), end_grads, ids, labels, loss, w.vocab, ws, False)
+        whole.append(loss.item())
+        pw.sgd_apply(list(zip(flat_p, flat_m, flat_g)), wk.LR, init_master=(s == 0))
+    torch.cuda.synchronize()
+    assert stage.status() == (0, 0)
+    for s in range(wk.STEPS):
+        mean = 0.5 * (res[0]["losses"][s] + res[1]["losses"][s])
+        assert abs(mean - whole[s]) < 2e-3 * whole[s], (s, res[0]["losses"], res[1]["losses"], whole)
+    assert whole[-1] < whole[0]
+    for got, want in zip(res[0]["params"], flat_p):
+        assert rel_l2(got.cuda(), np64(want)) < 1e-2
