@@ -56,7 +56,7 @@ __device__ __forceinline__ uint64_t splat2(float v) { return pack_f32x2(v, v); }
 // lane's loads are issued at once, the statistics need only warp shuffles (plus one shared-memory
 // hop when W > 1).  256-thread CTAs hold 8/W rows.
 template <int CH>
-__global__ void __launch_bounds__(kRowThreadsMax)
+__global__ void __launch_bounds__(kRowThreadsMax, 3)
 ln_fwd_kernel(const __nv_bfloat16* x, const __nv_bfloat16* gamma,
               const __nv_bfloat16* beta, int T, int d, float eps, __nv_bfloat16* h,
               float* mu, float* rstd, int W)
