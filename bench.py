@@ -34,7 +34,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram bytes read+written per GEMM launch (average over the 12 GEMM launches of a workload-2 step),
 # from the ncu capture summarised in profiles/gemm_pair_kernel_cfg2_dram_traffic.md; None for
 # workloads without a capture.
-GEMM_DRAM_TRAFFIC_PER_LAUNCH = {"cfg2_d2048_s1024_b8": 222.5e6}
+GEMM_DRAM_TRAFFIC_PER_LAUNCH = {"cfg2_d2048_s1024_b8": 220.7e6}
 
 
 def load_peaks():
