@@ -281,8 +281,15 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
         if (wpr > 1) {
             if (lane == 0) { red[par][0][warp] = s1; red[par][1][warp] = s2; }
             __syncthreads();
-            s1 = 0.f; s2 = 0.f;
-            for (int i = 0; i < wpr; ++i) { s1 += red[par][0][row_in_cta * wpr + i]; s2 += red[par][1][row_in_cta * wpr + i]; }
+            // every lane takes one warp's pair of partial sums; three exchange steps add up to eight of them
+            const int src = lane & (kMaxWarps - 1);      // every group of eight lanes holds the same eight values
+            s1 = src < wpr ? red[par][0][row_in_cta * wpr + src] : 0.f;
+            s2 = src < wpr ? red[par][1][row_in_cta * wpr + src] : 0.f;
+#pragma unroll
+            for (int o = kMaxWarps / 2; o > 0; o >>= 1) {
+                s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+                s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+            }
         }
         const uint64_t nmg2 = splat2(-s1 * inv_d), nmgx2 = splat2(-s2 * inv_d);
         if (live) {
