@@ -223,18 +223,25 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
     extern __shared__ uint4 ln_bwd_ring[];
     const uint32_t ring0 = smem_u32(ln_bwd_ring) + 16u * threadIdx.x;
     const uint32_t slot_stride = 16u * blockDim.x;
-    auto issue = [&](int rg, int stage) {
-        const int row = rg * rows_per_cta + row_in_cta;
-        const bool live = rg < row_groups && row < T;
+    // Rows are visited with a constant stride, so the element offsets of the row being fetched and of
+    // the row being computed are running sums (no 64-bit multiply per row).
+    const int row_step = gridDim.x * rows_per_cta;
+    const size_t off_step = static_cast<size_t>(row_step) * d;
+    int pf_row = blockIdx.x * rows_per_cta + row_in_cta;                 // next row to fetch
+    size_t pf_off = static_cast<size_t>(pf_row) * d + 8 * tr;
+    auto issue = [&](int stage) {
+        const bool live = pf_row < T;
 #pragma unroll
         for (int j = 0; j < CHUNKS; ++j) {
-            const size_t off = live ? static_cast<size_t>(row) * d + 8 * (tr + j * tpr) : 0;
+            const size_t off = live ? pf_off + 8 * j * tpr : 0;
             const uint32_t dst = ring0 + (stage * 3 * CHUNKS + j) * slot_stride;
             cp_async_16(dst, dh + off, live);
             cp_async_16(dst + CHUNKS * slot_stride, x + off, live);
             cp_async_16(dst + 2 * CHUNKS * slot_stride, resid ? resid + off : dh + off, live && resid != nullptr);   // no residual: zeros
         }
         cp_async_commit();
+        pf_row += row_step;
+        pf_off += off_step;
     };
     float n_m = 0.f, n_r = 0.f;
     auto fetch_stats = [&](int rg) {
@@ -244,16 +251,17 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
         n_r = live ? rstd[row] : 0.f;
     };
 #pragma unroll
-    for (int s = 0; s < kLnBwdDepth - 1; ++s) issue(blockIdx.x + s * gridDim.x, s);
+    for (int s = 0; s < kLnBwdDepth - 1; ++s) issue(s);
     fetch_stats(blockIdx.x);
     const float inv_d = 1.0f / d;
     int par = 0, stage = 0;
-    for (int rg = blockIdx.x; rg < row_groups; rg += gridDim.x, par ^= 1) {
-        const int row = rg * rows_per_cta + row_in_cta;
+    int row = blockIdx.x * rows_per_cta + row_in_cta;
+    size_t row_off = static_cast<size_t>(row) * d + 8 * tr;
+    for (int rg = blockIdx.x; rg < row_groups; rg += gridDim.x, par ^= 1, row += row_step, row_off += off_step) {
         const bool live = row < T;
         const float r = n_r;
         const uint64_t r2 = splat2(r), nmr2 = splat2(-n_m * r);
-        issue(rg + (kLnBwdDepth - 1) * gridDim.x, stage == 0 ? kLnBwdDepth - 1 : stage - 1);
+        issue(stage == 0 ? kLnBwdDepth - 1 : stage - 1);
         cp_async_wait<kLnBwdDepth - 1>();                  // this row's copies have landed
         uint64_t xh[CHUNKS][4], g[CHUNKS][4], dhv[CHUNKS][4], rs[CHUNKS][4];
         uint64_t s1p = 0ull, s2p = 0ull;
@@ -295,7 +303,7 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
         if (live) {
 #pragma unroll
             for (int j = 0; j < CHUNKS; ++j) {
-                const size_t off = static_cast<size_t>(row) * d + 8 * (tr + j * tpr);
+                const size_t off = row_off + 8 * j * tpr;
                 uint32_t w[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
