@@ -200,6 +200,11 @@ pw_status_t pw_layer_profile_begin(pw_layer_t* layer);
 pw_status_t pw_layer_profile_end(pw_layer_t* layer, pw_profile_t* out);
 /* Kernels launched through this handle since it was created (graph replays count their nodes). */
 pw_status_t pw_layer_launch_count(const pw_layer_t* layer, uint64_t* count);
+/* The backward pass runs its weight-gradient GEMMs and bias column sums on a library-owned side
+ * stream beside the data-gradient chain (default).  enabled = 0 keeps every kernel on the calling
+ * stream, in program order - the same kernels, the same results, one after the other: what a
+ * per-kernel time measured alone corresponds to.  Takes effect from the next call. */
+pw_status_t pw_layer_set_side_stream(pw_layer_t* layer, int enabled);
 
 /* ---- a pipeline stage: L layers x M micro-batches (Section 5.3, Table 2; dispatch modes of Section 5.1) ---- */
 
@@ -242,6 +247,7 @@ pw_status_t pw_stage_status(pw_stage_t* stage, int* device_status, int* site);
 pw_status_t pw_stage_profile_begin(pw_stage_t* stage);
 pw_status_t pw_stage_profile_end(pw_stage_t* stage, pw_profile_t* out);
 pw_status_t pw_stage_launch_count(const pw_stage_t* stage, uint64_t* count);
+pw_status_t pw_stage_set_side_stream(pw_stage_t* stage, int enabled);   /* as pw_layer_set_side_stream */
 
 /* ---- the whole small language model: embedding layer first, softmax layer last (Section 5.3) ----
  * The paper names the two end layers but prints no formula; the reading built here: token

@@ -42,7 +42,7 @@ EXPORTS = (
     "pw_lm_workspace_bytes", "pw_lm_step",
     "pw_op_embedding_fwd", "pw_op_embedding_bwd_scratch_bytes", "pw_op_embedding_bwd", "pw_op_softmax_xent",
     "pw_op_status_reset", "pw_op_selftest_wait_timeout", "pw_op_affine_f32", "pw_sgd_apply",
-    "pw_dp_slice", "pw_dp_reduce_apply", "pw_shared_alloc", "pw_shared_free", "pw_shared_open", "pw_shared_close",
+    "pw_layer_set_side_stream", "pw_stage_set_side_stream", "pw_dp_slice", "pw_dp_reduce_apply", "pw_shared_alloc", "pw_shared_free", "pw_shared_open", "pw_shared_close",
 )
 
 
@@ -155,6 +155,8 @@ def lib() -> ctypes.CDLL:
         L.pw_op_softmax_xent.argtypes = [vp, ci, vp, ci, ci, ctypes.c_float, vp, vp, vp]
         L.pw_op_selftest_wait_timeout.argtypes = [ctypes.c_uint64, ctypes.POINTER(ci), vp]
         L.pw_op_affine_f32.argtypes = [vp, ctypes.c_longlong, ctypes.c_float, ctypes.c_float, vp, vp]
+        L.pw_layer_set_side_stream.argtypes = [vp, ci]
+        L.pw_stage_set_side_stream.argtypes = [vp, ci]
         L.pw_dp_slice.argtypes = [ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int64),
                                   ctypes.POINTER(ctypes.c_int64)]
         L.pw_dp_reduce_apply.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(vp), ctypes.POINTER(vp), vp, ctypes.c_int64,
@@ -254,6 +256,9 @@ class Layer:
                                   ctypes.byref(_ptr12(grads)), int(accumulate), _p(ctx), _p(scratch),
                                   _stream(stream)))
 
+    def set_side_stream(self, enabled: bool):
+        _check(lib().pw_layer_set_side_stream(self._h, int(bool(enabled))))
+
     def status(self):
         c, s = ctypes.c_int(), ctypes.c_int()
         _check(lib().pw_layer_status(self._h, ctypes.byref(c), ctypes.byref(s)))
@@ -327,6 +332,9 @@ class Stage:
         nbytes = workspace.numel() * workspace.element_size() if workspace_bytes is None else workspace_bytes
         _check(lib().pw_lm_step(self._h, P, G, ctypes.byref(lp), ctypes.byref(lg), _p(ids), _p(labels), _p(loss), vocab,
                                 int(recompute), _p(workspace), nbytes, _stream(stream)))
+
+    def set_side_stream(self, enabled: bool):
+        _check(lib().pw_stage_set_side_stream(self._h, int(bool(enabled))))
 
     def status(self):
         c, s = ctypes.c_int(), ctypes.c_int()

@@ -76,6 +76,7 @@ struct LayerPlan {
     // lean ctx: h1, h2, a (and the statistics the re-derivation writes again) live in scratch
     bool lean;
     size_t off_lean_h1, off_lean_h2, off_lean_a, off_lean_stats;
+    size_t off_splitk;           // partial sums of GEMM tiles cut along K (main-stream GEMMs only)
 };
 
 }  // namespace pw
@@ -87,6 +88,7 @@ struct pw_layer {
     cudaStream_t aux = nullptr;     // side stream: weight gradients and bias column sums run beside the dgrad chain
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     uint64_t launches = 0;          // kernels launched (or replayed) through this handle
+    bool single_stream = false;     // pw_layer_set_side_stream(layer, 0): everything on the calling stream
     bool capturing = false;         // inside a stream capture: count launches into graph_nodes instead
     uint64_t graph_nodes = 0;
     // profiling: event pairs around every launch group
@@ -152,6 +154,7 @@ static void build_plan(const pw_layer_config_t& c, Runtime* rt, LayerPlan* p)
     if (c2 > part) part = c2;
     p->off_partials = s; s += align256(part);
     p->off_partials2 = s; s += align256(c1 > c2 ? c1 : c2);   // column sums on the side stream
+    p->off_splitk = s; s += align256(gemm_split_ws_bytes());
     p->off_lean_h1 = p->off_lean_h2 = p->off_lean_a = p->off_lean_stats = 0;
     if (p->lean) {
         p->off_lean_h1 = s; s += align256(T * d * 2);
@@ -194,9 +197,10 @@ static inline const uint8_t* at(const void* base, size_t off) { return static_ca
 
 static GemmArgs gemm_args(int layout, int epi, int act, int M, int N, int K, const void* A, int lda, const void* B,
                           int ldb, void* C, int ldc, const void* bias, const void* aux_in, int ld_aux, void* aux_out,
-                          int accumulate)
+                          int accumulate, void* split_ws = nullptr)
 {
     GemmArgs g;
+    g.split_ws = split_ws;
     g.layout = layout; g.epilogue = epi; g.act = act; g.M = M; g.N = N; g.K = K;
     g.A = A; g.lda = lda; g.B = B; g.ldb = ldb; g.C = C; g.ldc = ldc;
     g.bias = bias; g.aux_in = aux_in; g.ld_aux = ld_aux; g.aux_out = aux_out; g.accumulate = accumulate;
@@ -275,18 +279,20 @@ static pw_status_t enqueue_fwd(pw_layer_t* L, const pw_layer_params_t* P, const 
     void* mu1 = at(ctx, p.ctx_off[PW_CTX_MU1]); void* r1 = at(ctx, p.ctx_off[PW_CTX_R1]);
     void* mu2 = at(ctx, p.ctx_off[PW_CTX_MU2]); void* r2 = at(ctx, p.ctx_off[PW_CTX_R2]);
 
+    // GEMMs on the calling stream never overlap one another, so they may use the split-K scratch.
+    void* sk = scratch ? at(scratch, p.off_splitk) : nullptr;
     PW_DO(do_ln_fwd(L, x, P->ln1_gamma, P->ln1_beta, h1, mu1, r1, st));
     PW_DO(do_gemm(L, gemm_args(kTN, kEpiBias, act, T, 3 * d, d, h1, d, P->w_qkv, d, qkv, 3 * d, P->b_qkv,
-                                     nullptr, 0, nullptr, 0), st));
+                                     nullptr, 0, nullptr, 0, sk), st));
     PW_DO(do_attn_fwd(L, qkv, o, lse, st));
     PW_DO(do_gemm(L, gemm_args(kTN, kEpiBiasResid, act, T, d, d, o, d, P->w_o, d, x1, d, P->b_o, x, d,
-                                     nullptr, 0), st));
+                                     nullptr, 0, sk), st));
     PW_DO(do_ln_fwd(L, x1, P->ln2_gamma, P->ln2_beta, h2, mu2, r2, st));
     PW_DO(do_gemm(L, gemm_args(kTN, kEpiBiasGelu, act, T, F, d, h2, d, P->w_fc1, d, u, F, P->b_fc1, nullptr, 0,
-                                     a, 0), st));
+                                     a, 0, sk), st));
     if (with_fc2)
         PW_DO(do_gemm(L, gemm_args(kTN, kEpiBiasResid, act, T, d, F, a, F, P->w_fc2, F, y, d, P->b_fc2, x1, d,
-                                         nullptr, 0), st));
+                                         nullptr, 0, sk), st));
     return PW_OK;
 }
 
@@ -325,7 +331,7 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
     // streams; the side stream always rejoins before this call returns, so a captured graph sees
     // a plain fork/join.  While per-kernel profiling is on everything stays on one stream.
     static const bool no_side = getenv("PW_NO_SIDE_STREAM") != nullptr;   // tuning aid
-    cudaStream_t ax = (L->profiling || no_side) ? st : L->aux;
+    cudaStream_t ax = (L->profiling || L->single_stream || no_side) ? st : L->aux;
     auto order = [&](cudaEvent_t ev, cudaStream_t from, cudaStream_t to) -> pw_status_t {
         if (from == to) return PW_OK;
         cudaError_t e = cudaEventRecord(ev, from);
@@ -346,8 +352,9 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
     // y = x1 + a W2^T + b2  ->  du = (dy W2) * gelu'(u),  dW2 = dy^T a
     PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, d, F, T, dy, d, a, F, G->w_fc2, F, nullptr, nullptr, 0,
                                      nullptr, accumulate), ax));
+    void* sk = at(scratch, p.off_splitk);                // dgrad GEMMs run one after the other on the calling stream
     PW_DO(do_gemm(L, gemm_args(kNN, kEpiDGelu, act, T, F, d, dy, d, P->w_fc2, F, big, F, nullptr, u, F,
-                                     nullptr, 0), st));
+                                     nullptr, 0, sk), st));
     PW_DO(order(L->ev[1], st, ax));                      // du ready
     // u = h2 W1^T + b1  ->  dh2 = du W1,  dW1 = du^T h2,  db1 = colsum(du)
     if (rederive) PW_DO(do_ln_fwd(L, x1, P->ln2_gamma, P->ln2_beta, const_cast<void*>(h2), lean_st1, lean_st2, ax));
@@ -359,7 +366,7 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
         if (e != cudaSuccess) return fail_cuda("stream ordering", e);
     }
     PW_DO(do_gemm(L, gemm_args(kNN, kEpiNone, act, T, d, F, big, F, P->w_fc1, d, td0, d, nullptr, nullptr, 0,
-                                     nullptr, 0), st));
+                                     nullptr, 0, sk), st));
     // LN2 backward + residual: dx1 = dy + LNbwd(dh2); also db2 = colsum(dy), dbo = colsum(dx1)
     PW_DO(do_ln_bwd(L, td0, x1, mu2, r2, P->ln2_gamma, dy, dx1, G->ln2_gamma, G->ln2_beta,
                                 G->b_fc2, G->b_o, accumulate, part, st));
@@ -368,7 +375,7 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
     PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, d, d, T, dx1, d, o, d, G->w_o, d, nullptr, nullptr, 0,
                                      nullptr, accumulate), ax));
     PW_DO(do_gemm(L, gemm_args(kNN, kEpiNone, act, T, d, d, dx1, d, P->w_o, d, td0, d, nullptr, nullptr, 0,
-                                     nullptr, 0), st));
+                                     nullptr, 0, sk), st));
     // attention backward -> dqkv (reuses the du buffer)
     if (ax != st) {
         cudaError_t e = cudaStreamWaitEvent(st, L->ev[2], 0);
@@ -382,7 +389,7 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
                                      0, nullptr, accumulate), ax));
     PW_DO(do_colsum(L, big, 3 * d, G->b_qkv, accumulate, part2, ax));
     PW_DO(do_gemm(L, gemm_args(kNN, kEpiNone, act, T, d, 3 * d, big, 3 * d, P->w_qkv, d, td0, d, nullptr,
-                                     nullptr, 0, nullptr, 0), st));
+                                     nullptr, 0, nullptr, 0, sk), st));
     // LN1 backward + residual: dx = dx1 + LNbwd(dh1)
     PW_DO(do_ln_bwd(L, td0, x, mu1, r1, P->ln1_gamma, dx1, dx, G->ln1_gamma, G->ln1_beta, nullptr,
                                 nullptr, accumulate, part, st));
@@ -417,8 +424,9 @@ static pw_status_t read_status(DeviceStatus* dev, int* code, int* site)
     if (site) *site = h.site;
     // A kernel that gave up may have left the work counters of the persistent attention kernels
     // mid-count; the device is idle here, so they are put back to zero (the error stays recorded).
-    if (h.code != 0 && (h.sched[0] | h.sched[1] | h.sched[2] | h.sched[3] | h.sched[4] | h.sched[5]) != 0)
-        cudaMemset(reinterpret_cast<char*>(dev) + offsetof(DeviceStatus, sched), 0, sizeof(h.sched));
+    // (the same goes for the split-K tickets of the GEMM, which follow the counters in the struct)
+    if (h.code != 0)
+        cudaMemset(reinterpret_cast<char*>(dev) + offsetof(DeviceStatus, sched), 0, sizeof(h.sched) + sizeof(h.tickets));
     return PW_OK;
 }
 
@@ -718,7 +726,7 @@ pw_status_t pw_stage_run_chain(pw_stage_t* stage, const pw_layer_params_t* param
     // GRAPH: key = every pointer and setting that the captured launches bake in.
     std::vector<uint64_t> key;
     key.reserve(8 + 24 * L + 4 * M);
-    key.push_back(M); key.push_back(schedule); key.push_back(recompute);
+    key.push_back(M); key.push_back(schedule); key.push_back(recompute); key.push_back(stage->layer->single_stream ? 1 : 0);
     key.push_back(reinterpret_cast<uint64_t>(workspace));
     for (int l = 0; l < L; ++l) {
         const void* const* pp = reinterpret_cast<const void* const*>(&params[l]);
@@ -778,6 +786,18 @@ pw_status_t pw_stage_launch_count(const pw_stage_t* stage, uint64_t* count)
 {
     if (!stage) return fail(PW_ERR_INVALID_ARG, "stage is NULL");
     return pw_layer_launch_count(stage->layer, count);
+}
+
+pw_status_t pw_layer_set_side_stream(pw_layer_t* layer, int enabled)
+{
+    if (!layer) return fail(PW_ERR_INVALID_ARG, "layer is NULL");
+    layer->single_stream = enabled == 0;
+    return PW_OK;
+}
+pw_status_t pw_stage_set_side_stream(pw_stage_t* stage, int enabled)
+{
+    if (!stage) return fail(PW_ERR_INVALID_ARG, "stage is NULL");
+    return pw_layer_set_side_stream(stage->layer, enabled);
 }
 
 // ---------------------------------------------------------------------------------------- language model step
@@ -967,8 +987,11 @@ pw_status_t pw_op_gemm(int layout, int epilogue, int act, int M, int N, int K, c
                        int accumulate, void* stream)
 {
     PW_RT_OR_FAIL();
+    // The single-step calls share one status word and run one at a time, so this GEMM may cut the
+    // tiles of a thin last round along K; its scratch is allocated once per device, on first use.
+    if (!rt->split_ws && cudaMalloc(&rt->split_ws, gemm_split_ws_bytes()) != cudaSuccess) { rt->split_ws = nullptr; (void)cudaGetLastError(); }
     PW_OP(launch_gemm(rt, gemm_args(layout, epilogue, act, M, N, K, A, lda, B, ldb, C, ldc, bias, aux_in, ld_aux,
-                                    aux_out, accumulate), rt->op_status, static_cast<cudaStream_t>(stream)));
+                                    aux_out, accumulate, rt->split_ws), rt->op_status, static_cast<cudaStream_t>(stream)));
     return PW_OK;
 }
 

@@ -37,8 +37,10 @@ struct GemmParams {
     int accumulate, act;
     int m_tiles, n_tiles;
     int n_fastest;               // tile numbering: 1 = consecutive tiles share the A row panel, 0 = the B panel
-    int split_begin;             // tiles >= split_begin are issued as two half-width tiles (tail balancing)
+    int split_begin;             // tiles >= split_begin are issued as two units (tail balancing): half-width
+                                 // tiles in the one-CTA kernel, halves of the K range in the CTA-pair kernel
     int total_virtual;           // split_begin + 2 * (m_tiles*n_tiles - split_begin)
+    float* split_ws;             // CTA-pair kernel: where the K halves leave their partial sums
     DeviceStatus* status;
 };
 
@@ -104,10 +106,25 @@ __device__ __forceinline__ void epilogue_group(const uint32_t* v, int row, int c
 // store (rows >= M and columns >= N are clipped by the tensor map).  `taddr` addresses this warp's
 // lane quarter of the accumulator, row0 is the first of its 32 rows, pi selects which of the two
 // warps of the quarter it is (they take alternate column chunks).
-template <int EPI, bool SINGLE_SLAB = false>
+// Partial sums of one 32 x 32 accumulator chunk as the K halves of a cut tile exchange them: eight
+// 512-byte rows of [lane][4 floats], so that every access of a warp is one contiguous 512 bytes.
+__device__ __forceinline__ void add_partner_chunk(uint32_t (&v)[32], const float* partner_chunk, int lane)
+{
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float4 t = __ldcg(reinterpret_cast<const float4*>(partner_chunk + i * 128 + lane * 4));
+        v[4 * i] = __float_as_uint(__uint_as_float(v[4 * i]) + t.x);
+        v[4 * i + 1] = __float_as_uint(__uint_as_float(v[4 * i + 1]) + t.y);
+        v[4 * i + 2] = __float_as_uint(__uint_as_float(v[4 * i + 2]) + t.z);
+        v[4 * i + 3] = __float_as_uint(__uint_as_float(v[4 * i + 3]) + t.w);
+    }
+}
+
+template <int EPI, bool SINGLE_SLAB = false, bool SPLIT = false>
 __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, int bn, int pi, int pstride, int lane,
                                               uint8_t* slab, uint32_t slab_u32, uint32_t& nout, const CUtensorMap* tmC,
-                                              const CUtensorMap* tmAux, const GemmParams& p)
+                                              const CUtensorMap* tmAux, const GemmParams& p,
+                                              const float* partner = nullptr /* SPLIT: the other K half's partial sums, [chunk][1024] */)
 {
     const int row = row0 + lane;
     uint8_t* my_row = slab + lane * 128;
@@ -120,6 +137,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, 
             uint32_t v[32];
             tmem_ld32(taddr + s * 32, v);
             tc_wait_ld();
+            if constexpr (SPLIT) add_partner_chunk(v, partner + s * 1024, lane);
             if (lane == 0) bulk_wait_read0();
             __syncwarp();
 #pragma unroll
@@ -157,6 +175,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, 
             uint32_t v[32];
             tmem_ld32(taddr + ch * 32, v);
             tc_wait_ld();
+            if constexpr (SPLIT) add_partner_chunk(v, partner + ch * 1024, lane);
             uint4 o[4];
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
@@ -364,6 +383,20 @@ template <int EPI> struct PairCfg {
     static constexpr int kSmem = kStages * P_STAGE_BYTES + kEpiWarps * kSlab + 1024 + 256;
 };
 
+// Work unit v of the CTA-pair kernel: a whole tile, or - for the tiles of a thin last round - one
+// half of a tile's K range (slot = which cut tile, half = which half).
+struct PairUnit { int tile, kb0, kb1, slot, half; };
+__device__ __forceinline__ PairUnit pair_unit(const GemmParams& p, int v, int num_k)
+{
+    PairUnit u;
+    if (v < p.split_begin) { u.tile = v; u.kb0 = 0; u.kb1 = num_k; u.slot = -1; u.half = 0; return u; }
+    const int hv = v - p.split_begin;
+    u.slot = hv >> 1; u.half = hv & 1; u.tile = p.split_begin + u.slot;
+    u.kb0 = u.half ? num_k / 2 : 0;
+    u.kb1 = u.half ? num_k : num_k / 2;
+    return u;
+}
+
 template <bool A_MN, bool B_MN, int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairCfg<EPI>::kThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -383,7 +416,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t rank = cluster_ctarank();            // 0 = leader
     const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int num_k = (p.K + BK - 1) / BK;
-    const int total_tiles = p.m_tiles * p.n_tiles;      // pair tiles: m_tiles counts 256-row blocks
+    const int total_tiles = p.total_virtual;            // work units: whole pair tiles (m_tiles counts 256-row blocks) + K halves
     const int bn = p.bn, half_n = bn >> 1;
 
     if (threadIdx.x == 0) {
@@ -413,12 +446,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             const uint32_t pair_tx = 2u * (A_TILE_BYTES + half_n * BK * 2);
-            for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs) {
+            for (int unit = pair_id; unit < total_tiles && ok; unit += n_pairs) {
+                const PairUnit un = pair_unit(p, unit, num_k);
+                const int tile = un.tile;
                 const int mi = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles;
                 const int ni = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
                 const int m0 = mi * 256 + rank * 128;
                 const int n0 = ni * bn + rank * half_n;
-                for (int kb = 0; kb < num_k; ++kb) {
+                for (int kb = un.kb0; kb < un.kb1; ++kb) {
                     if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 700)) { ok = false; break; }
                     const uint32_t fb = mapa_shared(full0 + 8 * stage, 0);     // the leader's barrier
                     if (rank == 0) mbar_arrive_expect_tx(full0 + 8 * stage, pair_tx);
@@ -443,12 +478,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint32_t idesc = make_idesc_bf16(256, bn, A_MN, B_MN);
             uint32_t stage = 0, phase = 0, it = 0;
             bool ok = true;
-            for (int tile = pair_id; tile < total_tiles && ok; tile += n_pairs, ++it) {
+            for (int unit = pair_id; unit < total_tiles && ok; unit += n_pairs, ++it) {
+                const PairUnit un = pair_unit(p, unit, num_k);
                 const uint32_t buf = it & 1, acc_phase = (it >> 1) & 1;
                 if (!mbar_wait(acce0 + 8 * buf, acc_phase ^ 1, abort_flag, p.status, 710)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN_MAX;
-                for (int kb = 0; kb < num_k; ++kb) {
+                for (int kb = un.kb0; kb < un.kb1; ++kb) {
                     if (!mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 711)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_base = smem_u32(tiles + stage * P_STAGE_BYTES), b_base = a_base + A_TILE_BYTES;
@@ -458,7 +494,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                                     : make_smem_desc_sw128(a_base + kk * 32, 16, 1024);
                         const uint64_t bdesc = B_MN ? make_smem_desc_sw128(b_base + kk * 2048, 8192, 1024)
                                                     : make_smem_desc_sw128(b_base + kk * 32, 16, 1024);
-                        umma_f16_pair(d_tmem, adesc, bdesc, idesc, (kb | kk) != 0 ? 1u : 0u);
+                        umma_f16_pair(d_tmem, adesc, bdesc, idesc, (kb != un.kb0 || kk != 0) ? 1u : 0u);
                     }
                     umma_commit_pair(empty0 + 8 * stage, 3);     // frees the stage in both CTAs
                     if (++stage == P_STAGES) { stage = 0; phase ^= 1; }
@@ -471,7 +507,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         uint8_t* slab = slabs + (warp - 2) * PairCfg<EPI>::kSlab;
         const uint32_t slab_u32 = smem_u32(slab);
         uint32_t it = 0, nout = 0;
-        for (int tile = pair_id; tile < total_tiles; tile += n_pairs, ++it) {
+        for (int unit = pair_id; unit < total_tiles; unit += n_pairs, ++it) {
+            const PairUnit un = pair_unit(p, unit, num_k);
+            const int tile = un.tile;
             const int mi = p.n_fastest ? tile / p.n_tiles : tile % p.m_tiles;
             const int ni = p.n_fastest ? tile % p.n_tiles : tile / p.m_tiles;
             const int m0 = mi * 256 + rank * 128, n0 = ni * bn;
@@ -481,7 +519,42 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * BN_MAX;
-            epilogue_tile<EPI, NEPI == 16>(taddr, m0 + q * 32, n0, bn, pi, NEPI / 4, lane, slab, slab_u32, nout, &tmC, &tmAux, p);
+            if (EPI == kEpiF32 || un.slot < 0) {                 // (the fp32-output GEMMs are never cut)
+                epilogue_tile<EPI, NEPI == 16>(taddr, m0 + q * 32, n0, bn, pi, NEPI / 4, lane, slab, slab_u32, nout, &tmC, &tmAux, p);
+            } else {
+                // Half of a cut tile's K range.  Every epilogue warp leaves its part of the partial sums in
+                // the scratch, then draws a ticket shared with the same warp of the CTA that has the
+                // other half: the first of the two is finished, the second adds the first one's sums
+                // to its own (fp32, two addends: the result does not depend on who came first) and
+                // runs the epilogue.  Nobody waits for anybody.
+                const int nchunks = bn / 32;
+                const size_t region = static_cast<size_t>(nchunks) * 1024;       // floats per (slot, half, rank, quarter)
+                float* mine = p.split_ws + ((((static_cast<size_t>(un.slot) * 2 + un.half) * 2 + rank) * 4) + q) * region;
+                const float* other = p.split_ws + ((((static_cast<size_t>(un.slot) * 2 + (un.half ^ 1)) * 2 + rank) * 4) + q) * region;
+#pragma unroll 1
+                for (int ch = pi; ch < nchunks; ch += NEPI / 4) {
+                    if (n0 + ch * 32 >= p.N) break;
+                    uint32_t v[32];
+                    tmem_ld32(taddr + ch * 32, v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        __stcg(reinterpret_cast<float4*>(mine + ch * 1024 + i * 128 + lane * 4),
+                               make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
+                                           __uint_as_float(v[4 * i + 3])));
+                }
+                __threadfence();
+                __syncwarp();
+                int* ticket = &p.status->tickets[(un.slot * 2 + static_cast<int>(rank)) * 16 + (warp - 2)];
+                int before = 0;
+                if (lane == 0) before = atomicAdd(ticket, 1);
+                before = __shfl_sync(0xffffffffu, before, 0);
+                if (before != 0) {
+                    if (lane == 0) *ticket = 0;                                  // both halves have drawn: ready for the next launch
+                    __threadfence();
+                    epilogue_tile<EPI, NEPI == 16, true>(taddr, m0 + q * 32, n0, bn, pi, NEPI / 4, lane, slab, slab_u32, nout, &tmC, &tmAux, p, other);
+                }
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_shared(acce0 + 8 * buf, 0));
@@ -539,7 +612,7 @@ const char* launch_pair(Runtime* rt, const CUtensorMap& tmA, const CUtensorMap& 
                         const CUtensorMap& tmAux, const GemmParams& p, cudaStream_t stream)
 {
     auto kern = gemm_pair_kernel<A_MN, B_MN, EPI>;
-    const int total = p.m_tiles * p.n_tiles;
+    const int total = p.total_virtual;
     const int max_pairs = rt->sm_count / 2;
     const int pairs = total < max_pairs ? total : max_pairs;
     return launch_k(kern, dim3(2 * pairs), dim3(PairCfg<EPI>::kThreads), PairCfg<EPI>::kSmem, stream, tmA, tmB, tmC, tmAux, p) == cudaSuccess
@@ -603,6 +676,22 @@ static const char* launch_gemm_pair(Runtime* rt, const GemmArgs& a, DeviceStatus
     p.accumulate = a.accumulate; p.act = a.act;
     p.m_tiles = m_tiles; p.n_tiles = (a.N + bn - 1) / bn;
     p.split_begin = p.m_tiles * p.n_tiles; p.total_virtual = p.split_begin;
+    p.split_ws = nullptr;
+    {
+        // Tail balancing: when the last round of tiles would keep at most half of the CTA pairs busy,
+        // each of its tiles becomes two units of half the K range (needs the caller's scratch).
+        static const bool no_split = getenv("PW_GEMM_NO_SPLIT") != nullptr;   // tuning aid
+        const int total = p.m_tiles * p.n_tiles, num_k = (a.K + BK - 1) / BK;
+        const int rem = total % pairs;
+        static const int min_k = [] { const char* v = getenv("PW_GEMM_SPLIT_MIN_K"); return v ? atoi(v) : 64; }();   // tuning aid
+        // (short K ranges lose more to the second prologue and epilogue than the idle half round costs)
+        if (a.split_ws && !no_split && !f32_out && total > pairs && rem > 0 && 2 * rem <= pairs && rem <= kSplitMaxTiles &&
+            num_k >= min_k) {
+            p.split_begin = total - rem;
+            p.total_virtual = p.split_begin + 2 * rem;
+            p.split_ws = static_cast<float*>(a.split_ws);
+        }
+    }
     p.n_fastest = p.n_tiles < p.m_tiles ? 1 : 0;
     p.status = status;
     const int key = a.layout * 16 + a.epilogue;
@@ -617,6 +706,9 @@ static const char* launch_gemm_pair(Runtime* rt, const GemmArgs& a, DeviceStatus
         default: return "gemm: unsupported layout/epilogue combination";
     }
 }
+
+// Scratch for the K halves of cut tiles: (cut tile, half, CTA of the pair) x 128 rows x 256 columns, fp32.
+size_t gemm_split_ws_bytes() { return static_cast<size_t>(kSplitMaxTiles) * 2 * 2 * 128 * BN_MAX * sizeof(float); }
 
 const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cudaStream_t stream)
 {
@@ -673,6 +765,7 @@ const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cu
     p.m_tiles = m_tiles; p.n_tiles = (a.N + bn - 1) / bn;
     p.n_fastest = p.n_tiles < p.m_tiles ? 1 : 0;
     p.status = status;
+    p.split_ws = nullptr;
     {
         // Tail balancing: when the last round would leave at least half of the SMs idle, its
         // tiles are issued as two half-width tiles each.

@@ -13,10 +13,15 @@ namespace pw {
 // (0 = ok), word 1 = site id of the wait that gave up.
 // Words 2.. are the work counters of the persistent attention kernels: {next ticket, CTAs done}
 // per kernel.  They are zero between launches (the last CTA of a launch clears its pair).
+// A GEMM whose last round of tiles would leave at least half of the CTA pairs idle cuts each of those
+// tiles in two along K; the two halves meet through a ticket per (tile, CTA of the pair, epilogue warp).
+constexpr int kSplitMaxTiles = 40;                       // at most half of the CTA pairs' worth of tiles is cut
+constexpr int kSplitTickets = kSplitMaxTiles * 2 * 16;
 struct DeviceStatus {
     int code;
     int site;
     int sched[6];               // [0,1] attention fwd, [2,3] dQ, [4,5] dK/dV
+    int tickets[kSplitTickets]; // split-K hand-off of the GEMM; always back to zero when a kernel ends normally
 };
 
 constexpr int kStatusTimeout = 6;  // == PW_ERR_TIMEOUT

@@ -18,6 +18,7 @@ struct Runtime {
     int sm_count = 0;
     int cc_major = 0;
     void* encode_tiled = nullptr;      // cuTensorMapEncodeTiled, fetched through the runtime API
+    void* split_ws = nullptr;          // split-K scratch of the single-step GEMM call (allocated on first use)
     DeviceStatus* op_status = nullptr; // device memory, status block for pw_op_* calls
 };
 // Returns nullptr (and sets *err) if the device is not sm_100 or a CUDA call failed.
@@ -56,7 +57,11 @@ struct GemmArgs {
     const void* aux_in; int ld_aux;
     void* aux_out;
     int accumulate;
+    // Optional fp32 scratch of gemm_split_ws_bytes(): lets the tiles of a thin last round be cut in two
+    // along K.  Only for GEMMs that never run beside another GEMM using the same status word.
+    void* split_ws = nullptr;
 };
+size_t gemm_split_ws_bytes();
 // Encodes the two tensor maps and launches.  Returns nullptr on success, else a static message.
 const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cudaStream_t stream);
 

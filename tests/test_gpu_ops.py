@@ -294,3 +294,49 @@ def test_attention_random_shapes(pw, oracle64):
         assert rel_l2(o, ow) < ACT_TOL, (case, B, S, H, dh)
         assert np.allclose(lse.cpu().numpy(), lsew, atol=2e-3), (case, B, S, H, dh)
         assert rel_l2(dqkv, oracle64.attn_bwd(np64(qkv), np64(dout), B, S, H, dh)) < GRAD_TOL, (case, B, S, H, dh)
+
+
+def test_gemm_tiles_cut_along_k_are_exact_and_reproducible(pw):
+    """110 pair tiles on 74 CTA pairs: the 36 tiles of the last round are cut in two along K and the
+    halves meet through the scratch (bf16-output GEMMs with K >= 4096 only; the fp32-output layout
+    is run for comparison).  Integer operands make every partial sum exact, so the result must be
+    the exact product (rounded once to bf16 where the output is bf16), five times in a row (the
+    tickets are back at zero after every launch)."""
+    g = torch.Generator().manual_seed(9)
+    M, N, K = 2560, 2816, 4096
+    ri = lambda *s: torch.randint(-2, 3, s, generator=g).to(torch.bfloat16)
+    # TN: C = A B^T + bias + residual
+    A, B = ri(M, K), ri(N, K)
+    bias, resid = ri(N), ri(M, N)
+    want = (A.double() @ B.double().T + bias.double() + resid.double()).to(torch.bfloat16)
+    Ad, Bd, bd, rd = A.cuda(), B.cuda(), bias.cuda(), resid.cuda()
+    for _ in range(5):
+        C, check = guard_alloc((M, N), torch.bfloat16)
+        pw.op_gemm(pw.GEMM_TN, pw.EPI_BIAS_RESID, M, N, K, Ad, K, Bd, K, C, N, bias=bd, aux_in=rd, ld_aux=N)
+        torch.cuda.synchronize()
+        _status_ok(pw)
+        check()
+        assert torch.equal(C.cpu(), want)
+    # NN: C = A B  (dgrad: B stored [K, N])
+    Bn = ri(K, N)
+    want = (A.double() @ Bn.double()).to(torch.bfloat16)
+    C, check = guard_alloc((M, N), torch.bfloat16)
+    pw.op_gemm(pw.GEMM_NN, pw.EPI_NONE, M, N, K, Ad, K, Bn.cuda(), N, C, N)
+    torch.cuda.synchronize()
+    _status_ok(pw)
+    check()
+    assert torch.equal(C.cpu(), want)
+    # NT: C (+)= A^T B, fp32 (A stored [K, M], B stored [K, N])
+    At = ri(K, M)
+    want = At.double().T @ Bn.double()
+    C0 = torch.randint(-5, 6, (M, N), generator=g).float()
+    for accumulate in (False, True):
+        C, check = guard_alloc((M, N), torch.float32)
+        C.copy_(C0)
+        pw.op_gemm(pw.GEMM_NT, pw.EPI_F32, M, N, K, At.cuda(), M, Bn.cuda(), N, C, N, accumulate=accumulate)
+        torch.cuda.synchronize()
+        _status_ok(pw)
+        check()
+        assert torch.equal(C.double().cpu(), want + (C0.double() if accumulate else 0))
+    # a GEMM that is not cut still works afterwards
+    test_gemm_tn_integer_exact(pw)
