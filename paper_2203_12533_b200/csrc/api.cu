@@ -59,6 +59,8 @@ Runtime* get_runtime(const char** err)
         cudaMemset(rt->op_status, 0, sizeof(DeviceStatus)) != cudaSuccess) {
         delete rt; *err = "could not allocate the status word"; return nullptr;
     }
+    // split-K scratch of the single-step GEMM call; without it that call simply never cuts a tile
+    if (cudaMalloc(&rt->split_ws, gemm_split_ws_bytes()) != cudaSuccess) { rt->split_ws = nullptr; (void)cudaGetLastError(); }
     per_device[dev] = rt;
     return rt;
 }
@@ -988,8 +990,7 @@ pw_status_t pw_op_gemm(int layout, int epilogue, int act, int M, int N, int K, c
 {
     PW_RT_OR_FAIL();
     // The single-step calls share one status word and run one at a time, so this GEMM may cut the
-    // tiles of a thin last round along K; its scratch is allocated once per device, on first use.
-    if (!rt->split_ws && cudaMalloc(&rt->split_ws, gemm_split_ws_bytes()) != cudaSuccess) { rt->split_ws = nullptr; (void)cudaGetLastError(); }
+    // tiles of a thin last round along K (scratch allocated with the runtime, never on this path).
     PW_OP(launch_gemm(rt, gemm_args(layout, epilogue, act, M, N, K, A, lda, B, ldb, C, ldc, bias, aux_in, ld_aux,
                                     aux_out, accumulate, rt->split_ws), rt->op_status, static_cast<cudaStream_t>(stream)));
     return PW_OK;

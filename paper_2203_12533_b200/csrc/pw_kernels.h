@@ -18,7 +18,7 @@ struct Runtime {
     int sm_count = 0;
     int cc_major = 0;
     void* encode_tiled = nullptr;      // cuTensorMapEncodeTiled, fetched through the runtime API
-    void* split_ws = nullptr;          // split-K scratch of the single-step GEMM call (allocated on first use)
+    void* split_ws = nullptr;          // split-K scratch of the single-step GEMM call (allocated with the runtime)
     DeviceStatus* op_status = nullptr; // device memory, status block for pw_op_* calls
 };
 // Returns nullptr (and sets *err) if the device is not sm_100 or a CUDA call failed.
