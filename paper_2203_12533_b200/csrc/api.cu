@@ -1191,7 +1191,7 @@ pw_status_t pw_op_status_reset(void)
 {
     PW_RT_OR_FAIL();
     cudaError_t e = cudaDeviceSynchronize();
-    if (e == cudaSuccess) e = cudaMemset(rt->op_status, 0, 2 * sizeof(int));   // code and site; the work counters stay
+    if (e == cudaSuccess) e = cudaMemset(rt->op_status, 0, sizeof(DeviceStatus));   // the device is idle: code, site, counters, tickets
     return e == cudaSuccess ? PW_OK : fail_cuda("status reset", e);
 }
 
