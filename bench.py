@@ -346,17 +346,28 @@ def run_ours(args, w):
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    def timed(fn, steps):
+    def timed(fn, steps, per_step=None):
+        """Milliseconds for `steps` calls of fn (max over ranks).  per_step: a list that receives this
+        rank's time of every single step (one more event per step)."""
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        marks = []
         barrier()
         with torch.cuda.stream(stream):
             e0.record(stream)
             for _ in range(steps):
                 fn()
+                if per_step is not None:
+                    marks.append(torch.cuda.Event(enable_timing=True))
+                    marks[-1].record(stream)
             stream.wait_stream(s_d2h)                    # (end-to-end runs) the last results are on the host
             e1.record(stream)
         torch.cuda.synchronize(dev)
         ms = e0.elapsed_time(e1)
+        if per_step is not None:
+            prev = e0
+            for m in marks:
+                per_step.append(prev.elapsed_time(m))
+                prev = m
         barrier()
         return max_over_ranks(ms, world, dev)
 
@@ -369,8 +380,9 @@ def run_ours(args, w):
         raise SystemExit(f"device status {code} at site {site} after warm-up")
 
     n0 = stage.launch_count()
+    per_step = []
     with ClockSampler(local) as clocks:
-        ms_total = timed(step, args.steps)
+        ms_total = timed(step, args.steps, per_step)
     launches = stage.launch_count() - n0
     ms_step = ms_total / args.steps
     tokens_step = T * M
@@ -414,7 +426,8 @@ def run_ours(args, w):
     hw_flops = hw_flops_per_step(w)
     line = {
         "metric": "decoder-layer fwd+bwd tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+        "ms_per_step_median": statistics.median(per_step), "ms_per_step_best": min(per_step), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "d_model": w.d_model, "heads": f"{w.n_heads}x{w.head_dim}", "d_ff": w.d_ff,
                    "seq_len": w.seq_len, "microbatch": w.batch, "layers": L, "microbatches": M,
@@ -425,6 +438,7 @@ def run_ours(args, w):
         "tflops_hw": world * hw_flops / (ms_step * 1e-3) / 1e12,
         "frac_bf16_peak_burst": hw_flops / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
         "frac_bf16_peak_sustained": hw_flops / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+        "frac_bf16_nominal_2250": hw_flops / (ms_step * 1e-3) / 1e12 / 2250.0,   # datasheet dense bf16, for context
         "peaks": peaks,
         "clocks": clocks.summary(),
         "e2e": {"value": e2e_value, "unit": "tokens/s", "ms_per_step": ms_e2e, "steps": e2e_steps,
@@ -583,16 +597,25 @@ def run_ours_lm(args, w):
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    def timed(fn, steps):
+    def timed(fn, steps, per_step=None):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        marks = []
         barrier()
         with torch.cuda.stream(stream):
             e0.record(stream)
             for _ in range(steps):
                 fn()
+                if per_step is not None:
+                    marks.append(torch.cuda.Event(enable_timing=True))
+                    marks[-1].record(stream)
             e1.record(stream)
         torch.cuda.synchronize(dev)
         ms = e0.elapsed_time(e1)
+        if per_step is not None:
+            prev = e0
+            for m in marks:
+                per_step.append(prev.elapsed_time(m))
+                prev = m
         barrier()
         return max_over_ranks(ms, world, dev)
 
@@ -603,8 +626,9 @@ def run_ours_lm(args, w):
     if stage.status() != (0, 0):
         raise SystemExit(f"device status {stage.status()} after warm-up")
     n0 = stage.launch_count()
+    per_step = []
     with ClockSampler(local) as clocks:
-        ms_step = timed(step, args.steps) / args.steps
+        ms_step = timed(step, args.steps, per_step) / args.steps
     launches = stage.launch_count() - n0 + apply_launches * args.steps
     loss_after_timed = float(loss.item())
     stage.profile_begin()
@@ -641,7 +665,8 @@ def run_ours_lm(args, w):
     value = whole_job_value(T, world, ms_step)
     line = {
         "metric": "small-LM training step tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+        "ms_per_step_median": statistics.median(per_step), "ms_per_step_best": min(per_step), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "d_model": d, "heads": f"{w.n_heads}x{w.head_dim}", "d_ff": w.d_ff,
                    "seq_len": w.seq_len, "batch": w.batch, "layers": L, "vocab": V, "recompute": bool(w.recompute),
@@ -655,6 +680,7 @@ def run_ours_lm(args, w):
         "tflops_hw": world * hw_flops / (ms_step * 1e-3) / 1e12,
         "frac_bf16_peak_burst": hw_flops / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
         "frac_bf16_peak_sustained": hw_flops / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+        "frac_bf16_nominal_2250": hw_flops / (ms_step * 1e-3) / 1e12 / 2250.0,   # datasheet dense bf16, for context
         "peaks": peaks, "clocks": clocks.summary(),
         "e2e": {"value": world * T / (ms_e2e * 1e-3), "unit": "tokens/s", "ms_per_step": ms_e2e, "steps": e2e_steps,
                 "how": "pinned host ids, labels -> device and the loss -> pinned host every step",
