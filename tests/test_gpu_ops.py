@@ -340,3 +340,32 @@ def test_gemm_tiles_cut_along_k_are_exact_and_reproducible(pw):
         assert torch.equal(C.double().cpu(), want + (C0.double() if accumulate else 0))
     # a GEMM that is not cut still works afterwards
     test_gemm_tn_integer_exact(pw)
+
+
+@pytest.mark.parametrize("M,N,K", [(2056, 2312, 4104), (4096, 1280, 4096), (1288, 3848, 5000), (2304, 2304, 8200),
+                                    (8192, 2048, 4096)])
+def test_gemm_cut_tiles_ragged_shapes_are_exact(pw, M, N, K):
+    """Shapes whose last round of 256 x 256 tiles keeps at most half of the 74 CTA pairs busy (so its
+    tiles are cut along K), with ragged edges in every dimension: integer operands, exact result, for
+    the forward layout with the GeLU' -free epilogues and for the data-gradient layout."""
+    tiles = -(-M // 256) * -(-N // 256)
+    rem = tiles % 74
+    assert tiles > 74 and 0 < rem <= 37 and K >= 4096, (tiles, rem)      # the launcher's condition for cutting
+    g = torch.Generator().manual_seed(M + N + K)
+    ri = lambda *s: torch.randint(-2, 3, s, generator=g).to(torch.bfloat16)
+    A, B, Bn, bias = ri(M, K), ri(N, K), ri(K, N), ri(N)
+    Ad = A.cuda()
+    want = (A.double() @ B.double().T + bias.double()).to(torch.bfloat16)
+    C, check = guard_alloc((M, N), torch.bfloat16)
+    pw.op_gemm(pw.GEMM_TN, pw.EPI_BIAS, M, N, K, Ad, K, B.cuda(), K, C, N, bias=bias.cuda())
+    torch.cuda.synchronize()
+    _status_ok(pw)
+    check()
+    assert torch.equal(C.cpu(), want)
+    want = (A.double() @ Bn.double()).to(torch.bfloat16)
+    C, check = guard_alloc((M, N), torch.bfloat16)
+    pw.op_gemm(pw.GEMM_NN, pw.EPI_NONE, M, N, K, Ad, K, Bn.cuda(), N, C, N)
+    torch.cuda.synchronize()
+    _status_ok(pw)
+    check()
+    assert torch.equal(C.cpu(), want)
