@@ -248,3 +248,22 @@ def test_single_tile_layer(pw, oracle64):
     check_layer_against_oracle(pw, oracle64, w, random_ln=True)
     w = inputs.Workload("odd_tiles", 768, 12, 64, 384, 384, 1, sigma_w=0.03)    # S = 3 x 128: the last pair has one tile
     check_layer_against_oracle(pw, oracle64, w, random_ln=True, save_ctx=False)
+
+
+def test_side_stream_switch_changes_no_bit(pw):
+    """The backward pass with its weight-gradient GEMMs on the library's side stream (default) and
+    with every kernel on the calling stream gives the same bits."""
+    w = inputs.Workload("side", 512, 4, 128, 2048, 256, 4)
+    params = [p.cuda() for p in inputs.layer_params(w, 0, 0, random_ln=True)]
+    x, dy = inputs.microbatch(w, 0, 0)
+    xd, dyd = x.cuda().view(-1, w.d_model), dy.cuda().view(-1, w.d_model)
+    layer = make_layer(pw, w)
+    a = run_layer_gpu(pw, layer, params, xd, dyd)
+    layer.set_side_stream(False)
+    b = run_layer_gpu(pw, layer, params, xd, dyd)
+    layer.set_side_stream(True)
+    c = run_layer_gpu(pw, layer, params, xd, dyd)
+    for other in (b, c):
+        assert torch.equal(a["y"], other["y"]) and torch.equal(a["dx"], other["dx"])
+        for g0, g1 in zip(a["grads"], other["grads"]):
+            assert torch.equal(g0, g1)
