@@ -139,3 +139,32 @@ def test_lean_chain_and_lm_step_follow_the_full_save_set(pw):
         assert stage.status() == (0, 0)
         out[flags] = (loss.item(), eg[0], ws.numel())
     assert out[0][0] == out[1][0] and torch.equal(out[0][1], out[1][1]) and out[1][2] < out[0][2]
+
+
+def test_lean_chain_as_a_captured_graph_matches_the_stream_run(pw):
+    """The lean backward's extra kernels sit on the side stream; captured into a CUDA graph and
+    replayed twice they give the same bits as the plain asynchronous run."""
+    w = inputs.Workload("lean_graph", 256, 2, 128, 1024, 128, 2, n_layers=2, n_microbatches=2)
+    L, M = w.n_layers, w.n_microbatches
+    params = [[p.cuda() for p in inputs.layer_params(w, 0, l, random_ln=True)] for l in range(L)]
+    mbs = [inputs.microbatch(w, 0, m) for m in range(M)]
+    xs, dys = [x.cuda() for x, _ in mbs], [dy.cuda() for _, dy in mbs]
+    stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch, flags=pw.FLAG_LEAN_CTX)
+    ws = torch.empty(stage.workspace_bytes(M, pw.SCHEDULE_GPIPE, False), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+    outs = []
+    for mode, reps in ((pw.DISPATCH_ASYNC, 1), (pw.DISPATCH_GRAPH, 2)):
+        grads = [[torch.full(p.shape, float("nan"), dtype=torch.float32, device="cuda") for p in ps] for ps in params]
+        ys, dxs = [torch.empty_like(x) for x in xs], [torch.empty_like(x) for x in xs]
+        with torch.cuda.stream(stream):
+            for _ in range(reps):
+                stage.run_chain(params, grads, xs, dys, ys, dxs, ws, dispatch=mode, schedule=pw.SCHEDULE_GPIPE,
+                                recompute=False, stream=stream)
+        torch.cuda.synchronize()
+        assert stage.status() == (0, 0)
+        outs.append((ys, dxs, grads))
+    for a, b in zip(outs[0][0] + outs[0][1], outs[1][0] + outs[1][1]):
+        assert torch.equal(a, b)
+    for ga, gb in zip(outs[0][2], outs[1][2]):
+        for a, b in zip(ga, gb):
+            assert torch.equal(a, b)
