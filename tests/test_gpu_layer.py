@@ -209,6 +209,12 @@ def test_cfg2_full_size_parity(pw, oracle32):
     check_layer_against_oracle(pw, oracle32, inputs.WORKLOADS[2])
 
 
+def test_cfg5_layer_full_size_parity(pw, oracle32):
+    """One layer of workload 5 at its full size (d=1024, 16x64 heads, F=4096, S=1024, B=16: the 64-wide
+    heads in the launch configuration the benchmark times) against the fp32 oracle, every tensor."""
+    check_layer_against_oracle(pw, oracle32, inputs.WORKLOADS[5].with_(n_layers=1, vocab=0))
+
+
 # ------------------------------------------------------------------------------------------ full sizes of workloads 3 and 4
 @pytest.mark.parametrize("wid", [3, 4], ids=["cfg3_layer_full_size", "cfg4_full_size"])
 def test_full_size_wide_layer_by_the_causal_prefix_property(pw, oracle32, wid):
