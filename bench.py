@@ -32,7 +32,7 @@ sys.path.insert(0, ROOT)
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram bytes read+written per GEMM launch (average over the 12 GEMM launches of a workload-2 step),
-# from the ncu capture summarised in profiles/gemm_pair_kernel_cfg2_dram_traffic.md; None for
+# from one ncu pass (dram__bytes_read.sum + dram__bytes_write.sum) over those launches; None for
 # workloads without a capture.
 GEMM_DRAM_TRAFFIC_PER_LAUNCH = {"cfg2_d2048_s1024_b8": 220.7e6}
 
@@ -181,25 +181,27 @@ def isolated_elementwise(pw, w, peaks, dev, iters=30, nbuf=6):
 
 
 def gemm_roofline(g_flops, g_ms, g_n, tot_ms, ms_one_stream, steps, peaks, kernel, traffic):
-    """Roofline object of the GEMM family.  An event pair around every launch (the instrumented pass)
-    keeps each kernel's prologue from overlapping its predecessor's tail and adds launch latency, so
-    the bracketed per-launch time is longer than what the kernel costs inside the step (and longer
-    than ncu's serialised per-launch time).  The GEMM time per step is therefore taken as
-    (GEMM share of the bracketed times) x (event-timed step with every kernel on one stream and no
-    events between launches); the bracketed figures are reported beside it."""
+    """Roofline object of the GEMM family.  `achieved` is the literal figure: the algorithmic FLOPs of
+    the GEMM launches (2 M N K each) divided by the sum of their CUDA-event durations, each launch
+    bracketed by its own event pair on the launching stream (the instrumented pass).  An event pair
+    around every launch keeps a kernel's prologue from overlapping its predecessor's tail and adds
+    launch latency, so this is a lower bound on what the kernel does inside the un-instrumented step;
+    `achieved_in_step` apportions instead: (GEMM share of the bracketed times) x (event-timed step with
+    every kernel on one stream and no events between launches)."""
     share = g_ms / tot_ms
     ms_gemm_step = share * ms_one_stream
-    achieved = (g_flops / steps) / (ms_gemm_step * 1e-3) / 1e12
+    in_step = (g_flops / steps) / (ms_gemm_step * 1e-3) / 1e12
     bracketed = g_flops / (g_ms * 1e-3) / 1e12
     return {
-        "kernel": kernel, "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-        "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst cuBLAS bf16)",
-        "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
-        "flops_per_launch": g_flops / g_n, "ms_per_launch": ms_gemm_step / (g_n / steps), "launches_per_step": g_n / steps,
+        "kernel": kernel, "bound": "tensor", "achieved": bracketed, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+        "frac": bracketed / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst cuBLAS bf16)",
+        "frac_of_sustained_peak": bracketed / peaks["bf16_tflops_sustained"],
+        "flops_per_launch": g_flops / g_n, "ms_per_launch": g_ms / g_n, "launches_per_step": g_n / steps,
         "share_of_step": share,
-        "how": "share of the per-launch CUDA-event times x the event-timed one-stream step (no events between launches)",
-        "achieved_bracketed": bracketed, "frac_bracketed": bracketed / peaks["bf16_tflops"],
-        "ms_per_launch_bracketed": g_ms / g_n,
+        "how": "algorithmic FLOPs of the GEMM launches / sum of their per-launch CUDA-event durations (instrumented pass)",
+        "achieved_in_step": in_step, "frac_in_step": in_step / peaks["bf16_tflops"],
+        "ms_per_launch_in_step": ms_gemm_step / (g_n / steps),
+        "how_in_step": "GEMM share of the per-launch event times x the event-timed one-stream step (no events between launches)",
         "traffic": traffic,
     }
 
@@ -258,7 +260,10 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
-def run_ours(args, w):
+def run_ours(args, w, brief=False):
+    """Times workload w; returns the JSON line as a dict (rank 0) or None.  brief: the short form used
+    for the secondary workloads of the default run - device-resident steps and the per-class table
+    only (no end-to-end pass, no isolated kernels, no CPU baseline), single rank."""
     import torch
     import torch.distributed as dist
     from paper_2203_12533_b200 import binding as pw
@@ -266,10 +271,12 @@ def run_ours(args, w):
 
     rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if brief:
+        rank, world = 0, 1
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the product path)")
     torch.cuda.set_device(local)
-    if world > 1:
+    if world > 1 and not dist.is_initialized():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     pw.lib()
     peaks = load_peaks()
@@ -285,14 +292,17 @@ def run_ours(args, w):
     host_x, host_dy = [], []
     for m in range(M):
         x, dy = inputs.microbatch(w, args.seed, m)
-        host_x.append(x.view(T, d).pin_memory())
-        host_dy.append(dy.view(T, d).pin_memory())
+        host_x.append(x.view(T, d) if brief else x.view(T, d).pin_memory())
+        host_dy.append(dy.view(T, d) if brief else dy.view(T, d).pin_memory())
     xs = [t.to(dev) for t in host_x]
     dys = [t.to(dev) for t in host_dy]
     ys = [torch.empty_like(t) for t in xs]
     dxs = [torch.empty_like(t) for t in xs]
-    host_y = [torch.empty((T, d), dtype=torch.bfloat16).pin_memory() for _ in range(M)]
-    host_dx = [torch.empty((T, d), dtype=torch.bfloat16).pin_memory() for _ in range(M)]
+    if brief:
+        host_x = host_dy = host_y = host_dx = None
+    else:
+        host_y = [torch.empty((T, d), dtype=torch.bfloat16).pin_memory() for _ in range(M)]
+        host_dx = [torch.empty((T, d), dtype=torch.bfloat16).pin_memory() for _ in range(M)]
     ws_bytes = stage.workspace_bytes(M, schedule, w.recompute)
     workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
     stream = torch.cuda.Stream(device=dev)
@@ -303,11 +313,14 @@ def run_ours(args, w):
     # End to end: every step copies its x and dy from pinned host memory and reads its y and dx back.
     # Two device buffer sets and two copy streams pipeline the transfers behind the compute of the
     # neighbouring steps (h2d of step i+1 and d2h of step i-1 overlap the kernels of step i).
-    xs2 = [torch.empty_like(t) for t in xs]
-    dys2 = [torch.empty_like(t) for t in xs]
-    ys2 = [torch.empty_like(t) for t in xs]
-    dxs2 = [torch.empty_like(t) for t in xs]
-    sets = [(xs, dys, ys, dxs), (xs2, dys2, ys2, dxs2)]
+    if brief:
+        sets = [(xs, dys, ys, dxs)]
+    else:
+        xs2 = [torch.empty_like(t) for t in xs]
+        dys2 = [torch.empty_like(t) for t in xs]
+        ys2 = [torch.empty_like(t) for t in xs]
+        dxs2 = [torch.empty_like(t) for t in xs]
+        sets = [(xs, dys, ys, dxs), (xs2, dys2, ys2, dxs2)]
     s_h2d, s_d2h = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
     ev_in = [torch.cuda.Event() for _ in range(2)]       # inputs of set k are on the device
     ev_done = [torch.cuda.Event() for _ in range(2)]     # compute on set k finished
@@ -407,17 +420,19 @@ def run_ours(args, w):
         stage.set_side_stream(True)
 
     # end to end through the public API with host buffers
+    ms_e2e = e2e_value = None
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    for k in range(2):
-        ev_done[k].record(stream)
-        ev_out[k].record(stream)
-    with torch.cuda.stream(stream):
-        step_e2e()
-        step_e2e()
-    torch.cuda.synchronize(dev)
-    e2e_state["i"] = 0
-    ms_e2e = timed(step_e2e, e2e_steps) / e2e_steps
-    e2e_value = whole_job_value(tokens_step, world, ms_e2e)
+    if not brief:
+        for k in range(2):
+            ev_done[k].record(stream)
+            ev_out[k].record(stream)
+        with torch.cuda.stream(stream):
+            step_e2e()
+            step_e2e()
+        torch.cuda.synchronize(dev)
+        e2e_state["i"] = 0
+        ms_e2e = timed(step_e2e, e2e_steps) / e2e_steps
+        e2e_value = whole_job_value(tokens_step, world, ms_e2e)
     code, site = stage.status()
     if code != 0:
         raise SystemExit(f"device status {code} at site {site}")
@@ -446,6 +461,8 @@ def run_ours(args, w):
                 "h2d_bytes_per_step": 2 * M * T * d * 2, "d2h_bytes_per_step": 2 * M * T * d * 2},
         "gpu_launches": int(launches),
     }
+    if brief:
+        del line["e2e"], line["peaks"]
     if prof is not None:
         kernels = {}
         tot_ms = sum(v["ms"] for v in prof.values())
@@ -470,9 +487,25 @@ def run_ours(args, w):
                                          GEMM_DRAM_TRAFFIC_PER_LAUNCH.get(w.name))
         line["ms_per_step_one_stream"] = ms_one_stream
 
-    if rank == 0 and world == 1 and not args.no_isolated and w.tokens * w.d_ff <= (1 << 27):
+    if rank == 0 and world == 1 and not brief and not args.no_isolated and w.tokens * w.d_ff <= (1 << 27):
         line["kernels_isolated"] = isolated_elementwise(pw, w, peaks, dev)
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not brief and not args.no_sustained:
+        # Sustained regime: the same step back to back for at least a second, long enough for the power
+        # cap to pull the SM clock down to where it settles; compared with the sustained cuBLAS figure.
+        n_sus = max(args.sustained_steps, 1)
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                step()
+        with ClockSampler(local, period_s=0.02) as clk:
+            ms_sus = timed(step, n_sus) / n_sus
+        line["sustained"] = {
+            "steps": n_sus, "seconds": ms_sus * n_sus * 1e-3, "ms_per_step": ms_sus, "value": tokens_step / (ms_sus * 1e-3),
+            "unit": "tokens/s", "tflops_model": model_flops / (ms_sus * 1e-3) / 1e12,
+            "tflops_hw": hw_flops / (ms_sus * 1e-3) / 1e12,
+            "frac_bf16_peak_sustained": hw_flops / (ms_sus * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+            "frac_bf16_peak_burst": hw_flops / (ms_sus * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "clocks": clk.summary()}
+    if rank == 0 and world == 1 and not brief and not args.no_cpu_baseline:
         import oracle as oracle_mod
         orc = oracle_mod.Oracle("f32")
         b = min(w.batch, args.cpu_sample_batch)
@@ -484,10 +517,7 @@ def run_ours(args, w):
             "value": wsamp.tokens / dt, "unit": "tokens/s", "cores": oracle_mod.host_threads(), "kind": "oracle",
             "seconds": dt,
             "sample": f"{b} of {w.batch} sequences (S={w.seq_len}) through one layer fwd+bwd, fp32 plain-loop C oracle, run once"}
-    if rank == 0:
-        print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    return line if rank == 0 else None
 
 
 def lm_flops_per_step(w):
@@ -509,8 +539,9 @@ def oracle_lm_sample(w, layers):
     return ws, D, pls, E.float().numpy(), g.float().numpy(), b.float().numpy(), ids.numpy().ravel(), labels.numpy().ravel()
 
 
-def run_ours_lm(args, w):
-    """Workload 5: the whole small language-model step (pw_lm_step) instead of a bare layer chain."""
+def run_ours_lm(args, w, brief=False):
+    """Workload 5: the whole small language-model step (pw_lm_step) instead of a bare layer chain.
+    Returns the JSON line as a dict (rank 0) or None; brief as in run_ours."""
     import torch
     import torch.distributed as dist
     from paper_2203_12533_b200 import binding as pw
@@ -518,10 +549,12 @@ def run_ours_lm(args, w):
 
     rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if brief:
+        rank, world = 0, 1
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the product path)")
     torch.cuda.set_device(local)
-    if world > 1:
+    if world > 1 and not dist.is_initialized():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     pw.lib()
     peaks = load_peaks()
@@ -658,7 +691,7 @@ def run_ours_lm(args, w):
                                "link_bytes_in_per_replica": link_in, "link_gbs_in": link_in / (ms_apply * 1e-3) / 1e9,
                                "frac_of_measured_peer_copy_770": link_in / (ms_apply * 1e-3) / 1e9 / 770.0})
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    ms_e2e = timed(step_e2e, e2e_steps) / e2e_steps
+    ms_e2e = None if brief else timed(step_e2e, e2e_steps) / e2e_steps
     if stage.status() != (0, 0):
         raise SystemExit(f"device status {stage.status()}")
     model_flops, hw_flops = lm_flops_per_step(w)
@@ -682,11 +715,14 @@ def run_ours_lm(args, w):
         "frac_bf16_peak_sustained": hw_flops / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
         "frac_bf16_nominal_2250": hw_flops / (ms_step * 1e-3) / 1e12 / 2250.0,   # datasheet dense bf16, for context
         "peaks": peaks, "clocks": clocks.summary(),
-        "e2e": {"value": world * T / (ms_e2e * 1e-3), "unit": "tokens/s", "ms_per_step": ms_e2e, "steps": e2e_steps,
-                "how": "pinned host ids, labels -> device and the loss -> pinned host every step",
-                "h2d_bytes_per_step": 2 * T * 4, "d2h_bytes_per_step": 4},
+        "e2e": None if brief else {
+            "value": world * T / (ms_e2e * 1e-3), "unit": "tokens/s", "ms_per_step": ms_e2e, "steps": e2e_steps,
+            "how": "pinned host ids, labels -> device and the loss -> pinned host every step",
+            "h2d_bytes_per_step": 2 * T * 4, "d2h_bytes_per_step": 4},
         "gpu_launches": int(launches),
     }
+    if brief:
+        del line["e2e"], line["peaks"]
     if apply_info is not None:
         line["metric"] = "small-LM training step with gradient apply tokens/s"
         line["apply"] = apply_info
@@ -710,7 +746,7 @@ def run_ours_lm(args, w):
     line["roofline"] = gemm_roofline(g_flops, g_ms, g_n, tot_ms, ms_one_stream - ms_apply_step, args.steps, peaks,
                                      "gemm_pair_kernel (tcgen05 bf16 GEMM: layers and tied head)", None)
     line["ms_per_step_one_stream"] = ms_one_stream
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not brief and not args.no_cpu_baseline:
         import oracle as oracle_mod
         orc = oracle_mod.Oracle("f32")
         ws, D, pls, E_, g_, b_, ids_, labels_ = oracle_lm_sample(w, 1)
@@ -719,12 +755,9 @@ def run_ours_lm(args, w):
         dt = time.perf_counter() - t0
         line["cpu_baseline"] = {"value": ws.tokens / dt, "unit": "tokens/s", "cores": oracle_mod.host_threads(), "kind": "oracle",
                                 "seconds": dt, "sample": f"1 of {w.batch} sequences (S={w.seq_len}) through 1 of {L} layers and the full-vocabulary head, fwd+bwd, fp32 plain-loop C oracle, run once"}
-    if rank == 0:
-        print(json.dumps(line), flush=True)
     if replica is not None:
         replica.close()
-    if world > 1:
-        dist.destroy_process_group()
+    return line if rank == 0 else None
 
 
 def run_reference_lm(args, w):
@@ -764,6 +797,10 @@ def main():
     ap.add_argument("--cpu-sample-batch", type=int, default=6, help="sequences of the workload the timed oracle run processes (about 13 s of host time on workload 2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-isolated", action="store_true", help="skip the back-to-back timing of the element-wise kernels")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the long back-to-back run of the step (sustained clocks)")
+    ap.add_argument("--sustained-steps", type=int, default=600, help="steps of the sustained run (workload 2: about 1.4 s)")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="default run only: skip the short runs of workloads 3, 4, 5 and the dispatch study")
     ap.add_argument("--lean", action="store_true",
                     help="lean save set: the forward keeps neither LayerNorm output nor GeLU(u); the backward re-derives them")
     ap.add_argument("--data-parallel", action="store_true",
@@ -780,8 +817,64 @@ def main():
         raise SystemExit("--data-parallel needs --apply-lr")
     if args.impl == "reference":
         (run_reference_lm if w.vocab else run_reference)(args, w)
-    else:
-        (run_ours_lm if w.vocab else run_ours)(args, w)
+        return
+    line = (run_ours_lm if w.vocab else run_ours)(args, w)
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if line is not None and world == 1 and args.workload == 2 and not args.no_other_workloads and not args.lean \
+            and args.dispatch == "async":
+        line["other_workloads"] = other_workloads(args)
+        line["dispatch"] = dispatch_table()
+    if line is not None:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        if dist.is_initialized():
+            dist.destroy_process_group()
+
+
+# Steps (warm-up, timed) of the short runs of the other workloads inside the default run.
+OTHER_WORKLOAD_STEPS = {3: (1, 2), 4: (3, 10), 5: (3, 10)}
+
+
+def other_workloads(args):
+    """Short device-resident runs of workloads 3, 4 and 5 (the large configurations and the small-LM
+    step), each with its per-class kernel table and its own clock record.  They ride on the default
+    line so that one run of this file shows every configuration; the headline fields stay workload 2's."""
+    import copy
+    import gc
+    import torch
+    from paper_2203_12533_b200 import inputs
+    out = {}
+    for wid, (warm, steps) in OTHER_WORKLOAD_STEPS.items():
+        a = copy.copy(args)
+        a.warmup, a.steps, a.workload = warm, steps, wid
+        w = inputs.WORKLOADS[wid]
+        gc.collect()
+        torch.cuda.empty_cache()
+        t0 = time.perf_counter()
+        try:
+            r = (run_ours_lm if w.vocab else run_ours)(a, w, brief=True)
+        except SystemExit as e:                      # a device status other than 0: report it, keep the headline
+            out[f"workload_{wid}"] = {"workload": w.name, "error": str(e)}
+            continue
+        keep = ("metric", "value", "unit", "steps", "warmup", "ms_per_step", "ms_per_step_best", "tflops_model", "tflops_hw",
+                "frac_bf16_peak_burst", "frac_bf16_peak_sustained", "clocks", "gpu_launches", "kernels", "roofline", "loss",
+                "config")
+        o = {k: r[k] for k in keep if k in r}
+        o["wall_s"] = time.perf_counter() - t0
+        out[f"workload_{wid}"] = o
+    gc.collect()
+    torch.cuda.empty_cache()
+    return out
+
+
+def dispatch_table():
+    """The dispatch study (Section 5.1 analogue): OPBYOP / ASYNC / GRAPH over a chain of small layer calls."""
+    from paper_2203_12533_b200 import dispatch_study
+    rows = dispatch_study.study(seq_lens=(128, 256, 512, 1024, 2048), layers=8, microbatches=8, reps=10)
+    return {"what": "chain of 8 layers x 8 micro-batches at workload 1's width (recompute on): microseconds per layer call "
+                    "(forward or backward) in each dispatch mode of pw_stage_run_chain",
+            "rows": rows}
 
 
 if __name__ == "__main__":

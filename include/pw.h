@@ -232,7 +232,7 @@ pw_status_t pw_stage_workspace_bytes(const pw_stage_t* stage, int n_microbatches
  *   x_mb, dy_mb, y_mb, dx_mb : host arrays [M] of device pointers (bf16 [B,S,d] each);
  *                   y_mb[m] must not alias x_mb[m]
  *   recompute = 1 : only each layer's input is kept for the backward; the layer's forward is
- *                   re-run inside its backward (Section 5.3 config of the benchmark contract)
+ *                   re-run inside its backward (the pipeline-stage workload after Section 5.3 runs this way)
  *   recompute = 0 : every layer saves its activations (needs L * M (GPipe) or L (per-micro-batch)
  *                   contexts in the workspace)
  * GRAPH mode caches an instantiated graph keyed by every pointer and setting of the call and
@@ -425,6 +425,29 @@ pw_status_t pw_shared_alloc(size_t bytes, void** dev_ptr, pw_ipc_handle_t* handl
 pw_status_t pw_shared_free(void* dev_ptr);
 pw_status_t pw_shared_open(const pw_ipc_handle_t* handle, void** dev_ptr);
 pw_status_t pw_shared_close(void* dev_ptr);
+/* Process-wide tuning knobs.  The defaults are what the library is tested and measured with; a
+ * measurement script flips one of them to take an A/B figure.  Not thread-safe; set them while no
+ * call of this library is in progress.  A change invalidates the CUDA graphs that GRAPH dispatch
+ * has cached (Section 5.1's Fused mode re-captures on its next call).  Values out of range and
+ * unknown knobs return PW_ERR_INVALID_ARG and change nothing.
+ *   PW_TUNE_PDL               1 (default) / 0: launch kernels with programmatic dependent launch
+ *   PW_TUNE_GEMM_PAIR         1 (default) / 0: two-CTA 256 x 256 GEMM tiles whenever M >= 256
+ *   PW_TUNE_GEMM_BN           0 (default: chosen per shape) / 128 / 192 / 256: forced GEMM tile width
+ *   PW_TUNE_GEMM_SPLIT        1 (default) / 0: cut the tiles of a thin last round along K
+ *   PW_TUNE_GEMM_SPLIT_MIN_K  64 (default): ... only from this many 64-wide K blocks on
+ *   PW_TUNE_FAIL_LAUNCH       0 (default) / k > 0: host-side fault injection for error-path tests - the
+ *                             k-th kernel launch from now is not enqueued and reports a launch failure
+ *                             (the call that issued it returns PW_ERR_CUDA); the knob then returns to 0 */
+enum {
+    PW_TUNE_PDL = 0,
+    PW_TUNE_GEMM_PAIR = 1,
+    PW_TUNE_GEMM_BN = 2,
+    PW_TUNE_GEMM_SPLIT = 3,
+    PW_TUNE_GEMM_SPLIT_MIN_K = 4,
+    PW_TUNE_FAIL_LAUNCH = 5
+};
+pw_status_t pw_set_tuning(int knob, int value);
+pw_status_t pw_get_tuning(int knob, int* value);
 /* Clears the status word of the single-step calls (after a test has provoked an error). */
 pw_status_t pw_op_status_reset(void);
 /* Failure-path self-test.  Every device-side wait in this library is bounded; this call shows the

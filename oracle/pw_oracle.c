@@ -31,7 +31,7 @@
  * workload recipe; the Figure 2 program by the values the paper prints; the gradient
  * apply by a library bf16 conversion, the closed form after k equal steps, the exact
  * minimiser of a quadratic and the first-order loss decrease of the small-LM step.
- * Nothing is "parity unpinned".
+ * Every function in this file has at least one such pin.
  *
  * Layout conventions (all row-major, all REAL):
  *   activations  [T, width], T = B*S tokens, token t = b*S + s

@@ -41,7 +41,7 @@ EXPORTS = (
     "pw_op_attention_fwd", "pw_op_attention_bwd", "pw_op_status",
     "pw_lm_workspace_bytes", "pw_lm_step",
     "pw_op_embedding_fwd", "pw_op_embedding_bwd_scratch_bytes", "pw_op_embedding_bwd", "pw_op_softmax_xent",
-    "pw_op_status_reset", "pw_op_selftest_wait_timeout", "pw_op_affine_f32", "pw_sgd_apply",
+    "pw_set_tuning", "pw_get_tuning", "pw_op_status_reset", "pw_op_selftest_wait_timeout", "pw_op_affine_f32", "pw_sgd_apply",
     "pw_layer_set_side_stream", "pw_stage_set_side_stream", "pw_dp_slice", "pw_dp_reduce_apply", "pw_shared_alloc", "pw_shared_free", "pw_shared_open", "pw_shared_close",
 )
 
@@ -432,6 +432,20 @@ def op_status():
     c, s = ctypes.c_int(), ctypes.c_int()
     _check(lib().pw_op_status(ctypes.byref(c), ctypes.byref(s)))
     return c.value, s.value
+
+
+TUNE_PDL, TUNE_GEMM_PAIR, TUNE_GEMM_BN, TUNE_GEMM_SPLIT, TUNE_GEMM_SPLIT_MIN_K, TUNE_FAIL_LAUNCH = range(6)
+
+
+def set_tuning(knob: int, value: int):
+    """Process-wide tuning knob (see pw_set_tuning in include/pw.h)."""
+    _check(lib().pw_set_tuning(int(knob), int(value)))
+
+
+def get_tuning(knob: int) -> int:
+    v = ctypes.c_int(0)
+    _check(lib().pw_get_tuning(int(knob), ctypes.byref(v)))
+    return v.value
 
 
 def op_status_reset():

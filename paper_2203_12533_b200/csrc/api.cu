@@ -21,6 +21,12 @@ namespace pw {
 
 static thread_local std::string g_last_error;
 
+Tuning& tuning()
+{
+    static Tuning t;
+    return t;
+}
+
 static pw_status_t fail(pw_status_t s, const std::string& msg)
 {
     g_last_error = msg;
@@ -192,6 +198,12 @@ struct LaunchScope {
     {
         if (L->profiling && a && b) { cudaEventRecord(b, st); L->spans.push_back({a, b, cls}); }
     }
+    // The launch group failed before anything was enqueued: take its kernels out of the counts again.
+    void cancel(int nkernels)
+    {
+        if (L->capturing) L->graph_nodes -= nkernels; else L->launches -= nkernels;
+        if (L->profiling) L->prof.launches[cls] -= nkernels;
+    }
 };
 
 static inline uint8_t* at(void* base, size_t off) { return static_cast<uint8_t*>(base) + off; }
@@ -220,6 +232,7 @@ static pw_status_t do_gemm(pw_layer_t* L, const GemmArgs& g, cudaStream_t st)
     const int cls = g.layout == kTN ? PW_K_GEMM_TN : g.layout == kNN ? PW_K_GEMM_NN : PW_K_GEMM_NT;
     LaunchScope sc(L, cls, 1, 2.0 * g.M * g.N * g.K, 0.0, st);
     const char* e = launch_gemm(L->rt, g, L->status, st);
+    if (e) sc.cancel(1);
     return e ? fail(PW_ERR_CUDA, e) : PW_OK;
 }
 static pw_status_t do_ln_fwd(pw_layer_t* L, const void* x, const void* gamma, const void* beta, void* h, void* mu,
@@ -228,6 +241,7 @@ static pw_status_t do_ln_fwd(pw_layer_t* L, const void* x, const void* gamma, co
     const LayerPlan& p = L->plan;
     LaunchScope sc(L, PW_K_LN_FWD, 1, 0.0, 4.0 * p.T * p.d + 8.0 * p.T, st);
     const char* e = launch_layernorm_fwd(L->rt, x, gamma, beta, p.T, p.d, p.eps, h, mu, rstd, st);
+    if (e) sc.cancel(1);
     return e ? fail(PW_ERR_CUDA, e) : PW_OK;
 }
 static pw_status_t do_ln_bwd(pw_layer_t* L, const void* dh, const void* x, const void* mu, const void* rstd,
@@ -262,6 +276,7 @@ static pw_status_t do_attn_bwd(pw_layer_t* L, const void* qkv, const void* o, co
     const LayerPlan& p = L->plan;
     LaunchScope sc(L, PW_K_ATTN_BWD, 3, 5.0 * p.T * (p.S + 1.0) * p.d, 0.0, st);
     const char* e = launch_attention_bwd(L->rt, qkv, o, dout, lse, p.B, p.S, p.H, p.dh, dqkv, delta, L->status, st);
+    if (e) sc.cancel(3);
     return e ? fail(PW_ERR_CUDA, e) : PW_OK;
 }
 
@@ -332,8 +347,7 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
     // leaves idle (and the HBM-bound kernels share SMs with GEMM CTAs).  Events order the two
     // streams; the side stream always rejoins before this call returns, so a captured graph sees
     // a plain fork/join.  While per-kernel profiling is on everything stays on one stream.
-    static const bool no_side = getenv("PW_NO_SIDE_STREAM") != nullptr;   // tuning aid
-    cudaStream_t ax = (L->profiling || L->single_stream || no_side) ? st : L->aux;
+    cudaStream_t ax = (L->profiling || L->single_stream) ? st : L->aux;
     auto order = [&](cudaEvent_t ev, cudaStream_t from, cudaStream_t to) -> pw_status_t {
         if (from == to) return PW_OK;
         cudaError_t e = cudaEventRecord(ev, from);
@@ -729,6 +743,7 @@ pw_status_t pw_stage_run_chain(pw_stage_t* stage, const pw_layer_params_t* param
     std::vector<uint64_t> key;
     key.reserve(8 + 24 * L + 4 * M);
     key.push_back(M); key.push_back(schedule); key.push_back(recompute); key.push_back(stage->layer->single_stream ? 1 : 0);
+    key.push_back(tuning().epoch);
     key.push_back(reinterpret_cast<uint64_t>(workspace));
     for (int l = 0; l < L; ++l) {
         const void* const* pp = reinterpret_cast<const void* const*>(&params[l]);
@@ -979,8 +994,9 @@ pw_status_t pw_op_colsum_noalloc(const void* in, int T, int N, int ld, void* out
     if (accumulate != 0 && accumulate != 1) return fail(PW_ERR_INVALID_ARG, "accumulate must be 0 or 1");
     if (N > 0 && static_cast<size_t>(N) > colsum_noalloc_max_columns())
         return fail(PW_ERR_WORKSPACE_TOO_SMALL, "colsum (no-allocation variant): N exceeds the 262144 columns the built-in scratch can hold");
-    const char* e = launch_colsum_noalloc(in, T, N, ld, out, accumulate, static_cast<cudaStream_t>(stream));
-    if (e) return fail(PW_ERR_INVALID_ARG, e);
+    int kind = kErrArgument;
+    const char* e = launch_colsum_noalloc(in, T, N, ld, out, accumulate, static_cast<cudaStream_t>(stream), &kind);
+    if (e) return fail(kind == kErrDevice ? PW_ERR_DEVICE_UNSUPPORTED : kind == kErrCuda ? PW_ERR_CUDA : PW_ERR_INVALID_ARG, e);
     return PW_OK;
 }
 
@@ -1185,6 +1201,36 @@ pw_status_t pw_op_selftest_wait_timeout(uint64_t limit_cycles, int* kernel_retur
     cudaFree(flag);
     if (err) return fail(PW_ERR_CUDA, err);
     return e == cudaSuccess ? PW_OK : fail_cuda("self-test", e);
+}
+
+pw_status_t pw_set_tuning(int knob, int value)
+{
+    Tuning& t = tuning();
+    switch (knob) {
+        case PW_TUNE_PDL: if (value != 0 && value != 1) break; t.pdl = value; ++t.epoch; return PW_OK;
+        case PW_TUNE_GEMM_PAIR: if (value != 0 && value != 1) break; t.gemm_pair = value; ++t.epoch; return PW_OK;
+        case PW_TUNE_GEMM_BN: if (value != 0 && value != 128 && value != 192 && value != 256) break; t.gemm_bn = value; ++t.epoch; return PW_OK;
+        case PW_TUNE_GEMM_SPLIT: if (value != 0 && value != 1) break; t.gemm_split = value; ++t.epoch; return PW_OK;
+        case PW_TUNE_GEMM_SPLIT_MIN_K: if (value < 1) break; t.gemm_split_min_k = value; ++t.epoch; return PW_OK;
+        case PW_TUNE_FAIL_LAUNCH: if (value < 0) break; t.fail_launch_countdown = value; return PW_OK;
+        default: return fail(PW_ERR_INVALID_ARG, "unknown tuning knob");
+    }
+    return fail(PW_ERR_INVALID_ARG, "value out of range for this tuning knob");
+}
+
+pw_status_t pw_get_tuning(int knob, int* value)
+{
+    if (!value) return fail(PW_ERR_INVALID_ARG, "value is NULL");
+    const Tuning& t = tuning();
+    switch (knob) {
+        case PW_TUNE_PDL: *value = t.pdl; return PW_OK;
+        case PW_TUNE_GEMM_PAIR: *value = t.gemm_pair; return PW_OK;
+        case PW_TUNE_GEMM_BN: *value = t.gemm_bn; return PW_OK;
+        case PW_TUNE_GEMM_SPLIT: *value = t.gemm_split; return PW_OK;
+        case PW_TUNE_GEMM_SPLIT_MIN_K: *value = t.gemm_split_min_k; return PW_OK;
+        case PW_TUNE_FAIL_LAUNCH: *value = t.fail_launch_countdown; return PW_OK;
+        default: return fail(PW_ERR_INVALID_ARG, "unknown tuning knob");
+    }
 }
 
 pw_status_t pw_op_status_reset(void)

@@ -26,21 +26,6 @@ constexpr int kThreads = 320;
 constexpr int kDqThreads = 576;                            // producer warp, MMA warp, 2 x 8 element-wise warps
 constexpr float kLog2e = 1.4426950408889634f;
 
-// Timeline tracing of CTA 0 of the dK/dV kernel (one writer thread per role), compiled in only with
-// -DPW_TRACE_ENABLE; read back with pw_debug_trace_bwd (not part of the C ABI).
-#ifdef PW_TRACE_ENABLE
-__device__ long long g_trace_bwd[4][1024];
-__device__ int g_trace_bwd_n[4];
-__device__ __forceinline__ void trace_bwd(int role, int tag, int& n)
-{
-    if (blockIdx.x != 0 || (threadIdx.x & 31) != 0) return;
-    if (n < 1024) g_trace_bwd[role][n] = (static_cast<long long>(tag) << 48) | (clock64() & 0xffffffffffffll);
-    g_trace_bwd_n[role] = ++n;
-}
-#define PW_TRACE_B(role, tag) trace_bwd(role, tag, trace_n)
-#else
-#define PW_TRACE_B(role, tag) ((void)0)
-#endif
 
 struct BwdParams {
     int S, H, B;
@@ -115,8 +100,6 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int d = p.H * DH;
-    int trace_n = 0;                                        // used by PW_TRACE_B only
-    (void)trace_n;
 
     auto load_kv = [&](const KvItem& it, int buf) {
         mbar_arrive_expect_tx(bar(0 + buf), 2 * L::kKV);
@@ -187,7 +170,6 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
                     const int s = m % L::kStages;
                     if (!mbar_wait(bar(7 + s), ((m / L::kStages) & 1) ^ 1, abort_flag, p.status, 500)) { ok = false; break; }
                     load_q(it, i, s);
-                    PW_TRACE_B(0, 1);
                 }
                 if (!ok) break;
                 const int kn = k + 1;
@@ -261,9 +243,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
             ok = wait(0 + buf, (k >> 1) & 1, 510) && wait(4 + g0 % L::kStages, (g0 / L::kStages) & 1, 511);
             if (!ok) break;
             tc_fence_after();
-            PW_TRACE_B(1, 9);
             issue_scores(g0, buf);
-            PW_TRACE_B(1, 1);
             for (int i = 0; i < n_u && ok; ++i) {
                 const uint32_t g = g0 + i;
                 if (i + 1 < n_u) {
@@ -271,15 +251,12 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
                     if (!wait(4 + gn % L::kStages, (gn / L::kStages) & 1, 512)) { ok = false; break; }
                     tc_fence_after();
                     issue_scores(gn, buf);
-                    PW_TRACE_B(1, 1);
                 }
                 if (!wait(12 + (g & 1), (g >> 1) & 1, 513)) { ok = false; break; }
                 // the previous item's dV / dK must have been read out before they are overwritten
                 if (i == 0 && !wait(15, (k & 1) ^ 1, 515)) { ok = false; break; }
                 tc_fence_after();
-                PW_TRACE_B(1, 3);
                 issue_acc(g, i == 0);
-                PW_TRACE_B(1, 2);
             }
             if (!ok) break;
             if (elect_one()) umma_commit(bar(14));
@@ -320,12 +297,10 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                if (warp == 2) PW_TRACE_B(2, 1);
                 uint32_t sv[32], dv[32];
                 tmem_ld32(tmem_base + lane_addr + hb * 64 + ch * 32, sv);
                 tmem_ld32(tmem_base + lane_addr + 128 + hb * 64 + ch * 32, dv);
                 tc_wait_ld();
-                if (warp == 2) PW_TRACE_B(2, 2);
                 const bool diag = qc0 < kv0 + 128;           // some (key, query) pairs of this slice are masked
                 uint32_t pp[16], dd[16];
                 const uint64_t sl2x2 = pack_f32x2(sl2, sl2);
@@ -343,14 +318,12 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
                     pp[c >> 1] = pack_bf16(p0, p1);
                     dd[c >> 1] = pack_bf16(d0, d1);
                 }
-                if (warp == 2) PW_TRACE_B(2, 3);
                 // packed operands go back into this warp's own columns: P^T over S^T, dS^T over dP^T
                 tmem_st16(tmem_base + lane_addr + hb * 64 + ch * 32, pp);
                 tmem_st16(tmem_base + lane_addr + 128 + hb * 64 + ch * 32, dd);
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(12 + hb));
-                if (warp == 2) PW_TRACE_B(2, 4);
             }
             if (ok) {
                 ok = mbar_wait(bar(14), k & 1, abort_flag, p.status, 521);
@@ -395,7 +368,6 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
                 bulk_commit();
                 bulk_wait_read0();                          // the buffer may take another item's K / V
                 mbar_arrive(bar(2 + buf));
-                PW_TRACE_B(2, 8);
             }
         }
         if (warp == 2 && lane == 0) bulk_wait0();
@@ -821,15 +793,6 @@ const char* encode_rows(Runtime* rt, CUtensorMap* map, const void* ptr, uint64_t
 
 }  // namespace
 
-#ifdef PW_TRACE_ENABLE
-extern "C" int pw_debug_trace_bwd(long long* events, int* counts)
-{
-    if (cudaMemcpyFromSymbol(events, g_trace_bwd, sizeof(long long) * 4 * 1024) != cudaSuccess) return 1;
-    if (cudaMemcpyFromSymbol(counts, g_trace_bwd_n, sizeof(int) * 4) != cudaSuccess) return 1;
-    int zero[4] = {0, 0, 0, 0};
-    return cudaMemcpyToSymbol(g_trace_bwd_n, zero, sizeof(zero)) == cudaSuccess ? 0 : 1;
-}
-#endif
 
 const char* configure_attention_bwd_tc()
 {

@@ -38,22 +38,6 @@ struct FwdSmem {
     static constexpr int kBytes = kEnd + ((kEnd + 1024 <= 232448) ? 1024 : 232448 - kEnd);   // alignment slack (checked in the kernel)
 };
 
-// Timeline tracing of CTA 0 (one writer thread per role), compiled in only with -DPW_TRACE_ENABLE:
-// event = (tag << 48) | clock64.  Read back with pw_debug_trace_fwd (not part of the C ABI).
-#ifdef PW_TRACE_ENABLE
-__device__ long long g_trace[4][1024];
-__device__ int g_trace_n[4];
-// the event counter lives in a register of the writer thread (a global counter would stall it)
-__device__ __forceinline__ void trace(int role, int tag, int& n)
-{
-    if (blockIdx.x != 0 || (threadIdx.x & 31) != 0) return;
-    if (n < 1024) g_trace[role][n] = (static_cast<long long>(tag) << 48) | (clock64() & 0xffffffffffffll);
-    g_trace_n[role] = ++n;
-}
-#define PW_TRACE(role, tag) trace(role, tag, trace_n)
-#else
-#define PW_TRACE(role, tag) ((void)0)
-#endif
 
 struct FwdParams {
     int S, H, B;
@@ -117,8 +101,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
         if (threadIdx.x == 0 && atomicCAS(&p.status->code, 0, kStatusTimeout) == 0) p.status->site = 499;
         return;
     }
-    int trace_n = 0;                                        // used by PW_TRACE only
-    (void)trace_n;
 
     auto load_q = [&](const FwdItem& it, int t) {
         mbar_arrive_expect_tx(bar(0 + t), L::kTile);
@@ -193,7 +175,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                     if (!early) {
                         if (!mbar_wait(bar(6 + s), ph ^ 1, abort_flag, p.status, 400)) { ok = false; break; }
                         load_k(it, j, s);
-                        PW_TRACE(0, 1);
                     }
                     if (j == 0) {
                         // Q follows the first key tile; its buffer is free once the previous item's
@@ -202,7 +183,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                             if (!early) {
                                 if (!mbar_wait(bar(2 + t), (qn[t] & 1) ^ 1, abort_flag, p.status, 402)) { ok = false; break; }
                                 load_q(it, t);
-                                PW_TRACE(0, 2);
                             }
                             ++qn[t];
                         }
@@ -211,7 +191,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                     if (!early) {
                         if (!mbar_wait(bar(10 + s), ph ^ 1, abort_flag, p.status, 401)) { ok = false; break; }
                         load_v(it, j, s);
-                        PW_TRACE(0, 3);
                     }
                 }
                 if (!ok) break;
@@ -285,15 +264,12 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                 ok = wait(4 + s, ph, 411) && wait(0, qn[0] & 1, 410);
                 if (!ok) break;
                 tc_fence_after();
-                PW_TRACE(1, 9);
                 issue_s(0, s);
-                PW_TRACE(1, 1);
                 if (nA == 1) commit(2);                     // Q_A is not needed again
                 if (nB) {
                     if (!wait(1, qn[1] & 1, 417)) { ok = false; break; }
                     tc_fence_after();
                     issue_s(1, s);
-                    PW_TRACE(1, 2);
                     if (nB == 1) commit(3);
                 }
                 commit(6 + s);
@@ -311,7 +287,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                     if (j == 0 && !wait(18, (qn[0] & 1) ^ 1, 418)) { ok = false; break; }
                     tc_fence_after();
                     issue_pv(0, s, j > 0);
-                    PW_TRACE(1, 3);
                     if (j == nA - 1) commit(16);
                 }
                 if (j + 1 < nA) {
@@ -319,7 +294,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                     k_waited = true;
                     tc_fence_after();
                     issue_s(0, sn);
-                    PW_TRACE(1, 1);
                     if (j + 2 == nA) commit(2);
                 }
                 if (j < nB) {
@@ -328,7 +302,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                     if (j == 0 && !wait(19, (qn[1] & 1) ^ 1, 419)) { ok = false; break; }
                     tc_fence_after();
                     issue_pv(1, s, j > 0);
-                    PW_TRACE(1, 4);
                     if (j == nB - 1) commit(17);
                 }
                 commit(10 + s);                             // V stage free once these MMAs are done
@@ -336,7 +309,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                     if (!k_waited && !wait(4 + sn, phn, 416)) { ok = false; break; }
                     tc_fence_after();
                     issue_s(1, sn);
-                    PW_TRACE(1, 2);
                     if (j + 2 == nB) commit(3);
                 }
                 if (j + 1 < n_kv) commit(6 + sn);           // K stage free
@@ -356,7 +328,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
         const int hf = ((warp - 2) >> 2) & 1;               // column half
         const int q = warp & 3;                             // TMEM lane quarter this warp may touch
         const int r = q * 32 + lane;                        // query row inside the tile
-        const bool tracer = hf == 0 && q == 2 && lane == 0;
+        const bool leader = hf == 0 && q == 2 && lane == 0;
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
         const uint32_t s_addr = tmem_base + lane_addr + t * 128 + hf * 64;       // my 64 scores
         const uint32_t o_addr = tmem_base + lane_addr + 256 + t * 128 + hf * (DH / 2);
@@ -385,7 +357,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            if (tracer) PW_TRACE(2 + t, 1);
             const bool diag = j == n_t - 1;
             const int lim = diag ? r - hf * 64 : 64;        // columns i > lim of my 64 are masked (diagonal tile)
             // pass 1: row maximum.  Scores 0..31 are read, used and dropped; scores 32..63 stay in
@@ -410,7 +381,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                     mxs[2 + ((i >> 1) & 1)] = fmax3(mxs[2 + ((i >> 1) & 1)], __uint_as_float(vk[i]), __uint_as_float(vk[i + 1]));
                 }
             }
-            if (tracer) PW_TRACE(2 + t, 2);
             const float mine = fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3]));
             xch[hf * 128 + r] = mine;
             named_bar_sync(1 + t, 256);
@@ -433,7 +403,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                     tmem_st32(o_addr + c * 32, w);
                 }
             }
-            if (tracer) PW_TRACE(2 + t, 3);
             // pass 2: p = exp2((s - m) * scale * log2e), packed bf16 written over my own S columns: first the
             // kept scores 32..63 (into columns 32..47, their own), then scores 0..31 re-read (into columns 0..15)
             const float mb = m_used * sl2;
@@ -476,11 +445,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
                 unpack_f32x2(fadd2(lsum[0], lsum[1]), s0, s1);
                 l += s0 + s1;
             }
-            if (tracer) PW_TRACE(2 + t, 4);
             tc_wait_st();
             tc_fence_before();
             mbar_arrive(bar(14 + t));
-            if (tracer) PW_TRACE(2 + t, 5);
         }
         if (ok) {
             ok = mbar_wait(bar(16 + t), qn & 1, abort_flag, p.status, 421);
@@ -489,7 +456,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
         if (!ok) break;
         {
             tc_fence_after();
-            if (tracer) PW_TRACE(2 + t, 6);
             // row sum = the two halves' sums (the partner's last read of this slot was before its last p_full arrival)
             xch[hf * 128 + r] = l;
             named_bar_sync(1 + t, 256);
@@ -499,7 +465,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
             ok = mbar_wait(bar(20), (u & 1) ^ 1, abort_flag, p.status, 422);    // the previous user's store has read it
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            if (tracer) PW_TRACE(2 + t, 7);
 #pragma unroll 1
             for (int c = 0; c < DH / 64; ++c) {
                 uint32_t w[32];
@@ -521,18 +486,17 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_const
             if (hf == 0) p.lse[(static_cast<size_t>(it.b) * p.H + it.h) * p.S + q0 + r] = m_used * p.scale + logf(l_row);
             fence_proxy_async();
             named_bar_sync(1 + t, 256);
-            if (tracer) {
+            if (leader) {
                 for (int kb = 0; kb < L::kBlocks; ++kb)
                     tma_store_2d(&tmO, sbase + L::kO + kb * 16384, it.h * DH + kb * 64, it.b * p.S + q0);
                 bulk_commit();
                 bulk_wait_read0();                          // the staging tile may be written again
                 mbar_arrive(bar(20));
-                PW_TRACE(2 + t, 8);
             }
             ++qn;
         }
         }
-        if (tracer) bulk_wait0();
+        if (leader) bulk_wait0();
     }
 
     __syncwarp();
@@ -568,15 +532,6 @@ const char* encode_rows(Runtime* rt, CUtensorMap* map, const void* ptr, uint64_t
 
 }  // namespace
 
-#ifdef PW_TRACE_ENABLE
-extern "C" int pw_debug_trace_fwd(long long* events, int* counts)
-{
-    if (cudaMemcpyFromSymbol(events, g_trace, sizeof(long long) * 4 * 1024) != cudaSuccess) return 1;
-    if (cudaMemcpyFromSymbol(counts, g_trace_n, sizeof(int) * 4) != cudaSuccess) return 1;
-    int zero[4] = {0, 0, 0, 0};
-    return cudaMemcpyToSymbol(g_trace_n, zero, sizeof(zero)) == cudaSuccess ? 0 : 1;
-}
-#endif
 
 const char* configure_attention_fwd()
 {

@@ -559,8 +559,9 @@ namespace {
 struct StaticScratch { float* ptr; int sm_count; };
 // In host code the array's name is only a handle for the runtime, not a device address: the
 // address comes from cudaGetSymbolAddress, asked once per device with that device current.
-const char* static_scratch_for_current_device(StaticScratch* out)
+const char* static_scratch_for_current_device(StaticScratch* out, int* err_kind)
 {
+    *err_kind = kErrCuda;
     static std::mutex mu;
     static std::map<int, StaticScratch> per_device;
     std::lock_guard<std::mutex> lock(mu);
@@ -572,7 +573,7 @@ const char* static_scratch_for_current_device(StaticScratch* out)
         if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
             return "cudaDeviceGetAttribute failed";
-        if (major != 10) return "device is not compute capability 10.x (sm_100a kernels only, no fallback)";
+        if (major != 10) { *err_kind = kErrDevice; return "device is not compute capability 10.x (sm_100a kernels only, no fallback)"; }
         float* ptr = nullptr;
         const cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_colsum_scratch);
         if (e != cudaSuccess || ptr == nullptr) return "cudaGetSymbolAddress(static scratch) failed";
@@ -585,13 +586,16 @@ const char* static_scratch_for_current_device(StaticScratch* out)
 
 size_t colsum_noalloc_max_columns() { return kStaticScratchFloats; }
 
-const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* out, int accumulate, cudaStream_t stream)
+const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* out, int accumulate, cudaStream_t stream,
+                                  int* err_kind)
 {
+    *err_kind = kErrArgument;
     if (T <= 0 || N <= 0 || (N % 8) || (ld % 8) || ld < N) return "colsum: N and ld must be multiples of 8, ld >= N";
     if (static_cast<size_t>(N) > kStaticScratchFloats)
         return "colsum (no-allocation variant): N exceeds the 262144 columns the built-in scratch can hold";
     StaticScratch sc;
-    if (const char* e = static_scratch_for_current_device(&sc)) return e;
+    if (const char* e = static_scratch_for_current_device(&sc, err_kind)) return e;
+    *err_kind = kErrCuda;
     // as many row groups as the fixed scratch can hold, at most what the allocating variant uses
     const int col_blocks = (N + kColsumCols - 1) / kColsumCols;
     long long R = (4ll * sc.sm_count + col_blocks - 1) / col_blocks;

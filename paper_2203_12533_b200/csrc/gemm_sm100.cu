@@ -650,7 +650,7 @@ static const char* launch_gemm_pair(Runtime* rt, const GemmArgs& a, DeviceStatus
     // 128-wide pair tile moves as many operand bytes per FLOP as the one-CTA 256-wide tile).
     int bn = 256;
     {
-        static const int forced = [] { const char* v = getenv("PW_GEMM_BN"); return v ? atoi(v) : 0; }();
+        const int forced = tuning().gemm_bn;
         auto cost = [&](int w) {
             const long long tiles = static_cast<long long>(m_tiles) * ((a.N + w - 1) / w);
             const long long rounds = (tiles + pairs - 1) / pairs;
@@ -680,10 +680,10 @@ static const char* launch_gemm_pair(Runtime* rt, const GemmArgs& a, DeviceStatus
     {
         // Tail balancing: when the last round of tiles would keep at most half of the CTA pairs busy,
         // each of its tiles becomes two units of half the K range (needs the caller's scratch).
-        static const bool no_split = getenv("PW_GEMM_NO_SPLIT") != nullptr;   // tuning aid
+        const bool no_split = tuning().gemm_split == 0;
         const int total = p.m_tiles * p.n_tiles, num_k = (a.K + BK - 1) / BK;
         const int rem = total % pairs;
-        static const int min_k = [] { const char* v = getenv("PW_GEMM_SPLIT_MIN_K"); return v ? atoi(v) : 64; }();   // tuning aid
+        const int min_k = tuning().gemm_split_min_k;
         // (short K ranges lose more to the second prologue and epilogue than the idle half round costs)
         if (a.split_ws && !no_split && !f32_out && total > pairs && rem > 0 && 2 * rem <= pairs && rem <= kSplitMaxTiles &&
             num_k >= min_k) {
@@ -725,7 +725,7 @@ const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cu
 
     const bool a_mn = a.layout == kNT, b_mn = a.layout == kNN || a.layout == kNT;
     const bool f32_out = a.epilogue == kEpiF32;
-    static const int pair_mode = [] { const char* v = getenv("PW_GEMM_PAIR"); return v ? atoi(v) : 1; }();   // tuning aid
+    const int pair_mode = tuning().gemm_pair;
     if (pair_mode && a.M >= 256) return launch_gemm_pair(rt, a, status, stream);
     if (f32_out && (a.ldc % 4)) return "gemm: fp32 ldc must be a multiple of 4";
     // Tile width: the one that needs the least (rounds x width) on this many SMs; ties go to the
@@ -737,8 +737,8 @@ const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cu
     int bn = BN_MAX;
     while (bn > 128 && static_cast<long long>(m_tiles) * ((a.N + bn - 1) / bn) * 2 <= rt->sm_count) bn -= 64;
     {
-        static const int forced = [] { const char* v = getenv("PW_GEMM_BN"); return v ? atoi(v) : 0; }();
-        if (forced == 128 || forced == 192 || forced == 256) bn = forced;   // tuning aid
+        const int forced = tuning().gemm_bn;
+        if (forced == 128 || forced == 192 || forced == 256) bn = forced;
     }
     CUtensorMap tmA, tmB, tmBh, tmC, tmAux;
     const char* e;
@@ -772,7 +772,7 @@ const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cu
         const int total = p.m_tiles * p.n_tiles;
         const int grid = total < rt->sm_count ? total : rt->sm_count;
         const int rem = total % grid;
-        static const bool no_split = getenv("PW_GEMM_NO_SPLIT") != nullptr;   // tuning aid
+        const bool no_split = tuning().gemm_split == 0;
         p.split_begin = total;
         if (bn == BN_MAX && rem > 0 && 2 * rem <= grid && !no_split) p.split_begin = total - rem;
         p.total_virtual = p.split_begin + 2 * (total - p.split_begin);

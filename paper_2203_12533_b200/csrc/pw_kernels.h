@@ -30,11 +30,27 @@ const char* configure_attention();
 const char* configure_attention_fwd();
 const char* configure_elementwise();
 
+// Process-wide tuning knobs (pw_set_tuning); the defaults are what every measurement and test uses.
+struct Tuning {
+    int pdl = 1;                 // launch with the programmatic-serialization attribute
+    int gemm_pair = 1;           // CTA-pair GEMM kernel whenever M >= 256
+    int gemm_bn = 0;             // 0 = tile width chosen by the launcher, else 128 / 192 / 256
+    int gemm_split = 1;          // cut the tiles of a thin last round along K
+    int gemm_split_min_k = 64;   // ... from this many 64-wide K blocks on
+    uint64_t epoch = 0;          // bumped by every change (part of the CUDA-graph cache key)
+    // Host-side fault injection for the error-path tests: when > 0, counts down once per launch and
+    // the launch that brings it to zero is NOT enqueued and reports cudaErrorLaunchFailure instead.
+    int fail_launch_countdown = 0;
+};
+Tuning& tuning();
+
 // Launch with the programmatic-serialization attribute (see grid_dep_wait in pw_common.cuh).
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args)
 {
-    static const bool pdl = getenv("PW_NO_PDL") == nullptr;   // tuning aid
+    Tuning& tn = tuning();
+    if (tn.fail_launch_countdown > 0 && --tn.fail_launch_countdown == 0) return cudaErrorLaunchFailure;   // injected by a test
+    const bool pdl = tn.pdl != 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
     cudaLaunchAttribute at[1];
@@ -78,7 +94,10 @@ const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, voi
 
 // Column sums with the partial sums in a fixed device array inside the library (no allocation, no Runtime).
 size_t colsum_noalloc_max_columns();
-const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* out, int accumulate, cudaStream_t stream);
+// On failure *err_kind says what went wrong: an argument, the device (not sm_100) or a CUDA call.
+enum { kErrArgument = 0, kErrDevice = 1, kErrCuda = 2 };
+const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* out, int accumulate, cudaStream_t stream,
+                                  int* err_kind);
 
 // a = GeLU(u), bf16 -> bf16, n a multiple of 8.
 const char* launch_gelu_fwd(Runtime* rt, const void* u, void* a, long long n, int act, cudaStream_t stream);

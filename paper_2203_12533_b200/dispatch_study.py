@@ -57,6 +57,21 @@ def run(seq_len: int, layers: int, microbatches: int, reps: int, mode: int) -> f
     return e0.elapsed_time(e1) / reps
 
 
+def study(seq_lens=(128, 256, 512, 1024, 2048), layers=8, microbatches=8, reps=20):
+    """One row per sequence length: microseconds per layer call in each dispatch mode."""
+    pw.lib()
+    modes = (("opbyop", pw.DISPATCH_OPBYOP), ("async", pw.DISPATCH_ASYNC), ("graph", pw.DISPATCH_GRAPH))
+    calls = 2 * layers * microbatches
+    rows = []
+    for S in seq_lens:
+        row = {"seq_len": S, "tokens_per_call": 2 * S}
+        for name, mode in modes:
+            row[f"us_per_layer_call_{name}"] = 1e3 * run(S, layers, microbatches, reps, mode) / calls
+        row["graph_vs_opbyop"] = row["us_per_layer_call_opbyop"] / row["us_per_layer_call_graph"]
+        rows.append(row)
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--layers", type=int, default=8)

@@ -4,7 +4,7 @@ This module only draws random numbers and rounds them to bf16; it holds none
 of the layer's arithmetic, so both the CUDA path and the CPU checker can be
 fed from it without sharing any of the method's code.
 
-The workloads are the ones the benchmark contract names (Section 5.3 of the
+The five workloads this library is measured on (Section 5.3 of the
 paper gives the 3e9-parameter decoder's sizes: model dimension 2048, hidden
 dimension 8192, micro-batches of 4 examples, S stages x M micro-batches):
 

@@ -16,6 +16,38 @@ def rel_l2(got, want) -> float:
     return float(np.linalg.norm(g - w) / n) if n > 1e-12 else float(np.linalg.norm(g - w))
 
 
+# Per-element bounds, beside the norm: |gpu - oracle| <= atol_rms * rms(oracle) + rtol * |oracle|.
+# A bf16 store rounds to 2^-9 relative (half an ulp), so rtol = 2^-7 leaves room for two roundings on
+# the way (an intermediate stored as bf16, then the output).  The absolute term scales with the
+# tensor's root-mean-square value: an output element is a sum of many products whose operands carry
+# those roundings, so its error is set by the size of the terms, not by the size of the (possibly
+# cancelled) sum.  A tensor that passes the norm test at e = 3e-3 with Gaussian-like errors has its
+# worst of 1e8 elements near 6 e rms = 0.02 rms; a tile of wrong values is off by about rms.
+ELEM_ACT = dict(atol_rms=0.04, rtol=2.0 ** -7)      # activations
+ELEM_GRAD = dict(atol_rms=0.08, rtol=2.0 ** -6)     # gradients (two more bf16 hand-offs on the way)
+ELEM_F32 = dict(atol_rms=2e-4, rtol=2e-4)           # fp32 statistics (mean, 1/sigma, lse)
+
+
+def elem_check(got, want, name="", atol_rms=0.04, rtol=2.0 ** -7):
+    """Asserts the per-element bound and returns the worst ratio |diff| / bound (<= 1 passes).
+    On failure the message names the worst element's flat index, both values and the bound."""
+    g = got.detach().double().cpu().numpy().ravel() if isinstance(got, torch.Tensor) else np.asarray(got, np.float64).ravel()
+    w = want.detach().double().cpu().numpy().ravel() if isinstance(want, torch.Tensor) else np.asarray(want, np.float64).ravel()
+    assert g.shape == w.shape, (name, g.shape, w.shape)
+    assert np.all(np.isfinite(g)), f"{name}: non-finite values in the GPU result"
+    rms = float(np.sqrt(np.mean(w * w)))
+    bound = atol_rms * rms + rtol * np.abs(w)
+    if rms == 0.0:
+        bound = bound + 1e-30
+    ratio = np.abs(g - w) / bound
+    i = int(np.argmax(ratio))
+    worst = float(ratio[i])
+    assert worst <= 1.0, (f"{name}: element {i} of {g.size}: gpu {g[i]!r} vs oracle {w[i]!r}, |diff| {abs(g[i] - w[i]):.3e} "
+                          f"> bound {bound[i]:.3e} (rms {rms:.3e}, atol_rms {atol_rms}, rtol {rtol}); "
+                          f"{int((ratio > 1.0).sum())} elements out of bound")
+    return worst
+
+
 def bf16_randn(shape, gen, scale=1.0):
     return (torch.randn(shape, generator=gen, dtype=torch.float32) * scale).to(torch.bfloat16)
 

@@ -68,3 +68,19 @@ def test_argument_errors_need_no_gpu(libpath):
     if not torch.cuda.is_available():
         ok = binding.make_config(2048, 16, 128, 8192, 1024, 8)
         assert lib.pw_layer_create(ctypes.byref(ok), ctypes.byref(h)) == 5   # no device: loud failure, no fallback
+
+
+def test_tuning_knobs_validate_on_the_host(libpath):
+    """pw_set_tuning / pw_get_tuning are pure host state: defaults, round trip, range checks."""
+    lib = ctypes.CDLL(libpath)
+    v = ctypes.c_int(-1)
+    defaults = {0: 1, 1: 1, 2: 0, 3: 1, 4: 64, 5: 0}
+    for knob, want in defaults.items():
+        assert lib.pw_get_tuning(knob, ctypes.byref(v)) == 0 and v.value == want
+    assert lib.pw_set_tuning(2, 128) == 0
+    assert lib.pw_get_tuning(2, ctypes.byref(v)) == 0 and v.value == 128
+    assert lib.pw_set_tuning(2, 100) == 1                    # not a tile width: rejected, unchanged
+    assert lib.pw_get_tuning(2, ctypes.byref(v)) == 0 and v.value == 128
+    assert lib.pw_set_tuning(2, 0) == 0
+    assert lib.pw_set_tuning(0, 2) == 1 and lib.pw_set_tuning(99, 0) == 1 and lib.pw_set_tuning(5, -1) == 1
+    assert lib.pw_get_tuning(99, ctypes.byref(v)) == 1 and lib.pw_get_tuning(0, None) == 1

@@ -4,7 +4,21 @@ import pytest
 import torch
 
 from paper_2203_12533_b200 import inputs
-from tests.gpu_util import (ACT_TOL, GRAD_TOL, dims_of, make_layer, np64, rel_l2, run_layer_gpu)
+from tests.gpu_util import (ACT_TOL, GRAD_TOL, dims_of, elem_check, make_layer, np64, rel_l2, run_layer_gpu)
+
+# Element bounds for a whole layer.  Inside the layer the GPU path hands bf16 tensors from step to step
+# while the oracle keeps full precision, so an element differs by more than one output rounding: the
+# attention output of a position that sees only a few keys is as sensitive to the rounding of q and k as
+# a single softmax weight is (measured at workload-3 width: worst element 0.08 rms, 99.99 % below 0.04
+# rms, against 0.04 / 0.02 rms when the oracle is given the GPU's own qkv).  A mis-computed tile is off
+# by about one rms in every element, so these bounds still catch what the norm hides.  The single-step
+# tests (test_gpu_ops.py) use the tight bounds.
+LAYER_ACT = dict(atol_rms=0.2, rtol=2.0 ** -6)
+LAYER_GRAD = dict(atol_rms=0.3, rtol=2.0 ** -5)
+# statistics: a row mean is itself of size rms(x) / sqrt(d), and so is its error when x carries bf16
+# roundings - relative to the rms of the means that is a few 2^-9; 1 / sigma and lse move far less
+ELEM_STAT = dict(atol_rms=2e-3, rtol=2e-3)
+ELEM_MEAN = dict(atol_rms=2e-2, rtol=2e-3)
 
 pytestmark = pytest.mark.gpu
 
@@ -34,16 +48,22 @@ def check_layer_against_oracle(pw, oracle, w, random_ln=False, act=0, save_ctx=T
     yw, sv = oracle.layer_fwd(D, ps, cast(x))
     dxw, gw = oracle.layer_bwd(D, ps, cast(x), sv, cast(dy))
     errs = {"y": rel_l2(out["y"], yw)}
+    worst = {"y": elem_check(out["y"], yw, "y", **LAYER_ACT)}
     store = out["ctx"] if save_ctx else out["scratch"]
     for name in SAVED_BF16:
         errs[name] = rel_l2(layer.ctx_view(store, name), sv[name])
+        worst[name] = elem_check(layer.ctx_view(store, name), sv[name], name, **LAYER_ACT)
     for name in ("lse", "mu1", "r1", "mu2", "r2"):
         errs[name] = rel_l2(layer.ctx_view(store, name), sv[name])
+        worst[name] = elem_check(layer.ctx_view(store, name), sv[name], name, **(ELEM_MEAN if name.startswith("mu") else ELEM_STAT))
     gerrs = {"dx": rel_l2(out["dx"], dxw)}
+    worst["dx"] = elem_check(out["dx"], dxw, "dx", **LAYER_GRAD)
     for name, g, want in zip(pw.PARAM_NAMES, out["grads"], gw):
         gerrs["d" + name] = rel_l2(g, want)
+        worst["d" + name] = elem_check(g, want, "d" + name, **LAYER_GRAD)
     assert max(errs.values()) < ACT_TOL, errs
     assert max(gerrs.values()) < GRAD_TOL, gerrs
+    print("worst element ratios:", {k: round(v, 3) for k, v in worst.items()})
     return errs, gerrs
 
 
@@ -139,9 +159,9 @@ def test_wide_layers_at_reduced_token_count(pw, oracle32, d, H, F, S):
 
 
 # ------------------------------------------------------------------------------------------ stage chain
-def run_chain_gpu(pw, w, L, M, dispatch, schedule, recompute, seed=0):
+def run_chain_gpu(pw, w, L, M, dispatch, schedule, recompute, seed=0, random_ln=True):
     stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
-    params = [[p.cuda() for p in inputs.layer_params(w, seed, l, random_ln=True)] for l in range(L)]
+    params = [[p.cuda() for p in inputs.layer_params(w, seed, l, random_ln=random_ln)] for l in range(L)]
     grads = [[torch.full(p.shape, float("nan"), dtype=torch.float32, device="cuda") for p in ps] for ps in params]
     mbs = [inputs.microbatch(w, seed, m) for m in range(M)]
     xs = [x.cuda().view(-1, w.d_model) for x, _ in mbs]
@@ -246,6 +266,36 @@ def test_full_size_wide_layer_by_the_causal_prefix_property(pw, oracle32, wid):
     assert rel_l2(dx[:, :P, :].reshape(-1, w.d_model), dxw) < GRAD_TOL
     errs = {name: rel_l2(g, want) for name, g, want in zip(pw.PARAM_NAMES, out["grads"], gw)}
     assert max(errs.values()) < GRAD_TOL, errs
+
+
+def test_cfg4_full_size_parity(pw, oracle32):
+    """One layer of workload 4 at its full size (d = 8192, 64 x 128 heads, F = 32768, S = 2048, B = 1) against
+    the fp32 oracle: every saved tensor, every gradient, all 2048 positions (norm and element bounds).
+    The oracle needs about a minute and a half on 16 host cores."""
+    check_layer_against_oracle(pw, oracle32, inputs.WORKLOADS[4].with_(n_layers=1, n_microbatches=1))
+
+
+def test_cfg3_full_size_chain_one_microbatch(pw, oracle32):
+    """Workload 3's stage at its full size - four layers d = 4096, 32 x 128 heads, F = 16384, 4 x 2048 tokens,
+    activations recomputed, GPipe order - on one of its micro-batches, against the fp32 oracle's chain
+    with the same bf16 hand-off between layers: outputs, input gradients and all 48 parameter
+    gradients, norm and element bounds.  The oracle needs about five minutes on 16 host cores."""
+    w = inputs.WORKLOADS[3]
+    L, M = w.n_layers, 1
+    ys, dxs, grads = run_chain_gpu(pw, w, L, M, pw.DISPATCH_ASYNC, pw.SCHEDULE_GPIPE, True, random_ln=False)
+    D = dims_of(w)
+    pls = [[p.float().numpy() for p in inputs.layer_params(w, 0, l)] for l in range(L)]
+    x, dy = inputs.microbatch(w, 0, 0)
+    f32 = lambda t: t.float().numpy().reshape(w.tokens, w.d_model)
+    rt = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(torch.bfloat16).float().numpy()
+    yw, dxw, gw = oracle32.chain(D, pls, [f32(x)], [f32(dy)], handoff=rt)
+    assert rel_l2(ys[0], yw[0]) < ACT_TOL and rel_l2(dxs[0], dxw[0]) < GRAD_TOL
+    worst = {"y": elem_check(ys[0], yw[0], "y", **LAYER_ACT), "dx": elem_check(dxs[0], dxw[0], "dx", **LAYER_GRAD)}
+    for l in range(L):
+        for name, g, want in zip(pw.PARAM_NAMES, grads[l], gw[l]):
+            assert rel_l2(g, want) < GRAD_TOL, (l, name)
+            worst[f"L{l}.d{name}"] = elem_check(g, want, f"layer {l} d{name}", **LAYER_GRAD)
+    print("worst element ratios:", {k: round(v, 3) for k, v in worst.items()})
 
 
 def test_single_tile_layer(pw, oracle64):

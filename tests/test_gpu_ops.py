@@ -3,7 +3,8 @@ import numpy as np
 import pytest
 import torch
 
-from tests.gpu_util import ACT_TOL, GRAD_TOL, bf16_randn, guard_alloc, np64, rel_l2
+from tests.gpu_util import (ACT_TOL, ELEM_ACT, ELEM_F32, ELEM_GRAD, GRAD_TOL, bf16_randn, elem_check, guard_alloc, np64,
+                            rel_l2)
 
 pytestmark = pytest.mark.gpu
 
@@ -140,6 +141,9 @@ def test_layernorm_fwd_bwd(pw, oracle64, T, d):
     check_h()
     hw, muw, rw = oracle64.ln_fwd(np64(x), np64(gamma), np64(beta), 1e-5)
     assert rel_l2(h, hw) < ACT_TOL and rel_l2(mu, muw) < 1e-5 and rel_l2(r, rw) < 1e-5
+    elem_check(h, hw, "h", **ELEM_ACT)
+    elem_check(mu, muw, "mu", **ELEM_F32)
+    elem_check(r, rw, "rstd", **ELEM_F32)
 
     dx, check_dx = guard_alloc((T, d), torch.bfloat16)
     outs = [torch.full((d,), 3.0, device="cuda") for _ in range(4)]
@@ -152,7 +156,10 @@ def test_layernorm_fwd_bwd(pw, oracle64, T, d):
     dxw, dgw, dbw = oracle64.ln_bwd(np64(dh), np64(x), muw, rw, np64(gamma))
     dxw = dxw + np64(resid)
     assert rel_l2(dx, dxw) < GRAD_TOL
+    elem_check(dx, dxw, "dx", **ELEM_GRAD)
     assert rel_l2(outs[0], 2 * dgw) < GRAD_TOL and rel_l2(outs[1], 2 * dbw) < GRAD_TOL   # overwrite, then accumulate
+    elem_check(outs[0], 2 * dgw, "dgamma", **ELEM_GRAD)
+    elem_check(outs[1], 2 * dbw, "dbeta", **ELEM_GRAD)
     assert rel_l2(outs[2], 2 * np64(resid).sum(0)) < 1e-4
     assert rel_l2(outs[3], 2 * dxw.sum(0)) < GRAD_TOL
 
@@ -183,16 +190,56 @@ def test_attention_fwd_bwd(pw, oracle64, B, S, H, dh):
     check_o(); check_l()
     ow, lw = oracle64.attn_fwd(np64(qkv), B, S, H, dh)
     assert rel_l2(o, ow) < ACT_TOL
+    elem_check(o, ow, "o", **ELEM_ACT)
     assert np.abs(lse.double().cpu().numpy() - lw).max() < 1e-3
 
     dqkv, check_d = guard_alloc((B * S, 3 * d), torch.bfloat16)
     delta = torch.empty((B, H, S), device="cuda")
     pw.op_attention_bwd(qkv.cuda(), o, dout.cuda(), lse, B, S, H, dh, dqkv, delta)
     torch.cuda.synchronize()
+    _status_ok(pw)
     check_d()
     dw = oracle64.attn_bwd(np64(qkv), np64(dout), B, S, H, dh)
     for name, sl in (("dq", slice(0, d)), ("dk", slice(d, 2 * d)), ("dv", slice(2 * d, 3 * d))):
         assert rel_l2(dqkv[:, sl], dw[:, sl]) < GRAD_TOL, name
+        elem_check(dqkv[:, sl], dw[:, sl], name, **ELEM_GRAD)
+
+
+@pytest.mark.parametrize("S,dh", [(2048, 128), (2048, 64), (4096, 128), (4096, 64)])
+def test_attention_long_sequences_every_row(pw, oracle64, S, dh):
+    """Sequences of 16 and 32 key tiles (the 2048 tokens of workloads 3 and 4, and twice that): every
+    row of o, lse, dq, dk and dv against the oracle, by norm and element by element - the online
+    softmax rescales many times, the shared-memory rings wrap, and the work items of different weight
+    are drawn heaviest first.  A second backward call must give the same bits."""
+    g = torch.Generator().manual_seed(15 + S + dh)
+    B, H = 1, 2
+    d = H * dh
+    qkv = bf16_randn((B * S, 3 * d), g)
+    dout = bf16_randn((B * S, d), g)
+    o, check_o = guard_alloc((B * S, d), torch.bfloat16)
+    lse, check_l = guard_alloc((B, H, S), torch.float32)
+    pw.op_attention_fwd(qkv.cuda(), B, S, H, dh, o, lse)
+    torch.cuda.synchronize()
+    _status_ok(pw)
+    check_o(); check_l()
+    ow, lw = oracle64.attn_fwd(np64(qkv), B, S, H, dh)
+    assert rel_l2(o, ow) < ACT_TOL
+    elem_check(o, ow, "o", **ELEM_ACT)
+    assert np.abs(lse.double().cpu().numpy() - lw).max() < 1e-3
+    dqkv, check_d = guard_alloc((B * S, 3 * d), torch.bfloat16)
+    dqkv2 = torch.empty((B * S, 3 * d), dtype=torch.bfloat16, device="cuda")
+    delta = torch.empty((B, H, S), device="cuda")
+    pw.op_attention_bwd(qkv.cuda(), o, dout.cuda(), lse, B, S, H, dh, dqkv, delta)
+    delta.fill_(float("nan"))                          # nothing of the first call may be needed by the second
+    pw.op_attention_bwd(qkv.cuda(), o, dout.cuda(), lse, B, S, H, dh, dqkv2, delta)
+    torch.cuda.synchronize()
+    _status_ok(pw)
+    check_d()
+    assert torch.equal(dqkv, dqkv2)
+    dw = oracle64.attn_bwd(np64(qkv), np64(dout), B, S, H, dh)
+    for name, sl in (("dq", slice(0, d)), ("dk", slice(d, 2 * d)), ("dv", slice(2 * d, 3 * d))):
+        assert rel_l2(dqkv[:, sl], dw[:, sl]) < GRAD_TOL, name
+        elem_check(dqkv[:, sl], dw[:, sl], name, **ELEM_GRAD)
 
 
 def test_attention_is_causal_and_deterministic(pw):
@@ -292,8 +339,12 @@ def test_attention_random_shapes(pw, oracle64):
         _status_ok(pw)
         ow, lsew = oracle64.attn_fwd(np64(qkv), B, S, H, dh)
         assert rel_l2(o, ow) < ACT_TOL, (case, B, S, H, dh)
+        elem_check(o, ow, f"o case {case}", **ELEM_ACT)
         assert np.allclose(lse.cpu().numpy(), lsew, atol=2e-3), (case, B, S, H, dh)
-        assert rel_l2(dqkv, oracle64.attn_bwd(np64(qkv), np64(dout), B, S, H, dh)) < GRAD_TOL, (case, B, S, H, dh)
+        dw = oracle64.attn_bwd(np64(qkv), np64(dout), B, S, H, dh)
+        assert rel_l2(dqkv, dw) < GRAD_TOL, (case, B, S, H, dh)
+        for name, sl in (("dq", slice(0, d)), ("dk", slice(d, 2 * d)), ("dv", slice(2 * d, 3 * d))):
+            elem_check(dqkv[:, sl], dw[:, sl], f"{name} case {case}", **ELEM_GRAD)
 
 
 def test_gemm_tiles_cut_along_k_are_exact_and_reproducible(pw):

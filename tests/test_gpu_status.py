@@ -31,3 +31,37 @@ def test_bounded_wait_gives_up_reports_and_leaves_the_context_usable(pw):
     torch.cuda.synchronize()
     assert torch.equal(out, torch.full((256,), 64.0, device="cuda"))
     assert pw.op_status() == (0, 0)
+
+
+def test_injected_launch_failure_is_reported_and_nothing_of_that_launch_runs(pw):
+    """Host-side fault injection: the library's launch wrapper is told to refuse the k-th launch
+    before enqueueing it.  The call returns PW_ERR_CUDA with a message naming the kernel family,
+    the launch counter shows only the launches that really went out, the output of the refused
+    launch is untouched, the device status stays clean and the next call works."""
+    from paper_2203_12533_b200 import inputs
+    from tests.gpu_util import make_layer
+    w = inputs.WORKLOADS[1]
+    layer = make_layer(pw, w)
+    params = [p.cuda() for p in inputs.layer_params(w)]
+    x, _ = inputs.microbatch(w)
+    x = x.cuda().view(-1, w.d_model)
+    ctx = torch.empty(layer.ctx_bytes, dtype=torch.uint8, device="cuda")
+    scratch = torch.empty(layer.scratch_bytes, dtype=torch.uint8, device="cuda")
+    y = torch.full_like(x, 7.0)
+    for k, family in ((1, "layernorm"), (2, "gemm")):           # first launch of the forward is LN1, second the QKV GEMM
+        n0 = layer.launch_count()
+        pw.set_tuning(pw.TUNE_FAIL_LAUNCH, k)
+        with pytest.raises(pw.PwError) as e:
+            layer.fwd(params, x, y, ctx, scratch)
+        assert e.value.status == 4                              # PW_ERR_CUDA
+        assert family in str(e.value).lower()
+        assert pw.get_tuning(pw.TUNE_FAIL_LAUNCH) == 0          # one shot
+        assert layer.launch_count() - n0 == k - 1               # only the launches before the refused one
+        torch.cuda.synchronize()
+        assert torch.equal(y, torch.full_like(x, 7.0))          # the last GEMM, which writes y, never ran
+        assert layer.status() == (0, 0)
+    n0 = layer.launch_count()
+    layer.fwd(params, x, y, ctx, scratch)
+    torch.cuda.synchronize()
+    assert layer.launch_count() - n0 == 7 and layer.status() == (0, 0)
+    assert not torch.equal(y, torch.full_like(x, 7.0)) and torch.isfinite(y.float()).all()

@@ -34,10 +34,14 @@ def test_noalloc_colsum_matches_allocating_entry_point_twice(pw):
         part = torch.empty(pw.op_colsum_scratch_bytes(T, N), dtype=torch.uint8, device="cuda")
         pw.op_colsum(a, want, True, part)                           # existing entry point: want = base + sums
         got = base.clone()
-        before = torch.cuda.memory_allocated()
+        warm = base.clone()
+        pw.op_colsum_noalloc(a, warm, True)                         # the first call on a device looks up the array's address
+        torch.cuda.synchronize()
+        before, free_before = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
         pw.op_colsum_noalloc(a, got, True)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == before              # the binding allocated nothing either
+        assert torch.cuda.memory_allocated() == before              # the binding allocated nothing
+        assert torch.cuda.mem_get_info()[0] == free_before          # and neither did the library: the device's free memory is unchanged
         assert _rel(got, want) < 1e-5, (call, _rel(got, want))
         over = torch.empty(N, device="cuda")
         pw.op_colsum_noalloc(a, over, False)                        # overwrite mode ignores what `over` held
