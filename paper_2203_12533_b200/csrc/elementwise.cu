@@ -180,7 +180,8 @@ bool plan_warp_rows(int d, int* W, int* CH)
 // partials[(cta*rows_per_cta + row_in_cta)][4][d] = {dgamma, dbeta, sum resid, sum dx}.
 // The next row's three inputs are fetched before the current row's reduction, and the two row
 // sums share one barrier.
-constexpr int kLnBwdDepth = 4;
+// rows in the prefetch ring (six were measured slower than four at every width)
+__host__ __device__ constexpr int ln_bwd_depth(int) { return 4; }
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, bool valid)
 {
     const int n = valid ? 16 : 0;                       // 0: the 16 bytes are zero-filled, src is not read
@@ -202,6 +203,7 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
               const __nv_bfloat16* resid, int T, int d, __nv_bfloat16* dx,
               float* partials, int tpr, int rows_per_cta)
 {
+    constexpr int kDepth = ln_bwd_depth(CHUNKS);
     __shared__ float red[2][2][kMaxWarps];
     const int row_in_cta = threadIdx.x / tpr, tr = threadIdx.x % tpr;
     const int wpr = tpr >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -217,7 +219,7 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
     }
     const int row_groups = (T + rows_per_cta - 1) / rows_per_cta;
     // The three inputs of the rows this thread will handle travel through a private ring in
-    // shared memory, kLnBwdDepth - 1 rows ahead (16-byte asynchronous copies; a thread only ever
+    // shared memory, kDepth - 1 rows ahead (16-byte asynchronous copies; a thread only ever
     // reads what it fetched itself, so no barrier is involved).  Slot (stage, input, j) of thread
     // t is ring[((stage * 3 + input) * CHUNKS + j) * blockDim.x + t].
     extern __shared__ uint4 ln_bwd_ring[];
@@ -251,7 +253,7 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
         n_r = live ? rstd[row] : 0.f;
     };
 #pragma unroll
-    for (int s = 0; s < kLnBwdDepth - 1; ++s) issue(s);
+    for (int s = 0; s < kDepth - 1; ++s) issue(s);
     fetch_stats(blockIdx.x);
     const float inv_d = 1.0f / d;
     int par = 0, stage = 0;
@@ -261,8 +263,8 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
         const bool live = row < T;
         const float r = n_r;
         const uint64_t r2 = splat2(r), nmr2 = splat2(-n_m * r);
-        issue(stage == 0 ? kLnBwdDepth - 1 : stage - 1);
-        cp_async_wait<kLnBwdDepth - 1>();                  // this row's copies have landed
+        issue(stage == 0 ? kDepth - 1 : stage - 1);
+        cp_async_wait<kDepth - 1>();                  // this row's copies have landed
         uint64_t xh[CHUNKS][4], g[CHUNKS][4], dhv[CHUNKS][4], rs[CHUNKS][4];
         uint64_t s1p = 0ull, s2p = 0ull;
 #pragma unroll
@@ -279,7 +281,7 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
                 s2p = ffma2(g[j][k], xh[j][k], s2p);
             }
         }
-        stage = stage + 1 == kLnBwdDepth ? 0 : stage + 1;
+        stage = stage + 1 == kDepth ? 0 : stage + 1;
         fetch_stats(rg + gridDim.x);
         float s1, s1b, s2, s2b;
         unpack_f32x2(s1p, s1, s1b);
@@ -338,33 +340,48 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
     }
 }
 
-// out_q[c] (+)= sum over partial rows of partials[row][q][c].  CTA = 32 columns x 32 row lanes:
-// row lane y adds rows y, y+32, ... in order, then the 32 lane sums are added in order, so the
-// result does not depend on scheduling.  Up to 4 outputs (grid.y = quantity).
+// out_q[c] (+)= sum over partial rows of partials[row][q][c].  CTA = 64 columns x 16 row lanes, a thread
+// owns four consecutive columns (16-byte loads, eight rows in flight): row lane y adds rows y, y+16, ...
+// in order, then the 16 lane sums are added in order, so the result does not depend on scheduling.
+// Up to 4 outputs (grid.y = quantity).  n is a multiple of 4.
 struct ReduceOuts { float* out[4]; };
-__global__ void __launch_bounds__(1024)
+constexpr int kReduceCols = 64, kReduceLanes = 16;
+__global__ void __launch_bounds__(kReduceCols / 4 * kReduceLanes)
 reduce_partials_kernel(const float* partials, int nrows, int nq, int n, ReduceOuts outs, int accumulate)
 {
-    __shared__ float sm[32][33];
-    const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
-    const int c = blockIdx.x * 32 + cx;
+    __shared__ float4 sm[kReduceLanes][kReduceCols / 4];
+    const int cx = threadIdx.x & (kReduceCols / 4 - 1), ry = threadIdx.x / (kReduceCols / 4);
+    const int c = blockIdx.x * kReduceCols + cx * 4;
     const int q = blockIdx.y;
     float* out = outs.out[q];
     grid_dep_launch();
     grid_dep_wait();
     if (out == nullptr) return;
-    float s = 0.f;
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
     if (c < n) {
-#pragma unroll 4
-        for (int r = ry; r < nrows; r += 32) s += partials[(static_cast<size_t>(r) * nq + q) * n + c];
+        const size_t stride = static_cast<size_t>(nq) * n;             // floats between partial rows
+        const float* src = partials + static_cast<size_t>(q) * n + c;
+        int r = ry;
+        for (; r + 7 * kReduceLanes < nrows; r += 8 * kReduceLanes) {
+            float4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = *reinterpret_cast<const float4*>(src + (r + u * kReduceLanes) * stride);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
+        }
+        for (; r < nrows; r += kReduceLanes) {
+            const float4 v = *reinterpret_cast<const float4*>(src + r * stride);
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        }
     }
     sm[ry][cx] = s;
     __syncthreads();
     if (ry == 0 && c < n) {
-        float t = 0.f;
+        float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) t += sm[i][cx];
-        out[c] = accumulate ? out[c] + t : t;
+        for (int i = 0; i < kReduceLanes; ++i) { const float4 v = sm[i][cx]; t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w; }
+        if (accumulate) { t.x += out[c]; t.y += out[c + 1]; t.z += out[c + 2]; t.w += out[c + 3]; }
+        out[c] = t.x; out[c + 1] = t.y; out[c + 2] = t.z; out[c + 3] = t.w;
     }
 }
 
@@ -449,7 +466,7 @@ const char* launch_layernorm_fwd(Runtime* rt, const void* x, const void* gamma, 
 const char* configure_elementwise()
 {
     cudaError_t e = cudaSuccess;
-#define PW_LN_ATTR(C, B) if (e == cudaSuccess) e = cudaFuncSetAttribute(ln_bwd_kernel<C, B>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLnBwdDepth * 3 * C * kRowThreadsMax * 16)
+#define PW_LN_ATTR(C, B) if (e == cudaSuccess) e = cudaFuncSetAttribute(ln_bwd_kernel<C, B>, cudaFuncAttributeMaxDynamicSharedMemorySize, ln_bwd_depth(C) * 3 * C * kRowThreadsMax * 16)
     PW_LN_ATTR(1, true); PW_LN_ATTR(1, false); PW_LN_ATTR(2, true); PW_LN_ATTR(2, false); PW_LN_ATTR(4, true); PW_LN_ATTR(4, false);
 #undef PW_LN_ATTR
     return e == cudaSuccess ? nullptr : "could not raise the shared-memory limit of the layernorm kernels";
@@ -479,7 +496,7 @@ const char* launch_layernorm_bwd(Runtime* rt, const void* dh, const void* x, con
     auto Rs = static_cast<const float*>(rstd);
     auto P = static_cast<float*>(partials);
     cudaError_t le = cudaSuccess;
-    const size_t ring_bytes = static_cast<size_t>(kLnBwdDepth) * 3 * rp.chunks * rp.threads * 16;
+    const size_t ring_bytes = static_cast<size_t>(ln_bwd_depth(rp.chunks)) * 3 * rp.chunks * rp.threads * 16;
     const bool sums = db_resid != nullptr || db_dx != nullptr;
 #define PW_LN_BWD(C, B) le = launch_k(ln_bwd_kernel<C, B>, dim3(grid), dim3(rp.threads), ring_bytes, stream, DH, X, Mu, Rs, G, R, T, d, DX, P, rp.tpr, rp.rows_per_cta)
     switch (rp.chunks) {
@@ -493,8 +510,8 @@ const char* launch_layernorm_bwd(Runtime* rt, const void* dh, const void* x, con
     outs.out[0] = static_cast<float*>(dgamma); outs.out[1] = static_cast<float*>(dbeta);
     outs.out[2] = static_cast<float*>(db_resid); outs.out[3] = static_cast<float*>(db_dx);
     const int nq = sums ? 4 : 2;
-    dim3 rgrid((d + 31) / 32, nq);
-    return launch_k(reduce_partials_kernel, rgrid, dim3(1024), 0, stream, static_cast<const float*>(P), grid * rp.rows_per_cta, nq, d, outs, accumulate) == cudaSuccess
+    dim3 rgrid((d + kReduceCols - 1) / kReduceCols, nq);
+    return launch_k(reduce_partials_kernel, rgrid, dim3(kReduceCols / 4 * kReduceLanes), 0, stream, static_cast<const float*>(P), grid * rp.rows_per_cta, nq, d, outs, accumulate) == cudaSuccess
                ? nullptr : "layernorm bwd reduce launch failed";
 }
 
@@ -538,8 +555,8 @@ const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, voi
         return "colsum launch failed";
     ReduceOuts outs;
     outs.out[0] = static_cast<float*>(out); outs.out[1] = outs.out[2] = outs.out[3] = nullptr;
-    dim3 rgrid((N + 31) / 32, 1);
-    return launch_k(reduce_partials_kernel, rgrid, dim3(1024), 0, stream, static_cast<const float*>(partials), R, 1, N, outs, accumulate) == cudaSuccess
+    dim3 rgrid((N + kReduceCols - 1) / kReduceCols, 1);
+    return launch_k(reduce_partials_kernel, rgrid, dim3(kReduceCols / 4 * kReduceLanes), 0, stream, static_cast<const float*>(partials), R, 1, N, outs, accumulate) == cudaSuccess
                ? nullptr : "colsum reduce launch failed";
 }
 
@@ -608,8 +625,8 @@ const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* ou
     if (cudaGetLastError() != cudaSuccess) return "colsum launch failed";
     ReduceOuts outs;
     outs.out[0] = static_cast<float*>(out); outs.out[1] = outs.out[2] = outs.out[3] = nullptr;
-    dim3 rgrid((N + 31) / 32, 1);
-    reduce_partials_kernel<<<rgrid, 1024, 0, stream>>>(sc.ptr, static_cast<int>(R), 1, N, outs, accumulate);
+    dim3 rgrid((N + kReduceCols - 1) / kReduceCols, 1);
+    reduce_partials_kernel<<<rgrid, kReduceCols / 4 * kReduceLanes, 0, stream>>>(sc.ptr, static_cast<int>(R), 1, N, outs, accumulate);
     return cudaGetLastError() == cudaSuccess ? nullptr : "colsum reduce launch failed";
 }
 
