@@ -71,7 +71,16 @@ enum { PW_ACT_GELU_ERF = 0, PW_ACT_GELU_TANH = 1 };
  * the same bits as the first time, and GeLU of the bf16 pre-activations u, which may differ from
  * the forward's GeLU of the fp32 pre-activations in the last bf16 bit).  pw_layer_ctx_offset reports
  * size 0 for the three tensors; pw_layer_fwd then needs `scratch` even when ctx is given. */
-enum { PW_FLAG_LEAN_CTX = 1u };
+enum { PW_FLAG_LEAN_CTX = 1u, PW_FLAG_WHOLE_LAYER = 2u };
+/* PW_FLAG_WHOLE_LAYER: pw_layer_fwd and pw_layer_bwd are ONE cooperative kernel launch each instead of
+ * 7 and 19 - for calls so small that launches and hand-offs between kernels, not arithmetic, set the
+ * time (Section 5.1, Figures 5 and 6: computations shorter than the cost of issuing them).  Same
+ * tensors, same saved context, same bf16 hand-off points as the default path; results agree with
+ * it within rounding (different tile shapes and summation orders), bit-reproducibly.  Supported:
+ * head_dim 64, d_model <= 512, seq_len <= 1024, (batch * seq_len / 64) * (d_model / 64) <= 1024; not
+ * together with PW_FLAG_LEAN_CTX; pw_layer_fwd needs `scratch` even when ctx is given.  Anything else:
+ * PW_ERR_UNSUPPORTED_SHAPE / PW_ERR_INVALID_ARG from pw_layer_create.  A grid barrier that waits
+ * longer than about a second records PW_ERR_TIMEOUT in the status word and the kernel returns. */
 
 /* Static shape of a layer call - fixed for the life of the handle, like the static shapes of
  * a compiled function (Section 3).  Supported: head_dim in {64, 128}; n_heads*head_dim ==
@@ -88,7 +97,7 @@ typedef struct pw_layer_config {
     int32_t act;    /* PW_ACT_GELU_ERF (default) or PW_ACT_GELU_TANH */
     float ln_eps;   /* 0 means 1e-5 */
     int32_t causal; /* must be 1 */
-    uint32_t flags; /* 0, or PW_FLAG_LEAN_CTX */
+    uint32_t flags; /* 0, PW_FLAG_LEAN_CTX or PW_FLAG_WHOLE_LAYER */
 } pw_layer_config_t;
 
 /* The 12 parameters of a layer (bf16 device pointers). */
@@ -188,7 +197,8 @@ enum {
     PW_K_XENT = 8,      /* softmax / cross-entropy + loss mean (pw_lm_step)          */
     PW_K_EMBED = 9,     /* embedding lookup and its scatter-add backward (pw_lm_step) */
     PW_K_GELU = 10,     /* GeLU(u) re-derived in the backward of a PW_FLAG_LEAN_CTX layer */
-    PW_K_COUNT = 11
+    PW_K_WHOLE_LAYER = 11, /* forward or backward of a PW_FLAG_WHOLE_LAYER handle (one launch each) */
+    PW_K_COUNT = 12
 };
 typedef struct pw_profile {
     uint64_t launches[PW_K_COUNT]; /* kernel launches per class since profile_begin      */

@@ -21,6 +21,7 @@ STATUS_NAMES = {0: "PW_OK", 1: "PW_ERR_INVALID_ARG", 2: "PW_ERR_UNSUPPORTED_SHAP
                 4: "PW_ERR_CUDA", 5: "PW_ERR_DEVICE_UNSUPPORTED", 6: "PW_ERR_TIMEOUT", 7: "PW_ERR_INTERNAL"}
 ACT_GELU_ERF, ACT_GELU_TANH = 0, 1
 FLAG_LEAN_CTX = 1
+FLAG_WHOLE_LAYER = 2
 GEMM_TN, GEMM_NN, GEMM_NT = 0, 1, 2
 EPI_NONE, EPI_BIAS, EPI_BIAS_RESID, EPI_BIAS_GELU, EPI_DGELU, EPI_F32 = range(6)
 DISPATCH_OPBYOP, DISPATCH_ASYNC, DISPATCH_GRAPH = 0, 1, 2
@@ -73,12 +74,12 @@ class ApplyItem(ctypes.Structure):
 
 
 KERNEL_CLASSES = ("gemm_tn", "gemm_nn", "gemm_nt", "attn_fwd", "attn_bwd", "ln_fwd", "ln_bwd", "colsum", "xent", "embed",
-                  "gelu")
+                  "gelu", "whole_layer")
 
 
 class Profile(ctypes.Structure):
-    _fields_ = [("launches", ctypes.c_uint64 * 11), ("ms", ctypes.c_double * 11), ("flops", ctypes.c_double * 11),
-                ("bytes", ctypes.c_double * 11)]
+    _fields_ = [("launches", ctypes.c_uint64 * 12), ("ms", ctypes.c_double * 12), ("flops", ctypes.c_double * 12),
+                ("bytes", ctypes.c_double * 12)]
 
     def as_dict(self):
         return {n: dict(launches=int(self.launches[i]), ms=float(self.ms[i]), flops=float(self.flops[i]),

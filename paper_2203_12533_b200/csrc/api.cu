@@ -60,7 +60,7 @@ Runtime* get_runtime(const char** err)
         delete rt; *err = "cuTensorMapEncodeTiled not available from the driver"; return nullptr;
     }
     const char* ce;
-    if ((ce = configure_gemm()) || (ce = configure_attention()) || (ce = configure_attention_fwd()) || (ce = configure_elementwise())) { delete rt; *err = ce; return nullptr; }
+    if ((ce = configure_gemm()) || (ce = configure_attention()) || (ce = configure_attention_fwd()) || (ce = configure_elementwise()) || (ce = configure_whole_layer())) { delete rt; *err = ce; return nullptr; }
     if (cudaMalloc(reinterpret_cast<void**>(&rt->op_status), sizeof(DeviceStatus)) != cudaSuccess ||
         cudaMemset(rt->op_status, 0, sizeof(DeviceStatus)) != cudaSuccess) {
         delete rt; *err = "could not allocate the status word"; return nullptr;
@@ -85,6 +85,9 @@ struct LayerPlan {
     bool lean;
     size_t off_lean_h1, off_lean_h2, off_lean_a, off_lean_stats;
     size_t off_splitk;           // partial sums of GEMM tiles cut along K (main-stream GEMMs only)
+    // PW_FLAG_WHOLE_LAYER: forward and backward are one cooperative launch each
+    bool whole;
+    size_t off_whole_splitk;
 };
 
 }  // namespace pw
@@ -93,6 +96,7 @@ struct pw_layer {
     pw::LayerPlan plan;
     pw::Runtime* rt;
     pw::DeviceStatus* status;
+    unsigned* whole_sync = nullptr; // grid-barrier and split-K words of the whole-layer kernels (zero between launches)
     cudaStream_t aux = nullptr;     // side stream: weight gradients and bias column sums run beside the dgrad chain
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     uint64_t launches = 0;          // kernels launched (or replayed) through this handle
@@ -125,7 +129,9 @@ static pw_status_t validate_cfg(const pw_layer_config_t* c)
         return fail(PW_ERR_INVALID_ARG, "config has a non-positive dimension");
     if (c->act != PW_ACT_GELU_ERF && c->act != PW_ACT_GELU_TANH) return fail(PW_ERR_INVALID_ARG, "unknown activation");
     if (c->causal != 1) return fail(PW_ERR_UNSUPPORTED_SHAPE, "only causal attention is supported");
-    if ((c->flags & ~static_cast<uint32_t>(PW_FLAG_LEAN_CTX)) != 0) return fail(PW_ERR_INVALID_ARG, "unknown flag");
+    if ((c->flags & ~static_cast<uint32_t>(PW_FLAG_LEAN_CTX | PW_FLAG_WHOLE_LAYER)) != 0) return fail(PW_ERR_INVALID_ARG, "unknown flag");
+    if ((c->flags & PW_FLAG_LEAN_CTX) && (c->flags & PW_FLAG_WHOLE_LAYER))
+        return fail(PW_ERR_INVALID_ARG, "PW_FLAG_LEAN_CTX and PW_FLAG_WHOLE_LAYER exclude one another");
     if (c->ln_eps < 0.f) return fail(PW_ERR_INVALID_ARG, "ln_eps must be >= 0");
     if (c->head_dim != 64 && c->head_dim != 128) return fail(PW_ERR_UNSUPPORTED_SHAPE, "head_dim must be 64 or 128");
     if (static_cast<long long>(c->n_heads) * c->head_dim != c->d_model)
@@ -134,6 +140,10 @@ static pw_status_t validate_cfg(const pw_layer_config_t* c)
     if (c->d_ff % 128 != 0) return fail(PW_ERR_UNSUPPORTED_SHAPE, "d_ff must be a multiple of 128");
     if (c->seq_len % 128 != 0) return fail(PW_ERR_UNSUPPORTED_SHAPE, "seq_len must be a multiple of 128");
     if (static_cast<long long>(c->batch) * c->seq_len > (1ll << 24)) return fail(PW_ERR_UNSUPPORTED_SHAPE, "too many tokens per call");
+    if (c->flags & PW_FLAG_WHOLE_LAYER) {
+        const char* why = whole_layer_unsupported(c->batch * c->seq_len, c->d_model, c->n_heads, c->head_dim, c->d_ff, c->seq_len);
+        if (why) return fail(PW_ERR_UNSUPPORTED_SHAPE, why);
+    }
     return PW_OK;
 }
 
@@ -170,6 +180,9 @@ static void build_plan(const pw_layer_config_t& c, Runtime* rt, LayerPlan* p)
         p->off_lean_a = s; s += align256(T * F * 2);
         p->off_lean_stats = s; s += 2 * align256(T * 4);
     }
+    p->whole = (c.flags & PW_FLAG_WHOLE_LAYER) != 0;
+    p->off_whole_splitk = 0;
+    if (p->whole) { p->off_whole_splitk = s; s += align256(whole_layer_splitk_bytes(p->T, p->d)); }
     p->scratch_bytes = s;
 }
 
@@ -280,12 +293,48 @@ static pw_status_t do_attn_bwd(pw_layer_t* L, const void* qkv, const void* o, co
     return e ? fail(PW_ERR_CUDA, e) : PW_OK;
 }
 
+// One launch for the whole forward (or backward) of a PW_FLAG_WHOLE_LAYER handle.
+static pw_status_t do_whole_layer(pw_layer_t* L, const pw_layer_params_t* P, const void* x, void* y, const void* dy, void* dx,
+                                  const pw_layer_grads_t* G, int accumulate, void* ctx, void* scratch, bool with_fc2,
+                                  bool backward, cudaStream_t st)
+{
+    const LayerPlan& p = L->plan;
+    WholeLayerArgs a = {};
+    a.T = p.T; a.d = p.d; a.H = p.H; a.F = p.F; a.B = p.B; a.S = p.S; a.act = p.cfg.act;
+    a.accumulate = accumulate; a.with_fc2 = with_fc2 ? 1 : 0;
+    a.eps = p.eps; a.scale = 1.0f / sqrtf(static_cast<float>(p.dh));
+    a.x = x; a.y = y; a.dy = dy; a.dx = dx;
+    a.ln1_g = P->ln1_gamma; a.ln1_b = P->ln1_beta; a.w_qkv = P->w_qkv; a.b_qkv = P->b_qkv; a.w_o = P->w_o; a.b_o = P->b_o;
+    a.ln2_g = P->ln2_gamma; a.ln2_b = P->ln2_beta; a.w_fc1 = P->w_fc1; a.b_fc1 = P->b_fc1; a.w_fc2 = P->w_fc2; a.b_fc2 = P->b_fc2;
+    a.h1 = at(ctx, p.ctx_off[PW_CTX_H1]); a.qkv = at(ctx, p.ctx_off[PW_CTX_QKV]); a.o = at(ctx, p.ctx_off[PW_CTX_O]);
+    a.x1 = at(ctx, p.ctx_off[PW_CTX_X1]); a.h2 = at(ctx, p.ctx_off[PW_CTX_H2]); a.u = at(ctx, p.ctx_off[PW_CTX_U]);
+    a.a = at(ctx, p.ctx_off[PW_CTX_A]); a.lse = at(ctx, p.ctx_off[PW_CTX_LSE]);
+    a.mu1 = at(ctx, p.ctx_off[PW_CTX_MU1]); a.r1 = at(ctx, p.ctx_off[PW_CTX_R1]);
+    a.mu2 = at(ctx, p.ctx_off[PW_CTX_MU2]); a.r2 = at(ctx, p.ctx_off[PW_CTX_R2]);
+    a.big = at(scratch, p.off_big); a.td0 = at(scratch, p.off_td0); a.dx1 = at(scratch, p.off_td1);
+    if (G) {
+        a.g_ln1_g = G->ln1_gamma; a.g_ln1_b = G->ln1_beta; a.g_w_qkv = G->w_qkv; a.g_b_qkv = G->b_qkv; a.g_w_o = G->w_o;
+        a.g_b_o = G->b_o; a.g_ln2_g = G->ln2_gamma; a.g_ln2_b = G->ln2_beta; a.g_w_fc1 = G->w_fc1; a.g_b_fc1 = G->b_fc1;
+        a.g_w_fc2 = G->w_fc2; a.g_b_fc2 = G->b_fc2;
+    }
+    a.splitk = at(scratch, p.off_whole_splitk);
+    a.sync = L->whole_sync;
+    a.status = L->status;
+    const double T = p.T, d = p.d, F = p.F;
+    const double fwd_flops = 2.0 * T * d * (4.0 * d + 2.0 * F) + 2.0 * T * (p.S + 1.0) * d;
+    LaunchScope sc(L, PW_K_WHOLE_LAYER, 1, backward ? 2.0 * fwd_flops + T * (p.S + 1.0) * d : fwd_flops, 0.0, st);
+    const char* e = launch_whole_layer(L->rt, a, backward, st);
+    if (e) sc.cancel(1);
+    return e ? fail(PW_ERR_CUDA, e) : PW_OK;
+}
+
 // Forward into `ctx` (a ctx-shaped region).  with_fc2 = false stops after FC1/GeLU (all that a
 // recomputing backward needs).
 static pw_status_t enqueue_fwd(pw_layer_t* L, const pw_layer_params_t* P, const void* x, void* y, void* ctx,
                                void* scratch, bool with_fc2, cudaStream_t st)
 {
     const LayerPlan& p = L->plan;
+    if (p.whole) return do_whole_layer(L, P, x, y, nullptr, nullptr, nullptr, 0, ctx, scratch, with_fc2, false, st);
     const int T = p.T, d = p.d, F = p.F, act = p.cfg.act;
     void* h1 = p.lean ? at(scratch, p.off_lean_h1) : at(ctx, p.ctx_off[PW_CTX_H1]);
     void* h2 = p.lean ? at(scratch, p.off_lean_h2) : at(ctx, p.ctx_off[PW_CTX_H2]);
@@ -326,6 +375,7 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
         ctx = scratch;
         rederive = false;                                // the forward that just ran left them in scratch
     }
+    if (p.whole) return do_whole_layer(L, P, x, nullptr, dy, dx, G, accumulate, const_cast<void*>(ctx), scratch, false, true, st);
     const void* h1 = p.lean ? at(scratch, p.off_lean_h1) : at(ctx, p.ctx_off[PW_CTX_H1]);
     const void* h2 = p.lean ? at(scratch, p.off_lean_h2) : at(ctx, p.ctx_off[PW_CTX_H2]);
     const void* a = p.lean ? at(scratch, p.off_lean_a) : at(ctx, p.ctx_off[PW_CTX_A]);
@@ -485,6 +535,11 @@ pw_status_t pw_layer_create(const pw_layer_config_t* cfg, pw_layer_t** out)
     build_plan(*cfg, rt, &L->plan);
     cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&L->status), sizeof(DeviceStatus));
     if (e == cudaSuccess) e = cudaMemset(L->status, 0, sizeof(DeviceStatus));
+    if (e == cudaSuccess && L->plan.whole) {
+        const size_t bytes = (2 + kWholeLayerMaxTiles) * sizeof(unsigned);
+        e = cudaMalloc(reinterpret_cast<void**>(&L->whole_sync), bytes);
+        if (e == cudaSuccess) e = cudaMemset(L->whole_sync, 0, bytes);
+    }
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&L->aux, cudaStreamNonBlocking);
     for (int i = 0; i < 6 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&L->ev[i], cudaEventDisableTiming);
     if (e != cudaSuccess) { pw_layer_destroy(L); return fail_cuda("handle resources (status word, side stream, events)", e); }
@@ -500,6 +555,7 @@ void pw_layer_destroy(pw_layer_t* layer)
     for (auto e : layer->ev) if (e) cudaEventDestroy(e);
     if (layer->aux) cudaStreamDestroy(layer->aux);
     if (layer->status) cudaFree(layer->status);
+    if (layer->whole_sync) cudaFree(layer->whole_sync);
     delete layer;
 }
 
@@ -529,6 +585,7 @@ pw_status_t pw_layer_fwd(pw_layer_t* layer, const pw_layer_params_t* params, con
     if (ctx == nullptr && !aligned(scratch, 256)) return fail(PW_ERR_INVALID_ARG, "scratch must be 256-byte aligned when ctx is NULL");
     if (ctx != nullptr && !aligned(ctx, 256)) return fail(PW_ERR_INVALID_ARG, "ctx must be 256-byte aligned");
     if (layer->plan.lean && !aligned(scratch, 256)) return fail(PW_ERR_INVALID_ARG, "a lean-ctx layer needs a 256-byte aligned scratch in fwd");
+    if (layer->plan.whole && !aligned(scratch, 256)) return fail(PW_ERR_INVALID_ARG, "a whole-layer handle needs a 256-byte aligned scratch in fwd");
     return enqueue_fwd(layer, params, x, y, ctx ? ctx : scratch, scratch, true, static_cast<cudaStream_t>(stream));
 }
 

@@ -137,4 +137,27 @@ const char* launch_attention_bwd(Runtime* rt, const void* qkv, const void* o, co
                                  int B, int S, int H, int dh, void* dqkv, void* delta, DeviceStatus* status,
                                  cudaStream_t stream);
 
+// The layer's forward or backward as one cooperative launch (whole_layer.cu), for small shapes.
+// Tensor names are those of the layer plan: ctx tensors (h1 ... r2), backward temporaries (big =
+// du, later dqkv; td0 = dh2, dout, dh1; dx1), the 12 parameters and their fp32 gradients.
+constexpr int kWholeLayerMaxTiles = 1024;           // (tokens / 64) * (d_model / 64): one split-K ticket each
+struct WholeLayerArgs {
+    int T, d, H, F, B, S, act, accumulate, with_fc2;
+    int split_d, split_f, split_3d;                 // K slices of the GEMMs with [T, d] outputs (set by the launcher)
+    float eps, scale;
+    const void *x, *dy;
+    void *y, *dx;
+    const void *ln1_g, *ln1_b, *w_qkv, *b_qkv, *w_o, *b_o, *ln2_g, *ln2_b, *w_fc1, *b_fc1, *w_fc2, *b_fc2;
+    void *h1, *qkv, *o, *x1, *h2, *u, *a, *lse, *mu1, *r1, *mu2, *r2;
+    void *big, *td0, *dx1;
+    void *g_ln1_g, *g_ln1_b, *g_w_qkv, *g_b_qkv, *g_w_o, *g_b_o, *g_ln2_g, *g_ln2_b, *g_w_fc1, *g_b_fc1, *g_w_fc2, *g_b_fc2;
+    void* splitk;                                   // whole_layer_splitk_bytes() of fp32 partial tiles
+    unsigned* sync;                                 // 2 + kWholeLayerMaxTiles words, zero when the handle is created
+    DeviceStatus* status;
+};
+const char* configure_whole_layer();
+const char* whole_layer_unsupported(int T, int d, int H, int dh, int F, int S);   // nullptr if the shape is served
+size_t whole_layer_splitk_bytes(int T, int d);
+const char* launch_whole_layer(Runtime* rt, WholeLayerArgs a, bool backward, cudaStream_t stream);
+
 }  // namespace pw

@@ -1,0 +1,983 @@
+// One decoder layer's forward, or its backward, as ONE cooperative launch, for calls so small
+// (workload 1: 256 tokens, width 256, 1.2 GFLOP forward + backward) that launches, ramps and
+// hand-offs between kernels set the time, not arithmetic: the regime of the dispatch study of
+// Section 5.1 (Figures 5 and 6), where a computation is shorter than the cost of issuing it.
+//
+// The 7 forward / 19 backward steps of the layer become 5 / 7 phases of one persistent grid
+// (one 128-thread CTA per SM); a phase is a list of independent units (a 64 x 64 output tile of a
+// GEMM, a slice of its K range, 64 query or key rows of one head, four LayerNorm rows, 16 columns of
+// a bias sum) that the CTAs take round-robin, and phases are separated by a bounded grid barrier.
+// Steps that do not depend on one another share a phase (a data-gradient GEMM, the weight-gradient
+// GEMM and the bias sum that hang off the same tensor), LayerNorm is applied while a GEMM stages its
+// A rows, and rowsum(dO * O) is taken by the attention-backward units themselves.
+//
+// At these sizes a tile of 64 x 64 keeps 16 ... 144 SMs busy where the 128 x 256 tcgen05 tiles of
+// the large-shape kernels would keep 2 ... 8; the products run on mma.sync (m16n8k16, bf16 in, fp32
+// accumulate) from shared memory, which is far below the tcgen05 rate and does not matter here.
+// Every sum has a fixed order (split-K partial tiles are added by the last-arriving CTA in slice
+// order), so results are bit-reproducible.  Tensors, rounding points (bf16 hand-offs) and the saved
+// context are those of the multi-kernel path.
+#include "pw_kernels.h"
+
+namespace pw {
+namespace {
+
+constexpr int kThreads = 128;
+constexpr int kChunk = 64 * 64 * 2;                 // one 64 x 64 bf16 operand chunk
+constexpr int kStages = 3;
+constexpr int kMaxD = 512;                          // LayerNorm panel: 64 rows of the full width in shared memory
+constexpr int kMaxS = 1024;
+constexpr int kSmStage = 0;                         // kStages x (A chunk, B chunk); attention: Q/K/V/dO chunks
+constexpr int kSmPanel = kSmStage + kStages * 2 * kChunk;
+constexpr int kSmVec = kSmPanel + 64 * (kMaxD + 8) * 2;     // lse and delta of one (sequence, head)
+constexpr int kSmRed = kSmVec + 2 * kMaxS * 4;              // column-sum lanes
+constexpr int kSmFlag = kSmRed + 2 * 8 * 16 * 4;
+constexpr int kSmBytes = kSmFlag + 16;
+
+constexpr int kSiteBarrier = 900;
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t (&r)[4])
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm4t(uint32_t addr, uint32_t (&r)[4])
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ unsigned ld_acquire(const unsigned* p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ float ldcg_bf16(const uint16_t* p) { return __uint_as_float(static_cast<uint32_t>(__ldcg(p)) << 16); }
+
+// ---------------------------------------------------------------- grid barrier
+// sync[0] counts arrivals, sync[1] is the generation.  The last CTA to arrive clears the count and
+// bumps the generation; both words are back in a consistent state when the kernel ends, so the
+// next launch (or a replay of a captured graph) starts from where this one stopped.  A CTA that
+// waits longer than the limit records a timeout in the status word and every CTA leaves.
+__device__ bool grid_barrier(unsigned* sync, DeviceStatus* status, int* s_flag)
+{
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int ok = 1;
+        const unsigned gen = ld_acquire(sync + 1);
+        __threadfence();
+        const unsigned prev = atomicAdd(sync, 1u);
+        if (prev == gridDim.x - 1) {
+            atomicExch(sync, 0u);
+            __threadfence();
+            atomicAdd(sync + 1, 1u);
+        } else {
+            const long long t0 = clock64();
+            unsigned spins = 0;
+            while (ld_acquire(sync + 1) == gen) {
+                if ((++spins & 0xffu) == 0) {
+                    if (*reinterpret_cast<volatile int*>(&status->code) != 0) { ok = 0; break; }
+                    if (clock64() - t0 > kWaitCycles) {
+                        if (atomicCAS(&status->code, 0, kStatusTimeout) == 0) status->site = kSiteBarrier;
+                        ok = 0;
+                        break;
+                    }
+                }
+            }
+        }
+        __threadfence();
+        *s_flag = ok;
+    }
+    __syncthreads();
+    return *s_flag != 0;
+}
+
+// ---------------------------------------------------------------- operand chunks in shared memory
+// A chunk is 64 rows of 128 bytes; the 16-byte piece c of row r sits at piece c ^ (r & 7), which keeps
+// both ldmatrix forms free of bank conflicts.
+__device__ __forceinline__ uint32_t swz(int row, int piece) { return row * 128 + ((piece ^ (row & 7)) << 4); }
+
+__device__ __forceinline__ void stage_chunk(uint32_t dst, const uint16_t* src, size_t ld, int tid)
+{
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int q = tid + i * kThreads, row = q >> 3, piece = q & 7;
+        cp_async16(dst + swz(row, piece), src + row * ld + piece * 8);
+    }
+}
+// chunk stored [m or n][k]
+__device__ __forceinline__ void frag_a_k(uint32_t base, int r0, int kk, int lane, uint32_t (&a)[4])
+{
+    ldsm4(base + swz(r0 + (lane & 15), kk * 2 + (lane >> 4)), a);
+}
+__device__ __forceinline__ void frag_b_k(uint32_t base, int n0, int kk, int lane, uint32_t (&b)[4])
+{
+    ldsm4(base + swz(n0 + (lane & 7) + ((lane >> 4) << 3), kk * 2 + ((lane >> 3) & 1)), b);
+}
+// chunk stored [k][m or n]
+__device__ __forceinline__ void frag_a_mn(uint32_t base, int m0, int kk, int lane, uint32_t (&a)[4])
+{
+    ldsm4t(base + swz(kk * 16 + (lane & 7) + ((lane >> 4) << 3), (m0 >> 3) + ((lane >> 3) & 1)), a);
+}
+__device__ __forceinline__ void frag_b_mn(uint32_t base, int n0, int kk, int lane, uint32_t (&b)[4])
+{
+    ldsm4t(base + swz(kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), (n0 >> 3) + (lane >> 4)), b);
+}
+
+// ---------------------------------------------------------------- 64 x 64 output tile, K range [k0, k1)
+// C[m0.., n0..] = sum_k A(m, k) B(k, n).  A_MN: A is stored [K][M] (else [M][K]); B_MN: B is stored
+// [K][N] (else [N][K]); A_PANEL: the A rows are already in shared memory (LayerNorm output, full width).
+// Warp w owns rows 32 (w & 1) and columns 32 (w >> 1): acc[mi][ni][e] is row 16 mi + lane / 4 + 8 (e / 2),
+// column 8 ni + 2 (lane % 4) + e % 2 of that quarter.
+template <bool A_MN, bool B_MN, bool A_PANEL>
+__device__ void gemm_tile(float (&acc)[2][4][4], const uint16_t* A, size_t lda, const uint16_t* Bm, size_t ldb, int m0,
+                          int n0, int k0, int k1, uint32_t stage, uint32_t panel, int panel_stride)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, wm = (warp & 1) * 32, wn = (warp >> 1) * 32;
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.f;
+    const int nk = (k1 - k0) >> 6;
+    auto load = [&](int kc) {
+        const uint32_t sa = stage + (kc % kStages) * 2 * kChunk, sb = sa + kChunk;
+        const size_t kk0 = k0 + kc * 64;
+        if (!A_PANEL) stage_chunk(sa, A_MN ? A + kk0 * lda + m0 : A + m0 * lda + kk0, lda, tid);
+        stage_chunk(sb, B_MN ? Bm + kk0 * ldb + n0 : Bm + n0 * ldb + kk0, ldb, tid);
+    };
+#pragma unroll
+    for (int s = 0; s < kStages - 1; ++s) {
+        if (s < nk) load(s);
+        cp_async_commit();
+    }
+    for (int kc = 0; kc < nk; ++kc) {
+        cp_async_wait<kStages - 2>();
+        __syncthreads();
+        if (kc + kStages - 1 < nk) load(kc + kStages - 1);
+        cp_async_commit();
+        const uint32_t sa = stage + (kc % kStages) * 2 * kChunk, sb = sa + kChunk;
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+            uint32_t af[2][4], bf[2][4];
+#pragma unroll
+            for (int mi = 0; mi < 2; ++mi) {
+                if (A_PANEL) {
+                    const int row = wm + mi * 16 + (lane & 15), col = k0 + kc * 64 + kk * 16 + (lane >> 4) * 8;
+                    ldsm4(panel + row * panel_stride + col * 2, af[mi]);
+                } else if (A_MN) {
+                    frag_a_mn(sa, wm + mi * 16, kk, lane, af[mi]);
+                } else {
+                    frag_a_k(sa, wm + mi * 16, kk, lane, af[mi]);
+                }
+            }
+#pragma unroll
+            for (int np = 0; np < 2; ++np) {
+                if (B_MN) frag_b_mn(sb, wn + np * 16, kk, lane, bf[np]);
+                else frag_b_k(sb, wn + np * 16, kk, lane, bf[np]);
+            }
+#pragma unroll
+            for (int mi = 0; mi < 2; ++mi)
+#pragma unroll
+                for (int ni = 0; ni < 4; ++ni)
+                    mma16816(acc[mi][ni], af[mi], bf[ni >> 1][(ni & 1) * 2], bf[ni >> 1][(ni & 1) * 2 + 1]);
+        }
+    }
+    cp_async_wait<0>();
+    __syncthreads();                                        // the stage buffers may be refilled by the next unit
+}
+
+// Split-K: every slice stores its partial tile, the CTA that arrives last adds the slices in slice
+// order (its own included, from memory) and returns true: it then runs the epilogue.
+__device__ bool splitk_combine(float (&acc)[2][4][4], float* ws, unsigned* sem, int tile, int slice, int nslices, int* s_flag)
+{
+    if (nslices == 1) return true;
+    const int tid = threadIdx.x;
+    float* flat = &acc[0][0][0];
+    float4* mine = reinterpret_cast<float4*>(ws + static_cast<size_t>(tile * nslices + slice) * 4096);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) __stcg(mine + i * kThreads + tid, make_float4(flat[4 * i], flat[4 * i + 1], flat[4 * i + 2], flat[4 * i + 3]));
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned prev = atomicAdd(sem + tile, 1u);
+        const int last = prev == static_cast<unsigned>(nslices - 1);
+        if (last) atomicExch(sem + tile, 0u);
+        __threadfence();
+        *s_flag = last;
+    }
+    __syncthreads();
+    const bool last = *s_flag != 0;
+    __syncthreads();                                        // everyone has read the flag before it is written again
+    if (!last) return false;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) flat[i] = 0.f;
+    for (int s = 0; s < nslices; ++s) {
+        const float4* part = reinterpret_cast<const float4*>(ws + static_cast<size_t>(tile * nslices + s) * 4096);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float4 v = __ldcg(part + i * kThreads + tid);
+            flat[4 * i] += v.x; flat[4 * i + 1] += v.y; flat[4 * i + 2] += v.z; flat[4 * i + 3] += v.w;
+        }
+    }
+    return true;
+}
+
+// Calls f(row, col, v0, v1) for every pair of adjacent columns this thread holds of the tile at (m0, n0).
+template <typename F>
+__device__ __forceinline__ void for_each_pair(const float (&acc)[2][4][4], int m0, int n0, F f)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int r = m0 + (warp & 1) * 32 + (lane >> 2), c = n0 + (warp >> 1) * 32 + 2 * (lane & 3);
+#pragma unroll
+    for (int mi = 0; mi < 2; ++mi)
+#pragma unroll
+        for (int ni = 0; ni < 4; ++ni)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) f(r + mi * 16 + h * 8, c + ni * 8, acc[mi][ni][2 * h], acc[mi][ni][2 * h + 1]);
+}
+__device__ __forceinline__ void store_bf16x2(uint16_t* base, size_t idx, float v0, float v1)
+{
+    *reinterpret_cast<uint32_t*>(base + idx) = pack_bf16(v0, v1);
+}
+__device__ __forceinline__ void load_bf16x2(const uint16_t* base, size_t idx, float& v0, float& v1)
+{
+    const uint32_t v = __ldcg(reinterpret_cast<const uint32_t*>(base + idx));
+    v0 = bf16_lo(v); v1 = bf16_hi(v);
+}
+
+// ---------------------------------------------------------------- LayerNorm of 64 rows into the panel
+// Warp w normalises rows 16 w .. 16 w + 15 of the tile (two-pass statistics in fp32, like the
+// stand-alone kernel) and leaves h = (x - mean) * rstd * gamma + beta as bf16 in the panel; the CTA of
+// column tile 0 also writes h, mean and rstd to global memory for the backward pass.
+__device__ void ln_rows_to_panel(const uint16_t* x, const uint16_t* gamma, const uint16_t* beta, int d, float eps, int m0,
+                                 uint8_t* panel, int stride, bool write, uint16_t* h, float* mu, float* rstd)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, np = d >> 8;     // 16-byte pieces per lane
+    const float inv_d = 1.0f / d;
+    uint4 gq[2], bq[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+        if (i < np) {
+            gq[i] = __ldg(reinterpret_cast<const uint4*>(gamma) + lane + 32 * i);
+            bq[i] = __ldg(reinterpret_cast<const uint4*>(beta) + lane + 32 * i);
+        }
+    for (int batch = 0; batch < 2; ++batch) {
+        uint4 raw[8][2];                                    // eight rows in flight
+#pragma unroll
+        for (int rr = 0; rr < 8; ++rr)
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+                if (i < np)
+                    raw[rr][i] = __ldcg(reinterpret_cast<const uint4*>(x + static_cast<size_t>(m0 + warp * 16 + batch * 8 + rr) * d) + lane + 32 * i);
+#pragma unroll
+        for (int rr = 0; rr < 8; ++rr) {
+            const int row = warp * 16 + batch * 8 + rr;
+            float v[2][8];
+            float s = 0.f;
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+                if (i < np) {
+                    unpack8(raw[rr][i], v[i]);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) s += v[i][e];
+                }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            const float mean = s * inv_d;
+            float q = 0.f;
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+                if (i < np) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) { const float c = v[i][e] - mean; q = fmaf(c, c, q); }
+                }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+            const float rs = rsqrtf(q * inv_d + eps);
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+                if (i < np) {
+                    float g[8], b[8], y[8];
+                    unpack8(gq[i], g);
+                    unpack8(bq[i], b);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) y[e] = fmaf((v[i][e] - mean) * rs, g[e], b[e]);
+                    const uint4 out = pack8(y);
+                    *reinterpret_cast<uint4*>(panel + row * stride + (lane + 32 * i) * 16) = out;
+                    if (write) *(reinterpret_cast<uint4*>(h + static_cast<size_t>(m0 + row) * d) + lane + 32 * i) = out;
+                }
+            if (write && lane == 0) { mu[m0 + row] = mean; rstd[m0 + row] = rs; }
+        }
+    }
+}
+
+// ---------------------------------------------------------------- column sums (bias gradients, dgamma / dbeta)
+// One unit: 16 columns, 8 row lanes; lane sums are added in lane order.  With xhat_of != nullptr it
+// returns sum(in * xhat) in out0 and sum(in) in out1 (xhat = (xhat_of - mu) * rstd), else sum(in) in out0.
+__device__ void colsum_unit(const uint16_t* in, size_t ld, int T, int col0, const uint16_t* xhat_of, const float* mu,
+                            const float* rstd, float* out0, float* out1, int accumulate, float* red)
+{
+    const int tid = threadIdx.x, c = tid & 15, rl = tid >> 4;
+    float s0 = 0.f, s1 = 0.f;
+    if (xhat_of) {
+#pragma unroll 4
+        for (int row = rl; row < T; row += 8) {
+            const float g = ldcg_bf16(in + row * ld + col0 + c);
+            const float xh = (ldcg_bf16(xhat_of + row * ld + col0 + c) - __ldcg(mu + row)) * __ldcg(rstd + row);
+            s0 = fmaf(g, xh, s0);
+            s1 += g;
+        }
+    } else {
+#pragma unroll 8
+        for (int row = rl; row < T; row += 8) s0 += ldcg_bf16(in + row * ld + col0 + c);
+    }
+    red[rl * 16 + c] = s0;
+    red[128 + rl * 16 + c] = s1;
+    __syncthreads();
+    if (tid < 16) {
+        float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+        for (int l = 0; l < 8; ++l) { a0 += red[l * 16 + tid]; a1 += red[128 + l * 16 + tid]; }
+        out0[col0 + tid] = accumulate ? out0[col0 + tid] + a0 : a0;
+        if (xhat_of) out1[col0 + tid] = accumulate ? out1[col0 + tid] + a1 : a1;
+    }
+    __syncthreads();
+}
+
+// ---------------------------------------------------------------- LayerNorm backward, one row per warp
+// dx = resid + rstd * (g - mean(g) - xhat * mean(g * xhat)),  g = dh * gamma
+__device__ void ln_bwd_row(const uint16_t* dh, const uint16_t* x, const float* mu, const float* rstd, const uint16_t* gamma,
+                           const uint16_t* resid, uint16_t* dx, int d, int row)
+{
+    const int lane = threadIdx.x & 31, np = d >> 8;
+    const float m = __ldcg(mu + row), rs = __ldcg(rstd + row), inv_d = 1.0f / d;
+    float g[2][8], xh[2][8];
+    float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+        if (i < np) {
+            float a[8], b[8], c[8];
+            unpack8(__ldcg(reinterpret_cast<const uint4*>(dh + static_cast<size_t>(row) * d) + lane + 32 * i), a);
+            unpack8(__ldcg(reinterpret_cast<const uint4*>(x + static_cast<size_t>(row) * d) + lane + 32 * i), b);
+            unpack8(__ldg(reinterpret_cast<const uint4*>(gamma) + lane + 32 * i), c);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                g[i][e] = a[e] * c[e];
+                xh[i][e] = (b[e] - m) * rs;
+                s1 += g[i][e];
+                s2 = fmaf(g[i][e], xh[i][e], s2);
+            }
+        }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+        s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+    }
+    s1 *= inv_d; s2 *= inv_d;
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+        if (i < np) {
+            float r[8], y[8];
+            unpack8(__ldcg(reinterpret_cast<const uint4*>(resid + static_cast<size_t>(row) * d) + lane + 32 * i), r);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) y[e] = r[e] + rs * (g[i][e] - s1 - xh[i][e] * s2);
+            *(reinterpret_cast<uint4*>(dx + static_cast<size_t>(row) * d) + lane + 32 * i) = pack8(y);
+        }
+}
+
+// ---------------------------------------------------------------- attention units (head_dim 64)
+// rowsum(dO * O) of one row of one head: 64 products added in column order.
+__device__ __forceinline__ float delta_row(const uint16_t* dout, const uint16_t* o, size_t idx)
+{
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        float a[8], b[8];
+        unpack8(__ldcg(reinterpret_cast<const uint4*>(dout + idx) + i), a);
+        unpack8(__ldcg(reinterpret_cast<const uint4*>(o + idx) + i), b);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) s = fmaf(a[e], b[e], s);
+    }
+    return s;
+}
+
+// Forward: 64 query rows of one head; warp w owns rows 16 w .. 16 w + 15, scores and P stay in registers.
+__device__ void attn_fwd_unit(const WholeLayerArgs& p, int b, int h, int qb, uint32_t sm)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const size_t ld = 3 * static_cast<size_t>(p.d);
+    const uint16_t* qkv = static_cast<const uint16_t*>(p.qkv);
+    const uint16_t* base = qkv + static_cast<size_t>(b) * p.S * ld + h * 64;
+    const uint32_t sQ = sm, sK = sm + 2 * kChunk, sV = sm + 3 * kChunk;
+    const float sl2 = p.scale * 1.4426950408889634f;
+    stage_chunk(sQ, base + static_cast<size_t>(qb) * 64 * ld, ld, tid);
+    cp_async_commit();
+    uint32_t qf[4][4];
+    float oacc[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) oacc[i][e] = 0.f;
+    float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
+    for (int j = 0; j <= qb; ++j) {
+        stage_chunk(sK, base + static_cast<size_t>(j) * 64 * ld + p.d, ld, tid);
+        stage_chunk(sV, base + static_cast<size_t>(j) * 64 * ld + 2 * p.d, ld, tid);
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncthreads();
+        if (j == 0) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) frag_a_k(sQ, warp * 16, kk, lane, qf[kk]);
+        }
+        float s[8][4];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) s[i][e] = 0.f;
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                uint32_t bf[4];
+                frag_b_k(sK, np * 16, kk, lane, bf);
+                mma16816(s[2 * np], qf[kk], bf[0], bf[1]);
+                mma16816(s[2 * np + 1], qf[kk], bf[2], bf[3]);
+            }
+        float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int ni = 0; ni < 8; ++ni)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float t = s[ni][e] * sl2;
+                if (j == qb) {
+                    const int key = ni * 8 + 2 * (lane & 3) + (e & 1), row = warp * 16 + (lane >> 2) + 8 * (e >> 1);
+                    if (key > row) t = -INFINITY;
+                }
+                s[ni][e] = t;
+                mx[e >> 1] = fmaxf(mx[e >> 1], t);
+            }
+        float alpha[2];
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 1));
+            mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 2));
+            const float mn = fmaxf(m[hh], mx[hh]);
+            alpha[hh] = exp2f(m[hh] - mn);
+            m[hh] = mn;
+            l[hh] *= alpha[hh];
+        }
+#pragma unroll
+        for (int ni = 0; ni < 8; ++ni)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float pe = exp2f(s[ni][e] - m[e >> 1]);
+                s[ni][e] = pe;
+                l[e >> 1] += pe;
+                oacc[ni][e] *= alpha[e >> 1];
+            }
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+            uint32_t a[4] = {pack_bf16(s[2 * kk][0], s[2 * kk][1]), pack_bf16(s[2 * kk][2], s[2 * kk][3]),
+                             pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]), pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3])};
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                uint32_t bf[4];
+                frag_b_mn(sV, np * 16, kk, lane, bf);
+                mma16816(oacc[2 * np], a, bf[0], bf[1]);
+                mma16816(oacc[2 * np + 1], a, bf[2], bf[3]);
+            }
+        }
+        __syncthreads();                                    // K and V may be overwritten
+    }
+    uint16_t* o = static_cast<uint16_t*>(p.o);
+    float* lse = static_cast<float*>(p.lse);
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        l[hh] += __shfl_xor_sync(0xffffffffu, l[hh], 1);
+        l[hh] += __shfl_xor_sync(0xffffffffu, l[hh], 2);
+        const float inv = 1.0f / l[hh];
+        const int q = qb * 64 + warp * 16 + (lane >> 2) + 8 * hh;
+        const size_t row = static_cast<size_t>(b) * p.S + q;
+#pragma unroll
+        for (int ni = 0; ni < 8; ++ni)
+            store_bf16x2(o, row * p.d + h * 64 + ni * 8 + 2 * (lane & 3), oacc[ni][2 * hh] * inv, oacc[ni][2 * hh + 1] * inv);
+        if ((lane & 3) == 0) lse[(static_cast<size_t>(b) * p.H + h) * p.S + q] = m[hh] * 0.6931471805599453f + logf(l[hh]);
+    }
+}
+
+// Backward, dQ of 64 query rows of one head: per key block S and dP are rebuilt, dS = P (dP - delta)
+// goes straight from the accumulator registers into the A operand of dQ += dS K.
+__device__ void attn_dq_unit(const WholeLayerArgs& p, int b, int h, int qb, uint32_t sm, float* vec)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const size_t ld = 3 * static_cast<size_t>(p.d);
+    const uint16_t* base = static_cast<const uint16_t*>(p.qkv) + static_cast<size_t>(b) * p.S * ld + h * 64;
+    const uint16_t* dout = static_cast<const uint16_t*>(p.td0);
+    const uint16_t* o = static_cast<const uint16_t*>(p.o);
+    const uint32_t sQ = sm, sDO = sm + kChunk, sK = sm + 2 * kChunk, sV = sm + 3 * kChunk;
+    const float sl2 = p.scale * 1.4426950408889634f;
+    const size_t row0 = static_cast<size_t>(b) * p.S + qb * 64;
+    stage_chunk(sQ, base + static_cast<size_t>(qb) * 64 * ld, ld, tid);
+    stage_chunk(sDO, dout + row0 * p.d + h * 64, p.d, tid);
+    cp_async_commit();
+    if (tid < 64) vec[tid] = delta_row(dout, o, (row0 + tid) * p.d + h * 64);
+    float lse2[2], dlt[2];
+    uint32_t qf[4][4], dof[4][4];
+    float dq[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) dq[i][e] = 0.f;
+    for (int j = 0; j <= qb; ++j) {
+        stage_chunk(sK, base + static_cast<size_t>(j) * 64 * ld + p.d, ld, tid);
+        stage_chunk(sV, base + static_cast<size_t>(j) * 64 * ld + 2 * p.d, ld, tid);
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncthreads();
+        if (j == 0) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                frag_a_k(sQ, warp * 16, kk, lane, qf[kk]);
+                frag_a_k(sDO, warp * 16, kk, lane, dof[kk]);
+            }
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const int r = warp * 16 + (lane >> 2) + 8 * hh;
+                lse2[hh] = __ldcg(static_cast<const float*>(p.lse) + (static_cast<size_t>(b) * p.H + h) * p.S + qb * 64 + r) * 1.4426950408889634f;
+                dlt[hh] = vec[r];
+            }
+        }
+        float s[8][4], dp[8][4];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { s[i][e] = 0.f; dp[i][e] = 0.f; }
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                uint32_t bf[4];
+                frag_b_k(sK, np * 16, kk, lane, bf);
+                mma16816(s[2 * np], qf[kk], bf[0], bf[1]);
+                mma16816(s[2 * np + 1], qf[kk], bf[2], bf[3]);
+                frag_b_k(sV, np * 16, kk, lane, bf);
+                mma16816(dp[2 * np], dof[kk], bf[0], bf[1]);
+                mma16816(dp[2 * np + 1], dof[kk], bf[2], bf[3]);
+            }
+#pragma unroll
+        for (int ni = 0; ni < 8; ++ni)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float pe = exp2f(fmaf(s[ni][e], sl2, -lse2[e >> 1]));
+                if (j == qb) {
+                    const int key = ni * 8 + 2 * (lane & 3) + (e & 1), row = warp * 16 + (lane >> 2) + 8 * (e >> 1);
+                    if (key > row) pe = 0.f;
+                }
+                s[ni][e] = pe * (dp[ni][e] - dlt[e >> 1]);
+            }
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+            uint32_t a[4] = {pack_bf16(s[2 * kk][0], s[2 * kk][1]), pack_bf16(s[2 * kk][2], s[2 * kk][3]),
+                             pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]), pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3])};
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                uint32_t bf[4];
+                frag_b_mn(sK, np * 16, kk, lane, bf);
+                mma16816(dq[2 * np], a, bf[0], bf[1]);
+                mma16816(dq[2 * np + 1], a, bf[2], bf[3]);
+            }
+        }
+        __syncthreads();
+    }
+    uint16_t* dqkv = static_cast<uint16_t*>(p.big);
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        const size_t row = row0 + warp * 16 + (lane >> 2) + 8 * hh;
+#pragma unroll
+        for (int ni = 0; ni < 8; ++ni)
+            store_bf16x2(dqkv, row * ld + h * 64 + ni * 8 + 2 * (lane & 3), dq[ni][2 * hh] * p.scale, dq[ni][2 * hh + 1] * p.scale);
+    }
+}
+
+// Backward, dK and dV of 64 key rows of one head: per query block the transposed scores K Q^T and
+// V dO^T are built, so that P^T and dS^T come out of the accumulators as A operands.
+__device__ void attn_dkdv_unit(const WholeLayerArgs& p, int b, int h, int kb, uint32_t sm, float* vec)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const size_t ld = 3 * static_cast<size_t>(p.d);
+    const uint16_t* base = static_cast<const uint16_t*>(p.qkv) + static_cast<size_t>(b) * p.S * ld + h * 64;
+    const uint16_t* dout = static_cast<const uint16_t*>(p.td0);
+    const uint16_t* o = static_cast<const uint16_t*>(p.o);
+    const uint32_t sK = sm, sV = sm + kChunk, sQ = sm + 2 * kChunk, sDO = sm + 3 * kChunk;
+    const float sl2 = p.scale * 1.4426950408889634f;
+    const size_t seq0 = static_cast<size_t>(b) * p.S;
+    float* v_lse = vec;                                     // [S] lse * log2(e)
+    float* v_dlt = vec + kMaxS;                             // [S]
+    stage_chunk(sK, base + static_cast<size_t>(kb) * 64 * ld + p.d, ld, tid);
+    stage_chunk(sV, base + static_cast<size_t>(kb) * 64 * ld + 2 * p.d, ld, tid);
+    cp_async_commit();
+    for (int r = kb * 64 + tid; r < p.S; r += kThreads) {
+        v_lse[r] = __ldcg(static_cast<const float*>(p.lse) + (static_cast<size_t>(b) * p.H + h) * p.S + r) * 1.4426950408889634f;
+        v_dlt[r] = delta_row(dout, o, (seq0 + r) * p.d + h * 64);
+    }
+    uint32_t kf[4][4], vf[4][4];
+    float dk[8][4], dv[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { dk[i][e] = 0.f; dv[i][e] = 0.f; }
+    const int nqb = p.S >> 6;
+    for (int i = kb; i < nqb; ++i) {
+        stage_chunk(sQ, base + static_cast<size_t>(i) * 64 * ld, ld, tid);
+        stage_chunk(sDO, dout + (seq0 + i * 64) * p.d + h * 64, p.d, tid);
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncthreads();
+        if (i == kb) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                frag_a_k(sK, warp * 16, kk, lane, kf[kk]);
+                frag_a_k(sV, warp * 16, kk, lane, vf[kk]);
+            }
+        }
+        float st[8][4], dpt[8][4];
+#pragma unroll
+        for (int a = 0; a < 8; ++a)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { st[a][e] = 0.f; dpt[a][e] = 0.f; }
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                uint32_t bf[4];
+                frag_b_k(sQ, np * 16, kk, lane, bf);
+                mma16816(st[2 * np], kf[kk], bf[0], bf[1]);
+                mma16816(st[2 * np + 1], kf[kk], bf[2], bf[3]);
+                frag_b_k(sDO, np * 16, kk, lane, bf);
+                mma16816(dpt[2 * np], vf[kk], bf[0], bf[1]);
+                mma16816(dpt[2 * np + 1], vf[kk], bf[2], bf[3]);
+            }
+        // st -> P^T (kept for dV), dpt -> dS^T
+#pragma unroll
+        for (int ni = 0; ni < 8; ++ni)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int qcol = ni * 8 + 2 * (lane & 3) + (e & 1), q = i * 64 + qcol;
+                float pe = exp2f(fmaf(st[ni][e], sl2, -v_lse[q]));
+                if (i == kb) {
+                    const int key = warp * 16 + (lane >> 2) + 8 * (e >> 1);
+                    if (key > qcol) pe = 0.f;
+                }
+                st[ni][e] = pe;
+                dpt[ni][e] = pe * (dpt[ni][e] - v_dlt[q]);
+            }
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+            uint32_t a[4] = {pack_bf16(st[2 * kk][0], st[2 * kk][1]), pack_bf16(st[2 * kk][2], st[2 * kk][3]),
+                             pack_bf16(st[2 * kk + 1][0], st[2 * kk + 1][1]), pack_bf16(st[2 * kk + 1][2], st[2 * kk + 1][3])};
+            uint32_t c[4] = {pack_bf16(dpt[2 * kk][0], dpt[2 * kk][1]), pack_bf16(dpt[2 * kk][2], dpt[2 * kk][3]),
+                             pack_bf16(dpt[2 * kk + 1][0], dpt[2 * kk + 1][1]), pack_bf16(dpt[2 * kk + 1][2], dpt[2 * kk + 1][3])};
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                uint32_t bf[4];
+                frag_b_mn(sDO, np * 16, kk, lane, bf);
+                mma16816(dv[2 * np], a, bf[0], bf[1]);
+                mma16816(dv[2 * np + 1], a, bf[2], bf[3]);
+                frag_b_mn(sQ, np * 16, kk, lane, bf);
+                mma16816(dk[2 * np], c, bf[0], bf[1]);
+                mma16816(dk[2 * np + 1], c, bf[2], bf[3]);
+            }
+        }
+        __syncthreads();
+    }
+    uint16_t* dqkv = static_cast<uint16_t*>(p.big);
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        const size_t row = seq0 + kb * 64 + warp * 16 + (lane >> 2) + 8 * hh;
+#pragma unroll
+        for (int ni = 0; ni < 8; ++ni) {
+            const size_t at = row * ld + h * 64 + ni * 8 + 2 * (lane & 3);
+            store_bf16x2(dqkv, at + p.d, dk[ni][2 * hh] * p.scale, dk[ni][2 * hh + 1] * p.scale);
+            store_bf16x2(dqkv, at + 2 * p.d, dv[ni][2 * hh], dv[ni][2 * hh + 1]);
+        }
+    }
+}
+
+// ---------------------------------------------------------------- the phases
+struct Ctx {
+    const WholeLayerArgs& p;
+    uint8_t* smem;
+    uint32_t sm;                // shared-memory address of smem
+    int* flag;
+    unsigned* sem;
+    float* ws;
+};
+
+// Forward GEMM tile with bias and one of: nothing, residual, GeLU (writes u and a).
+enum { kFwdBias = 0, kFwdResid = 1, kFwdGelu = 2 };
+template <bool LN>
+__device__ void fwd_gemm_unit(const Ctx& c, int u, int mode, const uint16_t* A, int K, const uint16_t* W, const uint16_t* bias,
+                              int N, int nslices, const uint16_t* resid, uint16_t* out, uint16_t* out_act,
+                              const uint16_t* ln_g, const uint16_t* ln_b, uint16_t* ln_h, float* ln_mu, float* ln_rs)
+{
+    const WholeLayerArgs& p = c.p;
+    const int tile = u / nslices, slice = u % nslices, ntn = N >> 6, tm = tile / ntn, tn = tile % ntn;
+    const int m0 = tm * 64, n0 = tn * 64, kper = K / nslices;
+    float acc[2][4][4];
+    const int stride = (p.d + 8) * 2;
+    if (LN) {
+        ln_rows_to_panel(A, ln_g, ln_b, p.d, p.eps, m0, c.smem + kSmPanel, stride, tn == 0, ln_h, ln_mu, ln_rs);
+        gemm_tile<false, false, true>(acc, nullptr, 0, W, K, m0, n0, 0, K, c.sm + kSmStage, c.sm + kSmPanel, stride);
+    } else {
+        gemm_tile<false, false, false>(acc, A, K, W, K, m0, n0, slice * kper, (slice + 1) * kper, c.sm + kSmStage, 0, 0);
+        if (!splitk_combine(acc, c.ws, c.sem, tile, slice, nslices, c.flag)) return;
+    }
+    const int act = p.act;
+    for_each_pair(acc, m0, n0, [&](int row, int col, float v0, float v1) {
+        const uint32_t bb = __ldg(reinterpret_cast<const uint32_t*>(bias + col));
+        v0 += bf16_lo(bb); v1 += bf16_hi(bb);
+        const size_t idx = static_cast<size_t>(row) * N + col;
+        if (mode == kFwdResid) {
+            float r0, r1;
+            load_bf16x2(resid, idx, r0, r1);
+            v0 += r0; v1 += r1;
+        }
+        store_bf16x2(out, idx, v0, v1);
+        if (mode == kFwdGelu) {
+            gelu2(v0, v1, act);
+            store_bf16x2(out_act, idx, v0, v1);
+        }
+    });
+}
+
+// Data-gradient tile: out[T, N] = A[T, K] W[K, N] (W stored [K][N]); with u != nullptr the result is
+// multiplied by GeLU'(u).
+__device__ void dgrad_unit(const Ctx& c, int u, const uint16_t* A, int K, const uint16_t* W, int N, int nslices,
+                           const uint16_t* gelu_u, uint16_t* out)
+{
+    const int tile = u / nslices, slice = u % nslices, ntn = N >> 6, m0 = (tile / ntn) * 64, n0 = (tile % ntn) * 64;
+    const int kper = K / nslices;
+    float acc[2][4][4];
+    gemm_tile<false, true, false>(acc, A, K, W, N, m0, n0, slice * kper, (slice + 1) * kper, c.sm + kSmStage, 0, 0);
+    if (!splitk_combine(acc, c.ws, c.sem, tile, slice, nslices, c.flag)) return;
+    const int act = c.p.act;
+    for_each_pair(acc, m0, n0, [&](int row, int col, float v0, float v1) {
+        const size_t idx = static_cast<size_t>(row) * N + col;
+        if (gelu_u) {
+            float u0, u1;
+            load_bf16x2(gelu_u, idx, u0, u1);
+            gelu_grad_mul2(v0, v1, u0, u1, act);
+        }
+        store_bf16x2(out, idx, v0, v1);
+    });
+}
+
+// Weight-gradient tile: dW[M, N] (+)= A[T, M]^T B[T, N], fp32.
+__device__ void wgrad_unit(const Ctx& c, int u, const uint16_t* A, int M, const uint16_t* B, int N, float* dW)
+{
+    const int ntn = N >> 6, m0 = (u / ntn) * 64, n0 = (u % ntn) * 64;
+    float acc[2][4][4];
+    gemm_tile<true, true, false>(acc, A, M, B, N, m0, n0, 0, c.p.T, c.sm + kSmStage, 0, 0);
+    const int accumulate = c.p.accumulate;
+    for_each_pair(acc, m0, n0, [&](int row, int col, float v0, float v1) {
+        float2* dst = reinterpret_cast<float2*>(dW + static_cast<size_t>(row) * N + col);
+        if (accumulate) { const float2 old = *dst; v0 += old.x; v1 += old.y; }
+        *dst = make_float2(v0, v1);
+    });
+}
+
+__device__ __forceinline__ const uint16_t* cu16(const void* q) { return static_cast<const uint16_t*>(q); }
+__device__ __forceinline__ uint16_t* u16(void* q) { return static_cast<uint16_t*>(q); }
+__device__ __forceinline__ float* f32(void* q) { return static_cast<float*>(q); }
+
+__global__ void __launch_bounds__(kThreads, 1) whole_layer_fwd_kernel(const __grid_constant__ WholeLayerArgs p)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const Ctx c{p, smem, smem_u32(smem), reinterpret_cast<int*>(smem + kSmFlag), p.sync + 2, f32(p.splitk)};
+    if (*reinterpret_cast<volatile int*>(&p.status->code) != 0) return;
+    const int T = p.T, d = p.d, F = p.F, G = gridDim.x, tm = T >> 6;
+    // 1: qkv = LN1(x) Wqkv^T + bqkv (h1, mean, rstd written by the first column tile of each row block)
+    for (int u = blockIdx.x; u < tm * (3 * d >> 6); u += G)
+        fwd_gemm_unit<true>(c, u, kFwdBias, cu16(p.x), d, cu16(p.w_qkv), cu16(p.b_qkv), 3 * d, 1, nullptr, u16(p.qkv), nullptr,
+                            cu16(p.ln1_g), cu16(p.ln1_b), u16(p.h1), f32(p.mu1), f32(p.r1));
+    if (!grid_barrier(p.sync, p.status, c.flag)) return;
+    // 2: o = attention(qkv)
+    {
+        const int nqb = p.S >> 6, n = p.B * p.H * nqb;
+        for (int u = blockIdx.x; u < n; u += G) {
+            const int qb = nqb - 1 - u / (p.B * p.H), bh = u % (p.B * p.H);      // long rows first
+            attn_fwd_unit(p, bh / p.H, bh % p.H, qb, c.sm + kSmStage);
+        }
+    }
+    if (!grid_barrier(p.sync, p.status, c.flag)) return;
+    // 3: x1 = x + o Wo^T + bo
+    for (int u = blockIdx.x; u < tm * (d >> 6) * p.split_d; u += G)
+        fwd_gemm_unit<false>(c, u, kFwdResid, cu16(p.o), d, cu16(p.w_o), cu16(p.b_o), d, p.split_d, cu16(p.x), u16(p.x1), nullptr,
+                             nullptr, nullptr, nullptr, nullptr, nullptr);
+    if (!grid_barrier(p.sync, p.status, c.flag)) return;
+    // 4: u = LN2(x1) W1^T + b1, a = GeLU(u)
+    for (int u = blockIdx.x; u < tm * (F >> 6); u += G)
+        fwd_gemm_unit<true>(c, u, kFwdGelu, cu16(p.x1), d, cu16(p.w_fc1), cu16(p.b_fc1), F, 1, nullptr, u16(p.u), u16(p.a),
+                            cu16(p.ln2_g), cu16(p.ln2_b), u16(p.h2), f32(p.mu2), f32(p.r2));
+    if (!p.with_fc2) return;
+    if (!grid_barrier(p.sync, p.status, c.flag)) return;
+    // 5: y = x1 + a W2^T + b2
+    for (int u = blockIdx.x; u < tm * (d >> 6) * p.split_f; u += G)
+        fwd_gemm_unit<false>(c, u, kFwdResid, cu16(p.a), F, cu16(p.w_fc2), cu16(p.b_fc2), d, p.split_f, cu16(p.x1), u16(p.y), nullptr,
+                             nullptr, nullptr, nullptr, nullptr, nullptr);
+}
+
+__global__ void __launch_bounds__(kThreads, 1) whole_layer_bwd_kernel(const __grid_constant__ WholeLayerArgs p)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const Ctx c{p, smem, smem_u32(smem), reinterpret_cast<int*>(smem + kSmFlag), p.sync + 2, f32(p.splitk)};
+    if (*reinterpret_cast<volatile int*>(&p.status->code) != 0) return;
+    const int T = p.T, d = p.d, F = p.F, G = gridDim.x, tm = T >> 6, warp = threadIdx.x >> 5;
+    float* red = reinterpret_cast<float*>(smem + kSmRed);
+    float* vec = reinterpret_cast<float*>(smem + kSmVec);
+    const int acc = p.accumulate;
+    // 1: du = (dy W2) * GeLU'(u);  dW2 = dy^T a;  db2 = colsum(dy)
+    {
+        const int n0 = tm * (F >> 6), n1 = n0 + (d >> 6) * (F >> 6), n2 = n1 + (d >> 4);
+        for (int u = blockIdx.x; u < n2; u += G) {
+            if (u < n0) dgrad_unit(c, u, cu16(p.dy), d, cu16(p.w_fc2), F, 1, cu16(p.u), u16(p.big));
+            else if (u < n1) wgrad_unit(c, u - n0, cu16(p.dy), d, cu16(p.a), F, f32(p.g_w_fc2));
+            else colsum_unit(cu16(p.dy), d, T, (u - n1) * 16, nullptr, nullptr, nullptr, f32(p.g_b_fc2), nullptr, acc, red);
+        }
+    }
+    if (!grid_barrier(p.sync, p.status, c.flag)) return;
+    // 2: dh2 = du W1;  dW1 = du^T h2;  db1 = colsum(du)
+    {
+        const int n0 = tm * (d >> 6) * p.split_f, n1 = n0 + (F >> 6) * (d >> 6), n2 = n1 + (F >> 4);
+        for (int u = blockIdx.x; u < n2; u += G) {
+            if (u < n0) dgrad_unit(c, u, cu16(p.big), F, cu16(p.w_fc1), d, p.split_f, nullptr, u16(p.td0));
+            else if (u < n1) wgrad_unit(c, u - n0, cu16(p.big), F, cu16(p.h2), d, f32(p.g_w_fc1));
+            else colsum_unit(cu16(p.big), F, T, (u - n1) * 16, nullptr, nullptr, nullptr, f32(p.g_b_fc1), nullptr, acc, red);
+        }
+    }
+    if (!grid_barrier(p.sync, p.status, c.flag)) return;
+    // 3: dx1 = dy + LN2bwd(dh2);  dgamma2, dbeta2
+    {
+        const int n0 = T >> 2, n1 = n0 + (d >> 4);
+        for (int u = blockIdx.x; u < n1; u += G) {
+            if (u < n0) ln_bwd_row(cu16(p.td0), cu16(p.x1), f32(p.mu2), f32(p.r2), cu16(p.ln2_g), cu16(p.dy), u16(p.dx1), d, u * 4 + warp);
+            else colsum_unit(cu16(p.td0), d, T, (u - n0) * 16, cu16(p.x1), f32(p.mu2), f32(p.r2), f32(p.g_ln2_g), f32(p.g_ln2_b), acc, red);
+        }
+    }
+    if (!grid_barrier(p.sync, p.status, c.flag)) return;
+    // 4: dout = dx1 Wo;  dWo = dx1^T o;  dbo = colsum(dx1)
+    {
+        const int n0 = tm * (d >> 6) * p.split_d, n1 = n0 + (d >> 6) * (d >> 6), n2 = n1 + (d >> 4);
+        for (int u = blockIdx.x; u < n2; u += G) {
+            if (u < n0) dgrad_unit(c, u, cu16(p.dx1), d, cu16(p.w_o), d, p.split_d, nullptr, u16(p.td0));
+            else if (u < n1) wgrad_unit(c, u - n0, cu16(p.dx1), d, cu16(p.o), d, f32(p.g_w_o));
+            else colsum_unit(cu16(p.dx1), d, T, (u - n1) * 16, nullptr, nullptr, nullptr, f32(p.g_b_o), nullptr, acc, red);
+        }
+    }
+    if (!grid_barrier(p.sync, p.status, c.flag)) return;
+    // 5: dqkv = attention backward (delta is taken by each unit from dout and o)
+    {
+        const int nb = p.S >> 6, BH = p.B * p.H, n = BH * nb;
+        for (int u = blockIdx.x; u < 2 * n; u += G) {
+            const int v = u >> 1, blk = v / BH, bh = v % BH;
+            if (u & 1) attn_dq_unit(p, bh / p.H, bh % p.H, nb - 1 - blk, c.sm + kSmStage, vec);     // long rows first
+            else attn_dkdv_unit(p, bh / p.H, bh % p.H, blk, c.sm + kSmStage, vec);                  // long columns first
+            __syncthreads();
+        }
+    }
+    if (!grid_barrier(p.sync, p.status, c.flag)) return;
+    // 6: dh1 = dqkv Wqkv;  dWqkv = dqkv^T h1;  dbqkv = colsum(dqkv)
+    {
+        const int n0 = tm * (d >> 6) * p.split_3d, n1 = n0 + (3 * d >> 6) * (d >> 6), n2 = n1 + (3 * d >> 4);
+        for (int u = blockIdx.x; u < n2; u += G) {
+            if (u < n0) dgrad_unit(c, u, cu16(p.big), 3 * d, cu16(p.w_qkv), d, p.split_3d, nullptr, u16(p.td0));
+            else if (u < n1) wgrad_unit(c, u - n0, cu16(p.big), 3 * d, cu16(p.h1), d, f32(p.g_w_qkv));
+            else colsum_unit(cu16(p.big), 3 * d, T, (u - n1) * 16, nullptr, nullptr, nullptr, f32(p.g_b_qkv), nullptr, acc, red);
+        }
+    }
+    if (!grid_barrier(p.sync, p.status, c.flag)) return;
+    // 7: dx = dx1 + LN1bwd(dh1);  dgamma1, dbeta1
+    {
+        const int n0 = T >> 2, n1 = n0 + (d >> 4);
+        for (int u = blockIdx.x; u < n1; u += G) {
+            if (u < n0) ln_bwd_row(cu16(p.td0), cu16(p.x), f32(p.mu1), f32(p.r1), cu16(p.ln1_g), cu16(p.dx1), u16(p.dx), d, u * 4 + warp);
+            else colsum_unit(cu16(p.td0), d, T, (u - n0) * 16, cu16(p.x), f32(p.mu1), f32(p.r1), f32(p.g_ln1_g), f32(p.g_ln1_b), acc, red);
+        }
+    }
+}
+
+cudaError_t launch_coop(void (*kern)(const WholeLayerArgs), int grid, cudaStream_t st, const WholeLayerArgs& a)
+{
+    Tuning& tn = tuning();
+    if (tn.fail_launch_countdown > 0 && --tn.fail_launch_countdown == 0) return cudaErrorLaunchFailure;   // injected by a test
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kSmBytes; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeCooperative;
+    at[0].val.cooperative = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
+}  // namespace
+
+const char* configure_whole_layer()
+{
+    if (cudaFuncSetAttribute(whole_layer_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(whole_layer_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmBytes) != cudaSuccess)
+        return "could not set the whole-layer kernels' shared-memory size";
+    return nullptr;
+}
+
+const char* whole_layer_unsupported(int T, int d, int H, int dh, int F, int S)
+{
+    (void)H;
+    if (dh != 64) return "the whole-layer kernel needs head_dim 64";
+    if (d > kMaxD) return "the whole-layer kernel needs d_model <= 512";
+    if (S > kMaxS) return "the whole-layer kernel needs seq_len <= 1024";
+    if ((T >> 6) * (d >> 6) > kWholeLayerMaxTiles) return "the whole-layer kernel needs (tokens / 64) * (d_model / 64) <= 1024";
+    if (F % 64 != 0 || d % 256 != 0 || T % 64 != 0) return "the whole-layer kernel needs tokens and d_ff in multiples of 64";
+    return nullptr;
+}
+
+// Slices of the K range of a GEMM with `tiles` output tiles: as many as keep every slice at least
+// two 64-wide blocks long, divide the block count, and do not push the phase beyond one round of CTAs.
+static int pick_slices(int tiles, int K, int grid)
+{
+    const int blocks = K / 64;
+    int best = 1;
+    for (int s = 2; s <= 8; ++s)
+        if (blocks % s == 0 && blocks / s >= 2 && tiles * s <= grid) best = s;
+    return best;
+}
+
+size_t whole_layer_splitk_bytes(int T, int d) { return static_cast<size_t>(T >> 6) * (d >> 6) * 8 * 4096 * sizeof(float); }
+
+const char* launch_whole_layer(Runtime* rt, WholeLayerArgs a, bool backward, cudaStream_t stream)
+{
+    const int grid = rt->sm_count;
+    const int tiles = (a.T >> 6) * (a.d >> 6);
+    a.split_d = pick_slices(tiles, a.d, grid);
+    a.split_f = pick_slices(tiles, a.F, grid);
+    a.split_3d = pick_slices(tiles, 3 * a.d, grid);
+    const cudaError_t e = launch_coop(backward ? whole_layer_bwd_kernel : whole_layer_fwd_kernel, grid, stream, a);
+    return e == cudaSuccess ? nullptr : cudaGetErrorString(e);
+}
+
+}  // namespace pw

@@ -73,8 +73,8 @@ def dims_of(w):
     return Dims(w.batch, w.seq_len, w.d_model, w.n_heads, w.head_dim, w.d_ff)
 
 
-def make_layer(pw, w, act=0):
-    return pw.Layer(w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch, act=act)
+def make_layer(pw, w, act=0, flags=0):
+    return pw.Layer(w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch, act=act, flags=flags)
 
 
 def zeros_like_params(w, device="cuda"):

@@ -34,13 +34,13 @@ def pw():
     return binding
 
 
-def check_layer_against_oracle(pw, oracle, w, random_ln=False, act=0, save_ctx=True):
+def check_layer_against_oracle(pw, oracle, w, random_ln=False, act=0, save_ctx=True, flags=0):
     from oracle import Dims
     D = dims_of(w)
     D = Dims(D.B, D.S, D.d, D.H, D.dh, D.F, D.eps, act)
     params = inputs.layer_params(w, seed=0, layer=0, random_ln=random_ln)
     x, dy = inputs.microbatch(w, seed=0, m=0)
-    layer = make_layer(pw, w, act)
+    layer = make_layer(pw, w, act, flags)
     out = run_layer_gpu(pw, layer, [p.cuda() for p in params], x.cuda().view(-1, w.d_model),
                         dy.cuda().view(-1, w.d_model), save_ctx=save_ctx)
     cast = (lambda t: t.float().numpy()) if oracle.suf == "f32" else np64
@@ -159,8 +159,8 @@ def test_wide_layers_at_reduced_token_count(pw, oracle32, d, H, F, S):
 
 
 # ------------------------------------------------------------------------------------------ stage chain
-def run_chain_gpu(pw, w, L, M, dispatch, schedule, recompute, seed=0, random_ln=True, mbs=None):
-    stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
+def run_chain_gpu(pw, w, L, M, dispatch, schedule, recompute, seed=0, random_ln=True, mbs=None, flags=0, counts=None):
+    stage = pw.Stage(L, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch, flags=flags)
     params = [[p.cuda() for p in inputs.layer_params(w, seed, l, random_ln=random_ln)] for l in range(L)]
     grads = [[torch.full(p.shape, float("nan"), dtype=torch.float32, device="cuda") for p in ps] for ps in params]
     if mbs is None:
@@ -177,6 +177,8 @@ def run_chain_gpu(pw, w, L, M, dispatch, schedule, recompute, seed=0, random_ln=
             stage.run_chain(params, grads, xs, dys, ys, dxs, ws, dispatch, schedule, recompute, stream=stream)
     torch.cuda.synchronize()
     assert stage.status() == (0, 0)
+    if counts is not None:
+        counts.append(stage.launch_count() // reps)
     return ys, dxs, grads
 
 
