@@ -24,14 +24,16 @@ namespace {
 
 constexpr int kThreads = 128;
 constexpr int kChunk = 64 * 64 * 2;                 // one 64 x 64 bf16 operand chunk
-constexpr int kStages = 3;
+constexpr int kStages = 5;                            // four 64-wide K blocks in flight: K = 256 is one trip to L2
 constexpr int kMaxD = 512;                          // LayerNorm panel: 64 rows of the full width in shared memory
 constexpr int kMaxS = 1024;
 constexpr int kSmStage = 0;                         // kStages x (A chunk, B chunk); attention: Q/K/V/dO chunks
-constexpr int kSmPanel = kSmStage + kStages * 2 * kChunk;
+constexpr int kSmAux = kSmStage + kStages * 2 * kChunk;      // one chunk of an epilogue operand (residual, u)
+constexpr int kAccStride = 68;                               // floats per row of the accumulator tile (bank spread)
+constexpr int kSmAcc = kSmAux + kChunk;                      // 64 x 64 accumulators on their way to a rolled epilogue loop
+constexpr int kSmPanel = kSmAcc + 64 * kAccStride * 4;       // also the lanes of a column-sum unit (8 KB)
 constexpr int kSmVec = kSmPanel + 64 * (kMaxD + 8) * 2;     // lse and delta of one (sequence, head)
-constexpr int kSmRed = kSmVec + 2 * kMaxS * 4;              // column-sum lanes
-constexpr int kSmFlag = kSmRed + 2 * 8 * 16 * 4;
+constexpr int kSmFlag = kSmVec + 2 * kMaxS * 4;
 constexpr int kSmBytes = kSmFlag + 16;
 
 constexpr int kSiteBarrier = 900;
@@ -60,35 +62,38 @@ __device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], 
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ unsigned ld_acquire(const unsigned* p)
+__device__ __forceinline__ unsigned long long ld_acquire(const unsigned long long* p)
 {
-    unsigned v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ float ldcg_bf16(const uint16_t* p) { return __uint_as_float(static_cast<uint32_t>(__ldcg(p)) << 16); }
+__device__ __forceinline__ unsigned long long atom_add_acq_rel(unsigned long long* p, unsigned long long v)
+{
+    unsigned long long old;
+    asm volatile("atom.add.acq_rel.gpu.global.u64 %0, [%1], %2;" : "=l"(old) : "l"(p), "l"(v) : "memory");
+    return old;
+}
 
 // ---------------------------------------------------------------- grid barrier
-// sync[0] counts arrivals, sync[1] is the generation.  The last CTA to arrive clears the count and
-// bumps the generation; both words are back in a consistent state when the kernel ends, so the
-// next launch (or a replay of a captured graph) starts from where this one stopped.  A CTA that
-// waits longer than the limit records a timeout in the status word and every CTA leaves.
+// One 64-bit arrival counter that only ever grows: arrival number n belongs to barrier n / G and that
+// barrier is open once the counter reaches (n / G + 1) G, so one atomic per CTA is the whole
+// protocol and the last arrival is itself the release.  Every launch leaves the counter at a multiple
+// of G, which is all the next launch (or the replay of a captured graph) needs.  A CTA that waits
+// longer than the limit records a timeout in the status word and every CTA leaves.
 __device__ bool grid_barrier(unsigned* sync, DeviceStatus* status, int* s_flag)
 {
     __syncthreads();
     if (threadIdx.x == 0) {
         int ok = 1;
-        const unsigned gen = ld_acquire(sync + 1);
-        __threadfence();
-        const unsigned prev = atomicAdd(sync, 1u);
-        if (prev == gridDim.x - 1) {
-            atomicExch(sync, 0u);
-            __threadfence();
-            atomicAdd(sync + 1, 1u);
-        } else {
+        unsigned long long* count = reinterpret_cast<unsigned long long*>(sync);
+        const unsigned long long G = gridDim.x;
+        const unsigned long long mine = atom_add_acq_rel(count, 1ull);
+        const unsigned long long target = (mine / G + 1) * G;
+        if (mine + 1 < target) {
             const long long t0 = clock64();
             unsigned spins = 0;
-            while (ld_acquire(sync + 1) == gen) {
+            while (ld_acquire(count) < target) {
                 if ((++spins & 0xffu) == 0) {
                     if (*reinterpret_cast<volatile int*>(&status->code) != 0) { ok = 0; break; }
                     if (clock64() - t0 > kWaitCycles) {
@@ -99,7 +104,6 @@ __device__ bool grid_barrier(unsigned* sync, DeviceStatus* status, int* s_flag)
                 }
             }
         }
-        __threadfence();
         *s_flag = ok;
     }
     __syncthreads();
@@ -138,69 +142,81 @@ __device__ __forceinline__ void frag_b_mn(uint32_t base, int n0, int kk, int lan
     ldsm4t(base + swz(kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), (n0 >> 3) + (lane >> 4)), b);
 }
 
-// ---------------------------------------------------------------- 64 x 64 output tile, K range [k0, k1)
+// ---------------------------------------------------------------- 64 x 64 output tile, K range [k0, k0 + 64 nk)
 // C[m0.., n0..] = sum_k A(m, k) B(k, n).  A_MN: A is stored [K][M] (else [M][K]); B_MN: B is stored
 // [K][N] (else [N][K]); A_PANEL: the A rows are already in shared memory (LayerNorm output, full width).
 // Warp w owns rows 32 (w & 1) and columns 32 (w >> 1): acc[mi][ni][e] is row 16 mi + lane / 4 + 8 (e / 2),
-// column 8 ni + 2 (lane % 4) + e % 2 of that quarter.
+// column 8 ni + 2 (lane % 4) + e % 2 of that quarter.  prefetch() puts the first chunks in flight, so
+// that whatever the unit does before run() (LayerNorm of the A rows, loads of epilogue operands)
+// overlaps their way from L2.
 template <bool A_MN, bool B_MN, bool A_PANEL>
-__device__ void gemm_tile(float (&acc)[2][4][4], const uint16_t* A, size_t lda, const uint16_t* Bm, size_t ldb, int m0,
-                          int n0, int k0, int k1, uint32_t stage, uint32_t panel, int panel_stride)
-{
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, wm = (warp & 1) * 32, wn = (warp >> 1) * 32;
-#pragma unroll
-    for (int i = 0; i < 2; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.f;
-    const int nk = (k1 - k0) >> 6;
-    auto load = [&](int kc) {
+struct TileGemm {
+    const uint16_t* A; size_t lda;
+    const uint16_t* Bm; size_t ldb;
+    int m0, n0, k0, nk;
+    uint32_t stage;
+
+    __device__ __forceinline__ void load(int kc) const
+    {
+        const int tid = threadIdx.x;
         const uint32_t sa = stage + (kc % kStages) * 2 * kChunk, sb = sa + kChunk;
         const size_t kk0 = k0 + kc * 64;
         if (!A_PANEL) stage_chunk(sa, A_MN ? A + kk0 * lda + m0 : A + m0 * lda + kk0, lda, tid);
         stage_chunk(sb, B_MN ? Bm + kk0 * ldb + n0 : Bm + n0 * ldb + kk0, ldb, tid);
-    };
-#pragma unroll
-    for (int s = 0; s < kStages - 1; ++s) {
-        if (s < nk) load(s);
-        cp_async_commit();
     }
-    for (int kc = 0; kc < nk; ++kc) {
-        cp_async_wait<kStages - 2>();
-        __syncthreads();
-        if (kc + kStages - 1 < nk) load(kc + kStages - 1);
-        cp_async_commit();
-        const uint32_t sa = stage + (kc % kStages) * 2 * kChunk, sb = sa + kChunk;
+    __device__ __forceinline__ void prefetch() const
+    {
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-            uint32_t af[2][4], bf[2][4];
-#pragma unroll
-            for (int mi = 0; mi < 2; ++mi) {
-                if (A_PANEL) {
-                    const int row = wm + mi * 16 + (lane & 15), col = k0 + kc * 64 + kk * 16 + (lane >> 4) * 8;
-                    ldsm4(panel + row * panel_stride + col * 2, af[mi]);
-                } else if (A_MN) {
-                    frag_a_mn(sa, wm + mi * 16, kk, lane, af[mi]);
-                } else {
-                    frag_a_k(sa, wm + mi * 16, kk, lane, af[mi]);
-                }
-            }
-#pragma unroll
-            for (int np = 0; np < 2; ++np) {
-                if (B_MN) frag_b_mn(sb, wn + np * 16, kk, lane, bf[np]);
-                else frag_b_k(sb, wn + np * 16, kk, lane, bf[np]);
-            }
-#pragma unroll
-            for (int mi = 0; mi < 2; ++mi)
-#pragma unroll
-                for (int ni = 0; ni < 4; ++ni)
-                    mma16816(acc[mi][ni], af[mi], bf[ni >> 1][(ni & 1) * 2], bf[ni >> 1][(ni & 1) * 2 + 1]);
+        for (int s = 0; s < kStages - 1; ++s) {
+            if (s < nk) load(s);
+            cp_async_commit();
         }
     }
-    cp_async_wait<0>();
-    __syncthreads();                                        // the stage buffers may be refilled by the next unit
-}
+    __device__ __forceinline__ void run(float (&acc)[2][4][4], uint32_t panel, int panel_stride) const
+    {
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wm = (warp & 1) * 32, wn = (warp >> 1) * 32;
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.f;
+        for (int kc = 0; kc < nk; ++kc) {
+            cp_async_wait<kStages - 2>();
+            __syncthreads();
+            if (kc + kStages - 1 < nk) load(kc + kStages - 1);
+            cp_async_commit();
+            const uint32_t sa = stage + (kc % kStages) * 2 * kChunk, sb = sa + kChunk;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                uint32_t af[2][4], bf[2][4];
+#pragma unroll
+                for (int mi = 0; mi < 2; ++mi) {
+                    if (A_PANEL) {
+                        const int row = wm + mi * 16 + (lane & 15), col = k0 + kc * 64 + kk * 16 + (lane >> 4) * 8;
+                        ldsm4(panel + row * panel_stride + col * 2, af[mi]);
+                    } else if (A_MN) {
+                        frag_a_mn(sa, wm + mi * 16, kk, lane, af[mi]);
+                    } else {
+                        frag_a_k(sa, wm + mi * 16, kk, lane, af[mi]);
+                    }
+                }
+#pragma unroll
+                for (int np = 0; np < 2; ++np) {
+                    if (B_MN) frag_b_mn(sb, wn + np * 16, kk, lane, bf[np]);
+                    else frag_b_k(sb, wn + np * 16, kk, lane, bf[np]);
+                }
+#pragma unroll
+                for (int mi = 0; mi < 2; ++mi)
+#pragma unroll
+                    for (int ni = 0; ni < 4; ++ni)
+                        mma16816(acc[mi][ni], af[mi], bf[ni >> 1][(ni & 1) * 2], bf[ni >> 1][(ni & 1) * 2 + 1]);
+            }
+        }
+        cp_async_wait<0>();
+        __syncthreads();                                    // the stage buffers may be refilled by the next unit
+    }
+};
 
 // Split-K: every slice stores its partial tile, the CTA that arrives last adds the slices in slice
 // order (its own included, from memory) and returns true: it then runs the epilogue.
@@ -238,122 +254,129 @@ __device__ bool splitk_combine(float (&acc)[2][4][4], float* ws, unsigned* sem, 
     return true;
 }
 
-// Calls f(row, col, v0, v1) for every pair of adjacent columns this thread holds of the tile at (m0, n0).
-template <typename F>
-__device__ __forceinline__ void for_each_pair(const float (&acc)[2][4][4], int m0, int n0, F f)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int r = m0 + (warp & 1) * 32 + (lane >> 2), c = n0 + (warp >> 1) * 32 + 2 * (lane & 3);
-#pragma unroll
-    for (int mi = 0; mi < 2; ++mi)
-#pragma unroll
-        for (int ni = 0; ni < 4; ++ni)
-#pragma unroll
-            for (int h = 0; h < 2; ++h) f(r + mi * 16 + h * 8, c + ni * 8, acc[mi][ni][2 * h], acc[mi][ni][2 * h + 1]);
-}
 __device__ __forceinline__ void store_bf16x2(uint16_t* base, size_t idx, float v0, float v1)
 {
     *reinterpret_cast<uint32_t*>(base + idx) = pack_bf16(v0, v1);
 }
-__device__ __forceinline__ void load_bf16x2(const uint16_t* base, size_t idx, float& v0, float& v1)
-{
-    const uint32_t v = __ldcg(reinterpret_cast<const uint32_t*>(base + idx));
-    v0 = bf16_lo(v); v1 = bf16_hi(v);
-}
 
-// ---------------------------------------------------------------- LayerNorm of 64 rows into the panel
-// Warp w normalises rows 16 w .. 16 w + 15 of the tile (two-pass statistics in fp32, like the
-// stand-alone kernel) and leaves h = (x - mean) * rstd * gamma + beta as bf16 in the panel; the CTA of
-// column tile 0 also writes h, mean and rstd to global memory for the backward pass.
-__device__ void ln_rows_to_panel(const uint16_t* x, const uint16_t* gamma, const uint16_t* beta, int d, float eps, int m0,
-                                 uint8_t* panel, int stride, bool write, uint16_t* h, float* mu, float* rstd)
+// ---------------------------------------------------------------- LayerNorm of 64 rows in the panel
+// The 64 rows of x come into the panel by cp.async (ln_stage_rows, one commit group) and are normalised
+// in place by a short rolled loop - code that runs once per launch is paid for by instruction fetch,
+// not by arithmetic.  Warp w owns rows 16 w .. 16 w + 15, four at a time: eight lanes share a row (lane
+// % 8 owns the 16-byte pieces lane % 8 + 8 j), so a row sum is three shuffles.  Two-pass statistics
+// in fp32, like the stand-alone kernel; h = (x - mean) * rstd * gamma + beta replaces x as bf16 and,
+// from the CTA of column tile 0, goes to global memory with mean and rstd for the backward pass.
+__device__ __forceinline__ void ln_stage_rows(const uint16_t* x, int d, int m0, uint32_t panel, int stride)
 {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, np = d >> 8;     // 16-byte pieces per lane
+    const int per_row = d >> 3;                             // 16-byte pieces per row
+#pragma unroll 1
+    for (int q = threadIdx.x; q < 64 * per_row; q += kThreads) {
+        const int row = q / per_row, piece = q - row * per_row;
+        cp_async16(panel + row * stride + piece * 16, x + static_cast<size_t>(m0 + row) * d + piece * 8);
+    }
+}
+template <int NP>
+__device__ __forceinline__ void ln_rows_in_panel(const uint16_t* gamma, const uint16_t* beta, float eps, int m0, uint8_t* panel,
+                                                 int stride, bool write, uint16_t* h, float* mu, float* rstd)
+{
+    constexpr int d = 256 * NP, kPieces = 4 * NP;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, sub = lane & 7, rsel = lane >> 3;
     const float inv_d = 1.0f / d;
-    uint4 gq[2], bq[2];
+    uint4 gq[kPieces], bq[kPieces];
 #pragma unroll
-    for (int i = 0; i < 2; ++i)
-        if (i < np) {
-            gq[i] = __ldg(reinterpret_cast<const uint4*>(gamma) + lane + 32 * i);
-            bq[i] = __ldg(reinterpret_cast<const uint4*>(beta) + lane + 32 * i);
+    for (int j = 0; j < kPieces; ++j) {
+        gq[j] = __ldg(reinterpret_cast<const uint4*>(gamma) + sub + 8 * j);
+        bq[j] = __ldg(reinterpret_cast<const uint4*>(beta) + sub + 8 * j);
+    }
+#pragma unroll 1
+    for (int it = 0; it < 4; ++it) {
+        const int row = warp * 16 + it * 4 + rsel;
+        uint4* prow = reinterpret_cast<uint4*>(panel + row * stride);
+        float v[kPieces][8];
+        float s = 0.f;
+#pragma unroll
+        for (int j = 0; j < kPieces; ++j) {
+            unpack8(prow[sub + 8 * j], v[j]);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) s += v[j][e];
         }
-    for (int batch = 0; batch < 2; ++batch) {
-        uint4 raw[8][2];                                    // eight rows in flight
 #pragma unroll
-        for (int rr = 0; rr < 8; ++rr)
+        for (int o = 4; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        const float mean = s * inv_d;
+        float q = 0.f;
 #pragma unroll
-            for (int i = 0; i < 2; ++i)
-                if (i < np)
-                    raw[rr][i] = __ldcg(reinterpret_cast<const uint4*>(x + static_cast<size_t>(m0 + warp * 16 + batch * 8 + rr) * d) + lane + 32 * i);
+        for (int j = 0; j < kPieces; ++j)
 #pragma unroll
-        for (int rr = 0; rr < 8; ++rr) {
-            const int row = warp * 16 + batch * 8 + rr;
-            float v[2][8];
-            float s = 0.f;
+            for (int e = 0; e < 8; ++e) { const float c = v[j][e] - mean; q = fmaf(c, c, q); }
 #pragma unroll
-            for (int i = 0; i < 2; ++i)
-                if (i < np) {
-                    unpack8(raw[rr][i], v[i]);
+        for (int o = 4; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+        const float rs = rsqrtf(q * inv_d + eps);
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) s += v[i][e];
-                }
+        for (int j = 0; j < kPieces; ++j) {
+            float g[8], b[8], y[8];
+            unpack8(gq[j], g);
+            unpack8(bq[j], b);
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-            const float mean = s * inv_d;
-            float q = 0.f;
-#pragma unroll
-            for (int i = 0; i < 2; ++i)
-                if (i < np) {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) { const float c = v[i][e] - mean; q = fmaf(c, c, q); }
-                }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
-            const float rs = rsqrtf(q * inv_d + eps);
-#pragma unroll
-            for (int i = 0; i < 2; ++i)
-                if (i < np) {
-                    float g[8], b[8], y[8];
-                    unpack8(gq[i], g);
-                    unpack8(bq[i], b);
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) y[e] = fmaf((v[i][e] - mean) * rs, g[e], b[e]);
-                    const uint4 out = pack8(y);
-                    *reinterpret_cast<uint4*>(panel + row * stride + (lane + 32 * i) * 16) = out;
-                    if (write) *(reinterpret_cast<uint4*>(h + static_cast<size_t>(m0 + row) * d) + lane + 32 * i) = out;
-                }
-            if (write && lane == 0) { mu[m0 + row] = mean; rstd[m0 + row] = rs; }
+            for (int e = 0; e < 8; ++e) y[e] = fmaf((v[j][e] - mean) * rs, g[e], b[e]);
+            const uint4 out = pack8(y);
+            prow[sub + 8 * j] = out;
+            if (write) *(reinterpret_cast<uint4*>(h + static_cast<size_t>(m0 + row) * d) + sub + 8 * j) = out;
         }
+        if (write && sub == 0) { mu[m0 + row] = mean; rstd[m0 + row] = rs; }
     }
 }
 
 // ---------------------------------------------------------------- column sums (bias gradients, dgamma / dbeta)
-// One unit: 16 columns, 8 row lanes; lane sums are added in lane order.  With xhat_of != nullptr it
-// returns sum(in * xhat) in out0 and sum(in) in out1 (xhat = (xhat_of - mu) * rstd), else sum(in) in out0.
-__device__ void colsum_unit(const uint16_t* in, size_t ld, int T, int col0, const uint16_t* xhat_of, const float* mu,
-                            const float* rstd, float* out0, float* out1, int accumulate, float* red)
+// One unit: 32 columns (4 pieces of 16 bytes) x 32 row lanes, eight rows of a lane in flight (256
+// rows are one trip to L2); the lanes' sums are added in lane order.  With xhat_of != nullptr it
+// returns sum(in * xhat) in out0 and sum(in) in out1 (xhat = (xhat_of - mu) * rstd), else sum(in) in
+// out0.  red: 2 x 32 x 32 floats.
+__device__ __noinline__ void colsum_unit(const uint16_t* in, size_t ld, int T, int col0, const uint16_t* xhat_of, const float* mu,
+                                         const float* rstd, float* out0, float* out1, int accumulate, float* red)
 {
-    const int tid = threadIdx.x, c = tid & 15, rl = tid >> 4;
-    float s0 = 0.f, s1 = 0.f;
-    if (xhat_of) {
-#pragma unroll 4
-        for (int row = rl; row < T; row += 8) {
-            const float g = ldcg_bf16(in + row * ld + col0 + c);
-            const float xh = (ldcg_bf16(xhat_of + row * ld + col0 + c) - __ldcg(mu + row)) * __ldcg(rstd + row);
-            s0 = fmaf(g, xh, s0);
-            s1 += g;
+    const int tid = threadIdx.x, g = tid & 3, rl = tid >> 2;
+    float s0[8], s1[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { s0[e] = 0.f; s1[e] = 0.f; }
+    for (int r0 = rl; r0 < T; r0 += 32 * 8) {
+        uint4 a[8], b[8];
+        float m[8], rs[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int row = r0 + 32 * i;
+            if (row < T) {
+                a[i] = __ldcg(reinterpret_cast<const uint4*>(in + row * ld + col0) + g);
+                if (xhat_of) {
+                    b[i] = __ldcg(reinterpret_cast<const uint4*>(xhat_of + row * ld + col0) + g);
+                    m[i] = __ldcg(mu + row);
+                    rs[i] = __ldcg(rstd + row);
+                }
+            }
         }
-    } else {
-#pragma unroll 8
-        for (int row = rl; row < T; row += 8) s0 += ldcg_bf16(in + row * ld + col0 + c);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (r0 + 32 * i < T) {
+                float v[8];
+                unpack8(a[i], v);
+                if (xhat_of) {
+                    float xv[8];
+                    unpack8(b[i], xv);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) { s0[e] = fmaf(v[e], (xv[e] - m[i]) * rs[i], s0[e]); s1[e] += v[e]; }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) s0[e] += v[e];
+                }
+            }
+        }
     }
-    red[rl * 16 + c] = s0;
-    red[128 + rl * 16 + c] = s1;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { red[rl * 32 + g * 8 + e] = s0[e]; red[1024 + rl * 32 + g * 8 + e] = s1[e]; }
     __syncthreads();
-    if (tid < 16) {
+    if (tid < 32) {
         float a0 = 0.f, a1 = 0.f;
 #pragma unroll
-        for (int l = 0; l < 8; ++l) { a0 += red[l * 16 + tid]; a1 += red[128 + l * 16 + tid]; }
+        for (int l = 0; l < 32; ++l) { a0 += red[l * 32 + tid]; a1 += red[1024 + l * 32 + tid]; }
         out0[col0 + tid] = accumulate ? out0[col0 + tid] + a0 : a0;
         if (xhat_of) out1[col0 + tid] = accumulate ? out1[col0 + tid] + a1 : a1;
     }
@@ -362,28 +385,38 @@ __device__ void colsum_unit(const uint16_t* in, size_t ld, int T, int col0, cons
 
 // ---------------------------------------------------------------- LayerNorm backward, one row per warp
 // dx = resid + rstd * (g - mean(g) - xhat * mean(g * xhat)),  g = dh * gamma
-__device__ void ln_bwd_row(const uint16_t* dh, const uint16_t* x, const float* mu, const float* rstd, const uint16_t* gamma,
-                           const uint16_t* resid, uint16_t* dx, int d, int row)
+template <int NP>
+__device__ __forceinline__ void ln_bwd_row(const uint16_t* dh, const uint16_t* x, const float* mu, const float* rstd,
+                                           const uint16_t* gamma, const uint16_t* resid, uint16_t* dx, int row)
 {
-    const int lane = threadIdx.x & 31, np = d >> 8;
-    const float m = __ldcg(mu + row), rs = __ldcg(rstd + row), inv_d = 1.0f / d;
-    float g[2][8], xh[2][8];
+    constexpr int d = 256 * NP;
+    const int lane = threadIdx.x & 31;
+    const float inv_d = 1.0f / d;
+    uint4 qa[NP], qb[NP], qc[NP], qr[NP];
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+        qa[i] = __ldcg(reinterpret_cast<const uint4*>(dh + static_cast<size_t>(row) * d) + lane + 32 * i);
+        qb[i] = __ldcg(reinterpret_cast<const uint4*>(x + static_cast<size_t>(row) * d) + lane + 32 * i);
+        qr[i] = __ldcg(reinterpret_cast<const uint4*>(resid + static_cast<size_t>(row) * d) + lane + 32 * i);
+        qc[i] = __ldg(reinterpret_cast<const uint4*>(gamma) + lane + 32 * i);
+    }
+    const float m = __ldcg(mu + row), rs = __ldcg(rstd + row);
+    float g[NP][8], xh[NP][8];
     float s1 = 0.f, s2 = 0.f;
 #pragma unroll
-    for (int i = 0; i < 2; ++i)
-        if (i < np) {
-            float a[8], b[8], c[8];
-            unpack8(__ldcg(reinterpret_cast<const uint4*>(dh + static_cast<size_t>(row) * d) + lane + 32 * i), a);
-            unpack8(__ldcg(reinterpret_cast<const uint4*>(x + static_cast<size_t>(row) * d) + lane + 32 * i), b);
-            unpack8(__ldg(reinterpret_cast<const uint4*>(gamma) + lane + 32 * i), c);
+    for (int i = 0; i < NP; ++i) {
+        float a[8], b[8], c[8];
+        unpack8(qa[i], a);
+        unpack8(qb[i], b);
+        unpack8(qc[i], c);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                g[i][e] = a[e] * c[e];
-                xh[i][e] = (b[e] - m) * rs;
-                s1 += g[i][e];
-                s2 = fmaf(g[i][e], xh[i][e], s2);
-            }
+        for (int e = 0; e < 8; ++e) {
+            g[i][e] = a[e] * c[e];
+            xh[i][e] = (b[e] - m) * rs;
+            s1 += g[i][e];
+            s2 = fmaf(g[i][e], xh[i][e], s2);
         }
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         s1 += __shfl_xor_sync(0xffffffffu, s1, o);
@@ -391,14 +424,13 @@ __device__ void ln_bwd_row(const uint16_t* dh, const uint16_t* x, const float* m
     }
     s1 *= inv_d; s2 *= inv_d;
 #pragma unroll
-    for (int i = 0; i < 2; ++i)
-        if (i < np) {
-            float r[8], y[8];
-            unpack8(__ldcg(reinterpret_cast<const uint4*>(resid + static_cast<size_t>(row) * d) + lane + 32 * i), r);
+    for (int i = 0; i < NP; ++i) {
+        float r[8], y[8];
+        unpack8(qr[i], r);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) y[e] = r[e] + rs * (g[i][e] - s1 - xh[i][e] * s2);
-            *(reinterpret_cast<uint4*>(dx + static_cast<size_t>(row) * d) + lane + 32 * i) = pack8(y);
-        }
+        for (int e = 0; e < 8; ++e) y[e] = r[e] + rs * (g[i][e] - s1 - xh[i][e] * s2);
+        *(reinterpret_cast<uint4*>(dx + static_cast<size_t>(row) * d) + lane + 32 * i) = pack8(y);
+    }
 }
 
 // ---------------------------------------------------------------- attention units (head_dim 64)
@@ -418,15 +450,20 @@ __device__ __forceinline__ float delta_row(const uint16_t* dout, const uint16_t*
 }
 
 // Forward: 64 query rows of one head; warp w owns rows 16 w .. 16 w + 15, scores and P stay in registers.
-__device__ void attn_fwd_unit(const WholeLayerArgs& p, int b, int h, int qb, uint32_t sm)
+__device__ __noinline__ void attn_fwd_unit(const WholeLayerArgs& p, int b, int h, int qb, uint32_t sm)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const size_t ld = 3 * static_cast<size_t>(p.d);
     const uint16_t* qkv = static_cast<const uint16_t*>(p.qkv);
     const uint16_t* base = qkv + static_cast<size_t>(b) * p.S * ld + h * 64;
-    const uint32_t sQ = sm, sK = sm + 2 * kChunk, sV = sm + 3 * kChunk;
+    const uint32_t sQ = sm;                                 // K / V of block j in chunks 1 + 2 (j & 1), 2 + 2 (j & 1)
     const float sl2 = p.scale * 1.4426950408889634f;
+    auto load_kv = [&](int j) {
+        stage_chunk(sm + (1 + 2 * (j & 1)) * kChunk, base + static_cast<size_t>(j) * 64 * ld + p.d, ld, tid);
+        stage_chunk(sm + (2 + 2 * (j & 1)) * kChunk, base + static_cast<size_t>(j) * 64 * ld + 2 * p.d, ld, tid);
+    };
     stage_chunk(sQ, base + static_cast<size_t>(qb) * 64 * ld, ld, tid);
+    load_kv(0);
     cp_async_commit();
     uint32_t qf[4][4];
     float oacc[8][4];
@@ -436,11 +473,11 @@ __device__ void attn_fwd_unit(const WholeLayerArgs& p, int b, int h, int qb, uin
         for (int e = 0; e < 4; ++e) oacc[i][e] = 0.f;
     float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
     for (int j = 0; j <= qb; ++j) {
-        stage_chunk(sK, base + static_cast<size_t>(j) * 64 * ld + p.d, ld, tid);
-        stage_chunk(sV, base + static_cast<size_t>(j) * 64 * ld + 2 * p.d, ld, tid);
+        if (j < qb) load_kv(j + 1);                         // the next block travels while this one is used
         cp_async_commit();
-        cp_async_wait<0>();
+        cp_async_wait<1>();
         __syncthreads();
+        const uint32_t sK = sm + (1 + 2 * (j & 1)) * kChunk, sV = sK + kChunk;
         if (j == 0) {
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) frag_a_k(sQ, warp * 16, kk, lane, qf[kk]);
@@ -523,18 +560,23 @@ __device__ void attn_fwd_unit(const WholeLayerArgs& p, int b, int h, int qb, uin
 
 // Backward, dQ of 64 query rows of one head: per key block S and dP are rebuilt, dS = P (dP - delta)
 // goes straight from the accumulator registers into the A operand of dQ += dS K.
-__device__ void attn_dq_unit(const WholeLayerArgs& p, int b, int h, int qb, uint32_t sm, float* vec)
+__device__ __noinline__ void attn_dq_unit(const WholeLayerArgs& p, int b, int h, int qb, uint32_t sm, float* vec)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const size_t ld = 3 * static_cast<size_t>(p.d);
     const uint16_t* base = static_cast<const uint16_t*>(p.qkv) + static_cast<size_t>(b) * p.S * ld + h * 64;
     const uint16_t* dout = static_cast<const uint16_t*>(p.td0);
     const uint16_t* o = static_cast<const uint16_t*>(p.o);
-    const uint32_t sQ = sm, sDO = sm + kChunk, sK = sm + 2 * kChunk, sV = sm + 3 * kChunk;
+    const uint32_t sQ = sm, sDO = sm + kChunk;              // K / V of block j in chunks 2 + 2 (j & 1), 3 + 2 (j & 1)
     const float sl2 = p.scale * 1.4426950408889634f;
     const size_t row0 = static_cast<size_t>(b) * p.S + qb * 64;
+    auto load_kv = [&](int j) {
+        stage_chunk(sm + (2 + 2 * (j & 1)) * kChunk, base + static_cast<size_t>(j) * 64 * ld + p.d, ld, tid);
+        stage_chunk(sm + (3 + 2 * (j & 1)) * kChunk, base + static_cast<size_t>(j) * 64 * ld + 2 * p.d, ld, tid);
+    };
     stage_chunk(sQ, base + static_cast<size_t>(qb) * 64 * ld, ld, tid);
     stage_chunk(sDO, dout + row0 * p.d + h * 64, p.d, tid);
+    load_kv(0);
     cp_async_commit();
     if (tid < 64) vec[tid] = delta_row(dout, o, (row0 + tid) * p.d + h * 64);
     float lse2[2], dlt[2];
@@ -545,11 +587,11 @@ __device__ void attn_dq_unit(const WholeLayerArgs& p, int b, int h, int qb, uint
 #pragma unroll
         for (int e = 0; e < 4; ++e) dq[i][e] = 0.f;
     for (int j = 0; j <= qb; ++j) {
-        stage_chunk(sK, base + static_cast<size_t>(j) * 64 * ld + p.d, ld, tid);
-        stage_chunk(sV, base + static_cast<size_t>(j) * 64 * ld + 2 * p.d, ld, tid);
+        if (j < qb) load_kv(j + 1);
         cp_async_commit();
-        cp_async_wait<0>();
+        cp_async_wait<1>();
         __syncthreads();
+        const uint32_t sK = sm + (2 + 2 * (j & 1)) * kChunk, sV = sK + kChunk;
         if (j == 0) {
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
@@ -617,20 +659,25 @@ __device__ void attn_dq_unit(const WholeLayerArgs& p, int b, int h, int qb, uint
 
 // Backward, dK and dV of 64 key rows of one head: per query block the transposed scores K Q^T and
 // V dO^T are built, so that P^T and dS^T come out of the accumulators as A operands.
-__device__ void attn_dkdv_unit(const WholeLayerArgs& p, int b, int h, int kb, uint32_t sm, float* vec)
+__device__ __noinline__ void attn_dkdv_unit(const WholeLayerArgs& p, int b, int h, int kb, uint32_t sm, float* vec)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const size_t ld = 3 * static_cast<size_t>(p.d);
     const uint16_t* base = static_cast<const uint16_t*>(p.qkv) + static_cast<size_t>(b) * p.S * ld + h * 64;
     const uint16_t* dout = static_cast<const uint16_t*>(p.td0);
     const uint16_t* o = static_cast<const uint16_t*>(p.o);
-    const uint32_t sK = sm, sV = sm + kChunk, sQ = sm + 2 * kChunk, sDO = sm + 3 * kChunk;
+    const uint32_t sK = sm, sV = sm + kChunk;               // Q / dO of block i in chunks 2 + 2 (i & 1), 3 + 2 (i & 1)
     const float sl2 = p.scale * 1.4426950408889634f;
     const size_t seq0 = static_cast<size_t>(b) * p.S;
     float* v_lse = vec;                                     // [S] lse * log2(e)
     float* v_dlt = vec + kMaxS;                             // [S]
+    auto load_q = [&](int i) {
+        stage_chunk(sm + (2 + 2 * (i & 1)) * kChunk, base + static_cast<size_t>(i) * 64 * ld, ld, tid);
+        stage_chunk(sm + (3 + 2 * (i & 1)) * kChunk, dout + (seq0 + i * 64) * p.d + h * 64, p.d, tid);
+    };
     stage_chunk(sK, base + static_cast<size_t>(kb) * 64 * ld + p.d, ld, tid);
     stage_chunk(sV, base + static_cast<size_t>(kb) * 64 * ld + 2 * p.d, ld, tid);
+    load_q(kb);
     cp_async_commit();
     for (int r = kb * 64 + tid; r < p.S; r += kThreads) {
         v_lse[r] = __ldcg(static_cast<const float*>(p.lse) + (static_cast<size_t>(b) * p.H + h) * p.S + r) * 1.4426950408889634f;
@@ -644,11 +691,11 @@ __device__ void attn_dkdv_unit(const WholeLayerArgs& p, int b, int h, int kb, ui
         for (int e = 0; e < 4; ++e) { dk[i][e] = 0.f; dv[i][e] = 0.f; }
     const int nqb = p.S >> 6;
     for (int i = kb; i < nqb; ++i) {
-        stage_chunk(sQ, base + static_cast<size_t>(i) * 64 * ld, ld, tid);
-        stage_chunk(sDO, dout + (seq0 + i * 64) * p.d + h * 64, p.d, tid);
+        if (i + 1 < nqb) load_q(i + 1);
         cp_async_commit();
-        cp_async_wait<0>();
+        cp_async_wait<1>();
         __syncthreads();
+        const uint32_t sQ = sm + (2 + 2 * (i & 1)) * kChunk, sDO = sQ + kChunk;
         if (i == kb) {
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
@@ -729,77 +776,148 @@ struct Ctx {
     float* ws;
 };
 
-// Forward GEMM tile with bias and one of: nothing, residual, GeLU (writes u and a).
+// The accumulators leave the registers through a 64 x 64 fp32 tile in shared memory; the epilogue is
+// then a rolled loop over 16-byte pieces of the output (8 columns of a row per thread and turn), short
+// enough to stay in the instruction cache and storing whole 16-byte pieces.
+__device__ __forceinline__ void acc_to_smem(const float (&acc)[2][4][4], float* tile)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int r = (warp & 1) * 32 + (lane >> 2), c = (warp >> 1) * 32 + 2 * (lane & 3);
+#pragma unroll
+    for (int mi = 0; mi < 2; ++mi)
+#pragma unroll
+        for (int ni = 0; ni < 4; ++ni)
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+                *reinterpret_cast<float2*>(tile + (r + mi * 16 + h * 8) * kAccStride + c + ni * 8) =
+                    make_float2(acc[mi][ni][2 * h], acc[mi][ni][2 * h + 1]);
+    __syncthreads();
+}
+__device__ __forceinline__ void tile_piece(const float* tile, int row, int c8, float (&v)[8])
+{
+    const float4 a = *reinterpret_cast<const float4*>(tile + row * kAccStride + c8);
+    const float4 b = *reinterpret_cast<const float4*>(tile + row * kAccStride + c8 + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+
+// Forward GEMM tile with bias and one of: nothing, residual, GeLU (writes u and a).  The operand
+// chunks and the residual tile are requested first; LayerNorm (LN) runs while the weights travel.
 enum { kFwdBias = 0, kFwdResid = 1, kFwdGelu = 2 };
 template <bool LN>
-__device__ void fwd_gemm_unit(const Ctx& c, int u, int mode, const uint16_t* A, int K, const uint16_t* W, const uint16_t* bias,
-                              int N, int nslices, const uint16_t* resid, uint16_t* out, uint16_t* out_act,
-                              const uint16_t* ln_g, const uint16_t* ln_b, uint16_t* ln_h, float* ln_mu, float* ln_rs)
+__device__ __noinline__ void fwd_gemm_unit(const Ctx& c, int u, int mode, const uint16_t* A, int K, const uint16_t* W,
+                                           const uint16_t* bias, int N, int nslices, const uint16_t* resid, uint16_t* out,
+                                           uint16_t* out_act, const uint16_t* ln_g, const uint16_t* ln_b, uint16_t* ln_h,
+                                           float* ln_mu, float* ln_rs)
 {
     const WholeLayerArgs& p = c.p;
     const int tile = u / nslices, slice = u % nslices, ntn = N >> 6, tm = tile / ntn, tn = tile % ntn;
-    const int m0 = tm * 64, n0 = tn * 64, kper = K / nslices;
+    const int m0 = tm * 64, n0 = tn * 64, kper = K / nslices, tid = threadIdx.x;
     float acc[2][4][4];
+    const TileGemm<false, false, LN> g{A, static_cast<size_t>(K), W, static_cast<size_t>(K), m0, n0, LN ? 0 : slice * kper,
+                                       (LN ? K : kper) >> 6, c.sm + kSmStage};
     const int stride = (p.d + 8) * 2;
     if (LN) {
-        ln_rows_to_panel(A, ln_g, ln_b, p.d, p.eps, m0, c.smem + kSmPanel, stride, tn == 0, ln_h, ln_mu, ln_rs);
-        gemm_tile<false, false, true>(acc, nullptr, 0, W, K, m0, n0, 0, K, c.sm + kSmStage, c.sm + kSmPanel, stride);
+        ln_stage_rows(A, p.d, m0, c.sm + kSmPanel, stride);
+        cp_async_commit();
+    }
+    if (mode == kFwdResid) stage_chunk(c.sm + kSmAux, resid + static_cast<size_t>(m0) * N + n0, N, tid);   // rides with the first chunk
+    g.prefetch();
+    if (LN) {
+        cp_async_wait<kStages - 1>();                       // the rows of x have landed (the weight chunks may not have)
+        __syncthreads();
+        if (p.d == 256) ln_rows_in_panel<1>(ln_g, ln_b, p.eps, m0, c.smem + kSmPanel, stride, tn == 0, ln_h, ln_mu, ln_rs);
+        else ln_rows_in_panel<2>(ln_g, ln_b, p.eps, m0, c.smem + kSmPanel, stride, tn == 0, ln_h, ln_mu, ln_rs);
+        g.run(acc, c.sm + kSmPanel, stride);
     } else {
-        gemm_tile<false, false, false>(acc, A, K, W, K, m0, n0, slice * kper, (slice + 1) * kper, c.sm + kSmStage, 0, 0);
+        g.run(acc, 0, 0);
         if (!splitk_combine(acc, c.ws, c.sem, tile, slice, nslices, c.flag)) return;
     }
-    const int act = p.act;
-    for_each_pair(acc, m0, n0, [&](int row, int col, float v0, float v1) {
-        const uint32_t bb = __ldg(reinterpret_cast<const uint32_t*>(bias + col));
-        v0 += bf16_lo(bb); v1 += bf16_hi(bb);
-        const size_t idx = static_cast<size_t>(row) * N + col;
+    float* tl = reinterpret_cast<float*>(c.smem + kSmAcc);
+    acc_to_smem(acc, tl);
+    const int act = p.act, c8 = (tid & 7) * 8;
+    float bv[8];
+    unpack8(__ldg(reinterpret_cast<const uint4*>(bias + n0 + c8)), bv);
+#pragma unroll 1
+    for (int it = 0; it < 4; ++it) {
+        const int row = (tid >> 3) + it * 16;
+        float v[8];
+        tile_piece(tl, row, c8, v);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] += bv[e];
         if (mode == kFwdResid) {
-            float r0, r1;
-            load_bf16x2(resid, idx, r0, r1);
-            v0 += r0; v1 += r1;
+            float r[8];
+            unpack8(*reinterpret_cast<const uint4*>(c.smem + kSmAux + swz(row, tid & 7)), r);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[e] += r[e];
         }
-        store_bf16x2(out, idx, v0, v1);
+        const size_t idx = static_cast<size_t>(m0 + row) * N + n0 + c8;
+        *reinterpret_cast<uint4*>(out + idx) = pack8(v);
         if (mode == kFwdGelu) {
-            gelu2(v0, v1, act);
-            store_bf16x2(out_act, idx, v0, v1);
+#pragma unroll
+            for (int e = 0; e < 8; e += 2) gelu2(v[e], v[e + 1], act);
+            *reinterpret_cast<uint4*>(out_act + idx) = pack8(v);
         }
-    });
+    }
+    __syncthreads();                                        // the accumulator tile and the aux chunk may be rewritten
 }
 
 // Data-gradient tile: out[T, N] = A[T, K] W[K, N] (W stored [K][N]); with u != nullptr the result is
 // multiplied by GeLU'(u).
-__device__ void dgrad_unit(const Ctx& c, int u, const uint16_t* A, int K, const uint16_t* W, int N, int nslices,
-                           const uint16_t* gelu_u, uint16_t* out)
+__device__ __noinline__ void dgrad_unit(const Ctx& c, int u, const uint16_t* A, int K, const uint16_t* W, int N, int nslices,
+                                        const uint16_t* gelu_u, uint16_t* out)
 {
     const int tile = u / nslices, slice = u % nslices, ntn = N >> 6, m0 = (tile / ntn) * 64, n0 = (tile % ntn) * 64;
-    const int kper = K / nslices;
+    const int kper = K / nslices, tid = threadIdx.x;
     float acc[2][4][4];
-    gemm_tile<false, true, false>(acc, A, K, W, N, m0, n0, slice * kper, (slice + 1) * kper, c.sm + kSmStage, 0, 0);
+    const TileGemm<false, true, false> g{A, static_cast<size_t>(K), W, static_cast<size_t>(N), m0, n0, slice * kper, kper >> 6,
+                                         c.sm + kSmStage};
+    if (gelu_u) stage_chunk(c.sm + kSmAux, gelu_u + static_cast<size_t>(m0) * N + n0, N, tid);
+    g.prefetch();
+    g.run(acc, 0, 0);
     if (!splitk_combine(acc, c.ws, c.sem, tile, slice, nslices, c.flag)) return;
-    const int act = c.p.act;
-    for_each_pair(acc, m0, n0, [&](int row, int col, float v0, float v1) {
-        const size_t idx = static_cast<size_t>(row) * N + col;
+    float* tl = reinterpret_cast<float*>(c.smem + kSmAcc);
+    acc_to_smem(acc, tl);
+    const int act = c.p.act, c8 = (tid & 7) * 8;
+#pragma unroll 1
+    for (int it = 0; it < 4; ++it) {
+        const int row = (tid >> 3) + it * 16;
+        float v[8];
+        tile_piece(tl, row, c8, v);
         if (gelu_u) {
-            float u0, u1;
-            load_bf16x2(gelu_u, idx, u0, u1);
-            gelu_grad_mul2(v0, v1, u0, u1, act);
+            float uv[8];
+            unpack8(*reinterpret_cast<const uint4*>(c.smem + kSmAux + swz(row, tid & 7)), uv);
+#pragma unroll
+            for (int e = 0; e < 8; e += 2) gelu_grad_mul2(v[e], v[e + 1], uv[e], uv[e + 1], act);
         }
-        store_bf16x2(out, idx, v0, v1);
-    });
+        *reinterpret_cast<uint4*>(out + static_cast<size_t>(m0 + row) * N + n0 + c8) = pack8(v);
+    }
+    __syncthreads();
 }
 
 // Weight-gradient tile: dW[M, N] (+)= A[T, M]^T B[T, N], fp32.
-__device__ void wgrad_unit(const Ctx& c, int u, const uint16_t* A, int M, const uint16_t* B, int N, float* dW)
+__device__ __noinline__ void wgrad_unit(const Ctx& c, int u, const uint16_t* A, int M, const uint16_t* B, int N, float* dW)
 {
-    const int ntn = N >> 6, m0 = (u / ntn) * 64, n0 = (u % ntn) * 64;
+    const int ntn = N >> 6, m0 = (u / ntn) * 64, n0 = (u % ntn) * 64, tid = threadIdx.x;
     float acc[2][4][4];
-    gemm_tile<true, true, false>(acc, A, M, B, N, m0, n0, 0, c.p.T, c.sm + kSmStage, 0, 0);
-    const int accumulate = c.p.accumulate;
-    for_each_pair(acc, m0, n0, [&](int row, int col, float v0, float v1) {
-        float2* dst = reinterpret_cast<float2*>(dW + static_cast<size_t>(row) * N + col);
-        if (accumulate) { const float2 old = *dst; v0 += old.x; v1 += old.y; }
-        *dst = make_float2(v0, v1);
-    });
+    const TileGemm<true, true, false> g{A, static_cast<size_t>(M), B, static_cast<size_t>(N), m0, n0, 0, c.p.T >> 6, c.sm + kSmStage};
+    g.prefetch();
+    float4 old[8];
+    const int c4 = (tid & 15) * 4;
+    if (c.p.accumulate) {
+#pragma unroll
+        for (int it = 0; it < 8; ++it) old[it] = *reinterpret_cast<const float4*>(dW + static_cast<size_t>(m0 + (tid >> 4) + it * 8) * N + n0 + c4);
+    }
+    g.run(acc, 0, 0);
+    float* tl = reinterpret_cast<float*>(c.smem + kSmAcc);
+    acc_to_smem(acc, tl);
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+        const int row = (tid >> 4) + it * 8;
+        float4 v = *reinterpret_cast<const float4*>(tl + row * kAccStride + c4);
+        if (c.p.accumulate) { v.x += old[it].x; v.y += old[it].y; v.z += old[it].z; v.w += old[it].w; }
+        *reinterpret_cast<float4*>(dW + static_cast<size_t>(m0 + row) * N + n0 + c4) = v;
+    }
+    __syncthreads();
 }
 
 __device__ __forceinline__ const uint16_t* cu16(const void* q) { return static_cast<const uint16_t*>(q); }
@@ -849,45 +967,48 @@ __global__ void __launch_bounds__(kThreads, 1) whole_layer_bwd_kernel(const __gr
     const Ctx c{p, smem, smem_u32(smem), reinterpret_cast<int*>(smem + kSmFlag), p.sync + 2, f32(p.splitk)};
     if (*reinterpret_cast<volatile int*>(&p.status->code) != 0) return;
     const int T = p.T, d = p.d, F = p.F, G = gridDim.x, tm = T >> 6, warp = threadIdx.x >> 5;
-    float* red = reinterpret_cast<float*>(smem + kSmRed);
+    float* red = reinterpret_cast<float*>(smem + kSmPanel);
     float* vec = reinterpret_cast<float*>(smem + kSmVec);
     const int acc = p.accumulate;
     // 1: du = (dy W2) * GeLU'(u);  dW2 = dy^T a;  db2 = colsum(dy)
     {
-        const int n0 = tm * (F >> 6), n1 = n0 + (d >> 6) * (F >> 6), n2 = n1 + (d >> 4);
+        const int n0 = tm * (F >> 6), n1 = n0 + (d >> 6) * (F >> 6), n2 = n1 + (d >> 5);
         for (int u = blockIdx.x; u < n2; u += G) {
             if (u < n0) dgrad_unit(c, u, cu16(p.dy), d, cu16(p.w_fc2), F, 1, cu16(p.u), u16(p.big));
             else if (u < n1) wgrad_unit(c, u - n0, cu16(p.dy), d, cu16(p.a), F, f32(p.g_w_fc2));
-            else colsum_unit(cu16(p.dy), d, T, (u - n1) * 16, nullptr, nullptr, nullptr, f32(p.g_b_fc2), nullptr, acc, red);
+            else colsum_unit(cu16(p.dy), d, T, (u - n1) * 32, nullptr, nullptr, nullptr, f32(p.g_b_fc2), nullptr, acc, red);
         }
     }
     if (!grid_barrier(p.sync, p.status, c.flag)) return;
     // 2: dh2 = du W1;  dW1 = du^T h2;  db1 = colsum(du)
     {
-        const int n0 = tm * (d >> 6) * p.split_f, n1 = n0 + (F >> 6) * (d >> 6), n2 = n1 + (F >> 4);
+        const int n0 = tm * (d >> 6) * p.split_f, n1 = n0 + (F >> 6) * (d >> 6), n2 = n1 + (F >> 5);
         for (int u = blockIdx.x; u < n2; u += G) {
             if (u < n0) dgrad_unit(c, u, cu16(p.big), F, cu16(p.w_fc1), d, p.split_f, nullptr, u16(p.td0));
             else if (u < n1) wgrad_unit(c, u - n0, cu16(p.big), F, cu16(p.h2), d, f32(p.g_w_fc1));
-            else colsum_unit(cu16(p.big), F, T, (u - n1) * 16, nullptr, nullptr, nullptr, f32(p.g_b_fc1), nullptr, acc, red);
+            else colsum_unit(cu16(p.big), F, T, (u - n1) * 32, nullptr, nullptr, nullptr, f32(p.g_b_fc1), nullptr, acc, red);
         }
     }
     if (!grid_barrier(p.sync, p.status, c.flag)) return;
     // 3: dx1 = dy + LN2bwd(dh2);  dgamma2, dbeta2
     {
-        const int n0 = T >> 2, n1 = n0 + (d >> 4);
+        const int n0 = T >> 2, n1 = n0 + (d >> 5);
         for (int u = blockIdx.x; u < n1; u += G) {
-            if (u < n0) ln_bwd_row(cu16(p.td0), cu16(p.x1), f32(p.mu2), f32(p.r2), cu16(p.ln2_g), cu16(p.dy), u16(p.dx1), d, u * 4 + warp);
-            else colsum_unit(cu16(p.td0), d, T, (u - n0) * 16, cu16(p.x1), f32(p.mu2), f32(p.r2), f32(p.g_ln2_g), f32(p.g_ln2_b), acc, red);
+            if (u < n0) {
+                if (d == 256) ln_bwd_row<1>(cu16(p.td0), cu16(p.x1), f32(p.mu2), f32(p.r2), cu16(p.ln2_g), cu16(p.dy), u16(p.dx1), u * 4 + warp);
+                else ln_bwd_row<2>(cu16(p.td0), cu16(p.x1), f32(p.mu2), f32(p.r2), cu16(p.ln2_g), cu16(p.dy), u16(p.dx1), u * 4 + warp);
+            }
+            else colsum_unit(cu16(p.td0), d, T, (u - n0) * 32, cu16(p.x1), f32(p.mu2), f32(p.r2), f32(p.g_ln2_g), f32(p.g_ln2_b), acc, red);
         }
     }
     if (!grid_barrier(p.sync, p.status, c.flag)) return;
     // 4: dout = dx1 Wo;  dWo = dx1^T o;  dbo = colsum(dx1)
     {
-        const int n0 = tm * (d >> 6) * p.split_d, n1 = n0 + (d >> 6) * (d >> 6), n2 = n1 + (d >> 4);
+        const int n0 = tm * (d >> 6) * p.split_d, n1 = n0 + (d >> 6) * (d >> 6), n2 = n1 + (d >> 5);
         for (int u = blockIdx.x; u < n2; u += G) {
             if (u < n0) dgrad_unit(c, u, cu16(p.dx1), d, cu16(p.w_o), d, p.split_d, nullptr, u16(p.td0));
             else if (u < n1) wgrad_unit(c, u - n0, cu16(p.dx1), d, cu16(p.o), d, f32(p.g_w_o));
-            else colsum_unit(cu16(p.dx1), d, T, (u - n1) * 16, nullptr, nullptr, nullptr, f32(p.g_b_o), nullptr, acc, red);
+            else colsum_unit(cu16(p.dx1), d, T, (u - n1) * 32, nullptr, nullptr, nullptr, f32(p.g_b_o), nullptr, acc, red);
         }
     }
     if (!grid_barrier(p.sync, p.status, c.flag)) return;
@@ -904,20 +1025,23 @@ __global__ void __launch_bounds__(kThreads, 1) whole_layer_bwd_kernel(const __gr
     if (!grid_barrier(p.sync, p.status, c.flag)) return;
     // 6: dh1 = dqkv Wqkv;  dWqkv = dqkv^T h1;  dbqkv = colsum(dqkv)
     {
-        const int n0 = tm * (d >> 6) * p.split_3d, n1 = n0 + (3 * d >> 6) * (d >> 6), n2 = n1 + (3 * d >> 4);
+        const int n0 = tm * (d >> 6) * p.split_3d, n1 = n0 + (3 * d >> 6) * (d >> 6), n2 = n1 + (3 * d >> 5);
         for (int u = blockIdx.x; u < n2; u += G) {
             if (u < n0) dgrad_unit(c, u, cu16(p.big), 3 * d, cu16(p.w_qkv), d, p.split_3d, nullptr, u16(p.td0));
             else if (u < n1) wgrad_unit(c, u - n0, cu16(p.big), 3 * d, cu16(p.h1), d, f32(p.g_w_qkv));
-            else colsum_unit(cu16(p.big), 3 * d, T, (u - n1) * 16, nullptr, nullptr, nullptr, f32(p.g_b_qkv), nullptr, acc, red);
+            else colsum_unit(cu16(p.big), 3 * d, T, (u - n1) * 32, nullptr, nullptr, nullptr, f32(p.g_b_qkv), nullptr, acc, red);
         }
     }
     if (!grid_barrier(p.sync, p.status, c.flag)) return;
     // 7: dx = dx1 + LN1bwd(dh1);  dgamma1, dbeta1
     {
-        const int n0 = T >> 2, n1 = n0 + (d >> 4);
+        const int n0 = T >> 2, n1 = n0 + (d >> 5);
         for (int u = blockIdx.x; u < n1; u += G) {
-            if (u < n0) ln_bwd_row(cu16(p.td0), cu16(p.x), f32(p.mu1), f32(p.r1), cu16(p.ln1_g), cu16(p.dx1), u16(p.dx), d, u * 4 + warp);
-            else colsum_unit(cu16(p.td0), d, T, (u - n0) * 16, cu16(p.x), f32(p.mu1), f32(p.r1), f32(p.g_ln1_g), f32(p.g_ln1_b), acc, red);
+            if (u < n0) {
+                if (d == 256) ln_bwd_row<1>(cu16(p.td0), cu16(p.x), f32(p.mu1), f32(p.r1), cu16(p.ln1_g), cu16(p.dx1), u16(p.dx), u * 4 + warp);
+                else ln_bwd_row<2>(cu16(p.td0), cu16(p.x), f32(p.mu1), f32(p.r1), cu16(p.ln1_g), cu16(p.dx1), u16(p.dx), u * 4 + warp);
+            }
+            else colsum_unit(cu16(p.td0), d, T, (u - n0) * 32, cu16(p.x), f32(p.mu1), f32(p.r1), f32(p.g_ln1_g), f32(p.g_ln1_b), acc, red);
         }
     }
 }
@@ -956,12 +1080,15 @@ const char* whole_layer_unsupported(int T, int d, int H, int dh, int F, int S)
     return nullptr;
 }
 
-// Slices of the K range of a GEMM with `tiles` output tiles: as many as keep every slice at least
-// two 64-wide blocks long, divide the block count, and do not push the phase beyond one round of CTAs.
+// Slices of the K range of a GEMM with `tiles` output tiles.  Meeting the other slices costs three
+// trips to L2 (partial tile out, ticket, partial tiles back in), about as much as eight 64-wide
+// blocks of products, so only long K ranges are cut: into as many slices as keep every slice at
+// least two blocks long, divide the block count, and do not push the phase beyond one round of CTAs.
 static int pick_slices(int tiles, int K, int grid)
 {
     const int blocks = K / 64;
     int best = 1;
+    if (blocks < 12) return 1;
     for (int s = 2; s <= 8; ++s)
         if (blocks % s == 0 && blocks / s >= 2 && tiles * s <= grid) best = s;
     return best;

@@ -10,7 +10,9 @@ every layer call), ASYNC (enqueue everything) and GRAPH (one captured CUDA graph
     python -m paper_2203_12533_b200.dispatch_study [--layers 8] [--microbatches 8] [--reps 20]
 
 prints one JSON line per (sequence length, mode): layer calls per second and microseconds per
-call, for a chain of ``layers`` x ``microbatches`` x 2 calls at the width of workload 1.
+call, for a chain of ``layers`` x ``microbatches`` x 2 calls at the width of workload 1.  Where the
+shape allows it, each mode is also run with PW_FLAG_WHOLE_LAYER (a layer call is then one kernel
+launch instead of 7 or 19): the step the paper's Fused mode takes one level further down.
 """
 from __future__ import annotations
 
@@ -23,11 +25,14 @@ from . import binding as pw
 from . import inputs
 
 
-def run(seq_len: int, layers: int, microbatches: int, reps: int, mode: int) -> float:
+WHOLE_LAYER_MAX_SEQ = 1024
+
+
+def run(seq_len: int, layers: int, microbatches: int, reps: int, mode: int, flags: int = 0) -> float:
     """Milliseconds per chain (L x M forward calls + L x M backward calls)."""
     w = inputs.WORKLOADS[1].with_(seq_len=seq_len, n_layers=layers, n_microbatches=microbatches)
     dev = torch.device("cuda")
-    stage = pw.Stage(layers, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
+    stage = pw.Stage(layers, w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch, flags=flags)
     params = [[p.to(dev) for p in inputs.layer_params(w, 0, l)] for l in range(layers)]
     grads = [[torch.zeros(p.shape, dtype=torch.float32, device=dev) for p in ps] for ps in params]
     xs, dys = [], []
@@ -68,6 +73,9 @@ def study(seq_lens=(128, 256, 512, 1024, 2048), layers=8, microbatches=8, reps=2
         for name, mode in modes:
             row[f"us_per_layer_call_{name}"] = 1e3 * run(S, layers, microbatches, reps, mode) / calls
         row["graph_vs_opbyop"] = row["us_per_layer_call_opbyop"] / row["us_per_layer_call_graph"]
+        if S <= WHOLE_LAYER_MAX_SEQ:
+            for name, mode in modes:
+                row[f"us_per_layer_call_whole_layer_{name}"] = 1e3 * run(S, layers, microbatches, reps, mode, pw.FLAG_WHOLE_LAYER) / calls
         rows.append(row)
     return rows
 
@@ -82,11 +90,14 @@ def main():
     pw.lib()
     modes = (("opbyop", pw.DISPATCH_OPBYOP), ("async", pw.DISPATCH_ASYNC), ("graph", pw.DISPATCH_GRAPH))
     for S in args.seq_lens:
-        for name, mode in modes:
-            ms = run(S, args.layers, args.microbatches, args.reps, mode)
-            calls = 2 * args.layers * args.microbatches
-            print(json.dumps({"seq_len": S, "tokens_per_call": 2 * S, "mode": name, "ms_per_chain": ms,
-                              "us_per_layer_call": 1e3 * ms / calls, "layer_calls_per_s": calls / (ms * 1e-3)}), flush=True)
+        for flags in (0, pw.FLAG_WHOLE_LAYER):
+            if flags and S > WHOLE_LAYER_MAX_SEQ:
+                continue
+            for name, mode in modes:
+                ms = run(S, args.layers, args.microbatches, args.reps, mode, flags)
+                calls = 2 * args.layers * args.microbatches
+                print(json.dumps({"seq_len": S, "tokens_per_call": 2 * S, "mode": name, "whole_layer": bool(flags), "ms_per_chain": ms,
+                                  "us_per_layer_call": 1e3 * ms / calls, "layer_calls_per_s": calls / (ms * 1e-3)}), flush=True)
 
 
 if __name__ == "__main__":
