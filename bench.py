@@ -873,7 +873,8 @@ def dispatch_table():
     from paper_2203_12533_b200 import dispatch_study
     rows = dispatch_study.study(seq_lens=(128, 256, 512, 1024, 2048), layers=8, microbatches=8, reps=10)
     return {"what": "chain of 8 layers x 8 micro-batches at workload 1's width (recompute on): microseconds per layer call "
-                    "(forward or backward) in each dispatch mode of pw_stage_run_chain",
+                    "(forward or backward) in each dispatch mode of pw_stage_run_chain; the whole_layer columns are the same chain with "
+                    "PW_FLAG_WHOLE_LAYER (one cooperative launch per layer call), for the shapes that path serves",
             "rows": rows}
 
 

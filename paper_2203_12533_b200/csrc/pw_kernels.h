@@ -143,7 +143,7 @@ const char* launch_attention_bwd(Runtime* rt, const void* qkv, const void* o, co
 constexpr int kWholeLayerMaxTiles = 1024;           // (tokens / 64) * (d_model / 64): one split-K ticket each
 struct WholeLayerArgs {
     int T, d, H, F, B, S, act, accumulate, with_fc2;
-    int split_d, split_f, split_3d;                 // K slices of the GEMMs with [T, d] outputs (set by the launcher)
+    int split_o, split_fc2, split_dh2, split_dh1;   // K slices of the GEMMs with [T, d] outputs (set by the launcher)
     float eps, scale;
     const void *x, *dy;
     void *y, *dx;

@@ -4,7 +4,7 @@
 // Section 5.1 (Figures 5 and 6), where a computation is shorter than the cost of issuing it.
 //
 // The 7 forward / 19 backward steps of the layer become 5 / 7 phases of one persistent grid
-// (one 128-thread CTA per SM); a phase is a list of independent units (a 64 x 64 output tile of a
+// (one 256-thread CTA per SM); a phase is a list of independent units (a 64 x 64 output tile of a
 // GEMM, a slice of its K range, 64 query or key rows of one head, four LayerNorm rows, 16 columns of
 // a bias sum) that the CTAs take round-robin, and phases are separated by a bounded grid barrier.
 // Steps that do not depend on one another share a phase (a data-gradient GEMM, the weight-gradient
@@ -22,7 +22,7 @@
 namespace pw {
 namespace {
 
-constexpr int kThreads = 128;
+constexpr int kThreads = 256;                        // 8 warps
 constexpr int kChunk = 64 * 64 * 2;                 // one 64 x 64 bf16 operand chunk
 constexpr int kStages = 5;                            // four 64-wide K blocks in flight: K = 256 is one trip to L2
 constexpr int kMaxD = 512;                          // LayerNorm panel: 64 rows of the full width in shared memory
@@ -31,7 +31,7 @@ constexpr int kSmStage = 0;                         // kStages x (A chunk, B chu
 constexpr int kSmAux = kSmStage + kStages * 2 * kChunk;      // one chunk of an epilogue operand (residual, u)
 constexpr int kAccStride = 68;                               // floats per row of the accumulator tile (bank spread)
 constexpr int kSmAcc = kSmAux + kChunk;                      // 64 x 64 accumulators on their way to a rolled epilogue loop
-constexpr int kSmPanel = kSmAcc + 64 * kAccStride * 4;       // also the lanes of a column-sum unit (8 KB)
+constexpr int kSmPanel = kSmAcc + 64 * kAccStride * 4;       // also the lanes of a column-sum unit (16 KB) and the attention merges
 constexpr int kSmVec = kSmPanel + 64 * (kMaxD + 8) * 2;     // lse and delta of one (sequence, head)
 constexpr int kSmFlag = kSmVec + 2 * kMaxS * 4;
 constexpr int kSmBytes = kSmFlag + 16;
@@ -118,7 +118,7 @@ __device__ __forceinline__ uint32_t swz(int row, int piece) { return row * 128 +
 __device__ __forceinline__ void stage_chunk(uint32_t dst, const uint16_t* src, size_t ld, int tid)
 {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < 512 / kThreads; ++i) {
         const int q = tid + i * kThreads, row = q >> 3, piece = q & 7;
         cp_async16(dst + swz(row, piece), src + row * ld + piece * 8);
     }
@@ -145,8 +145,8 @@ __device__ __forceinline__ void frag_b_mn(uint32_t base, int n0, int kk, int lan
 // ---------------------------------------------------------------- 64 x 64 output tile, K range [k0, k0 + 64 nk)
 // C[m0.., n0..] = sum_k A(m, k) B(k, n).  A_MN: A is stored [K][M] (else [M][K]); B_MN: B is stored
 // [K][N] (else [N][K]); A_PANEL: the A rows are already in shared memory (LayerNorm output, full width).
-// Warp w owns rows 32 (w & 1) and columns 32 (w >> 1): acc[mi][ni][e] is row 16 mi + lane / 4 + 8 (e / 2),
-// column 8 ni + 2 (lane % 4) + e % 2 of that quarter.  prefetch() puts the first chunks in flight, so
+// Warp w owns rows 32 (w & 1) and columns 16 (w >> 1): acc[mi][ni][e] is row 16 mi + lane / 4 + 8 (e / 2),
+// column 8 ni + 2 (lane % 4) + e % 2 of that eighth.  prefetch() puts the first chunks in flight, so
 // that whatever the unit does before run() (LayerNorm of the A rows, loads of epilogue operands)
 // overlaps their way from L2.
 template <bool A_MN, bool B_MN, bool A_PANEL>
@@ -172,13 +172,13 @@ struct TileGemm {
             cp_async_commit();
         }
     }
-    __device__ __forceinline__ void run(float (&acc)[2][4][4], uint32_t panel, int panel_stride) const
+    __device__ __forceinline__ void run(float (&acc)[2][2][4], uint32_t panel, int panel_stride) const
     {
-        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wm = (warp & 1) * 32, wn = (warp >> 1) * 32;
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wm = (warp & 1) * 32, wn = (warp >> 1) * 16;
 #pragma unroll
         for (int i = 0; i < 2; ++i)
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
+            for (int j = 0; j < 2; ++j)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.f;
         for (int kc = 0; kc < nk; ++kc) {
@@ -189,7 +189,7 @@ struct TileGemm {
             const uint32_t sa = stage + (kc % kStages) * 2 * kChunk, sb = sa + kChunk;
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
-                uint32_t af[2][4], bf[2][4];
+                uint32_t af[2][4], bf[4];
 #pragma unroll
                 for (int mi = 0; mi < 2; ++mi) {
                     if (A_PANEL) {
@@ -201,16 +201,12 @@ struct TileGemm {
                         frag_a_k(sa, wm + mi * 16, kk, lane, af[mi]);
                     }
                 }
-#pragma unroll
-                for (int np = 0; np < 2; ++np) {
-                    if (B_MN) frag_b_mn(sb, wn + np * 16, kk, lane, bf[np]);
-                    else frag_b_k(sb, wn + np * 16, kk, lane, bf[np]);
-                }
+                if (B_MN) frag_b_mn(sb, wn, kk, lane, bf);
+                else frag_b_k(sb, wn, kk, lane, bf);
 #pragma unroll
                 for (int mi = 0; mi < 2; ++mi)
 #pragma unroll
-                    for (int ni = 0; ni < 4; ++ni)
-                        mma16816(acc[mi][ni], af[mi], bf[ni >> 1][(ni & 1) * 2], bf[ni >> 1][(ni & 1) * 2 + 1]);
+                    for (int ni = 0; ni < 2; ++ni) mma16816(acc[mi][ni], af[mi], bf[ni * 2], bf[ni * 2 + 1]);
             }
         }
         cp_async_wait<0>();
@@ -220,14 +216,14 @@ struct TileGemm {
 
 // Split-K: every slice stores its partial tile, the CTA that arrives last adds the slices in slice
 // order (its own included, from memory) and returns true: it then runs the epilogue.
-__device__ bool splitk_combine(float (&acc)[2][4][4], float* ws, unsigned* sem, int tile, int slice, int nslices, int* s_flag)
+__device__ bool splitk_combine(float (&acc)[2][2][4], float* ws, unsigned* sem, int tile, int slice, int nslices, int* s_flag)
 {
     if (nslices == 1) return true;
     const int tid = threadIdx.x;
     float* flat = &acc[0][0][0];
     float4* mine = reinterpret_cast<float4*>(ws + static_cast<size_t>(tile * nslices + slice) * 4096);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) __stcg(mine + i * kThreads + tid, make_float4(flat[4 * i], flat[4 * i + 1], flat[4 * i + 2], flat[4 * i + 3]));
+    for (int i = 0; i < 4; ++i) __stcg(mine + i * kThreads + tid, make_float4(flat[4 * i], flat[4 * i + 1], flat[4 * i + 2], flat[4 * i + 3]));
     __threadfence();
     __syncthreads();
     if (tid == 0) {
@@ -242,11 +238,11 @@ __device__ bool splitk_combine(float (&acc)[2][4][4], float* ws, unsigned* sem, 
     __syncthreads();                                        // everyone has read the flag before it is written again
     if (!last) return false;
 #pragma unroll
-    for (int i = 0; i < 32; ++i) flat[i] = 0.f;
+    for (int i = 0; i < 16; ++i) flat[i] = 0.f;
     for (int s = 0; s < nslices; ++s) {
         const float4* part = reinterpret_cast<const float4*>(ws + static_cast<size_t>(tile * nslices + s) * 4096);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < 4; ++i) {
             const float4 v = __ldcg(part + i * kThreads + tid);
             flat[4 * i] += v.x; flat[4 * i + 1] += v.y; flat[4 * i + 2] += v.z; flat[4 * i + 3] += v.w;
         }
@@ -262,7 +258,7 @@ __device__ __forceinline__ void store_bf16x2(uint16_t* base, size_t idx, float v
 // ---------------------------------------------------------------- LayerNorm of 64 rows in the panel
 // The 64 rows of x come into the panel by cp.async (ln_stage_rows, one commit group) and are normalised
 // in place by a short rolled loop - code that runs once per launch is paid for by instruction fetch,
-// not by arithmetic.  Warp w owns rows 16 w .. 16 w + 15, four at a time: eight lanes share a row (lane
+// not by arithmetic.  Warp w owns rows 8 w .. 8 w + 7, four at a time: eight lanes share a row (lane
 // % 8 owns the 16-byte pieces lane % 8 + 8 j), so a row sum is three shuffles.  Two-pass statistics
 // in fp32, like the stand-alone kernel; h = (x - mean) * rstd * gamma + beta replaces x as bf16 and,
 // from the CTA of column tile 0, goes to global memory with mean and rstd for the backward pass.
@@ -289,8 +285,8 @@ __device__ __forceinline__ void ln_rows_in_panel(const uint16_t* gamma, const ui
         bq[j] = __ldg(reinterpret_cast<const uint4*>(beta) + sub + 8 * j);
     }
 #pragma unroll 1
-    for (int it = 0; it < 4; ++it) {
-        const int row = warp * 16 + it * 4 + rsel;
+    for (int it = 0; it < 2; ++it) {
+        const int row = warp * 8 + it * 4 + rsel;
         uint4* prow = reinterpret_cast<uint4*>(panel + row * stride);
         float v[kPieces][8];
         float s = 0.f;
@@ -327,10 +323,10 @@ __device__ __forceinline__ void ln_rows_in_panel(const uint16_t* gamma, const ui
 }
 
 // ---------------------------------------------------------------- column sums (bias gradients, dgamma / dbeta)
-// One unit: 32 columns (4 pieces of 16 bytes) x 32 row lanes, eight rows of a lane in flight (256
+// One unit: 32 columns (4 pieces of 16 bytes) x 64 row lanes, eight rows of a lane in flight (512
 // rows are one trip to L2); the lanes' sums are added in lane order.  With xhat_of != nullptr it
 // returns sum(in * xhat) in out0 and sum(in) in out1 (xhat = (xhat_of - mu) * rstd), else sum(in) in
-// out0.  red: 2 x 32 x 32 floats.
+// out0.  red: 2 x 64 x 32 floats.
 __device__ __noinline__ void colsum_unit(const uint16_t* in, size_t ld, int T, int col0, const uint16_t* xhat_of, const float* mu,
                                          const float* rstd, float* out0, float* out1, int accumulate, float* red)
 {
@@ -338,12 +334,12 @@ __device__ __noinline__ void colsum_unit(const uint16_t* in, size_t ld, int T, i
     float s0[8], s1[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) { s0[e] = 0.f; s1[e] = 0.f; }
-    for (int r0 = rl; r0 < T; r0 += 32 * 8) {
+    for (int r0 = rl; r0 < T; r0 += 64 * 8) {
         uint4 a[8], b[8];
         float m[8], rs[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            const int row = r0 + 32 * i;
+            const int row = r0 + 64 * i;
             if (row < T) {
                 a[i] = __ldcg(reinterpret_cast<const uint4*>(in + row * ld + col0) + g);
                 if (xhat_of) {
@@ -355,7 +351,7 @@ __device__ __noinline__ void colsum_unit(const uint16_t* in, size_t ld, int T, i
         }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            if (r0 + 32 * i < T) {
+            if (r0 + 64 * i < T) {
                 float v[8];
                 unpack8(a[i], v);
                 if (xhat_of) {
@@ -371,12 +367,12 @@ __device__ __noinline__ void colsum_unit(const uint16_t* in, size_t ld, int T, i
         }
     }
 #pragma unroll
-    for (int e = 0; e < 8; ++e) { red[rl * 32 + g * 8 + e] = s0[e]; red[1024 + rl * 32 + g * 8 + e] = s1[e]; }
+    for (int e = 0; e < 8; ++e) { red[rl * 32 + g * 8 + e] = s0[e]; red[2048 + rl * 32 + g * 8 + e] = s1[e]; }
     __syncthreads();
     if (tid < 32) {
         float a0 = 0.f, a1 = 0.f;
 #pragma unroll
-        for (int l = 0; l < 32; ++l) { a0 += red[l * 32 + tid]; a1 += red[1024 + l * 32 + tid]; }
+        for (int l = 0; l < 64; ++l) { a0 += red[l * 32 + tid]; a1 += red[2048 + l * 32 + tid]; }
         out0[col0 + tid] = accumulate ? out0[col0 + tid] + a0 : a0;
         if (xhat_of) out1[col0 + tid] = accumulate ? out1[col0 + tid] + a1 : a1;
     }
@@ -449,10 +445,13 @@ __device__ __forceinline__ float delta_row(const uint16_t* dout, const uint16_t*
     return s;
 }
 
-// Forward: 64 query rows of one head; warp w owns rows 16 w .. 16 w + 15, scores and P stay in registers.
-__device__ __noinline__ void attn_fwd_unit(const WholeLayerArgs& p, int b, int h, int qb, uint32_t sm)
+// Forward: 64 query rows of one head.  Warps w and w + 4 share rows 16 (w % 4) .. + 15; each takes one
+// half (32 keys) of every 64-key block and runs its own online softmax over its keys, with scores and P
+// in registers; the two partial results (running maximum, sum, unnormalised O) are merged at the end
+// through shared memory.  `mrg` is 4 x (16 x 64 + 32) floats.
+__device__ __noinline__ void attn_fwd_unit(const WholeLayerArgs& p, int b, int h, int qb, uint32_t sm, float* mrg)
 {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, rw = warp & 3, kh = warp >> 2;
     const size_t ld = 3 * static_cast<size_t>(p.d);
     const uint16_t* qkv = static_cast<const uint16_t*>(p.qkv);
     const uint16_t* base = qkv + static_cast<size_t>(b) * p.S * ld + h * 64;
@@ -465,7 +464,6 @@ __device__ __noinline__ void attn_fwd_unit(const WholeLayerArgs& p, int b, int h
     stage_chunk(sQ, base + static_cast<size_t>(qb) * 64 * ld, ld, tid);
     load_kv(0);
     cp_async_commit();
-    uint32_t qf[4][4];
     float oacc[8][4];
 #pragma unroll
     for (int i = 0; i < 8; ++i)
@@ -478,91 +476,122 @@ __device__ __noinline__ void attn_fwd_unit(const WholeLayerArgs& p, int b, int h
         cp_async_wait<1>();
         __syncthreads();
         const uint32_t sK = sm + (1 + 2 * (j & 1)) * kChunk, sV = sK + kChunk;
-        if (j == 0) {
+        float s[4][4];
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) frag_a_k(sQ, warp * 16, kk, lane, qf[kk]);
-        }
-        float s[8][4];
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
+        for (int i = 0; i < 4; ++i)
 #pragma unroll
             for (int e = 0; e < 4; ++e) s[i][e] = 0.f;
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk)
+        for (int kk = 0; kk < 4; ++kk) {
+            uint32_t qf[4];
+            frag_a_k(sQ, rw * 16, kk, lane, qf);
 #pragma unroll
-            for (int np = 0; np < 4; ++np) {
+            for (int np = 0; np < 2; ++np) {
                 uint32_t bf[4];
-                frag_b_k(sK, np * 16, kk, lane, bf);
-                mma16816(s[2 * np], qf[kk], bf[0], bf[1]);
-                mma16816(s[2 * np + 1], qf[kk], bf[2], bf[3]);
+                frag_b_k(sK, kh * 32 + np * 16, kk, lane, bf);
+                mma16816(s[2 * np], qf, bf[0], bf[1]);
+                mma16816(s[2 * np + 1], qf, bf[2], bf[3]);
             }
+        }
         float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
-        for (int ni = 0; ni < 8; ++ni)
+        for (int ni = 0; ni < 4; ++ni)
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 float t = s[ni][e] * sl2;
                 if (j == qb) {
-                    const int key = ni * 8 + 2 * (lane & 3) + (e & 1), row = warp * 16 + (lane >> 2) + 8 * (e >> 1);
+                    const int key = kh * 32 + ni * 8 + 2 * (lane & 3) + (e & 1), row = rw * 16 + (lane >> 2) + 8 * (e >> 1);
                     if (key > row) t = -INFINITY;
                 }
                 s[ni][e] = t;
                 mx[e >> 1] = fmaxf(mx[e >> 1], t);
             }
-        float alpha[2];
+        float alpha[2], mb[2];
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
             mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 1));
             mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 2));
             const float mn = fmaxf(m[hh], mx[hh]);
-            alpha[hh] = exp2f(m[hh] - mn);
+            mb[hh] = mn == -INFINITY ? 0.f : mn;            // a half may see only masked keys of a row
+            alpha[hh] = exp2f(m[hh] - mb[hh]);
             m[hh] = mn;
             l[hh] *= alpha[hh];
         }
 #pragma unroll
-        for (int ni = 0; ni < 8; ++ni)
+        for (int ni = 0; ni < 4; ++ni)
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const float pe = exp2f(s[ni][e] - m[e >> 1]);
+                const float pe = exp2f(s[ni][e] - mb[e >> 1]);
                 s[ni][e] = pe;
                 l[e >> 1] += pe;
-                oacc[ni][e] *= alpha[e >> 1];
             }
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
+        for (int ni = 0; ni < 8; ++ni)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) oacc[ni][e] *= alpha[e >> 1];
+#pragma unroll
+        for (int kk = 0; kk < 2; ++kk) {
             uint32_t a[4] = {pack_bf16(s[2 * kk][0], s[2 * kk][1]), pack_bf16(s[2 * kk][2], s[2 * kk][3]),
                              pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]), pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3])};
 #pragma unroll
             for (int np = 0; np < 4; ++np) {
                 uint32_t bf[4];
-                frag_b_mn(sV, np * 16, kk, lane, bf);
+                frag_b_mn(sV, np * 16, kh * 2 + kk, lane, bf);
                 mma16816(oacc[2 * np], a, bf[0], bf[1]);
                 mma16816(oacc[2 * np + 1], a, bf[2], bf[3]);
             }
         }
         __syncthreads();                                    // K and V may be overwritten
     }
-    uint16_t* o = static_cast<uint16_t*>(p.o);
-    float* lse = static_cast<float*>(p.lse);
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
         l[hh] += __shfl_xor_sync(0xffffffffu, l[hh], 1);
         l[hh] += __shfl_xor_sync(0xffffffffu, l[hh], 2);
-        const float inv = 1.0f / l[hh];
-        const int q = qb * 64 + warp * 16 + (lane >> 2) + 8 * hh;
-        const size_t row = static_cast<size_t>(b) * p.S + q;
-#pragma unroll
-        for (int ni = 0; ni < 8; ++ni)
-            store_bf16x2(o, row * p.d + h * 64 + ni * 8 + 2 * (lane & 3), oacc[ni][2 * hh] * inv, oacc[ni][2 * hh + 1] * inv);
-        if ((lane & 3) == 0) lse[(static_cast<size_t>(b) * p.H + h) * p.S + q] = m[hh] * 0.6931471805599453f + logf(l[hh]);
     }
+    // merge: the upper half hands (m, l, O) to the lower half
+    float* mine = mrg + rw * (16 * 64 + 32);
+    if (kh == 1) {
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int r = (lane >> 2) + 8 * hh;
+#pragma unroll
+            for (int ni = 0; ni < 8; ++ni)
+                *reinterpret_cast<float2*>(mine + r * 64 + ni * 8 + 2 * (lane & 3)) = make_float2(oacc[ni][2 * hh], oacc[ni][2 * hh + 1]);
+            if ((lane & 3) == 0) { mine[1024 + r] = m[hh]; mine[1040 + r] = l[hh]; }
+        }
+    }
+    __syncthreads();
+    if (kh == 0) {
+        uint16_t* o = static_cast<uint16_t*>(p.o);
+        float* lse = static_cast<float*>(p.lse);
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int r = (lane >> 2) + 8 * hh;
+            const float m2 = mine[1024 + r], l2 = mine[1040 + r];
+            const float mt = fmaxf(m[hh], m2);              // the lower half always sees key 0: finite
+            const float c1 = exp2f(m[hh] - mt), c2 = m2 == -INFINITY ? 0.f : exp2f(m2 - mt);
+            const float lt = l[hh] * c1 + l2 * c2, inv = 1.0f / lt;
+            const int q = qb * 64 + rw * 16 + r;
+            const size_t row = static_cast<size_t>(b) * p.S + q;
+#pragma unroll
+            for (int ni = 0; ni < 8; ++ni) {
+                const float2 o2 = *reinterpret_cast<const float2*>(mine + r * 64 + ni * 8 + 2 * (lane & 3));
+                store_bf16x2(o, row * p.d + h * 64 + ni * 8 + 2 * (lane & 3), (oacc[ni][2 * hh] * c1 + o2.x * c2) * inv,
+                             (oacc[ni][2 * hh + 1] * c1 + o2.y * c2) * inv);
+            }
+            if ((lane & 3) == 0) lse[(static_cast<size_t>(b) * p.H + h) * p.S + q] = mt * 0.6931471805599453f + logf(lt);
+        }
+    }
+    __syncthreads();                                        // the merge area may be rewritten by the next unit
 }
 
 // Backward, dQ of 64 query rows of one head: per key block S and dP are rebuilt, dS = P (dP - delta)
-// goes straight from the accumulator registers into the A operand of dQ += dS K.
-__device__ __noinline__ void attn_dq_unit(const WholeLayerArgs& p, int b, int h, int qb, uint32_t sm, float* vec)
+// goes straight from the accumulator registers into the A operand of dQ += dS K.  Warps w and w + 4
+// share rows 16 (w % 4) .. + 15 and split every key block in halves; the two partial dQ are added (lower
+// half first) through shared memory.  `mrg` is 4 x 16 x 64 floats.
+__device__ __noinline__ void attn_dq_unit(const WholeLayerArgs& p, int b, int h, int qb, uint32_t sm, float* vec, float* mrg)
 {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, rw = warp & 3, kh = warp >> 2;
     const size_t ld = 3 * static_cast<size_t>(p.d);
     const uint16_t* base = static_cast<const uint16_t*>(p.qkv) + static_cast<size_t>(b) * p.S * ld + h * 64;
     const uint16_t* dout = static_cast<const uint16_t*>(p.td0);
@@ -580,7 +609,9 @@ __device__ __noinline__ void attn_dq_unit(const WholeLayerArgs& p, int b, int h,
     cp_async_commit();
     if (tid < 64) vec[tid] = delta_row(dout, o, (row0 + tid) * p.d + h * 64);
     float lse2[2], dlt[2];
-    uint32_t qf[4][4], dof[4][4];
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh)
+        lse2[hh] = __ldcg(static_cast<const float*>(p.lse) + (static_cast<size_t>(b) * p.H + h) * p.S + qb * 64 + rw * 16 + (lane >> 2) + 8 * hh) * 1.4426950408889634f;
     float dq[8][4];
 #pragma unroll
     for (int i = 0; i < 8; ++i)
@@ -594,74 +625,87 @@ __device__ __noinline__ void attn_dq_unit(const WholeLayerArgs& p, int b, int h,
         const uint32_t sK = sm + (2 + 2 * (j & 1)) * kChunk, sV = sK + kChunk;
         if (j == 0) {
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-                frag_a_k(sQ, warp * 16, kk, lane, qf[kk]);
-                frag_a_k(sDO, warp * 16, kk, lane, dof[kk]);
-            }
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                const int r = warp * 16 + (lane >> 2) + 8 * hh;
-                lse2[hh] = __ldcg(static_cast<const float*>(p.lse) + (static_cast<size_t>(b) * p.H + h) * p.S + qb * 64 + r) * 1.4426950408889634f;
-                dlt[hh] = vec[r];
-            }
+            for (int hh = 0; hh < 2; ++hh) dlt[hh] = vec[rw * 16 + (lane >> 2) + 8 * hh];
         }
-        float s[8][4], dp[8][4];
+        float s[4][4], dp[4][4];
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
+        for (int i = 0; i < 4; ++i)
 #pragma unroll
             for (int e = 0; e < 4; ++e) { s[i][e] = 0.f; dp[i][e] = 0.f; }
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk)
+        for (int kk = 0; kk < 4; ++kk) {
+            uint32_t qf[4], dof[4];
+            frag_a_k(sQ, rw * 16, kk, lane, qf);
+            frag_a_k(sDO, rw * 16, kk, lane, dof);
 #pragma unroll
-            for (int np = 0; np < 4; ++np) {
+            for (int np = 0; np < 2; ++np) {
                 uint32_t bf[4];
-                frag_b_k(sK, np * 16, kk, lane, bf);
-                mma16816(s[2 * np], qf[kk], bf[0], bf[1]);
-                mma16816(s[2 * np + 1], qf[kk], bf[2], bf[3]);
-                frag_b_k(sV, np * 16, kk, lane, bf);
-                mma16816(dp[2 * np], dof[kk], bf[0], bf[1]);
-                mma16816(dp[2 * np + 1], dof[kk], bf[2], bf[3]);
+                frag_b_k(sK, kh * 32 + np * 16, kk, lane, bf);
+                mma16816(s[2 * np], qf, bf[0], bf[1]);
+                mma16816(s[2 * np + 1], qf, bf[2], bf[3]);
+                frag_b_k(sV, kh * 32 + np * 16, kk, lane, bf);
+                mma16816(dp[2 * np], dof, bf[0], bf[1]);
+                mma16816(dp[2 * np + 1], dof, bf[2], bf[3]);
             }
+        }
 #pragma unroll
-        for (int ni = 0; ni < 8; ++ni)
+        for (int ni = 0; ni < 4; ++ni)
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 float pe = exp2f(fmaf(s[ni][e], sl2, -lse2[e >> 1]));
                 if (j == qb) {
-                    const int key = ni * 8 + 2 * (lane & 3) + (e & 1), row = warp * 16 + (lane >> 2) + 8 * (e >> 1);
+                    const int key = kh * 32 + ni * 8 + 2 * (lane & 3) + (e & 1), row = rw * 16 + (lane >> 2) + 8 * (e >> 1);
                     if (key > row) pe = 0.f;
                 }
                 s[ni][e] = pe * (dp[ni][e] - dlt[e >> 1]);
             }
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
+        for (int kk = 0; kk < 2; ++kk) {
             uint32_t a[4] = {pack_bf16(s[2 * kk][0], s[2 * kk][1]), pack_bf16(s[2 * kk][2], s[2 * kk][3]),
                              pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]), pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3])};
 #pragma unroll
             for (int np = 0; np < 4; ++np) {
                 uint32_t bf[4];
-                frag_b_mn(sK, np * 16, kk, lane, bf);
+                frag_b_mn(sK, np * 16, kh * 2 + kk, lane, bf);
                 mma16816(dq[2 * np], a, bf[0], bf[1]);
                 mma16816(dq[2 * np + 1], a, bf[2], bf[3]);
             }
         }
         __syncthreads();
     }
-    uint16_t* dqkv = static_cast<uint16_t*>(p.big);
+    float* mine = mrg + rw * (16 * 64);
+    if (kh == 1) {
 #pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-        const size_t row = row0 + warp * 16 + (lane >> 2) + 8 * hh;
+        for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
-        for (int ni = 0; ni < 8; ++ni)
-            store_bf16x2(dqkv, row * ld + h * 64 + ni * 8 + 2 * (lane & 3), dq[ni][2 * hh] * p.scale, dq[ni][2 * hh + 1] * p.scale);
+            for (int ni = 0; ni < 8; ++ni)
+                *reinterpret_cast<float2*>(mine + ((lane >> 2) + 8 * hh) * 64 + ni * 8 + 2 * (lane & 3)) = make_float2(dq[ni][2 * hh], dq[ni][2 * hh + 1]);
     }
+    __syncthreads();
+    if (kh == 0) {
+        uint16_t* dqkv = static_cast<uint16_t*>(p.big);
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int r = (lane >> 2) + 8 * hh;
+            const size_t row = row0 + rw * 16 + r;
+#pragma unroll
+            for (int ni = 0; ni < 8; ++ni) {
+                const float2 o2 = *reinterpret_cast<const float2*>(mine + r * 64 + ni * 8 + 2 * (lane & 3));
+                store_bf16x2(dqkv, row * ld + h * 64 + ni * 8 + 2 * (lane & 3), (dq[ni][2 * hh] + o2.x) * p.scale,
+                             (dq[ni][2 * hh + 1] + o2.y) * p.scale);
+            }
+        }
+    }
+    __syncthreads();
 }
 
 // Backward, dK and dV of 64 key rows of one head: per query block the transposed scores K Q^T and
-// V dO^T are built, so that P^T and dS^T come out of the accumulators as A operands.
-__device__ __noinline__ void attn_dkdv_unit(const WholeLayerArgs& p, int b, int h, int kb, uint32_t sm, float* vec)
+// V dO^T are built, so that P^T and dS^T come out of the accumulators as A operands.  Warps w and w + 4
+// share keys 16 (w % 4) .. + 15 and split every query block in halves; the partial dK and dV are added
+// (lower half first) through shared memory.  `mrg` is 2 x 4 x 16 x 64 floats.
+__device__ __noinline__ void attn_dkdv_unit(const WholeLayerArgs& p, int b, int h, int kb, uint32_t sm, float* vec, float* mrg)
 {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, rw = warp & 3, qh = warp >> 2;
     const size_t ld = 3 * static_cast<size_t>(p.d);
     const uint16_t* base = static_cast<const uint16_t*>(p.qkv) + static_cast<size_t>(b) * p.S * ld + h * 64;
     const uint16_t* dout = static_cast<const uint16_t*>(p.td0);
@@ -683,7 +727,6 @@ __device__ __noinline__ void attn_dkdv_unit(const WholeLayerArgs& p, int b, int 
         v_lse[r] = __ldcg(static_cast<const float*>(p.lse) + (static_cast<size_t>(b) * p.H + h) * p.S + r) * 1.4426950408889634f;
         v_dlt[r] = delta_row(dout, o, (seq0 + r) * p.d + h * 64);
     }
-    uint32_t kf[4][4], vf[4][4];
     float dk[8][4], dv[8][4];
 #pragma unroll
     for (int i = 0; i < 8; ++i)
@@ -696,46 +739,43 @@ __device__ __noinline__ void attn_dkdv_unit(const WholeLayerArgs& p, int b, int 
         cp_async_wait<1>();
         __syncthreads();
         const uint32_t sQ = sm + (2 + 2 * (i & 1)) * kChunk, sDO = sQ + kChunk;
-        if (i == kb) {
+        float st[4][4], dpt[4][4];
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-                frag_a_k(sK, warp * 16, kk, lane, kf[kk]);
-                frag_a_k(sV, warp * 16, kk, lane, vf[kk]);
-            }
-        }
-        float st[8][4], dpt[8][4];
-#pragma unroll
-        for (int a = 0; a < 8; ++a)
+        for (int a = 0; a < 4; ++a)
 #pragma unroll
             for (int e = 0; e < 4; ++e) { st[a][e] = 0.f; dpt[a][e] = 0.f; }
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk)
+        for (int kk = 0; kk < 4; ++kk) {
+            uint32_t kf[4], vf[4];
+            frag_a_k(sK, rw * 16, kk, lane, kf);
+            frag_a_k(sV, rw * 16, kk, lane, vf);
 #pragma unroll
-            for (int np = 0; np < 4; ++np) {
+            for (int np = 0; np < 2; ++np) {
                 uint32_t bf[4];
-                frag_b_k(sQ, np * 16, kk, lane, bf);
-                mma16816(st[2 * np], kf[kk], bf[0], bf[1]);
-                mma16816(st[2 * np + 1], kf[kk], bf[2], bf[3]);
-                frag_b_k(sDO, np * 16, kk, lane, bf);
-                mma16816(dpt[2 * np], vf[kk], bf[0], bf[1]);
-                mma16816(dpt[2 * np + 1], vf[kk], bf[2], bf[3]);
+                frag_b_k(sQ, qh * 32 + np * 16, kk, lane, bf);
+                mma16816(st[2 * np], kf, bf[0], bf[1]);
+                mma16816(st[2 * np + 1], kf, bf[2], bf[3]);
+                frag_b_k(sDO, qh * 32 + np * 16, kk, lane, bf);
+                mma16816(dpt[2 * np], vf, bf[0], bf[1]);
+                mma16816(dpt[2 * np + 1], vf, bf[2], bf[3]);
             }
+        }
         // st -> P^T (kept for dV), dpt -> dS^T
 #pragma unroll
-        for (int ni = 0; ni < 8; ++ni)
+        for (int ni = 0; ni < 4; ++ni)
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const int qcol = ni * 8 + 2 * (lane & 3) + (e & 1), q = i * 64 + qcol;
+                const int qcol = qh * 32 + ni * 8 + 2 * (lane & 3) + (e & 1), q = i * 64 + qcol;
                 float pe = exp2f(fmaf(st[ni][e], sl2, -v_lse[q]));
                 if (i == kb) {
-                    const int key = warp * 16 + (lane >> 2) + 8 * (e >> 1);
+                    const int key = rw * 16 + (lane >> 2) + 8 * (e >> 1);
                     if (key > qcol) pe = 0.f;
                 }
                 st[ni][e] = pe;
                 dpt[ni][e] = pe * (dpt[ni][e] - v_dlt[q]);
             }
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
+        for (int kk = 0; kk < 2; ++kk) {
             uint32_t a[4] = {pack_bf16(st[2 * kk][0], st[2 * kk][1]), pack_bf16(st[2 * kk][2], st[2 * kk][3]),
                              pack_bf16(st[2 * kk + 1][0], st[2 * kk + 1][1]), pack_bf16(st[2 * kk + 1][2], st[2 * kk + 1][3])};
             uint32_t c[4] = {pack_bf16(dpt[2 * kk][0], dpt[2 * kk][1]), pack_bf16(dpt[2 * kk][2], dpt[2 * kk][3]),
@@ -743,27 +783,46 @@ __device__ __noinline__ void attn_dkdv_unit(const WholeLayerArgs& p, int b, int 
 #pragma unroll
             for (int np = 0; np < 4; ++np) {
                 uint32_t bf[4];
-                frag_b_mn(sDO, np * 16, kk, lane, bf);
+                frag_b_mn(sDO, np * 16, qh * 2 + kk, lane, bf);
                 mma16816(dv[2 * np], a, bf[0], bf[1]);
                 mma16816(dv[2 * np + 1], a, bf[2], bf[3]);
-                frag_b_mn(sQ, np * 16, kk, lane, bf);
+                frag_b_mn(sQ, np * 16, qh * 2 + kk, lane, bf);
                 mma16816(dk[2 * np], c, bf[0], bf[1]);
                 mma16816(dk[2 * np + 1], c, bf[2], bf[3]);
             }
         }
         __syncthreads();
     }
-    uint16_t* dqkv = static_cast<uint16_t*>(p.big);
+    float* mk = mrg + rw * (16 * 64);
+    float* mv = mrg + 4 * 16 * 64 + rw * (16 * 64);
+    if (qh == 1) {
 #pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-        const size_t row = seq0 + kb * 64 + warp * 16 + (lane >> 2) + 8 * hh;
+        for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
-        for (int ni = 0; ni < 8; ++ni) {
-            const size_t at = row * ld + h * 64 + ni * 8 + 2 * (lane & 3);
-            store_bf16x2(dqkv, at + p.d, dk[ni][2 * hh] * p.scale, dk[ni][2 * hh + 1] * p.scale);
-            store_bf16x2(dqkv, at + 2 * p.d, dv[ni][2 * hh], dv[ni][2 * hh + 1]);
+            for (int ni = 0; ni < 8; ++ni) {
+                const int at = ((lane >> 2) + 8 * hh) * 64 + ni * 8 + 2 * (lane & 3);
+                *reinterpret_cast<float2*>(mk + at) = make_float2(dk[ni][2 * hh], dk[ni][2 * hh + 1]);
+                *reinterpret_cast<float2*>(mv + at) = make_float2(dv[ni][2 * hh], dv[ni][2 * hh + 1]);
+            }
+    }
+    __syncthreads();
+    if (qh == 0) {
+        uint16_t* dqkv = static_cast<uint16_t*>(p.big);
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int r = (lane >> 2) + 8 * hh;
+            const size_t row = seq0 + kb * 64 + rw * 16 + r;
+#pragma unroll
+            for (int ni = 0; ni < 8; ++ni) {
+                const int at = r * 64 + ni * 8 + 2 * (lane & 3);
+                const float2 k2 = *reinterpret_cast<const float2*>(mk + at), v2 = *reinterpret_cast<const float2*>(mv + at);
+                const size_t dst = row * ld + h * 64 + ni * 8 + 2 * (lane & 3);
+                store_bf16x2(dqkv, dst + p.d, (dk[ni][2 * hh] + k2.x) * p.scale, (dk[ni][2 * hh + 1] + k2.y) * p.scale);
+                store_bf16x2(dqkv, dst + 2 * p.d, dv[ni][2 * hh] + v2.x, dv[ni][2 * hh + 1] + v2.y);
+            }
         }
     }
+    __syncthreads();
 }
 
 // ---------------------------------------------------------------- the phases
@@ -779,14 +838,14 @@ struct Ctx {
 // The accumulators leave the registers through a 64 x 64 fp32 tile in shared memory; the epilogue is
 // then a rolled loop over 16-byte pieces of the output (8 columns of a row per thread and turn), short
 // enough to stay in the instruction cache and storing whole 16-byte pieces.
-__device__ __forceinline__ void acc_to_smem(const float (&acc)[2][4][4], float* tile)
+__device__ __forceinline__ void acc_to_smem(const float (&acc)[2][2][4], float* tile)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int r = (warp & 1) * 32 + (lane >> 2), c = (warp >> 1) * 32 + 2 * (lane & 3);
+    const int r = (warp & 1) * 32 + (lane >> 2), c = (warp >> 1) * 16 + 2 * (lane & 3);
 #pragma unroll
     for (int mi = 0; mi < 2; ++mi)
 #pragma unroll
-        for (int ni = 0; ni < 4; ++ni)
+        for (int ni = 0; ni < 2; ++ni)
 #pragma unroll
             for (int h = 0; h < 2; ++h)
                 *reinterpret_cast<float2*>(tile + (r + mi * 16 + h * 8) * kAccStride + c + ni * 8) =
@@ -812,7 +871,7 @@ __device__ __noinline__ void fwd_gemm_unit(const Ctx& c, int u, int mode, const 
     const WholeLayerArgs& p = c.p;
     const int tile = u / nslices, slice = u % nslices, ntn = N >> 6, tm = tile / ntn, tn = tile % ntn;
     const int m0 = tm * 64, n0 = tn * 64, kper = K / nslices, tid = threadIdx.x;
-    float acc[2][4][4];
+    float acc[2][2][4];
     const TileGemm<false, false, LN> g{A, static_cast<size_t>(K), W, static_cast<size_t>(K), m0, n0, LN ? 0 : slice * kper,
                                        (LN ? K : kper) >> 6, c.sm + kSmStage};
     const int stride = (p.d + 8) * 2;
@@ -838,8 +897,8 @@ __device__ __noinline__ void fwd_gemm_unit(const Ctx& c, int u, int mode, const 
     float bv[8];
     unpack8(__ldg(reinterpret_cast<const uint4*>(bias + n0 + c8)), bv);
 #pragma unroll 1
-    for (int it = 0; it < 4; ++it) {
-        const int row = (tid >> 3) + it * 16;
+    for (int it = 0; it < 2; ++it) {
+        const int row = (tid >> 3) + it * 32;
         float v[8];
         tile_piece(tl, row, c8, v);
 #pragma unroll
@@ -868,7 +927,7 @@ __device__ __noinline__ void dgrad_unit(const Ctx& c, int u, const uint16_t* A, 
 {
     const int tile = u / nslices, slice = u % nslices, ntn = N >> 6, m0 = (tile / ntn) * 64, n0 = (tile % ntn) * 64;
     const int kper = K / nslices, tid = threadIdx.x;
-    float acc[2][4][4];
+    float acc[2][2][4];
     const TileGemm<false, true, false> g{A, static_cast<size_t>(K), W, static_cast<size_t>(N), m0, n0, slice * kper, kper >> 6,
                                          c.sm + kSmStage};
     if (gelu_u) stage_chunk(c.sm + kSmAux, gelu_u + static_cast<size_t>(m0) * N + n0, N, tid);
@@ -879,8 +938,8 @@ __device__ __noinline__ void dgrad_unit(const Ctx& c, int u, const uint16_t* A, 
     acc_to_smem(acc, tl);
     const int act = c.p.act, c8 = (tid & 7) * 8;
 #pragma unroll 1
-    for (int it = 0; it < 4; ++it) {
-        const int row = (tid >> 3) + it * 16;
+    for (int it = 0; it < 2; ++it) {
+        const int row = (tid >> 3) + it * 32;
         float v[8];
         tile_piece(tl, row, c8, v);
         if (gelu_u) {
@@ -898,21 +957,21 @@ __device__ __noinline__ void dgrad_unit(const Ctx& c, int u, const uint16_t* A, 
 __device__ __noinline__ void wgrad_unit(const Ctx& c, int u, const uint16_t* A, int M, const uint16_t* B, int N, float* dW)
 {
     const int ntn = N >> 6, m0 = (u / ntn) * 64, n0 = (u % ntn) * 64, tid = threadIdx.x;
-    float acc[2][4][4];
+    float acc[2][2][4];
     const TileGemm<true, true, false> g{A, static_cast<size_t>(M), B, static_cast<size_t>(N), m0, n0, 0, c.p.T >> 6, c.sm + kSmStage};
     g.prefetch();
-    float4 old[8];
+    float4 old[4];
     const int c4 = (tid & 15) * 4;
     if (c.p.accumulate) {
 #pragma unroll
-        for (int it = 0; it < 8; ++it) old[it] = *reinterpret_cast<const float4*>(dW + static_cast<size_t>(m0 + (tid >> 4) + it * 8) * N + n0 + c4);
+        for (int it = 0; it < 4; ++it) old[it] = *reinterpret_cast<const float4*>(dW + static_cast<size_t>(m0 + (tid >> 4) + it * 16) * N + n0 + c4);
     }
     g.run(acc, 0, 0);
     float* tl = reinterpret_cast<float*>(c.smem + kSmAcc);
     acc_to_smem(acc, tl);
 #pragma unroll
-    for (int it = 0; it < 8; ++it) {
-        const int row = (tid >> 4) + it * 8;
+    for (int it = 0; it < 4; ++it) {
+        const int row = (tid >> 4) + it * 16;
         float4 v = *reinterpret_cast<const float4*>(tl + row * kAccStride + c4);
         if (c.p.accumulate) { v.x += old[it].x; v.y += old[it].y; v.z += old[it].z; v.w += old[it].w; }
         *reinterpret_cast<float4*>(dW + static_cast<size_t>(m0 + row) * N + n0 + c4) = v;
@@ -940,13 +999,13 @@ __global__ void __launch_bounds__(kThreads, 1) whole_layer_fwd_kernel(const __gr
         const int nqb = p.S >> 6, n = p.B * p.H * nqb;
         for (int u = blockIdx.x; u < n; u += G) {
             const int qb = nqb - 1 - u / (p.B * p.H), bh = u % (p.B * p.H);      // long rows first
-            attn_fwd_unit(p, bh / p.H, bh % p.H, qb, c.sm + kSmStage);
+            attn_fwd_unit(p, bh / p.H, bh % p.H, qb, c.sm + kSmStage, reinterpret_cast<float*>(smem + kSmPanel));
         }
     }
     if (!grid_barrier(p.sync, p.status, c.flag)) return;
     // 3: x1 = x + o Wo^T + bo
-    for (int u = blockIdx.x; u < tm * (d >> 6) * p.split_d; u += G)
-        fwd_gemm_unit<false>(c, u, kFwdResid, cu16(p.o), d, cu16(p.w_o), cu16(p.b_o), d, p.split_d, cu16(p.x), u16(p.x1), nullptr,
+    for (int u = blockIdx.x; u < tm * (d >> 6) * p.split_o; u += G)
+        fwd_gemm_unit<false>(c, u, kFwdResid, cu16(p.o), d, cu16(p.w_o), cu16(p.b_o), d, p.split_o, cu16(p.x), u16(p.x1), nullptr,
                              nullptr, nullptr, nullptr, nullptr, nullptr);
     if (!grid_barrier(p.sync, p.status, c.flag)) return;
     // 4: u = LN2(x1) W1^T + b1, a = GeLU(u)
@@ -956,8 +1015,8 @@ __global__ void __launch_bounds__(kThreads, 1) whole_layer_fwd_kernel(const __gr
     if (!p.with_fc2) return;
     if (!grid_barrier(p.sync, p.status, c.flag)) return;
     // 5: y = x1 + a W2^T + b2
-    for (int u = blockIdx.x; u < tm * (d >> 6) * p.split_f; u += G)
-        fwd_gemm_unit<false>(c, u, kFwdResid, cu16(p.a), F, cu16(p.w_fc2), cu16(p.b_fc2), d, p.split_f, cu16(p.x1), u16(p.y), nullptr,
+    for (int u = blockIdx.x; u < tm * (d >> 6) * p.split_fc2; u += G)
+        fwd_gemm_unit<false>(c, u, kFwdResid, cu16(p.a), F, cu16(p.w_fc2), cu16(p.b_fc2), d, p.split_fc2, cu16(p.x1), u16(p.y), nullptr,
                              nullptr, nullptr, nullptr, nullptr, nullptr);
 }
 
@@ -972,31 +1031,31 @@ __global__ void __launch_bounds__(kThreads, 1) whole_layer_bwd_kernel(const __gr
     const int acc = p.accumulate;
     // 1: du = (dy W2) * GeLU'(u);  dW2 = dy^T a;  db2 = colsum(dy)
     {
-        const int n0 = tm * (F >> 6), n1 = n0 + (d >> 6) * (F >> 6), n2 = n1 + (d >> 5);
+        const int n0 = (d >> 6) * (F >> 6), n1 = n0 + tm * (F >> 6), n2 = n1 + (d >> 5);
         for (int u = blockIdx.x; u < n2; u += G) {
-            if (u < n0) dgrad_unit(c, u, cu16(p.dy), d, cu16(p.w_fc2), F, 1, cu16(p.u), u16(p.big));
-            else if (u < n1) wgrad_unit(c, u - n0, cu16(p.dy), d, cu16(p.a), F, f32(p.g_w_fc2));
+            if (u < n0) wgrad_unit(c, u, cu16(p.dy), d, cu16(p.a), F, f32(p.g_w_fc2));
+            else if (u < n1) dgrad_unit(c, u - n0, cu16(p.dy), d, cu16(p.w_fc2), F, 1, cu16(p.u), u16(p.big));
             else colsum_unit(cu16(p.dy), d, T, (u - n1) * 32, nullptr, nullptr, nullptr, f32(p.g_b_fc2), nullptr, acc, red);
         }
     }
     if (!grid_barrier(p.sync, p.status, c.flag)) return;
     // 2: dh2 = du W1;  dW1 = du^T h2;  db1 = colsum(du)
     {
-        const int n0 = tm * (d >> 6) * p.split_f, n1 = n0 + (F >> 6) * (d >> 6), n2 = n1 + (F >> 5);
+        const int n0 = (F >> 6) * (d >> 6), n1 = n0 + tm * (d >> 6) * p.split_dh2, n2 = n1 + (F >> 5);
         for (int u = blockIdx.x; u < n2; u += G) {
-            if (u < n0) dgrad_unit(c, u, cu16(p.big), F, cu16(p.w_fc1), d, p.split_f, nullptr, u16(p.td0));
-            else if (u < n1) wgrad_unit(c, u - n0, cu16(p.big), F, cu16(p.h2), d, f32(p.g_w_fc1));
+            if (u < n0) wgrad_unit(c, u, cu16(p.big), F, cu16(p.h2), d, f32(p.g_w_fc1));
+            else if (u < n1) dgrad_unit(c, u - n0, cu16(p.big), F, cu16(p.w_fc1), d, p.split_dh2, nullptr, u16(p.td0));
             else colsum_unit(cu16(p.big), F, T, (u - n1) * 32, nullptr, nullptr, nullptr, f32(p.g_b_fc1), nullptr, acc, red);
         }
     }
     if (!grid_barrier(p.sync, p.status, c.flag)) return;
-    // 3: dx1 = dy + LN2bwd(dh2);  dgamma2, dbeta2
+    // 3: dx1 = dy + LN2bwd(dh2) (a row per warp);  dgamma2, dbeta2
     {
-        const int n0 = T >> 2, n1 = n0 + (d >> 5);
+        const int n0 = T >> 3, n1 = n0 + (d >> 5);
         for (int u = blockIdx.x; u < n1; u += G) {
             if (u < n0) {
-                if (d == 256) ln_bwd_row<1>(cu16(p.td0), cu16(p.x1), f32(p.mu2), f32(p.r2), cu16(p.ln2_g), cu16(p.dy), u16(p.dx1), u * 4 + warp);
-                else ln_bwd_row<2>(cu16(p.td0), cu16(p.x1), f32(p.mu2), f32(p.r2), cu16(p.ln2_g), cu16(p.dy), u16(p.dx1), u * 4 + warp);
+                if (d == 256) ln_bwd_row<1>(cu16(p.td0), cu16(p.x1), f32(p.mu2), f32(p.r2), cu16(p.ln2_g), cu16(p.dy), u16(p.dx1), u * 8 + warp);
+                else ln_bwd_row<2>(cu16(p.td0), cu16(p.x1), f32(p.mu2), f32(p.r2), cu16(p.ln2_g), cu16(p.dy), u16(p.dx1), u * 8 + warp);
             }
             else colsum_unit(cu16(p.td0), d, T, (u - n0) * 32, cu16(p.x1), f32(p.mu2), f32(p.r2), f32(p.g_ln2_g), f32(p.g_ln2_b), acc, red);
         }
@@ -1004,10 +1063,10 @@ __global__ void __launch_bounds__(kThreads, 1) whole_layer_bwd_kernel(const __gr
     if (!grid_barrier(p.sync, p.status, c.flag)) return;
     // 4: dout = dx1 Wo;  dWo = dx1^T o;  dbo = colsum(dx1)
     {
-        const int n0 = tm * (d >> 6) * p.split_d, n1 = n0 + (d >> 6) * (d >> 6), n2 = n1 + (d >> 5);
+        const int n0 = (d >> 6) * (d >> 6), n1 = n0 + tm * (d >> 6) * p.split_o, n2 = n1 + (d >> 5);
         for (int u = blockIdx.x; u < n2; u += G) {
-            if (u < n0) dgrad_unit(c, u, cu16(p.dx1), d, cu16(p.w_o), d, p.split_d, nullptr, u16(p.td0));
-            else if (u < n1) wgrad_unit(c, u - n0, cu16(p.dx1), d, cu16(p.o), d, f32(p.g_w_o));
+            if (u < n0) wgrad_unit(c, u, cu16(p.dx1), d, cu16(p.o), d, f32(p.g_w_o));
+            else if (u < n1) dgrad_unit(c, u - n0, cu16(p.dx1), d, cu16(p.w_o), d, p.split_o, nullptr, u16(p.td0));
             else colsum_unit(cu16(p.dx1), d, T, (u - n1) * 32, nullptr, nullptr, nullptr, f32(p.g_b_o), nullptr, acc, red);
         }
     }
@@ -1017,29 +1076,29 @@ __global__ void __launch_bounds__(kThreads, 1) whole_layer_bwd_kernel(const __gr
         const int nb = p.S >> 6, BH = p.B * p.H, n = BH * nb;
         for (int u = blockIdx.x; u < 2 * n; u += G) {
             const int v = u >> 1, blk = v / BH, bh = v % BH;
-            if (u & 1) attn_dq_unit(p, bh / p.H, bh % p.H, nb - 1 - blk, c.sm + kSmStage, vec);     // long rows first
-            else attn_dkdv_unit(p, bh / p.H, bh % p.H, blk, c.sm + kSmStage, vec);                  // long columns first
+            if (u & 1) attn_dq_unit(p, bh / p.H, bh % p.H, nb - 1 - blk, c.sm + kSmStage, vec, red);     // long rows first
+            else attn_dkdv_unit(p, bh / p.H, bh % p.H, blk, c.sm + kSmStage, vec, red);                  // long columns first
             __syncthreads();
         }
     }
     if (!grid_barrier(p.sync, p.status, c.flag)) return;
     // 6: dh1 = dqkv Wqkv;  dWqkv = dqkv^T h1;  dbqkv = colsum(dqkv)
     {
-        const int n0 = tm * (d >> 6) * p.split_3d, n1 = n0 + (3 * d >> 6) * (d >> 6), n2 = n1 + (3 * d >> 5);
+        const int n0 = (3 * d >> 6) * (d >> 6), n1 = n0 + tm * (d >> 6) * p.split_dh1, n2 = n1 + (3 * d >> 5);
         for (int u = blockIdx.x; u < n2; u += G) {
-            if (u < n0) dgrad_unit(c, u, cu16(p.big), 3 * d, cu16(p.w_qkv), d, p.split_3d, nullptr, u16(p.td0));
-            else if (u < n1) wgrad_unit(c, u - n0, cu16(p.big), 3 * d, cu16(p.h1), d, f32(p.g_w_qkv));
+            if (u < n0) wgrad_unit(c, u, cu16(p.big), 3 * d, cu16(p.h1), d, f32(p.g_w_qkv));
+            else if (u < n1) dgrad_unit(c, u - n0, cu16(p.big), 3 * d, cu16(p.w_qkv), d, p.split_dh1, nullptr, u16(p.td0));
             else colsum_unit(cu16(p.big), 3 * d, T, (u - n1) * 32, nullptr, nullptr, nullptr, f32(p.g_b_qkv), nullptr, acc, red);
         }
     }
     if (!grid_barrier(p.sync, p.status, c.flag)) return;
     // 7: dx = dx1 + LN1bwd(dh1);  dgamma1, dbeta1
     {
-        const int n0 = T >> 2, n1 = n0 + (d >> 5);
+        const int n0 = T >> 3, n1 = n0 + (d >> 5);
         for (int u = blockIdx.x; u < n1; u += G) {
             if (u < n0) {
-                if (d == 256) ln_bwd_row<1>(cu16(p.td0), cu16(p.x), f32(p.mu1), f32(p.r1), cu16(p.ln1_g), cu16(p.dx1), u16(p.dx), u * 4 + warp);
-                else ln_bwd_row<2>(cu16(p.td0), cu16(p.x), f32(p.mu1), f32(p.r1), cu16(p.ln1_g), cu16(p.dx1), u16(p.dx), u * 4 + warp);
+                if (d == 256) ln_bwd_row<1>(cu16(p.td0), cu16(p.x), f32(p.mu1), f32(p.r1), cu16(p.ln1_g), cu16(p.dx1), u16(p.dx), u * 8 + warp);
+                else ln_bwd_row<2>(cu16(p.td0), cu16(p.x), f32(p.mu1), f32(p.r1), cu16(p.ln1_g), cu16(p.dx1), u16(p.dx), u * 8 + warp);
             }
             else colsum_unit(cu16(p.td0), d, T, (u - n0) * 32, cu16(p.x), f32(p.mu1), f32(p.r1), f32(p.g_ln1_g), f32(p.g_ln1_b), acc, red);
         }
@@ -1083,9 +1142,11 @@ const char* whole_layer_unsupported(int T, int d, int H, int dh, int F, int S)
 // Slices of the K range of a GEMM with `tiles` output tiles.  Meeting the other slices costs three
 // trips to L2 (partial tile out, ticket, partial tiles back in), about as much as eight 64-wide
 // blocks of products, so only long K ranges are cut: into as many slices as keep every slice at
-// least two blocks long, divide the block count, and do not push the phase beyond one round of CTAs.
-static int pick_slices(int tiles, int K, int grid)
+// least two blocks long, divide the block count, and fit into `room` CTAs - what one round of the grid
+// has left beside the other GEMM of the phase (the short column-sum units go to a second round).
+static int pick_slices(int tiles, int K, int room)
 {
+    const int grid = room;
     const int blocks = K / 64;
     int best = 1;
     if (blocks < 12) return 1;
@@ -1100,9 +1161,10 @@ const char* launch_whole_layer(Runtime* rt, WholeLayerArgs a, bool backward, cud
 {
     const int grid = rt->sm_count;
     const int tiles = (a.T >> 6) * (a.d >> 6);
-    a.split_d = pick_slices(tiles, a.d, grid);
-    a.split_f = pick_slices(tiles, a.F, grid);
-    a.split_3d = pick_slices(tiles, 3 * a.d, grid);
+    a.split_o = pick_slices(tiles, a.d, grid - (a.d >> 6) * (a.d >> 6));
+    a.split_fc2 = pick_slices(tiles, a.F, grid);
+    a.split_dh2 = pick_slices(tiles, a.F, grid - (a.F >> 6) * (a.d >> 6));
+    a.split_dh1 = pick_slices(tiles, 3 * a.d, grid - (3 * a.d >> 6) * (a.d >> 6));
     const cudaError_t e = launch_coop(backward ? whole_layer_bwd_kernel : whole_layer_fwd_kernel, grid, stream, a);
     return e == cudaSuccess ? nullptr : cudaGetErrorString(e);
 }
