@@ -192,13 +192,15 @@ enum {
     PW_K_ATTN_FWD = 3,
     PW_K_ATTN_BWD = 4,  /* delta + dq + dkdv kernels          */
     PW_K_LN_FWD = 5,
-    PW_K_LN_BWD = 6,    /* main kernel + partial reduction    */
-    PW_K_COLSUM = 7,    /* main kernel + partial reduction    */
+    PW_K_LN_BWD = 6,    /* main kernel (+ partial reduction when called as a single step) */
+    PW_K_COLSUM = 7,    /* main kernel (+ partial reduction when called as a single step) */
     PW_K_XENT = 8,      /* softmax / cross-entropy + loss mean (pw_lm_step)          */
     PW_K_EMBED = 9,     /* embedding lookup and its scatter-add backward (pw_lm_step) */
     PW_K_GELU = 10,     /* GeLU(u) re-derived in the backward of a PW_FLAG_LEAN_CTX layer */
     PW_K_WHOLE_LAYER = 11, /* forward or backward of a PW_FLAG_WHOLE_LAYER handle (one launch each) */
-    PW_K_COUNT = 12
+    PW_K_REDUCE = 12,   /* one launch per layer backward: fixed-order sums of the partial rows that its two
+                           LayerNorm backward kernels and its two bias column sums left (8 gradient vectors) */
+    PW_K_COUNT = 13
 };
 typedef struct pw_profile {
     uint64_t launches[PW_K_COUNT]; /* kernel launches per class since profile_begin      */
@@ -361,6 +363,18 @@ pw_status_t pw_op_embedding_bwd(const int32_t* ids, const void* dx0, int T, int 
 pw_status_t pw_op_softmax_xent(void* logits, int ld, const int32_t* labels, int T, int V, float grad_scale,
                                void* lse, void* loss_rows, void* stream);
 
+/* The output projection's data gradient with the first step of attention backward folded into its
+ * epilogue (the backward of Section 5.3's Transformer layer; the fusion itself is this library's):
+ *   C bf16 [M,N] = A [M,K] B [K,N]   (PW_GEMM_NN operands: dout = dx1 Wo), and
+ *   row_dot fp32 [M / seq_len, N / head_dim, seq_len]: row_dot[b][h][s] = sum over the head_dim
+ *   columns c of head h of acc[b * seq_len + s][c] * other[b * seq_len + s][c], with acc the fp32
+ *   product before it is rounded to bf16 and other bf16 [M,N] (row stride ld_other) = the attention
+ *   output o; this is the rowsum(dO * O) that pw_op_attention_bwd otherwise computes itself.
+ * head_dim 64 or 128 dividing N; seq_len dividing M; M, N, K multiples of 8; pointers 16-byte
+ * aligned (row_dot: 4).  Errors: PW_ERR_CUDA with a message for a shape the GEMM refuses. */
+pw_status_t pw_op_gemm_rowdot(int M, int N, int K, const void* A, int lda, const void* B, int ldb, void* C, int ldc,
+                              const void* other, int ld_other, int head_dim, int seq_len, void* row_dot, void* stream);
+
 /* Causal attention forward on packed qkv (bf16 [T,3d]); o bf16 [T,d]; lse fp32 [B,H,S].
  * The attention kernels are persistent and hand out their work through counters that live
  * beside the status word: the pw_op_attention_* calls of one device share one set, so two of them
@@ -369,7 +383,9 @@ pw_status_t pw_op_softmax_xent(void* logits, int ld, const int32_t* labels, int 
 pw_status_t pw_op_attention_fwd(const void* qkv, int B, int S, int H, int dh, void* o, void* lse, void* stream);
 
 /* Causal attention backward.  dout bf16 [T,d]; dqkv bf16 [T,3d] (same packing as qkv);
- * delta: fp32 device scratch [B,H,S] (receives rowsum(dout*o)). */
+ * delta: fp32 device scratch [B,H,S] (receives rowsum(dout*o)).  With o = NULL the call takes
+ * delta as an input - already filled, e.g. by pw_op_gemm_rowdot - and launches two kernels
+ * instead of three. */
 pw_status_t pw_op_attention_bwd(const void* qkv, const void* o, const void* dout, const void* lse, int B, int S,
                                 int H, int dh, void* dqkv, void* delta, void* stream);
 

@@ -38,7 +38,7 @@ EXPORTS = (
     "pw_stage_create", "pw_stage_destroy", "pw_stage_workspace_bytes", "pw_stage_run_chain", "pw_stage_status",
     "pw_stage_profile_begin", "pw_stage_profile_end", "pw_stage_launch_count",
     "pw_op_layernorm_fwd", "pw_op_layernorm_bwd_scratch_bytes", "pw_op_layernorm_bwd",
-    "pw_op_colsum_scratch_bytes", "pw_op_colsum", "pw_op_colsum_noalloc", "pw_op_gemm",
+    "pw_op_colsum_scratch_bytes", "pw_op_colsum", "pw_op_colsum_noalloc", "pw_op_gemm", "pw_op_gemm_rowdot",
     "pw_op_attention_fwd", "pw_op_attention_bwd", "pw_op_status",
     "pw_lm_workspace_bytes", "pw_lm_step",
     "pw_op_embedding_fwd", "pw_op_embedding_bwd_scratch_bytes", "pw_op_embedding_bwd", "pw_op_softmax_xent",
@@ -74,12 +74,12 @@ class ApplyItem(ctypes.Structure):
 
 
 KERNEL_CLASSES = ("gemm_tn", "gemm_nn", "gemm_nt", "attn_fwd", "attn_bwd", "ln_fwd", "ln_bwd", "colsum", "xent", "embed",
-                  "gelu", "whole_layer")
+                  "gelu", "whole_layer", "reduce")
 
 
 class Profile(ctypes.Structure):
-    _fields_ = [("launches", ctypes.c_uint64 * 12), ("ms", ctypes.c_double * 12), ("flops", ctypes.c_double * 12),
-                ("bytes", ctypes.c_double * 12)]
+    _fields_ = [("launches", ctypes.c_uint64 * 13), ("ms", ctypes.c_double * 13), ("flops", ctypes.c_double * 13),
+                ("bytes", ctypes.c_double * 13)]
 
     def as_dict(self):
         return {n: dict(launches=int(self.launches[i]), ms=float(self.ms[i]), flops=float(self.flops[i]),
@@ -143,6 +143,7 @@ def lib() -> ctypes.CDLL:
         L.pw_op_colsum.argtypes = [vp, ci, ci, ci, vp, ci, vp, vp]
         L.pw_op_colsum_noalloc.argtypes = [vp, ci, ci, ci, vp, ci, vp]
         L.pw_op_gemm.argtypes = [ci, ci, ci, ci, ci, ci, vp, ci, vp, ci, vp, ci, vp, vp, ci, vp, ci, vp]
+        L.pw_op_gemm_rowdot.argtypes = [ci, ci, ci, vp, ci, vp, ci, vp, ci, vp, ci, ci, ci, vp, vp]
         L.pw_op_attention_fwd.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp]
         L.pw_op_attention_bwd.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, vp]
         L.pw_op_status.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci)]
@@ -418,6 +419,11 @@ def op_gemm(layout, epilogue, M, N, K, A, lda, B, ldb, C, ldc, bias=None, aux_in
             accumulate=False, act=ACT_GELU_ERF, stream=None):
     _check(lib().pw_op_gemm(layout, epilogue, act, M, N, K, _p(A), lda, _p(B), ldb, _p(C), ldc, _p(bias), _p(aux_in),
                             ld_aux, _p(aux_out), int(accumulate), _stream(stream)))
+
+
+def op_gemm_rowdot(M, N, K, A, lda, B, ldb, C, ldc, other, ld_other, head_dim, seq_len, row_dot, stream=None):
+    _check(lib().pw_op_gemm_rowdot(M, N, K, _p(A), lda, _p(B), ldb, _p(C), ldc, _p(other), ld_other, head_dim, seq_len,
+                                   _p(row_dot), _stream(stream)))
 
 
 def op_attention_fwd(qkv, B, S, H, dh, o, lse, stream=None):

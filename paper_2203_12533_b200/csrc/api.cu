@@ -80,7 +80,7 @@ struct LayerPlan {
     float eps;
     size_t ctx_off[PW_CTX_COUNT], ctx_size[PW_CTX_COUNT], ctx_bytes;
     // scratch = [ctx-shaped region used when the caller passes ctx == NULL] [backward temporaries]
-    size_t off_big, off_td0, off_td1, off_delta, off_partials, off_partials2, scratch_bytes;
+    size_t off_big, off_td0, off_td1, off_delta, off_partials, off_partials2, off_partials3, off_partials4, scratch_bytes;
     // lean ctx: h1, h2, a (and the statistics the re-derivation writes again) live in scratch
     bool lean;
     size_t off_lean_h1, off_lean_h2, off_lean_a, off_lean_stats;
@@ -171,7 +171,11 @@ static void build_plan(const pw_layer_config_t& c, Runtime* rt, LayerPlan* p)
     if (c1 > part) part = c1;
     if (c2 > part) part = c2;
     p->off_partials = s; s += align256(part);
-    p->off_partials2 = s; s += align256(c1 > c2 ? c1 : c2);   // column sums on the side stream
+    // The four sets of partial rows of a backward call (LN2, LN1, the two bias column sums) are
+    // summed by one launch at the end of the call, so each has a region of its own.
+    p->off_partials2 = s; s += align256(c1);                                           // db1 column sums (side stream)
+    p->off_partials3 = s; s += align256(layernorm_bwd_scratch_bytes(rt, p->T, p->d));  // LN1 backward
+    p->off_partials4 = s; s += align256(c2);                                           // dbqkv column sums (side stream)
     p->off_splitk = s; s += align256(gemm_split_ws_bytes());
     p->off_lean_h1 = p->off_lean_h2 = p->off_lean_a = p->off_lean_stats = 0;
     if (p->lean) {
@@ -259,20 +263,32 @@ static pw_status_t do_ln_fwd(pw_layer_t* L, const void* x, const void* gamma, co
 }
 static pw_status_t do_ln_bwd(pw_layer_t* L, const void* dh, const void* x, const void* mu, const void* rstd,
                              const void* gamma, const void* resid, void* dx, void* dgamma, void* dbeta, void* db_resid,
-                             void* db_dx, int accumulate, void* partials, cudaStream_t st)
+                             void* db_dx, int accumulate, void* partials, cudaStream_t st, ReduceJob* defer = nullptr)
 {
+    // defer: the partial rows are left for a later launch_reduce_jobs (the caller collects the jobs)
     const LayerPlan& p = L->plan;
-    LaunchScope sc(L, PW_K_LN_BWD, 2, 0.0, 8.0 * p.T * p.d + 8.0 * p.T, st);
-    const char* e = launch_layernorm_bwd(L->rt, dh, x, mu, rstd, gamma, resid, p.T, p.d, dx, dgamma, dbeta, db_resid,
-                                         db_dx, accumulate, partials, st);
+    LaunchScope sc(L, PW_K_LN_BWD, defer ? 1 : 2, 0.0, 8.0 * p.T * p.d + 8.0 * p.T, st);
+    const char* e = defer
+        ? launch_layernorm_bwd_partial(L->rt, dh, x, mu, rstd, gamma, resid, p.T, p.d, dx, dgamma, dbeta, db_resid, db_dx,
+                                       partials, defer, st)
+        : launch_layernorm_bwd(L->rt, dh, x, mu, rstd, gamma, resid, p.T, p.d, dx, dgamma, dbeta, db_resid, db_dx,
+                               accumulate, partials, st);
     return e ? fail(PW_ERR_CUDA, e) : PW_OK;
 }
 static pw_status_t do_colsum(pw_layer_t* L, const void* in, int N, void* out, int accumulate, void* partials,
-                             cudaStream_t st)
+                             cudaStream_t st, ReduceJob* defer = nullptr)
 {
     const LayerPlan& p = L->plan;
-    LaunchScope sc(L, PW_K_COLSUM, 2, 0.0, 2.0 * p.T * N, st);
-    const char* e = launch_colsum(L->rt, in, p.T, N, N, out, accumulate, partials, st);
+    LaunchScope sc(L, PW_K_COLSUM, defer ? 1 : 2, 0.0, 2.0 * p.T * N, st);
+    const char* e = defer ? launch_colsum_partial(L->rt, in, p.T, N, N, out, partials, defer, st)
+                          : launch_colsum(L->rt, in, p.T, N, N, out, accumulate, partials, st);
+    return e ? fail(PW_ERR_CUDA, e) : PW_OK;
+}
+static pw_status_t do_reduce(pw_layer_t* L, const ReduceJob* jobs, int njobs, int accumulate, cudaStream_t st)
+{
+    LaunchScope sc(L, PW_K_REDUCE, 1, 0.0, 0.0, st);
+    const char* e = launch_reduce_jobs(jobs, njobs, accumulate, st);
+    if (e) sc.cancel(1);
     return e ? fail(PW_ERR_CUDA, e) : PW_OK;
 }
 // Attention FLOPs count the visible (causal) pairs only: 2 T (S+1) d forward, 2.5x that backward.
@@ -287,9 +303,10 @@ static pw_status_t do_attn_bwd(pw_layer_t* L, const void* qkv, const void* o, co
                                void* dqkv, void* delta, cudaStream_t st)
 {
     const LayerPlan& p = L->plan;
-    LaunchScope sc(L, PW_K_ATTN_BWD, 3, 5.0 * p.T * (p.S + 1.0) * p.d, 0.0, st);
+    const int nk = o ? 3 : 2;                            // o == nullptr: delta was filled by the GEMM that made dout
+    LaunchScope sc(L, PW_K_ATTN_BWD, nk, 5.0 * p.T * (p.S + 1.0) * p.d, 0.0, st);
     const char* e = launch_attention_bwd(L->rt, qkv, o, dout, lse, p.B, p.S, p.H, p.dh, dqkv, delta, L->status, st);
-    if (e) sc.cancel(3);
+    if (e) sc.cancel(nk);
     return e ? fail(PW_ERR_CUDA, e) : PW_OK;
 }
 
@@ -391,6 +408,9 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
     void* part = at(scratch, p.off_partials);
 
     void* part2 = at(scratch, p.off_partials2);
+    void* part3 = at(scratch, p.off_partials3);
+    void* part4 = at(scratch, p.off_partials4);
+    ReduceJob jobs[4];                                   // LN2, db1, LN1, dbqkv: summed by one launch at the end
 
     // The weight gradients and the bias column sums hang off the dgrad chain, so they run on a
     // side stream: their CTAs fill the SMs that the last, partly filled round of a dgrad GEMM
@@ -426,7 +446,7 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
     if (rederive) PW_DO(do_ln_fwd(L, x1, P->ln2_gamma, P->ln2_beta, const_cast<void*>(h2), lean_st1, lean_st2, ax));
     PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, F, d, T, big, F, h2, d, G->w_fc1, d, nullptr, nullptr, 0,
                                      nullptr, accumulate), ax));
-    PW_DO(do_colsum(L, big, F, G->b_fc1, accumulate, part2, ax));
+    PW_DO(do_colsum(L, big, F, G->b_fc1, accumulate, part2, ax, &jobs[1]));
     if (ax != st) {                                      // remembered: du may be overwritten only after these two
         cudaError_t e = cudaEventRecord(L->ev[2], ax);
         if (e != cudaSuccess) return fail_cuda("stream ordering", e);
@@ -435,31 +455,37 @@ static pw_status_t enqueue_bwd(pw_layer_t* L, const pw_layer_params_t* P, const 
                                      nullptr, 0, sk), st));
     // LN2 backward + residual: dx1 = dy + LNbwd(dh2); also db2 = colsum(dy), dbo = colsum(dx1)
     PW_DO(do_ln_bwd(L, td0, x1, mu2, r2, P->ln2_gamma, dy, dx1, G->ln2_gamma, G->ln2_beta,
-                                G->b_fc2, G->b_o, accumulate, part, st));
+                                G->b_fc2, G->b_o, accumulate, part, st, &jobs[0]));
     PW_DO(order(L->ev[3], st, ax));                      // dx1 ready
     // x1 = x + o Wo^T + bo  ->  dout = dx1 Wo,  dWo = dx1^T o
     PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, d, d, T, dx1, d, o, d, G->w_o, d, nullptr, nullptr, 0,
                                      nullptr, accumulate), ax));
-    PW_DO(do_gemm(L, gemm_args(kNN, kEpiNone, act, T, d, d, dx1, d, P->w_o, d, td0, d, nullptr, nullptr, 0,
-                                     nullptr, 0, sk), st));
+    // (the epilogue also takes delta = rowsum(dout * o) per token and head, which attention backward starts from)
+    {
+        GemmArgs g = gemm_args(kNN, kEpiRowDot, act, T, d, d, dx1, d, P->w_o, d, td0, d, nullptr, o, d, nullptr, 0, sk);
+        g.row_dot = delta; g.head_dim = p.dh; g.seq_len = p.S;
+        PW_DO(do_gemm(L, g, st));
+    }
     // attention backward -> dqkv (reuses the du buffer)
     if (ax != st) {
         cudaError_t e = cudaStreamWaitEvent(st, L->ev[2], 0);
         if (e != cudaSuccess) return fail_cuda("stream ordering", e);
     }
-    PW_DO(do_attn_bwd(L, qkv, o, td0, lse, big, delta, st));
+    PW_DO(do_attn_bwd(L, qkv, nullptr, td0, lse, big, delta, st));
     PW_DO(order(L->ev[4], st, ax));                      // dqkv ready
     // qkv = h1 Wqkv^T + bqkv  ->  dh1 = dqkv Wqkv,  dWqkv = dqkv^T h1,  dbqkv = colsum(dqkv)
     if (rederive) PW_DO(do_ln_fwd(L, x, P->ln1_gamma, P->ln1_beta, const_cast<void*>(h1), lean_st1, lean_st2, ax));
     PW_DO(do_gemm(L, gemm_args(kNT, kEpiF32, act, 3 * d, d, T, big, 3 * d, h1, d, G->w_qkv, d, nullptr, nullptr,
                                      0, nullptr, accumulate), ax));
-    PW_DO(do_colsum(L, big, 3 * d, G->b_qkv, accumulate, part2, ax));
+    PW_DO(do_colsum(L, big, 3 * d, G->b_qkv, accumulate, part4, ax, &jobs[3]));
     PW_DO(do_gemm(L, gemm_args(kNN, kEpiNone, act, T, d, 3 * d, big, 3 * d, P->w_qkv, d, td0, d, nullptr,
                                      nullptr, 0, nullptr, 0, sk), st));
     // LN1 backward + residual: dx = dx1 + LNbwd(dh1)
     PW_DO(do_ln_bwd(L, td0, x, mu1, r1, P->ln1_gamma, dx1, dx, G->ln1_gamma, G->ln1_beta, nullptr,
-                                nullptr, accumulate, part, st));
+                                nullptr, accumulate, part3, st, &jobs[2]));
     PW_DO(order(L->ev[5], ax, st));                      // join
+    // dgamma1/2, dbeta1/2, db2, dbo, db1, dbqkv: eight vectors, one fixed-order launch
+    PW_DO(do_reduce(L, jobs, 4, accumulate, st));
     return PW_OK;
 }
 
@@ -1069,6 +1095,16 @@ pw_status_t pw_op_gemm(int layout, int epilogue, int act, int M, int N, int K, c
     return PW_OK;
 }
 
+pw_status_t pw_op_gemm_rowdot(int M, int N, int K, const void* A, int lda, const void* B, int ldb, void* C, int ldc,
+                              const void* other, int ld_other, int head_dim, int seq_len, void* row_dot, void* stream)
+{
+    PW_RT_OR_FAIL();
+    GemmArgs g = gemm_args(kNN, kEpiRowDot, 0, M, N, K, A, lda, B, ldb, C, ldc, nullptr, other, ld_other, nullptr, 0, rt->split_ws);
+    g.row_dot = row_dot; g.head_dim = head_dim; g.seq_len = seq_len;
+    PW_OP(launch_gemm(rt, g, rt->op_status, static_cast<cudaStream_t>(stream)));
+    return PW_OK;
+}
+
 pw_status_t pw_op_attention_fwd(const void* qkv, int B, int S, int H, int dh, void* o, void* lse, void* stream)
 {
     PW_RT_OR_FAIL();
@@ -1081,7 +1117,7 @@ pw_status_t pw_op_attention_bwd(const void* qkv, const void* o, const void* dout
                                 int dh, void* dqkv, void* delta, void* stream)
 {
     PW_RT_OR_FAIL();
-    if (!aligned(qkv, 16) || !aligned(o, 16) || !aligned(dout, 16) || !lse || !aligned(dqkv, 16) || !delta)
+    if (!aligned(qkv, 16) || (o && !aligned(o, 16)) || !aligned(dout, 16) || !lse || !aligned(dqkv, 16) || !delta)
         return fail(PW_ERR_INVALID_ARG, "attention bwd: NULL or misaligned pointer");
     PW_OP(launch_attention_bwd(rt, qkv, o, dout, lse, B, S, H, dh, dqkv, delta, rt->op_status, static_cast<cudaStream_t>(stream)));
     return PW_OK;

@@ -1,5 +1,6 @@
-// Attention backward, host side: delta = rowsum(dO * O) (HBM-bound, below), then the two tcgen05
-// kernels of attention_bwd_sm100.cu (dq; dk and dv).
+// Attention backward, host side: delta = rowsum(dO * O) (HBM-bound, below; skipped when the GEMM that
+// produced dO already took the sums in its epilogue), then the two tcgen05 kernels of
+// attention_bwd_sm100.cu (dq; dk and dv).
 #include "pw_kernels.h"
 
 namespace pw {
@@ -71,7 +72,7 @@ const char* launch_attention_bwd(Runtime* rt, const void* qkv, const void* o, co
                                  cudaStream_t stream)
 {
     if (B <= 0 || H <= 0 || S <= 0 || (S % 128) != 0 || (dh != 64 && dh != 128)) return "attention: unsupported shape";
-    {
+    if (o != nullptr) {                                      // o == nullptr: delta already holds rowsum(dout * o)
         const size_t total = static_cast<size_t>(B) * S * H * (dh / 8);
         if (total >= (1ull << 31)) return "attention: too many (token, head) pairs for the row-dot kernel";
         if (launch_k(attn_delta_kernel, dim3(static_cast<unsigned>((total + 1023) / 1024)), dim3(256), 0, stream,

@@ -340,27 +340,31 @@ ln_bwd_kernel(const __nv_bfloat16* dh, const __nv_bfloat16* x,
     }
 }
 
-// out_q[c] (+)= sum over partial rows of partials[row][q][c].  CTA = 64 columns x 16 row lanes, a thread
+// out[c] (+)= sum over partial rows r of src[r * stride + c], for up to eight (src, out) entries in one
+// launch (grid.y = entry): the partial rows of the two LayerNorm backward kernels and of the two bias
+// column sums of a layer's backward end up in one launch.  CTA = 64 columns x 16 row lanes, a thread
 // owns four consecutive columns (16-byte loads, eight rows in flight): row lane y adds rows y, y+16, ...
 // in order, then the 16 lane sums are added in order, so the result does not depend on scheduling.
-// Up to 4 outputs (grid.y = quantity).  n is a multiple of 4.
-struct ReduceOuts { float* out[4]; };
+// n is a multiple of 4.
+struct ReduceEntry { const float* src; float* out; int nrows, n; long long stride; };
+struct ReduceTable { ReduceEntry e[kReduceMaxEntries]; };
 constexpr int kReduceCols = 64, kReduceLanes = 16;
 __global__ void __launch_bounds__(kReduceCols / 4 * kReduceLanes)
-reduce_partials_kernel(const float* partials, int nrows, int nq, int n, ReduceOuts outs, int accumulate)
+reduce_partials_kernel(const __grid_constant__ ReduceTable tab, int accumulate)
 {
     __shared__ float4 sm[kReduceLanes][kReduceCols / 4];
     const int cx = threadIdx.x & (kReduceCols / 4 - 1), ry = threadIdx.x / (kReduceCols / 4);
     const int c = blockIdx.x * kReduceCols + cx * 4;
-    const int q = blockIdx.y;
-    float* out = outs.out[q];
+    const ReduceEntry& en = tab.e[blockIdx.y];
+    float* out = en.out;
+    const int n = en.n, nrows = en.nrows;
     grid_dep_launch();
     grid_dep_wait();
-    if (out == nullptr) return;
+    if (out == nullptr || blockIdx.x * kReduceCols >= n) return;
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
     if (c < n) {
-        const size_t stride = static_cast<size_t>(nq) * n;             // floats between partial rows
-        const float* src = partials + static_cast<size_t>(q) * n + c;
+        const size_t stride = static_cast<size_t>(en.stride);          // floats between partial rows
+        const float* src = en.src + c;
         int r = ry;
         for (; r + 7 * kReduceLanes < nrows; r += 8 * kReduceLanes) {
             float4 v[8];
@@ -479,10 +483,11 @@ size_t layernorm_bwd_scratch_bytes(Runtime* rt, int T, int d)
     return static_cast<size_t>(ln_bwd_grid(rt, T, rp)) * rp.rows_per_cta * 4 * d * sizeof(float);
 }
 
-const char* launch_layernorm_bwd(Runtime* rt, const void* dh, const void* x, const void* mu, const void* rstd,
-                                 const void* gamma, const void* resid, int T, int d, void* dx, void* dgamma,
-                                 void* dbeta, void* db_resid, void* db_dx, int accumulate, void* partials,
-                                 cudaStream_t stream)
+// Main kernel only: the partial rows stay in `partials` and `job` says how to reduce them.
+const char* launch_layernorm_bwd_partial(Runtime* rt, const void* dh, const void* x, const void* mu, const void* rstd,
+                                         const void* gamma, const void* resid, int T, int d, void* dx, void* dgamma,
+                                         void* dbeta, void* db_resid, void* db_dx, void* partials, ReduceJob* job,
+                                         cudaStream_t stream)
 {
     RowPlan rp;
     if (T <= 0 || !plan_rows(d, &rp)) return "layernorm: unsupported row width";
@@ -506,13 +511,43 @@ const char* launch_layernorm_bwd(Runtime* rt, const void* dh, const void* x, con
     }
 #undef PW_LN_BWD
     if (le != cudaSuccess) return "layernorm bwd launch failed";
-    ReduceOuts outs;
-    outs.out[0] = static_cast<float*>(dgamma); outs.out[1] = static_cast<float*>(dbeta);
-    outs.out[2] = static_cast<float*>(db_resid); outs.out[3] = static_cast<float*>(db_dx);
-    const int nq = sums ? 4 : 2;
-    dim3 rgrid((d + kReduceCols - 1) / kReduceCols, nq);
-    return launch_k(reduce_partials_kernel, rgrid, dim3(kReduceCols / 4 * kReduceLanes), 0, stream, static_cast<const float*>(P), grid * rp.rows_per_cta, nq, d, outs, accumulate) == cudaSuccess
-               ? nullptr : "layernorm bwd reduce launch failed";
+    job->partials = P; job->nrows = grid * rp.rows_per_cta; job->nq = sums ? 4 : 2; job->n = d;
+    job->out[0] = static_cast<float*>(dgamma); job->out[1] = static_cast<float*>(dbeta);
+    job->out[2] = static_cast<float*>(db_resid); job->out[3] = static_cast<float*>(db_dx);
+    return nullptr;
+}
+
+// One launch for the partial rows of up to four jobs (at most eight output vectors in all).
+const char* launch_reduce_jobs(const ReduceJob* jobs, int njobs, int accumulate, cudaStream_t stream)
+{
+    ReduceTable tab = {};
+    int ne = 0, max_n = 0;
+    for (int j = 0; j < njobs; ++j)
+        for (int q = 0; q < jobs[j].nq; ++q) {
+            if (jobs[j].out[q] == nullptr) continue;
+            if (ne == kReduceMaxEntries) return "reduce: too many output vectors for one launch";
+            ReduceEntry& en = tab.e[ne++];
+            en.src = jobs[j].partials + static_cast<size_t>(q) * jobs[j].n;
+            en.out = jobs[j].out[q];
+            en.nrows = jobs[j].nrows; en.n = jobs[j].n;
+            en.stride = static_cast<long long>(jobs[j].nq) * jobs[j].n;
+            if (en.n > max_n) max_n = en.n;
+        }
+    if (ne == 0) return nullptr;
+    dim3 rgrid((max_n + kReduceCols - 1) / kReduceCols, ne);
+    return launch_k(reduce_partials_kernel, rgrid, dim3(kReduceCols / 4 * kReduceLanes), 0, stream, tab, accumulate) == cudaSuccess
+               ? nullptr : "partial-row reduce launch failed";
+}
+
+const char* launch_layernorm_bwd(Runtime* rt, const void* dh, const void* x, const void* mu, const void* rstd,
+                                 const void* gamma, const void* resid, int T, int d, void* dx, void* dgamma,
+                                 void* dbeta, void* db_resid, void* db_dx, int accumulate, void* partials,
+                                 cudaStream_t stream)
+{
+    ReduceJob job;
+    const char* e = launch_layernorm_bwd_partial(rt, dh, x, mu, rstd, gamma, resid, T, d, dx, dgamma, dbeta, db_resid, db_dx,
+                                                 partials, &job, stream);
+    return e ? e : launch_reduce_jobs(&job, 1, accumulate, stream);
 }
 
 // y = x * scale + shift on fp32 vectors: the node type of the paper's Figure 2 program (a: x*2,
@@ -545,19 +580,25 @@ size_t colsum_scratch_bytes(Runtime* rt, int T, int N)
     return static_cast<size_t>(colsum_splits(rt, T, N)) * N * sizeof(float);
 }
 
-const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, void* out, int accumulate,
-                          void* partials, cudaStream_t stream)
+const char* launch_colsum_partial(Runtime* rt, const void* in, int T, int N, int ld, void* out, void* partials,
+                                  ReduceJob* job, cudaStream_t stream)
 {
     if (T <= 0 || N <= 0 || (N % 8) || (ld % 8)) return "colsum: N and ld must be multiples of 8";
     const int R = colsum_splits(rt, T, N);
     dim3 grid((N + kColsumCols - 1) / kColsumCols, R);
     if (launch_k(colsum_kernel, grid, dim3(256), 0, stream, static_cast<const __nv_bfloat16*>(in), T, N, ld, static_cast<float*>(partials)) != cudaSuccess)
         return "colsum launch failed";
-    ReduceOuts outs;
-    outs.out[0] = static_cast<float*>(out); outs.out[1] = outs.out[2] = outs.out[3] = nullptr;
-    dim3 rgrid((N + kReduceCols - 1) / kReduceCols, 1);
-    return launch_k(reduce_partials_kernel, rgrid, dim3(kReduceCols / 4 * kReduceLanes), 0, stream, static_cast<const float*>(partials), R, 1, N, outs, accumulate) == cudaSuccess
-               ? nullptr : "colsum reduce launch failed";
+    job->partials = static_cast<const float*>(partials); job->nrows = R; job->nq = 1; job->n = N;
+    job->out[0] = static_cast<float*>(out); job->out[1] = job->out[2] = job->out[3] = nullptr;
+    return nullptr;
+}
+
+const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, void* out, int accumulate,
+                          void* partials, cudaStream_t stream)
+{
+    ReduceJob job;
+    const char* e = launch_colsum_partial(rt, in, T, N, ld, out, partials, &job, stream);
+    return e ? e : launch_reduce_jobs(&job, 1, accumulate, stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -623,10 +664,11 @@ const char* launch_colsum_noalloc(const void* in, int T, int N, int ld, void* ou
     dim3 grid(col_blocks, static_cast<unsigned>(R));
     colsum_kernel<<<grid, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(in), T, N, ld, sc.ptr);
     if (cudaGetLastError() != cudaSuccess) return "colsum launch failed";
-    ReduceOuts outs;
-    outs.out[0] = static_cast<float*>(out); outs.out[1] = outs.out[2] = outs.out[3] = nullptr;
+    ReduceTable tab = {};
+    tab.e[0].src = sc.ptr; tab.e[0].out = static_cast<float*>(out);
+    tab.e[0].nrows = static_cast<int>(R); tab.e[0].n = N; tab.e[0].stride = N;
     dim3 rgrid((N + kReduceCols - 1) / kReduceCols, 1);
-    reduce_partials_kernel<<<rgrid, kReduceCols / 4 * kReduceLanes, 0, stream>>>(sc.ptr, static_cast<int>(R), 1, N, outs, accumulate);
+    reduce_partials_kernel<<<rgrid, kReduceCols / 4 * kReduceLanes, 0, stream>>>(tab, accumulate);
     return cudaGetLastError() == cudaSuccess ? nullptr : "colsum reduce launch failed";
 }
 

@@ -41,6 +41,7 @@ struct GemmParams {
                                  // tiles in the one-CTA kernel, halves of the K range in the CTA-pair kernel
     int total_virtual;           // split_begin + 2 * (m_tiles*n_tiles - split_begin)
     float* split_ws;             // CTA-pair kernel: where the K halves leave their partial sums
+    float* row_dot; int head_dim, seq_len;   // kEpiRowDot: per (row, head) dot products with aux_in, [B, H, S]
     DeviceStatus* status;
 };
 
@@ -157,14 +158,20 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, 
         // swizzle) used alternately, so one store is always in flight behind the math.
         const int nchunks = bn / 32;
         const uint32_t sw = (lane >> 1) & 3;
+        // The warps of a lane quarter take alternate chunks - except with the row-dot epilogue, where each
+        // takes a run of neighbouring chunks, so that all columns of a head meet in one thread.
+        const int ch_first = EPI == kEpiRowDot ? pi * (nchunks / pstride) : pi;
+        const int ch_step = EPI == kEpiRowDot ? 1 : pstride;
+        const int ch_end = EPI == kEpiRowDot ? ch_first + nchunks / pstride : nchunks;
+        float dot = 0.f;
 #pragma unroll 1
-        for (int ch = pi; ch < nchunks; ch += pstride) {
+        for (int ch = ch_first; ch < ch_end; ch += ch_step) {
             const int col0 = n0 + ch * 32;
             if (col0 >= p.N) break;
             // residual / saved pre-activation of this chunk: requested before the TMEM load so that the
             // (row-strided, L2-latency) reads overlap it
             uint4 aux[4] = {};
-            if constexpr (EPI == kEpiBiasResid || EPI == kEpiDGelu) {
+            if constexpr (EPI == kEpiBiasResid || EPI == kEpiDGelu || EPI == kEpiRowDot) {
                 if (row < p.M) {
 #pragma unroll
                     for (int g = 0; g < 4; ++g)
@@ -182,6 +189,12 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, 
                 float f[8];
                 epilogue_group<EPI>(v + 8 * g, row, col0 + g * 8, p, aux[g], f);
                 o[g] = pack8(f);
+                if constexpr (EPI == kEpiRowDot) {
+                    float r[8];
+                    unpack8(aux[g], r);                      // zeros beyond M and N
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) dot = fmaf(f[j], r[j], dot);
+                }
                 if constexpr (EPI == kEpiBiasGelu) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) v[8 * g + j] = __float_as_uint(f[j]);   // fp32 pre-activation, kept for GeLU
@@ -202,6 +215,15 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, int row0, int n0, 
                 }
             };
             store_chunk(o, tmC);
+            if constexpr (EPI == kEpiRowDot) {
+                if ((col0 + 32) % p.head_dim == 0) {         // last chunk of a head: its row sums are complete
+                    if (row < p.M) {
+                        const int b = row / p.seq_len, sq = row - b * p.seq_len, h = col0 / p.head_dim;
+                        p.row_dot[(static_cast<size_t>(b) * (p.N / p.head_dim) + h) * p.seq_len + sq] = dot;
+                    }
+                    dot = 0.f;
+                }
+            }
             if constexpr (EPI == kEpiBiasGelu) {
                 // GeLU of the fp32 pre-activation, evaluated while the store above drains the slab
 #pragma unroll
@@ -636,7 +658,7 @@ const char* configure_gemm()
 {
     const bool ok = set_attr<false, false, kEpiNone>() && set_attr<false, false, kEpiBias>() &&
                     set_attr<false, false, kEpiBiasResid>() && set_attr<false, false, kEpiBiasGelu>() &&
-                    set_attr<false, true, kEpiNone>() && set_attr<false, true, kEpiDGelu>() &&
+                    set_attr<false, true, kEpiNone>() && set_attr<false, true, kEpiDGelu>() && set_attr<false, true, kEpiRowDot>() &&
                     set_attr<true, true, kEpiF32>();
     return ok ? nullptr : "cudaFuncSetAttribute(gemm) failed";
 }
@@ -658,6 +680,7 @@ static const char* launch_gemm_pair(Runtime* rt, const GemmArgs& a, DeviceStatus
         };
         if (cost(128) < cost(256)) bn = 128;
         if (forced == 128 || forced == 256) bn = forced;
+        if (a.epilogue == kEpiRowDot) bn = 256;              // an epilogue warp must own whole heads (128 columns)
     }
     CUtensorMap tmA, tmB, tmC, tmAux;
     const char* e;
@@ -677,6 +700,7 @@ static const char* launch_gemm_pair(Runtime* rt, const GemmArgs& a, DeviceStatus
     p.m_tiles = m_tiles; p.n_tiles = (a.N + bn - 1) / bn;
     p.split_begin = p.m_tiles * p.n_tiles; p.total_virtual = p.split_begin;
     p.split_ws = nullptr;
+    p.row_dot = static_cast<float*>(a.row_dot); p.head_dim = a.head_dim; p.seq_len = a.seq_len;
     {
         // Tail balancing: when the last round of tiles would keep at most half of the CTA pairs busy,
         // each of its tiles becomes two units of half the K range (needs the caller's scratch).
@@ -685,7 +709,7 @@ static const char* launch_gemm_pair(Runtime* rt, const GemmArgs& a, DeviceStatus
         const int rem = total % pairs;
         const int min_k = tuning().gemm_split_min_k;
         // (short K ranges lose more to the second prologue and epilogue than the idle half round costs)
-        if (a.split_ws && !no_split && !f32_out && total > pairs && rem > 0 && 2 * rem <= pairs && rem <= kSplitMaxTiles &&
+        if (a.split_ws && !no_split && !f32_out && a.epilogue != kEpiRowDot && total > pairs && rem > 0 && 2 * rem <= pairs && rem <= kSplitMaxTiles &&
             num_k >= min_k) {
             p.split_begin = total - rem;
             p.total_virtual = p.split_begin + 2 * rem;
@@ -702,6 +726,7 @@ static const char* launch_gemm_pair(Runtime* rt, const GemmArgs& a, DeviceStatus
         case kTN * 16 + kEpiBiasGelu: return launch_pair<false, false, kEpiBiasGelu>(rt, tmA, tmB, tmC, tmAux, p, stream);
         case kNN * 16 + kEpiNone: return launch_pair<false, true, kEpiNone>(rt, tmA, tmB, tmC, tmAux, p, stream);
         case kNN * 16 + kEpiDGelu: return launch_pair<false, true, kEpiDGelu>(rt, tmA, tmB, tmC, tmAux, p, stream);
+        case kNN * 16 + kEpiRowDot: return launch_pair<false, true, kEpiRowDot>(rt, tmA, tmB, tmC, tmAux, p, stream);
         case kNT * 16 + kEpiF32: return launch_pair<true, true, kEpiF32>(rt, tmA, tmB, tmC, tmAux, p, stream);
         default: return "gemm: unsupported layout/epilogue combination";
     }
@@ -718,7 +743,10 @@ const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cu
     auto misaligned = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15) != 0; };
     if (!a.A || !a.B || !a.C || misaligned(a.A) || misaligned(a.B) || misaligned(a.C)) return "gemm: null or misaligned operand";
     const bool need_bias = a.epilogue == kEpiBias || a.epilogue == kEpiBiasResid || a.epilogue == kEpiBiasGelu;
-    const bool need_aux_in = a.epilogue == kEpiBiasResid || a.epilogue == kEpiDGelu;
+    const bool need_aux_in = a.epilogue == kEpiBiasResid || a.epilogue == kEpiDGelu || a.epilogue == kEpiRowDot;
+    if (a.epilogue == kEpiRowDot &&
+        (!a.row_dot || (a.head_dim != 64 && a.head_dim != 128) || (a.N % a.head_dim) || a.seq_len <= 0 || (a.M % a.seq_len)))
+        return "gemm: the row-dot epilogue needs an output, head_dim 64 or 128 dividing N, and seq_len dividing M";
     if (need_bias && (!a.bias || misaligned(a.bias))) return "gemm: epilogue needs a 16-byte aligned bias";
     if (need_aux_in && (!a.aux_in || misaligned(a.aux_in) || (a.ld_aux % 8))) return "gemm: epilogue needs aux_in";
     if (a.epilogue == kEpiBiasGelu && (!a.aux_out || misaligned(a.aux_out))) return "gemm: epilogue needs aux_out";
@@ -739,6 +767,7 @@ const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cu
     {
         const int forced = tuning().gemm_bn;
         if (forced == 128 || forced == 192 || forced == 256) bn = forced;
+        if (a.epilogue == kEpiRowDot) bn = BN_MAX;           // an epilogue warp must own whole heads (128 columns)
     }
     CUtensorMap tmA, tmB, tmBh, tmC, tmAux;
     const char* e;
@@ -766,6 +795,7 @@ const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cu
     p.n_fastest = p.n_tiles < p.m_tiles ? 1 : 0;
     p.status = status;
     p.split_ws = nullptr;
+    p.row_dot = static_cast<float*>(a.row_dot); p.head_dim = a.head_dim; p.seq_len = a.seq_len;
     {
         // Tail balancing: when the last round would leave at least half of the SMs idle, its
         // tiles are issued as two half-width tiles each.
@@ -774,7 +804,7 @@ const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cu
         const int rem = total % grid;
         const bool no_split = tuning().gemm_split == 0;
         p.split_begin = total;
-        if (bn == BN_MAX && rem > 0 && 2 * rem <= grid && !no_split) p.split_begin = total - rem;
+        if (bn == BN_MAX && rem > 0 && 2 * rem <= grid && !no_split && a.epilogue != kEpiRowDot) p.split_begin = total - rem;
         p.total_virtual = p.split_begin + 2 * (total - p.split_begin);
     }
 
@@ -786,6 +816,7 @@ const char* launch_gemm(Runtime* rt, const GemmArgs& a, DeviceStatus* status, cu
         case kTN * 16 + kEpiBiasGelu: return launch_inst<false, false, kEpiBiasGelu>(rt, tmA, tmB, tmBh, tmC, tmAux, p, stream);
         case kNN * 16 + kEpiNone: return launch_inst<false, true, kEpiNone>(rt, tmA, tmB, tmBh, tmC, tmAux, p, stream);
         case kNN * 16 + kEpiDGelu: return launch_inst<false, true, kEpiDGelu>(rt, tmA, tmB, tmBh, tmC, tmAux, p, stream);
+        case kNN * 16 + kEpiRowDot: return launch_inst<false, true, kEpiRowDot>(rt, tmA, tmB, tmBh, tmC, tmAux, p, stream);
         case kNT * 16 + kEpiF32: return launch_inst<true, true, kEpiF32>(rt, tmA, tmB, tmBh, tmC, tmAux, p, stream);
         default: return "gemm: unsupported layout/epilogue combination";
     }

@@ -61,7 +61,8 @@ inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_
 }
 
 enum GemmLayout { kTN = 0, kNN = 1, kNT = 2 };
-enum GemmEpi { kEpiNone = 0, kEpiBias = 1, kEpiBiasResid = 2, kEpiBiasGelu = 3, kEpiDGelu = 4, kEpiF32 = 5 };
+enum GemmEpi { kEpiNone = 0, kEpiBias = 1, kEpiBiasResid = 2, kEpiBiasGelu = 3, kEpiDGelu = 4, kEpiF32 = 5,
+               kEpiRowDot = 6 /* C bf16 = acc, and rowdot[b][h][s] = sum over the columns of head h of acc * aux_in */ };
 
 struct GemmArgs {
     int layout, epilogue, act;
@@ -76,6 +77,10 @@ struct GemmArgs {
     // Optional fp32 scratch of gemm_split_ws_bytes(): lets the tiles of a thin last round be cut in two
     // along K.  Only for GEMMs that never run beside another GEMM using the same status word.
     void* split_ws = nullptr;
+    // kEpiRowDot (the output projection's data gradient, C = dO): per (row, head) dot products of the
+    // fp32 result with aux_in (= O) go to row_dot as fp32 [B, H, S], rows being tokens b * S + s and
+    // heads head_dim consecutive columns - the rowsum(dO * O) that attention backward starts from.
+    void* row_dot = nullptr; int head_dim = 0, seq_len = 0;
 };
 size_t gemm_split_ws_bytes();
 // Encodes the two tensor maps and launches.  Returns nullptr on success, else a static message.
@@ -91,6 +96,24 @@ const char* launch_layernorm_bwd(Runtime* rt, const void* dh, const void* x, con
 size_t colsum_scratch_bytes(Runtime* rt, int T, int N);
 const char* launch_colsum(Runtime* rt, const void* in, int T, int N, int ld, void* out, int accumulate,
                           void* partials, cudaStream_t stream);
+
+// The LayerNorm backward and the column-sum kernels leave one partial row per CTA slot; a second,
+// fixed-order kernel adds them up.  The *_partial launchers run the first kernel only and describe
+// the second in a ReduceJob, so that a caller with several of them (a layer's backward has four)
+// can finish them all with one launch_reduce_jobs - at most kReduceMaxEntries output vectors.
+constexpr int kReduceMaxEntries = 8;
+struct ReduceJob {
+    const float* partials;      // [nrows][nq][n]
+    int nrows, nq, n;
+    float* out[4];              // out[q] (+)= sum over rows of partials[.][q][.]; nullptr: skip
+};
+const char* launch_layernorm_bwd_partial(Runtime* rt, const void* dh, const void* x, const void* mu, const void* rstd,
+                                         const void* gamma, const void* resid, int T, int d, void* dx, void* dgamma,
+                                         void* dbeta, void* db_resid, void* db_dx, void* partials, ReduceJob* job,
+                                         cudaStream_t stream);
+const char* launch_colsum_partial(Runtime* rt, const void* in, int T, int N, int ld, void* out, void* partials,
+                                  ReduceJob* job, cudaStream_t stream);
+const char* launch_reduce_jobs(const ReduceJob* jobs, int njobs, int accumulate, cudaStream_t stream);
 
 // Column sums with the partial sums in a fixed device array inside the library (no allocation, no Runtime).
 size_t colsum_noalloc_max_columns();

@@ -84,6 +84,47 @@ def test_gemm_nn_dgrad(pw, oracle64, M, N, K, epi):
     assert rel_l2(C, dx) < GRAD_TOL
 
 
+@pytest.mark.parametrize("B,S,H,dh,K", [(2, 128, 4, 128, 512), (3, 128, 6, 64, 384), (1, 640, 3, 128, 384), (1, 128, 2, 64, 128),
+                                        (4, 256, 16, 128, 2048)])
+def test_gemm_rowdot_epilogue(pw, oracle64, B, S, H, dh, K):
+    """dout = dx1 Wo with delta[b][h][s] = sum over head h's columns of dout * o taken in the epilogue;
+    the same delta then drives pw_op_attention_bwd (o = None) to the same dqkv as the three-kernel call."""
+    g = torch.Generator().manual_seed(31)
+    M, N = B * S, H * dh
+    A, W = bf16_randn((M, K), g), bf16_randn((K, N), g, 0.1)
+    O = bf16_randn((M, N), g)
+    C, check = guard_alloc((M, N), torch.bfloat16)
+    delta, check_d = guard_alloc((B, H, S), torch.float32)
+    pw.op_gemm_rowdot(M, N, K, A.cuda(), K, W.cuda(), N, C, N, O.cuda(), N, dh, S, delta)
+    torch.cuda.synchronize()
+    _status_ok(pw)
+    check(); check_d()
+    dout, _, _ = oracle64.linear_bwd(np.zeros((M, N)), np64(W), np64(A))     # dout[t][n] = sum_k A[t][k] W[k][n]
+    assert rel_l2(C, dout) < GRAD_TOL
+    elem_check(C, dout, "dout", **ELEM_GRAD)
+    want = (dout * np64(O)).reshape(B, S, H, dh).sum(-1).transpose(0, 2, 1)  # [B, H, S]
+    assert rel_l2(delta, want) < 1e-4
+    elem_check(delta, want, "delta", **ELEM_F32)
+    # bitwise repeatable
+    C2, d2 = torch.empty_like(C), torch.empty_like(delta)
+    pw.op_gemm_rowdot(M, N, K, A.cuda(), K, W.cuda(), N, C2, N, O.cuda(), N, dh, S, d2)
+    torch.cuda.synchronize()
+    assert torch.equal(C, C2) and torch.equal(delta, d2)
+    if S % 128 == 0:
+        qkv = bf16_randn((M, 3 * N), g).cuda()
+        o_dev, lse = torch.empty((M, N), dtype=torch.bfloat16, device="cuda"), torch.empty((B, H, S), device="cuda")
+        pw.op_attention_fwd(qkv, B, S, H, dh, o_dev, lse)
+        dq_a, dq_b = torch.empty_like(qkv), torch.empty_like(qkv)
+        dl = torch.empty((B, H, S), device="cuda")
+        pw.op_gemm_rowdot(M, N, K, A.cuda(), K, W.cuda(), N, C2, N, o_dev, N, dh, S, d2)
+        pw.op_attention_bwd(qkv, o_dev, C2, lse, B, S, H, dh, dq_a, dl)        # delta by the row-dot kernel (from bf16 dout)
+        pw.op_attention_bwd(qkv, None, C2, lse, B, S, H, dh, dq_b, d2)         # delta from the GEMM epilogue (from fp32 dout)
+        torch.cuda.synchronize()
+        _status_ok(pw)
+        assert rel_l2(d2, dl) < 5e-3
+        assert rel_l2(dq_b, dq_a) < 5e-3
+
+
 @pytest.mark.parametrize("M,N,K", SHAPES)
 @pytest.mark.parametrize("accumulate", [False, True])
 def test_gemm_nt_wgrad(pw, oracle64, M, N, K, accumulate):
