@@ -286,7 +286,9 @@ static pw_status_t do_colsum(pw_layer_t* L, const void* in, int N, void* out, in
 }
 static pw_status_t do_reduce(pw_layer_t* L, const ReduceJob* jobs, int njobs, int accumulate, cudaStream_t st)
 {
-    LaunchScope sc(L, PW_K_REDUCE, 1, 0.0, 0.0, st);
+    double bytes = 0.0;                                  // the partial rows it reads (they are still in L2 more often than not)
+    for (int j = 0; j < njobs; ++j) bytes += 4.0 * jobs[j].nrows * jobs[j].nq * jobs[j].n;
+    LaunchScope sc(L, PW_K_REDUCE, 1, 0.0, bytes, st);
     const char* e = launch_reduce_jobs(jobs, njobs, accumulate, st);
     if (e) sc.cancel(1);
     return e ? fail(PW_ERR_CUDA, e) : PW_OK;
