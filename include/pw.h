@@ -463,17 +463,33 @@ pw_status_t pw_shared_close(void* dev_ptr);
  *   PW_TUNE_GEMM_SPLIT_MIN_K  64 (default): ... only from this many 64-wide K blocks on
  *   PW_TUNE_FAIL_LAUNCH       0 (default) / k > 0: host-side fault injection for error-path tests - the
  *                             k-th kernel launch from now is not enqueued and reports a launch failure
- *                             (the call that issued it returns PW_ERR_CUDA); the knob then returns to 0 */
+ *                             (the call that issued it returns PW_ERR_CUDA); the knob then returns to 0
+ *   PW_TUNE_NVTX              0 (default) / 1: NVTX ranges ("pw_layer_fwd", "pw_layer_bwd",
+ *                             "pw_stage_run_chain", "pw_lm_step", "pw_sgd_apply") around the host side of those
+ *                             calls, for timeline tools; without a tool attached a range costs a function call */
 enum {
     PW_TUNE_PDL = 0,
     PW_TUNE_GEMM_PAIR = 1,
     PW_TUNE_GEMM_BN = 2,
     PW_TUNE_GEMM_SPLIT = 3,
     PW_TUNE_GEMM_SPLIT_MIN_K = 4,
-    PW_TUNE_FAIL_LAUNCH = 5
+    PW_TUNE_FAIL_LAUNCH = 5,
+    PW_TUNE_NVTX = 6
 };
 pw_status_t pw_set_tuning(int knob, int value);
 pw_status_t pw_get_tuning(int knob, int* value);
+/* Logging (the paper's monitoring side channel has no counterpart here; this is the library's own).
+ * The library prints nothing by default.  pw_set_log installs a process-wide sink:
+ *   level PW_LOG_OFF (default), PW_LOG_ERROR: every failure, with the text pw_last_error() would give;
+ *   PW_LOG_INFO: also one line per pw_layer_create / pw_stage_create (shapes, workspace sizes) and per
+ *   pw_stage_run_chain / pw_lm_step call (dispatch mode, layers, micro-batches).
+ * fn(level, message, user) is called on the calling thread, before the failing call returns; message is
+ * only valid during the call.  fn = NULL writes "pw: <message>" lines to stderr.  No environment
+ * variable is read. */
+enum { PW_LOG_OFF = 0, PW_LOG_ERROR = 1, PW_LOG_INFO = 2 };
+typedef void (*pw_log_fn)(int level, const char* message, void* user);
+pw_status_t pw_set_log(int level, pw_log_fn fn, void* user);
+
 /* Clears the status word of the single-step calls (after a test has provoked an error). */
 pw_status_t pw_op_status_reset(void);
 /* Failure-path self-test.  Every device-side wait in this library is bounded; this call shows the

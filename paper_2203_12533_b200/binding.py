@@ -42,7 +42,7 @@ EXPORTS = (
     "pw_op_attention_fwd", "pw_op_attention_bwd", "pw_op_status",
     "pw_lm_workspace_bytes", "pw_lm_step",
     "pw_op_embedding_fwd", "pw_op_embedding_bwd_scratch_bytes", "pw_op_embedding_bwd", "pw_op_softmax_xent",
-    "pw_set_tuning", "pw_get_tuning", "pw_op_status_reset", "pw_op_selftest_wait_timeout", "pw_op_affine_f32", "pw_sgd_apply",
+    "pw_set_tuning", "pw_get_tuning", "pw_set_log", "pw_op_status_reset", "pw_op_selftest_wait_timeout", "pw_op_affine_f32", "pw_sgd_apply",
     "pw_layer_set_side_stream", "pw_stage_set_side_stream", "pw_dp_slice", "pw_dp_reduce_apply", "pw_shared_alloc", "pw_shared_free", "pw_shared_open", "pw_shared_close",
 )
 
@@ -441,12 +441,26 @@ def op_status():
     return c.value, s.value
 
 
-TUNE_PDL, TUNE_GEMM_PAIR, TUNE_GEMM_BN, TUNE_GEMM_SPLIT, TUNE_GEMM_SPLIT_MIN_K, TUNE_FAIL_LAUNCH = range(6)
+TUNE_PDL, TUNE_GEMM_PAIR, TUNE_GEMM_BN, TUNE_GEMM_SPLIT, TUNE_GEMM_SPLIT_MIN_K, TUNE_FAIL_LAUNCH, TUNE_NVTX = range(7)
+LOG_OFF, LOG_ERROR, LOG_INFO = range(3)
+LOG_FN = ctypes.CFUNCTYPE(None, ctypes.c_int, ctypes.c_char_p, ctypes.c_void_p)
 
 
 def set_tuning(knob: int, value: int):
     """Process-wide tuning knob (see pw_set_tuning in include/pw.h)."""
     _check(lib().pw_set_tuning(int(knob), int(value)))
+
+
+_log_keepalive = None
+
+
+def set_log(level: int, fn=None):
+    """pw_set_log: fn(level, message) or None for stderr; the ctypes thunk is kept alive here."""
+    global _log_keepalive
+    thunk = LOG_FN(lambda lv, msg, user: fn(lv, msg.decode())) if fn is not None else LOG_FN(0)
+    lib().pw_set_log.argtypes = [ctypes.c_int, LOG_FN, ctypes.c_void_p]
+    _check(lib().pw_set_log(int(level), thunk, None))
+    _log_keepalive = thunk
 
 
 def get_tuning(knob: int) -> int:

@@ -14,6 +14,8 @@
 #include <string>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "../../include/pw.h"
 #include "pw_kernels.h"
 
@@ -27,11 +29,40 @@ Tuning& tuning()
     return t;
 }
 
+// Log sink (pw_set_log): process-wide, guarded by a mutex; nothing is printed unless a level is set.
+struct LogSink { int level = 0; pw_log_fn fn = nullptr; void* user = nullptr; };
+static LogSink g_log;
+static std::mutex g_log_mu;
+static void log_line(int level, const std::string& msg)
+{
+    LogSink sink;
+    {
+        std::lock_guard<std::mutex> lock(g_log_mu);
+        sink = g_log;
+    }
+    if (sink.level < level) return;
+    if (sink.fn) sink.fn(level, msg.c_str(), sink.user);
+    else fprintf(stderr, "pw: %s\n", msg.c_str());
+}
+static bool log_enabled(int level)
+{
+    std::lock_guard<std::mutex> lock(g_log_mu);
+    return g_log.level >= level;
+}
+
 static pw_status_t fail(pw_status_t s, const std::string& msg)
 {
     g_last_error = msg;
+    log_line(PW_LOG_ERROR, std::string(pw_status_string(s)) + ": " + msg);
     return s;
 }
+
+// NVTX range around the host side of an entry point (PW_TUNE_NVTX); the v3 header needs no library.
+struct NvtxRange {
+    bool on;
+    explicit NvtxRange(const char* name) : on(tuning().nvtx != 0) { if (on) nvtxRangePushA(name); }
+    ~NvtxRange() { if (on) nvtxRangePop(); }
+};
 static pw_status_t fail_cuda(const char* what, cudaError_t e)
 {
     return fail(PW_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
@@ -571,6 +602,13 @@ pw_status_t pw_layer_create(const pw_layer_config_t* cfg, pw_layer_t** out)
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&L->aux, cudaStreamNonBlocking);
     for (int i = 0; i < 6 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&L->ev[i], cudaEventDisableTiming);
     if (e != cudaSuccess) { pw_layer_destroy(L); return fail_cuda("handle resources (status word, side stream, events)", e); }
+    if (log_enabled(PW_LOG_INFO)) {
+        const LayerPlan& p = L->plan;
+        log_line(PW_LOG_INFO, "pw_layer_create: d_model " + std::to_string(p.d) + ", " + std::to_string(p.H) + " heads x " + std::to_string(p.dh) +
+                                  ", d_ff " + std::to_string(p.F) + ", " + std::to_string(p.B) + " x " + std::to_string(p.S) + " tokens, ctx " +
+                                  std::to_string(p.ctx_bytes) + " bytes, scratch " + std::to_string(p.scratch_bytes) + " bytes" +
+                                  (p.lean ? ", lean save set" : "") + (p.whole ? ", whole-layer kernels" : ""));
+    }
     *out = L;
     return PW_OK;
 }
@@ -606,6 +644,7 @@ pw_status_t pw_layer_ctx_offset(const pw_layer_t* layer, int which, size_t* offs
 pw_status_t pw_layer_fwd(pw_layer_t* layer, const pw_layer_params_t* params, const void* x, void* y, void* ctx,
                          void* scratch, void* stream)
 {
+    NvtxRange nv("pw_layer_fwd");
     if (!layer || !params) return fail(PW_ERR_INVALID_ARG, "layer or params is NULL");
     if (!params_ok(params)) return fail(PW_ERR_INVALID_ARG, "a parameter pointer is NULL or not 16-byte aligned");
     if (!aligned(x, 16) || !aligned(y, 16)) return fail(PW_ERR_INVALID_ARG, "x or y is NULL or misaligned");
@@ -620,6 +659,7 @@ pw_status_t pw_layer_fwd(pw_layer_t* layer, const pw_layer_params_t* params, con
 pw_status_t pw_layer_bwd(pw_layer_t* layer, const pw_layer_params_t* params, const void* x, const void* dy, void* dx,
                          const pw_layer_grads_t* grads, int accumulate, const void* ctx, void* scratch, void* stream)
 {
+    NvtxRange nv("pw_layer_bwd");
     if (!layer || !params || !grads) return fail(PW_ERR_INVALID_ARG, "layer, params or grads is NULL");
     if (!params_ok(params)) return fail(PW_ERR_INVALID_ARG, "a parameter pointer is NULL or not 16-byte aligned");
     if (!grads_ok(grads)) return fail(PW_ERR_INVALID_ARG, "a gradient pointer is NULL or not 16-byte aligned");
@@ -685,6 +725,7 @@ pw_status_t pw_stage_create(const pw_layer_config_t* cfg, int n_layers, pw_stage
     st->layer = L;
     st->n_layers = n_layers;
     *out = st;
+    if (log_enabled(PW_LOG_INFO)) log_line(PW_LOG_INFO, "pw_stage_create: " + std::to_string(n_layers) + " layers of the shape above");
     return PW_OK;
 }
 
@@ -802,11 +843,15 @@ pw_status_t pw_stage_run_chain(pw_stage_t* stage, const pw_layer_params_t* param
                                void* const* dx_mb, int n_microbatches, int dispatch_mode, int schedule, int recompute,
                                void* workspace, size_t workspace_bytes, void* stream)
 {
+    NvtxRange nv("pw_stage_run_chain");
     if (!stage || !params || !grads || !x_mb || !dy_mb || !y_mb || !dx_mb)
         return fail(PW_ERR_INVALID_ARG, "a required pointer is NULL");
     if (dispatch_mode < PW_DISPATCH_OPBYOP || dispatch_mode > PW_DISPATCH_GRAPH) return fail(PW_ERR_INVALID_ARG, "unknown dispatch mode");
     StageLayout lay;
     pw_status_t s = stage_layout(stage, n_microbatches, schedule, recompute, &lay);
+    if (s == PW_OK && log_enabled(PW_LOG_INFO))
+        log_line(PW_LOG_INFO, std::string("pw_stage_run_chain: ") + (dispatch_mode == PW_DISPATCH_OPBYOP ? "OPBYOP" : dispatch_mode == PW_DISPATCH_ASYNC ? "ASYNC" : "GRAPH") +
+                                  ", " + std::to_string(stage->n_layers) + " layers x " + std::to_string(n_microbatches) + " micro-batches" + (recompute ? ", recompute" : ""));
     if (s != PW_OK) return s;
     if (!aligned(workspace, 256)) return fail(PW_ERR_INVALID_ARG, "workspace is NULL or not 256-byte aligned");
     if (workspace_bytes < lay.total) return fail(PW_ERR_WORKSPACE_TOO_SMALL, "workspace smaller than pw_stage_workspace_bytes reports");
@@ -948,6 +993,7 @@ pw_status_t pw_lm_step(pw_stage_t* stage, const pw_layer_params_t* params, const
                        const pw_lm_params_t* lm, const pw_lm_grads_t* lm_grads, const int32_t* ids, const int32_t* labels,
                        float* loss, int vocab, int recompute, void* workspace, size_t workspace_bytes, void* stream)
 {
+    NvtxRange nv("pw_lm_step");
     if (!stage || !params || !grads || !lm || !lm_grads || !ids || !labels || !loss)
         return fail(PW_ERR_INVALID_ARG, "a required pointer is NULL");
     LmLayout lay;
@@ -1167,6 +1213,7 @@ pw_status_t pw_op_affine_f32(const void* x, long long n, float scale, float shif
 pw_status_t pw_sgd_apply(const pw_apply_item_t* items, int n_items, float lr, float grad_scale, int init_master,
                          void* stream)
 {
+    NvtxRange nv("pw_sgd_apply");
     PW_RT_OR_FAIL();
     if (!items || n_items <= 0) return fail(PW_ERR_INVALID_ARG, "gradient apply: no items");
     if (!(lr >= 0.0f) || !(grad_scale > 0.0f) || !std::isfinite(lr) || !std::isfinite(grad_scale))
@@ -1298,6 +1345,14 @@ pw_status_t pw_op_selftest_wait_timeout(uint64_t limit_cycles, int* kernel_retur
     return e == cudaSuccess ? PW_OK : fail_cuda("self-test", e);
 }
 
+pw_status_t pw_set_log(int level, pw_log_fn fn, void* user)
+{
+    if (level < PW_LOG_OFF || level > PW_LOG_INFO) return fail(PW_ERR_INVALID_ARG, "unknown log level");
+    std::lock_guard<std::mutex> lock(g_log_mu);
+    g_log.level = level; g_log.fn = fn; g_log.user = user;
+    return PW_OK;
+}
+
 pw_status_t pw_set_tuning(int knob, int value)
 {
     Tuning& t = tuning();
@@ -1308,6 +1363,7 @@ pw_status_t pw_set_tuning(int knob, int value)
         case PW_TUNE_GEMM_SPLIT: if (value != 0 && value != 1) break; t.gemm_split = value; ++t.epoch; return PW_OK;
         case PW_TUNE_GEMM_SPLIT_MIN_K: if (value < 1) break; t.gemm_split_min_k = value; ++t.epoch; return PW_OK;
         case PW_TUNE_FAIL_LAUNCH: if (value < 0) break; t.fail_launch_countdown = value; return PW_OK;
+        case PW_TUNE_NVTX: if (value != 0 && value != 1) break; t.nvtx = value; return PW_OK;
         default: return fail(PW_ERR_INVALID_ARG, "unknown tuning knob");
     }
     return fail(PW_ERR_INVALID_ARG, "value out of range for this tuning knob");
@@ -1324,6 +1380,7 @@ pw_status_t pw_get_tuning(int knob, int* value)
         case PW_TUNE_GEMM_SPLIT: *value = t.gemm_split; return PW_OK;
         case PW_TUNE_GEMM_SPLIT_MIN_K: *value = t.gemm_split_min_k; return PW_OK;
         case PW_TUNE_FAIL_LAUNCH: *value = t.fail_launch_countdown; return PW_OK;
+        case PW_TUNE_NVTX: *value = t.nvtx; return PW_OK;
         default: return fail(PW_ERR_INVALID_ARG, "unknown tuning knob");
     }
 }

@@ -37,6 +37,7 @@ struct Tuning {
     int gemm_bn = 0;             // 0 = tile width chosen by the launcher, else 128 / 192 / 256
     int gemm_split = 1;          // cut the tiles of a thin last round along K
     int gemm_split_min_k = 64;   // ... from this many 64-wide K blocks on
+    int nvtx = 0;                // NVTX ranges around the host side of the main entry points
     uint64_t epoch = 0;          // bumped by every change (part of the CUDA-graph cache key)
     // Host-side fault injection for the error-path tests: when > 0, counts down once per launch and
     // the launch that brings it to zero is NOT enqueued and reports cudaErrorLaunchFailure instead.

@@ -74,7 +74,7 @@ def test_tuning_knobs_validate_on_the_host(libpath):
     """pw_set_tuning / pw_get_tuning are pure host state: defaults, round trip, range checks."""
     lib = ctypes.CDLL(libpath)
     v = ctypes.c_int(-1)
-    defaults = {0: 1, 1: 1, 2: 0, 3: 1, 4: 64, 5: 0}
+    defaults = {0: 1, 1: 1, 2: 0, 3: 1, 4: 64, 5: 0, 6: 0}
     for knob, want in defaults.items():
         assert lib.pw_get_tuning(knob, ctypes.byref(v)) == 0 and v.value == want
     assert lib.pw_set_tuning(2, 128) == 0
@@ -84,3 +84,26 @@ def test_tuning_knobs_validate_on_the_host(libpath):
     assert lib.pw_set_tuning(2, 0) == 0
     assert lib.pw_set_tuning(0, 2) == 1 and lib.pw_set_tuning(99, 0) == 1 and lib.pw_set_tuning(5, -1) == 1
     assert lib.pw_get_tuning(99, ctypes.byref(v)) == 1 and lib.pw_get_tuning(0, None) == 1
+
+
+def test_log_sink_receives_failures_and_nvtx_ranges_cost_nothing_without_a_tool(libpath):
+    """pw_set_log: an argument error reaches the callback with the text of pw_last_error (no GPU needed);
+    level 0 is silent again.  PW_TUNE_NVTX only switches ranges on: the failing call below runs through one."""
+    lib = ctypes.CDLL(libpath)
+    lib.pw_last_error.restype = ctypes.c_char_p
+    LOGFN = ctypes.CFUNCTYPE(None, ctypes.c_int, ctypes.c_char_p, ctypes.c_void_p)
+    seen = []
+    cb = LOGFN(lambda level, msg, user: seen.append((level, msg.decode())))
+    lib.pw_set_log.argtypes = [ctypes.c_int, LOGFN, ctypes.c_void_p]
+    assert lib.pw_set_log(7, cb, None) == 1                                  # unknown level
+    assert lib.pw_set_log(1, cb, None) == 0
+    assert lib.pw_set_tuning(6, 1) == 0
+    h = ctypes.c_void_p()
+    assert lib.pw_layer_create(None, ctypes.byref(h)) == 1
+    assert lib.pw_layer_fwd(None, None, None, None, None, None, None) == 1   # inside an NVTX range, no tool attached
+    assert lib.pw_set_tuning(6, 0) == 0
+    assert len(seen) == 2 and all(level == 1 for level, _ in seen)
+    assert seen[0][1].startswith("PW_ERR_INVALID_ARG: ") and lib.pw_last_error().decode() in seen[1][1]
+    assert lib.pw_set_log(0, LOGFN(0), None) == 0
+    assert lib.pw_layer_create(None, ctypes.byref(h)) == 1
+    assert len(seen) == 2

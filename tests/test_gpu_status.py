@@ -65,3 +65,37 @@ def test_injected_launch_failure_is_reported_and_nothing_of_that_launch_runs(pw)
     torch.cuda.synchronize()
     assert layer.launch_count() - n0 == 7 and layer.status() == (0, 0)
     assert not torch.equal(y, torch.full_like(x, 7.0)) and torch.isfinite(y.float()).all()
+
+
+def test_info_log_and_nvtx_ranges_on_a_live_step(pw):
+    """With the log sink at INFO and NVTX ranges on, creating a layer and running a forward produce the
+    documented lines and change nothing in the result (no timeline tool is attached: the ranges are calls
+    into an empty dispatch table)."""
+    from paper_2203_12533_b200 import inputs
+    w = inputs.WORKLOADS[1]
+    params = [p.cuda() for p in inputs.layer_params(w, 0, 0)]
+    x, _ = inputs.microbatch(w, 0, 0)
+    xd = x.cuda().view(-1, w.d_model)
+
+    def forward():
+        layer = pw.Layer(w.d_model, w.n_heads, w.head_dim, w.d_ff, w.seq_len, w.batch)
+        y = torch.empty_like(xd)
+        ctx = torch.empty(layer.ctx_bytes, dtype=torch.uint8, device="cuda")
+        scratch = torch.empty(layer.scratch_bytes, dtype=torch.uint8, device="cuda")
+        layer.fwd(params, xd, y, ctx, scratch)
+        torch.cuda.synchronize()
+        assert layer.status() == (0, 0)
+        return y
+
+    want = forward()
+    lines = []
+    pw.set_log(pw.LOG_INFO, lambda level, msg: lines.append((level, msg)))
+    pw.set_tuning(pw.TUNE_NVTX, 1)
+    try:
+        got = forward()
+    finally:
+        pw.set_tuning(pw.TUNE_NVTX, 0)
+        pw.set_log(pw.LOG_OFF)
+    assert torch.equal(got, want)
+    assert any(level == pw.LOG_INFO and msg.startswith("pw_layer_create: d_model 256, 4 heads x 64") for level, msg in lines)
+    assert not any(level == pw.LOG_ERROR for level, _ in lines)
