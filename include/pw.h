@@ -73,7 +73,7 @@ enum { PW_ACT_GELU_ERF = 0, PW_ACT_GELU_TANH = 1 };
  * size 0 for the three tensors; pw_layer_fwd then needs `scratch` even when ctx is given. */
 enum { PW_FLAG_LEAN_CTX = 1u, PW_FLAG_WHOLE_LAYER = 2u };
 /* PW_FLAG_WHOLE_LAYER: pw_layer_fwd and pw_layer_bwd are ONE cooperative kernel launch each instead of
- * 7 and 19 - for calls so small that launches and hand-offs between kernels, not arithmetic, set the
+ * 7 and 15 - for calls so small that launches and hand-offs between kernels, not arithmetic, set the
  * time (Section 5.1, Figures 5 and 6: computations shorter than the cost of issuing them).  Same
  * tensors, same saved context, same bf16 hand-off points as the default path; results agree with
  * it within rounding (different tile shapes and summation orders), bit-reproducibly.  Supported:

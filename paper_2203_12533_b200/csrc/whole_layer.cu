@@ -3,7 +3,7 @@
 // hand-offs between kernels set the time, not arithmetic: the regime of the dispatch study of
 // Section 5.1 (Figures 5 and 6), where a computation is shorter than the cost of issuing it.
 //
-// The 7 forward / 19 backward steps of the layer become 5 / 7 phases of one persistent grid
+// The 7 forward / 15 backward launches of the multi-kernel path become 5 / 7 phases of one persistent grid
 // (one 256-thread CTA per SM); a phase is a list of independent units (a 64 x 64 output tile of a
 // GEMM, a slice of its K range, 64 query or key rows of one head, four LayerNorm rows, 16 columns of
 // a bias sum) that the CTAs take round-robin, and phases are separated by a bounded grid barrier.

@@ -12,7 +12,7 @@ every layer call), ASYNC (enqueue everything) and GRAPH (one captured CUDA graph
 prints one JSON line per (sequence length, mode): layer calls per second and microseconds per
 call, for a chain of ``layers`` x ``microbatches`` x 2 calls at the width of workload 1.  Where the
 shape allows it, each mode is also run with PW_FLAG_WHOLE_LAYER (a layer call is then one kernel
-launch instead of 7 or 19): the step the paper's Fused mode takes one level further down.
+launch instead of 7 or 15): the step the paper's Fused mode takes one level further down.
 """
 from __future__ import annotations
 
