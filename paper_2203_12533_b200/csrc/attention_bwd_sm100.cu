@@ -44,7 +44,14 @@ struct KvSmem {
     static constexpr int kBlocks = DH / 64;
     static constexpr int kKV = 128 * DH * 2;                 // K_j or V_j tile
     static constexpr int kSub = 64 * DH * 2;                 // one 64-row sub-tile of Q or dO
-    static constexpr int kStages = 3;
+    static constexpr int kStages = DH == 64 ? 5 : 3;         // Q_u / dO_u ring (the scores run kBufs - 1 sub-tiles ahead of the accumulation)
+    static constexpr int kBufs = DH == 64 ? 3 : 2;           // S^T / dP^T buffers in TMEM: with 64-wide heads dV and dK leave room for a third pair
+    // TMEM columns: S^T buffer b at 64 b, dP^T buffer b at kDP + 64 b, then dV and dK (DH columns each)
+    static constexpr int kDP = 64 * kBufs, kDV = 128 * kBufs, kDK = kDV + (DH == 64 ? 64 : 128);
+    // barriers: 0,1 kv_full[buffer] | 2,3 kv_empty[buffer] | kQF+s q_full[stage] | kQE+s q_empty[stage] | kSF+b st_full[b]
+    //   kPF+b p_full[b] (256 arrivals) | kAF acc_full | kAE acc_empty (256 arrivals) | kIF+i item_full | kIE+i item_empty (9 arrivals)
+    static constexpr int kQF = 4, kQE = kQF + kStages, kSF = kQE + kStages, kPF = kSF + kBufs, kAF = kPF + kBufs, kAE = kAF + 1,
+                         kIF = kAE + 1, kIE = kIF + 2, kNumBars = kIE + 2;
     static constexpr int kK = 0;                             // item buffer i: K_j at i*2*kKV, V_j right after (two buffers)
     static constexpr int kQ = 4 * kKV;                       // ring: stage s holds Q_u at kQ + s*2*kSub, dO_u right after
     static constexpr int kBars = kQ + kStages * 2 * kSub;
@@ -81,12 +88,11 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
     uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(sm);
     uint64_t* bars = reinterpret_cast<uint64_t*>(sm + L::kBars);
-    // barrier map: 0,1 kv_full[buffer] | 2,3 kv_empty[buffer] | 4..6 q_full[stage] | 7..9 q_empty[stage]
-    //   10,11 st_full[hb] | 12,13 p_full[hb] (256 arrivals) | 14 acc_full | 15 acc_empty (256 arrivals)
-    //   16,17 item_full | 18,19 item_empty (9 arrivals)
+    // (barrier map: see KvSmem)
     const uint32_t bar0 = smem_u32(bars);
     auto bar = [&](int i) { return bar0 + 8u * i; };
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
+    static_assert(L::kNumBars <= 28, "barriers and the words behind them share 256 bytes");
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 28);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* item_slot = reinterpret_cast<volatile int*>(tmem_slot + 2);   // two entries
     auto draw = [&]() {
@@ -110,22 +116,22 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
         }
     };
     auto load_q = [&](const KvItem& it, int i, int s) {     // Q_u and dO_u, u = 2j + i
-        mbar_arrive_expect_tx(bar(4 + s), 2 * L::kSub);
+        mbar_arrive_expect_tx(bar(L::kQF + s), 2 * L::kSub);
         const uint32_t qs = sbase + L::kQ + s * 2 * L::kSub, gs = qs + L::kSub;
         const int qrow = it.b * p.S + (2 * it.j + i) * 64;
         for (int kb = 0; kb < L::kBlocks; ++kb) {
-            tma_load_2d(qs + kb * 8192, &tmQ, it.h * DH + kb * 64, qrow, bar(4 + s));
-            tma_load_2d(gs + kb * 8192, &tmDO, it.h * DH + kb * 64, qrow, bar(4 + s));
+            tma_load_2d(qs + kb * 8192, &tmQ, it.h * DH + kb * 64, qrow, bar(L::kQF + s));
+            tma_load_2d(gs + kb * 8192, &tmDO, it.h * DH + kb * 64, qrow, bar(L::kQF + s));
         }
     };
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 12; ++i) mbar_init(bar(i), 1);
-        mbar_init(bar(12), 256); mbar_init(bar(13), 256);
-        mbar_init(bar(14), 1);
-        mbar_init(bar(15), 256);
-        mbar_init(bar(16), 1); mbar_init(bar(17), 1);
-        mbar_init(bar(18), 9); mbar_init(bar(19), 9);
+        for (int i = 0; i < L::kPF; ++i) mbar_init(bar(i), 1);
+        for (int i = 0; i < L::kBufs; ++i) mbar_init(bar(L::kPF + i), 256);
+        mbar_init(bar(L::kAF), 1);
+        mbar_init(bar(L::kAE), 256);
+        mbar_init(bar(L::kIF), 1); mbar_init(bar(L::kIF + 1), 1);
+        mbar_init(bar(L::kIE), 9); mbar_init(bar(L::kIE + 1), 9);
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async();
@@ -138,7 +144,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
         KvItem it;
         const int idx0 = draw();
         item_slot[0] = idx0;
-        mbar_arrive(bar(16));
+        mbar_arrive(bar(L::kIF));
         if (kv_item(p, idx0, it)) {
             load_kv(it, 0);
             for (; early < it.n_u && early < L::kStages; ++early) load_q(it, early, early);
@@ -152,7 +158,6 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    // TMEM columns: S^T buffers at 0 / 64, dP^T buffers at 128 / 192, dV at 256, dK at 384
 
     if (warp == 0) {
         if (lane == 0) {
@@ -168,15 +173,15 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
                 for (int i = 0; i < it.n_u && ok; ++i, ++m) {
                     if (k == 0 && i < early) continue;
                     const int s = m % L::kStages;
-                    if (!mbar_wait(bar(7 + s), ((m / L::kStages) & 1) ^ 1, abort_flag, p.status, 500)) { ok = false; break; }
+                    if (!mbar_wait(bar(L::kQE + s), ((m / L::kStages) & 1) ^ 1, abort_flag, p.status, 500)) { ok = false; break; }
                     load_q(it, i, s);
                 }
                 if (!ok) break;
                 const int kn = k + 1;
-                if (!mbar_wait(bar(18 + (kn & 1)), ((kn >> 1) & 1) ^ 1, abort_flag, p.status, 502)) break;
+                if (!mbar_wait(bar(L::kIE + (kn & 1)), ((kn >> 1) & 1) ^ 1, abort_flag, p.status, 502)) break;
                 idx = draw();
                 item_slot[kn & 1] = idx;
-                mbar_arrive(bar(16 + (kn & 1)));
+                mbar_arrive(bar(L::kIF + (kn & 1)));
             }
         }
     } else if (warp == 1) {
@@ -185,44 +190,42 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
         constexpr uint32_t idesc_acc = make_idesc_bf16(128, DH, false, true);
         const uint32_t tb = __shfl_sync(0xffffffffu, tmem_base, 0);
         const uint32_t sb = __shfl_sync(0xffffffffu, sbase, 0);
-        auto issue_scores = [&](uint32_t g, int buf) {      // S^T and dP^T of stream position g into buffer g & 1
-            const int s = g % L::kStages, hb = g & 1;
+        auto issue_scores = [&](uint32_t g, int buf) {      // S^T and dP^T of stream position g into buffer g % kBufs
+            const int s = g % L::kStages, hb = g % L::kBufs;
             const uint64_t desc_k = make_smem_desc_sw128(sb + L::kK + buf * 2 * L::kKV, 16, 1024);
             const uint64_t desc_v = desc_advance(desc_k, L::kKV);
             const uint64_t dq = make_smem_desc_sw128(sb + L::kQ + s * 2 * L::kSub, 16, 1024), dg = desc_advance(dq, L::kSub);
             const uint32_t st = tb + hb * 64;
             if (elect_one()) {
+                // the two products are independent accumulation chains: their steps alternate, so that a step
+                // never has to wait for the one before it to leave the pipe
 #pragma unroll
                 for (int kb = 0; kb < L::kBlocks; ++kb)
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
+                    for (int kk = 0; kk < 4; ++kk) {
                         umma_f16(st, desc_advance(desc_k, kb * 16384 + kk * 32), desc_advance(dq, kb * 8192 + kk * 32),
                                  idesc_st, (kb | kk) ? 1u : 0u);
-#pragma unroll
-                for (int kb = 0; kb < L::kBlocks; ++kb)
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        umma_f16(st + 128, desc_advance(desc_v, kb * 16384 + kk * 32), desc_advance(dg, kb * 8192 + kk * 32),
+                        umma_f16(st + L::kDP, desc_advance(desc_v, kb * 16384 + kk * 32), desc_advance(dg, kb * 8192 + kk * 32),
                                  idesc_st, (kb | kk) ? 1u : 0u);
-                umma_commit(bar(10 + hb));
+                    }
+                umma_commit(bar(L::kSF + hb));
             }
             __syncwarp();
         };
         auto issue_acc = [&](uint32_t g, bool first) {      // dV += P^T dO_u, dK += dS^T Q_u
-            const int s = g % L::kStages, hb = g & 1;
+            const int s = g % L::kStages, hb = g % L::kBufs;
             const uint64_t dq = make_smem_desc_sw128(sb + L::kQ + s * 2 * L::kSub, 8192, 1024), dg = desc_advance(dq, L::kSub);
             const uint32_t pt = tb + hb * 64;
             const uint32_t acc0 = first ? 0u : 1u;
             if (elect_one()) {
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    umma_f16_ta(tb + 256, pt + (ks >> 1) * 32 + (ks & 1) * 8, desc_advance(dg, ks * 2048), idesc_acc,
+                for (int ks = 0; ks < 4; ++ks) {             // dV and dK alternate (independent accumulators)
+                    umma_f16_ta(tb + L::kDV, pt + (ks >> 1) * 32 + (ks & 1) * 8, desc_advance(dg, ks * 2048), idesc_acc,
                                 ks ? 1u : acc0);
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    umma_f16_ta(tb + 384, pt + 128 + (ks >> 1) * 32 + (ks & 1) * 8, desc_advance(dq, ks * 2048), idesc_acc,
+                    umma_f16_ta(tb + L::kDK, pt + L::kDP + (ks >> 1) * 32 + (ks & 1) * 8, desc_advance(dq, ks * 2048), idesc_acc,
                                 ks ? 1u : acc0);
-                umma_commit(bar(7 + s));                    // Q_u / dO_u stage free
+                }
+                umma_commit(bar(L::kQE + s));               // Q_u / dO_u stage free
             }
             __syncwarp();
         };
@@ -234,32 +237,39 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
         bool ok = true;
         KvItem it;
         for (int k = 0; ok; ++k) {
-            if (!wait(16 + (k & 1), (k >> 1) & 1, 514)) break;
+            if (!wait(L::kIF + (k & 1), (k >> 1) & 1, 514)) break;
             const int idx = __shfl_sync(0xffffffffu, item_slot[k & 1], 0);   // broadcast: everything derived from it is warp-uniform
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(18 + (k & 1)));
+            if (lane == 0) mbar_arrive(bar(L::kIE + (k & 1)));
             if (!kv_item(p, idx, it)) break;
             const int buf = k & 1, n_u = it.n_u;
-            ok = wait(0 + buf, (k >> 1) & 1, 510) && wait(4 + g0 % L::kStages, (g0 / L::kStages) & 1, 511);
+            // the scores run kBufs - 1 sub-tiles ahead of the accumulation products
+            constexpr int kAhead = L::kBufs - 1;
+            ok = wait(0 + buf, (k >> 1) & 1, 510);
+            for (int a = 0; a < kAhead && a < n_u && ok; ++a) {
+                const uint32_t ga = g0 + a;
+                ok = wait(L::kQF + ga % L::kStages, (ga / L::kStages) & 1, 511);
+                if (!ok) break;
+                tc_fence_after();
+                issue_scores(ga, buf);
+            }
             if (!ok) break;
-            tc_fence_after();
-            issue_scores(g0, buf);
             for (int i = 0; i < n_u && ok; ++i) {
                 const uint32_t g = g0 + i;
-                if (i + 1 < n_u) {
-                    const uint32_t gn = g + 1;
-                    if (!wait(4 + gn % L::kStages, (gn / L::kStages) & 1, 512)) { ok = false; break; }
+                if (i + kAhead < n_u) {
+                    const uint32_t gn = g + kAhead;
+                    if (!wait(L::kQF + gn % L::kStages, (gn / L::kStages) & 1, 512)) { ok = false; break; }
                     tc_fence_after();
                     issue_scores(gn, buf);
                 }
-                if (!wait(12 + (g & 1), (g >> 1) & 1, 513)) { ok = false; break; }
+                if (!wait(L::kPF + g % L::kBufs, (g / L::kBufs) & 1, 513)) { ok = false; break; }
                 // the previous item's dV / dK must have been read out before they are overwritten
-                if (i == 0 && !wait(15, (k & 1) ^ 1, 515)) { ok = false; break; }
+                if (i == 0 && !wait(L::kAE, (k & 1) ^ 1, 515)) { ok = false; break; }
                 tc_fence_after();
                 issue_acc(g, i == 0);
             }
             if (!ok) break;
-            if (elect_one()) umma_commit(bar(14));
+            if (elect_one()) umma_commit(bar(L::kAF));
             __syncwarp();
             g0 += n_u;
         }
@@ -272,18 +282,18 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
         bool ok = true;
         KvItem it;
         for (int k = 0; ok; ++k) {
-            ok = mbar_wait(bar(16 + (k & 1)), (k >> 1) & 1, abort_flag, p.status, 522);
+            ok = mbar_wait(bar(L::kIF + (k & 1)), (k >> 1) & 1, abort_flag, p.status, 522);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const int idx = item_slot[k & 1];
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(18 + (k & 1)));
+            if (lane == 0) mbar_arrive(bar(L::kIE + (k & 1)));
             if (!kv_item(p, idx, it)) break;
             const int kv0 = it.j * 128, u0 = 2 * it.j;
             const float* lse_row = p.lse + (static_cast<size_t>(it.b) * p.H + it.h) * p.S;
             const float* dl_row = p.delta + (static_cast<size_t>(it.b) * p.H + it.h) * p.S;
             for (int i = 0; i < it.n_u; ++i, ++g) {
-                const int hb = g & 1, qc0 = (u0 + i) * 64 + ch * 32;   // first query column of this thread's slice
+                const int hb = g % L::kBufs, qc0 = (u0 + i) * 64 + ch * 32;   // first query column of this thread's slice
                 // -lse*log2e and -delta of this slice's 32 queries, as two-wide operands
                 uint64_t nl2[16], ndl[16];
 #pragma unroll
@@ -293,13 +303,13 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
                     nl2[2 * gg] = pack_f32x2(-a.x * kLog2e, -a.y * kLog2e); nl2[2 * gg + 1] = pack_f32x2(-a.z * kLog2e, -a.w * kLog2e);
                     ndl[2 * gg] = pack_f32x2(-c.x, -c.y); ndl[2 * gg + 1] = pack_f32x2(-c.z, -c.w);
                 }
-                ok = mbar_wait(bar(10 + hb), (g >> 1) & 1, abort_flag, p.status, 520);
+                ok = mbar_wait(bar(L::kSF + hb), (g / L::kBufs) & 1, abort_flag, p.status, 520);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
                 uint32_t sv[32], dv[32];
                 tmem_ld32(tmem_base + lane_addr + hb * 64 + ch * 32, sv);
-                tmem_ld32(tmem_base + lane_addr + 128 + hb * 64 + ch * 32, dv);
+                tmem_ld32(tmem_base + lane_addr + L::kDP + hb * 64 + ch * 32, dv);
                 tc_wait_ld();
                 const bool diag = qc0 < kv0 + 128;           // some (key, query) pairs of this slice are masked
                 uint32_t pp[16], dd[16];
@@ -320,13 +330,13 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
                 }
                 // packed operands go back into this warp's own columns: P^T over S^T, dS^T over dP^T
                 tmem_st16(tmem_base + lane_addr + hb * 64 + ch * 32, pp);
-                tmem_st16(tmem_base + lane_addr + 128 + hb * 64 + ch * 32, dd);
+                tmem_st16(tmem_base + lane_addr + L::kDP + hb * 64 + ch * 32, dd);
                 tc_wait_st();
                 tc_fence_before();
-                mbar_arrive(bar(12 + hb));
+                mbar_arrive(bar(L::kPF + hb));
             }
             if (ok) {
-                ok = mbar_wait(bar(14), k & 1, abort_flag, p.status, 521);
+                ok = mbar_wait(bar(L::kAF), k & 1, abort_flag, p.status, 521);
                 ok = __all_sync(0xffffffffu, ok);
             }
             if (!ok) break;
@@ -341,11 +351,11 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmKV,   // qkv, box 
                 for (int c = 0; c < DH / 64; ++c) {
                     const int col0 = ch * (DH / 2) + c * 32;
                     uint32_t v[32];
-                    tmem_ld32(tmem_base + lane_addr + 256 + which * 128 + col0, v);
+                    tmem_ld32(tmem_base + lane_addr + (which == 0 ? L::kDV : L::kDK) + col0, v);
                     tc_wait_ld();
                     if (which == 1 && c == DH / 64 - 1) {    // dV and dK have left TMEM: the next item may overwrite them
                         tc_fence_before();
-                        mbar_arrive(bar(15));
+                        mbar_arrive(bar(L::kAE));
                     }
 #pragma unroll
                     for (int gq = 0; gq < 4; ++gq) {
